@@ -1,0 +1,190 @@
+/*
+ * oasis.h -- C ABI of the B200 (sm_100a) implementation of the OasisKV per-decode-step
+ * hot path: lookahead scoring of KV blocks, per-head top-k selection, host->HBM block
+ * gather, and sparse paged decode attention (OasisKV, Sec. 4.2-4.3, 5.1-5.2).
+ *
+ * Conventions shared by every call
+ *   - Every buffer is caller-owned.  Unless a parameter says "host", a pointer must be
+ *     dereferenceable by the GPU: device memory, or pinned host memory mapped into the
+ *     device address space (unified addressing).  The library allocates nothing, keeps
+ *     no state besides the last-error string, never synchronises and never blocks: each
+ *     call validates its scalar arguments on the host, enqueues its kernels on `stream`
+ *     (a cudaStream_t passed as void*; NULL = the legacy default stream) and returns.
+ *   - Return value: OASIS_OK or an oasis_status_t error.  On error nothing was enqueued
+ *     and oasis_last_error() describes the problem.  Contents of device arrays are not
+ *     validated on the host; out-of-range block ids or slots are the caller's error.
+ *   - bf16 tensors are raw 16-bit patterns, dense and row-major with the innermost index
+ *     last, and their base addresses must be 16-byte aligned (OASIS_ERR_INVALID_ARG
+ *     otherwise).  head_dim must be 128 and block_size 16 (OASIS_ERR_UNSUPPORTED
+ *     otherwise); n_q_heads must be a multiple of n_kv_heads.
+ *   - One "entry" is the K part then the V part of one (block, KV head):
+ *     [2][16][128] bf16 = 8192 contiguous bytes.  The full-KV pool is
+ *     [n_phys_blocks][n_kv_heads] entries (the paper's Head-Token-Dimension order,
+ *     Sec. 4.3); the HBM working-set pool is [n_slots] entries.
+ *   - Query head a reads KV head a / (n_q_heads / n_kv_heads).
+ */
+#ifndef OASIS_H
+#define OASIS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    OASIS_OK = 0,
+    OASIS_ERR_INVALID_ARG = 1, /* null pointer, misaligned buffer, inconsistent sizes   */
+    OASIS_ERR_UNSUPPORTED = 2, /* a shape this build has no kernel for                   */
+    OASIS_ERR_CUDA = 3,        /* a CUDA runtime call or kernel launch failed            */
+    OASIS_ERR_WORKSPACE = 4    /* workspace missing or smaller than required             */
+} oasis_status_t;
+
+typedef enum { OASIS_REDUCE_MAX = 0, OASIS_REDUCE_SUM = 1 } oasis_reduce_t;
+
+typedef struct {
+    int32_t batch;      /* B: requests in the step                                  */
+    int32_t n_q_heads;  /* Hq                                                        */
+    int32_t n_kv_heads; /* Hkv                                                       */
+    int32_t head_dim;   /* 128                                                       */
+    int32_t block_size; /* 16 tokens per KV block                                    */
+    int32_t max_blocks; /* row stride of every per-request block array               */
+} oasis_dims_t;
+
+#define OASIS_ENTRY_BYTES 8192
+#define OASIS_MAX_K 2048 /* largest k accepted by oasis_select_topk */
+
+/*
+ * Step 0 -- block summaries (Sec. 4.2.1: the coordinate-wise minimum and maximum of the
+ * keys of each logical block; Sec. 5.2: two summary rows per block, 1/16 of the KV size).
+ * For request b and every KV head h, (re)builds the summaries of logical blocks
+ * j = first_block[b] .. first_block[b] + n_blocks[b] - 1 from the K part of entry
+ * (block_table[b][j], h) of kv_pool.
+ *   kv_pool        full-KV pool (device memory, or mapped pinned host memory)
+ *   block_table    [B][max_blocks] int32, logical -> physical block
+ *   first_block, n_blocks   [B] int32 (device)
+ *   max_new_blocks host-side upper bound of n_blocks[b]; sizes the launch (blocks past
+ *                  n_blocks[b] are skipped on the device)
+ *   summaries      [B][Hkv][max_blocks][2][128] bf16, row 0 = min, row 1 = max; only the
+ *                  requested blocks are written
+ */
+int oasis_build_summaries(const oasis_dims_t *dims, const void *kv_pool,
+                          const int32_t *block_table, const int32_t *first_block,
+                          const int32_t *n_blocks, int32_t max_new_blocks, void *summaries,
+                          void *stream);
+
+/*
+ * Step 1 -- block scores from the lookahead (draft) queries (Sec. 4.2.1: each draft query
+ * scans the summaries and ranks all logical blocks independently for every KV head).
+ * For one query row q and block j the estimate is the upper bound that min/max summaries
+ * admit, U(q, j) = sum_x max(q_x * min_jx, q_x * max_jx), accumulated in fp32.  The
+ * n_draft * (Hq/Hkv) rows that share KV head h are reduced with max (OASIS_REDUCE_MAX) or
+ * sum (OASIS_REDUCE_SUM).
+ *   q_draft        draft queries, bf16, element (b, t, a, x) at
+ *                  q_draft[b * q_batch_stride + (t * Hq + a) * 128 + x]; q_batch_stride is
+ *                  in elements, a multiple of 8 (n_draft*Hq*128 when dense; larger when
+ *                  the drafts are a view into the stacked verify-step queries)
+ *   n_full_blocks  [B] int32 (device): blocks j < n_full_blocks[b] are candidates
+ *   scores         [B][Hkv][max_blocks] fp32; -inf for j >= n_full_blocks[b]
+ * n_draft * (Hq/Hkv) may not exceed 128.
+ */
+int oasis_score_blocks(const oasis_dims_t *dims, const void *q_draft, int64_t q_batch_stride,
+                       int32_t n_draft, const void *summaries, const int32_t *n_full_blocks,
+                       int32_t reduce_mode, float *scores, void *stream);
+
+/*
+ * Step 2 -- top-k blocks per (request, KV head) plus the always-kept local blocks
+ * (Sec. 5.2: K selected blocks and the active local block; no sink tokens).
+ * With K_eff = min(k, n_full_blocks[b]):
+ *   sel[b][h][0 .. K_eff)   block ids by descending score, equal scores by ascending id
+ *   sel[b][h][K_eff .. k)   -1
+ *   sel[b][h][k], [k+1]     the local blocks n_full_blocks[b] .. ceil((seq_len[b] +
+ *                           n_q_tokens) / 16) - 1 (at most two), else -1
+ * Scores are compared as fp32; -0 equals +0; NaN is not supported.
+ * Optional gather lists (both NULL, or both given), one request per sel column:
+ *   stage_idx   [B][Hkv][k+2] int64: block_table[b][sel] * Hkv + h, or -1 for a -1 column
+ *   stage_slots [B][Hkv][k+2] int32: (b * Hkv + h) * (k + 2) + column
+ *   seq_len     [B] int32 (device): history tokens before this step
+ * 1 <= k <= OASIS_MAX_K; max_blocks <= 49152.
+ */
+int oasis_select_topk(const oasis_dims_t *dims, const float *scores,
+                      const int32_t *n_full_blocks, const int32_t *seq_len,
+                      int32_t n_q_tokens, int32_t k, const int32_t *block_table, int32_t *sel,
+                      int64_t *stage_idx, int32_t *stage_slots, void *stream);
+
+/*
+ * Step 3 -- gather of selected entries from the host-resident full KV cache into HBM
+ * slots (Sec. 5.1: a gather kernel reads the selected block-head entries from the pinned
+ * CPU cache through unified addressing and writes them into the resident GPU pages).
+ *   hbm_pool[slots[i]] = host_kv[idx[i]]   for i < n, 8192-byte entries; idx[i] < 0: skip
+ *   host_kv   full-KV pool: pinned host memory mapped for the device (or device memory)
+ *   idx       [n] int64 (device), slots [n] int32 (device); two requests must not name
+ *             the same slot
+ * Typically enqueued on a side stream so that it overlaps other layers' compute.
+ */
+int oasis_stage_blocks(const void *host_kv, const int64_t *idx, const int32_t *slots,
+                       int32_t n, void *hbm_pool, void *stream);
+
+/*
+ * Step 4 -- sparse paged decode attention over the staged working set (Sec. 4.2.1: the
+ * stacked normal and draft queries run over one resident KV working set in one call;
+ * Sec. 4.3: the selected key and value blocks share one ordering).
+ * Query token t of request b sits at position seq_len[b] + t.  For KV head h the keys are
+ * the tokens i of every column c with blk_tbl[b][h][c] = j >= 0 whose position
+ * j * 16 + i <= seq_len[b] + t, read from entry slot_tbl[b][h][c] of hbm_pool.
+ * out = softmax(scale * q K^T) V with bf16 tensor-core products and fp32 accumulation.
+ *   q, out      [B][n_q_tokens][Hq][128] bf16
+ *   slot_tbl, blk_tbl   [B][Hkv][n_cols] int32 (device)
+ *   lse         optional [B][n_q_tokens][Hq] fp32: natural-log sum of exponentials
+ *   workspace   device scratch of at least oasis_attn_workspace_bytes() bytes, 16-byte
+ *               aligned; its contents need no initialisation and are undefined afterwards.
+ *               May be NULL when that function returns 0.
+ * n_q_tokens * (Hq/Hkv) may not exceed 128.  A query row that sees no key yields zeros
+ * (lse = -inf).
+ */
+int oasis_sparse_attn(const oasis_dims_t *dims, const void *q, int32_t n_q_tokens,
+                      const void *hbm_pool, const int32_t *slot_tbl, const int32_t *blk_tbl,
+                      int32_t n_cols, const int32_t *seq_len, float scale, void *out,
+                      float *lse, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Scratch bytes oasis_sparse_attn needs for these shapes on the current device. */
+size_t oasis_attn_workspace_bytes(const oasis_dims_t *dims, int32_t n_q_tokens,
+                                  int32_t n_cols);
+
+/*
+ * KV selection stage -- delta selection with capped eviction (Sec. 4.2.3; the cap is a
+ * fraction of K, Sec. 5.5.1: cap = floor(ratio * K)).  Each (b, h) row owns n_res resident
+ * columns: resident[b][h][c] is the logical block held in column c (-1 = empty) and
+ * stamp[b][h][c] the step at which it was last selected.  With pred = sel[b][h][0..k):
+ *   1. a resident block that is in pred stays in place; its stamp becomes `step`;
+ *   2. the predicted blocks that are not resident are the candidates, in rank order;
+ *   3. the columns whose block is not in pred are eviction targets, least recently
+ *      selected first (empty columns first; equal stamps by ascending column);
+ *   4. candidate i replaces target i for i < min(cap, #candidates, #targets): the column
+ *      takes the block and stamp `step`, and a gather request is emitted:
+ *      plan_idx = block_table[b][block] * Hkv + h, plan_slots = row * slot_stride + column
+ *      with row = b * Hkv + h.  All other columns are left unchanged.
+ *   sel         [B][Hkv][sel_cols] int32, k <= sel_cols
+ *   resident, stamp   [B][Hkv][n_res] int32, updated in place (resident can serve as the
+ *               first n_res columns of an attention blk_tbl when n_res == its row length)
+ *   plan_idx [B][Hkv][cap] int64, plan_slots [B][Hkv][cap] int32: unused requests have
+ *               idx = -1; n_admitted [B][Hkv] int32 (may be NULL)
+ * 1 <= k <= OASIS_MAX_K, 1 <= n_res <= OASIS_MAX_K, 0 <= cap <= k.
+ */
+int oasis_plan_delta(const oasis_dims_t *dims, const int32_t *sel, int32_t sel_cols, int32_t k,
+                     const int32_t *block_table, int32_t *resident, int32_t *stamp,
+                     int32_t n_res, int32_t slot_stride, int32_t cap, int32_t step,
+                     int64_t *plan_idx, int32_t *plan_slots, int32_t *n_admitted,
+                     void *stream);
+
+/* Description of the calling thread's most recent error ("" if none). Static storage. */
+const char *oasis_last_error(void);
+
+/* Library version, "major.minor". */
+const char *oasis_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OASIS_H */

@@ -1,0 +1,174 @@
+"""Python names for the C-ABI calls of include/oasis.h -- argument marshalling only.
+
+Every function takes torch tensors (device memory, or pinned host memory for the full-KV
+pool), checks dtype / contiguity, hands raw pointers to liboasis.so and raises
+`OasisError` when the library reports a failure.  All arithmetic happens in the CUDA
+kernels; there is no CPU fallback: if liboasis.so has not been built
+(`python -m paper_2608_08097_b200.build`), the first call raises.
+"""
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liboasis.so")
+
+REDUCE_MAX, REDUCE_SUM = 0, 1
+ENTRY_BYTES = 8192
+SYMBOLS = ("oasis_build_summaries", "oasis_score_blocks", "oasis_select_topk",
+           "oasis_stage_blocks", "oasis_sparse_attn", "oasis_attn_workspace_bytes",
+           "oasis_plan_delta", "oasis_last_error", "oasis_version")
+
+
+class OasisError(RuntimeError):
+    pass
+
+
+class _Dims(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("batch", "n_q_heads", "n_kv_heads", "head_dim", "block_size", "max_blocks")]
+
+
+@dataclass(frozen=True)
+class Dims:
+    batch: int
+    n_q_heads: int
+    n_kv_heads: int
+    max_blocks: int
+    head_dim: int = 128
+    block_size: int = 16
+
+    def c(self):
+        return _Dims(self.batch, self.n_q_heads, self.n_kv_heads, self.head_dim, self.block_size,
+                     self.max_blocks)
+
+
+_lib = None
+
+
+def lib():
+    """Loads liboasis.so once; raises OasisError if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise OasisError("%s not found: build it with `python -m paper_2608_08097_b200.build` "
+                             "(there is no CPU fallback)" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, f32, sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float,
+                                 ctypes.c_size_t)
+        dp = ctypes.POINTER(_Dims)
+        L.oasis_build_summaries.argtypes = [dp, vp, vp, vp, vp, i32, vp, vp]
+        L.oasis_score_blocks.argtypes = [dp, vp, i64, i32, vp, vp, i32, vp, vp]
+        L.oasis_select_topk.argtypes = [dp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]
+        L.oasis_stage_blocks.argtypes = [vp, vp, vp, i32, vp, vp]
+        L.oasis_sparse_attn.argtypes = [dp, vp, i32, vp, vp, vp, i32, vp, f32, vp, vp, vp, sz, vp]
+        L.oasis_attn_workspace_bytes.argtypes = [dp, i32, i32]
+        L.oasis_attn_workspace_bytes.restype = sz
+        L.oasis_plan_delta.argtypes = [dp, vp, i32, i32, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
+        for name in ("oasis_build_summaries", "oasis_score_blocks", "oasis_select_topk",
+                     "oasis_stage_blocks", "oasis_sparse_attn", "oasis_plan_delta"):
+            getattr(L, name).restype = ctypes.c_int
+        L.oasis_last_error.restype = ctypes.c_char_p
+        L.oasis_version.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def last_error() -> str:
+    return lib().oasis_last_error().decode()
+
+
+def _check(rc, name):
+    if rc != 0:
+        raise OasisError("%s failed with status %d: %s" % (name, rc, last_error()))
+
+
+def _ptr(t, dtype=None, name="tensor"):
+    if t is None:
+        return None
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError("%s: expected %s, got %s" % (name, dtype, t.dtype))
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % name)
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def build_summaries(dims, kv_pool, block_table, first_block, n_blocks, max_new_blocks, summaries,
+                    stream=None):
+    d = dims.c()
+    _check(lib().oasis_build_summaries(
+        ctypes.byref(d), _ptr(kv_pool, torch.bfloat16, "kv_pool"),
+        _ptr(block_table, torch.int32, "block_table"), _ptr(first_block, torch.int32, "first_block"),
+        _ptr(n_blocks, torch.int32, "n_blocks"), int(max_new_blocks),
+        _ptr(summaries, torch.bfloat16, "summaries"), _stream(stream)), "oasis_build_summaries")
+
+
+def score_blocks(dims, q_draft, n_draft, summaries, n_full_blocks, scores, reduce_mode=REDUCE_MAX,
+                 q_batch_stride=None, stream=None):
+    """q_draft may be a view into the stacked queries (q[:, 1:]): only its batch stride may
+    differ from the dense layout."""
+    if q_draft.dtype != torch.bfloat16:
+        raise TypeError("q_draft: expected bfloat16")
+    if q_batch_stride is None:
+        if q_draft.dim() != 4 or q_draft.stride()[1:] != (q_draft.shape[2] * q_draft.shape[3], q_draft.shape[3], 1):
+            raise ValueError("q_draft must be [B][Td][Hq][128] with dense inner dimensions")
+        q_batch_stride = q_draft.stride(0) if q_draft.shape[0] > 1 else q_draft[0].numel()
+    d = dims.c()
+    _check(lib().oasis_score_blocks(
+        ctypes.byref(d), ctypes.c_void_p(q_draft.data_ptr()), int(q_batch_stride), int(n_draft),
+        _ptr(summaries, torch.bfloat16, "summaries"), _ptr(n_full_blocks, torch.int32, "n_full_blocks"),
+        int(reduce_mode), _ptr(scores, torch.float32, "scores"), _stream(stream)), "oasis_score_blocks")
+
+
+def select_topk(dims, scores, n_full_blocks, seq_len, n_q_tokens, k, block_table, sel,
+                stage_idx=None, stage_slots=None, stream=None):
+    d = dims.c()
+    _check(lib().oasis_select_topk(
+        ctypes.byref(d), _ptr(scores, torch.float32, "scores"),
+        _ptr(n_full_blocks, torch.int32, "n_full_blocks"), _ptr(seq_len, torch.int32, "seq_len"),
+        int(n_q_tokens), int(k), _ptr(block_table, torch.int32, "block_table"),
+        _ptr(sel, torch.int32, "sel"), _ptr(stage_idx, torch.int64, "stage_idx"),
+        _ptr(stage_slots, torch.int32, "stage_slots"), _stream(stream)), "oasis_select_topk")
+
+
+def stage_blocks(host_kv, idx, slots, n, hbm_pool, stream=None):
+    _check(lib().oasis_stage_blocks(
+        _ptr(host_kv, torch.bfloat16, "host_kv"), _ptr(idx, torch.int64, "idx"),
+        _ptr(slots, torch.int32, "slots"), int(n), _ptr(hbm_pool, torch.bfloat16, "hbm_pool"),
+        _stream(stream)), "oasis_stage_blocks")
+
+
+def attn_workspace_bytes(dims, n_q_tokens, n_cols) -> int:
+    d = dims.c()
+    return int(lib().oasis_attn_workspace_bytes(ctypes.byref(d), int(n_q_tokens), int(n_cols)))
+
+
+def sparse_attn(dims, q, n_q_tokens, hbm_pool, slot_tbl, blk_tbl, n_cols, seq_len, scale, out,
+                lse=None, workspace=None, stream=None):
+    d = dims.c()
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().oasis_sparse_attn(
+        ctypes.byref(d), _ptr(q, torch.bfloat16, "q"), int(n_q_tokens),
+        _ptr(hbm_pool, torch.bfloat16, "hbm_pool"), _ptr(slot_tbl, torch.int32, "slot_tbl"),
+        _ptr(blk_tbl, torch.int32, "blk_tbl"), int(n_cols), _ptr(seq_len, torch.int32, "seq_len"),
+        float(scale), _ptr(out, torch.bfloat16, "out"), _ptr(lse, torch.float32, "lse"),
+        _ptr(workspace, None, "workspace"), ws_bytes, _stream(stream)), "oasis_sparse_attn")
+
+
+def plan_delta(dims, sel, k, block_table, resident, stamp, slot_stride, cap, step, plan_idx,
+               plan_slots, n_admitted=None, stream=None):
+    d = dims.c()
+    _check(lib().oasis_plan_delta(
+        ctypes.byref(d), _ptr(sel, torch.int32, "sel"), int(sel.shape[-1]), int(k),
+        _ptr(block_table, torch.int32, "block_table"), _ptr(resident, torch.int32, "resident"),
+        _ptr(stamp, torch.int32, "stamp"), int(resident.shape[-1]), int(slot_stride), int(cap),
+        int(step), _ptr(plan_idx, torch.int64, "plan_idx"), _ptr(plan_slots, torch.int32, "plan_slots"),
+        _ptr(n_admitted, torch.int32, "n_admitted"), _stream(stream)), "oasis_plan_delta")

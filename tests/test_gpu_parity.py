@@ -1,0 +1,370 @@
+"""GPU parity tests: the CUDA library (through its C ABI) against the CPU oracle, element by
+element, on the same seeded inputs.  Index work must be bit-exact (fp32 near-ties adjudicated
+with the oracle's double-precision scores); attention within atol 2e-3 / rtol 1e-2."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_08097_b200 import synth
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2608_08097_b200 import build
+    build.build()
+    from paper_2608_08097_b200 import binding, pipeline
+    binding.lib()
+    return binding, pipeline
+
+
+def run_gpu_path(pipeline, lay, k, step=0, reduce_mode=0, kv_on="pinned", want_lse=True):
+    """All five calls on the GPU for one layer / step.  kv_on: where the full-KV pool lives."""
+    cfg = lay.cfg
+    dev = torch.device("cuda")
+    L = pipeline.DecodeLayer(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_blocks, k, cfg.n_q_tokens,
+                             device=dev, want_lse=want_lse)
+    if kv_on == "pinned":
+        kv = lay.host_kv if lay.host_kv.is_pinned() else lay.host_kv.pin_memory()
+    else:
+        kv = lay.host_kv.to(dev)
+    table = lay.block_table.to(dev)
+    n_full = lay.n_full_steps[step].to(dev)
+    seq_len = lay.seq_len_steps[step].to(dev)
+    q = lay.q_steps[step].to(dev)
+    zeros = torch.zeros(cfg.batch, dtype=torch.int32, device=dev)
+    L.build_summaries(kv, table, zeros, n_full, cfg.max_blocks)
+    L.score(q, n_full, reduce_mode=reduce_mode)
+    L.select(n_full, seq_len, table)
+    L.stage(kv)
+    L.attend(q, seq_len)
+    torch.cuda.synchronize()
+    return L, dict(kv=kv, table=table, n_full=n_full, seq_len=seq_len, q=q)
+
+
+def compare_path(oracle, pipeline, lay, k, step=0, reduce_mode=0, kv_on="pinned"):
+    L, dv = run_gpu_path(pipeline, lay, k, step, reduce_mode, kv_on)
+    ref = pu.oracle_layer(oracle, lay, k, reduce_mode, step)
+    cfg = lay.cfg
+    pu.assert_summaries_equal(pu.np_u16(L.summaries), ref["summ"], ref["n_full"])
+    gs = L.scores.cpu().numpy()
+    pu.assert_scores_close(gs, ref["s32"], ref["s64"], ref["n_full"])
+    gsel = L.sel.cpu().numpy()
+    n_adj = pu.assert_sel_parity(gsel, ref["sel"], ref["s64"], k)
+    # gather lists follow the GPU's own selection exactly
+    table = lay.block_table.numpy()
+    gidx, gslots = L.stage_idx.cpu().numpy(), L.stage_slots.cpu().numpy()
+    want_idx = np.where(gsel < 0, -1, np.take_along_axis(
+        np.broadcast_to(table[:, None, :], gsel.shape[:2] + (table.shape[1],)), np.maximum(gsel, 0), axis=2)
+        .astype(np.int64) * cfg.n_kv_heads + np.arange(cfg.n_kv_heads)[None, :, None])
+    assert np.array_equal(gidx, want_idx)
+    assert np.array_equal(gslots.reshape(-1), np.arange(gslots.size))
+    # staged pool: bit-exact copy of the requested entries
+    want_pool = np.zeros_like(ref["pool"])
+    oracle.stage_blocks(pu.np_u16(lay.host_kv).reshape(-1, 2, 16, 128), gidx, gslots, want_pool)
+    assert np.array_equal(pu.np_u16(L.pool), want_pool)
+    # attention on the GPU's own selection vs the oracle on that same selection
+    slot_tbl = np.arange(gsel.size, dtype=np.int32).reshape(gsel.shape)
+    ref_attn = oracle.sparse_attn(ref["q"], want_pool, slot_tbl, gsel, ref["seq_len"],
+                                  np.float32(1.0 / math.sqrt(128.0)), cfg.n_kv_heads)
+    pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref_attn["out32"])
+    np.testing.assert_allclose(L.lse.cpu().numpy(), ref_attn["lse"], rtol=1e-3, atol=2e-3)
+    # and attention on the ORACLE's selection and pool (independent of the GPU's choices)
+    if n_adj:
+        dev = torch.device("cuda")
+        L.pool.copy_(torch.from_numpy(ref["pool"].view(np.int16)).view(torch.bfloat16).to(dev))
+        L.attend(dv["q"], dv["seq_len"], blk_tbl=torch.from_numpy(ref["sel"]).to(dev))
+        torch.cuda.synchronize()
+        pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref["attn"]["out32"])
+    return L, ref, n_adj
+
+
+SMALL = [
+    # several tiles and a ragged tail in every dimension; shapes follow the five configurations
+    ("c1", dict(base="c1_single", context=1040, k_blocks=24), dict()),
+    ("c1_perm_ragged", dict(base="c1_single", batch=3, context=1232, k_blocks=16), dict(permute_table=True, ragged=True)),
+    ("c2", dict(base="c2_reasoning", batch=3, context=2064, k_blocks=40, layers=1, steps=1), dict(ragged=True)),
+    ("c3_zipf", dict(base="c3_longctx", batch=2, context=4112, k_blocks=128, layers=1), dict()),
+    ("c4_gqa8", dict(base="c4_gqa8", batch=2, context=2064, k_blocks=48, layers=1), dict(ragged=True)),
+    ("c5_td1", dict(base="c5_sweep", batch=2, context=1552, k_blocks=32, n_draft=1), dict()),
+    ("c5_td2", dict(base="c5_sweep", batch=2, context=1552, k_blocks=64, n_draft=2), dict(ragged=True)),
+    ("c5_td8", dict(base="c5_sweep", batch=2, context=1552, k_blocks=8, n_draft=8), dict()),
+    ("full_budget", dict(base="c1_single", batch=2, context=528, k_blocks=64), dict(ragged=True)),
+]
+
+
+def make_cfg(spec):
+    spec = dict(spec)
+    base = synth.CONFIGS[spec.pop("base")]
+    return synth.scaled(base, **spec)
+
+
+@pytest.mark.parametrize("name,spec,kw", SMALL, ids=[s[0] for s in SMALL])
+def test_whole_path_small(oracle, gpu, name, spec, kw):
+    _, pipeline = gpu
+    cfg = make_cfg(spec)
+    lay = synth.make_layer(cfg, seed=11, **kw)
+    compare_path(oracle, pipeline, lay, cfg.k_blocks)
+
+
+def test_full_budget_equals_dense_attention(oracle, gpu):
+    """Budget >= number of blocks: the GPU path must reproduce dense causal attention."""
+    _, pipeline = gpu
+    cfg = synth.scaled(synth.C1, batch=2, context=400, k_blocks=40)     # 25 full blocks, partial local block
+    lay = synth.make_layer(cfg, seed=5)
+    L, _ = run_gpu_path(pipeline, lay, cfg.k_blocks)
+    kv = lay.host_kv.float().numpy()
+    q = lay.q.float().numpy()
+    scale = 1.0 / math.sqrt(128.0)
+    G = cfg.group
+    out = pu.bf16_to_f32_np(L.out)
+    for b in range(cfg.batch):
+        blocks = kv[lay.block_table[b].numpy()]                        # [mb][Hkv][2][16][128]
+        for t in range(cfg.n_q_tokens):
+            n_vis = cfg.context + t + 1
+            for a in range(0, cfg.n_q_heads, 5):
+                h = a // G
+                K = blocks[:, h, 0].reshape(-1, 128)[:n_vis].astype(np.float64)
+                V = blocks[:, h, 1].reshape(-1, 128)[:n_vis].astype(np.float64)
+                logits = K @ q[b, t, a].astype(np.float64) * scale
+                w = np.exp(logits - logits.max())
+                want = (w[:, None] * V).sum(0) / w.sum()
+                assert np.all(np.abs(out[b, t, a] - want) <= pu.ATTN_ATOL + pu.ATTN_RTOL * np.abs(want))
+
+
+def test_sum_reduce_mode(oracle, gpu):
+    _, pipeline = gpu
+    cfg = synth.scaled(synth.C1, batch=2, context=1040, k_blocks=24, n_draft=3)
+    lay = synth.make_layer(cfg, seed=2, ragged=True)
+    compare_path(oracle, pipeline, lay, cfg.k_blocks, reduce_mode=1)
+
+
+def test_kv_pool_in_device_memory(oracle, gpu):
+    _, pipeline = gpu
+    cfg = synth.scaled(synth.C1, batch=2, context=784, k_blocks=16)
+    lay = synth.make_layer(cfg, seed=4, permute_table=True)
+    compare_path(oracle, pipeline, lay, cfg.k_blocks, kv_on="device")
+
+
+@pytest.mark.parametrize("Hq,Hkv,Td", [(8, 8, 1), (16, 8, 1), (32, 8, 2), (32, 8, 7), (64, 8, 5), (40, 8, 8), (128, 8, 8)])
+def test_row_counts(oracle, gpu, Hq, Hkv, Td):
+    """R = Td*G from 1 to 128 score rows; T*G from 2 to 144 would exceed 128, so Td is capped."""
+    _, pipeline = gpu
+    G = Hq // Hkv
+    if (Td + 1) * G > 128:
+        Td = 128 // G - 1
+    cfg = synth.scaled(synth.C1, batch=1, n_q_heads=Hq, n_kv_heads=Hkv, context=656, k_blocks=12, n_draft=Td)
+    lay = synth.make_layer(cfg, seed=6)
+    compare_path(oracle, pipeline, lay, cfg.k_blocks)
+
+
+def test_consecutive_steps_with_growing_context(oracle, gpu):
+    """Drift workload: 20 decode steps, the local block fills up and a new full block (with its
+    summary) appears; late steps need two local blocks (committed + T > 16)."""
+    binding, pipeline = gpu
+    cfg = synth.scaled(synth.C2, batch=2, context=1024, k_blocks=16, layers=1, steps=20)
+    lay = synth.make_layer(cfg, seed=9)
+    dev = torch.device("cuda")
+    L = pipeline.DecodeLayer(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_blocks, cfg.k_blocks,
+                             cfg.n_q_tokens, device=dev)
+    kv = lay.host_kv.pin_memory()
+    table = lay.block_table.to(dev)
+    kv_np = pu.np_u16(lay.host_kv)
+    summ_ref = None
+    for s in range(cfg.steps):
+        n_full = lay.n_full_steps[s].to(dev)
+        seq_len = lay.seq_len_steps[s].to(dev)
+        q = lay.q_steps[s].to(dev)
+        if s == 0:
+            first = torch.zeros(cfg.batch, dtype=torch.int32, device=dev)
+            count = n_full
+            max_new = cfg.max_blocks
+        else:                                  # incremental: only blocks completed since the last step
+            first = lay.n_full_steps[s - 1].to(dev)
+            count = (lay.n_full_steps[s] - lay.n_full_steps[s - 1]).to(dev)
+            max_new = 1
+        L.build_summaries(kv, table, first, count, max_new)
+        L.score(q, n_full)
+        L.select(n_full, seq_len, table)
+        L.stage(kv)
+        L.attend(q, seq_len)
+        torch.cuda.synchronize()
+        ref = pu.oracle_layer(oracle, lay, cfg.k_blocks, 0, s)
+        pu.assert_summaries_equal(pu.np_u16(L.summaries), ref["summ"], ref["n_full"])
+        gsel = L.sel.cpu().numpy()
+        n_adj = pu.assert_sel_parity(gsel, ref["sel"], ref["s64"], cfg.k_blocks)
+        if 12 <= s < 16:
+            assert (gsel[:, :, cfg.k_blocks + 1] >= 0).all()            # second local block in use
+        if n_adj == 0:
+            pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref["attn"]["out32"])
+
+
+def _select_only(binding, scores, n_full, seq_len, T, k, table=None, with_lists=True):
+    dev = torch.device("cuda")
+    B, Hkv, mb = scores.shape
+    dims = binding.Dims(B, Hkv, Hkv, mb)
+    sel = torch.full((B, Hkv, k + 2), -7, dtype=torch.int32, device=dev)
+    idx = torch.full((B, Hkv, k + 2), -7, dtype=torch.int64, device=dev) if with_lists else None
+    slots = torch.full((B, Hkv, k + 2), -7, dtype=torch.int32, device=dev) if with_lists else None
+    if table is None:
+        table = np.arange(B * mb, dtype=np.int32).reshape(B, mb)
+    binding.select_topk(dims, torch.from_numpy(scores).to(dev), torch.tensor(n_full, dtype=torch.int32, device=dev),
+                        torch.tensor(seq_len, dtype=torch.int32, device=dev), T, k, torch.from_numpy(table).to(dev),
+                        sel, idx, slots)
+    torch.cuda.synchronize()
+    return sel.cpu().numpy(), (idx.cpu().numpy() if with_lists else None)
+
+
+@pytest.mark.parametrize("n,k", [(1, 1), (5, 3), (31, 31), (33, 40), (64, 9), (1000, 128), (4096, 512),
+                                 (8192, 128), (8192, 2048), (20000, 1), (49147, 300)])
+def test_select_exact_with_ties(oracle, gpu, n, k):
+    """Integer-valued scores: masses of exact ties, so the lowest-index rule decides; exact match."""
+    binding, _ = gpu
+    rng = np.random.default_rng(n * 31 + k)
+    B, Hkv = 2, 3
+    mb = n + 5                                                       # 49147 + 5 = 49152, the largest row
+    scores = rng.integers(-4, 5, (B, Hkv, mb)).astype(np.float32)
+    scores[0, 0, :] = 1.5                                           # a row of all-equal scores
+    scores[1, 1, : min(n, 7)] = [0.0, -0.0, 0.0, -0.0, 0.0, -0.0, 0.0][: min(n, 7)]   # signed zeros are equal
+    n_full = [n, max(0, n - 3)]
+    seq_len = [n * 16 + 3, max(0, n - 3) * 16 + 14]
+    table = rng.permutation(B * mb).astype(np.int32).reshape(B, mb)
+    got, gidx = _select_only(binding, scores, n_full, seq_len, 5, k, table)
+    want, widx, _ = oracle.select_topk(scores, n_full, seq_len, 5, k, table)
+    assert np.array_equal(got, want)
+    assert np.array_equal(gidx, widx)
+
+
+def test_select_no_full_blocks_and_no_lists(oracle, gpu):
+    binding, _ = gpu
+    scores = np.zeros((1, 2, 8), np.float32)
+    got, _ = _select_only(binding, scores, [0], [3], 5, 4, with_lists=False)
+    assert (got[:, :, :4] == -1).all() and (got[:, :, 4] == 0).all() and (got[:, :, 5] == -1).all()
+    got, _ = _select_only(binding, scores, [0], [13], 5, 4, with_lists=False)
+    assert (got[:, :, 4] == 0).all() and (got[:, :, 5] == 1).all()
+
+
+def test_select_random_floats_large(oracle, gpu):
+    binding, _ = gpu
+    rng = np.random.default_rng(77)
+    scores = (rng.standard_normal((4, 8, 8200)) * 50 + 100).astype(np.float32)
+    scores[2] = -np.abs(scores[2])                                   # negative scores
+    scores[3, :, ::2] *= 1e-30                                       # wide dynamic range
+    n_full = [8192, 8000, 4097, 8192]
+    seq = [nf * 16 for nf in n_full]
+    for k in (1, 128, 513):
+        got, _ = _select_only(binding, scores, n_full, seq, 5, k)
+        want = oracle.select_topk(scores, n_full, seq, 5, k, np.arange(4 * 8200, dtype=np.int32).reshape(4, 8200),
+                                  want_stage=False)
+        assert np.array_equal(got, want)
+
+
+def test_stage_skips_negative_and_keeps_other_slots(oracle, gpu):
+    binding, _ = gpu
+    dev = torch.device("cuda")
+    rng = np.random.default_rng(3)
+    host = torch.from_numpy(rng.integers(0, 2 ** 15, (300, 2, 16, 128), dtype=np.int16)).view(torch.bfloat16).pin_memory()
+    pool = torch.from_numpy(np.full((200, 2, 16, 128), 0x3ABC, np.int16)).view(torch.bfloat16).to(dev)
+    n = 150
+    idx = rng.permutation(300)[:n].astype(np.int64)
+    idx[::7] = -1
+    slots = rng.permutation(200)[:n].astype(np.int32)
+    binding.stage_blocks(host, torch.from_numpy(idx).to(dev), torch.from_numpy(slots).to(dev), n, pool)
+    torch.cuda.synchronize()
+    want = np.full((200, 2, 16, 128), 0x3ABC, np.uint16)
+    oracle.stage_blocks(pu.np_u16(host), idx, slots, want)
+    assert np.array_equal(pu.np_u16(pool), want)
+    binding.stage_blocks(host, torch.from_numpy(idx).to(dev), torch.from_numpy(slots).to(dev), 0, pool)   # n = 0: no-op
+
+
+def test_attention_padding_rows_and_empty_columns(oracle, gpu):
+    """Columns of -1 anywhere in the table (not only at the end), rows that see nothing."""
+    binding, pipeline = gpu
+    cfg = synth.scaled(synth.C1, batch=2, context=640, k_blocks=20)
+    lay = synth.make_layer(cfg, seed=8)
+    L, dv = run_gpu_path(pipeline, lay, cfg.k_blocks)
+    sel = L.sel.cpu().numpy().copy()
+    sel[:, :, 3::4] = -1                                              # punch holes
+    sel[1, 2, :] = -1                                                 # one row sees no key at all
+    dev = torch.device("cuda")
+    L.attend(dv["q"], dv["seq_len"], blk_tbl=torch.from_numpy(sel).to(dev))
+    torch.cuda.synchronize()
+    slot_tbl = np.arange(sel.size, dtype=np.int32).reshape(sel.shape)
+    ref = oracle.sparse_attn(pu.np_u16(lay.q), pu.np_u16(L.pool), slot_tbl, sel, lay.seq_len.numpy(),
+                             np.float32(1.0 / math.sqrt(128.0)), cfg.n_kv_heads)
+    pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref["out32"])
+    G = cfg.group
+    assert (pu.bf16_to_f32_np(L.out)[1, :, 2 * G:3 * G] == 0).all()
+    assert np.isneginf(L.lse.cpu().numpy()[1, :, 2 * G:3 * G]).all()
+
+
+def test_empty_batch_is_a_no_op(gpu):
+    binding, _ = gpu
+    dev = torch.device("cuda")
+    dims = binding.Dims(0, 32, 8, 64)
+    e16 = torch.empty(16, dtype=torch.bfloat16, device=dev)
+    e32 = torch.empty(16, dtype=torch.int32, device=dev)
+    ef = torch.empty(16, dtype=torch.float32, device=dev)
+    binding.build_summaries(dims, e16, e32, e32, e32, 4, e16)
+    binding.score_blocks(dims, e16, 4, e16, e32, ef, q_batch_stride=4 * 32 * 128)
+    binding.select_topk(dims, ef, e32, e32, 5, 4, e32, e32)
+    binding.sparse_attn(dims, e16, 5, e16, e32, e32, 6, e32, 0.1, e16)
+    torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("cap_ratio", [0.05, 0.2, 1.0])
+def test_plan_delta_matches_oracle_over_steps(oracle, gpu, cap_ratio):
+    """Delta selection + capped eviction (KV selection stage) over the drift workload: resident
+    table, stamps and gather plan must equal the oracle's exactly at every step, and after the
+    planned gathers every resident column must hold exactly its block's bytes."""
+    binding, pipeline = gpu
+    cfg = synth.scaled(synth.C2, batch=2, context=2048, k_blocks=32, layers=1, steps=12)
+    lay = synth.make_layer(cfg, seed=21)
+    dev = torch.device("cuda")
+    k = cfg.k_blocks
+    cap = max(1, int(math.floor(cap_ratio * k)))
+    L = pipeline.DecodeLayer(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_blocks, k, cfg.n_q_tokens, device=dev)
+    kv = lay.host_kv.pin_memory()
+    kv_np = pu.np_u16(lay.host_kv).reshape(-1, 2, 16, 128)
+    table = lay.block_table.to(dev)
+    B, Hkv = cfg.batch, cfg.n_kv_heads
+    resident = torch.full((B, Hkv, k), -1, dtype=torch.int32, device=dev)
+    stamp = torch.zeros((B, Hkv, k), dtype=torch.int32, device=dev)
+    plan_idx = torch.empty((B, Hkv, cap), dtype=torch.int64, device=dev)
+    plan_slots = torch.empty((B, Hkv, cap), dtype=torch.int32, device=dev)
+    n_adm = torch.empty((B, Hkv), dtype=torch.int32, device=dev)
+    res_ref = np.full((B, Hkv, k), -1, np.int32)
+    stamp_ref = np.zeros((B, Hkv, k), np.int32)
+    zeros = torch.zeros(B, dtype=torch.int32, device=dev)
+    L.build_summaries(kv, table, zeros, lay.n_full_steps[-1].to(dev), cfg.max_blocks)
+    for s in range(cfg.steps):
+        n_full = lay.n_full_steps[s].to(dev)
+        L.score(lay.q_steps[s].to(dev), n_full)
+        L.select(n_full, lay.seq_len_steps[s].to(dev), table)
+        binding.plan_delta(L.dims, L.sel, k, table, resident, stamp, L.cols, cap, s + 1, plan_idx, plan_slots, n_adm)
+        binding.stage_blocks(kv, plan_idx, plan_slots, plan_idx.numel(), L.pool)
+        torch.cuda.synchronize()
+        sel_np = L.sel.cpu().numpy()
+        ridx, rslots, radm = oracle.plan_delta(sel_np, lay.block_table.numpy(), res_ref, stamp_ref, k, cap, s + 1, L.cols)
+        assert np.array_equal(resident.cpu().numpy(), res_ref)
+        assert np.array_equal(stamp.cpu().numpy(), stamp_ref)
+        assert np.array_equal(n_adm.cpu().numpy(), radm)
+        gi, gs = plan_idx.cpu().numpy(), plan_slots.cpu().numpy()
+        assert np.array_equal(gi, ridx)
+        assert np.array_equal(np.where(gi >= 0, gs, 0), np.where(ridx >= 0, rslots, 0))
+        assert (radm <= cap).all()
+        # the pool mirrors the resident table
+        pool_np = pu.np_u16(L.pool)
+        for b in range(B):
+            for h in range(Hkv):
+                for c in range(0, k, 5):
+                    j = res_ref[b, h, c]
+                    if j >= 0:
+                        src = int(lay.block_table[b, j]) * Hkv + h
+                        assert np.array_equal(pool_np[(b * Hkv + h) * L.cols + c], kv_np[src])
