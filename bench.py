@@ -1,0 +1,491 @@
+#!/usr/bin/env python
+"""Benchmark of the OasisKV decode hot path on B200: one JSON line per run.
+
+A "step" is one decode step of the reasoning-style workload (batch 16, 32 layers, 32 q / 8 KV
+heads, 32,768-token context in 16-token blocks, budget 2,048 tokens, 4 draft tokens, drifting
+heavy hitters): per layer, sparse attention over the working set staged by the previous step,
+then summary update, block scoring with the draft queries, top-k, and the gather of the
+selected blocks on a side stream.  metric = tokens/s per layer = batch / (step time / layers).
+
+  value : full-KV pool mirrored in HBM (all inputs resident in HBM), fetch-all gather.
+  e2e   : full-KV pool in pinned host memory (the gather crosses the host link), queries copied
+          host->device and outputs device->host inside every step, fetch-all gather.
+Extra keys report the capped-delta gather, the gather's GB/s against the measured pinned
+host->device peak, the per-kernel HBM rooflines, lookahead recall and the CPU-oracle baseline.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+"""
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2608_08097_b200 import synth  # noqa: E402
+
+METRIC = "sparse decode-attn+select tokens/s per layer"
+UNIT = "tokens/s/layer"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=None, help="override the number of layers (debugging)")
+    ap.add_argument("--batch", type=int, default=None, help="override the batch (debugging)")
+    ap.add_argument("--context", type=int, default=None, help="override the context length (debugging)")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--fetch-ratio", type=float, default=0.05, help="cap of the delta gather, fraction of K")
+    ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--skip-cpu", action="store_true")
+    return ap.parse_args()
+
+
+def workload(args):
+    kw = {}
+    if args.layers:
+        kw["layers"] = args.layers
+    if args.batch:
+        kw["batch"] = args.batch
+    if args.context:
+        kw["context"] = args.context
+    need_steps = args.steps + max(args.warmup, 3) + 1
+    if need_steps > synth.C2.steps:
+        kw["steps"] = need_steps
+    return synth.scaled(synth.C2, **kw) if kw else synth.C2
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while a region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        fd, self.path = tempfile.mkstemp(suffix=".csv")
+        os.close(fd)
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        rows = []
+        with open(self.path) as f:
+            for line in f:
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) >= 7:
+                    try:
+                        rows.append((float(parts[0]), float(parts[1]), parts[3:7]))
+                    except ValueError:
+                        pass
+        os.unlink(self.path)
+        if rows:
+            clocks = sorted(r[0] for r in rows)
+            out["sm_mhz"] = clocks[len(clocks) // 2]
+            out["sm_max_mhz"] = rows[0][1]
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            out["reasons"] = [n for i, n in enumerate(names) if any(r[2][i].lower().startswith("active") for r in rows)]
+            out["samples"] = len(rows)
+        return out
+
+
+def dist_setup(args):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl" if torch.cuda.is_available() else "gloo")
+    return world, rank, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(x, world, device):
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# ------------------------------------------------------------------------------------------- ours
+
+
+def time_pinned_h2d(device):
+    """Pinned host -> device copy bandwidth, 1 GiB, best of 10 (GB/s)."""
+    n = 1 << 30
+    src = torch.empty(n, dtype=torch.uint8, pin_memory=True)
+    dst = torch.empty(n, dtype=torch.uint8, device=device)
+    best = 0.0
+    for _ in range(10):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        dst.copy_(src, non_blocking=True)
+        b.record()
+        b.synchronize()
+        best = max(best, n / (a.elapsed_time(b) * 1e-3) / 1e9)
+    del src, dst
+    return best
+
+
+class Bench:
+    def __init__(self, args, cfg, device, rank):
+        from paper_2608_08097_b200 import build
+        build.build()
+        from paper_2608_08097_b200 import binding, pipeline
+        binding.lib()
+        self.args, self.cfg, self.dev, self.rank = args, cfg, device, rank
+        self.binding, self.pipeline = binding, pipeline
+        self.n_layers = cfg.layers
+        self.host_kv, self.mirror, self.tables = [], [], []
+        self.q_dev, self.q_true_dev = [], []
+        self.sample_layer = None
+
+    def generate(self, want_mirror, want_host):
+        cfg = self.cfg
+        t0 = time.time()
+        for l in range(self.n_layers):
+            P = cfg.batch * cfg.max_blocks
+            host = torch.empty((P, cfg.n_kv_heads, 2, 16, 128), dtype=torch.bfloat16, pin_memory=True)
+            lay = synth.make_layer(cfg, seed=self.args.seed + 7919 * self.rank, layer=l, device=self.dev, out_kv=host)
+            self.tables.append(lay.block_table.to(self.dev))
+            self.q_dev.append(lay.q_steps.to(self.dev))
+            self.q_true_dev.append(lay.q_true_steps.to(self.dev))
+            if want_mirror:
+                self.mirror.append(host.to(self.dev, non_blocking=False))
+            if want_host:
+                self.host_kv.append(host)
+            if l == 0:
+                self.seq_steps = lay.seq_len_steps.clone()
+                self.sample_layer = lay if want_host else None
+            if not want_host:
+                del host
+        S = cfg.steps
+        seq = self.seq_steps                                            # [S][B] int32 (host)
+        self.seq_dev = seq.to(self.dev)
+        self.first_dev = (seq // 16).to(torch.int32).to(self.dev)       # full blocks before the step's commit
+        self.seq_next_dev = (seq + 1).to(torch.int32).to(self.dev)
+        self.nfull_next_dev = ((seq + 1) // 16).to(torch.int32).to(self.dev)
+        self.n_new_dev = (self.nfull_next_dev - self.first_dev).contiguous()
+        self.gen_seconds = time.time() - t0
+
+    def engine(self, mode, kv_list, cap=None):
+        cfg = self.cfg
+        eng = self.pipeline.DecodeEngine(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_blocks, cfg.k_blocks,
+                                         cfg.n_q_tokens, self.n_layers, self.dev, mode=mode, cap=cap)
+        for l in range(self.n_layers):
+            eng.attach(l, kv_list[l], self.tables[l])
+        eng.prime([self.q_dev[l][0] for l in range(self.n_layers)], self.first_dev[0].contiguous(), self.seq_dev[0].contiguous())
+        return eng
+
+    def run_steps(self, eng, steps, timers=None, e2e=False, q_pinned=None, out_pinned=None, q_stage=None):
+        for s in steps:
+            if e2e:
+                q_list = q_stage
+                q_host = [q_pinned[l][s] for l in range(self.n_layers)]
+            else:
+                q_list = [self.q_dev[l][s] for l in range(self.n_layers)]
+                q_host = None
+            eng.step(q_list, self.seq_dev[s], self.first_dev[s], self.n_new_dev[s], self.nfull_next_dev[s],
+                     self.seq_next_dev[s], step_stamp=s + 1, timers=timers, q_host=q_host,
+                     out_host=out_pinned if e2e else None)
+
+    def timed(self, eng, world, W, K, e2e=False, collect=True, **kw):
+        """W warm-up steps, then exactly K timed steps; returns (ms per step, timers, clocks)."""
+        self.run_steps(eng, range(0, W), e2e=e2e, **kw)
+        eng.join()
+        torch.cuda.synchronize()
+        timers = {"score": [], "select": [], "attn": [], "stage": []} if collect else None
+        sampler = ClockSampler(self.dev.index or 0)
+        sampler.start()
+        barrier(world)
+        torch.cuda.synchronize()
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = eng.launches
+        start.record(eng.main)
+        self.run_steps(eng, range(W, W + K), timers=timers, e2e=e2e, **kw)
+        eng.join()
+        end.record(eng.main)
+        torch.cuda.synchronize()
+        barrier(world)
+        clocks = sampler.stop()
+        ms = start.elapsed_time(end) / K
+        ms = max_over_ranks(ms, world, self.dev)
+        launches = eng.launches - l0
+        per_kernel = {}
+        if timers:
+            for name, pairs in timers.items():
+                if pairs:
+                    per_kernel[name] = sum(a.elapsed_time(b) for a, b in pairs) / len(pairs) * 1e3   # us per launch
+        return ms, per_kernel, clocks, launches
+
+    def recall(self, eng, steps):
+        """Share of the draft-predicted top-k also chosen by the true next-step queries."""
+        cfg = self.cfg
+        tot, n = 0.0, 0
+        for l in range(0, self.n_layers, max(1, self.n_layers // 4)):
+            L = eng.layers[l]
+            sel_true = torch.empty_like(L.sel)
+            for s in steps:
+                with torch.cuda.stream(eng.main):
+                    L.score(self.q_dev[l][s], self.nfull_next_dev[s])
+                    L.select(self.nfull_next_dev[s], self.seq_next_dev[s], self.tables[l])
+                    sel_draft = L.sel.clone()
+                    L.score_queries(self.q_true_dev[l][s], self.nfull_next_dev[s])
+                    L.select(self.nfull_next_dev[s], self.seq_next_dev[s], self.tables[l], sel=sel_true)
+                eng.main.synchronize()
+                a = sel_draft[..., :cfg.k_blocks]
+                b = sel_true[..., :cfg.k_blocks]
+                hit = (a[..., :, None] == b[..., None, :]).any(-1).float().mean().item()
+                tot, n = tot + hit, n + 1
+        return tot / max(n, 1)
+
+
+def algorithmic_bytes(cfg, seq_steps, steps):
+    """Per-launch algorithmic bytes of the scoring and attention kernels, averaged over steps."""
+    B, Hkv, T, Hq = cfg.batch, cfg.n_kv_heads, cfg.n_q_tokens, cfg.n_q_heads
+    score, attn = 0.0, 0.0
+    for s in steps:
+        L = seq_steps[s].to(torch.int64)
+        nfull_next = (L + 1) // 16
+        score += float((nfull_next * Hkv * (512 + 4)).sum())
+        nfull = L // 16
+        n_local = (L + T + 15) // 16 - nfull
+        cols = torch.minimum(nfull, torch.tensor(cfg.k_blocks)) + n_local
+        attn += float((cols * Hkv * 8192).sum()) + 2.0 * B * T * Hq * 128 * 2
+    return score / len(steps), attn / len(steps)
+
+
+def cpu_baseline(cfg, lay, budget_s=20.0):
+    """The oracle, as it stands, on this host: one layer of one step, request by request
+    (score + top-k + gather + attention), until about `budget_s` seconds are spent."""
+    import numpy as np
+    from oracle import oracle
+    oracle.lib()
+    kv = synth.u16(lay.host_kv)
+    table = lay.block_table.numpy()
+    mb = cfg.max_blocks
+    done, t_used = 0, 0.0
+    for b in range(cfg.batch):
+        tb = table[b:b + 1]
+        n_full = lay.n_full.numpy()[b:b + 1]
+        seq = lay.seq_len.numpy()[b:b + 1]
+        q = synth.u16(lay.q[b:b + 1])
+        summ = oracle.build_summaries(kv, tb, np.zeros(1, np.int32), n_full)          # set-up, not timed
+        t0 = time.perf_counter()
+        s32, _ = oracle.score_blocks(q[:, 1:], summ, n_full)
+        sel, idx, slots = oracle.select_topk(s32, n_full, seq, cfg.n_q_tokens, cfg.k_blocks, tb)
+        pool = np.zeros((cfg.n_kv_heads * (cfg.k_blocks + 2), 2, 16, 128), np.uint16)
+        oracle.stage_blocks(kv.reshape(-1, 2, 16, 128), idx, slots, pool)
+        oracle.sparse_attn(q, pool, slots.reshape(1, cfg.n_kv_heads, -1), sel, seq,
+                           np.float32(1.0 / math.sqrt(128.0)), cfg.n_kv_heads)
+        t_used += time.perf_counter() - t0
+        done += 1
+        if t_used >= budget_s:
+            break
+    return {"value": done / t_used, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": "layer 0, step 0, %d of %d requests, score+top-k+gather+attention, single thread (%.1f s)"
+                      % (done, cfg.batch, t_used)}
+
+
+def run_ours(args):
+    world, rank, local = dist_setup(args)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    cfg = workload(args)
+    W, K = max(args.warmup, 3), args.steps
+    hbm_peak, peak_kind = measured_peaks()
+    bench = Bench(args, cfg, dev, rank)
+    h2d_peak = time_pinned_h2d(dev)
+    bench.generate(want_mirror=True, want_host=not args.skip_e2e)
+
+    # ---- value: everything resident in HBM ---------------------------------------------------
+    eng = bench.engine("fetch_all", bench.mirror)
+    ms, per_kernel, clocks, launches = bench.timed(eng, world, W, K)
+    steps = range(W, W + K)
+    score_bytes, attn_bytes = algorithmic_bytes(cfg, bench.seq_steps, steps)
+    kern = {}
+    for name, nbytes in (("score", score_bytes), ("attn", attn_bytes)):
+        if name in per_kernel:
+            gbs = nbytes / (per_kernel[name] * 1e-6) / 1e9
+            kern[name] = {"us": round(per_kernel[name], 2), "algorithmic_MB": round(nbytes / 1e6, 2),
+                          "GBps": round(gbs, 1), "frac_of_measured": round(gbs / hbm_peak, 3),
+                          "frac_of_8TBps": round(gbs / 8000.0, 3)}
+    stage_bytes = cfg.batch * cfg.n_kv_heads * (cfg.k_blocks + 1) * 8192
+    if "stage" in per_kernel:
+        kern["stage_hbm_to_hbm"] = {"us": round(per_kernel["stage"], 2),
+                                    "GBps_read_plus_write": round(2 * stage_bytes / (per_kernel["stage"] * 1e-6) / 1e9, 1)}
+    if "select" in per_kernel:
+        kern["select"] = {"us": round(per_kernel["select"], 2)}
+    dominant = max(("score", "attn"), key=lambda n: per_kernel.get(n, 0.0))
+    value = cfg.batch * world / (ms * 1e-3 / cfg.layers)
+    recall = bench.recall(eng, range(W, min(W + 4, W + K)))
+
+    # compute only (no gather), for the overlap accounting
+    extra = {}
+    eng_d = bench.engine("delta", bench.mirror, cap=max(1, int(math.floor(args.fetch_ratio * cfg.k_blocks))))
+    ms_d, _, _, _ = bench.timed(eng_d, world, W, K, collect=False)
+    extra["value_delta_cap"] = {"fetch_ratio": args.fetch_ratio, "ms_per_step": round(ms_d, 4),
+                                "value": round(cfg.batch * world / (ms_d * 1e-3 / cfg.layers), 1)}
+    del eng_d, eng
+    bench.mirror.clear()
+    torch.cuda.empty_cache()
+
+    # ---- e2e: KV in pinned host memory, queries in / outputs out every step -----------------------
+    e2e = None
+    if not args.skip_e2e:
+        q_pinned = [q.cpu().pin_memory() for q in bench.q_dev]
+        q_stage = [torch.empty_like(bench.q_dev[l][0]) for l in range(cfg.layers)]
+        out_pinned = [torch.empty((cfg.batch, cfg.n_q_tokens, cfg.n_q_heads, 128), dtype=torch.bfloat16,
+                                  pin_memory=True) for _ in range(cfg.layers)]
+        kw = dict(q_pinned=q_pinned, out_pinned=out_pinned, q_stage=q_stage)
+        Ke = min(K, 8)
+        eng = bench.engine("fetch_all", bench.host_kv)
+        ms_e, pk_e, _, _ = bench.timed(eng, world, W, Ke, e2e=True, **kw)
+        h2d = cfg.layers * (stage_bytes + cfg.batch * cfg.n_q_tokens * cfg.n_q_heads * 128 * 2)
+        d2h = cfg.layers * cfg.batch * cfg.n_q_tokens * cfg.n_q_heads * 128 * 2
+        e2e = {"value": round(cfg.batch * world / (ms_e * 1e-3 / cfg.layers), 1), "unit": UNIT,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "ms_per_step": round(ms_e, 3),
+               "steps": Ke, "gather": "fetch-all (every selected block crosses the host link each step)"}
+        if "stage" in pk_e:
+            gbs = stage_bytes / (pk_e["stage"] * 1e-6) / 1e9
+            extra["staged"] = {"GBps_overlapped": round(gbs, 2), "pinned_h2d_peak_GBps": round(h2d_peak, 2),
+                               "frac_of_h2d_peak": round(gbs / h2d_peak, 3), "us_per_layer": round(pk_e["stage"], 1)}
+        del eng
+        cap = max(1, int(math.floor(args.fetch_ratio * cfg.k_blocks)))
+        eng = bench.engine("delta", bench.host_kv, cap=cap)
+        ms_ed, pk_ed, _, _ = bench.timed(eng, world, W, K, e2e=True, **kw)
+        extra["e2e_delta_cap"] = {"fetch_ratio": args.fetch_ratio, "cap_blocks": cap, "ms_per_step": round(ms_ed, 4),
+                                  "value": round(cfg.batch * world / (ms_ed * 1e-3 / cfg.layers), 1),
+                                  "h2d_bytes_per_step": int(cfg.layers * cfg.batch * cfg.n_kv_heads * (cap + 1) * 8192)}
+        del eng
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.skip_cpu and bench.sample_layer is not None:
+        cpu = cpu_baseline(cfg, bench.sample_layer)
+
+    if rank == 0:
+        d = kern.get(dominant, {})
+        line = {
+            "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": round(ms, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "configs[1] reasoning-style decode: batch %d, %d layers, %dq/%dkv heads, d128, "
+                                   "context %d (+1 per step), 16-token blocks, budget %d tokens, %d draft tokens"
+                                   % (cfg.batch, cfg.layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.context,
+                                      cfg.k_blocks * 16, cfg.n_draft),
+                       "global_batch": cfg.batch * world, "parallelism": "replicas x%d" % world,
+                       "l2": "inputs larger than L2: each step streams %d layers x %.0f MB of distinct summaries + staged KV"
+                             % (cfg.layers, (score_bytes + attn_bytes) / 1e6),
+                       "gather": "fetch-all from an HBM mirror of the full KV (value); pinned host (e2e)"},
+            "gpu_launches": launches,
+            "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"]},
+            "roofline": {"bound": "hbm", "kernel": dominant, "achieved": d.get("GBps"), "peak": hbm_peak,
+                         "unit": "GB/s", "frac": d.get("frac_of_measured"), "traffic": None,
+                         "peak_kind": peak_kind + " (STREAM-style copy)"},
+            "kernels": kern,
+            "recall_lookahead_topk": round(recall, 4),
+            "e2e": e2e, "cpu_baseline": cpu, "setup_seconds": round(bench.gen_seconds, 1),
+        }
+        line.update(extra)
+        print(json.dumps(line))
+
+
+# -------------------------------------------------------------------------------------- reference
+
+
+def run_reference(args):
+    """The CPU oracle, as it stands, timed on this host's cores on the same workload; every
+    step is a bounded sample (one request of one layer)."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    from oracle import oracle
+    oracle.lib()
+    cfg = workload(args)
+    one = synth.scaled(cfg, batch=1, layers=1, steps=1)
+    lay = synth.make_layer(one, seed=args.seed, layer=0, device="cpu")
+    kv = synth.u16(lay.host_kv)
+    table, n_full, seq = lay.block_table.numpy(), lay.n_full.numpy(), lay.seq_len.numpy()
+    q = synth.u16(lay.q)
+    summ = oracle.build_summaries(kv, table, np.zeros(1, np.int32), n_full)
+
+    def one_step():
+        s32, _ = oracle.score_blocks(q[:, 1:], summ, n_full)
+        sel, idx, slots = oracle.select_topk(s32, n_full, seq, one.n_q_tokens, one.k_blocks, table)
+        pool = np.zeros((one.n_kv_heads * (one.k_blocks + 2), 2, 16, 128), np.uint16)
+        oracle.stage_blocks(kv.reshape(-1, 2, 16, 128), idx, slots, pool)
+        oracle.sparse_attn(q, pool, slots.reshape(1, one.n_kv_heads, -1), sel, seq,
+                           np.float32(1.0 / math.sqrt(128.0)), one.n_kv_heads)
+
+    W, K = max(args.warmup, 1), args.steps
+    for _ in range(W):
+        one_step()
+    t0 = time.perf_counter()
+    for _ in range(K):
+        one_step()
+    dt = (time.perf_counter() - t0) / K
+    value = 1.0 / dt                     # one request through one layer per sample
+    sample = "each step = 1 request x 1 layer of the workload (score+top-k+gather+attention), single thread"
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world,
+            "steps": K, "warmup": W, "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "configs[1] reasoning-style decode (bounded sample): %s" % sample},
+            "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

@@ -165,18 +165,24 @@ size_t oasis_attn_workspace_bytes(const oasis_dims_t *dims, int32_t n_q_tokens,
  *      takes the block and stamp `step`, and a gather request is emitted:
  *      plan_idx = block_table[b][block] * Hkv + h, plan_slots = row * slot_stride + column
  *      with row = b * Hkv + h.  All other columns are left unchanged.
- *   sel         [B][Hkv][sel_cols] int32, k <= sel_cols
- *   resident, stamp   [B][Hkv][n_res] int32, updated in place (resident can serve as the
- *               first n_res columns of an attention blk_tbl when n_res == its row length)
- *   plan_idx [B][Hkv][cap] int64, plan_slots [B][Hkv][cap] int32: unused requests have
- *               idx = -1; n_admitted [B][Hkv] int32 (may be NULL)
- * 1 <= k <= OASIS_MAX_K, 1 <= n_res <= OASIS_MAX_K, 0 <= cap <= k.
+ *   5. the n_local (0..2) always-kept local blocks sel[b][h][k .. k+n_local) (Sec. 4.3:
+ *      the selected blocks and a local window stay in GPU memory) are copied to columns
+ *      n_res .. n_res+n_local-1 of the row, stamps untouched, and requested unconditionally.
+ *   sel         [B][Hkv][sel_cols] int32, k + n_local <= sel_cols
+ *   resident, stamp   [B][Hkv][res_stride] int32, updated in place, res_stride >= n_res +
+ *               n_local; with res_stride = n_res + n_local, resident is directly the blk_tbl
+ *               of oasis_sparse_attn
+ *   plan_idx [B][Hkv][cap + n_local] int64, plan_slots (same shape) int32: the pairs first,
+ *               then the local blocks; unused requests have idx = -1
+ *   n_admitted  [B][Hkv] int32 number of pairs (may be NULL)
+ * 1 <= k <= OASIS_MAX_K, 1 <= n_res <= OASIS_MAX_K, 0 <= cap <= k, slot_stride >= n_res +
+ * n_local, max_blocks <= 524288.
  */
 int oasis_plan_delta(const oasis_dims_t *dims, const int32_t *sel, int32_t sel_cols, int32_t k,
                      const int32_t *block_table, int32_t *resident, int32_t *stamp,
-                     int32_t n_res, int32_t slot_stride, int32_t cap, int32_t step,
-                     int64_t *plan_idx, int32_t *plan_slots, int32_t *n_admitted,
-                     void *stream);
+                     int32_t n_res, int32_t res_stride, int32_t n_local, int32_t slot_stride,
+                     int32_t cap, int32_t step, int64_t *plan_idx, int32_t *plan_slots,
+                     int32_t *n_admitted, void *stream);
 
 /* Description of the calling thread's most recent error ("" if none). Static storage. */
 const char *oasis_last_error(void);

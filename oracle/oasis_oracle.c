@@ -381,11 +381,16 @@ double oasis_oracle_topk_recall(int32_t rows, int32_t cols, int32_t k,
  *      resident[target] = candidate, stamp[target] = step, and the pair is emitted as
  *      a gather request (source entry block_table[b][cand]*Hkv + h, destination slot
  *      row*slot_stride + target); every other column is left unchanged.
- * plan_idx / plan_slots hold cap requests per row, unused ones with idx = -1.
- * n_admitted[row] receives the number of pairs.
+ *   5. Sec. 4.3 keeps a local window next to the selected blocks: the n_local always-kept
+ *      local block ids sel[row][k .. k+n_local) are copied to columns n_res .. n_res+n_local-1
+ *      of the row (their stamps untouched) and requested unconditionally.
+ * resident / stamp rows are res_stride apart (res_stride >= n_res + n_local).
+ * plan_idx / plan_slots hold cap + n_local requests per row (pairs first, then the local
+ * blocks), unused ones with idx = -1.  n_admitted[row] receives the number of pairs.
  */
 void oasis_oracle_plan_delta(int32_t B, int32_t Hkv, int32_t max_blocks, int32_t k,
-                             int32_t sel_cols, int32_t n_res, int32_t slot_stride,
+                             int32_t sel_cols, int32_t n_res, int32_t res_stride,
+                             int32_t n_local, int32_t slot_stride,
                              int32_t cap, int32_t step, const int32_t *sel,
                              const int32_t *block_table, int32_t *resident,
                              int32_t *stamp, int64_t *plan_idx, int32_t *plan_slots,
@@ -397,8 +402,9 @@ void oasis_oracle_plan_delta(int32_t B, int32_t Hkv, int32_t max_blocks, int32_t
         for (int32_t h = 0; h < Hkv; ++h) {
             const int64_t row = (int64_t)b * Hkv + h;
             const int32_t *pred = sel + row * sel_cols;
-            int32_t *res = resident + row * n_res;
-            int32_t *stp = stamp + row * n_res;
+            int32_t *res = resident + row * res_stride;
+            int32_t *stp = stamp + row * res_stride;
+            const int32_t plan_cols = cap + n_local;
             int32_t n_cand = 0, n_target = 0;
             /* 1 + 3a: hits keep their column; the others are eviction targets */
             for (int32_t c = 0; c < n_res; ++c) {
@@ -436,19 +442,28 @@ void oasis_oracle_plan_delta(int32_t B, int32_t Hkv, int32_t max_blocks, int32_t
             int32_t n_pair = cap;
             if (n_cand < n_pair) n_pair = n_cand;
             if (n_target < n_pair) n_pair = n_target;
-            for (int32_t i = 0; i < cap; ++i) {
-                plan_idx[row * cap + i] = -1;
-                plan_slots[row * cap + i] = 0;
+            for (int32_t i = 0; i < plan_cols; ++i) {
+                plan_idx[row * plan_cols + i] = -1;
+                plan_slots[row * plan_cols + i] = 0;
             }
             for (int32_t i = 0; i < n_pair; ++i) {
                 int32_t c = target[i];
                 res[c] = cand[i];
                 stp[c] = step;
-                plan_idx[row * cap + i] =
+                plan_idx[row * plan_cols + i] =
                     (int64_t)block_table[(int64_t)b * max_blocks + cand[i]] * Hkv + h;
-                plan_slots[row * cap + i] = (int32_t)(row * slot_stride + c);
+                plan_slots[row * plan_cols + i] = (int32_t)(row * slot_stride + c);
             }
             n_admitted[row] = n_pair;
+            /* 5: the local window */
+            for (int32_t i = 0; i < n_local; ++i) {
+                int32_t j = pred[k + i];
+                res[n_res + i] = j;
+                plan_slots[row * plan_cols + cap + i] = (int32_t)(row * slot_stride + n_res + i);
+                if (j >= 0)
+                    plan_idx[row * plan_cols + cap + i] =
+                        (int64_t)block_table[(int64_t)b * max_blocks + j] * Hkv + h;
+            }
         }
     }
     free(cand);

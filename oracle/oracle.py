@@ -131,19 +131,22 @@ def topk_recall(sel_draft, sel_true, k):
     return float(lib().oasis_oracle_topk_recall(rows, cols, int(k), _p(sel_draft), _p(sel_true)))
 
 
-def plan_delta(sel, block_table, resident, stamp, k, cap, step, slot_stride):
-    """Updates resident/stamp [B][Hkv][n_res] in place; returns (plan_idx int64
-    [B][Hkv][cap], plan_slots int32 [B][Hkv][cap], n_admitted [B][Hkv])."""
+def plan_delta(sel, block_table, resident, stamp, k, cap, step, slot_stride, n_res=None, n_local=0):
+    """Updates resident/stamp [B][Hkv][res_stride] in place (n_res eviction-managed columns,
+    then n_local local-block columns); returns (plan_idx int64 [B][Hkv][cap+n_local],
+    plan_slots int32 (same shape), n_admitted [B][Hkv])."""
     sel, block_table = _i32(sel), _i32(block_table)
     assert resident.dtype == np.int32 and resident.flags.c_contiguous
     assert stamp.dtype == np.int32 and stamp.flags.c_contiguous
     B, Hkv, sel_cols = sel.shape
-    n_res = resident.shape[-1]
+    res_stride = resident.shape[-1]
+    n_res = res_stride - n_local if n_res is None else n_res
     max_blocks = block_table.shape[-1]
-    plan_idx = np.empty((B, Hkv, max(cap, 0)), dtype=np.int64)
-    plan_slots = np.empty((B, Hkv, max(cap, 0)), dtype=np.int32)
+    plan_idx = np.empty((B, Hkv, max(cap, 0) + n_local), dtype=np.int64)
+    plan_slots = np.empty((B, Hkv, max(cap, 0) + n_local), dtype=np.int32)
     n_adm = np.empty((B, Hkv), dtype=np.int32)
-    lib().oasis_oracle_plan_delta(B, Hkv, max_blocks, int(k), sel_cols, n_res, int(slot_stride),
-                                  int(cap), int(step), _p(sel), _p(block_table), _p(resident),
-                                  _p(stamp), _p(plan_idx), _p(plan_slots), _p(n_adm))
+    lib().oasis_oracle_plan_delta(B, Hkv, max_blocks, int(k), sel_cols, int(n_res), int(res_stride),
+                                  int(n_local), int(slot_stride), int(cap), int(step), _p(sel),
+                                  _p(block_table), _p(resident), _p(stamp), _p(plan_idx),
+                                  _p(plan_slots), _p(n_adm))
     return plan_idx, plan_slots, n_adm

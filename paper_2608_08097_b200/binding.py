@@ -66,7 +66,7 @@ def lib():
         L.oasis_sparse_attn.argtypes = [dp, vp, i32, vp, vp, vp, i32, vp, f32, vp, vp, vp, sz, vp]
         L.oasis_attn_workspace_bytes.argtypes = [dp, i32, i32]
         L.oasis_attn_workspace_bytes.restype = sz
-        L.oasis_plan_delta.argtypes = [dp, vp, i32, i32, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
+        L.oasis_plan_delta.argtypes = [dp, vp, i32, i32, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
         for name in ("oasis_build_summaries", "oasis_score_blocks", "oasis_select_topk",
                      "oasis_stage_blocks", "oasis_sparse_attn", "oasis_plan_delta"):
             getattr(L, name).restype = ctypes.c_int
@@ -164,11 +164,14 @@ def sparse_attn(dims, q, n_q_tokens, hbm_pool, slot_tbl, blk_tbl, n_cols, seq_le
 
 
 def plan_delta(dims, sel, k, block_table, resident, stamp, slot_stride, cap, step, plan_idx,
-               plan_slots, n_admitted=None, stream=None):
+               plan_slots, n_admitted=None, n_local=0, stream=None):
+    """resident / stamp are [B][Hkv][n_res + n_local]; plan lists [B][Hkv][cap + n_local]."""
     d = dims.c()
+    res_stride = int(resident.shape[-1])
     _check(lib().oasis_plan_delta(
         ctypes.byref(d), _ptr(sel, torch.int32, "sel"), int(sel.shape[-1]), int(k),
         _ptr(block_table, torch.int32, "block_table"), _ptr(resident, torch.int32, "resident"),
-        _ptr(stamp, torch.int32, "stamp"), int(resident.shape[-1]), int(slot_stride), int(cap),
-        int(step), _ptr(plan_idx, torch.int64, "plan_idx"), _ptr(plan_slots, torch.int32, "plan_slots"),
-        _ptr(n_admitted, torch.int32, "n_admitted"), _stream(stream)), "oasis_plan_delta")
+        _ptr(stamp, torch.int32, "stamp"), res_stride - int(n_local), res_stride, int(n_local),
+        int(slot_stride), int(cap), int(step), _ptr(plan_idx, torch.int64, "plan_idx"),
+        _ptr(plan_slots, torch.int32, "plan_slots"), _ptr(n_admitted, torch.int32, "n_admitted"),
+        _stream(stream)), "oasis_plan_delta")

@@ -18,7 +18,7 @@ struct PlanParams {
     long long *plan_idx;
     int32_t *plan_slots;
     int32_t *n_admitted;
-    int Hkv, max_blocks, sel_cols, k, n_res, slot_stride, cap, step, sort_len, bitmap_words;
+    int Hkv, max_blocks, sel_cols, k, n_res, res_stride, n_local, slot_stride, cap, step, sort_len, bitmap_words;
 };
 
 constexpr int kPlanThreads = 256;
@@ -39,8 +39,9 @@ plan_delta_kernel(const PlanParams p)
     const int row = blockIdx.x;
     const int b = row / p.Hkv, h = row % p.Hkv;
     const int32_t *pred = p.sel + (long long)row * p.sel_cols;
-    int32_t *res = p.resident + (long long)row * p.n_res;
-    int32_t *stp = p.stamp + (long long)row * p.n_res;
+    int32_t *res = p.resident + (long long)row * p.res_stride;
+    int32_t *stp = p.stamp + (long long)row * p.res_stride;
+    const int plan_cols = p.cap + p.n_local;
 
     for (int i = tid; i < 2 * p.bitmap_words; i += kPlanThreads) pred_bits[i] = 0;
     if (tid == 0) sh_n_target = 0;
@@ -127,8 +128,16 @@ plan_delta_kernel(const PlanParams p)
             idx = (long long)p.block_table[(long long)b * p.max_blocks + j] * p.Hkv + h;
             slot = row * p.slot_stride + c;
         }
-        p.plan_idx[(long long)row * p.cap + i] = idx;
-        p.plan_slots[(long long)row * p.cap + i] = slot;
+        p.plan_idx[(long long)row * plan_cols + i] = idx;
+        p.plan_slots[(long long)row * plan_cols + i] = slot;
+    }
+    // the always-kept local blocks (Sec. 4.3: selected blocks plus a local window)
+    for (int i = tid; i < p.n_local; i += kPlanThreads) {
+        const int j = pred[p.k + i];
+        res[p.n_res + i] = j;
+        p.plan_slots[(long long)row * plan_cols + p.cap + i] = row * p.slot_stride + p.n_res + i;
+        p.plan_idx[(long long)row * plan_cols + p.cap + i] =
+            (j < 0 || j >= p.max_blocks) ? -1ll : (long long)p.block_table[(long long)b * p.max_blocks + j] * p.Hkv + h;
     }
     if (tid == 0 && p.n_admitted) p.n_admitted[row] = n_pair;
 }
@@ -137,7 +146,8 @@ plan_delta_kernel(const PlanParams p)
 
 extern "C" int oasis_plan_delta(const oasis_dims_t *dims, const int32_t *sel, int32_t sel_cols, int32_t k,
                                 const int32_t *block_table, int32_t *resident, int32_t *stamp,
-                                int32_t n_res, int32_t slot_stride, int32_t cap, int32_t step,
+                                int32_t n_res, int32_t res_stride, int32_t n_local, int32_t slot_stride,
+                                int32_t cap, int32_t step,
                                 int64_t *plan_idx, int32_t *plan_slots, int32_t *n_admitted, void *stream)
 {
     using namespace oasis;
@@ -149,9 +159,14 @@ extern "C" int oasis_plan_delta(const oasis_dims_t *dims, const int32_t *sel, in
     if (n_res < 1 || n_res > OASIS_MAX_K)
         return fail(OASIS_ERR_INVALID_ARG, "oasis_plan_delta: n_res %d outside [1, %d]", n_res, OASIS_MAX_K);
     if (cap < 0 || cap > k) return fail(OASIS_ERR_INVALID_ARG, "oasis_plan_delta: cap %d outside [0, k]", cap);
-    if (cap > 0 && (!plan_idx || !plan_slots))
+    if (n_local < 0 || n_local > 2 || k + n_local > sel_cols)
+        return fail(OASIS_ERR_INVALID_ARG, "oasis_plan_delta: n_local %d (k %d, sel_cols %d)", n_local, k, sel_cols);
+    if (res_stride < n_res + n_local)
+        return fail(OASIS_ERR_INVALID_ARG, "oasis_plan_delta: res_stride %d < n_res + n_local = %d", res_stride, n_res + n_local);
+    if (cap + n_local > 0 && (!plan_idx || !plan_slots))
         return fail(OASIS_ERR_INVALID_ARG, "oasis_plan_delta: plan_idx / plan_slots are NULL");
-    if (slot_stride < n_res) return fail(OASIS_ERR_INVALID_ARG, "oasis_plan_delta: slot_stride %d < n_res %d", slot_stride, n_res);
+    if (slot_stride < n_res + n_local)
+        return fail(OASIS_ERR_INVALID_ARG, "oasis_plan_delta: slot_stride %d < n_res + n_local = %d", slot_stride, n_res + n_local);
     if ((long long)dims->batch * dims->n_kv_heads * slot_stride > 0x7fffffffLL)
         return fail(OASIS_ERR_UNSUPPORTED, "oasis_plan_delta: more than 2^31 slots");
     if (dims->max_blocks > (1 << 19))
@@ -162,7 +177,7 @@ extern "C" int oasis_plan_delta(const oasis_dims_t *dims, const int32_t *sel, in
     p.sel = sel; p.block_table = block_table; p.resident = resident; p.stamp = stamp;
     p.plan_idx = (long long *)plan_idx; p.plan_slots = plan_slots; p.n_admitted = n_admitted;
     p.Hkv = dims->n_kv_heads; p.max_blocks = dims->max_blocks; p.sel_cols = sel_cols; p.k = k;
-    p.n_res = n_res; p.slot_stride = slot_stride; p.cap = cap; p.step = step;
+    p.n_res = n_res; p.res_stride = res_stride; p.n_local = n_local; p.slot_stride = slot_stride; p.cap = cap; p.step = step;
     int sort_len = 2;
     while (sort_len < n_res) sort_len <<= 1;
     p.sort_len = sort_len;

@@ -74,3 +74,140 @@ class DecodeLayer:
                           self.sel if blk_tbl is None else blk_tbl, self.cols, seq_len, self.scale,
                           self.out, lse=self.lse, workspace=self.workspace, stream=stream)
         return self.out
+
+
+class DecodeEngine:
+    """Sequencing of one decode step across layers, after the paper's asynchronous prefetch
+    pipeline (Sec. 4.2.2): on the foreground stream each layer runs attention over the working
+    set that the previous step's prediction staged, then this step's prediction (summary
+    update for newly completed blocks, scoring with the draft queries, top-k); the transfer
+    of what was selected runs on a side stream and is awaited, per layer, only by the next
+    step's attention of that same layer.
+
+    mode "fetch_all": every selected block is gathered each step (k + 2 requests per row).
+    mode "delta": delta selection with capped eviction (Sec. 4.2.3) bounds the gather to
+    `cap` blocks per (request, KV head) per step plus the local blocks.
+    """
+
+    def __init__(self, batch, n_q_heads, n_kv_heads, max_blocks, k, n_q_tokens, n_layers,
+                 device="cuda", mode="fetch_all", cap=None):
+        assert mode in ("fetch_all", "delta")
+        self.mode, self.k, self.T, self.n_layers = mode, k, n_q_tokens, n_layers
+        self.device = torch.device(device)
+        self.layers = [DecodeLayer(batch, n_q_heads, n_kv_heads, max_blocks, k, n_q_tokens, device)
+                       for _ in range(n_layers)]
+        self.kv = [None] * n_layers
+        self.table = [None] * n_layers
+        self.main = torch.cuda.Stream(device=self.device)
+        self.side = torch.cuda.Stream(device=self.device)
+        self.sel_done = [torch.cuda.Event() for _ in range(n_layers)]
+        self.stage_done = [torch.cuda.Event() for _ in range(n_layers)]
+        self.launches = 0
+        self.cap = cap
+        if mode == "delta":
+            assert cap is not None and 0 <= cap <= k
+            dev, rows = self.device, (batch, n_kv_heads)
+            self.resident = [torch.full(rows + (k + 2,), -1, dtype=torch.int32, device=dev) for _ in range(n_layers)]
+            self.stamp = [torch.zeros(rows + (k + 2,), dtype=torch.int32, device=dev) for _ in range(n_layers)]
+            self.plan_idx = [torch.empty(rows + (cap + 2,), dtype=torch.int64, device=dev) for _ in range(n_layers)]
+            self.plan_slots = [torch.empty(rows + (cap + 2,), dtype=torch.int32, device=dev) for _ in range(n_layers)]
+        self._splits = oasis.attn_workspace_bytes(self.layers[0].dims, n_q_tokens, k + 2) > 0 if n_layers else False
+
+    def attach(self, layer, kv_src, block_table):
+        """kv_src: the layer's full-KV pool (pinned host memory, or device memory)."""
+        self.kv[layer], self.table[layer] = kv_src, block_table
+
+    def blk_tbl(self, layer):
+        return self.resident[layer] if self.mode == "delta" else self.layers[layer].sel
+
+    def _predict_and_transfer(self, l, q, first_block, n_new, max_new, n_full_next, seq_next, timers, plan=None):
+        L = self.layers[l]
+        ms = self.main
+        with torch.cuda.stream(ms):
+            L.build_summaries(self.kv[l], self.table[l], first_block, n_new, max_new)
+            t0 = self._tick(timers, "score")
+            L.score(q, n_full_next)
+            self._tock(timers, "score", t0)
+            t0 = self._tick(timers, "select")
+            L.select(n_full_next, seq_next, self.table[l])
+            self._tock(timers, "select", t0)
+            self.launches += 3
+            if self.mode == "delta":
+                plan_idx = self.plan_idx[l] if plan is None else plan[0]
+                plan_slots = self.plan_slots[l] if plan is None else plan[1]
+                oasis.plan_delta(L.dims, L.sel, self.k, self.table[l], self.resident[l], self.stamp[l],
+                                 L.cols, plan_idx.shape[-1] - 2, self._stamp_now, plan_idx, plan_slots, n_local=2)
+                self.launches += 1
+            self.sel_done[l].record(ms)
+        with torch.cuda.stream(self.side):
+            self.side.wait_event(self.sel_done[l])
+            t0 = self._tick(timers, "stage", self.side)
+            if self.mode == "delta":
+                oasis.stage_blocks(self.kv[l], plan_idx, plan_slots, plan_idx.numel(), L.pool)
+            else:
+                L.stage(self.kv[l])
+            self._tock(timers, "stage", t0, self.side)
+            self.launches += 1
+            self.stage_done[l].record(self.side)
+
+    @staticmethod
+    def _tick(timers, name, stream=None):
+        if timers is None or name not in timers:
+            return None
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record(stream if stream is not None else torch.cuda.current_stream())
+        return ev
+
+    @staticmethod
+    def _tock(timers, name, start, stream=None):
+        if start is None:
+            return
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record(stream if stream is not None else torch.cuda.current_stream())
+        timers[name].append((start, ev))
+
+    def prime(self, q_list, n_full_next, seq_next, step_stamp=0):
+        """Before the first step: build every summary and run one prediction + transfer per
+        layer, as the step before the first one would have done."""
+        self._stamp_now = step_stamp
+        B = self.layers[0].B
+        zeros = torch.zeros(B, dtype=torch.int32, device=self.device)
+        plan = None
+        if self.mode == "delta":        # the initial working set is admitted whole (cap = k)
+            rows = (B, self.layers[0].Hkv, self.k + 2)
+            plan = (torch.empty(rows, dtype=torch.int64, device=self.device),
+                    torch.empty(rows, dtype=torch.int32, device=self.device))
+        for l in range(self.n_layers):
+            self._predict_and_transfer(l, q_list[l], zeros, n_full_next, self.layers[l].mb, n_full_next, seq_next,
+                                       None, plan)
+            if plan is not None:
+                self.side.synchronize()  # the shared priming plan is reused by the next layer
+        self.main.synchronize()
+        self.side.synchronize()
+
+    def step(self, q_list, seq_len, first_block, n_new, n_full_next, seq_next, step_stamp=0,
+             timers=None, q_host=None, out_host=None):
+        """One decode step over all layers.  seq_len: history tokens of this step; the
+        prediction works on the next step's view (n_full_next, seq_next).  With q_host /
+        out_host (pinned tensors per layer) the step's queries are copied in and its outputs
+        copied out inside the step (end-to-end mode)."""
+        self._stamp_now = step_stamp
+        ms = self.main
+        for l in range(self.n_layers):
+            L = self.layers[l]
+            with torch.cuda.stream(ms):
+                if q_host is not None:
+                    q_list[l].copy_(q_host[l], non_blocking=True)
+                ms.wait_event(self.stage_done[l])
+                t0 = self._tick(timers, "attn")
+                L.attend(q_list[l], seq_len, blk_tbl=self.blk_tbl(l))
+                self._tock(timers, "attn", t0)
+                self.launches += 2 if self._splits else 1
+                if out_host is not None:
+                    out_host[l].copy_(L.out, non_blocking=True)
+            self._predict_and_transfer(l, q_list[l], first_block, n_new, 1, n_full_next, seq_next, timers)
+
+    def join(self):
+        """Makes the foreground stream wait for every transfer in flight."""
+        for l in range(self.n_layers):
+            self.main.wait_event(self.stage_done[l])

@@ -94,8 +94,10 @@ def test_argument_validation_of_each_call(L):
     assert lib.oasis_sparse_attn(d, one, 5, one, one, one, 130, one, 1.0, one, null, null, 0, null) == 4
     assert "workspace" in L.last_error()
     assert lib.oasis_sparse_attn(d, one, 5, one, one, one, 130, one, 1.0, one, null, one, need - 1, null) == 4
-    assert lib.oasis_plan_delta(d, one, 130, 128, one, one, one, 130, 130, 200, 1, one, one, null, null) == 1
-    assert lib.oasis_plan_delta(d, one, 130, 128, one, one, one, 130, 100, 6, 1, one, one, null, null) == 1
+    assert lib.oasis_plan_delta(d, one, 130, 128, one, one, one, 128, 130, 2, 130, 200, 1, one, one, null, null) == 1
+    assert lib.oasis_plan_delta(d, one, 130, 128, one, one, one, 128, 130, 2, 100, 6, 1, one, one, null, null) == 1
+    assert lib.oasis_plan_delta(d, one, 130, 128, one, one, one, 128, 129, 2, 130, 6, 1, one, one, null, null) == 1
+    assert lib.oasis_plan_delta(d, one, 129, 128, one, one, one, 128, 130, 2, 130, 6, 1, one, one, null, null) == 1
     empty = L.Dims(0, 32, 8, 64).c()
     assert lib.oasis_score_blocks(ctypes.byref(empty), one, dense, 4, one, one, 0, one, null) == 0
 

@@ -1,0 +1,97 @@
+"""GPU parity of the multi-layer decode engine (the launch sequence bench.py times): at every
+step each layer's attention must equal the oracle's attention over the working set that the
+previous step's lookahead prediction selected, in fetch-all and in capped-delta mode."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_08097_b200 import synth
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+SCALE = np.float32(1.0 / math.sqrt(128.0))
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2608_08097_b200 import build
+    build.build()
+    from paper_2608_08097_b200 import binding, pipeline
+    binding.lib()
+    return binding, pipeline
+
+
+def oracle_prediction(oracle, lay, summ_cache, q_step, n_full, seq):
+    """Selection made from the draft queries of step q_step for a step whose view is (n_full, seq)."""
+    cfg = lay.cfg
+    kv = pu.np_u16(lay.host_kv)
+    table = lay.block_table.numpy()
+    summ = oracle.build_summaries(kv, table, np.zeros(cfg.batch, np.int32), n_full)
+    q = pu.np_u16(lay.q_steps[q_step])
+    s32, s64 = oracle.score_blocks(q[:, 1:], summ, n_full)
+    sel, idx, slots = oracle.select_topk(s32, n_full, seq, cfg.n_q_tokens, cfg.k_blocks, table)
+    return sel, idx, slots, s64
+
+
+@pytest.mark.parametrize("mode,cap", [("fetch_all", None), ("delta", 3), ("delta", 16)])
+def test_engine_steps_match_oracle(oracle, gpu, mode, cap):
+    binding, pipeline = gpu
+    dev = torch.device("cuda")
+    n_layers, S = 3, 19
+    cfg = synth.scaled(synth.C2, batch=2, context=1536, k_blocks=16, layers=n_layers, steps=S)
+    k, B, Hkv = cfg.k_blocks, cfg.batch, cfg.n_kv_heads
+    lays = [synth.make_layer(cfg, seed=31, layer=l) for l in range(n_layers)]
+    eng = pipeline.DecodeEngine(B, cfg.n_q_heads, Hkv, cfg.max_blocks, k, cfg.n_q_tokens, n_layers, dev,
+                                mode=mode, cap=cap)
+    kvs = [lay.host_kv.pin_memory() for lay in lays]
+    for l, lay in enumerate(lays):
+        eng.attach(l, kvs[l], lay.block_table.to(dev))
+    seq = lays[0].seq_len_steps                                   # [S][B]
+    q_dev = [lay.q_steps.to(dev) for lay in lays]
+    to_dev = lambda t: t.to(torch.int32).contiguous().to(dev)
+    eng.prime([q_dev[l][0] for l in range(n_layers)], to_dev(seq[0] // 16), to_dev(seq[0]))
+
+    # oracle-side state
+    pools = [np.zeros((B * Hkv * (k + 2), 2, 16, 128), np.uint16) for _ in range(n_layers)]
+    slot_tbl = np.arange(B * Hkv * (k + 2), dtype=np.int32).reshape(B, Hkv, k + 2)
+    res = [np.full((B, Hkv, k + 2), -1, np.int32) for _ in range(n_layers)]
+    stp = [np.zeros((B, Hkv, k + 2), np.int32) for _ in range(n_layers)]
+    blk = [None] * n_layers
+
+    def oracle_transfer(l, sel, idx, slots, cap_now, stamp):
+        kv = pu.np_u16(lays[l].host_kv).reshape(-1, 2, 16, 128)
+        if mode == "delta":
+            pidx, pslots, _ = oracle.plan_delta(sel, lays[l].block_table.numpy(), res[l], stp[l], k, cap_now, stamp,
+                                                k + 2, n_local=2)
+            oracle.stage_blocks(kv, pidx, pslots, pools[l])
+            blk[l] = res[l].copy()
+        else:
+            oracle.stage_blocks(kv, idx, slots, pools[l])
+            blk[l] = sel.copy()
+
+    for l in range(n_layers):
+        sel, idx, slots, _ = oracle_prediction(oracle, lays[l], None, 0, (seq[0] // 16).numpy(), seq[0].numpy())
+        oracle_transfer(l, sel, idx, slots, k, 0)
+
+    for s in range(S):
+        eng.step([q_dev[l][s] for l in range(n_layers)], to_dev(seq[s]), to_dev(seq[s] // 16),
+                 to_dev((seq[s] + 1) // 16 - seq[s] // 16), to_dev((seq[s] + 1) // 16), to_dev(seq[s] + 1),
+                 step_stamp=s + 1)
+        eng.join()
+        torch.cuda.synchronize()
+        for l in range(n_layers):
+            # attention of this step ran over the working set predicted one step earlier
+            ref = oracle.sparse_attn(pu.np_u16(lays[l].q_steps[s]), pools[l], slot_tbl, blk[l], seq[s].numpy(), SCALE, Hkv)
+            pu.assert_attn_close(pu.bf16_to_f32_np(eng.layers[l].out), ref["out32"])
+            # this step's prediction and transfer, for the next step
+            sel, idx, slots, s64 = oracle_prediction(oracle, lays[l], None, s, ((seq[s] + 1) // 16).numpy(),
+                                                     (seq[s] + 1).numpy())
+            gsel = eng.layers[l].sel.cpu().numpy()
+            assert pu.assert_sel_parity(gsel, sel, s64, k) == 0, "near-tie in a test that expects none"
+            oracle_transfer(l, sel, idx, slots, cap if cap is not None else k, s + 1)
+            assert np.array_equal(eng.blk_tbl(l).cpu().numpy(), blk[l])
+            assert np.array_equal(pu.np_u16(eng.layers[l].pool), pools[l])

@@ -334,24 +334,26 @@ def test_plan_delta_matches_oracle_over_steps(oracle, gpu, cap_ratio):
     kv_np = pu.np_u16(lay.host_kv).reshape(-1, 2, 16, 128)
     table = lay.block_table.to(dev)
     B, Hkv = cfg.batch, cfg.n_kv_heads
-    resident = torch.full((B, Hkv, k), -1, dtype=torch.int32, device=dev)
-    stamp = torch.zeros((B, Hkv, k), dtype=torch.int32, device=dev)
-    plan_idx = torch.empty((B, Hkv, cap), dtype=torch.int64, device=dev)
-    plan_slots = torch.empty((B, Hkv, cap), dtype=torch.int32, device=dev)
+    resident = torch.full((B, Hkv, k + 2), -1, dtype=torch.int32, device=dev)
+    stamp = torch.zeros((B, Hkv, k + 2), dtype=torch.int32, device=dev)
+    plan_idx = torch.empty((B, Hkv, cap + 2), dtype=torch.int64, device=dev)
+    plan_slots = torch.empty((B, Hkv, cap + 2), dtype=torch.int32, device=dev)
     n_adm = torch.empty((B, Hkv), dtype=torch.int32, device=dev)
-    res_ref = np.full((B, Hkv, k), -1, np.int32)
-    stamp_ref = np.zeros((B, Hkv, k), np.int32)
+    res_ref = np.full((B, Hkv, k + 2), -1, np.int32)
+    stamp_ref = np.zeros((B, Hkv, k + 2), np.int32)
     zeros = torch.zeros(B, dtype=torch.int32, device=dev)
     L.build_summaries(kv, table, zeros, lay.n_full_steps[-1].to(dev), cfg.max_blocks)
     for s in range(cfg.steps):
         n_full = lay.n_full_steps[s].to(dev)
         L.score(lay.q_steps[s].to(dev), n_full)
         L.select(n_full, lay.seq_len_steps[s].to(dev), table)
-        binding.plan_delta(L.dims, L.sel, k, table, resident, stamp, L.cols, cap, s + 1, plan_idx, plan_slots, n_adm)
+        binding.plan_delta(L.dims, L.sel, k, table, resident, stamp, L.cols, cap, s + 1, plan_idx, plan_slots, n_adm,
+                           n_local=2)
         binding.stage_blocks(kv, plan_idx, plan_slots, plan_idx.numel(), L.pool)
         torch.cuda.synchronize()
         sel_np = L.sel.cpu().numpy()
-        ridx, rslots, radm = oracle.plan_delta(sel_np, lay.block_table.numpy(), res_ref, stamp_ref, k, cap, s + 1, L.cols)
+        ridx, rslots, radm = oracle.plan_delta(sel_np, lay.block_table.numpy(), res_ref, stamp_ref, k, cap, s + 1, L.cols,
+                                               n_local=2)
         assert np.array_equal(resident.cpu().numpy(), res_ref)
         assert np.array_equal(stamp.cpu().numpy(), stamp_ref)
         assert np.array_equal(n_adm.cpu().numpy(), radm)
@@ -363,7 +365,7 @@ def test_plan_delta_matches_oracle_over_steps(oracle, gpu, cap_ratio):
         pool_np = pu.np_u16(L.pool)
         for b in range(B):
             for h in range(Hkv):
-                for c in range(0, k, 5):
+                for c in list(range(0, k, 5)) + [k, k + 1]:
                     j = res_ref[b, h, c]
                     if j >= 0:
                         src = int(lay.block_table[b, j]) * Hkv + h

@@ -518,6 +518,19 @@ def test_plan_delta_hand_worked_example(oracle):
     assert n.reshape(-1).tolist() == [2] and idx.reshape(-1).tolist() == [1020, 1021, -1, -1]
 
 
+def test_plan_delta_local_window(oracle):
+    # two local columns after three managed ones: the ids in sel[k..k+2) are mirrored and always requested
+    pred = np.array([[[7, 8, 9, 40, -1]]], np.int32)                      # k = 3, locals 40 and none
+    res = np.array([[[7, 5, 6, 99, 99]]], np.int32)
+    stp = np.array([[[4, 1, 2, 77, 78]]], np.int32)
+    table = (np.arange(100, dtype=np.int32) + 1000).reshape(1, 100)
+    idx, slots, n = oracle.plan_delta(pred, table, res, stp, 3, 1, 9, slot_stride=8, n_local=2)
+    assert res.reshape(-1).tolist() == [7, 8, 6, 40, -1]                   # 8 replaces the oldest (block 5)
+    assert stp.reshape(-1).tolist() == [9, 9, 2, 77, 78]                   # local stamps untouched
+    assert idx.reshape(-1).tolist() == [1008, 1040, -1] and slots.reshape(-1).tolist()[:2] == [1, 3]
+    assert slots.reshape(-1).tolist()[2] == 4 and n.reshape(-1).tolist() == [1]
+
+
 def test_plan_delta_invariants(oracle):
     rng = np.random.default_rng(26)
     Hkv, k, n_res, nblk = 3, 12, 12, 60
