@@ -19,9 +19,7 @@ import argparse
 import json
 import math
 import os
-import subprocess
 import sys
-import tempfile
 import threading
 import time
 
@@ -40,7 +38,7 @@ UNIT = "tokens/s/layer"
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--steps", type=int, default=48)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=None, help="override the number of layers (debugging)")
@@ -77,50 +75,49 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while a region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    """Samples the SM clock and the clock-event (throttle) reasons through NVML, read-only,
+    every few milliseconds from a thread while a timed region runs."""
+    REASONS = (("hw_slowdown", 0x8), ("hw_thermal_slowdown", 0x40), ("sw_thermal_slowdown", 0x20),
+               ("sw_power_cap", 0x4))
 
     def __init__(self, index):
-        self.index, self.proc, self.path = index, None, None
+        self.index, self.thread, self.stop_flag = index, None, threading.Event()
+        self.clocks, self.reason_bits, self.max_mhz = [], 0, None
+
+    def _run(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            idx = self.index
+            if visible:
+                try:
+                    idx = int(visible.split(",")[self.index])
+                except ValueError:
+                    pass
+            h = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM)
+            while not self.stop_flag.is_set():
+                self.clocks.append(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM))
+                self.reason_bits |= int(pynvml.nvmlDeviceGetCurrentClocksEventReasons(h))
+                time.sleep(0.004)
+        except Exception:          # NVML missing or refused: report no samples
+            pass
 
     def start(self):
-        fd, self.path = tempfile.mkstemp(suffix=".csv")
-        os.close(fd)
-        try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
-        except OSError:
-            self.proc = None
+        self.thread = threading.Thread(target=self._run, daemon=True)
+        self.thread.start()
+        time.sleep(0.02)
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.proc is None:
-            return out
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-        rows = []
-        with open(self.path) as f:
-            for line in f:
-                parts = [p.strip() for p in line.split(",")]
-                if len(parts) >= 7:
-                    try:
-                        rows.append((float(parts[0]), float(parts[1]), parts[3:7]))
-                    except ValueError:
-                        pass
-        os.unlink(self.path)
-        if rows:
-            clocks = sorted(r[0] for r in rows)
-            out["sm_mhz"] = clocks[len(clocks) // 2]
-            out["sm_max_mhz"] = rows[0][1]
-            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-            out["reasons"] = [n for i, n in enumerate(names) if any(r[2][i].lower().startswith("active") for r in rows)]
-            out["samples"] = len(rows)
+        self.stop_flag.set()
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        out = {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": len(self.clocks)}
+        if self.clocks:
+            c = sorted(self.clocks)
+            out["sm_mhz"] = c[len(c) // 2]
+            out["reasons"] = [n for n, bit in self.REASONS if self.reason_bits & bit]
         return out
 
 
@@ -423,7 +420,8 @@ def run_ours(args):
                              % (cfg.layers, (score_bytes + attn_bytes) / 1e6),
                        "gather": "fetch-all from an HBM mirror of the full KV (value); pinned host (e2e)"},
             "gpu_launches": launches,
-            "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"]},
+            "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
+                       "samples": clocks["samples"]},
             "roofline": {"bound": "hbm", "kernel": dominant, "achieved": d.get("GBps"), "peak": hbm_peak,
                          "unit": "GB/s", "frac": d.get("frac_of_measured"), "traffic": None,
                          "peak_kind": peak_kind + " (STREAM-style copy)"},

@@ -1,0 +1,46 @@
+"""Multi-rank plumbing of bench.py on CPU: two gloo ranks, barrier + max-over-ranks timing,
+whole-job aggregation; and the reference arm under torchrun (rank 0 alone prints)."""
+import json
+import os
+import socket
+import subprocess
+import sys
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def torchrun(script_args, nproc=2, timeout=600):
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(nproc),
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port())] + script_args
+    env = dict(os.environ, CUDA_VISIBLE_DEVICES="", OMP_NUM_THREADS="1")
+    return subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=timeout)
+
+
+def json_lines(text):
+    return [json.loads(l) for l in text.splitlines() if l.startswith("{")]
+
+
+def test_two_rank_timing_is_max_over_ranks_and_value_is_whole_job():
+    r = torchrun([os.path.join("tests", "dist_worker.py"), "--gpus", "2", "--steps", "4"])
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = json_lines(r.stdout)
+    assert len(lines) == 1                                  # rank 0 alone prints
+    out = lines[0]
+    assert out["world"] == 2 and out["ms"] == 15.0          # slowest rank
+    assert abs(out["value"] - 16 * 2 / (15e-3 / 32)) < 1e-6  # both replicas' tokens over that time
+
+
+def test_reference_arm_under_torchrun_prints_once():
+    r = torchrun(["bench.py", "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "1",
+                  "--context", "4096"])
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = json_lines(r.stdout)
+    assert len(lines) == 1 and lines[0]["impl"] == "reference"
+    assert lines[0]["cpu_baseline"]["kind"] == "oracle" and lines[0]["e2e"]["h2d_bytes_per_step"] == 0
+    assert lines[0]["value"] > 0
