@@ -153,6 +153,33 @@ size_t oasis_attn_workspace_bytes(const oasis_dims_t *dims, int32_t n_q_tokens,
                                   int32_t n_cols);
 
 /*
+ * Sparse attention with built-in scratch memory.  (This entry point has no counterpart in the
+ * paper: it is a packaging variant of step 4.)
+ * Same computation, arguments and results as oasis_sparse_attn, but the caller passes no
+ * workspace: the split-KV partials go to a fixed array of oasis_static_scratch_bytes() bytes
+ * (4 MiB) that is part of the library image, so every GPU that loads the library holds that
+ * much memory until the process exits.  It is meant for callers that cannot provide scratch
+ * memory themselves -- an engine that gave all free device memory to its KV-cache pool at
+ * start-up, or a decode loop that must not call cudaMalloc (it can fail at that point and it
+ * synchronises the device).  The call allocates and frees nothing.
+ *   - Shapes whose partials need more than the array holds are rejected with
+ *     OASIS_ERR_WORKSPACE (the message states both sizes); use oasis_sparse_attn for those.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call before any stream capture begins.
+ *   - All calls share the one array.  It keeps whatever the previous call left in it, which is
+ *     harmless (every partial is written before it is read), but two calls whose kernels
+ *     overlap on the GPU (different streams) race on it: serialise them.
+ */
+int oasis_sparse_attn_static_scratch(const oasis_dims_t *dims, const void *q, int32_t n_q_tokens,
+                                     const void *hbm_pool, const int32_t *slot_tbl,
+                                     const int32_t *blk_tbl, int32_t n_cols,
+                                     const int32_t *seq_len, float scale, void *out, float *lse,
+                                     void *stream);
+
+/* Size in bytes of the built-in scratch array used by oasis_sparse_attn_static_scratch. */
+size_t oasis_static_scratch_bytes(void);
+
+/*
  * KV selection stage -- delta selection with capped eviction (Sec. 4.2.3; the cap is a
  * fraction of K, Sec. 5.5.1: cap = floor(ratio * K)).  Each (b, h) row owns n_res resident
  * columns: resident[b][h][c] is the logical block held in column c (-1 = empty) and

@@ -19,7 +19,8 @@ REDUCE_MAX, REDUCE_SUM = 0, 1
 ENTRY_BYTES = 8192
 SYMBOLS = ("oasis_build_summaries", "oasis_score_blocks", "oasis_select_topk",
            "oasis_stage_blocks", "oasis_sparse_attn", "oasis_attn_workspace_bytes",
-           "oasis_plan_delta", "oasis_last_error", "oasis_version")
+           "oasis_plan_delta", "oasis_last_error", "oasis_version",
+           "oasis_sparse_attn_static_scratch", "oasis_static_scratch_bytes")
 
 
 class OasisError(RuntimeError):
@@ -64,6 +65,10 @@ def lib():
         L.oasis_select_topk.argtypes = [dp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]
         L.oasis_stage_blocks.argtypes = [vp, vp, vp, i32, vp, vp]
         L.oasis_sparse_attn.argtypes = [dp, vp, i32, vp, vp, vp, i32, vp, f32, vp, vp, vp, sz, vp]
+        L.oasis_sparse_attn_static_scratch.argtypes = [dp, vp, i32, vp, vp, vp, i32, vp, f32, vp, vp, vp]
+        L.oasis_sparse_attn_static_scratch.restype = ctypes.c_int
+        L.oasis_static_scratch_bytes.argtypes = []
+        L.oasis_static_scratch_bytes.restype = sz
         L.oasis_attn_workspace_bytes.argtypes = [dp, i32, i32]
         L.oasis_attn_workspace_bytes.restype = sz
         L.oasis_plan_delta.argtypes = [dp, vp, i32, i32, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
@@ -161,6 +166,24 @@ def sparse_attn(dims, q, n_q_tokens, hbm_pool, slot_tbl, blk_tbl, n_cols, seq_le
         _ptr(blk_tbl, torch.int32, "blk_tbl"), int(n_cols), _ptr(seq_len, torch.int32, "seq_len"),
         float(scale), _ptr(out, torch.bfloat16, "out"), _ptr(lse, torch.float32, "lse"),
         _ptr(workspace, None, "workspace"), ws_bytes, _stream(stream)), "oasis_sparse_attn")
+
+
+def static_scratch_bytes() -> int:
+    return int(lib().oasis_static_scratch_bytes())
+
+
+def sparse_attn_static_scratch(dims, q, n_q_tokens, hbm_pool, slot_tbl, blk_tbl, n_cols, seq_len, scale,
+                               out, lse=None, stream=None):
+    """oasis_sparse_attn for callers that cannot hand over scratch memory (no free device memory
+    left to allocate from, or no cudaMalloc allowed in the decode loop): the partial results go
+    to a 4 MiB array built into the library.  Calls sharing a GPU must not overlap."""
+    d = dims.c()
+    _check(lib().oasis_sparse_attn_static_scratch(
+        ctypes.byref(d), _ptr(q, torch.bfloat16, "q"), int(n_q_tokens),
+        _ptr(hbm_pool, torch.bfloat16, "hbm_pool"), _ptr(slot_tbl, torch.int32, "slot_tbl"),
+        _ptr(blk_tbl, torch.int32, "blk_tbl"), int(n_cols), _ptr(seq_len, torch.int32, "seq_len"),
+        float(scale), _ptr(out, torch.bfloat16, "out"), _ptr(lse, torch.float32, "lse"),
+        _stream(stream)), "oasis_sparse_attn_static_scratch")
 
 
 def plan_delta(dims, sel, k, block_table, resident, stamp, slot_stride, cap, step, plan_idx,

@@ -455,3 +455,113 @@ extern "C" int oasis_sparse_attn(const oasis_dims_t *dims, const void *q, int32_
     }
     return OASIS_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Sparse attention with built-in scratch memory.
+//
+// oasis_sparse_attn needs a caller-supplied workspace whenever it splits the column list.  Some
+// callers have no way to supply one: an inference engine that hands every free byte of the
+// device to its KV-cache pool at start-up has nothing left to carve scratch from later, and a
+// decode loop cannot afford cudaMalloc, which may fail at that point and synchronises the device
+// when it succeeds.  For them the split-KV partials live in the fixed array below, which is part
+// of the library image: every GPU that loads the library holds these bytes until the process
+// exits.
+//
+// In host code `g_attn_scratch` is only a stand-in for the device array -- its host address is
+// not a device address -- so the device address is looked up once per device with
+// cudaGetSymbolAddress (with that device current) and that pointer is what the kernels get.
+#include <mutex>
+
+namespace oasis {
+
+constexpr size_t kStaticScratchBytes = 4u << 20;      // 4 MiB
+constexpr int kMaxDevices = 64;
+
+static __device__ __align__(256) unsigned char g_attn_scratch[kStaticScratchBytes];
+
+static std::mutex g_scratch_mutex;
+static void *g_scratch_ptr[kMaxDevices] = {};          // device address of g_attn_scratch, per device
+
+// Device address of the scratch array on the current device; looked up on first use.
+static int static_scratch(void **out)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "oasis_sparse_attn_static_scratch: cudaGetDevice: %s", cudaGetErrorString(e));
+    if (dev < 0 || dev >= kMaxDevices)
+        return fail(OASIS_ERR_UNSUPPORTED, "oasis_sparse_attn_static_scratch: device ordinal %d >= %d", dev, kMaxDevices);
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_ptr[dev]) {
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_attn_scratch);
+        if (e != cudaSuccess || !p) {
+            cudaGetLastError();
+            return fail(OASIS_ERR_CUDA, "oasis_sparse_attn_static_scratch: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+        }
+        g_scratch_ptr[dev] = p;
+    }
+    *out = g_scratch_ptr[dev];
+    return OASIS_OK;
+}
+
+}  // namespace oasis
+
+extern "C" size_t oasis_static_scratch_bytes(void) { return oasis::kStaticScratchBytes; }
+
+extern "C" int oasis_sparse_attn_static_scratch(const oasis_dims_t *dims, const void *q, int32_t n_q_tokens,
+                                                const void *hbm_pool, const int32_t *slot_tbl,
+                                                const int32_t *blk_tbl, int32_t n_cols, const int32_t *seq_len,
+                                                float scale, void *out, float *lse, void *stream)
+{
+    using namespace oasis;
+    if (int rc = check_dims(dims)) return rc;
+    if (!q || !hbm_pool || !slot_tbl || !blk_tbl || !seq_len || !out)
+        return fail(OASIS_ERR_INVALID_ARG, "oasis_sparse_attn_static_scratch: NULL pointer argument");
+    if (!aligned16(q) || !aligned16(hbm_pool) || !aligned16(out))
+        return fail(OASIS_ERR_INVALID_ARG, "oasis_sparse_attn_static_scratch: q, hbm_pool and out must be 16-byte aligned");
+    if (n_q_tokens < 1 || n_cols < 1)
+        return fail(OASIS_ERR_INVALID_ARG, "oasis_sparse_attn_static_scratch: n_q_tokens %d, n_cols %d", n_q_tokens, n_cols);
+    const int G = dims->n_q_heads / dims->n_kv_heads;
+    if (n_q_tokens * G > 128)
+        return fail(OASIS_ERR_UNSUPPORTED, "oasis_sparse_attn_static_scratch: n_q_tokens * group = %d rows > 128", n_q_tokens * G);
+    if (dims->batch == 0) return OASIS_OK;
+    const AttnPlan pl = attn_plan(dims, n_q_tokens, n_cols);
+    if (pl.workspace > kStaticScratchBytes)
+        return fail(OASIS_ERR_WORKSPACE,
+                    "oasis_sparse_attn_static_scratch: these shapes need %zu bytes of scratch, the built-in array holds %zu; "
+                    "use oasis_sparse_attn with a caller-owned workspace",
+                    pl.workspace, kStaticScratchBytes);
+    if (pl.items > 0x7fffffffLL) return fail(OASIS_ERR_UNSUPPORTED, "oasis_sparse_attn_static_scratch: grid too large");
+    void *scratch = nullptr;
+    if (int rc = static_scratch(&scratch)) return rc;
+
+    AttnParams p;
+    p.q = (const uint8_t *)q; p.pool = (const uint8_t *)hbm_pool;
+    p.slot_tbl = slot_tbl; p.blk_tbl = blk_tbl; p.seq_len = seq_len;
+    p.out = (uint8_t *)out; p.lse = lse;
+    p.part_o = (float *)scratch;
+    p.part_lse = p.part_o + (size_t)pl.items * pl.rows_per_group * kHeadDim;
+    p.scale_log2 = scale * kLog2e;
+    p.T = n_q_tokens; p.Hq = dims->n_q_heads; p.Hkv = dims->n_kv_heads; p.G = G;
+    p.n_cols = n_cols; p.R = n_q_tokens * G;
+    p.n_splits = pl.n_splits; p.cols_per_split = pl.cols_per_split;
+    p.n_groups = pl.n_groups; p.rows_per_group = pl.rows_per_group;
+
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t smem = (size_t)pl.n_mt * 16 * kRowBytes + (size_t)kAttnWarps * kAttnStages * kEntryBytes;
+    cudaError_t e;
+    if (pl.n_mt == 1) {
+        e = cudaFuncSetAttribute(sparse_attn_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) sparse_attn_kernel<1><<<(unsigned)pl.items, kAttnWarps * 32, smem, st>>>(p);
+    } else {
+        e = cudaFuncSetAttribute(sparse_attn_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) sparse_attn_kernel<2><<<(unsigned)pl.items, kAttnWarps * 32, smem, st>>>(p);
+    }
+    if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "oasis_sparse_attn_static_scratch: %s", cudaGetErrorString(e));
+    if (int rc = check_launch("oasis_sparse_attn_static_scratch")) return rc;
+    if (pl.n_splits > 1) {
+        attn_combine_kernel<<<(unsigned)((long long)dims->batch * dims->n_kv_heads * p.R), 128, 0, st>>>(p);
+        return check_launch("oasis_sparse_attn_static_scratch (combine)");
+    }
+    return OASIS_OK;
+}
