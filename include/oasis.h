@@ -211,6 +211,15 @@ int oasis_plan_delta(const oasis_dims_t *dims, const int32_t *sel, int32_t sel_c
                      int32_t cap, int32_t step, int64_t *plan_idx, int32_t *plan_slots,
                      int32_t *n_admitted, void *stream);
 
+/*
+ * Registers a device word (int32, zero-initialised by the caller, or NULL to unregister) in
+ * which kernels record a non-zero code if one of their internal waits (on a shared-memory
+ * barrier of an asynchronous copy or tensor-core operation) runs out of its iteration bound.
+ * Such a kernel stops working and returns; its outputs are then undefined.  The word is
+ * process-wide and is only ever written with a compare-and-swap from zero.
+ */
+int oasis_set_error_word(int32_t *device_word);
+
 /* Description of the calling thread's most recent error ("" if none). Static storage. */
 const char *oasis_last_error(void);
 

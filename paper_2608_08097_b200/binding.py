@@ -20,7 +20,7 @@ ENTRY_BYTES = 8192
 SYMBOLS = ("oasis_build_summaries", "oasis_score_blocks", "oasis_select_topk",
            "oasis_stage_blocks", "oasis_sparse_attn", "oasis_attn_workspace_bytes",
            "oasis_plan_delta", "oasis_last_error", "oasis_version",
-           "oasis_sparse_attn_static_scratch", "oasis_static_scratch_bytes")
+           "oasis_sparse_attn_static_scratch", "oasis_static_scratch_bytes", "oasis_set_error_word")
 
 
 class OasisError(RuntimeError):
@@ -75,10 +75,19 @@ def lib():
         for name in ("oasis_build_summaries", "oasis_score_blocks", "oasis_select_topk",
                      "oasis_stage_blocks", "oasis_sparse_attn", "oasis_plan_delta"):
             getattr(L, name).restype = ctypes.c_int
+        L.oasis_set_error_word.argtypes = [vp]
+        L.oasis_set_error_word.restype = ctypes.c_int
         L.oasis_last_error.restype = ctypes.c_char_p
         L.oasis_version.restype = ctypes.c_char_p
         _lib = L
     return _lib
+
+
+def set_error_word(word):
+    """Registers an int32 device tensor (one element, zero) that kernels flag on an internal
+    wait time-out; None unregisters."""
+    _check(lib().oasis_set_error_word(None if word is None else ctypes.c_void_p(word.data_ptr())),
+           "oasis_set_error_word")
 
 
 def last_error() -> str:

@@ -62,7 +62,16 @@ int sm_count()
     return cached;
 }
 
+static int32_t *g_error_word = nullptr;
+int32_t *error_word() { return g_error_word; }
+
 }  // namespace oasis
+
+extern "C" int oasis_set_error_word(int32_t *device_word)
+{
+    oasis::g_error_word = device_word;
+    return OASIS_OK;
+}
 
 extern "C" const char *oasis_last_error(void) { return oasis::g_last_error; }
 extern "C" const char *oasis_version(void) { return "0.1"; }

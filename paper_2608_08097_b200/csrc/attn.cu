@@ -5,14 +5,16 @@
 // are packed into the M dimension of the tensor-core tiles, so each K/V block is read from
 // HBM once per item however many rows use it.
 //
-// A CTA has four warps.  Warp w owns the columns c0 + w, c0 + w + 4, ... of its item: it
-// fetches each 8 KiB entry with sixteen 16-byte cp.async per lane into a private 3-deep
-// shared-memory ring (XOR-swizzled 16-byte chunks, so ldmatrix is conflict-free), computes
-// S = Q K^T for the 16 keys with mma.sync.m16n8k16 (bf16 in, fp32 out), applies the causal
-// limit of local blocks, updates a running max / sum in fp32 (online softmax, quad shuffles
-// for the row reductions), rounds P to bf16 and accumulates O += P V on the tensor cores.
-// The ring is warp-private, so the main loop has no CTA-wide barrier.  At the end the four
-// warps' (m, l, O) are merged through shared memory; if the column list was split, the
+// A CTA has four column slots; slot s owns the columns c0 + s, c0 + s + 4, ... of its item.
+// A slot is served by one warp per 16-row m-tile (one or two warps): together they fetch each
+// 8 KiB entry with 16-byte cp.async into the slot's private 3-deep shared-memory ring
+// (XOR-swizzled 16-byte chunks, so ldmatrix is conflict-free) and meet on the slot's named
+// barrier; each warp then computes S = Q K^T for its 16 rows x 16 keys with mma.sync.m16n8k16
+// (bf16 in, fp32 out), applies the causal limit (local blocks only), keeps a running max / sum
+// in fp32 (online softmax, quad shuffles; the running max is only raised when a row's new max
+// exceeds it by 2^8, so the accumulator is rarely rescaled), rounds P to bf16 and accumulates
+// O += P V on the tensor cores.  There is no CTA-wide barrier in the main loop.  At the end
+// the slots' (m, l, O) are merged through shared memory; if the column list was split, the
 // item's normalised partial output and its log-sum-exp go to the workspace and a second
 // small kernel merges the splits.
 // Algorithmic traffic: 8 KiB per (request, KV head, column) plus Q and O.
@@ -22,7 +24,7 @@
 
 namespace oasis {
 
-constexpr int kAttnWarps = 4;
+constexpr int kAttnSlots = 4;       // column slots per CTA (each served by one warp per m-tile)
 constexpr int kAttnStages = 3;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -47,17 +49,26 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk)   // byte offset ins
     return (uint32_t)(row * kRowBytes + ((chunk ^ (row & 7)) << 4));
 }
 
+__device__ __forceinline__ void slot_barrier(int id, int nthreads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
 template <int N_MT>
-__global__ void __launch_bounds__(kAttnWarps * 32, 2)
+__global__ void __launch_bounds__(kAttnSlots * N_MT * 32, 2)
 sparse_attn_kernel(const AttnParams p)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     constexpr int QROWS = N_MT * 16;
+    constexpr int SLOT_THREADS = N_MT * 32;
+    constexpr int NTHREADS = kAttnSlots * SLOT_THREADS;
     uint8_t *q_sm = smem;                                  // [QROWS][256 B], swizzled
-    uint8_t *kv_sm = smem + QROWS * kRowBytes;             // [warps][stages][8 KiB]
+    uint8_t *kv_sm = smem + QROWS * kRowBytes;             // [slots][stages][8 KiB]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t4 = lane & 3;
+    const int mt = warp % N_MT, slot = warp / N_MT;
+    const int slot_lane = mt * 32 + lane;                  // 0 .. SLOT_THREADS-1
 
     // item -> (bh, split, row group); groups of one (bh, split) are adjacent in the grid
     int item = blockIdx.x;
@@ -72,7 +83,7 @@ sparse_attn_kernel(const AttnParams p)
     const int L = p.seq_len[b];
 
     // ---- Q rows of this group -> shared memory (zero rows past nrows) -------------------------
-    for (int i = tid; i < QROWS * 16; i += blockDim.x) {
+    for (int i = tid; i < QROWS * 16; i += NTHREADS) {
         const int r = i >> 4, ch = i & 15;
         uint4 v = make_uint4(0, 0, 0, 0);
         if (r < nrows) {
@@ -84,71 +95,67 @@ sparse_attn_kernel(const AttnParams p)
     }
     __syncthreads();
 
-    // causal limit (last visible position) of the two rows this lane owns in every m-tile
-    int limit[N_MT][2];
+    // causal limit (last visible position) of the two rows this lane owns: rows g and g + 8 of m-tile mt
+    int limit[2];
 #pragma unroll
-    for (int mt = 0; mt < N_MT; ++mt) {
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            const int r = mt * 16 + g + 8 * e;
-            limit[mt][e] = (r < nrows) ? L + (row0 + r) / p.G : -1;
-        }
+    for (int e = 0; e < 2; ++e) {
+        const int r = mt * 16 + g + 8 * e;
+        limit[e] = (r < nrows) ? L + (row0 + r) / p.G : -1;
     }
 
-    float o[N_MT][16][4];
-    float m_run[N_MT][2], l_run[N_MT][2];
+    float o[16][4];
+    float m_run[2] = {-CUDART_INF_F, -CUDART_INF_F}, l_run[2] = {0.f, 0.f};
 #pragma unroll
-    for (int mt = 0; mt < N_MT; ++mt) {
-        m_run[mt][0] = m_run[mt][1] = -CUDART_INF_F;
-        l_run[mt][0] = l_run[mt][1] = 0.f;
+    for (int nt = 0; nt < 16; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+
+    // Q fragments of this warp's m-tile stay in registers when the CTA is small enough to afford them
+    constexpr bool kQInRegs = (N_MT == 1);
+    uint32_t qf[kQInRegs ? 8 : 1][4];
+    const int lm = lane >> 3, lr = lane & 7;               // ldmatrix: matrix index, row within it
+    const uint32_t q_u32 = smem_u32(q_sm);
+    if constexpr (kQInRegs) {
 #pragma unroll
-        for (int nt = 0; nt < 16; ++nt) o[mt][nt][0] = o[mt][nt][1] = o[mt][nt][2] = o[mt][nt][3] = 0.f;
+        for (int ks = 0; ks < 8; ++ks)
+            ldmatrix_x4(qf[ks], q_u32 + swz(mt * 16 + (lm & 1) * 8 + lr, ks * 2 + (lm >> 1)));
     }
 
-    // Q fragments stay in registers when there is a single m-tile
-    uint32_t qf[N_MT == 1 ? 8 : 1][4];
-    if constexpr (N_MT == 1) {
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            const int m = lane >> 3, r = lane & 7;
-            ldmatrix_x4(qf[ks], smem_u32(q_sm + swz((m & 1) * 8 + r, ks * 2 + (m >> 1))));
-        }
-    }
-
-    // ---- this warp's columns ---------------------------------------------------------------------
-    const int my_first = c0 + warp;
-    const int n_mine = (c1 > my_first) ? (c1 - my_first + kAttnWarps - 1) / kAttnWarps : 0;
+    // ---- this slot's columns ---------------------------------------------------------------------
+    const int my_first = c0 + slot;
+    const int n_mine = (c1 > my_first) ? (c1 - my_first + kAttnSlots - 1) / kAttnSlots : 0;
     const int32_t *slot_row = p.slot_tbl + (long long)bh * p.n_cols;
     const int32_t *blk_row = p.blk_tbl + (long long)bh * p.n_cols;
-    uint8_t *ring = kv_sm + warp * (kAttnStages * kEntryBytes);
-    const uint32_t ring_u32 = smem_u32(ring);
+    const uint32_t ring_u32 = smem_u32(kv_sm + slot * (kAttnStages * kEntryBytes));
 
-    // lane i of a 32-column window holds the table entries of this warp's column i
+    // lane i of a 32-column window holds the table entries of this slot's column i
     int win_slot = -1, win_blk = -1;
     auto load_window = [&](int first_i) {
-        const int c = my_first + (first_i + lane) * kAttnWarps;
+        const int c = my_first + (first_i + lane) * kAttnSlots;
         win_blk = (first_i + lane < n_mine) ? blk_row[c] : -1;
         win_slot = (win_blk >= 0) ? slot_row[c] : -1;
     };
-    auto issue = [&](int i, int slot) {             // fetch this warp's i-th column into ring stage i % stages
-        if (slot >= 0) {
-            const uint8_t *src = p.pool + (long long)slot * kEntryBytes;
+    auto issue = [&](int i, int entry) {           // fetch this slot's i-th column into ring stage i % stages
+        if (entry >= 0) {
+            const uint8_t *src = p.pool + (long long)entry * kEntryBytes;
             const uint32_t dst = ring_u32 + (i % kAttnStages) * kEntryBytes;
 #pragma unroll
-            for (int c = 0; c < 16; ++c) {
-                const int gch = lane + 32 * c;                 // 16-byte chunk of the entry
+            for (int c = 0; c < 16 / N_MT; ++c) {
+                const int gch = slot_lane + SLOT_THREADS * c;          // 16-byte chunk of the entry
                 const int part = gch >> 8, r = (gch >> 4) & 15, ch = gch & 15;
                 cp_async16(dst + part * kPartBytes + swz(r, ch), src + gch * 16);
             }
         }
         cp_async_commit();
     };
+    auto slot_sync = [&]() {
+        if constexpr (N_MT == 1) __syncwarp();
+        else slot_barrier(1 + slot, SLOT_THREADS);
+    };
 
     load_window(0);
 #pragma unroll
     for (int s = 0; s < kAttnStages - 1; ++s) {
-        const int slot = __shfl_sync(0xffffffffu, win_slot, s);     // s < 32 always
-        issue(s, s < n_mine ? slot : -1);
+        const int entry = __shfl_sync(0xffffffffu, win_slot, s);     // s < 32 always
+        issue(s, s < n_mine ? entry : -1);
     }
 
     for (int i = 0; i < n_mine; ++i) {
@@ -156,156 +163,144 @@ sparse_attn_kernel(const AttnParams p)
         // prefetch column i + stages - 1 (its ring stage was released at the end of iteration i - 1)
         {
             const int nx = i + kAttnStages - 1;
-            int slot = -1;
+            int entry = -1;
             if (nx < n_mine) {
-                // the window covers columns [32 * (i / 32), +32); nx may fall into the next one
-                const int base = (i >> 5) << 5;
-                if (nx < base + 32) slot = __shfl_sync(0xffffffffu, win_slot, nx - base);
+                const int base = (i >> 5) << 5;                      // the window covers [base, base + 32)
+                if (nx < base + 32) entry = __shfl_sync(0xffffffffu, win_slot, nx - base);
                 else {
-                    const int c = my_first + nx * kAttnWarps;
+                    const int c = my_first + nx * kAttnSlots;
                     const int bk = blk_row[c];
-                    slot = bk >= 0 ? slot_row[c] : -1;
+                    entry = bk >= 0 ? slot_row[c] : -1;
                 }
             }
-            issue(nx, slot);
+            issue(nx, entry);
         }
         const int blk = __shfl_sync(0xffffffffu, win_blk, i & 31);
         cp_async_wait<kAttnStages - 1>();
-        __syncwarp();
+        slot_sync();                                   // every thread's share of the entry has landed
         if (blk >= 0) {
             const uint32_t k_u32 = ring_u32 + (i % kAttnStages) * kEntryBytes;
             const uint32_t v_u32 = k_u32 + kPartBytes;
 
-            // ---- S = Q K^T for 16 keys -------------------------------------------------------------
-            float s[N_MT][2][4];
+            // ---- S = Q K^T: 16 rows x 16 keys -------------------------------------------------------
+            float s[2][4];
 #pragma unroll
-            for (int mt = 0; mt < N_MT; ++mt)
-#pragma unroll
-                for (int nt = 0; nt < 2; ++nt) s[mt][nt][0] = s[mt][nt][1] = s[mt][nt][2] = s[mt][nt][3] = 0.f;
+            for (int nt = 0; nt < 2; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
-                uint32_t kf[4];
-                {
-                    const int m = lane >> 3, r = lane & 7;
-                    ldmatrix_x4(kf, k_u32 + swz((m >> 1) * 8 + r, ks * 2 + (m & 1)));
-                }
+                uint32_t kf[4], a[4];
+                ldmatrix_x4(kf, k_u32 + swz((lm >> 1) * 8 + lr, ks * 2 + (lm & 1)));
+                if constexpr (kQInRegs) {
 #pragma unroll
-                for (int mt = 0; mt < N_MT; ++mt) {
-                    uint32_t a[4];
-                    if constexpr (N_MT == 1) {
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) a[e] = qf[ks][e];
-                    } else {
-                        const int m = lane >> 3, r = lane & 7;
-                        ldmatrix_x4(a, smem_u32(q_sm + swz(mt * 16 + (m & 1) * 8 + r, ks * 2 + (m >> 1))));
-                    }
-                    mma_bf16_16816(s[mt][0], a, kf[0], kf[1]);
-                    mma_bf16_16816(s[mt][1], a, kf[2], kf[3]);
+                    for (int e = 0; e < 4; ++e) a[e] = qf[ks][e];
+                } else {
+                    ldmatrix_x4(a, q_u32 + swz(mt * 16 + (lm & 1) * 8 + lr, ks * 2 + (lm >> 1)));
                 }
+                mma_bf16_16816(s[0], a, kf[0], kf[1]);
+                mma_bf16_16816(s[1], a, kf[2], kf[3]);
             }
 
-            // ---- online softmax -----------------------------------------------------------------------
+            // ---- online softmax with a lazily raised running max -----------------------------------------
             const int pos0 = blk * kBlock;                       // position of key 0 of the block
-            uint32_t pf[N_MT][4];
+            const bool masked = pos0 + kBlock - 1 > L;           // only local blocks reach past the history
+            float x[2][4], mxs[2];
+            bool raise = false;
 #pragma unroll
-            for (int mt = 0; mt < N_MT; ++mt) {
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {                    // e = 0: row g, e = 1: row g + 8
-                    float x[4];                                  // keys 2*t4, 2*t4+1, 8+2*t4, 8+2*t4+1
-                    x[0] = s[mt][0][2 * e]; x[1] = s[mt][0][2 * e + 1];
-                    x[2] = s[mt][1][2 * e]; x[3] = s[mt][1][2 * e + 1];
-                    const int lim = limit[mt][e] - pos0;         // keys with index <= lim are visible
+            for (int e = 0; e < 2; ++e) {                        // e = 0: row g, e = 1: row g + 8
+                x[e][0] = s[0][2 * e]; x[e][1] = s[0][2 * e + 1];        // keys 2*t4, 2*t4+1
+                x[e][2] = s[1][2 * e]; x[e][3] = s[1][2 * e + 1];        // keys 8+2*t4, 8+2*t4+1
+                if (masked) {
+                    const int lim = limit[e] - pos0;             // keys with index <= lim are visible
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         const int key = (c >> 1) * 8 + 2 * t4 + (c & 1);
-                        x[c] = key <= lim ? x[c] * p.scale_log2 : -CUDART_INF_F;
-                    }
-                    float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
-                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                    const float m_new = fmaxf(m_run[mt][e], mx);
-                    const float m_use = m_new == -CUDART_INF_F ? 0.f : m_new;
-                    const float alpha = fast_exp2(m_run[mt][e] - m_use);
-                    m_run[mt][e] = m_new;
-                    // round P to bf16 first and sum the rounded values, so that the normaliser
-                    // matches what the tensor cores multiply with V
-                    const __nv_bfloat162 p01 = __floats2bfloat162_rn(fast_exp2(x[0] - m_use), fast_exp2(x[1] - m_use));
-                    const __nv_bfloat162 p23 = __floats2bfloat162_rn(fast_exp2(x[2] - m_use), fast_exp2(x[3] - m_use));
-                    const float2 f01 = __bfloat1622float2(p01), f23 = __bfloat1622float2(p23);
-                    l_run[mt][e] = l_run[mt][e] * alpha + (f01.x + f01.y) + (f23.x + f23.y);
-                    pf[mt][e] = *reinterpret_cast<const uint32_t *>(&p01);         // a0 / a1: keys 0..7
-                    pf[mt][2 + e] = *reinterpret_cast<const uint32_t *>(&p23);     // a2 / a3: keys 8..15
-#pragma unroll
-                    for (int nt = 0; nt < 16; ++nt) {
-                        o[mt][nt][2 * e] *= alpha;
-                        o[mt][nt][2 * e + 1] *= alpha;
+                        if (key > lim) x[e][c] = -CUDART_INF_F;
                     }
                 }
+                float mx = fmaxf(fmaxf(x[e][0], x[e][1]), fmaxf(x[e][2], x[e][3]));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                mxs[e] = mx * p.scale_log2;                      // scale > 0: max commutes with scaling
+                raise |= mxs[e] > m_run[e] + 8.0f;               // also true for the first visible key
+            }
+            if (__any_sync(0xffffffffu, raise)) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const float m_new = mxs[e] > m_run[e] + 8.0f ? mxs[e] : m_run[e];
+                    const float alpha = m_new == -CUDART_INF_F ? 1.f : fast_exp2(m_run[e] - m_new);
+                    m_run[e] = m_new;
+                    l_run[e] *= alpha;
+#pragma unroll
+                    for (int nt = 0; nt < 16; ++nt) {
+                        o[nt][2 * e] *= alpha;
+                        o[nt][2 * e + 1] *= alpha;
+                    }
+                }
+            }
+            uint32_t pf[4];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const float neg_m = m_run[e] == -CUDART_INF_F ? 0.f : -m_run[e];
+                float pr[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) pr[c] = fast_exp2(fmaf(x[e][c], p.scale_log2, neg_m));
+                l_run[e] += (pr[0] + pr[1]) + (pr[2] + pr[3]);
+                pf[e] = pack_bf16x2(pr[0], pr[1]);               // a0 / a1: keys 0..7
+                pf[2 + e] = pack_bf16x2(pr[2], pr[3]);           // a2 / a3: keys 8..15
             }
 
             // ---- O += P V --------------------------------------------------------------------------------
 #pragma unroll
             for (int np = 0; np < 8; ++np) {
                 uint32_t vf[4];
-                {
-                    const int m = lane >> 3, r = lane & 7;
-                    ldmatrix_x4_trans(vf, v_u32 + swz((m & 1) * 8 + r, np * 2 + (m >> 1)));
-                }
-#pragma unroll
-                for (int mt = 0; mt < N_MT; ++mt) {
-                    mma_bf16_16816(o[mt][2 * np], pf[mt], vf[0], vf[1]);
-                    mma_bf16_16816(o[mt][2 * np + 1], pf[mt], vf[2], vf[3]);
-                }
+                ldmatrix_x4_trans(vf, v_u32 + swz((lm & 1) * 8 + lr, np * 2 + (lm >> 1)));
+                mma_bf16_16816(o[2 * np], pf, vf[0], vf[1]);
+                mma_bf16_16816(o[2 * np + 1], pf, vf[2], vf[3]);
             }
         }
-        __syncwarp();        // every lane is done with this ring stage before it is refilled
+        slot_sync();         // every thread of the slot is done with this ring stage before it is refilled
     }
     cp_async_wait<0>();
 
-    // ---- merge the four warps through shared memory ----------------------------------------------------
+    // ---- merge the four slots through shared memory ----------------------------------------------------
 #pragma unroll
-    for (int mt = 0; mt < N_MT; ++mt)
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            float l = l_run[mt][e];
-            l += __shfl_xor_sync(0xffffffffu, l, 1);
-            l += __shfl_xor_sync(0xffffffffu, l, 2);
-            l_run[mt][e] = l;
-        }
+    for (int e = 0; e < 2; ++e) {
+        float l = l_run[e];
+        l += __shfl_xor_sync(0xffffffffu, l, 1);
+        l += __shfl_xor_sync(0xffffffffu, l, 2);
+        l_run[e] = l;
+    }
     __syncthreads();                                        // all rings idle: reuse them
-    float *mo = reinterpret_cast<float *>(kv_sm);           // [warps][QROWS][128]
-    float *mm = mo + kAttnWarps * QROWS * kHeadDim;         // [warps][QROWS]
-    float *ml = mm + kAttnWarps * QROWS;                    // [warps][QROWS]
+    float *mo = reinterpret_cast<float *>(kv_sm);           // [slots][QROWS][128]
+    float *mm = mo + kAttnSlots * QROWS * kHeadDim;         // [slots][QROWS]
+    float *ml = mm + kAttnSlots * QROWS;                    // [slots][QROWS]
 #pragma unroll
-    for (int mt = 0; mt < N_MT; ++mt) {
+    for (int e = 0; e < 2; ++e) {
+        const int r = mt * 16 + g + 8 * e;
+        float *dst = mo + ((slot * QROWS + r) * kHeadDim);
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            const int r = mt * 16 + g + 8 * e;
-            float *dst = mo + ((warp * QROWS + r) * kHeadDim);
-#pragma unroll
-            for (int nt = 0; nt < 16; ++nt)
-                *reinterpret_cast<float2 *>(dst + nt * 8 + 2 * t4) = make_float2(o[mt][nt][2 * e], o[mt][nt][2 * e + 1]);
-            if (t4 == 0) {
-                mm[warp * QROWS + r] = m_run[mt][e];
-                ml[warp * QROWS + r] = l_run[mt][e];
-            }
+        for (int nt = 0; nt < 16; ++nt)
+            *reinterpret_cast<float2 *>(dst + nt * 8 + 2 * t4) = make_float2(o[nt][2 * e], o[nt][2 * e + 1]);
+        if (t4 == 0) {
+            mm[slot * QROWS + r] = m_run[e];
+            ml[slot * QROWS + r] = l_run[e];
         }
     }
     __syncthreads();
 
-    const int d = tid;                                       // 128 threads <-> 128 output dims
-    for (int r = 0; r < nrows; ++r) {
-        float mw[kAttnWarps], mx = -CUDART_INF_F;
+    const int d = tid & (kHeadDim - 1);                      // 128 threads <-> 128 output dims
+    for (int r = tid >> 7; r < nrows; r += NTHREADS / kHeadDim) {
+        float mw[kAttnSlots], mx = -CUDART_INF_F;
 #pragma unroll
-        for (int w = 0; w < kAttnWarps; ++w) {
+        for (int w = 0; w < kAttnSlots; ++w) {
             mw[w] = mm[w * QROWS + r];
             mx = fmaxf(mx, mw[w]);
         }
         float acc = 0.f, den = 0.f;
         if (mx > -CUDART_INF_F) {
 #pragma unroll
-            for (int w = 0; w < kAttnWarps; ++w) {
-                const float f = fast_exp2(mw[w] - mx);       // 0 for a warp that saw no key
+            for (int w = 0; w < kAttnSlots; ++w) {
+                const float f = fast_exp2(mw[w] - mx);       // 0 for a slot that saw no key
                 acc += f * mo[(w * QROWS + r) * kHeadDim + d];
                 den += f * ml[w * QROWS + r];
             }
@@ -389,6 +384,28 @@ static AttnPlan attn_plan(const oasis_dims_t *dims, int T, int n_cols)
     return pl;
 }
 
+// Enqueues the attention kernel (and the split combine) for a plan.
+static int launch_attn(const AttnPlan &pl, const AttnParams &p, long long combine_ctas, cudaStream_t st,
+                       const char *who)
+{
+    const size_t smem = (size_t)pl.n_mt * 16 * kRowBytes + (size_t)kAttnSlots * kAttnStages * kEntryBytes;
+    cudaError_t e;
+    if (pl.n_mt == 1) {
+        e = cudaFuncSetAttribute(sparse_attn_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) sparse_attn_kernel<1><<<(unsigned)pl.items, kAttnSlots * 32, smem, st>>>(p);
+    } else {
+        e = cudaFuncSetAttribute(sparse_attn_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) sparse_attn_kernel<2><<<(unsigned)pl.items, kAttnSlots * 64, smem, st>>>(p);
+    }
+    if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "%s: %s", who, cudaGetErrorString(e));
+    if (int rc = check_launch(who)) return rc;
+    if (pl.n_splits > 1) {
+        attn_combine_kernel<<<(unsigned)combine_ctas, 128, 0, st>>>(p);
+        return check_launch(who);
+    }
+    return OASIS_OK;
+}
+
 }  // namespace oasis
 
 extern "C" size_t oasis_attn_workspace_bytes(const oasis_dims_t *dims, int32_t n_q_tokens, int32_t n_cols)
@@ -437,23 +454,7 @@ extern "C" int oasis_sparse_attn(const oasis_dims_t *dims, const void *q, int32_
     p.n_splits = pl.n_splits; p.cols_per_split = pl.cols_per_split;
     p.n_groups = pl.n_groups; p.rows_per_group = pl.rows_per_group;
 
-    cudaStream_t st = (cudaStream_t)stream;
-    const size_t smem = (size_t)pl.n_mt * 16 * kRowBytes + (size_t)kAttnWarps * kAttnStages * kEntryBytes;
-    cudaError_t e;
-    if (pl.n_mt == 1) {
-        e = cudaFuncSetAttribute(sparse_attn_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess) sparse_attn_kernel<1><<<(unsigned)pl.items, kAttnWarps * 32, smem, st>>>(p);
-    } else {
-        e = cudaFuncSetAttribute(sparse_attn_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess) sparse_attn_kernel<2><<<(unsigned)pl.items, kAttnWarps * 32, smem, st>>>(p);
-    }
-    if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "oasis_sparse_attn: %s", cudaGetErrorString(e));
-    if (int rc = check_launch("oasis_sparse_attn")) return rc;
-    if (pl.n_splits > 1) {
-        attn_combine_kernel<<<(unsigned)((long long)dims->batch * dims->n_kv_heads * p.R), 128, 0, st>>>(p);
-        return check_launch("oasis_sparse_attn (combine)");
-    }
-    return OASIS_OK;
+    return launch_attn(pl, p, (long long)dims->batch * dims->n_kv_heads * p.R, (cudaStream_t)stream, "oasis_sparse_attn");
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -547,21 +548,6 @@ extern "C" int oasis_sparse_attn_static_scratch(const oasis_dims_t *dims, const 
     p.n_splits = pl.n_splits; p.cols_per_split = pl.cols_per_split;
     p.n_groups = pl.n_groups; p.rows_per_group = pl.rows_per_group;
 
-    cudaStream_t st = (cudaStream_t)stream;
-    const size_t smem = (size_t)pl.n_mt * 16 * kRowBytes + (size_t)kAttnWarps * kAttnStages * kEntryBytes;
-    cudaError_t e;
-    if (pl.n_mt == 1) {
-        e = cudaFuncSetAttribute(sparse_attn_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess) sparse_attn_kernel<1><<<(unsigned)pl.items, kAttnWarps * 32, smem, st>>>(p);
-    } else {
-        e = cudaFuncSetAttribute(sparse_attn_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess) sparse_attn_kernel<2><<<(unsigned)pl.items, kAttnWarps * 32, smem, st>>>(p);
-    }
-    if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "oasis_sparse_attn_static_scratch: %s", cudaGetErrorString(e));
-    if (int rc = check_launch("oasis_sparse_attn_static_scratch")) return rc;
-    if (pl.n_splits > 1) {
-        attn_combine_kernel<<<(unsigned)((long long)dims->batch * dims->n_kv_heads * p.R), 128, 0, st>>>(p);
-        return check_launch("oasis_sparse_attn_static_scratch (combine)");
-    }
-    return OASIS_OK;
+    return launch_attn(pl, p, (long long)dims->batch * dims->n_kv_heads * p.R, (cudaStream_t)stream,
+                       "oasis_sparse_attn_static_scratch");
 }

@@ -20,6 +20,7 @@ int fail(int code, const char *fmt, ...);
 int check_dims(const oasis_dims_t *dims);
 int check_launch(const char *what);   // cudaGetLastError() -> status
 int sm_count();                       // multiprocessors of the current device (148 if unknown)
+int32_t *error_word();                // device word registered with oasis_set_error_word (or NULL)
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

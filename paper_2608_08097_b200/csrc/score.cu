@@ -19,6 +19,8 @@
 // Algorithmic traffic: 512 B read + 4 B written per (request, KV head, block).
 #include <math_constants.h>
 
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace oasis {
@@ -180,6 +182,10 @@ score_blocks_kernel(const ScoreParams p)
     }
 }
 
+int score_blocks_tc(const oasis_dims_t *dims, const void *q_draft, int64_t q_batch_stride, int32_t n_draft,
+                    const void *summaries, const int32_t *n_full_blocks, int32_t reduce_mode, float *scores,
+                    int32_t *err_word, cudaStream_t st);          // score_tc.cu
+
 }  // namespace oasis
 
 extern "C" int oasis_score_blocks(const oasis_dims_t *dims, const void *q_draft,
@@ -202,6 +208,14 @@ extern "C" int oasis_score_blocks(const oasis_dims_t *dims, const void *q_draft,
     if (q_batch_stride < (int64_t)n_draft * dims->n_q_heads * kHeadDim || q_batch_stride % 8 != 0)
         return fail(OASIS_ERR_INVALID_ARG, "oasis_score_blocks: q_batch_stride %lld", (long long)q_batch_stride);
     if (dims->batch == 0) return OASIS_OK;
+    if ((long long)dims->batch * dims->n_kv_heads * dims->max_blocks > 0x7fffffffLL)
+        return fail(OASIS_ERR_UNSUPPORTED, "oasis_score_blocks: more than 2^31 summary rows");
+    {
+        static const bool legacy = getenv("OASIS_SCORE_MMA_SYNC") != nullptr;   // development switch
+        if (!legacy)
+            return score_blocks_tc(dims, q_draft, q_batch_stride, n_draft, summaries, n_full_blocks, reduce_mode,
+                                   scores, error_word(), (cudaStream_t)stream);
+    }
 
     ScoreParams p;
     p.q = (const uint8_t *)q_draft;

@@ -1,0 +1,421 @@
+// Step 1 on the 5th-generation tensor cores: block scores from the draft queries (Sec. 4.2.1).
+//
+// As in score.cu, U(q, j) = q^- . min_j + q^+ . max_j, so the scores of the R query rows that
+// share a KV head against a run of blocks are one small dense contraction.  Here the blocks
+// are the M dimension (swap-AB): for a tile of 128 consecutive blocks
+//     D[128 blocks x N] = A[128 x 256] (summaries, [min | max], K-major)  x  B[256 x N] (q^- | q^+)
+// with N = R rounded up to 16, followed by a max (or sum) over the N columns of every row.
+//
+// A persistent CTA per SM walks a contiguous range of tiles with three warp roles:
+//   warp 0     TMA producer: four 2-D tensor copies (128 rows x 128 B, 128-byte swizzle) per tile
+//              into a ring of 64 KiB stages, completion on mbarriers; it also builds the
+//              (q^- | q^+) operand of every new (request, KV head) in the same swizzled layout.
+//   warp 1     one thread issues 16 tcgen05.mma (128 x N x 16, bf16 -> fp32) per tile into one of
+//              two TMEM accumulators and commits to the stage's "empty" and the accumulator's
+//              "full" barrier.
+//   warps 2-5  epilogue: tcgen05.ld of the thread's TMEM lane (= one block), max / sum over its N
+//              columns, one coalesced fp32 store per block.
+// Bytes in flight are bounded by shared memory (up to three 64 KiB stages per SM), not by
+// registers; the tensor work per tile is tiny, so the kernel is HBM bound.
+// Every wait is bounded: on a timeout the thread records a code in the error word (if one was
+// registered), stops working and the CTA releases its TMEM and returns.
+// Algorithmic traffic: 512 B read + 4 B written per (request, KV head, block).
+#include <cuda.h>
+#include <math_constants.h>
+
+#include "common.cuh"
+
+namespace oasis {
+
+constexpr int kTcThreads = 192;
+constexpr int kTileBlocks = 128;
+constexpr int kATileBytes = kTileBlocks * kSummaryBytes;   // 64 KiB
+constexpr int kSubTileBytes = kTileBlocks * 128;           // one 64-element K chunk of the tile: 16 KiB
+constexpr int kMaxStages = 3;
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+struct ScoreTcParams {
+    const uint8_t *q;
+    long long q_batch_stride;
+    const int32_t *n_full;
+    float *scores;
+    int32_t *err;
+    int Hq, Hkv, G, R, N, max_blocks, tiles_per_bh, reduce_sum, stages, tmem_cols, n_bbuf;
+    long long total_tiles;
+};
+
+// ---- PTX wrappers -----------------------------------------------------------------------------------
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait: false (and an error code) if the phase did not complete within the spin limit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t *err, int code)
+{
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    if (err) atomicCAS(err, 0, code);
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major operand stored as rows of 128 bytes with the
+// 128-byte swizzle (8-row groups 1024 bytes apart).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3ffffu) >> 4);          // start address
+    d |= (uint64_t)1 << 16;                           // leading-dimension byte offset (unused here)
+    d |= (uint64_t)(1024 >> 4) << 32;                 // stride between 8-row groups
+    d |= (uint64_t)1 << 46;                           // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                           // 128-byte swizzle
+    return d;
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t a_u32 = base;                                        // [stages][64 KiB]
+    const uint32_t b_bytes = (uint32_t)p.N * kSummaryBytes;
+    const uint32_t b_u32 = a_u32 + (uint32_t)p.stages * kATileBytes;     // [2][N][512 B] as 4 sub-tiles of N x 128 B
+    uint8_t *b_ptr = base_ptr + (size_t)p.stages * kATileBytes;
+    const uint32_t bar_u32 = b_u32 + p.n_bbuf * b_bytes;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(b_ptr + p.n_bbuf * b_bytes + 128);
+    auto bar_full = [&](int s) { return bar_u32 + 8u * s; };
+    auto bar_empty = [&](int s) { return bar_u32 + 8u * (kMaxStages + s); };
+    auto bar_acc_full = [&](int a) { return bar_u32 + 8u * (2 * kMaxStages + a); };
+    auto bar_acc_empty = [&](int a) { return bar_u32 + 8u * (2 * kMaxStages + 2 + a); };
+    auto bar_b_full = [&](int a) { return bar_u32 + 8u * (2 * kMaxStages + 4 + a); };
+    auto bar_b_empty = [&](int a) { return bar_u32 + 8u * (2 * kMaxStages + 6 + a); };
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    const long long t0 = p.total_tiles * blockIdx.x / gridDim.x;
+    const long long t1 = p.total_tiles * (blockIdx.x + 1) / gridDim.x;
+
+    // First tile at or after t (and before t1) that has candidate blocks; t1 if there is none.
+    auto next_active = [&](long long t) {
+        for (; t < t1; ++t) {
+            const long long bh = t / p.tiles_per_bh;
+            const int j0 = (int)(t % p.tiles_per_bh) * kTileBlocks;
+            if (j0 < p.n_full[(int)(bh / p.Hkv)]) break;
+        }
+        return t;
+    };
+    // (q^- | q^+) rows of one (request, KV head), K-major, 128-byte swizzle: element k of row n
+    // lives in sub-tile k / 64.  `nthr` threads (index `me`) share the work; loads are issued
+    // eight at a time so their latencies overlap.
+    auto build_b = [&](long long bh, int buf, int me, int nthr) {
+        const int b = (int)(bh / p.Hkv), h = (int)(bh % p.Hkv);
+        uint8_t *dstb = b_ptr + (size_t)buf * b_bytes;
+        const int tasks = p.N * 16;                              // 16-byte chunks of the query rows
+        for (int i0 = me; i0 < tasks; i0 += nthr * 8) {
+            uint4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + nthr * u;
+                v[u] = make_uint4(0, 0, 0, 0);
+                const int n = i >> 4, c = i & 15;
+                if (i < tasks && (n < p.R || !p.reduce_sum)) {
+                    const int r = n % p.R;
+                    const int tq = r / p.G, a = h * p.G + r % p.G;
+                    v[u] = *reinterpret_cast<const uint4 *>(
+                        p.q + ((long long)b * p.q_batch_stride + ((long long)tq * p.Hq + a) * kHeadDim) * 2 + c * 16);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + nthr * u;
+                if (i >= tasks) continue;
+                const int n = i >> 4, c = i & 15;
+                const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f);
+                uint4 neg, pos;
+                const __nv_bfloat162 *f = reinterpret_cast<const __nv_bfloat162 *>(&v[u]);
+                __nv_bfloat162 *n2 = reinterpret_cast<__nv_bfloat162 *>(&neg);
+                __nv_bfloat162 *p2 = reinterpret_cast<__nv_bfloat162 *>(&pos);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    n2[e] = __hmin2(f[e], zero2);
+                    p2[e] = __hmax2(f[e], zero2);
+                }
+                const int sub = c >> 3, ch = (c & 7) ^ (n & 7);
+                uint8_t *row = dstb + n * 128 + ch * 16;
+                *reinterpret_cast<uint4 *>(row + (size_t)sub * p.N * 128) = neg;          // k in [0, 128): min rows
+                *reinterpret_cast<uint4 *>(row + (size_t)(2 + sub) * p.N * 128) = pos;    // k in [128, 256): max rows
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    };
+
+    if (tid == 0) {
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(bar_acc_full(a), 1);
+            mbar_init(bar_acc_empty(a), 4);
+            mbar_init(bar_b_full(a), 1);
+            mbar_init(bar_b_empty(a), 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)p.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    // The operand of the first (request, KV head) is built by the whole CTA while the barriers and
+    // the tensor memory are being set up.
+    const long long t_first = next_active(t0);
+    if (t_first < t1) build_b(t_first / p.tiles_per_bh, 0, tid, kTcThreads);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    if (tid == 0 && t_first < t1) mbar_arrive(bar_b_full(0));
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- producer
+        int it = 0, bo = 0;
+        bool alive = true;
+        long long t = t_first;
+        while (t < t1 && alive) {
+            const long long bh = t / p.tiles_per_bh;
+            const int j0 = (int)(t % p.tiles_per_bh) * kTileBlocks;
+            if (lane == 0) {
+                const int s = it % p.stages;
+                alive = mbar_wait(bar_empty(s), ((it / p.stages) & 1) ^ 1, p.err, 12);
+                if (alive) {
+                    mbar_arrive_expect_tx(bar_full(s), kATileBytes);
+                    const int y = (int)(bh * p.max_blocks + j0);
+#pragma unroll
+                    for (int kc = 0; kc < 4; ++kc)
+                        tma_load_2d(a_u32 + s * kATileBytes + kc * kSubTileBytes, &tmap, kc * 64, y, bar_full(s));
+                }
+            }
+            alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
+            ++it;
+            // one tile ahead: if the next tile belongs to another (request, KV head), build its operand now,
+            // while this tile's copies are in flight
+            const long long tn = next_active(t + 1);
+            if (alive && tn < t1 && tn / p.tiles_per_bh != bh) {
+                ++bo;
+                const int buf = bo % p.n_bbuf;
+                alive = mbar_wait(bar_b_empty(buf), ((bo / p.n_bbuf) & 1) ^ 1, p.err, 11);
+                if (alive) {
+                    build_b(tn / p.tiles_per_bh, buf, lane, 32);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_b_full(buf));
+                }
+            }
+            t = tn;
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.N >> 3) << 17) |
+                                   ((uint32_t)(kTileBlocks >> 4) << 24);
+            int it = 0, bo = -1;
+            long long cur_bh = -1;
+            bool alive = true;
+            for (long long t = t0; t < t1 && alive; ++t) {
+                const long long bh = t / p.tiles_per_bh;
+                const int j0 = (int)(t % p.tiles_per_bh) * kTileBlocks;
+                const int b = (int)(bh / p.Hkv);
+                if (j0 >= p.n_full[b]) continue;
+                if (bh != cur_bh) {
+                    if (bo >= 0) tc_commit(bar_b_empty(bo % p.n_bbuf));   // earlier MMAs no longer read that operand
+                    cur_bh = bh;
+                    ++bo;
+                    alive = mbar_wait(bar_b_full(bo % p.n_bbuf), (bo / p.n_bbuf) & 1, p.err, 21);
+                    if (!alive) break;
+                }
+                const int acc = it & 1, s = it % p.stages;
+                alive = mbar_wait(bar_acc_empty(acc), ((it >> 1) & 1) ^ 1, p.err, 22) &&
+                        mbar_wait(bar_full(s), (it / p.stages) & 1, p.err, 23);
+                if (!alive) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.N);
+                const uint32_t a_tile = a_u32 + s * kATileBytes;
+                const uint32_t b_tile = b_u32 + (bo % p.n_bbuf) * b_bytes;
+#pragma unroll
+                for (int kc = 0; kc < 4; ++kc) {
+#pragma unroll
+                    for (int k4 = 0; k4 < 4; ++k4) {
+                        const uint64_t ad = smem_desc_sw128(a_tile + kc * kSubTileBytes + k4 * 32);
+                        const uint64_t bd = smem_desc_sw128(b_tile + kc * p.N * 128 + k4 * 32);
+                        tc_mma_bf16(d_tmem, ad, bd, idesc, (kc | k4) ? 1u : 0u);
+                    }
+                }
+                tc_commit(bar_empty(s));         // the stage may be refilled once these MMAs have read it
+                tc_commit(bar_acc_full(acc));    // the accumulator is complete
+                ++it;
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue (warps 2..5)
+        const int quarter = warp & 3;            // TMEM lanes [32 * quarter, +32) belong to this warp
+        int it = 0;
+        bool alive = true;
+        for (long long t = t0; t < t1 && alive; ++t) {
+            const long long bh = t / p.tiles_per_bh;
+            const int j0 = (int)(t % p.tiles_per_bh) * kTileBlocks;
+            const int b = (int)(bh / p.Hkv);
+            const int nf = p.n_full[b];
+            const int j = j0 + quarter * 32 + lane;
+            float *out = p.scores + bh * p.max_blocks;
+            if (j0 >= nf) {
+                if (j < p.max_blocks) out[j] = -CUDART_INF_F;
+                continue;
+            }
+            const int acc = it & 1;
+            alive = mbar_wait(bar_acc_full(acc), (it >> 1) & 1, p.err, 31);
+            if (!alive) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.N);
+            float res = p.reduce_sum ? 0.f : -CUDART_INF_F;
+            for (int c = 0; c < p.N; c += 16) {
+                uint32_t v[16];
+                tc_ld16(taddr + c, v);
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                    const float f = __uint_as_float(v[e]);
+                    res = p.reduce_sum ? res + f : fmaxf(res, f);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acc_empty(acc));
+            if (j < p.max_blocks) out[j] = j < nf ? res : -CUDART_INF_F;
+            ++it;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols)
+                     : "memory");
+    }
+}
+
+// ---- host side -----------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)ptr;
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+int score_blocks_tc(const oasis_dims_t *dims, const void *q_draft, int64_t q_batch_stride, int32_t n_draft,
+                    const void *summaries, const int32_t *n_full_blocks, int32_t reduce_mode, float *scores,
+                    int32_t *err_word, cudaStream_t st)
+{
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return fail(OASIS_ERR_CUDA, "oasis_score_blocks: cuTensorMapEncodeTiled is not available");
+    const int G = dims->n_q_heads / dims->n_kv_heads;
+    const int R = n_draft * G;
+    const int N = (R + 15) / 16 * 16;
+    const long long rows = (long long)dims->batch * dims->n_kv_heads * dims->max_blocks;
+
+    CUtensorMap tmap;
+    const cuuint64_t gdim[2] = {256, (cuuint64_t)rows};
+    const cuuint64_t gstride[1] = {(cuuint64_t)kSummaryBytes};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kTileBlocks};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult cr = encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(summaries), gdim, gstride, box,
+                         estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return fail(OASIS_ERR_CUDA, "oasis_score_blocks: cuTensorMapEncodeTiled failed (%d)", (int)cr);
+
+    ScoreTcParams p;
+    p.q = (const uint8_t *)q_draft;
+    p.q_batch_stride = q_batch_stride;
+    p.n_full = n_full_blocks;
+    p.scores = scores;
+    p.err = err_word;
+    p.Hq = dims->n_q_heads; p.Hkv = dims->n_kv_heads; p.G = G; p.R = R; p.N = N;
+    p.max_blocks = dims->max_blocks;
+    p.tiles_per_bh = (dims->max_blocks + kTileBlocks - 1) / kTileBlocks;
+    p.reduce_sum = reduce_mode == OASIS_REDUCE_SUM;
+    p.stages = N <= 32 ? 3 : 2;
+    p.n_bbuf = N <= 64 ? 2 : 1;          // 2 x 64 KiB of tiles + the operand(s) must fit in 227 KiB
+    int cols = 32;
+    while (cols < 2 * N) cols <<= 1;
+    p.tmem_cols = cols;
+    p.total_tiles = (long long)dims->batch * dims->n_kv_heads * p.tiles_per_bh;
+    const size_t smem = 1024 + (size_t)p.stages * kATileBytes + (size_t)p.n_bbuf * N * kSummaryBytes + 256;
+    cudaError_t e = cudaFuncSetAttribute(score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "oasis_score_blocks: shared memory %zu B: %s", smem, cudaGetErrorString(e));
+    long long grid = p.total_tiles < sm_count() ? p.total_tiles : sm_count();
+    score_tc_kernel<<<(unsigned)grid, kTcThreads, smem, st>>>(tmap, p);
+    return check_launch("oasis_score_blocks");
+}
+
+}  // namespace oasis
