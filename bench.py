@@ -31,6 +31,9 @@ import torch  # noqa: E402
 
 from paper_2608_08097_b200 import synth  # noqa: E402
 
+# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (configs[1] shapes)
+TRAFFIC_BYTES = {"score": None, "attn": None}
+
 METRIC = "sparse decode-attn+select tokens/s per layer"
 UNIT = "tokens/s/layer"
 
@@ -217,24 +220,28 @@ class Bench:
         eng.prime([self.q_dev[l][0] for l in range(self.n_layers)], self.first_dev[0].contiguous(), self.seq_dev[0].contiguous())
         return eng
 
-    def run_steps(self, eng, steps, timers=None, e2e=False, q_pinned=None, out_pinned=None, q_stage=None):
-        for s in steps:
-            if e2e:
-                q_list = q_stage
-                q_host = [q_pinned[l][s] for l in range(self.n_layers)]
-            else:
-                q_list = [self.q_dev[l][s] for l in range(self.n_layers)]
-                q_host = None
-            eng.step(q_list, self.seq_dev[s], self.first_dev[s], self.n_new_dev[s], self.nfull_next_dev[s],
-                     self.seq_next_dev[s], step_stamp=s + 1, timers=timers, q_host=q_host,
-                     out_host=out_pinned if e2e else None)
+    def step_args(self, s, e2e, q_pinned, q_stage, out_pinned):
+        if e2e:
+            q_list = q_stage
+            q_host = [q_pinned[l][s] for l in range(self.n_layers)]
+        else:
+            q_list = [self.q_dev[l][s] for l in range(self.n_layers)]
+            q_host = None
+        args = (q_list, self.seq_dev[s], self.first_dev[s], self.n_new_dev[s], self.nfull_next_dev[s],
+                self.seq_next_dev[s])
+        kw = dict(step_stamp=s + 1, q_host=q_host, out_host=out_pinned if e2e else None)
+        return args, kw
 
-    def timed(self, eng, world, W, K, e2e=False, collect=True, **kw):
-        """W warm-up steps, then exactly K timed steps; returns (ms per step, timers, clocks)."""
-        self.run_steps(eng, range(0, W), e2e=e2e, **kw)
-        eng.join()
+    def timed(self, eng, world, W, K, e2e=False, q_pinned=None, out_pinned=None, q_stage=None):
+        """Every step is captured into a CUDA graph; W warm-up replays, then exactly K timed
+        replays bracketed by barrier + synchronize.  Returns (ms per step, clocks, launches)."""
+        graphs = []
+        for s in range(W + K):
+            args, kw = self.step_args(s, e2e, q_pinned, q_stage, out_pinned)
+            graphs.append(eng.capture_step(*args, **kw))
+        for s in range(W):
+            eng.replay(graphs[s])
         torch.cuda.synchronize()
-        timers = {"score": [], "select": [], "attn": [], "stage": []} if collect else None
         sampler = ClockSampler(self.dev.index or 0)
         sampler.start()
         barrier(world)
@@ -242,21 +249,25 @@ class Bench:
         start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         l0 = eng.launches
         start.record(eng.main)
-        self.run_steps(eng, range(W, W + K), timers=timers, e2e=e2e, **kw)
-        eng.join()
+        for s in range(W, W + K):
+            eng.replay(graphs[s])
         end.record(eng.main)
         torch.cuda.synchronize()
         barrier(world)
         clocks = sampler.stop()
-        ms = start.elapsed_time(end) / K
-        ms = max_over_ranks(ms, world, self.dev)
-        launches = eng.launches - l0
-        per_kernel = {}
-        if timers:
-            for name, pairs in timers.items():
-                if pairs:
-                    per_kernel[name] = sum(a.elapsed_time(b) for a, b in pairs) / len(pairs) * 1e3   # us per launch
-        return ms, per_kernel, clocks, launches
+        ms = max_over_ranks(start.elapsed_time(end) / K, world, self.dev)
+        return ms, clocks, eng.launches - l0
+
+    def kernel_times(self, eng, W, K, e2e=False, q_pinned=None, out_pinned=None, q_stage=None):
+        """Per-kernel durations (us per launch) with CUDA events on the launching streams, over
+        the same steps launched eagerly on the same three streams."""
+        timers = {"score": [], "select": [], "attn": [], "stage": []}
+        for s in range(W, W + K):
+            args, kw = self.step_args(s, e2e, q_pinned, q_stage, out_pinned)
+            eng.step(*args, timers=timers, **kw)
+        eng.join()
+        torch.cuda.synchronize()
+        return {n: sum(a.elapsed_time(b) for a, b in p) / len(p) * 1e3 for n, p in timers.items() if p}
 
     def recall(self, eng, steps):
         """Share of the draft-predicted top-k also chosen by the true next-step queries."""
@@ -327,6 +338,27 @@ def cpu_baseline(cfg, lay, budget_s=20.0):
                       % (done, cfg.batch, t_used)}
 
 
+def kernel_rooflines(per_kernel, score_bytes, attn_bytes, hbm_peak):
+    kern = {}
+    for name, nbytes in (("score", score_bytes), ("attn", attn_bytes)):
+        if name in per_kernel:
+            gbs = nbytes / (per_kernel[name] * 1e-6) / 1e9
+            kern[name] = {"us": round(per_kernel[name], 2), "algorithmic_MB": round(nbytes / 1e6, 2),
+                          "GBps": round(gbs, 1), "frac_of_measured": round(gbs / hbm_peak, 3),
+                          "frac_of_8TBps": round(gbs / 8000.0, 3)}
+    for name in ("select", "stage"):
+        if name in per_kernel:
+            kern[name] = {"us": round(per_kernel[name], 2)}
+    return kern
+
+
+def staged_entries(eng):
+    """Gather requests actually issued by the last step, per layer (delta mode: admitted pairs + local blocks)."""
+    if eng.mode == "delta":
+        return sum(int((p >= 0).sum().item()) for p in eng.plan_idx) / max(1, eng.n_layers)
+    return sum(int((L.stage_idx >= 0).sum().item()) for L in eng.layers) / max(1, eng.n_layers)
+
+
 def run_ours(args):
     world, rank, local = dist_setup(args)
     if not torch.cuda.is_available():
@@ -339,40 +371,35 @@ def run_ours(args):
     bench = Bench(args, cfg, dev, rank)
     h2d_peak = time_pinned_h2d(dev)
     bench.generate(want_mirror=True, want_host=not args.skip_e2e)
-
-    # ---- value: everything resident in HBM ---------------------------------------------------
-    eng = bench.engine("fetch_all", bench.mirror)
-    ms, per_kernel, clocks, launches = bench.timed(eng, world, W, K)
+    cap = max(1, int(math.floor(args.fetch_ratio * cfg.k_blocks)))
     steps = range(W, W + K)
     score_bytes, attn_bytes = algorithmic_bytes(cfg, bench.seq_steps, steps)
-    kern = {}
-    for name, nbytes in (("score", score_bytes), ("attn", attn_bytes)):
-        if name in per_kernel:
-            gbs = nbytes / (per_kernel[name] * 1e-6) / 1e9
-            kern[name] = {"us": round(per_kernel[name], 2), "algorithmic_MB": round(nbytes / 1e6, 2),
-                          "GBps": round(gbs, 1), "frac_of_measured": round(gbs / hbm_peak, 3),
-                          "frac_of_8TBps": round(gbs / 8000.0, 3)}
-    stage_bytes = cfg.batch * cfg.n_kv_heads * (cfg.k_blocks + 1) * 8192
-    if "stage" in per_kernel:
-        kern["stage_hbm_to_hbm"] = {"us": round(per_kernel["stage"], 2),
-                                    "GBps_read_plus_write": round(2 * stage_bytes / (per_kernel["stage"] * 1e-6) / 1e9, 1)}
-    if "select" in per_kernel:
-        kern["select"] = {"us": round(per_kernel["select"], 2)}
-    dominant = max(("score", "attn"), key=lambda n: per_kernel.get(n, 0.0))
-    value = cfg.batch * world / (ms * 1e-3 / cfg.layers)
-    recall = bench.recall(eng, range(W, min(W + 4, W + K)))
-
-    # compute only (no gather), for the overlap accounting
+    tok = cfg.batch * world * cfg.layers          # tokens/s/layer = batch / (step time / layers)
     extra = {}
-    eng_d = bench.engine("delta", bench.mirror, cap=max(1, int(math.floor(args.fetch_ratio * cfg.k_blocks))))
-    ms_d, _, _, _ = bench.timed(eng_d, world, W, K, collect=False)
-    extra["value_delta_cap"] = {"fetch_ratio": args.fetch_ratio, "ms_per_step": round(ms_d, 4),
-                                "value": round(cfg.batch * world / (ms_d * 1e-3 / cfg.layers), 1)}
-    del eng_d, eng
+
+    # ---- value: everything resident in HBM, capped-delta gather (the paper's default operating point) ----
+    eng = bench.engine("delta", bench.mirror, cap=cap)
+    ms, clocks, launches = bench.timed(eng, world, W, K)
+    value = tok / (ms * 1e-3)
+    recall = bench.recall(eng, range(W, min(W + 4, W + K)))
+    del eng
+    eng = bench.engine("delta", bench.mirror, cap=cap)        # instrumented eager pass, fresh state
+    for s in range(W):
+        a, kw = bench.step_args(s, False, None, None, None)
+        eng.step(*a, **kw)
+    per_kernel = bench.kernel_times(eng, W, min(K, 16))
+    kern = kernel_rooflines(per_kernel, score_bytes, attn_bytes, hbm_peak)
+    dominant = max(("score", "attn"), key=lambda n: per_kernel.get(n, 0.0))
+    del eng
+    eng = bench.engine("fetch_all", bench.mirror)
+    ms_f, _, _ = bench.timed(eng, world, W, K)
+    extra["value_fetch_all"] = {"ms_per_step": round(ms_f, 4), "value": round(tok / (ms_f * 1e-3), 1),
+                                "gather": "all K+1 blocks per (request, KV head) every step, HBM mirror -> pool"}
+    del eng
     bench.mirror.clear()
     torch.cuda.empty_cache()
 
-    # ---- e2e: KV in pinned host memory, queries in / outputs out every step -----------------------
+    # ---- e2e: KV in pinned host memory, queries in / outputs out every step --------------------------------
     e2e = None
     if not args.skip_e2e:
         q_pinned = [q.cpu().pin_memory() for q in bench.q_dev]
@@ -380,25 +407,34 @@ def run_ours(args):
         out_pinned = [torch.empty((cfg.batch, cfg.n_q_tokens, cfg.n_q_heads, 128), dtype=torch.bfloat16,
                                   pin_memory=True) for _ in range(cfg.layers)]
         kw = dict(q_pinned=q_pinned, out_pinned=out_pinned, q_stage=q_stage)
+        qo_bytes = cfg.batch * cfg.n_q_tokens * cfg.n_q_heads * 128 * 2
+        eng = bench.engine("delta", bench.host_kv, cap=cap)
+        ms_e, _, _ = bench.timed(eng, world, W, K, e2e=True, **kw)
+        n_req = staged_entries(eng)
+        pk = bench.kernel_times(eng, W, min(K, 8), e2e=True, **kw)
+        e2e = {"value": round(tok / (ms_e * 1e-3), 1), "unit": UNIT,
+               "h2d_bytes_per_step": int(cfg.layers * (n_req * 8192 + qo_bytes)),
+               "d2h_bytes_per_step": int(cfg.layers * qo_bytes), "ms_per_step": round(ms_e, 4), "steps": K,
+               "gather": "capped delta: at most %d new blocks per (request, KV head) per step + local blocks, "
+                         "zero-copy from pinned host memory" % cap}
+        if "stage" in pk:
+            gbs = n_req * 8192 / (pk["stage"] * 1e-6) / 1e9
+            extra["staged_delta"] = {"requests_per_layer": round(n_req, 1), "us_per_layer": round(pk["stage"], 1),
+                                     "GBps_overlapped": round(gbs, 2), "pinned_h2d_peak_GBps": round(h2d_peak, 2),
+                                     "frac_of_h2d_peak": round(gbs / h2d_peak, 3)}
+        del eng
         Ke = min(K, 8)
         eng = bench.engine("fetch_all", bench.host_kv)
-        ms_e, pk_e, _, _ = bench.timed(eng, world, W, Ke, e2e=True, **kw)
-        h2d = cfg.layers * (stage_bytes + cfg.batch * cfg.n_q_tokens * cfg.n_q_heads * 128 * 2)
-        d2h = cfg.layers * cfg.batch * cfg.n_q_tokens * cfg.n_q_heads * 128 * 2
-        e2e = {"value": round(cfg.batch * world / (ms_e * 1e-3 / cfg.layers), 1), "unit": UNIT,
-               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "ms_per_step": round(ms_e, 3),
-               "steps": Ke, "gather": "fetch-all (every selected block crosses the host link each step)"}
-        if "stage" in pk_e:
-            gbs = stage_bytes / (pk_e["stage"] * 1e-6) / 1e9
-            extra["staged"] = {"GBps_overlapped": round(gbs, 2), "pinned_h2d_peak_GBps": round(h2d_peak, 2),
-                               "frac_of_h2d_peak": round(gbs / h2d_peak, 3), "us_per_layer": round(pk_e["stage"], 1)}
-        del eng
-        cap = max(1, int(math.floor(args.fetch_ratio * cfg.k_blocks)))
-        eng = bench.engine("delta", bench.host_kv, cap=cap)
-        ms_ed, pk_ed, _, _ = bench.timed(eng, world, W, K, e2e=True, **kw)
-        extra["e2e_delta_cap"] = {"fetch_ratio": args.fetch_ratio, "cap_blocks": cap, "ms_per_step": round(ms_ed, 4),
-                                  "value": round(cfg.batch * world / (ms_ed * 1e-3 / cfg.layers), 1),
-                                  "h2d_bytes_per_step": int(cfg.layers * cfg.batch * cfg.n_kv_heads * (cap + 1) * 8192)}
+        ms_ef, _, _ = bench.timed(eng, world, W, Ke, e2e=True, **kw)
+        n_req_f = staged_entries(eng)
+        pk_f = bench.kernel_times(eng, W, min(Ke, 4), e2e=True, **kw)
+        extra["e2e_fetch_all"] = {"ms_per_step": round(ms_ef, 3), "value": round(tok / (ms_ef * 1e-3), 1), "steps": Ke,
+                                  "h2d_bytes_per_step": int(cfg.layers * (n_req_f * 8192 + qo_bytes))}
+        if "stage" in pk_f:
+            gbs = n_req_f * 8192 / (pk_f["stage"] * 1e-6) / 1e9
+            extra["staged_fetch_all"] = {"us_per_layer": round(pk_f["stage"], 1), "GBps_overlapped": round(gbs, 2),
+                                         "pinned_h2d_peak_GBps": round(h2d_peak, 2),
+                                         "frac_of_h2d_peak": round(gbs / h2d_peak, 3)}
         del eng
 
     cpu = None
@@ -418,13 +454,16 @@ def run_ours(args):
                        "global_batch": cfg.batch * world, "parallelism": "replicas x%d" % world,
                        "l2": "inputs larger than L2: each step streams %d layers x %.0f MB of distinct summaries + staged KV"
                              % (cfg.layers, (score_bytes + attn_bytes) / 1e6),
-                       "gather": "fetch-all from an HBM mirror of the full KV (value); pinned host (e2e)"},
+                       "gather": "delta selection with capped eviction, fetch ratio %.2f (cap %d blocks per head per "
+                                 "step); full KV in an HBM mirror (value) / pinned host memory (e2e)" % (args.fetch_ratio, cap),
+                       "launch": "each decode step is one CUDA graph over three streams (attention / prediction / transfer)"},
             "gpu_launches": launches,
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
                        "samples": clocks["samples"]},
             "roofline": {"bound": "hbm", "kernel": dominant, "achieved": d.get("GBps"), "peak": hbm_peak,
-                         "unit": "GB/s", "frac": d.get("frac_of_measured"), "traffic": None,
-                         "peak_kind": peak_kind + " (STREAM-style copy)"},
+                         "unit": "GB/s", "frac": d.get("frac_of_measured"), "traffic": TRAFFIC_BYTES.get(dominant),
+                         "peak_kind": peak_kind + " (STREAM-style copy)",
+                         "timing": "CUDA events around each launch on its stream, same steps launched eagerly"},
             "kernels": kern,
             "recall_lookahead_topk": round(recall, 4),
             "e2e": e2e, "cpu_baseline": cpu, "setup_seconds": round(bench.gen_seconds, 1),

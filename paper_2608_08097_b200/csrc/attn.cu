@@ -20,6 +20,8 @@
 // Algorithmic traffic: 8 KiB per (request, KV head, column) plus Q and O.
 #include <math_constants.h>
 
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace oasis {
@@ -358,18 +360,36 @@ struct AttnPlan {
     size_t workspace;
 };
 
+// The tcgen05 kernel (attn_tc.cu) is the product path; the mma.sync kernel above stays as a
+// development cross-check behind an environment switch.
+static bool use_tc()
+{
+    static const bool legacy = getenv("OASIS_ATTN_MMA_SYNC") != nullptr;
+    return !legacy;
+}
+
+int launch_attn_tc(const oasis_dims_t *dims, const void *q, int n_q_tokens, const void *hbm_pool,
+                   const int32_t *slot_tbl, const int32_t *blk_tbl, int n_cols, const int32_t *seq_len, float scale,
+                   void *out, float *lse, float *part_o, float *part_lse, int n_splits, int cols_per_split,
+                   int stages, int32_t *err_word, cudaStream_t st, const char *who);      // attn_tc.cu
+
 static AttnPlan attn_plan(const oasis_dims_t *dims, int T, int n_cols)
 {
     AttnPlan pl;
     const int G = dims->n_q_heads / dims->n_kv_heads;
     const int R = T * G;
-    pl.n_groups = (R + 31) / 32;
-    pl.rows_per_group = (R + pl.n_groups - 1) / pl.n_groups;
+    if (use_tc()) {                      // all rows of a KV head in one CTA (M = 128)
+        pl.n_groups = 1;
+        pl.rows_per_group = R;
+    } else {
+        pl.n_groups = (R + 31) / 32;
+        pl.rows_per_group = (R + pl.n_groups - 1) / pl.n_groups;
+    }
     pl.n_mt = pl.rows_per_group <= 16 ? 1 : 2;
     const long long base = (long long)dims->batch * dims->n_kv_heads * pl.n_groups;
     // All CTAs should be resident at once (two per SM): a bandwidth-bound kernel then has no
     // tail.  Split the column list only as far as that allows, at least 8 columns per split.
-    const long long slots = 2LL * sm_count();
+    const long long slots = (use_tc() ? 1LL : 2LL) * sm_count();   // resident CTAs: the tcgen05 kernel runs one per SM
     long long s = base > 0 ? slots / base : 1;
     const long long max_s = (n_cols + 7) / 8;
     if (s > max_s) s = max_s;
@@ -385,9 +405,19 @@ static AttnPlan attn_plan(const oasis_dims_t *dims, int T, int n_cols)
 }
 
 // Enqueues the attention kernel (and the split combine) for a plan.
-static int launch_attn(const AttnPlan &pl, const AttnParams &p, long long combine_ctas, cudaStream_t st,
-                       const char *who)
+static int launch_attn(const oasis_dims_t *dims, const AttnPlan &pl, const AttnParams &p, const void *q,
+                       const void *pool, float scale, long long combine_ctas, cudaStream_t st, const char *who)
 {
+    if (use_tc()) {
+        if (int rc = launch_attn_tc(dims, q, p.T, pool, p.slot_tbl, p.blk_tbl, p.n_cols, p.seq_len, scale, p.out, p.lse,
+                                    p.part_o, p.part_lse, pl.n_splits, pl.cols_per_split, 7, error_word(), st, who))
+            return rc;
+        if (pl.n_splits > 1) {
+            attn_combine_kernel<<<(unsigned)combine_ctas, 128, 0, st>>>(p);
+            return check_launch(who);
+        }
+        return OASIS_OK;
+    }
     const size_t smem = (size_t)pl.n_mt * 16 * kRowBytes + (size_t)kAttnSlots * kAttnStages * kEntryBytes;
     cudaError_t e;
     if (pl.n_mt == 1) {
@@ -454,7 +484,8 @@ extern "C" int oasis_sparse_attn(const oasis_dims_t *dims, const void *q, int32_
     p.n_splits = pl.n_splits; p.cols_per_split = pl.cols_per_split;
     p.n_groups = pl.n_groups; p.rows_per_group = pl.rows_per_group;
 
-    return launch_attn(pl, p, (long long)dims->batch * dims->n_kv_heads * p.R, (cudaStream_t)stream, "oasis_sparse_attn");
+    return launch_attn(dims, pl, p, q, hbm_pool, scale, (long long)dims->batch * dims->n_kv_heads * p.R,
+                       (cudaStream_t)stream, "oasis_sparse_attn");
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -548,6 +579,6 @@ extern "C" int oasis_sparse_attn_static_scratch(const oasis_dims_t *dims, const 
     p.n_splits = pl.n_splits; p.cols_per_split = pl.cols_per_split;
     p.n_groups = pl.n_groups; p.rows_per_group = pl.rows_per_group;
 
-    return launch_attn(pl, p, (long long)dims->batch * dims->n_kv_heads * p.R, (cudaStream_t)stream,
-                       "oasis_sparse_attn_static_scratch");
+    return launch_attn(dims, pl, p, q, hbm_pool, scale, (long long)dims->batch * dims->n_kv_heads * p.R,
+                       (cudaStream_t)stream, "oasis_sparse_attn_static_scratch");
 }

@@ -1,0 +1,569 @@
+// Step 4 on the 5th-generation tensor cores: sparse paged decode attention (Sec. 4.2.1, 4.3).
+//
+// Work item = (request, KV head, split of the column list).  All query rows that share the KV
+// head (G heads x T verify-step tokens, at most 128) form the M = 128 rows of every MMA, so each
+// staged K/V block is read from HBM once.  A tile is four columns = 64 keys (32 KiB of K and V).
+//
+//   warp 0     TMA producer: per block four 2-D tensor copies (16 rows x 128 B, 128-byte swizzle:
+//              the two 64-dim halves of its K rows and of its V rows) gathered by slot id into a
+//              ring of 32 KiB stages; completion on the stage's mbarrier.
+//   warp 1     one thread issues the MMAs: S = Q K^T (8 x tcgen05.mma 128x64x16, both operands in
+//              shared memory) into one of two S buffers in tensor memory, and O += P V
+//              (4 x tcgen05.mma 128x128x16, P read from tensor memory, V from shared memory in its
+//              natural key-major layout).  S of tile i+1 is issued before P V of tile i, so the
+//              softmax of tile i overlaps the next Q K^T.
+//   warps 2-5  softmax, one thread per MMA row: tcgen05.ld of the row's logits, masking on local
+//              blocks only, exp2 against a running reference maximum that is raised lazily (only
+//              when a logit exceeds it by 2^8; the O row is then rescaled in tensor memory),
+//              running sum in a register, P rounded to bf16 and written back over S with
+//              tcgen05.st.  No cross-thread reduction exists anywhere in the softmax.
+//              A warp can only reach its own quarter of the 128 tensor-memory lanes, and a single
+//              warp's instruction rate bounds the softmax; so when the query rows fit in 32 (64)
+//              lanes they are replicated into all four (two) lane ranges, and each copy takes one
+//              (two) of the tile's four blocks, writing P = 0 for the others.  The copies' partial
+//              (max, sum, O) are merged through shared memory after the last tile.
+// After the merge the rows are normalised and written as bf16 (or, when the column list is
+// split, as a normalised partial plus its log-sum-exp to the workspace).
+// Every wait is bounded; a timeout records a code in the error word and the CTA winds down.
+// Algorithmic traffic: 8 KiB per (request, KV head, column) plus Q and O.
+#include <cuda.h>
+#include <math_constants.h>
+
+#include <cstdlib>
+
+#include "common.cuh"
+#include "tc_common.cuh"
+
+namespace oasis {
+
+constexpr int kAtThreads = 192;
+constexpr int kAtTileCols = 4;                              // blocks per tile
+constexpr int kAtTileKeys = kAtTileCols * kBlock;           // 64
+constexpr int kAtStageBytes = kAtTileCols * kEntryBytes;    // 32 KiB: one 8 KiB image per block
+// Shared-memory image of one block (one 5-D tensor copy): [row group 0..1][dim half 0..1][K, V][8 rows][128 B].
+constexpr int kImgGroup = 4096, kImgHalf = 2048, kImgPart = 1024;
+constexpr int kAtSBufs = 4;                                 // S / P buffers in tensor memory (Q K^T runs 3 tiles ahead)
+constexpr int kAtQBytes = 0;                                // Q lives in tensor memory
+constexpr int kAtMaxStages = 7;
+constexpr int kAtTmemCols = 512;                            // S buffers [0,256), O [256,384), Q [384,448)
+constexpr float kAtLog2e = 1.4426950408889634f;
+constexpr float kAtLn2 = 0.6931471805599453f;
+
+struct AttnTcParams {
+    const uint8_t *q;
+    const int32_t *slot_tbl;
+    const int32_t *blk_tbl;
+    const int32_t *seq_len;
+    uint8_t *out;
+    float *lse;
+    float *part_o;
+    float *part_lse;
+    int32_t *err;
+    float scale_log2;
+    int T, Hq, Hkv, G, n_cols, R, n_splits, cols_per_split, stages;
+};
+
+__device__ __forceinline__ void tc_mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&v)[16])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
+}
+__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t (&v)[8])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// K-major operand with 128-byte rows and the 128-byte swizzle is described by smem_desc_sw128().
+// MN-major operand (V: rows = keys, 64 dims = 128 bytes per row and half): 8-key groups 1024 bytes
+// apart, the second 64-dim half `half_stride` bytes further.
+__device__ __forceinline__ uint64_t smem_desc_sw128_mn(uint32_t addr, uint32_t half_stride, uint32_t group_stride)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)((half_stride >> 4) & 0x3fffu) << 16;   // leading-dimension byte offset
+    d |= (uint64_t)((group_stride >> 4) & 0x3fffu) << 32;  // stride between 8-key groups
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// K-major operand, 128-byte swizzle, 8-row groups `group_stride` bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128_k(uint32_t addr, uint32_t group_stride)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)((group_stride >> 4) & 0x3fffu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, int c3, int c4,
+                                            uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
+        : "memory");
+}
+
+template <int COPIES>
+__global__ void __launch_bounds__(kAtThreads, 1)
+sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcParams p)
+{
+    constexpr int RPC = 128 / COPIES;                       // MMA rows per copy of the query rows
+    constexpr int BPC = kAtTileCols / COPIES;               // blocks of a tile each copy handles
+    constexpr int KPC = BPC * kBlock;                       // keys of a tile each copy handles
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t kv_u32 = base + kAtQBytes;                        // [stages][32 KiB]
+    uint8_t *misc = base_ptr + kAtQBytes + (size_t)p.stages * kAtStageBytes;
+    const uint32_t bar_u32 = smem_u32(misc);
+    auto bar_full = [&](int s) { return bar_u32 + 8u * s; };
+    auto bar_empty = [&](int s) { return bar_u32 + 8u * (kAtMaxStages + s); };
+    auto bar_s_full = [&](int a) { return bar_u32 + 8u * (2 * kAtMaxStages + a); };
+    auto bar_p_full = [&](int a) { return bar_u32 + 8u * (2 * kAtMaxStages + kAtSBufs + a); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 8 * (2 * kAtMaxStages + 2 * kAtSBufs + 2));
+    int32_t *tile_blk = reinterpret_cast<int32_t *>(misc + 8 * (2 * kAtMaxStages + 2 * kAtSBufs + 4));   // [stages][4]
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int split = blockIdx.x % p.n_splits;
+    const int bh = blockIdx.x / p.n_splits;
+    const int b = bh / p.Hkv, h = bh % p.Hkv;
+    const int c0 = split * p.cols_per_split;
+    const int c1 = min(c0 + p.cols_per_split, p.n_cols);
+    const int n_tiles = (c1 - c0 + kAtTileCols - 1) / kAtTileCols;
+    const int L = p.seq_len[b];
+    const int32_t *slot_row = p.slot_tbl + (long long)bh * p.n_cols;
+    const int32_t *blk_row = p.blk_tbl + (long long)bh * p.n_cols;
+
+    // ---- set-up: barriers, tensor memory, Q operand, zeroed stages ------------------------------------
+    if (tid == 0) {
+        for (int s = 0; s < kAtMaxStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+        for (int a = 0; a < kAtSBufs; ++a) { mbar_init(bar_s_full(a), 1); mbar_init(bar_p_full(a), 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)kAtTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_o = tmem_base + kAtSBufs * kAtTileKeys;
+    const uint32_t tmem_q = tmem_o + kHeadDim;                       // Q as the A operand: 128 rows x 64 packed columns
+    if (warp >= 2) {
+        // every softmax thread owns one MMA row: it loads that row of Q (rows are replicated across the copies,
+        // rows past R are zero) and stores it to its tensor-memory lane
+        const int m_row = (warp & 3) * 32 + lane;
+        const int r = m_row % RPC;
+        uint4 v[16];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) v[c] = make_uint4(0, 0, 0, 0);
+        if (r < p.R) {
+            const int tq = r / p.G, a = h * p.G + r % p.G;
+            const uint4 *src = reinterpret_cast<const uint4 *>(p.q + ((((long long)b * p.T + tq) * p.Hq + a) * kHeadDim) * 2);
+#pragma unroll
+            for (int c = 0; c < 16; ++c) v[c] = src[c];
+        }
+        const uint32_t q_lane = tmem_q + ((uint32_t)((warp & 3) * 32) << 16);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const uint32_t w[16] = {v[4 * c].x, v[4 * c].y, v[4 * c].z, v[4 * c].w, v[4 * c + 1].x, v[4 * c + 1].y,
+                                    v[4 * c + 1].z, v[4 * c + 1].w, v[4 * c + 2].x, v[4 * c + 2].y, v[4 * c + 2].z,
+                                    v[4 * c + 2].w, v[4 * c + 3].x, v[4 * c + 3].y, v[4 * c + 3].z, v[4 * c + 3].w};
+            tc_st16(q_lane + c * 16, w);
+        }
+        tc_wait_st();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- producer
+        bool alive = true;
+        // Table entries are read 32 columns (eight tiles) at a time, lane j holding column j of the window, and the
+        // next window is requested as soon as the current one starts, so no table load sits on the critical path.
+        auto load_window = [&](int first_col, int &wblk, int &wslot) {
+            const int c = first_col + lane;
+            wblk = c < c1 ? blk_row[c] : -1;
+            wslot = c < c1 ? slot_row[c] : -1;
+        };
+        int cur_blk, cur_slot, nxt_blk = -1, nxt_slot = -1;
+        load_window(c0, cur_blk, cur_slot);
+        for (int i = 0; i < n_tiles && alive; ++i) {
+            if ((i & 7) == 0) {
+                if (i > 0) { cur_blk = nxt_blk; cur_slot = nxt_slot; }
+                load_window(c0 + (i + 8) * kAtTileCols, nxt_blk, nxt_slot);
+            }
+            const int src_lane = (i & 7) * kAtTileCols + (lane & 3);
+            int blk = __shfl_sync(0xffffffffu, cur_blk, src_lane);
+            const int slot = __shfl_sync(0xffffffffu, cur_slot, src_lane);
+            if (lane >= kAtTileCols) blk = -1;
+            const int s = i % p.stages;
+            if (lane == 0) alive = mbar_wait(bar_empty(s), ((i / p.stages) & 1) ^ 1, p.err, 41);
+            alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
+            if (!alive) break;
+            const unsigned valid = __ballot_sync(0xffffffffu, lane < kAtTileCols && blk >= 0);
+            if (lane < kAtTileCols) {
+                tile_blk[s * kAtTileCols + lane] = blk;
+                if (blk < 0) {
+                    // a missing block contributes P = 0, which must not meet stale NaN bit patterns in V
+                    uint8_t *img = base_ptr + kAtQBytes + (size_t)s * kAtStageBytes + lane * kEntryBytes;
+                    for (int u = 0; u < 4; ++u)                      // (row group, dim half) units of the V part
+                        for (int j = 0; j < kImgPart / 16; ++j)
+                            *reinterpret_cast<uint4 *>(img + (u >> 1) * kImgGroup + (u & 1) * kImgHalf + kImgPart + j * 16) =
+                                make_uint4(0, 0, 0, 0);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive_expect_tx(bar_full(s), (uint32_t)__popc(valid) * kEntryBytes);
+            __syncwarp();
+            if (lane < kAtTileCols && blk >= 0)                       // the whole 8 KiB entry in one copy
+                tma_load_5d(kv_u32 + s * kAtStageBytes + lane * kEntryBytes, &tmap, 0, 0, 2 * slot, 0, 0, bar_full(s));
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0 && n_tiles > 0) {
+            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAtTileKeys >> 3) << 17) | (8u << 24);
+            const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(128 >> 3) << 17) | (8u << 24);
+            bool alive = true;
+            // descriptors: the operand start address occupies the low 14 bits (16-byte units), so offsets are added there
+            const uint64_t k_desc0 = smem_desc_sw128_k(kv_u32, kImgGroup);
+            const uint64_t v_desc0 = smem_desc_sw128_mn(kv_u32 + kImgPart, kImgHalf, kImgGroup);
+            // Event-driven issue: whichever of "next Q K^T" (its tile has landed and an S buffer is free) and
+            // "next P V" (its P has been written) is ready goes first, so a late tile never delays a P V and
+            // with it the release of a stage.
+            int qk_next = 0, pv_next = 0;
+            uint32_t idle = 0;
+            while (pv_next < n_tiles) {
+                bool progressed = false;
+                if (qk_next < n_tiles && qk_next < pv_next + kAtSBufs) {
+                    const int i = qk_next, s = i % p.stages;
+                    if (mbar_test(bar_full(s), (i / p.stages) & 1)) {
+                        tc_fence_after();
+                        const uint64_t k_desc = k_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
+                        const uint32_t d_tmem = tmem_base + (uint32_t)((i % kAtSBufs) * kAtTileKeys);
+#pragma unroll
+                        for (int kc = 0; kc < 2; ++kc)
+#pragma unroll
+                            for (int k4 = 0; k4 < 4; ++k4)
+                                tc_mma_bf16_ts(d_tmem, tmem_q + (kc * 4 + k4) * 8,
+                                                   k_desc + (uint64_t)((kc * kImgHalf + k4 * 32) >> 4), idesc_qk,
+                                                   (kc | k4) ? 1u : 0u);
+                        tc_commit(bar_s_full(i % kAtSBufs));
+                        ++qk_next;
+                        progressed = true;
+                    }
+                }
+                if (pv_next < qk_next) {
+                    const int i = pv_next, s = i % p.stages;
+                    if (mbar_test(bar_p_full(i % kAtSBufs), (i / kAtSBufs) & 1)) {
+                        tc_fence_after();
+                        const uint64_t v_desc = v_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
+                        const uint32_t p_tmem = tmem_base + (uint32_t)((i % kAtSBufs) * kAtTileKeys);
+#pragma unroll
+                        for (int ks = 0; ks < kAtTileCols; ++ks)           // 16 keys per MMA = one block image
+                            tc_mma_bf16_ts(tmem_o, p_tmem + ks * 8, v_desc + (uint64_t)((ks * kEntryBytes) >> 4),
+                                               idesc_pv, (i | ks) ? 1u : 0u);
+                        tc_commit(bar_empty(s));         // stage free, and O complete up to this tile
+                        ++pv_next;
+                        progressed = true;
+                    }
+                }
+                if (progressed) idle = 0;
+                else if (++idle > kSpinLimit * 8u) {     // bounded: give up, flag, let the CTA wind down
+                    if (p.err) atomicCAS(p.err, 0, 53);
+                    break;
+                }
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- softmax, one thread per MMA row
+        const int quarter = warp & 3;
+        const int m_row = quarter * 32 + lane;                      // MMA row = tensor-memory lane
+        const int copy = m_row / RPC, row = m_row % RPC;            // which copy of the rows, which query row
+        const bool live_row = row < p.R;
+        const bool live_warp = (quarter * 32) % RPC < p.R;          // some lane of this warp holds a query row
+        const int limit = live_row ? L + row / p.G : -1;            // last visible position of this row
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        float m_ref = -CUDART_INF_F, l_sum = 0.f;
+        bool alive = true;
+        for (int i = 0; i < n_tiles && alive; ++i) {
+            alive = mbar_wait(bar_s_full(i % kAtSBufs), (i / kAtSBufs) & 1, p.err, 61);
+            if (!alive) break;
+            tc_fence_after();
+            const uint32_t s_tmem = tmem_base + lane_base + (uint32_t)((i % kAtSBufs) * kAtTileKeys);
+            if (live_warp) {
+                const int s = i % p.stages;
+                int nvis[BPC];                                      // visible keys of each of this copy's blocks
+                bool masked = false;
+#pragma unroll
+                for (int c = 0; c < BPC; ++c) {
+                    const int blk = tile_blk[s * kAtTileCols + copy * BPC + c];
+                    int n = blk < 0 ? 0 : limit - blk * kBlock + 1;
+                    n = max(0, min(n, kBlock));
+                    nvis[c] = n;
+                    masked |= n < kBlock;
+                }
+                masked = __any_sync(0xffffffffu, masked);
+                float x[KPC];
+                {
+                    uint32_t v[BPC][16];
+#pragma unroll
+                    for (int c = 0; c < BPC; ++c) tc_ld16_nowait(s_tmem + (copy * BPC + c) * 16, v[c]);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int c = 0; c < BPC; ++c)
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) x[c * 16 + e] = __uint_as_float(v[c][e]);
+                }
+                if (masked) {
+#pragma unroll
+                    for (int c = 0; c < BPC; ++c)
+#pragma unroll
+                        for (int e = 0; e < 16; ++e)
+                            if (e >= nvis[c]) x[c * 16 + e] = -CUDART_INF_F;
+                }
+                float mx4[4] = {x[0], x[1], x[2], x[3]};
+#pragma unroll
+                for (int e = 4; e < KPC; e += 4) {
+                    mx4[0] = fmaxf(mx4[0], x[e]); mx4[1] = fmaxf(mx4[1], x[e + 1]);
+                    mx4[2] = fmaxf(mx4[2], x[e + 2]); mx4[3] = fmaxf(mx4[3], x[e + 3]);
+                }
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                const float mxs = mx * p.scale_log2;
+                const bool raise = mxs > m_ref + 8.0f;
+                if (__any_sync(0xffffffffu, raise)) {
+                    // the O rows must be complete up to tile i-1 before they are rescaled
+                    // (its stage is released by the commit that follows that P V; with at least four stages in the
+                    // ring the phase parity of that barrier is unambiguous)
+                    if (i > 0) alive = mbar_wait(bar_empty((i - 1) % p.stages), ((i - 1) / p.stages) & 1, p.err, 62);
+                    tc_fence_after();
+                    const float m_new = raise ? mxs : m_ref;
+                    const float alpha = m_new == -CUDART_INF_F ? 1.f : fast_exp2(m_ref - m_new);
+                    m_ref = m_new;
+                    l_sum *= alpha;
+                    if (i > 0) {
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            uint32_t v[16];
+                            tc_ld16(tmem_o + lane_base + c * 16, v);
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
+                            tc_st16(tmem_o + lane_base + c * 16, v);
+                        }
+                        tc_wait_st();
+                    }
+                }
+                const float neg_m = m_ref == -CUDART_INF_F ? 0.f : -m_ref;
+                float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+                // P of the whole tile is 32 packed columns; this copy owns columns [copy*KPC/2, +KPC/2), the rest is 0
+                uint32_t pk[KPC / 2];
+#pragma unroll
+                for (int e = 0; e < KPC / 2; ++e) {
+                    const float p0 = fast_exp2(fmaf(x[2 * e], p.scale_log2, neg_m));
+                    const float p1 = fast_exp2(fmaf(x[2 * e + 1], p.scale_log2, neg_m));
+                    sum4[e & 3] += p0 + p1;
+                    pk[e] = pack_bf16x2(p0, p1);
+                }
+                l_sum += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+#pragma unroll
+                for (int g8 = 0; g8 < 4; ++g8) {                    // four groups of 8 packed columns = four blocks
+                    uint32_t w8[8];
+                    const int own = g8 - copy * BPC;                // index among this copy's blocks, if in [0, BPC)
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        uint32_t val = 0u;
+#pragma unroll
+                        for (int c = 0; c < BPC; ++c)
+                            if (own == c) val = pk[c * 8 + e];
+                        w8[e] = val;
+                    }
+                    tc_st8(s_tmem + g8 * 8, w8);
+                }
+                tc_wait_st();
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_p_full(i % kAtSBufs));
+        }
+        // ---- epilogue: merge the copies, normalise, write out ----------------------------------------------
+        if (alive && n_tiles > 0)
+            alive = mbar_wait(bar_empty((n_tiles - 1) % p.stages), ((n_tiles - 1) / p.stages) & 1, p.err, 63);
+        tc_fence_after();
+        // the K/V ring is idle now: stage the O rows there.  [128 MMA rows][132 floats], then max and sum.
+        float *o_sm = reinterpret_cast<float *>(base_ptr + kAtQBytes);
+        float *m_sm = o_sm + 128 * 132;
+        float *l_sm = m_sm + 128;
+        if (COPIES > 1) {
+            if (live_warp && alive && n_tiles > 0) {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    uint32_t v[16];
+                    tc_ld16(tmem_o + lane_base + c * 16, v);
+                    float4 *dst = reinterpret_cast<float4 *>(o_sm + m_row * 132 + c * 16);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        dst[e] = make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]),
+                                             __uint_as_float(v[4 * e + 2]), __uint_as_float(v[4 * e + 3]));
+                }
+            }
+            m_sm[m_row] = m_ref;
+            l_sm[m_row] = l_sum;
+            asm volatile("bar.sync 1, 128;" ::: "memory");          // the four softmax warps
+        }
+        {
+            // thread -> (query row, slice of the 128 output dims)
+            const int t = quarter * 32 + lane;
+            const int orow_idx = t % RPC, dpart = t / RPC;
+            constexpr int DLEN = kHeadDim / COPIES;
+            const int d0 = dpart * DLEN;
+            float acc[DLEN];
+            if (COPIES == 1) {                                       // the thread's own O row, read by the whole warp
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    uint32_t v[16];
+                    if (n_tiles > 0 && live_warp && alive) tc_ld16(tmem_o + lane_base + c * 16, v);
+#pragma unroll
+                    for (int e = 0; e < 16; ++e)
+                        acc[(c * 16 + e) % DLEN] = (n_tiles > 0 && live_warp && alive) ? __uint_as_float(v[e]) : 0.f;
+                }
+            }
+            if (orow_idx < p.R && alive) {
+                float mx = -CUDART_INF_F, den = 0.f;
+                if (COPIES == 1) {
+                    mx = m_ref;
+                    den = l_sum;
+                } else {
+                    float mw[COPIES], wt[COPIES];
+#pragma unroll
+                    for (int c = 0; c < COPIES; ++c) {
+                        mw[c] = m_sm[c * RPC + orow_idx];
+                        mx = fmaxf(mx, mw[c]);
+                    }
+#pragma unroll
+                    for (int c = 0; c < COPIES; ++c) {
+                        wt[c] = mx == -CUDART_INF_F ? 0.f : fast_exp2(mw[c] - mx);
+                        den += wt[c] * l_sm[c * RPC + orow_idx];
+                    }
+#pragma unroll
+                    for (int e = 0; e < DLEN; ++e) acc[e] = 0.f;
+                    if (n_tiles > 0) {
+#pragma unroll
+                        for (int c = 0; c < COPIES; ++c) {
+                            if (wt[c] == 0.f) continue;                  // a copy that saw no key holds no O row
+                            const float4 *src = reinterpret_cast<const float4 *>(o_sm + (c * RPC + orow_idx) * 132 + d0);
+#pragma unroll
+                            for (int e = 0; e < DLEN / 4; ++e) {
+                                const float4 f = src[e];
+                                acc[4 * e] += wt[c] * f.x; acc[4 * e + 1] += wt[c] * f.y;
+                                acc[4 * e + 2] += wt[c] * f.z; acc[4 * e + 3] += wt[c] * f.w;
+                            }
+                        }
+                    }
+                }
+                const float inv = den > 0.f ? 1.f / den : 0.f;
+                const float lse2 = den > 0.f ? mx + log2f(den) : -CUDART_INF_F;
+                const int tq = orow_idx / p.G, a = h * p.G + orow_idx % p.G;
+                const long long orow = ((long long)b * p.T + tq) * p.Hq + a;
+                if (p.n_splits == 1) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(p.out + (orow * kHeadDim + d0) * 2);
+#pragma unroll
+                    for (int e = 0; e < DLEN / 8; ++e)
+                        dst[e] = make_uint4(pack_bf16x2(acc[8 * e] * inv, acc[8 * e + 1] * inv),
+                                            pack_bf16x2(acc[8 * e + 2] * inv, acc[8 * e + 3] * inv),
+                                            pack_bf16x2(acc[8 * e + 4] * inv, acc[8 * e + 5] * inv),
+                                            pack_bf16x2(acc[8 * e + 6] * inv, acc[8 * e + 7] * inv));
+                    if (p.lse && dpart == 0) p.lse[orow] = lse2 * kAtLn2;
+                } else {
+                    float4 *dst = reinterpret_cast<float4 *>(p.part_o + ((long long)blockIdx.x * p.R + orow_idx) * kHeadDim + d0);
+#pragma unroll
+                    for (int e = 0; e < DLEN / 4; ++e)
+                        dst[e] = make_float4(acc[4 * e] * inv, acc[4 * e + 1] * inv, acc[4 * e + 2] * inv, acc[4 * e + 3] * inv);
+                    if (dpart == 0) p.part_lse[(long long)blockIdx.x * p.R + orow_idx] = lse2;
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kAtTmemCols)
+                     : "memory");
+    }
+}
+
+// ---- host side -----------------------------------------------------------------------------------------
+
+size_t attn_tc_smem_bytes(int stages) { return 1024 + kAtQBytes + (size_t)stages * kAtStageBytes + 512; }
+
+int launch_attn_tc(const oasis_dims_t *dims, const void *q, int n_q_tokens, const void *hbm_pool,
+                   const int32_t *slot_tbl, const int32_t *blk_tbl, int n_cols, const int32_t *seq_len, float scale,
+                   void *out, float *lse, float *part_o, float *part_lse, int n_splits, int cols_per_split,
+                   int stages, int32_t *err_word, cudaStream_t st, const char *who)
+{
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return fail(OASIS_ERR_CUDA, "%s: cuTensorMapEncodeTiled is not available", who);
+    // The pool is seen as rows of 256 bytes, 32 per entry.  Its size is not an argument of the call:
+    // the extent only bounds the coordinates, and slot ids always stay inside the caller's pool.
+    // dims (innermost first): 64 elements of a row half | 8 rows of a row group | 4 KiB parts (K, V) of all entries |
+    // the two 64-dim halves of a row | the two 8-row groups of a part.  One box = one whole 8 KiB entry, landing as
+    // [group][half][part][8 rows][128 B], so that 8-row groups of consecutive blocks are uniformly 4096 bytes apart.
+    CUtensorMap tmap;
+    const cuuint64_t gdim[5] = {64, 8, (cuuint64_t)1 << 31, 2, 2};
+    const cuuint64_t gstride[4] = {256, 4096, 128, 2048};
+    const cuuint32_t box[5] = {64, 8, 2, 2, 2};
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    CUresult cr = encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(hbm_pool), gdim, gstride, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return fail(OASIS_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed (%d)", who, (int)cr);
+
+    AttnTcParams p;
+    p.q = (const uint8_t *)q; p.slot_tbl = slot_tbl; p.blk_tbl = blk_tbl; p.seq_len = seq_len;
+    p.out = (uint8_t *)out; p.lse = lse; p.part_o = part_o; p.part_lse = part_lse; p.err = err_word;
+    p.scale_log2 = scale * kAtLog2e;
+    p.T = n_q_tokens; p.Hq = dims->n_q_heads; p.Hkv = dims->n_kv_heads; p.G = p.Hq / p.Hkv;
+    p.n_cols = n_cols; p.R = n_q_tokens * p.G; p.n_splits = n_splits; p.cols_per_split = cols_per_split;
+    p.stages = stages;
+    const size_t smem = attn_tc_smem_bytes(stages);
+    const long long grid = (long long)dims->batch * dims->n_kv_heads * n_splits;
+    cudaError_t e;
+#define OASIS_ATTN_TC_LAUNCH(C)                                                                                        \
+    do {                                                                                                               \
+        e = cudaFuncSetAttribute(sparse_attn_tc_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);     \
+        if (e == cudaSuccess) sparse_attn_tc_kernel<C><<<(unsigned)grid, kAtThreads, smem, st>>>(tmap, p);             \
+    } while (0)
+    if (p.R <= 32) OASIS_ATTN_TC_LAUNCH(4);
+    else if (p.R <= 64) OASIS_ATTN_TC_LAUNCH(2);
+    else OASIS_ATTN_TC_LAUNCH(1);
+#undef OASIS_ATTN_TC_LAUNCH
+    if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "%s: shared memory %zu B: %s", who, smem, cudaGetErrorString(e));
+    return check_launch(who);
+}
+
+}  // namespace oasis

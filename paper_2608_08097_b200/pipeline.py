@@ -78,11 +78,16 @@ class DecodeLayer:
 
 class DecodeEngine:
     """Sequencing of one decode step across layers, after the paper's asynchronous prefetch
-    pipeline (Sec. 4.2.2): on the foreground stream each layer runs attention over the working
-    set that the previous step's prediction staged, then this step's prediction (summary
-    update for newly completed blocks, scoring with the draft queries, top-k); the transfer
-    of what was selected runs on a side stream and is awaited, per layer, only by the next
-    step's attention of that same layer.
+    pipeline (Sec. 4.2.2).  Three streams:
+      foreground  attention of every layer over the working set that the previous step's
+                  prediction staged;
+      prediction  summary update for newly completed blocks, scoring with the draft queries,
+                  top-k and (delta mode) the transfer plan -- the tables a layer's attention
+                  reads are only rewritten after that attention has finished;
+      transfer    the gather of what was selected, awaited, per layer, only by the next step's
+                  attention of that same layer.
+    A whole step can be captured into a CUDA graph (`capture_step`) and replayed, which removes
+    the host launch cost of its ~250 kernels.
 
     mode "fetch_all": every selected block is gathered each step (k + 2 requests per row).
     mode "delta": delta selection with capped eviction (Sec. 4.2.3) bounds the gather to
@@ -99,11 +104,11 @@ class DecodeEngine:
         self.kv = [None] * n_layers
         self.table = [None] * n_layers
         self.main = torch.cuda.Stream(device=self.device)
+        self.pred = torch.cuda.Stream(device=self.device)
         self.side = torch.cuda.Stream(device=self.device)
-        self.sel_done = [torch.cuda.Event() for _ in range(n_layers)]
-        self.stage_done = [torch.cuda.Event() for _ in range(n_layers)]
         self.launches = 0
         self.cap = cap
+        self.stage_done = [None] * n_layers          # event of the layer's latest transfer
         if mode == "delta":
             assert cap is not None and 0 <= cap <= k
             dev, rows = self.device, (batch, n_kv_heads)
@@ -120,56 +125,68 @@ class DecodeEngine:
     def blk_tbl(self, layer):
         return self.resident[layer] if self.mode == "delta" else self.layers[layer].sel
 
-    def _predict_and_transfer(self, l, q, first_block, n_new, max_new, n_full_next, seq_next, timers, plan=None):
-        L = self.layers[l]
-        ms = self.main
-        with torch.cuda.stream(ms):
+    @staticmethod
+    def _tick(timers, name, stream):
+        if timers is None or name not in timers:
+            return None
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record(stream)
+        return ev
+
+    @staticmethod
+    def _tock(timers, name, start, stream):
+        if start is None:
+            return
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record(stream)
+        timers[name].append((start, ev))
+
+    def _predict(self, l, q, first_block, n_new, max_new, n_full_next, seq_next, stamp, timers,
+                 attn_done=None, plan=None):
+        """Prediction chain of one layer on the prediction stream; returns the event after which
+        the layer's gather may start."""
+        L, ps = self.layers[l], self.pred
+        with torch.cuda.stream(ps):
             L.build_summaries(self.kv[l], self.table[l], first_block, n_new, max_new)
-            t0 = self._tick(timers, "score")
+            t0 = self._tick(timers, "score", ps)
             L.score(q, n_full_next)
-            self._tock(timers, "score", t0)
-            t0 = self._tick(timers, "select")
+            self._tock(timers, "score", t0, ps)
+            if attn_done is not None:
+                ps.wait_event(attn_done)            # sel / resident are read by this step's attention
+            t0 = self._tick(timers, "select", ps)
             L.select(n_full_next, seq_next, self.table[l])
-            self._tock(timers, "select", t0)
+            self._tock(timers, "select", t0, ps)
             self.launches += 3
             if self.mode == "delta":
                 plan_idx = self.plan_idx[l] if plan is None else plan[0]
                 plan_slots = self.plan_slots[l] if plan is None else plan[1]
                 oasis.plan_delta(L.dims, L.sel, self.k, self.table[l], self.resident[l], self.stamp[l],
-                                 L.cols, plan_idx.shape[-1] - 2, self._stamp_now, plan_idx, plan_slots, n_local=2)
+                                 L.cols, plan_idx.shape[-1] - 2, stamp, plan_idx, plan_slots, n_local=2)
                 self.launches += 1
-            self.sel_done[l].record(ms)
-        with torch.cuda.stream(self.side):
-            self.side.wait_event(self.sel_done[l])
-            t0 = self._tick(timers, "stage", self.side)
+            ev = torch.cuda.Event()
+            ev.record(ps)
+        return ev
+
+    def _transfer(self, l, ready, timers, plan=None):
+        L, ss = self.layers[l], self.side
+        with torch.cuda.stream(ss):
+            ss.wait_event(ready)
+            t0 = self._tick(timers, "stage", ss)
             if self.mode == "delta":
+                plan_idx = self.plan_idx[l] if plan is None else plan[0]
+                plan_slots = self.plan_slots[l] if plan is None else plan[1]
                 oasis.stage_blocks(self.kv[l], plan_idx, plan_slots, plan_idx.numel(), L.pool)
             else:
                 L.stage(self.kv[l])
-            self._tock(timers, "stage", t0, self.side)
+            self._tock(timers, "stage", t0, ss)
             self.launches += 1
-            self.stage_done[l].record(self.side)
-
-    @staticmethod
-    def _tick(timers, name, stream=None):
-        if timers is None or name not in timers:
-            return None
-        ev = torch.cuda.Event(enable_timing=True)
-        ev.record(stream if stream is not None else torch.cuda.current_stream())
-        return ev
-
-    @staticmethod
-    def _tock(timers, name, start, stream=None):
-        if start is None:
-            return
-        ev = torch.cuda.Event(enable_timing=True)
-        ev.record(stream if stream is not None else torch.cuda.current_stream())
-        timers[name].append((start, ev))
+            ev = torch.cuda.Event()
+            ev.record(ss)
+        self.stage_done[l] = ev
 
     def prime(self, q_list, n_full_next, seq_next, step_stamp=0):
         """Before the first step: build every summary and run one prediction + transfer per
         layer, as the step before the first one would have done."""
-        self._stamp_now = step_stamp
         B = self.layers[0].B
         zeros = torch.zeros(B, dtype=torch.int32, device=self.device)
         plan = None
@@ -178,12 +195,13 @@ class DecodeEngine:
             plan = (torch.empty(rows, dtype=torch.int64, device=self.device),
                     torch.empty(rows, dtype=torch.int32, device=self.device))
         for l in range(self.n_layers):
-            self._predict_and_transfer(l, q_list[l], zeros, n_full_next, self.layers[l].mb, n_full_next, seq_next,
-                                       None, plan)
+            ready = self._predict(l, q_list[l], zeros, n_full_next, self.layers[l].mb, n_full_next, seq_next,
+                                  step_stamp, None, plan=plan)
+            self._transfer(l, ready, None, plan=plan)
             if plan is not None:
                 self.side.synchronize()  # the shared priming plan is reused by the next layer
-        self.main.synchronize()
-        self.side.synchronize()
+        torch.cuda.synchronize(self.device)
+        self.stage_done = [None] * self.n_layers     # everything has completed
 
     def step(self, q_list, seq_len, first_block, n_new, n_full_next, seq_next, step_stamp=0,
              timers=None, q_host=None, out_host=None):
@@ -191,23 +209,61 @@ class DecodeEngine:
         prediction works on the next step's view (n_full_next, seq_next).  With q_host /
         out_host (pinned tensors per layer) the step's queries are copied in and its outputs
         copied out inside the step (end-to-end mode)."""
-        self._stamp_now = step_stamp
         ms = self.main
         for l in range(self.n_layers):
             L = self.layers[l]
             with torch.cuda.stream(ms):
+                q_ready = None
                 if q_host is not None:
                     q_list[l].copy_(q_host[l], non_blocking=True)
-                ms.wait_event(self.stage_done[l])
-                t0 = self._tick(timers, "attn")
+                    q_ready = torch.cuda.Event()
+                    q_ready.record(ms)
+                if self.stage_done[l] is not None:
+                    ms.wait_event(self.stage_done[l])
+                t0 = self._tick(timers, "attn", ms)
                 L.attend(q_list[l], seq_len, blk_tbl=self.blk_tbl(l))
-                self._tock(timers, "attn", t0)
+                self._tock(timers, "attn", t0, ms)
                 self.launches += 2 if self._splits else 1
+                attn_done = torch.cuda.Event()
+                attn_done.record(ms)
                 if out_host is not None:
                     out_host[l].copy_(L.out, non_blocking=True)
-            self._predict_and_transfer(l, q_list[l], first_block, n_new, 1, n_full_next, seq_next, timers)
+            if q_ready is not None:
+                self.pred.wait_event(q_ready)
+            ready = self._predict(l, q_list[l], first_block, n_new, 1, n_full_next, seq_next, step_stamp, timers,
+                                  attn_done=attn_done)
+            self._transfer(l, ready, timers)
 
     def join(self):
-        """Makes the foreground stream wait for every transfer in flight."""
-        for l in range(self.n_layers):
-            self.main.wait_event(self.stage_done[l])
+        """Makes the foreground stream wait for everything the other streams have in flight."""
+        ev = torch.cuda.Event()
+        ev.record(self.pred)
+        self.main.wait_event(ev)
+        ev2 = torch.cuda.Event()
+        ev2.record(self.side)
+        self.main.wait_event(ev2)
+        self.stage_done = [None] * self.n_layers
+
+    def capture_step(self, *args, **kwargs):
+        """Captures one step (same arguments as `step`) into a CUDA graph on the foreground
+        stream and returns it; `graph.replay()` must be issued on that stream, and a replay
+        completes only when all three streams' work of the step has completed."""
+        torch.cuda.synchronize(self.device)
+        self.stage_done = [None] * self.n_layers
+        before = self.launches
+        g = torch.cuda.CUDAGraph()
+        fork = torch.cuda.Event()
+        with torch.cuda.graph(g, stream=self.main, capture_error_mode="thread_local"):
+            fork.record(self.main)
+            self.pred.wait_event(fork)
+            self.side.wait_event(fork)
+            self.step(*args, **kwargs)
+            self.join()
+        g.launches = self.launches - before
+        self.launches = before
+        return g
+
+    def replay(self, graph):
+        with torch.cuda.stream(self.main):
+            graph.replay()
+        self.launches += graph.launches

@@ -37,8 +37,9 @@ def oracle_prediction(oracle, lay, summ_cache, q_step, n_full, seq):
     return sel, idx, slots, s64
 
 
-@pytest.mark.parametrize("mode,cap", [("fetch_all", None), ("delta", 3), ("delta", 16)])
-def test_engine_steps_match_oracle(oracle, gpu, mode, cap):
+@pytest.mark.parametrize("mode,cap,graph", [("fetch_all", None, False), ("delta", 3, False), ("delta", 16, False),
+                                            ("fetch_all", None, True), ("delta", 3, True)])
+def test_engine_steps_match_oracle(oracle, gpu, mode, cap, graph):
     binding, pipeline = gpu
     dev = torch.device("cuda")
     n_layers, S = 3, 19
@@ -78,10 +79,15 @@ def test_engine_steps_match_oracle(oracle, gpu, mode, cap):
         oracle_transfer(l, sel, idx, slots, k, 0)
 
     for s in range(S):
-        eng.step([q_dev[l][s] for l in range(n_layers)], to_dev(seq[s]), to_dev(seq[s] // 16),
-                 to_dev((seq[s] + 1) // 16 - seq[s] // 16), to_dev((seq[s] + 1) // 16), to_dev(seq[s] + 1),
-                 step_stamp=s + 1)
-        eng.join()
+        args = ([q_dev[l][s] for l in range(n_layers)], to_dev(seq[s]), to_dev(seq[s] // 16),
+                to_dev((seq[s] + 1) // 16 - seq[s] // 16), to_dev((seq[s] + 1) // 16), to_dev(seq[s] + 1))
+        if graph:                                    # the step captured into a CUDA graph and replayed
+            keep = args
+            g = eng.capture_step(*args, step_stamp=s + 1)
+            eng.replay(g)
+        else:
+            eng.step(*args, step_stamp=s + 1)
+            eng.join()
         torch.cuda.synchronize()
         for l in range(n_layers):
             # attention of this step ran over the working set predicted one step earlier
