@@ -122,11 +122,14 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
-template <int COPIES>
+// MMA_M = 64 halves the tensor work when the query rows fit; its rows live in tensor-memory lanes
+// (m % 16) + 32 * (m / 16), i.e. sixteen per softmax warp.
+template <int MMA_M, int COPIES>
 __global__ void __launch_bounds__(kAtThreads, 1)
 sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcParams p)
 {
-    constexpr int RPC = 128 / COPIES;                       // MMA rows per copy of the query rows
+    constexpr int RPC = MMA_M / COPIES;                     // MMA rows per copy of the query rows
+    constexpr int LANES = MMA_M / 4;                        // lanes of each softmax warp that hold an MMA row
     constexpr int BPC = kAtTileCols / COPIES;               // blocks of a tile each copy handles
     constexpr int KPC = BPC * kBlock;                       // keys of a tile each copy handles
     extern __shared__ uint8_t smem_raw[];
@@ -174,12 +177,12 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
     if (warp >= 2) {
         // every softmax thread owns one MMA row: it loads that row of Q (rows are replicated across the copies,
         // rows past R are zero) and stores it to its tensor-memory lane
-        const int m_row = (warp & 3) * 32 + lane;
+        const int m_row = (warp & 3) * LANES + lane;
         const int r = m_row % RPC;
         uint4 v[16];
 #pragma unroll
         for (int c = 0; c < 16; ++c) v[c] = make_uint4(0, 0, 0, 0);
-        if (r < p.R) {
+        if (lane < LANES && r < p.R) {
             const int tq = r / p.G, a = h * p.G + r % p.G;
             const uint4 *src = reinterpret_cast<const uint4 *>(p.q + ((((long long)b * p.T + tq) * p.Hq + a) * kHeadDim) * 2);
 #pragma unroll
@@ -246,8 +249,8 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0 && n_tiles > 0) {
-            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAtTileKeys >> 3) << 17) | (8u << 24);
-            const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(128 >> 3) << 17) | (8u << 24);
+            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAtTileKeys >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
+            const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
             bool alive = true;
             // descriptors: the operand start address occupies the low 14 bits (16-byte units), so offsets are added there
             const uint64_t k_desc0 = smem_desc_sw128_k(kv_u32, kImgGroup);
@@ -302,10 +305,11 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
     } else {
         // ---------------------------------------------------------------- softmax, one thread per MMA row
         const int quarter = warp & 3;
-        const int m_row = quarter * 32 + lane;                      // MMA row = tensor-memory lane
+        const int m_row = quarter * LANES + (lane % LANES);         // MMA row held by this tensor-memory lane
         const int copy = m_row / RPC, row = m_row % RPC;            // which copy of the rows, which query row
-        const bool live_row = row < p.R;
-        const bool live_warp = (quarter * 32) % RPC < p.R;          // some lane of this warp holds a query row
+        const bool has_row = lane < LANES;
+        const bool live_row = has_row && row < p.R;
+        const bool live_warp = (quarter * LANES) % RPC < p.R;       // some lane of this warp holds a query row
         const int limit = live_row ? L + row / p.G : -1;            // last visible position of this row
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         float m_ref = -CUDART_INF_F, l_sum = 0.f;
@@ -426,17 +430,21 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
                     float4 *dst = reinterpret_cast<float4 *>(o_sm + m_row * 132 + c * 16);
 #pragma unroll
                     for (int e = 0; e < 4; ++e)
-                        dst[e] = make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]),
+                        if (has_row) dst[e] = make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]),
                                              __uint_as_float(v[4 * e + 2]), __uint_as_float(v[4 * e + 3]));
                 }
             }
-            m_sm[m_row] = m_ref;
-            l_sm[m_row] = l_sum;
+            if (has_row) {
+                m_sm[m_row] = m_ref;
+                l_sm[m_row] = l_sum;
+            }
             asm volatile("bar.sync 1, 128;" ::: "memory");          // the four softmax warps
         }
         {
             // thread -> (query row, slice of the 128 output dims)
-            const int t = quarter * 32 + lane;
+            // one copy: the thread that holds a row writes it; several copies: the MMA_M (row, slice) tasks go to
+            // the first MMA_M softmax threads
+            const int t = COPIES == 1 ? (has_row ? m_row : MMA_M) : quarter * 32 + lane;
             const int orow_idx = t % RPC, dpart = t / RPC;
             constexpr int DLEN = kHeadDim / COPIES;
             const int d0 = dpart * DLEN;
@@ -451,7 +459,7 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
                         acc[(c * 16 + e) % DLEN] = (n_tiles > 0 && live_warp && alive) ? __uint_as_float(v[e]) : 0.f;
                 }
             }
-            if (orow_idx < p.R && alive) {
+            if (t < MMA_M && orow_idx < p.R && alive) {
                 float mx = -CUDART_INF_F, den = 0.f;
                 if (COPIES == 1) {
                     mx = m_ref;
@@ -553,14 +561,15 @@ int launch_attn_tc(const oasis_dims_t *dims, const void *q, int n_q_tokens, cons
     const size_t smem = attn_tc_smem_bytes(stages);
     const long long grid = (long long)dims->batch * dims->n_kv_heads * n_splits;
     cudaError_t e;
-#define OASIS_ATTN_TC_LAUNCH(C)                                                                                        \
+#define OASIS_ATTN_TC_LAUNCH(M, C)                                                                                     \
     do {                                                                                                               \
-        e = cudaFuncSetAttribute(sparse_attn_tc_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);     \
-        if (e == cudaSuccess) sparse_attn_tc_kernel<C><<<(unsigned)grid, kAtThreads, smem, st>>>(tmap, p);             \
+        e = cudaFuncSetAttribute(sparse_attn_tc_kernel<M, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
+        if (e == cudaSuccess) sparse_attn_tc_kernel<M, C><<<(unsigned)grid, kAtThreads, smem, st>>>(tmap, p);          \
     } while (0)
-    if (p.R <= 32) OASIS_ATTN_TC_LAUNCH(4);
-    else if (p.R <= 64) OASIS_ATTN_TC_LAUNCH(2);
-    else OASIS_ATTN_TC_LAUNCH(1);
+    if (p.R <= 16) OASIS_ATTN_TC_LAUNCH(64, 4);          // four copies of <= 16 rows, one block of a tile each
+    else if (p.R <= 32) OASIS_ATTN_TC_LAUNCH(64, 2);     // two copies of <= 32 rows, two blocks each
+    else if (p.R <= 64) OASIS_ATTN_TC_LAUNCH(64, 1);
+    else OASIS_ATTN_TC_LAUNCH(128, 1);
 #undef OASIS_ATTN_TC_LAUNCH
     if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "%s: shared memory %zu B: %s", who, smem, cudaGetErrorString(e));
     return check_launch(who);

@@ -180,7 +180,47 @@ select_topk_kernel(const SelectParams p)
     __syncthreads();
 
     // ---- 4. bitonic sort, descending ------------------------------------------------------------
-    if (k_eff > 1) {
+    if (k_eff > 1 && p.sort_len <= 128) {
+        // up to 128 winners: one warp sorts them in registers (element e = 32 * j + lane), exchanging
+        // across lanes with shuffles -- no CTA-wide barrier per stage
+        if (warp == 0) {
+            unsigned long long v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[j] = (32 * j + lane < p.sort_len) ? cand[32 * j + lane] : 0ull;
+#pragma unroll
+            for (int size = 2; size <= 128; size <<= 1) {
+#pragma unroll
+                for (int stride = size >> 1; stride > 0; stride >>= 1) {
+                    if (stride >= 32) {                       // partner lives in the same lane
+                        const int dj = stride >> 5;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            if ((j & dj) == 0) {
+                                const int e = 32 * j + lane;
+                                const bool descending = (e & size) == 0;
+                                const unsigned long long x = v[j], y = v[j | dj];
+                                if ((x < y) == descending) { v[j] = y; v[j | dj] = x; }
+                            }
+                        }
+                    } else {                                   // partner lives in lane ^ stride
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int e = 32 * j + lane;
+                            const unsigned long long other = __shfl_xor_sync(0xffffffffu, v[j], stride);
+                            const bool lower = (lane & stride) == 0;          // this lane holds the pair's first element
+                            const bool descending = (e & size) == 0;
+                            const bool keep_max = lower == descending;
+                            v[j] = keep_max ? (v[j] > other ? v[j] : other) : (v[j] < other ? v[j] : other);
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (32 * j + lane < p.sort_len) cand[32 * j + lane] = v[j];
+        }
+        __syncthreads();
+    } else if (k_eff > 1) {
         const int len = p.sort_len;
         for (int size = 2; size <= len; size <<= 1) {
             for (int stride = size >> 1; stride > 0; stride >>= 1) {
@@ -251,7 +291,7 @@ extern "C" int oasis_select_topk(const oasis_dims_t *dims, const float *scores,
     while (sort_len < k) sort_len <<= 1;
     p.sort_len = sort_len;
     int threads = 128;
-    while (threads < 1024 && threads * 4 < dims->max_blocks) threads <<= 1;
+    while (threads < 1024 && threads * 16 < dims->max_blocks) threads <<= 1;   // ~16 keys per thread
     const size_t smem = (size_t)sort_len * 8 + (size_t)dims->max_blocks * 4;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -78,11 +78,11 @@ class DecodeLayer:
 
 class DecodeEngine:
     """Sequencing of one decode step across layers, after the paper's asynchronous prefetch
-    pipeline (Sec. 4.2.2).  Three streams:
+    pipeline (Sec. 4.2.2).  Four streams:
       foreground  attention of every layer over the working set that the previous step's
                   prediction staged;
-      prediction  summary update for newly completed blocks, scoring with the draft queries,
-                  top-k and (delta mode) the transfer plan -- the tables a layer's attention
+      prediction  summary update for newly completed blocks and scoring with the draft queries;
+      selection   top-k and (delta mode) the transfer plan -- the tables a layer's attention
                   reads are only rewritten after that attention has finished;
       transfer    the gather of what was selected, awaited, per layer, only by the next step's
                   attention of that same layer.
@@ -105,6 +105,7 @@ class DecodeEngine:
         self.table = [None] * n_layers
         self.main = torch.cuda.Stream(device=self.device)
         self.pred = torch.cuda.Stream(device=self.device)
+        self.selq = torch.cuda.Stream(device=self.device)
         self.side = torch.cuda.Stream(device=self.device)
         self.launches = 0
         self.cap = cap
@@ -145,17 +146,23 @@ class DecodeEngine:
                  attn_done=None, plan=None):
         """Prediction chain of one layer on the prediction stream; returns the event after which
         the layer's gather may start."""
-        L, ps = self.layers[l], self.pred
+        L, ps, qs = self.layers[l], self.pred, self.selq
         with torch.cuda.stream(ps):
             L.build_summaries(self.kv[l], self.table[l], first_block, n_new, max_new)
             t0 = self._tick(timers, "score", ps)
             L.score(q, n_full_next)
             self._tock(timers, "score", t0, ps)
+            scored = torch.cuda.Event()
+            scored.record(ps)
+        # top-k and the transfer plan run on their own stream, so that waiting for this layer's attention does
+        # not hold back the next layer's scoring
+        with torch.cuda.stream(qs):
+            qs.wait_event(scored)
             if attn_done is not None:
-                ps.wait_event(attn_done)            # sel / resident are read by this step's attention
-            t0 = self._tick(timers, "select", ps)
+                qs.wait_event(attn_done)            # sel / resident are read by this step's attention
+            t0 = self._tick(timers, "select", qs)
             L.select(n_full_next, seq_next, self.table[l])
-            self._tock(timers, "select", t0, ps)
+            self._tock(timers, "select", t0, qs)
             self.launches += 3
             if self.mode == "delta":
                 plan_idx = self.plan_idx[l] if plan is None else plan[0]
@@ -164,7 +171,7 @@ class DecodeEngine:
                                  L.cols, plan_idx.shape[-1] - 2, stamp, plan_idx, plan_slots, n_local=2)
                 self.launches += 1
             ev = torch.cuda.Event()
-            ev.record(ps)
+            ev.record(qs)
         return ev
 
     def _transfer(self, l, ready, timers, plan=None):
@@ -236,12 +243,10 @@ class DecodeEngine:
 
     def join(self):
         """Makes the foreground stream wait for everything the other streams have in flight."""
-        ev = torch.cuda.Event()
-        ev.record(self.pred)
-        self.main.wait_event(ev)
-        ev2 = torch.cuda.Event()
-        ev2.record(self.side)
-        self.main.wait_event(ev2)
+        for st in (self.pred, self.selq, self.side):
+            ev = torch.cuda.Event()
+            ev.record(st)
+            self.main.wait_event(ev)
         self.stage_done = [None] * self.n_layers
 
     def capture_step(self, *args, **kwargs):
@@ -256,6 +261,7 @@ class DecodeEngine:
         with torch.cuda.graph(g, stream=self.main, capture_error_mode="thread_local"):
             fork.record(self.main)
             self.pred.wait_event(fork)
+            self.selq.wait_event(fork)
             self.side.wait_event(fork)
             self.step(*args, **kwargs)
             self.join()
