@@ -212,6 +212,19 @@ int oasis_plan_delta(const oasis_dims_t *dims, const int32_t *sel, int32_t sel_c
                      int32_t *n_admitted, void *stream);
 
 /*
+ * Head-union block set (Sec. 4.4.1, partial transfer: per layer the per-head selected sets are
+ * united at block granularity -- a block is included if at least one KV head selected it -- and
+ * the index of every included block is sent with its data).
+ *   sel         [B][Hkv][sel_cols] int32; columns [0, k) of every head take part, negative = none
+ *   union_idx   [B][max_union] int32: the distinct block ids of request b in ascending order,
+ *               then -1; ids beyond max_union are dropped
+ *   n_union     [B] int32: size of the union (also when it exceeds max_union)
+ * 1 <= k <= sel_cols, max_union >= 1, max_blocks <= 1048576.
+ */
+int oasis_union_blocks(const oasis_dims_t *dims, const int32_t *sel, int32_t sel_cols, int32_t k,
+                       int32_t max_union, int32_t *union_idx, int32_t *n_union, void *stream);
+
+/*
  * Registers a device word (int32, zero-initialised by the caller, or NULL to unregister) in
  * which kernels record a non-zero code if one of their internal waits (on a shared-memory
  * barrier of an asynchronous copy or tensor-core operation) runs out of its iteration bound.

@@ -469,3 +469,35 @@ void oasis_oracle_plan_delta(int32_t B, int32_t Hkv, int32_t max_blocks, int32_t
     free(cand);
     free(target);
 }
+
+/* ---------------------------------------------------------------- head-union set
+ * Sec. 4.4.1 (partial transfer): per layer, the union over the KV heads of a request's
+ * selected sets at block granularity -- a block is included if at least one head selected
+ * it -- and the index of every included block travels with its data.
+ * For request b: the distinct ids among sel[b][h][0..k) over all h (negative = none), in
+ * ascending order, written to union_idx[b][0..n) and padded with -1 up to max_union;
+ * n_union[b] = n (the ids beyond max_union, if any, are dropped but still counted).
+ */
+void oasis_oracle_union_blocks(int32_t B, int32_t Hkv, int32_t max_blocks, int32_t sel_cols,
+                               int32_t k, const int32_t *sel, int32_t max_union,
+                               int32_t *union_idx, int32_t *n_union)
+{
+    uint8_t *seen = (uint8_t *)malloc((size_t)(max_blocks > 0 ? max_blocks : 1));
+    for (int32_t b = 0; b < B; ++b) {
+        memset(seen, 0, (size_t)(max_blocks > 0 ? max_blocks : 1));
+        for (int32_t h = 0; h < Hkv; ++h)
+            for (int32_t r = 0; r < k; ++r) {
+                int32_t j = sel[((int64_t)b * Hkv + h) * sel_cols + r];
+                if (j >= 0 && j < max_blocks) seen[j] = 1;
+            }
+        int32_t n = 0;
+        for (int32_t j = 0; j < max_blocks; ++j) {
+            if (!seen[j]) continue;
+            if (n < max_union) union_idx[(int64_t)b * max_union + n] = j;
+            ++n;
+        }
+        for (int32_t i = n; i < max_union; ++i) union_idx[(int64_t)b * max_union + i] = -1;
+        n_union[b] = n;
+    }
+    free(seen);
+}

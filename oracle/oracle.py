@@ -150,3 +150,13 @@ def plan_delta(sel, block_table, resident, stamp, k, cap, step, slot_stride, n_r
                                   _p(block_table), _p(resident), _p(stamp), _p(plan_idx),
                                   _p(plan_slots), _p(n_adm))
     return plan_idx, plan_slots, n_adm
+
+
+def union_blocks(sel, k, max_blocks, max_union):
+    """sel [B][Hkv][cols] -> (union_idx [B][max_union] ascending, -1 padded; n_union [B])."""
+    sel = _i32(sel)
+    B, Hkv, cols = sel.shape
+    idx = np.empty((B, max_union), dtype=np.int32)
+    n = np.empty((B,), dtype=np.int32)
+    lib().oasis_oracle_union_blocks(B, Hkv, int(max_blocks), cols, int(k), _p(sel), int(max_union), _p(idx), _p(n))
+    return idx, n

@@ -20,7 +20,7 @@ ENTRY_BYTES = 8192
 SYMBOLS = ("oasis_build_summaries", "oasis_score_blocks", "oasis_select_topk",
            "oasis_stage_blocks", "oasis_sparse_attn", "oasis_attn_workspace_bytes",
            "oasis_plan_delta", "oasis_last_error", "oasis_version",
-           "oasis_sparse_attn_static_scratch", "oasis_static_scratch_bytes", "oasis_set_error_word")
+           "oasis_sparse_attn_static_scratch", "oasis_static_scratch_bytes", "oasis_set_error_word", "oasis_union_blocks")
 
 
 class OasisError(RuntimeError):
@@ -75,6 +75,8 @@ def lib():
         for name in ("oasis_build_summaries", "oasis_score_blocks", "oasis_select_topk",
                      "oasis_stage_blocks", "oasis_sparse_attn", "oasis_plan_delta"):
             getattr(L, name).restype = ctypes.c_int
+        L.oasis_union_blocks.argtypes = [dp, vp, i32, i32, i32, vp, vp, vp]
+        L.oasis_union_blocks.restype = ctypes.c_int
         L.oasis_set_error_word.argtypes = [vp]
         L.oasis_set_error_word.restype = ctypes.c_int
         L.oasis_last_error.restype = ctypes.c_char_p
@@ -87,7 +89,7 @@ def set_error_word(word):
     """Registers an int32 device tensor (one element, zero) that kernels flag on an internal
     wait time-out; None unregisters."""
     _check(lib().oasis_set_error_word(None if word is None else ctypes.c_void_p(word.data_ptr())),
-           "oasis_set_error_word")
+           "oasis_set_error_word", "oasis_union_blocks")
 
 
 def last_error() -> str:
@@ -175,6 +177,15 @@ def sparse_attn(dims, q, n_q_tokens, hbm_pool, slot_tbl, blk_tbl, n_cols, seq_le
         _ptr(blk_tbl, torch.int32, "blk_tbl"), int(n_cols), _ptr(seq_len, torch.int32, "seq_len"),
         float(scale), _ptr(out, torch.bfloat16, "out"), _ptr(lse, torch.float32, "lse"),
         _ptr(workspace, None, "workspace"), ws_bytes, _stream(stream)), "oasis_sparse_attn")
+
+
+def union_blocks(dims, sel, k, union_idx, n_union, stream=None):
+    """union_idx [B][max_union] int32, n_union [B] int32: distinct selected blocks over all KV heads."""
+    d = dims.c()
+    _check(lib().oasis_union_blocks(
+        ctypes.byref(d), _ptr(sel, torch.int32, "sel"), int(sel.shape[-1]), int(k), int(union_idx.shape[-1]),
+        _ptr(union_idx, torch.int32, "union_idx"), _ptr(n_union, torch.int32, "n_union"), _stream(stream)),
+        "oasis_union_blocks")
 
 
 def static_scratch_bytes() -> int:

@@ -370,3 +370,25 @@ def test_plan_delta_matches_oracle_over_steps(oracle, gpu, cap_ratio):
                     if j >= 0:
                         src = int(lay.block_table[b, j]) * Hkv + h
                         assert np.array_equal(pool_np[(b * Hkv + h) * L.cols + c], kv_np[src])
+
+
+@pytest.mark.parametrize("nblk,k,Hkv", [(50, 9, 4), (2056, 128, 8), (8200, 512, 8), (40000, 64, 2)])
+def test_union_blocks_matches_oracle(oracle, gpu, nblk, k, Hkv):
+    """Head-union set of partial transfer: exact match with the oracle, also when the list is too short."""
+    binding, _ = gpu
+    dev = torch.device("cuda")
+    rng = np.random.default_rng(nblk + k)
+    B = 3
+    sel = np.stack([np.stack([rng.permutation(nblk)[:k] for _ in range(Hkv)]) for _ in range(B)]).astype(np.int32)
+    sel = np.concatenate([sel, np.full((B, Hkv, 2), 5, np.int32)], axis=2)
+    sel[1, 0, : k // 2] = -1
+    sel[2, :, :k] = sel[2, 0:1, :k]
+    dims = binding.Dims(B, Hkv, Hkv, nblk)
+    for max_union in (Hkv * k, max(1, k // 2)):
+        idx = torch.full((B, max_union), -7, dtype=torch.int32, device=dev)
+        n = torch.full((B,), -7, dtype=torch.int32, device=dev)
+        binding.union_blocks(dims, torch.from_numpy(sel).to(dev), k, idx, n)
+        torch.cuda.synchronize()
+        want_idx, want_n = oracle.union_blocks(sel, k, nblk, max_union)
+        assert np.array_equal(n.cpu().numpy(), want_n)
+        assert np.array_equal(idx.cpu().numpy(), want_idx)

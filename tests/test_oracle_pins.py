@@ -570,6 +570,23 @@ def test_plan_delta_invariants(oracle):
             assert np.array_equal(stp[0, h][untouched], before_stamp[0, h][untouched])
 
 
+def test_union_blocks_matches_numpy_unique(oracle):
+    rng = np.random.default_rng(27)
+    B, Hkv, k, nblk = 3, 4, 9, 50
+    sel = np.stack([np.stack([rng.permutation(nblk)[:k] for _ in range(Hkv)]) for _ in range(B)]).astype(np.int32)
+    sel = np.concatenate([sel, np.full((B, Hkv, 2), 7, np.int32)], axis=2)          # local columns are not part of it
+    sel[1, 2, 3:6] = -1                                                              # unused ranks
+    sel[2, :, :k] = sel[2, 0:1, :k]                                                  # all heads agree: the union is one set
+    idx, n = oracle.union_blocks(sel, k, nblk, Hkv * k)
+    for b in range(B):
+        want = np.unique(sel[b, :, :k][sel[b, :, :k] >= 0])
+        assert n[b] == len(want) and np.array_equal(idx[b, :n[b]], want) and (idx[b, n[b]:] == -1).all()
+    assert n[2] == k and k <= n[0] <= Hkv * k
+    # a list shorter than the union: truncated, but the count is the true size
+    idx2, n2 = oracle.union_blocks(sel, k, nblk, 5)
+    assert np.array_equal(idx2[0], idx[0, :5]) and n2[0] == n[0]
+
+
 def test_fetch_cap_reading_against_the_papers_table(oracle):
     """Table 'Fetch-cap ablation' (Sec. 5.5.1): GB per step, GB/s and tok/s per fetch ratio.
     With one committed token per request per step, requests = tok/s * (GB per step / GB/s).
