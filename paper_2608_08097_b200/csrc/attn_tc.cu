@@ -1,27 +1,30 @@
 // Step 4 on the 5th-generation tensor cores: sparse paged decode attention (Sec. 4.2.1, 4.3).
 //
 // Work item = (request, KV head, split of the column list).  All query rows that share the KV
-// head (G heads x T verify-step tokens, at most 128) form the M = 128 rows of every MMA, so each
-// staged K/V block is read from HBM once.  A tile is four columns = 64 keys (32 KiB of K and V).
+// head (G heads x T verify-step tokens, at most 128) are the M rows of every MMA (M = 64 when
+// they fit, else 128), so each staged K/V block is read from HBM once.  A tile is four columns
+// = 64 keys (32 KiB of K and V); one CTA per SM keeps a ring of seven such stages in flight.
 //
-//   warp 0     TMA producer: per block four 2-D tensor copies (16 rows x 128 B, 128-byte swizzle:
-//              the two 64-dim halves of its K rows and of its V rows) gathered by slot id into a
-//              ring of 32 KiB stages; completion on the stage's mbarrier.
-//   warp 1     one thread issues the MMAs: S = Q K^T (8 x tcgen05.mma 128x64x16, both operands in
-//              shared memory) into one of two S buffers in tensor memory, and O += P V
-//              (4 x tcgen05.mma 128x128x16, P read from tensor memory, V from shared memory in its
-//              natural key-major layout).  S of tile i+1 is issued before P V of tile i, so the
-//              softmax of tile i overlaps the next Q K^T.
+//   warp 0     TMA producer: one 5-D tensor copy per block brings its whole 8 KiB entry (gathered
+//              by slot id) as [row group][dim half][K, V][8 rows][128 B] with the 128-byte swizzle,
+//              so that the 8-row groups of consecutive blocks are uniformly 4 KiB apart and both
+//              the K operand (K-major) and the V operand (key-major) can be described to the MMA.
+//              Slot / block tables are read 32 columns at a time, one window ahead.
+//   warp 1     one thread issues the MMAs, event driven: S = Q K^T (8 x tcgen05.mma M x 64 x 16,
+//              Q read from tensor memory, K from shared memory) into one of four S buffers as soon
+//              as a tile has landed, and O += P V (4 x tcgen05.mma M x 128 x 16, P read from tensor
+//              memory, V from shared memory) as soon as the tile's P is written; the commit after
+//              P V releases the stage.
 //   warps 2-5  softmax, one thread per MMA row: tcgen05.ld of the row's logits, masking on local
 //              blocks only, exp2 against a running reference maximum that is raised lazily (only
 //              when a logit exceeds it by 2^8; the O row is then rescaled in tensor memory),
 //              running sum in a register, P rounded to bf16 and written back over S with
 //              tcgen05.st.  No cross-thread reduction exists anywhere in the softmax.
-//              A warp can only reach its own quarter of the 128 tensor-memory lanes, and a single
-//              warp's instruction rate bounds the softmax; so when the query rows fit in 32 (64)
-//              lanes they are replicated into all four (two) lane ranges, and each copy takes one
-//              (two) of the tile's four blocks, writing P = 0 for the others.  The copies' partial
-//              (max, sum, O) are merged through shared memory after the last tile.
+//              A warp only reaches its own quarter of the tensor-memory lanes and a single warp's
+//              instruction rate bounds the softmax, so when the query rows fit several times into
+//              the M rows they are replicated (2 or 4 copies) and each copy takes its share of the
+//              tile's four blocks, writing P = 0 for the others.  The copies' partial (max, sum, O)
+//              are merged through shared memory after the last tile.
 // After the merge the rows are normalised and written as bf16 (or, when the column list is
 // split, as a normalised partial plus its log-sum-exp to the workspace).
 // Every wait is bounded; a timeout records a code in the error word and the CTA winds down.
