@@ -10,12 +10,14 @@
 //              so that the 8-row groups of consecutive blocks are uniformly 4 KiB apart and both
 //              the K operand (K-major) and the V operand (key-major) can be described to the MMA.
 //              Slot / block tables are read 32 columns at a time, one window ahead.
-//   warp 1     one thread issues the MMAs, event driven: S = Q K^T (8 x tcgen05.mma M x 64 x 16,
-//              Q read from tensor memory, K from shared memory) into one of four S buffers as soon
-//              as a tile has landed, and O += P V (4 x tcgen05.mma M x 128 x 16, P read from tensor
-//              memory, V from shared memory) as soon as the tile's P is written; the commit after
-//              P V releases the stage.
-//   warps 2-5  softmax, one thread per MMA row: tcgen05.ld of the row's logits, masking on local
+//   warp 1     one thread issues S = Q K^T (8 x tcgen05.mma M x 64 x 16, Q read from tensor memory,
+//              K from shared memory) into one of four S buffers as soon as a tile has landed and
+//              the buffer's previous P V has completed.
+//   warp 2     one thread issues O += P V (4 x tcgen05.mma M x 128 x 16, P read from tensor memory,
+//              V from shared memory) as soon as the tile's P is written; the commit after P V
+//              releases the stage.  Issuing a tcgen05.mma costs its thread about 50-60 cycles,
+//              so two issuers halve the per-tile issue time, which otherwise bounds the loop.
+//   warps 3-6  softmax, one thread per MMA row: tcgen05.ld of the row's logits, masking on local
 //              blocks only, exp2 against a running reference maximum that is raised lazily (only
 //              when a logit exceeds it by 2^8; the O row is then rescaled in tensor memory),
 //              running sum in a register, P rounded to bf16 and written back over S with
@@ -39,7 +41,7 @@
 
 namespace oasis {
 
-constexpr int kAtThreads = 192;
+constexpr int kAtThreads = 224;                             // producer, Q K^T issuer, P V issuer, four softmax warps
 constexpr int kAtTileCols = 4;                              // blocks per tile
 constexpr int kAtTileKeys = kAtTileCols * kBlock;           // 64
 constexpr int kAtStageBytes = kAtTileCols * kEntryBytes;    // 32 KiB: one 8 KiB image per block
@@ -177,7 +179,7 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tmem_o = tmem_base + kAtSBufs * kAtTileKeys;
     const uint32_t tmem_q = tmem_o + kHeadDim;                       // Q as the A operand: 128 rows x 64 packed columns
-    if (warp >= 2) {
+    if (warp >= 3) {
         // every softmax thread owns one MMA row: it loads that row of Q (rows are replicated across the copies,
         // rows past R are zero) and stores it to its tensor-memory lane
         const int m_row = (warp & 3) * LANES + lane;
@@ -217,7 +219,9 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
         };
         int cur_blk, cur_slot, nxt_blk = -1, nxt_slot = -1;
         load_window(c0, cur_blk, cur_slot);
-        for (int i = 0; i < n_tiles && alive; ++i) {
+        int s = 0;
+        uint32_t ph = 1;                                             // parity of the "empty" phase to wait for
+        for (int i = 0; i < n_tiles && alive; ++i, ph ^= (s + 1 == p.stages), s = (s + 1 == p.stages) ? 0 : s + 1) {
             if ((i & 7) == 0) {
                 if (i > 0) { cur_blk = nxt_blk; cur_slot = nxt_slot; }
                 load_window(c0 + (i + 8) * kAtTileCols, nxt_blk, nxt_slot);
@@ -226,8 +230,7 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
             int blk = __shfl_sync(0xffffffffu, cur_blk, src_lane);
             const int slot = __shfl_sync(0xffffffffu, cur_slot, src_lane);
             if (lane >= kAtTileCols) blk = -1;
-            const int s = i % p.stages;
-            if (lane == 0) alive = mbar_wait(bar_empty(s), ((i / p.stages) & 1) ^ 1, p.err, 41);
+            if (lane == 0) alive = mbar_wait(bar_empty(s), ph, p.err, 41);
             alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
             if (!alive) break;
             const unsigned valid = __ballot_sync(0xffffffffu, lane < kAtTileCols && blk >= 0);
@@ -250,59 +253,60 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
                 tma_load_5d(kv_u32 + s * kAtStageBytes + lane * kEntryBytes, &tmap, 0, 0, 2 * slot, 0, 0, bar_full(s));
         }
     } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0 && n_tiles > 0) {
+        // ---------------------------------------------------------------- Q K^T issuer
+        if (lane == 0) {
             const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAtTileKeys >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
-            const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
-            bool alive = true;
             // descriptors: the operand start address occupies the low 14 bits (16-byte units), so offsets are added there
             const uint64_t k_desc0 = smem_desc_sw128_k(kv_u32, kImgGroup);
+            bool alive = true;
+            int s = 0, sb = 0, s_old = 0;                            // stage and S buffer of tile i; stage of tile i - kAtSBufs
+            uint32_t ph = 0, ph_old = 0;
+            for (int i = 0; i < n_tiles && alive; ++i) {
+                // the S buffer also held P of tile i - kAtSBufs: its P V must have completed
+                if (i >= kAtSBufs) {
+                    alive = mbar_wait(bar_empty(s_old), ph_old, p.err, 51);
+                    ph_old ^= (s_old + 1 == p.stages);
+                    s_old = (s_old + 1 == p.stages) ? 0 : s_old + 1;
+                }
+                alive = alive && mbar_wait(bar_full(s), ph, p.err, 52);
+                if (!alive) break;
+                tc_fence_after();
+                const uint64_t k_desc = k_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(sb * kAtTileKeys);
+#pragma unroll
+                for (int kc = 0; kc < 2; ++kc)
+#pragma unroll
+                    for (int k4 = 0; k4 < 4; ++k4)
+                        tc_mma_bf16_ts(d_tmem, tmem_q + (kc * 4 + k4) * 8, k_desc + (uint64_t)((kc * kImgHalf + k4 * 32) >> 4),
+                                       idesc_qk, (kc | k4) ? 1u : 0u);
+                tc_commit(bar_s_full(sb));
+                ph ^= (s + 1 == p.stages);
+                s = (s + 1 == p.stages) ? 0 : s + 1;
+                sb = (sb + 1) & (kAtSBufs - 1);
+            }
+        }
+    } else if (warp == 2) {
+        // ---------------------------------------------------------------- P V issuer
+        if (lane == 0) {
+            const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
             const uint64_t v_desc0 = smem_desc_sw128_mn(kv_u32 + kImgPart, kImgHalf, kImgGroup);
-            // Event-driven issue: whichever of "next Q K^T" (its tile has landed and an S buffer is free) and
-            // "next P V" (its P has been written) is ready goes first, so a late tile never delays a P V and
-            // with it the release of a stage.
-            int qk_next = 0, pv_next = 0;
-            uint32_t idle = 0;
-            while (pv_next < n_tiles) {
-                bool progressed = false;
-                if (qk_next < n_tiles && qk_next < pv_next + kAtSBufs) {
-                    const int i = qk_next, s = i % p.stages;
-                    if (mbar_test(bar_full(s), (i / p.stages) & 1)) {
-                        tc_fence_after();
-                        const uint64_t k_desc = k_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
-                        const uint32_t d_tmem = tmem_base + (uint32_t)((i % kAtSBufs) * kAtTileKeys);
+            bool alive = true;
+            int s = 0, sb = 0;
+            uint32_t ph_p = 0;
+            for (int i = 0; i < n_tiles && alive; ++i) {
+                alive = mbar_wait(bar_p_full(sb), ph_p, p.err, 53);
+                if (!alive) break;
+                tc_fence_after();
+                const uint64_t v_desc = v_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
+                const uint32_t p_tmem = tmem_base + (uint32_t)(sb * kAtTileKeys);
 #pragma unroll
-                        for (int kc = 0; kc < 2; ++kc)
-#pragma unroll
-                            for (int k4 = 0; k4 < 4; ++k4)
-                                tc_mma_bf16_ts(d_tmem, tmem_q + (kc * 4 + k4) * 8,
-                                                   k_desc + (uint64_t)((kc * kImgHalf + k4 * 32) >> 4), idesc_qk,
-                                                   (kc | k4) ? 1u : 0u);
-                        tc_commit(bar_s_full(i % kAtSBufs));
-                        ++qk_next;
-                        progressed = true;
-                    }
-                }
-                if (pv_next < qk_next) {
-                    const int i = pv_next, s = i % p.stages;
-                    if (mbar_test(bar_p_full(i % kAtSBufs), (i / kAtSBufs) & 1)) {
-                        tc_fence_after();
-                        const uint64_t v_desc = v_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
-                        const uint32_t p_tmem = tmem_base + (uint32_t)((i % kAtSBufs) * kAtTileKeys);
-#pragma unroll
-                        for (int ks = 0; ks < kAtTileCols; ++ks)           // 16 keys per MMA = one block image
-                            tc_mma_bf16_ts(tmem_o, p_tmem + ks * 8, v_desc + (uint64_t)((ks * kEntryBytes) >> 4),
-                                               idesc_pv, (i | ks) ? 1u : 0u);
-                        tc_commit(bar_empty(s));         // stage free, and O complete up to this tile
-                        ++pv_next;
-                        progressed = true;
-                    }
-                }
-                if (progressed) idle = 0;
-                else if (++idle > kSpinLimit * 8u) {     // bounded: give up, flag, let the CTA wind down
-                    if (p.err) atomicCAS(p.err, 0, 53);
-                    break;
-                }
+                for (int ks = 0; ks < kAtTileCols; ++ks)               // 16 keys per MMA = one block image
+                    tc_mma_bf16_ts(tmem_o, p_tmem + ks * 8, v_desc + (uint64_t)((ks * kEntryBytes) >> 4), idesc_pv,
+                                   (i | ks) ? 1u : 0u);
+                tc_commit(bar_empty(s));                             // stage free, and O complete up to this tile
+                s = (s + 1 == p.stages) ? 0 : s + 1;
+                sb = (sb + 1) & (kAtSBufs - 1);
+                ph_p ^= (sb == 0);
             }
         }
     } else {
@@ -317,13 +321,14 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         float m_ref = -CUDART_INF_F, l_sum = 0.f;
         bool alive = true;
+        int s = 0, s_prev = 0;                                      // ring stage of tile i and of tile i - 1
+        uint32_t ph_prev = 0;                                       // parity of the "empty" phase that ends tile i - 1
         for (int i = 0; i < n_tiles && alive; ++i) {
             alive = mbar_wait(bar_s_full(i % kAtSBufs), (i / kAtSBufs) & 1, p.err, 61);
             if (!alive) break;
             tc_fence_after();
             const uint32_t s_tmem = tmem_base + lane_base + (uint32_t)((i % kAtSBufs) * kAtTileKeys);
             if (live_warp) {
-                const int s = i % p.stages;
                 int nvis[BPC];                                      // visible keys of each of this copy's blocks
                 bool masked = false;
 #pragma unroll
@@ -366,7 +371,7 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
                     // the O rows must be complete up to tile i-1 before they are rescaled
                     // (its stage is released by the commit that follows that P V; with at least four stages in the
                     // ring the phase parity of that barrier is unambiguous)
-                    if (i > 0) alive = mbar_wait(bar_empty((i - 1) % p.stages), ((i - 1) / p.stages) & 1, p.err, 62);
+                    if (i > 0) alive = mbar_wait(bar_empty(s_prev), ph_prev, p.err, 62);
                     tc_fence_after();
                     const float m_new = raise ? mxs : m_ref;
                     const float alpha = m_new == -CUDART_INF_F ? 1.f : fast_exp2(m_ref - m_new);
@@ -415,6 +420,9 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_p_full(i % kAtSBufs));
+            if (i > 0) ph_prev ^= (s_prev + 1 == p.stages);
+            s_prev = s;
+            s = (s + 1 == p.stages) ? 0 : s + 1;
         }
         // ---- epilogue: merge the copies, normalise, write out ----------------------------------------------
         if (alive && n_tiles > 0)
