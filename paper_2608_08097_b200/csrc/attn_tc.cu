@@ -167,45 +167,52 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
         for (int a = 0; a < kAtSBufs; ++a) { mbar_init(bar_s_full(a), 1); mbar_init(bar_p_full(a), 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)kAtTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_o = tmem_base + kAtSBufs * kAtTileKeys;
-    const uint32_t tmem_q = tmem_o + kHeadDim;                       // Q as the A operand: 128 rows x 64 packed columns
-    if (warp >= 3) {
-        // every softmax thread owns one MMA row: it loads that row of Q (rows are replicated across the copies,
-        // rows past R are zero) and stores it to its tensor-memory lane
-        const int m_row = (warp & 3) * LANES + lane;
-        const int r = m_row % RPC;
+    __syncthreads();                             // the barriers exist; the producer starts copying right away
+    uint32_t tmem_base = 0, tmem_o = 0, tmem_q = 0;
+    if (warp != 0) {
+        // Meanwhile: warp 1 allocates the tensor memory, and every softmax thread, owner of one MMA row, loads
+        // that row of Q (rows are replicated across the copies, rows past R are zero) and then stores it to its
+        // tensor-memory lane.
+        if (warp == 1) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)kAtTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
         uint4 v[16];
+        if (warp >= 3) {
+            const int m_row = (warp & 3) * LANES + lane;
+            const int r = m_row % RPC;
 #pragma unroll
-        for (int c = 0; c < 16; ++c) v[c] = make_uint4(0, 0, 0, 0);
-        if (lane < LANES && r < p.R) {
-            const int tq = r / p.G, a = h * p.G + r % p.G;
-            const uint4 *src = reinterpret_cast<const uint4 *>(p.q + ((((long long)b * p.T + tq) * p.Hq + a) * kHeadDim) * 2);
+            for (int c = 0; c < 16; ++c) v[c] = make_uint4(0, 0, 0, 0);
+            if (lane < LANES && r < p.R) {
+                const int tq = r / p.G, a = h * p.G + r % p.G;
+                const uint4 *src = reinterpret_cast<const uint4 *>(p.q + ((((long long)b * p.T + tq) * p.Hq + a) * kHeadDim) * 2);
 #pragma unroll
-            for (int c = 0; c < 16; ++c) v[c] = src[c];
+                for (int c = 0; c < 16; ++c) v[c] = src[c];
+            }
         }
-        const uint32_t q_lane = tmem_q + ((uint32_t)((warp & 3) * 32) << 16);
+        tc_fence_before();
+        asm volatile("bar.sync 2, %0;" ::"n"(kAtThreads - 32) : "memory");
+        tc_fence_after();
+        tmem_base = *tmem_slot;
+        tmem_o = tmem_base + kAtSBufs * kAtTileKeys;
+        tmem_q = tmem_o + kHeadDim;                                  // Q as the A operand: 128 rows x 64 packed columns
+        if (warp >= 3) {
+            const uint32_t q_lane = tmem_q + ((uint32_t)((warp & 3) * 32) << 16);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const uint32_t w[16] = {v[4 * c].x, v[4 * c].y, v[4 * c].z, v[4 * c].w, v[4 * c + 1].x, v[4 * c + 1].y,
-                                    v[4 * c + 1].z, v[4 * c + 1].w, v[4 * c + 2].x, v[4 * c + 2].y, v[4 * c + 2].z,
-                                    v[4 * c + 2].w, v[4 * c + 3].x, v[4 * c + 3].y, v[4 * c + 3].z, v[4 * c + 3].w};
-            tc_st16(q_lane + c * 16, w);
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t w[16] = {v[4 * c].x, v[4 * c].y, v[4 * c].z, v[4 * c].w, v[4 * c + 1].x, v[4 * c + 1].y,
+                                        v[4 * c + 1].z, v[4 * c + 1].w, v[4 * c + 2].x, v[4 * c + 2].y, v[4 * c + 2].z,
+                                        v[4 * c + 2].w, v[4 * c + 3].x, v[4 * c + 3].y, v[4 * c + 3].z, v[4 * c + 3].w};
+                tc_st16(q_lane + c * 16, w);
+            }
+            tc_wait_st();
         }
-        tc_wait_st();
+        tc_fence_before();
+        asm volatile("bar.sync 2, %0;" ::"n"(kAtThreads - 32) : "memory");
+        tc_fence_after();
     }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
 
     if (warp == 0) {
         // ---------------------------------------------------------------- producer

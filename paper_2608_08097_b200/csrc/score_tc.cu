@@ -132,20 +132,24 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)p.tmem_cols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    // The operand of the first (request, KV head) is built by the whole CTA while the barriers and
-    // the tensor memory are being set up.
+    __syncthreads();                             // the barriers exist; the producer starts copying right away
     const long long t_first = next_active(t0);
-    if (t_first < t1) build_b(t_first / p.tiles_per_bh, 0, tid, kTcThreads);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-    if (tid == 0 && t_first < t1) mbar_arrive(bar_b_full(0));
+    uint32_t tmem_base = 0;
+    if (warp != 0) {
+        // Meanwhile the other five warps allocate the tensor memory and build the operand of the first
+        // (request, KV head).
+        if (warp == 1) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)p.tmem_cols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
+        if (t_first < t1) build_b(t_first / p.tiles_per_bh, 0, tid - 32, kTcThreads - 32);
+        tc_fence_before();
+        asm volatile("bar.sync 1, %0;" ::"n"(kTcThreads - 32) : "memory");
+        tc_fence_after();
+        tmem_base = *tmem_slot;
+        if (tid == 32 && t_first < t1) mbar_arrive(bar_b_full(0));
+    }
 
     if (warp == 0) {
         // ---------------------------------------------------------------- producer
