@@ -27,6 +27,7 @@ stage_blocks_kernel(const uint8_t *__restrict__ host_kv, const long long *__rest
         uint4 v[16];
 #pragma unroll
         for (int c = 0; c < 16; ++c) v[c] = ld_stream_v4(src + c * 512);
+        asm volatile("" ::: "memory");          // keeps the stores behind all sixteen loads
 #pragma unroll
         for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4 *>(dst + c * 512) = v[c];
     }

@@ -86,6 +86,8 @@ class DecodeEngine:
                   reads are only rewritten after that attention has finished;
       transfer    the gather of what was selected, awaited, per layer, only by the next step's
                   attention of that same layer.
+    In end-to-end mode a fifth stream uploads the step's queries (all layers, before the first
+    gather) and downloads each layer's output.
     A whole step can be captured into a CUDA graph (`capture_step`) and replayed, which removes
     the host launch cost of its ~250 kernels.
 
@@ -107,6 +109,7 @@ class DecodeEngine:
         self.pred = torch.cuda.Stream(device=self.device)
         self.selq = torch.cuda.Stream(device=self.device)
         self.side = torch.cuda.Stream(device=self.device)
+        self.copy = torch.cuda.Stream(device=self.device)     # end-to-end mode: query upload, output download
         self.launches = 0
         self.cap = cap
         self.stage_done = [None] * n_layers          # event of the layer's latest transfer
@@ -216,15 +219,29 @@ class DecodeEngine:
         prediction works on the next step's view (n_full_next, seq_next).  With q_host /
         out_host (pinned tensors per layer) the step's queries are copied in and its outputs
         copied out inside the step (end-to-end mode)."""
-        ms = self.main
+        ms, cs = self.main, self.copy
+        q_ready = [None] * self.n_layers
+        if q_host is not None or out_host is not None:
+            # the copy stream starts after everything the previous step left on the other streams
+            for st in (ms, self.pred):
+                ev = torch.cuda.Event()
+                ev.record(st)
+                cs.wait_event(ev)
+        if q_host is not None:
+            # All of the step's queries cross the host link before its first gather: the zero-copy gathers keep
+            # thousands of reads in flight on the link and would starve DMA copies queued beside them, which
+            # would serialise gather(l) -> attention(l + 1).
+            with torch.cuda.stream(cs):
+                for l in range(self.n_layers):
+                    q_list[l].copy_(q_host[l], non_blocking=True)
+                    q_ready[l] = torch.cuda.Event()
+                    q_ready[l].record(cs)
+            self.side.wait_event(q_ready[-1])
         for l in range(self.n_layers):
             L = self.layers[l]
             with torch.cuda.stream(ms):
-                q_ready = None
-                if q_host is not None:
-                    q_list[l].copy_(q_host[l], non_blocking=True)
-                    q_ready = torch.cuda.Event()
-                    q_ready.record(ms)
+                if q_ready[l] is not None:
+                    ms.wait_event(q_ready[l])
                 if self.stage_done[l] is not None:
                     ms.wait_event(self.stage_done[l])
                 t0 = self._tick(timers, "attn", ms)
@@ -233,17 +250,23 @@ class DecodeEngine:
                 self.launches += 2 if self._splits else 1
                 attn_done = torch.cuda.Event()
                 attn_done.record(ms)
-                if out_host is not None:
+            if out_host is not None:
+                cs.wait_event(attn_done)
+                with torch.cuda.stream(cs):
                     out_host[l].copy_(L.out, non_blocking=True)
-            if q_ready is not None:
-                self.pred.wait_event(q_ready)
+            if q_ready[l] is not None:
+                self.pred.wait_event(q_ready[l])
             ready = self._predict(l, q_list[l], first_block, n_new, 1, n_full_next, seq_next, step_stamp, timers,
                                   attn_done=attn_done)
             self._transfer(l, ready, timers)
+        if out_host is not None:
+            ev = torch.cuda.Event()                  # the next step's attention overwrites the output buffers
+            ev.record(cs)
+            ms.wait_event(ev)
 
     def join(self):
         """Makes the foreground stream wait for everything the other streams have in flight."""
-        for st in (self.pred, self.selq, self.side):
+        for st in (self.pred, self.selq, self.side, self.copy):
             ev = torch.cuda.Event()
             ev.record(st)
             self.main.wait_event(ev)
@@ -252,7 +275,7 @@ class DecodeEngine:
     def capture_step(self, *args, **kwargs):
         """Captures one step (same arguments as `step`) into a CUDA graph on the foreground
         stream and returns it; `graph.replay()` must be issued on that stream, and a replay
-        completes only when all three streams' work of the step has completed."""
+        completes only when all streams' work of the step has completed."""
         torch.cuda.synchronize(self.device)
         self.stage_done = [None] * self.n_layers
         before = self.launches
@@ -263,6 +286,7 @@ class DecodeEngine:
             self.pred.wait_event(fork)
             self.selq.wait_event(fork)
             self.side.wait_event(fork)
+            self.copy.wait_event(fork)
             self.step(*args, **kwargs)
             self.join()
         g.launches = self.launches - before
