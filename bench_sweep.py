@@ -1,0 +1,203 @@
+"""Secondary measurements of the sparse-decode path on one B200 (not part of the `bench.py` contract).
+
+    python bench_sweep.py [--layers 8] [--steps 16] [--what ratio,c5,stage]
+
+Prints one JSON line per section:
+  ratio   configs[1] (reasoning-style decode) at several fetch ratios of the capped delta gather
+          (Sec. 5.5.1) plus the uncapped delta and fetch-all: step time with everything in HBM,
+          end-to-end step time with the KV pool in pinned host memory, the exposed transfer time,
+          admitted entries per (request, KV head) per step, and the break-even fetch fraction
+          rho* = link bandwidth x compute time / cold bytes.
+  c5      the budget x draft-length sweep (configs[4]): solo kernel times and roofline fractions of
+          scoring / top-k / attention, and lookahead recall per cell.
+  stage   the gather kernel alone on random entries of a pinned pool, against the DMA copy peak.
+Inputs are synthetic (the generators of `synth`); nothing here touches the CPU oracle.
+"""
+import argparse
+import json
+import math
+import os
+import sys
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import bench as B                                        # noqa: E402
+from paper_2608_08097_b200 import synth                  # noqa: E402
+
+
+def graph_time(fn, n_rot, iters=32, warm=4):
+    """Median of 5 graph replays of `iters` launches rotating over `n_rot` working sets (us per launch)."""
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        for i in range(warm):
+            fn(i % n_rot)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=st):
+        for i in range(iters):
+            fn(i % n_rot)
+    ts = []
+    for _ in range(5):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b) * 1e3 / iters)
+    ts.sort()
+    return ts[2]
+
+
+def section_ratio(args, dev, hbm_peak):
+    """Fetch-ratio sweep on the reasoning-style workload (fewer layers than the bench, same per-layer sizes)."""
+    W, K = 3, args.steps
+    cfg = synth.scaled(synth.C2, layers=args.layers, steps=W + K + 2)
+    ns = argparse.Namespace(seed=args.seed, skip_e2e=False, skip_cpu=True, fetch_ratio=0.05, layers=args.layers,
+                            batch=None, context=None, gpus=1, steps=K, warmup=W)
+    bench = B.Bench(ns, cfg, dev, 0)
+    h2d_peak = B.time_pinned_h2d(dev)
+    bench.generate(want_mirror=True, want_host=True)
+    q_pinned = [q.cpu().pin_memory() for q in bench.q_dev]
+    q_stage = [torch.empty_like(bench.q_dev[l][0]) for l in range(cfg.layers)]
+    out_pinned = [torch.empty((cfg.batch, cfg.n_q_tokens, cfg.n_q_heads, 128), dtype=torch.bfloat16, pin_memory=True)
+                  for _ in range(cfg.layers)]
+    kw = dict(q_pinned=q_pinned, out_pinned=out_pinned, q_stage=q_stage)
+    rows = cfg.batch * cfg.n_kv_heads
+    cold_bytes = rows * (cfg.k_blocks + 1) * 8192                       # per layer: every selected block + the local one
+    out = []
+    for ratio in (0.01, 0.02, 0.05, 0.10, 0.20, 1.0, None):              # 1.0: uncapped delta; None: fetch all
+        if ratio is None:
+            mode, cap, name = "fetch_all", None, "all"
+        else:
+            mode, cap, name = "delta", max(1, int(math.floor(ratio * cfg.k_blocks))), "%.2f" % ratio
+        eng = bench.engine(mode, bench.mirror, cap=cap)
+        ms_v, _, _ = bench.timed(eng, 1, W, K)
+        del eng
+        eng = bench.engine(mode, bench.host_kv, cap=cap)
+        ms_e, _, _ = bench.timed(eng, 1, W, K, e2e=True, **kw)
+        if mode == "delta":
+            adm = sum(int((p[..., :cap] >= 0).sum().item()) for p in eng.plan_idx) / (cfg.layers * rows)
+            loc = sum(int((p[..., cap:] >= 0).sum().item()) for p in eng.plan_idx) / (cfg.layers * rows)
+        else:
+            adm = sum(int((L.stage_idx[..., :cfg.k_blocks] >= 0).sum().item()) for L in eng.layers) / (cfg.layers * rows)
+            loc = sum(int((L.stage_idx[..., cfg.k_blocks:] >= 0).sum().item()) for L in eng.layers) / (cfg.layers * rows)
+        del eng
+        bytes_layer = rows * (adm + loc) * 8192
+        out.append({
+            "fetch_ratio": name, "cap_blocks": cap,
+            "value_us_per_layer": round(ms_v * 1e3 / cfg.layers, 1),
+            "e2e_us_per_layer": round(ms_e * 1e3 / cfg.layers, 1),
+            "exposed_us_per_layer": round((ms_e - ms_v) * 1e3 / cfg.layers, 1),
+            "tokens_per_s_per_layer_value": round(cfg.batch * cfg.layers / (ms_v * 1e-3), 1),
+            "tokens_per_s_per_layer_e2e": round(cfg.batch * cfg.layers / (ms_e * 1e-3), 1),
+            "admitted_per_row_last_step": round(adm, 2), "local_per_row": round(loc, 2),
+            "fetched_fraction_of_budget": round(adm / cfg.k_blocks, 4),
+            "staged_MB_per_layer": round(bytes_layer / 1e6, 2),
+            "staged_GBps_over_e2e_step": round(bytes_layer / (ms_e * 1e-3 / cfg.layers) / 1e9, 2),
+        })
+    t_compute = out[2]["value_us_per_layer"] * 1e-6                      # the default operating point
+    link = 0.91 * h2d_peak * 1e9                                         # what the zero-copy gather reaches alone
+    print(json.dumps({"section": "ratio", "workload": "configs[1], %d layers, %d timed steps" % (cfg.layers, K),
+                      "pinned_h2d_peak_GBps": round(h2d_peak, 2), "cold_MB_per_layer": round(cold_bytes / 1e6, 1),
+                      "break_even_fetch_fraction": round(link * t_compute / cold_bytes, 4),
+                      "break_even_note": "rho* = 0.91 x pinned peak x value-mode time per layer / cold bytes per layer",
+                      "rows": out}))
+
+
+def section_c5(args, dev, hbm_peak):
+    """Budget x draft-length sweep: kernels alone (graph replay over rotating working sets) and recall."""
+    from paper_2608_08097_b200 import pipeline
+    base = synth.scaled(synth.C5, n_draft=8, layers=1, steps=1)
+    lay = synth.make_layer(base, seed=args.seed, layer=0, device=dev)
+    kv = lay.host_kv.to(dev)
+    table, n_full, seq = lay.block_table.to(dev), lay.n_full.to(dev), lay.seq_len.to(dev)
+    Bq, Hq, Hkv, mb = base.batch, base.n_q_heads, base.n_kv_heads, base.max_blocks
+    zeros = torch.zeros(Bq, dtype=torch.int32, device=dev)
+    nf = int(lay.n_full[0])
+    n_rot = 3                                                            # 3 x 268 MB of summaries > 2 x L2
+    cells = []
+    for K in (32, 64, 128, 256, 512):
+        for Td in (1, 2, 4, 8):
+            T = Td + 1
+            Ls = [pipeline.DecodeLayer(Bq, Hq, Hkv, mb, K, T, dev) for _ in range(n_rot)]
+            q = lay.q[:, :T].contiguous().to(dev)
+            q_true = lay.q_true[:, :Td].contiguous().to(dev)
+            for L in Ls:
+                L.build_summaries(kv, table, zeros, n_full, mb)
+                L.score(q, n_full)
+                L.select(n_full, seq, table)
+                L.stage(kv)
+            torch.cuda.synchronize()
+            t_score = graph_time(lambda i: Ls[i].score(q, n_full), n_rot)
+            t_sel = graph_time(lambda i: Ls[i].select(n_full, seq, table), n_rot)
+            t_attn = graph_time(lambda i: Ls[i].attend(q, seq), n_rot)
+            sel_draft = Ls[0].sel.clone()
+            sel_true = torch.empty_like(sel_draft)
+            Ls[0].score_queries(q_true, n_full)
+            Ls[0].select(n_full, seq, table, sel=sel_true)
+            torch.cuda.synchronize()
+            a, b = sel_draft[..., :K], sel_true[..., :K]
+            recall = (a[..., :, None] == b[..., None, :]).any(-1).float().mean().item()
+            sb = Bq * Hkv * nf * 516
+            ab = Bq * Hkv * (min(K, nf) + 1) * 8192 + 2 * Bq * T * Hq * 256
+            cells.append({"K": K, "Td": Td, "score_us": round(t_score, 1), "score_frac": round(sb / t_score / 1e3 / hbm_peak, 3),
+                          "select_us": round(t_sel, 1), "attn_us": round(t_attn, 1),
+                          "attn_frac": round(ab / t_attn / 1e3 / hbm_peak, 3),
+                          "tokens_per_s_per_layer": round(Bq / ((t_score + t_sel + t_attn) * 1e-6), 1),
+                          "recall": round(recall, 4)})
+            del Ls
+            torch.cuda.empty_cache()
+    print(json.dumps({"section": "c5", "workload": "configs[4]: batch 16, 32q/8kv heads, context 65536, one layer "
+                      "(3 rotating copies of the summaries and pools), kernels alone; frac = algorithmic bytes / time / "
+                      "measured copy peak; tokens/s/layer from the serial sum score + top-k + attention",
+                      "hbm_peak_GBps": hbm_peak, "cells": cells}))
+
+
+def section_stage(args, dev, hbm_peak):
+    """The gather kernel alone: random 8 KiB entries of a 2 GiB pinned pool into HBM slots."""
+    from paper_2608_08097_b200 import binding as oasis
+    h2d_peak = B.time_pinned_h2d(dev)
+    P = 262144
+    host = torch.empty((P, 2, 16, 128), dtype=torch.bfloat16, pin_memory=True)
+    host.view(torch.int16).random_(0, 1000)
+    pool = torch.zeros((20000, 2, 16, 128), dtype=torch.bfloat16, device=dev)
+    g = torch.Generator()
+    g.manual_seed(args.seed)
+    rows = []
+    for n, pad in ((896, 1024), (4096, 4096), (16640, 16640)):
+        idxs, slots = [], []
+        for _ in range(8):
+            idx = torch.full((pad,), -1, dtype=torch.int64)
+            idx[torch.randperm(pad, generator=g)[:n]] = torch.randint(0, P, (n,), generator=g)
+            idxs.append(idx.to(dev))
+            slots.append(torch.arange(pad, dtype=torch.int32, device=dev))
+        us = graph_time(lambda i: oasis.stage_blocks(host, idxs[i], slots[i], pad, pool), 8, iters=8, warm=8)
+        rows.append({"requests": n, "list_length": pad, "us": round(us, 1), "GBps": round(n * 8192 / us / 1e3, 2),
+                     "frac_of_h2d_peak": round(n * 8192 / us / 1e3 / h2d_peak, 3)})
+    print(json.dumps({"section": "stage", "pinned_h2d_peak_GBps": round(h2d_peak, 2), "rows": rows}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--layers", type=int, default=8)
+    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--what", default="ratio,c5,stage")
+    args = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench_sweep.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    from paper_2608_08097_b200 import build
+    build.build()
+    hbm_peak, _ = B.measured_peaks()
+    for what in args.what.split(","):
+        {"ratio": section_ratio, "c5": section_c5, "stage": section_stage}[what](args, dev, hbm_peak)
+        torch.cuda.empty_cache()
+
+
+if __name__ == "__main__":
+    main()

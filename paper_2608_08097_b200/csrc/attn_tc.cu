@@ -1,8 +1,8 @@
 // Step 4 on the 5th-generation tensor cores: sparse paged decode attention (Sec. 4.2.1, 4.3).
 //
 // Work item = (request, KV head, split of the column list).  All query rows that share the KV
-// head (G heads x T verify-step tokens, at most 128) are the M rows of every MMA (M = 64 when
-// they fit, else 128), so each staged K/V block is read from HBM once.  A tile is four columns
+// head (G heads x T verify-step tokens, at most 128) are the M rows of every MMA (M = 64 for up to
+// 32 rows, else 128), so each staged K/V block is read from HBM once.  A tile is four columns
 // = 64 keys (32 KiB of K and V); one CTA per SM keeps a ring of seven such stages in flight.
 //
 //   warp 0     TMA producer: one 5-D tensor copy per block brings its whole 8 KiB entry (gathered
@@ -586,7 +586,7 @@ int launch_attn_tc(const oasis_dims_t *dims, const void *q, int n_q_tokens, cons
     } while (0)
     if (p.R <= 16) OASIS_ATTN_TC_LAUNCH(64, 4);          // four copies of <= 16 rows, one block of a tile each
     else if (p.R <= 32) OASIS_ATTN_TC_LAUNCH(64, 2);     // two copies of <= 32 rows, two blocks each
-    else if (p.R <= 64) OASIS_ATTN_TC_LAUNCH(64, 1);
+    else if (p.R <= 64) OASIS_ATTN_TC_LAUNCH(128, 2);    // two copies of <= 64 rows: half the softmax work per thread
     else OASIS_ATTN_TC_LAUNCH(128, 1);
 #undef OASIS_ATTN_TC_LAUNCH
     if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "%s: shared memory %zu B: %s", who, smem, cudaGetErrorString(e));
