@@ -6,15 +6,18 @@
 //     D[128 blocks x N] = A[128 x 256] (summaries, [min | max], K-major)  x  B[256 x N] (q^- | q^+)
 // with N = R rounded up to 16, followed by a max (or sum) over the N columns of every row.
 //
-// A persistent CTA per SM walks a contiguous range of tiles with three warp roles:
+// A persistent CTA per SM walks a contiguous range of tiles with four warp roles:
 //   warp 0     TMA producer: four 2-D tensor copies (128 rows x 128 B, 128-byte swizzle) per tile
-//              into a ring of 64 KiB stages, completion on mbarriers; it also builds the
-//              (q^- | q^+) operand of every new (request, KV head) in the same swizzled layout.
+//              into a ring of 64 KiB stages, completion on mbarriers.  It starts right after the
+//              barrier set-up, while the other warps allocate the tensor memory and build the
+//              (q^- | q^+) operand of the first (request, KV head) in the same swizzled layout.
 //   warp 1     one thread issues 16 tcgen05.mma (128 x N x 16, bf16 -> fp32) per tile into one of
 //              two TMEM accumulators and commits to the stage's "empty" and the accumulator's
 //              "full" barrier.
 //   warps 2-5  epilogue: tcgen05.ld of the thread's TMEM lane (= one block), max / sum over its N
 //              columns, one coalesced fp32 store per block.
+//   warp 6     builds the (q^- | q^+) operand of every further (request, KV head) of the CTA's range
+//              ahead of time, into whichever of the two operand buffers is free.
 // Bytes in flight are bounded by shared memory (up to three 64 KiB stages per SM), not by
 // registers; the tensor work per tile is tiny, so the kernel is HBM bound.
 // Every wait is bounded: on a timeout the thread records a code in the error word (if one was
@@ -28,7 +31,7 @@
 
 namespace oasis {
 
-constexpr int kTcThreads = 192;
+constexpr int kTcThreads = 224;
 constexpr int kTileBlocks = 128;
 constexpr int kATileBytes = kTileBlocks * kSummaryBytes;   // 64 KiB
 constexpr int kSubTileBytes = kTileBlocks * 128;           // one 64-element K chunk of the tile: 16 KiB
@@ -153,7 +156,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
 
     if (warp == 0) {
         // ---------------------------------------------------------------- producer
-        int it = 0, bo = 0;
+        int it = 0;
         bool alive = true;
         long long t = t_first;
         while (t < t1 && alive) {
@@ -172,19 +175,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
             }
             alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
             ++it;
-            // one tile ahead: if the next tile belongs to another (request, KV head), build its operand now,
-            // while this tile's copies are in flight
             const long long tn = next_active(t + 1);
-            if (alive && tn < t1 && tn / p.tiles_per_bh != bh) {
-                ++bo;
-                const int buf = bo % p.n_bbuf;
-                alive = mbar_wait(bar_b_empty(buf), ((bo / p.n_bbuf) & 1) ^ 1, p.err, 11);
-                if (alive) {
-                    build_b(tn / p.tiles_per_bh, buf, lane, 32);
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_b_full(buf));
-                }
-            }
             t = tn;
         }
     } else if (warp == 1) {
@@ -228,6 +219,26 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
                 tc_commit(bar_acc_full(acc));    // the accumulator is complete
                 ++it;
             }
+        }
+    } else if (warp == 6) {
+        // ---------------------------------------------------------------- operand builder
+        // Walks the CTA's tiles ahead of everyone else and builds (q^- | q^+) of every further (request, KV head)
+        // as soon as an operand buffer is free, so neither the copies nor the MMAs ever wait for it.
+        int bo = 0;
+        bool alive = true;
+        long long cur_bh = t_first < t1 ? t_first / p.tiles_per_bh : -1;
+        for (long long t = t_first < t1 ? next_active(t_first + 1) : t1; t < t1 && alive; t = next_active(t + 1)) {
+            const long long bh = t / p.tiles_per_bh;
+            if (bh == cur_bh) continue;
+            cur_bh = bh;
+            ++bo;
+            const int buf = bo % p.n_bbuf;
+            if (lane == 0) alive = mbar_wait(bar_b_empty(buf), ((bo / p.n_bbuf) & 1) ^ 1, p.err, 11);
+            alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
+            if (!alive) break;
+            build_b(bh, buf, lane, 32);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_b_full(buf));
         }
     } else {
         // ---------------------------------------------------------------- epilogue (warps 2..5)
