@@ -37,9 +37,11 @@ def oracle_prediction(oracle, lay, summ_cache, q_step, n_full, seq):
     return sel, idx, slots, s64
 
 
-@pytest.mark.parametrize("mode,cap,graph", [("fetch_all", None, False), ("delta", 3, False), ("delta", 16, False),
-                                            ("fetch_all", None, True), ("delta", 3, True)])
-def test_engine_steps_match_oracle(oracle, gpu, mode, cap, graph):
+@pytest.mark.parametrize("mode,cap,graph,e2e", [("fetch_all", None, False, False), ("delta", 3, False, False),
+                                                ("delta", 16, False, False), ("fetch_all", None, True, False),
+                                                ("delta", 3, True, False), ("delta", 3, False, True),
+                                                ("delta", 3, True, True)])
+def test_engine_steps_match_oracle(oracle, gpu, mode, cap, graph, e2e):
     binding, pipeline = gpu
     dev = torch.device("cuda")
     n_layers, S = 3, 19
@@ -54,6 +56,11 @@ def test_engine_steps_match_oracle(oracle, gpu, mode, cap, graph):
     seq = lays[0].seq_len_steps                                   # [S][B]
     q_dev = [lay.q_steps.to(dev) for lay in lays]
     to_dev = lambda t: t.to(torch.int32).contiguous().to(dev)
+    # end-to-end mode: the step uploads its queries from pinned memory and downloads its outputs
+    q_pin = [lay.q_steps.pin_memory() for lay in lays] if e2e else None
+    q_stage = [torch.empty_like(q_dev[l][0]) for l in range(n_layers)] if e2e else None
+    out_pin = [torch.zeros((B, cfg.n_q_tokens, cfg.n_q_heads, 128), dtype=torch.bfloat16).pin_memory()
+               for _ in range(n_layers)] if e2e else None
     eng.prime([q_dev[l][0] for l in range(n_layers)], to_dev(seq[0] // 16), to_dev(seq[0]))
 
     # oracle-side state
@@ -79,17 +86,23 @@ def test_engine_steps_match_oracle(oracle, gpu, mode, cap, graph):
         oracle_transfer(l, sel, idx, slots, k, 0)
 
     for s in range(S):
-        args = ([q_dev[l][s] for l in range(n_layers)], to_dev(seq[s]), to_dev(seq[s] // 16),
+        args = (q_stage if e2e else [q_dev[l][s] for l in range(n_layers)], to_dev(seq[s]), to_dev(seq[s] // 16),
                 to_dev((seq[s] + 1) // 16 - seq[s] // 16), to_dev((seq[s] + 1) // 16), to_dev(seq[s] + 1))
+        kw = dict(step_stamp=s + 1)
+        if e2e:
+            kw.update(q_host=[q_pin[l][s] for l in range(n_layers)], out_host=out_pin)
         if graph:                                    # the step captured into a CUDA graph and replayed
             keep = args
-            g = eng.capture_step(*args, step_stamp=s + 1)
+            g = eng.capture_step(*args, **kw)
             eng.replay(g)
         else:
-            eng.step(*args, step_stamp=s + 1)
+            eng.step(*args, **kw)
             eng.join()
         torch.cuda.synchronize()
         for l in range(n_layers):
+            if e2e:                                  # what arrived in host memory is what the device holds
+                assert torch.equal(out_pin[l], eng.layers[l].out.cpu())
+                assert torch.equal(q_stage[l].cpu(), lays[l].q_steps[s])
             # attention of this step ran over the working set predicted one step earlier
             ref = oracle.sparse_attn(pu.np_u16(lays[l].q_steps[s]), pools[l], slot_tbl, blk[l], seq[s].numpy(), SCALE, Hkv)
             pu.assert_attn_close(pu.bf16_to_f32_np(eng.layers[l].out), ref["out32"])
