@@ -501,3 +501,51 @@ void oasis_oracle_union_blocks(int32_t B, int32_t Hkv, int32_t max_blocks, int32
     }
     free(seen);
 }
+
+/* ---------------------------------------------------------------- dense -> sparse hand-over
+ * Sec. 4.3: "A request initially performs prefill and decoding densely ...  Once its context
+ * exceeds the sparsification threshold, [the system] copies the full KV cache to CPU memory";
+ * both pools keep their blocks in Head-Token-Dimension order and each has its own page table.
+ * The dense GPU pool holds keys and values separately, dense_k / dense_v [P_gpu][Hkv][bs][d];
+ * the CPU pool holds one entry [K part | V part] per (block, head).  For request b and logical
+ * blocks j = first_block[b] .. first_block[b] + n_blocks[b] - 1 (those below max_blocks):
+ *   host_kv[(block_table[b][j] * Hkv + h)] = [ dense_k[(gpu_table[b][j] * Hkv + h)] |
+ *                                              dense_v[(gpu_table[b][j] * Hkv + h)] ]
+ * and, when summaries is given, the block's min / max rows are taken from the copied keys
+ * exactly as in step 0.
+ */
+void oasis_oracle_offload_blocks(int32_t B, int32_t Hkv, int32_t d, int32_t bs, int32_t max_blocks,
+                                 const uint16_t *dense_k, const uint16_t *dense_v,
+                                 const int32_t *gpu_table, const int32_t *block_table,
+                                 const int32_t *first_block, const int32_t *n_blocks,
+                                 uint16_t *host_kv, uint16_t *summaries)
+{
+    const int64_t part = (int64_t)bs * d;
+    for (int32_t b = 0; b < B; ++b) {
+        for (int32_t j = first_block[b]; j < first_block[b] + n_blocks[b]; ++j) {
+            if (j < 0 || j >= max_blocks) continue;
+            int64_t src = gpu_table[(int64_t)b * max_blocks + j];
+            int64_t dst = block_table[(int64_t)b * max_blocks + j];
+            for (int32_t h = 0; h < Hkv; ++h) {
+                const uint16_t *k = dense_k + (src * Hkv + h) * part;
+                const uint16_t *v = dense_v + (src * Hkv + h) * part;
+                uint16_t *entry = host_kv + (dst * Hkv + h) * 2 * part;
+                memcpy(entry, k, (size_t)part * sizeof(uint16_t));
+                memcpy(entry + part, v, (size_t)part * sizeof(uint16_t));
+                if (!summaries) continue;
+                uint16_t *row_min = summaries + ((((int64_t)b * Hkv + h) * max_blocks + j) * 2 + 0) * d;
+                uint16_t *row_max = row_min + d;
+                for (int32_t x = 0; x < d; ++x) {
+                    uint16_t lo = k[x], hi = k[x];
+                    for (int32_t i = 1; i < bs; ++i) {
+                        uint16_t t = k[(int64_t)i * d + x];
+                        if (bf16_to_f32(t) < bf16_to_f32(lo)) lo = t;
+                        if (bf16_to_f32(t) > bf16_to_f32(hi)) hi = t;
+                    }
+                    row_min[x] = lo;
+                    row_max[x] = hi;
+                }
+            }
+        }
+    }
+}

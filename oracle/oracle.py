@@ -160,3 +160,19 @@ def union_blocks(sel, k, max_blocks, max_union):
     n = np.empty((B,), dtype=np.int32)
     lib().oasis_oracle_union_blocks(B, Hkv, int(max_blocks), cols, int(k), _p(sel), int(max_union), _p(idx), _p(n))
     return idx, n
+
+
+def offload_blocks(dense_k, dense_v, gpu_table, block_table, first_block, n_blocks, host_kv, summaries=None):
+    """dense_k / dense_v [P_gpu][Hkv][bs][d] u16 -> entries of host_kv [P_cpu][Hkv][2][bs][d] u16 (in
+    place); summaries [B][Hkv][max_blocks][2][d] u16 are updated in place when given."""
+    dense_k, dense_v = _u16(dense_k), _u16(dense_v)
+    gpu_table, block_table = _i32(gpu_table), _i32(block_table)
+    first_block, n_blocks = _i32(first_block), _i32(n_blocks)
+    _, Hkv, bs, d = dense_k.shape
+    B, max_blocks = block_table.shape
+    assert host_kv.dtype == np.uint16 and host_kv.flags.c_contiguous
+    if summaries is not None:
+        assert summaries.dtype == np.uint16 and summaries.flags.c_contiguous
+    lib().oasis_oracle_offload_blocks(B, Hkv, d, bs, max_blocks, _p(dense_k), _p(dense_v), _p(gpu_table),
+                                      _p(block_table), _p(first_block), _p(n_blocks), _p(host_kv), _p(summaries))
+    return host_kv

@@ -621,3 +621,78 @@ def test_kv_footprint_worked_numbers():
     req = per_token * float(gold["context_tokens"])
     assert req / 1e9 == pytest.approx(float(gold["request_GB"]), abs=0.05)
     assert math.floor(float(gold["hbm_GB"]) / float(gold["request_GB"])) == int(gold["b_max"])
+
+
+# --------------------------------------------------------------------------- dense -> sparse hand-over
+
+
+def _handover_case(rng, B=3, Hkv=4, bs=16, d=128, mb=12):
+    Pg, Pc = B * mb + 5, B * mb + 7
+    kb, kf = rand_bf16(rng, (Pg, Hkv, bs, d))
+    vb, _ = rand_bf16(rng, (Pg, Hkv, bs, d))
+    gpu_table = rng.permutation(Pg)[:B * mb].reshape(B, mb).astype(np.int32)
+    cpu_table = rng.permutation(Pc)[:B * mb].reshape(B, mb).astype(np.int32)
+    return kb, kf, vb, gpu_table, cpu_table, Pc
+
+
+def test_offload_matches_numpy_definition_and_leaves_other_entries_alone(oracle):
+    """Entry (cpu block, head) = [K | V] of (gpu block, head), written out with numpy fancy indexing;
+    entries outside the requested ranges keep their canary."""
+    rng = np.random.default_rng(70)
+    kb, _, vb, gt, ct, Pc = _handover_case(rng)
+    B, mb = gt.shape
+    Hkv = kb.shape[1]
+    first = np.array([0, 3, 5], np.int32)
+    n = np.array([mb, 4, 0], np.int32)                              # whole request / a middle range / nothing
+    host = np.full((Pc, Hkv, 2, 16, 128), 0xBEEF, np.uint16)
+    oracle.offload_blocks(kb, vb, gt, ct, first, n, host)
+    want = np.full_like(host, 0xBEEF)
+    for b in range(B):
+        js = np.arange(first[b], first[b] + n[b])
+        want[ct[b, js]] = np.stack([kb[gt[b, js]], vb[gt[b, js]]], axis=2)
+    assert np.array_equal(host, want)
+    # a transposed K / V or a swapped table would show here: the two halves differ and the tables are permutations
+    assert not np.array_equal(kb, vb) and not np.array_equal(gt, ct)
+
+
+def test_offload_then_gather_returns_the_dense_blocks(oracle):
+    """Round trip: what the hand-over wrote to the CPU pool, gathered back by step 3, is the dense data."""
+    rng = np.random.default_rng(71)
+    kb, _, vb, gt, ct, Pc = _handover_case(rng, B=2, Hkv=2, mb=6)
+    B, mb = gt.shape
+    Hkv = kb.shape[1]
+    host = np.zeros((Pc, Hkv, 2, 16, 128), np.uint16)
+    oracle.offload_blocks(kb, vb, gt, ct, np.zeros(B, np.int32), np.full(B, mb, np.int32), host)
+    b, h = 1, 1
+    idx = (ct[b].astype(np.int64) * Hkv + h)
+    pool = np.zeros((mb, 2, 16, 128), np.uint16)
+    oracle.stage_blocks(host.reshape(-1, 2, 16, 128), idx, np.arange(mb, dtype=np.int32), pool)
+    assert np.array_equal(pool[:, 0], kb[gt[b], h]) and np.array_equal(pool[:, 1], vb[gt[b], h])
+
+
+def test_offload_summaries_are_the_min_and_max_of_the_copied_keys(oracle):
+    rng = np.random.default_rng(72)
+    kb, kf, vb, gt, ct, Pc = _handover_case(rng)
+    B, mb = gt.shape
+    Hkv = kb.shape[1]
+    first = np.array([0, 2, 1], np.int32)
+    n = np.array([mb, 5, 20], np.int32)                             # the last range runs past max_blocks: clipped
+    host = np.zeros((Pc, Hkv, 2, 16, 128), np.uint16)
+    summ = np.full((B, Hkv, mb, 2, 128), 0x7FC0, np.uint16)         # NaN canary
+    oracle.offload_blocks(kb, vb, gt, ct, first, n, host, summ)
+    got = oracle.bf16_to_f32(summ)
+    for b in range(B):
+        for j in range(mb):
+            inside = first[b] <= j < first[b] + n[b]
+            for h in range(Hkv):
+                if inside:
+                    keys = kf[gt[b, j], h]                          # [16][128]
+                    assert np.array_equal(got[b, h, j, 0], keys.min(axis=0))
+                    assert np.array_equal(got[b, h, j, 1], keys.max(axis=0))
+                else:
+                    assert np.all(summ[b, h, j] == 0x7FC0)
+    # and they agree with step 0 run on the pool the hand-over filled
+    again = oracle.build_summaries(host, ct, np.zeros(B, np.int32), np.full(B, mb, np.int32))
+    sel = [(b, j) for b in range(B) for j in range(mb) if first[b] <= j < first[b] + n[b]]
+    for b, j in sel:
+        assert np.array_equal(summ[b, :, j], again[b, :, j])
