@@ -10,7 +10,8 @@ Prints one JSON line per section:
           rho* = link bandwidth x compute time / cold bytes.
   c5      the budget x draft-length sweep (configs[4]): solo kernel times and roofline fractions of
           scoring / top-k / attention, and lookahead recall per cell.
-  stage   the gather kernel alone on random entries of a pinned pool, against the DMA copy peak.
+  stage   the gather kernel alone on random entries of a pinned pool, against the DMA copy peak, and the
+          dense -> sparse hand-over (device blocks -> pinned entries + summaries) alone.
 Inputs are synthetic (the generators of `synth`); nothing here touches the CPU oracle.
 """
 import argparse
@@ -177,7 +178,20 @@ def section_stage(args, dev, hbm_peak):
         us = graph_time(lambda i: oasis.stage_blocks(host, idxs[i], slots[i], pad, pool), 8, iters=8, warm=8)
         rows.append({"requests": n, "list_length": pad, "us": round(us, 1), "GBps": round(n * 8192 / us / 1e3, 2),
                      "frac_of_h2d_peak": round(n * 8192 / us / 1e3 / h2d_peak, 3)})
-    print(json.dumps({"section": "stage", "pinned_h2d_peak_GBps": round(h2d_peak, 2), "rows": rows}))
+    # the hand-over in the other direction: dense key / value blocks (HBM) -> entries of the pinned pool + summaries
+    Bq, Hkv, mb = 8, 8, 2048                                            # 16,384 blocks x 8 heads x 8 KiB = 1 GiB
+    dims = oasis.Dims(Bq, 32, Hkv, mb)
+    dk = torch.randn((Bq * mb, Hkv, 16, 128), device=dev).to(torch.bfloat16)
+    dv = torch.randn((Bq * mb, Hkv, 16, 128), device=dev).to(torch.bfloat16)
+    tbl = torch.arange(Bq * mb, dtype=torch.int32, device=dev).view(Bq, mb)
+    summ = torch.empty((Bq, Hkv, mb, 2, 128), dtype=torch.bfloat16, device=dev)
+    first = torch.zeros(Bq, dtype=torch.int32, device=dev)
+    n = torch.full((Bq,), mb, dtype=torch.int32, device=dev)
+    host1 = host.view(-1)[:Bq * mb * Hkv * 2 * 16 * 128].view(Bq * mb, Hkv, 2, 16, 128)
+    us = graph_time(lambda i: oasis.offload_blocks(dims, dk, dv, tbl, tbl, first, n, mb, host1, summ), 1, iters=2, warm=1)
+    gb = Bq * mb * Hkv * 8192 / 1e9
+    offload = {"blocks": Bq * mb, "GB": round(gb, 3), "ms": round(us / 1e3, 2), "GBps_to_host": round(gb / (us * 1e-6), 2)}
+    print(json.dumps({"section": "stage", "pinned_h2d_peak_GBps": round(h2d_peak, 2), "rows": rows, "offload": offload}))
 
 
 def main():

@@ -75,6 +75,29 @@ int oasis_build_summaries(const oasis_dims_t *dims, const void *kv_pool,
                           void *stream);
 
 /*
+ * Dense -> sparse hand-over (Sec. 4.3: a request prefills and decodes densely; once its context
+ * exceeds the sparsification threshold the full KV cache is copied to CPU memory and only the
+ * selected blocks and a local window stay on the GPU; both pools keep their blocks in
+ * Head-Token-Dimension order, each behind its own page table).
+ * For request b and logical blocks j = first_block[b] .. first_block[b] + n_blocks[b] - 1 (those
+ * below max_blocks) and every KV head h:
+ *   host_kv entry (block_table[b][j], h) = [ dense_k block (gpu_table[b][j], h) |
+ *                                            dense_v block (gpu_table[b][j], h) ]
+ * and, when summaries is not NULL, summaries[b][h][j] is built from the copied keys as in step 0
+ * (pass NULL for a partially filled block, which has no final summary yet).
+ *   dense_k, dense_v   [P_gpu][Hkv][16][128] bf16 (device): the dense pool's key / value blocks
+ *   gpu_table          [B][max_blocks] int32 (device): logical -> physical block of the dense pool
+ *   block_table        [B][max_blocks] int32 (device): logical -> physical block of host_kv
+ *   max_new_blocks     host-side upper bound of n_blocks[b]; sizes the launch
+ *   host_kv            full-KV pool of 8192-byte entries: mapped pinned host memory (or device memory)
+ * The working set of the first sparse step is then selected and gathered by steps 1-3 as usual.
+ */
+int oasis_offload_blocks(const oasis_dims_t *dims, const void *dense_k, const void *dense_v,
+                         const int32_t *gpu_table, const int32_t *block_table,
+                         const int32_t *first_block, const int32_t *n_blocks, int32_t max_new_blocks,
+                         void *host_kv, void *summaries, void *stream);
+
+/*
  * Step 1 -- block scores from the lookahead (draft) queries (Sec. 4.2.1: each draft query
  * scans the summaries and ranks all logical blocks independently for every KV head).
  * For one query row q and block j the estimate is the upper bound that min/max summaries

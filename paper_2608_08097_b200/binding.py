@@ -20,7 +20,8 @@ ENTRY_BYTES = 8192
 SYMBOLS = ("oasis_build_summaries", "oasis_score_blocks", "oasis_select_topk",
            "oasis_stage_blocks", "oasis_sparse_attn", "oasis_attn_workspace_bytes",
            "oasis_plan_delta", "oasis_last_error", "oasis_version",
-           "oasis_sparse_attn_static_scratch", "oasis_static_scratch_bytes", "oasis_set_error_word", "oasis_union_blocks")
+           "oasis_sparse_attn_static_scratch", "oasis_static_scratch_bytes", "oasis_set_error_word", "oasis_union_blocks",
+           "oasis_offload_blocks")
 
 
 class OasisError(RuntimeError):
@@ -76,6 +77,8 @@ def lib():
                      "oasis_stage_blocks", "oasis_sparse_attn", "oasis_plan_delta"):
             getattr(L, name).restype = ctypes.c_int
         L.oasis_union_blocks.argtypes = [dp, vp, i32, i32, i32, vp, vp, vp]
+        L.oasis_offload_blocks.argtypes = [dp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
+        L.oasis_offload_blocks.restype = ctypes.c_int
         L.oasis_union_blocks.restype = ctypes.c_int
         L.oasis_set_error_word.argtypes = [vp]
         L.oasis_set_error_word.restype = ctypes.c_int
@@ -89,7 +92,7 @@ def set_error_word(word):
     """Registers an int32 device tensor (one element, zero) that kernels flag on an internal
     wait time-out; None unregisters."""
     _check(lib().oasis_set_error_word(None if word is None else ctypes.c_void_p(word.data_ptr())),
-           "oasis_set_error_word", "oasis_union_blocks")
+           "oasis_set_error_word")
 
 
 def last_error() -> str:
@@ -186,6 +189,19 @@ def union_blocks(dims, sel, k, union_idx, n_union, stream=None):
         ctypes.byref(d), _ptr(sel, torch.int32, "sel"), int(sel.shape[-1]), int(k), int(union_idx.shape[-1]),
         _ptr(union_idx, torch.int32, "union_idx"), _ptr(n_union, torch.int32, "n_union"), _stream(stream)),
         "oasis_union_blocks")
+
+
+def offload_blocks(dims, dense_k, dense_v, gpu_table, block_table, first_block, n_blocks, max_new_blocks,
+                   host_kv, summaries=None, stream=None):
+    """Dense -> sparse hand-over: dense_k / dense_v [P_gpu][Hkv][16][128] -> entries of host_kv (and the
+    copied blocks' summaries when given)."""
+    d = dims.c()
+    _check(lib().oasis_offload_blocks(
+        ctypes.byref(d), _ptr(dense_k, torch.bfloat16, "dense_k"), _ptr(dense_v, torch.bfloat16, "dense_v"),
+        _ptr(gpu_table, torch.int32, "gpu_table"), _ptr(block_table, torch.int32, "block_table"),
+        _ptr(first_block, torch.int32, "first_block"), _ptr(n_blocks, torch.int32, "n_blocks"), int(max_new_blocks),
+        _ptr(host_kv, torch.bfloat16, "host_kv"), _ptr(summaries, torch.bfloat16, "summaries"), _stream(stream)),
+        "oasis_offload_blocks")
 
 
 def static_scratch_bytes() -> int:

@@ -194,18 +194,37 @@ class DecodeEngine:
             ev.record(ss)
         self.stage_done[l] = ev
 
-    def prime(self, q_list, n_full_next, seq_next, step_stamp=0):
-        """Before the first step: build every summary and run one prediction + transfer per
-        layer, as the step before the first one would have done."""
+    def handover(self, layer, dense_k, dense_v, gpu_table, seq_len):
+        """Dense -> sparse transition of one layer (Sec. 4.3): every block of the dense GPU pool that
+        holds tokens of a request is copied to the attached full-KV pool; the full blocks get their
+        summaries on the way, the partially filled last block does not.  `prime(...,
+        summaries_ready=True)` then selects and gathers the first working set."""
+        L = self.layers[layer]
+        torch.cuda.current_stream(self.device).synchronize()      # seq_len may still be in flight on the caller's stream
+        with torch.cuda.stream(self.pred):                        # the small tensors are made on the stream that reads them
+            n_full = (seq_len // 16).to(torch.int32)
+            n_part = ((seq_len + 15) // 16).to(torch.int32) - n_full
+            zeros = torch.zeros_like(n_full)
+            oasis.offload_blocks(L.dims, dense_k, dense_v, gpu_table, self.table[layer], zeros, n_full, L.mb,
+                                 self.kv[layer], L.summaries)
+            oasis.offload_blocks(L.dims, dense_k, dense_v, gpu_table, self.table[layer], n_full, n_part, 1,
+                                 self.kv[layer], None)
+        self.launches += 2
+
+    def prime(self, q_list, n_full_next, seq_next, step_stamp=0, summaries_ready=False):
+        """Before the first step: build every summary (unless the hand-over already did) and run one
+        prediction + transfer per layer, as the step before the first one would have done."""
         B = self.layers[0].B
         zeros = torch.zeros(B, dtype=torch.int32, device=self.device)
+        n_build = zeros if summaries_ready else n_full_next
+        torch.cuda.current_stream(self.device).synchronize()      # `zeros` is read on the engine's own streams
         plan = None
         if self.mode == "delta":        # the initial working set is admitted whole (cap = k)
             rows = (B, self.layers[0].Hkv, self.k + 2)
             plan = (torch.empty(rows, dtype=torch.int64, device=self.device),
                     torch.empty(rows, dtype=torch.int32, device=self.device))
         for l in range(self.n_layers):
-            ready = self._predict(l, q_list[l], zeros, n_full_next, self.layers[l].mb, n_full_next, seq_next,
+            ready = self._predict(l, q_list[l], zeros, n_build, self.layers[l].mb, n_full_next, seq_next,
                                   step_stamp, None, plan=plan)
             self._transfer(l, ready, None, plan=plan)
             if plan is not None:

@@ -114,3 +114,55 @@ def test_engine_steps_match_oracle(oracle, gpu, mode, cap, graph, e2e):
             oracle_transfer(l, sel, idx, slots, cap if cap is not None else k, s + 1)
             assert np.array_equal(eng.blk_tbl(l).cpu().numpy(), blk[l])
             assert np.array_equal(pu.np_u16(eng.layers[l].pool), pools[l])
+
+
+def test_handover_from_dense_pool_then_decode(oracle, gpu):
+    """Dense -> sparse transition (Sec. 4.3): the engine starts from dense GPU key / value pools behind their
+    own (permuted) page table, copies them to an empty pinned CPU pool with the summaries built on the way,
+    then selects, gathers and attends.  The CPU pool must equal the generator's pool byte for byte and the
+    first sparse step must match the oracle."""
+    binding, pipeline = gpu
+    dev = torch.device("cuda")
+    cfg = synth.scaled(synth.C2, batch=2, context=1544, k_blocks=16, layers=1, steps=2)    # 96 full blocks + 8 tokens
+    k, B, Hkv, mb = cfg.k_blocks, cfg.batch, cfg.n_kv_heads, cfg.max_blocks
+    lay = synth.make_layer(cfg, seed=33, layer=0, permute_table=True)
+    seq = lay.seq_len_steps
+    # the dense pool: the same blocks, keys and values apart, at permuted physical positions
+    g = torch.Generator()
+    g.manual_seed(5)
+    P = lay.host_kv.shape[0]
+    perm = torch.randperm(P, generator=g)
+    inv = torch.empty_like(perm)
+    inv[perm] = torch.arange(P)
+    dense_k = lay.host_kv[perm][:, :, 0].contiguous().to(dev)                # dense block p holds CPU block perm[p]
+    dense_v = lay.host_kv[perm][:, :, 1].contiguous().to(dev)
+    gpu_table = inv[lay.block_table.long()].to(torch.int32).to(dev)          # logical -> dense physical
+    host = torch.zeros_like(lay.host_kv).pin_memory()
+
+    eng = pipeline.DecodeEngine(B, cfg.n_q_heads, Hkv, mb, k, cfg.n_q_tokens, 1, dev, mode="fetch_all")
+    eng.attach(0, host, lay.block_table.to(dev))
+    to_dev = lambda t: t.to(torch.int32).contiguous().to(dev)
+    eng.handover(0, dense_k, dense_v, gpu_table, to_dev(seq[0]))
+    q_dev = lay.q_steps.to(dev)
+    eng.prime([q_dev[0]], to_dev(seq[0] // 16), to_dev(seq[0]), summaries_ready=True)
+    torch.cuda.synchronize()
+
+    n_any = (int(seq[0].max()) + 15) // 16
+    used = lay.block_table[:, :n_any].reshape(-1).long()
+    assert torch.equal(host[used], lay.host_kv[used])
+    kv = pu.np_u16(lay.host_kv)
+    n_full0 = (seq[0] // 16).numpy()
+    summ = oracle.build_summaries(kv, lay.block_table.numpy(), np.zeros(B, np.int32), n_full0)
+    pu.assert_summaries_equal(pu.np_u16(eng.layers[0].summaries), summ, n_full0)
+
+    sel, idx, slots, _ = oracle_prediction(oracle, lay, None, 0, n_full0, seq[0].numpy())
+    pool = np.zeros((B * Hkv * (k + 2), 2, 16, 128), np.uint16)
+    oracle.stage_blocks(kv.reshape(-1, 2, 16, 128), idx, slots, pool)
+    slot_tbl = np.arange(B * Hkv * (k + 2), dtype=np.int32).reshape(B, Hkv, k + 2)
+    args = ([q_dev[0]], to_dev(seq[0]), to_dev(seq[0] // 16), to_dev((seq[0] + 1) // 16 - seq[0] // 16),
+            to_dev((seq[0] + 1) // 16), to_dev(seq[0] + 1))
+    eng.step(*args, step_stamp=1)
+    eng.join()
+    torch.cuda.synchronize()
+    ref = oracle.sparse_attn(pu.np_u16(lay.q_steps[0]), pool, slot_tbl, sel, seq[0].numpy(), SCALE, Hkv)
+    pu.assert_attn_close(pu.bf16_to_f32_np(eng.layers[0].out), ref["out32"])

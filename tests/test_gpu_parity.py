@@ -392,3 +392,57 @@ def test_union_blocks_matches_oracle(oracle, gpu, nblk, k, Hkv):
         want_idx, want_n = oracle.union_blocks(sel, k, nblk, max_union)
         assert np.array_equal(n.cpu().numpy(), want_n)
         assert np.array_equal(idx.cpu().numpy(), want_idx)
+
+
+@pytest.mark.parametrize("dst", ["pinned", "device"])
+def test_offload_blocks_matches_oracle(oracle, gpu, dst):
+    """Dense -> sparse hand-over: byte-exact CPU-pool entries and summaries, permuted page tables on both
+    sides, ragged ranges (one running past max_blocks, one empty), untouched entries keep their canary."""
+    binding, _ = gpu
+    dev = torch.device("cuda")
+    rng = np.random.default_rng(81)
+    B, Hkv, mb = 3, 8, 21
+    Pg, Pc = B * mb + 3, B * mb + 9
+    k = torch.from_numpy(rng.standard_normal((Pg, Hkv, 16, 128)).astype(np.float32)).to(torch.bfloat16)
+    v = torch.from_numpy(rng.standard_normal((Pg, Hkv, 16, 128)).astype(np.float32)).to(torch.bfloat16)
+    gt = torch.from_numpy(rng.permutation(Pg)[:B * mb].reshape(B, mb).astype(np.int32))
+    ct = torch.from_numpy(rng.permutation(Pc)[:B * mb].reshape(B, mb).astype(np.int32))
+    first = torch.tensor([0, 4, 7], dtype=torch.int32)
+    n = torch.tensor([mb, 30, 0], dtype=torch.int32)
+    dims = binding.Dims(B, 32, Hkv, mb)
+    for with_summ in (True, False):
+        host = torch.full((Pc, Hkv, 2, 16, 128), -3.0, dtype=torch.bfloat16)
+        host = host.pin_memory() if dst == "pinned" else host.to(dev)
+        summ = torch.full((B, Hkv, mb, 2, 128), 7.0, dtype=torch.bfloat16, device=dev)
+        want_host = pu.np_u16(torch.full((Pc, Hkv, 2, 16, 128), -3.0, dtype=torch.bfloat16)).copy()
+        want_summ = pu.np_u16(torch.full((B, Hkv, mb, 2, 128), 7.0, dtype=torch.bfloat16)).copy()
+        oracle.offload_blocks(pu.np_u16(k), pu.np_u16(v), gt.numpy(), ct.numpy(), first.numpy(), n.numpy(), want_host,
+                              want_summ if with_summ else None)
+        binding.offload_blocks(dims, k.to(dev), v.to(dev), gt.to(dev), ct.to(dev), first.to(dev), n.to(dev), mb,
+                               host, summ if with_summ else None)
+        torch.cuda.synchronize()
+        assert np.array_equal(pu.np_u16(host), want_host)
+        assert np.array_equal(pu.np_u16(summ), want_summ)
+
+
+def test_error_word_registration(gpu):
+    """A registered error word stays zero over a normal launch and can be unregistered again."""
+    binding, pipeline = gpu
+    dev = torch.device("cuda")
+    word = torch.zeros(1, dtype=torch.int32, device=dev)
+    binding.set_error_word(word)
+    try:
+        cfg = synth.scaled(synth.C1, batch=1, context=528, k_blocks=8)
+        lay = synth.make_layer(cfg, seed=3)
+        L = pipeline.DecodeLayer(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_blocks, cfg.k_blocks, cfg.n_q_tokens, dev)
+        kv = lay.host_kv.to(dev)
+        table, n_full, seq, q = (t.to(dev) for t in (lay.block_table, lay.n_full, lay.seq_len, lay.q))
+        L.build_summaries(kv, table, torch.zeros_like(n_full), n_full, cfg.max_blocks)
+        L.score(q, n_full)
+        L.select(n_full, seq, table)
+        L.stage(kv)
+        L.attend(q, seq)
+        torch.cuda.synchronize()
+        assert int(word.item()) == 0
+    finally:
+        binding.set_error_word(None)
