@@ -260,7 +260,7 @@ class Bench:
 
     def kernel_times(self, eng, W, K, e2e=False, q_pinned=None, out_pinned=None, q_stage=None):
         """Per-kernel durations (us per launch) with CUDA events on the launching streams, over
-        the same steps launched eagerly on the same three streams."""
+        the same steps launched eagerly on the engine's streams."""
         timers = {"score": [], "select": [], "attn": [], "stage": []}
         for s in range(W, W + K):
             args, kw = self.step_args(s, e2e, q_pinned, q_stage, out_pinned)

@@ -1,6 +1,7 @@
 // Step 1 on the 5th-generation tensor cores: block scores from the draft queries (Sec. 4.2.1).
 //
-// As in score.cu, U(q, j) = q^- . min_j + q^+ . max_j, so the scores of the R query rows that
+// Since max(q_x * min_jx, q_x * max_jx) = q_x^- * min_jx + q_x^+ * max_jx with q^- = min(q, 0) and q^+ = max(q, 0),
+// U(q, j) = q^- . min_j + q^+ . max_j, so the scores of the R query rows that
 // share a KV head against a run of blocks are one small dense contraction.  Here the blocks
 // are the M dimension (swap-AB): for a tile of 128 consecutive blocks
 //     D[128 blocks x N] = A[128 x 256] (summaries, [min | max], K-major)  x  B[256 x N] (q^- | q^+)
