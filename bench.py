@@ -427,6 +427,12 @@ def run_ours(args):
         kern.setdefault(name, {})["us_in_step"] = round(us, 2)
     dominant = max(("score", "attn"), key=lambda n: solo.get(n, 0.0))
     del eng
+    # the whole step against the HBM roofline: scoring + attention bytes of all layers over the step time
+    step_gbs = (score_bytes + attn_bytes) * cfg.layers / (ms * 1e-3) / 1e9
+    extra["step_hbm"] = {"algorithmic_MB_per_layer": round((score_bytes + attn_bytes) / 1e6, 2),
+                         "achieved_GBps": round(step_gbs, 1), "frac_of_measured": round(step_gbs / hbm_peak, 3),
+                         "note": "scoring + attention bytes of all layers / step time; the two kernels each need "
+                                 "every SM (one CTA per SM) and alternate, so the step is about the sum of both"}
     eng = bench.engine("fetch_all", bench.mirror)
     ms_f, _, _ = bench.timed(eng, world, W, K)
     extra["value_fetch_all"] = {"ms_per_step": round(ms_f, 4), "value": round(tok / (ms_f * 1e-3), 1),
