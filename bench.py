@@ -32,7 +32,7 @@ import torch  # noqa: E402
 from paper_2608_08097_b200 import synth  # noqa: E402
 
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (configs[1] shapes)
-TRAFFIC_BYTES = {"score": 142.1e6, "attn": 140.2e6}
+TRAFFIC_BYTES = {"score": 142.1e6, "attn": 140.2e6, "layer": 282.3e6}
 
 METRIC = "sparse decode-attn+select tokens/s per layer"
 UNIT = "tokens/s/layer"
@@ -261,7 +261,7 @@ class Bench:
     def kernel_times(self, eng, W, K, e2e=False, q_pinned=None, out_pinned=None, q_stage=None):
         """Per-kernel durations (us per launch) with CUDA events on the launching streams, over
         the same steps launched eagerly on the engine's streams."""
-        timers = {"score": [], "select": [], "attn": [], "stage": []}
+        timers = {"score": [], "select": [], "attn": [], "layer": [], "stage": []}
         for s in range(W, W + K):
             args, kw = self.step_args(s, e2e, q_pinned, q_stage, out_pinned)
             eng.step(*args, timers=timers, **kw)
@@ -279,6 +279,9 @@ class Bench:
             "score": lambda l: eng.layers[l].score(self.q_dev[l][s], self.nfull_next_dev[s]),
             "attn": lambda l: eng.layers[l].attend(self.q_dev[l][s], self.seq_dev[s], blk_tbl=eng.blk_tbl(l)),
         }
+        if eng.fused:        # the launch the step actually makes: attention + scoring of a layer in one kernel
+            calls["layer"] = lambda l: eng.layers[l].attend_and_score(self.q_dev[l][s], self.seq_dev[s], self.nfull_next_dev[s],
+                                                                      blk_tbl=eng.blk_tbl(l))
         for name, fn in calls.items():
             torch.cuda.synchronize()
             with torch.cuda.stream(st):
@@ -373,7 +376,7 @@ def cpu_baseline(cfg, lay, budget_s=20.0):
 
 def kernel_rooflines(per_kernel, score_bytes, attn_bytes, hbm_peak):
     kern = {}
-    for name, nbytes in (("score", score_bytes), ("attn", attn_bytes)):
+    for name, nbytes in (("score", score_bytes), ("attn", attn_bytes), ("layer", score_bytes + attn_bytes)):
         if name in per_kernel:
             gbs = nbytes / (per_kernel[name] * 1e-6) / 1e9
             kern[name] = {"us": round(per_kernel[name], 2), "algorithmic_MB": round(nbytes / 1e6, 2),
@@ -425,7 +428,8 @@ def run_ours(args):
     kern = kernel_rooflines(solo, score_bytes, attn_bytes, hbm_peak)
     for name, us in per_kernel.items():          # the same launches inside the four-stream step (they share HBM there)
         kern.setdefault(name, {})["us_in_step"] = round(us, 2)
-    dominant = max(("score", "attn"), key=lambda n: solo.get(n, 0.0))
+    dominant = "layer" if "layer" in solo else max(("score", "attn"), key=lambda n: solo.get(n, 0.0))
+    fused = "layer" in solo
     del eng
     # the whole step against the HBM roofline: scoring + attention bytes of all layers over the step time
     step_gbs = (score_bytes + attn_bytes) * cfg.layers / (ms * 1e-3) / 1e9
@@ -498,7 +502,9 @@ def run_ours(args):
                              % (cfg.layers, (score_bytes + attn_bytes) / 1e6),
                        "gather": "delta selection with capped eviction, fetch ratio %.2f (cap %d blocks per head per "
                                  "step); full KV in an HBM mirror (value) / pinned host memory (e2e)" % (args.fetch_ratio, cap),
-                       "launch": "each decode step is one CUDA graph over four streams (attention / scoring / selection / transfer)"},
+                       "launch": "each decode step is one CUDA graph over four streams; a layer's attention and scoring are "
+                                 "one fused launch (oasis_attn_and_score)" if fused else
+                                 "each decode step is one CUDA graph over four streams (attention / scoring / selection / transfer)"},
             "gpu_launches": launches,
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
                        "samples": clocks["samples"]},
@@ -506,7 +512,9 @@ def run_ours(args):
                          "unit": "GB/s", "frac": d.get("frac_of_measured"), "traffic": TRAFFIC_BYTES.get(dominant),
                          "peak_kind": peak_kind + " (STREAM-style copy)",
                          "timing": "CUDA events around a graph of one launch per layer (32 distinct working sets), "
-                                   "kernel alone on its stream; us_in_step = same launch inside the four-stream step"},
+                                   "kernel alone on its stream; us_in_step = same launch inside the four-stream step; "
+                                   "'layer' = the fused attention + scoring launch the step makes, 'score' and 'attn' = "
+                                   "the two separate kernels, for comparison"},
             "kernels": kern,
             "recall_lookahead_topk": round(recall, 4),
             "e2e": e2e, "cpu_baseline": cpu, "setup_seconds": round(bench.gen_seconds, 1),

@@ -176,6 +176,27 @@ size_t oasis_attn_workspace_bytes(const oasis_dims_t *dims, int32_t n_q_tokens,
                                   int32_t n_cols);
 
 /*
+ * Steps 4 and 1 of one layer in a single launch (Sec. 4.2.2: a layer's attention over the working set
+ * staged by the previous step and its look-ahead scoring for the next step are independent).  Same
+ * arguments, arithmetic and results as oasis_sparse_attn (q .. lse) followed by oasis_score_blocks
+ * (q_draft .. scores); no workspace is needed.  One persistent thread block per SM first attends one
+ * (request, KV head) row and then scores its share of the layer's blocks over the same shared-memory
+ * ring, the shares sized so that every SM moves the same number of bytes.
+ * Only shapes with  SMs / 2 < B * Hkv <= SMs,  n_q_tokens * (Hq/Hkv) <= 128,  n_draft * (Hq/Hkv) <= 32
+ * and a shared-memory footprint within 227 KiB are taken (oasis_attn_and_score_supported tells); others
+ * return OASIS_ERR_UNSUPPORTED: make the two calls.
+ *   q_batch_stride   elements between consecutive requests of q_draft (0 = dense)
+ */
+int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int32_t n_q_tokens, const void *hbm_pool,
+                         const int32_t *slot_tbl, const int32_t *blk_tbl, int32_t n_cols,
+                         const int32_t *seq_len, float scale, void *out, float *lse, const void *q_draft,
+                         int64_t q_batch_stride, int32_t n_draft, const void *summaries,
+                         const int32_t *n_full_blocks, int32_t reduce_mode, float *scores, void *stream);
+
+/* 1 if oasis_attn_and_score takes these shapes on the current device, else 0. */
+int oasis_attn_and_score_supported(const oasis_dims_t *dims, int32_t n_q_tokens, int32_t n_draft);
+
+/*
  * Sparse attention with built-in scratch memory.  (This entry point has no counterpart in the
  * paper: it is a packaging variant of step 4.)
  * Same computation, arguments and results as oasis_sparse_attn, but the caller passes no

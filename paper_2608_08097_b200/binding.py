@@ -21,7 +21,7 @@ SYMBOLS = ("oasis_build_summaries", "oasis_score_blocks", "oasis_select_topk",
            "oasis_stage_blocks", "oasis_sparse_attn", "oasis_attn_workspace_bytes",
            "oasis_plan_delta", "oasis_last_error", "oasis_version",
            "oasis_sparse_attn_static_scratch", "oasis_static_scratch_bytes", "oasis_set_error_word", "oasis_union_blocks",
-           "oasis_offload_blocks")
+           "oasis_offload_blocks", "oasis_attn_and_score", "oasis_attn_and_score_supported")
 
 
 class OasisError(RuntimeError):
@@ -79,6 +79,11 @@ def lib():
         L.oasis_union_blocks.argtypes = [dp, vp, i32, i32, i32, vp, vp, vp]
         L.oasis_offload_blocks.argtypes = [dp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.oasis_offload_blocks.restype = ctypes.c_int
+        L.oasis_attn_and_score.argtypes = [dp, vp, i32, vp, vp, vp, i32, vp, ctypes.c_float, vp, vp, vp, ctypes.c_int64, i32, vp, vp,
+                                           i32, vp, vp]
+        L.oasis_attn_and_score.restype = ctypes.c_int
+        L.oasis_attn_and_score_supported.argtypes = [dp, i32, i32]
+        L.oasis_attn_and_score_supported.restype = ctypes.c_int
         L.oasis_union_blocks.restype = ctypes.c_int
         L.oasis_set_error_word.argtypes = [vp]
         L.oasis_set_error_word.restype = ctypes.c_int
@@ -202,6 +207,28 @@ def offload_blocks(dims, dense_k, dense_v, gpu_table, block_table, first_block, 
         _ptr(first_block, torch.int32, "first_block"), _ptr(n_blocks, torch.int32, "n_blocks"), int(max_new_blocks),
         _ptr(host_kv, torch.bfloat16, "host_kv"), _ptr(summaries, torch.bfloat16, "summaries"), _stream(stream)),
         "oasis_offload_blocks")
+
+
+def attn_and_score(dims, q, n_q_tokens, hbm_pool, slot_tbl, blk_tbl, n_cols, seq_len, scale, out, q_draft, n_draft,
+                   summaries, n_full_blocks, scores, lse=None, reduce_mode=REDUCE_MAX, q_batch_stride=None, stream=None):
+    """Steps 4 and 1 of one layer in one launch; raises OasisError (status 2) for shapes outside the fused
+    launch, which take sparse_attn + score_blocks instead."""
+    d = dims.c()
+    if q_batch_stride is None:
+        q_batch_stride = n_draft * dims.n_q_heads * 128
+    _check(lib().oasis_attn_and_score(
+        ctypes.byref(d), _ptr(q, torch.bfloat16, "q"), int(n_q_tokens), _ptr(hbm_pool, torch.bfloat16, "hbm_pool"),
+        _ptr(slot_tbl, torch.int32, "slot_tbl"), _ptr(blk_tbl, torch.int32, "blk_tbl"), int(n_cols),
+        _ptr(seq_len, torch.int32, "seq_len"), ctypes.c_float(scale), _ptr(out, torch.bfloat16, "out"),
+        _ptr(lse, torch.float32, "lse"), ctypes.c_void_p(q_draft.data_ptr()), ctypes.c_int64(int(q_batch_stride)),
+        int(n_draft), _ptr(summaries, torch.bfloat16, "summaries"), _ptr(n_full_blocks, torch.int32, "n_full_blocks"),
+        int(reduce_mode), _ptr(scores, torch.float32, "scores"), _stream(stream)), "oasis_attn_and_score")
+
+
+def attn_and_score_supported(dims, n_q_tokens, n_draft) -> bool:
+    """Whether oasis_attn_and_score takes these shapes on the current device."""
+    d = dims.c()
+    return bool(lib().oasis_attn_and_score_supported(ctypes.byref(d), int(n_q_tokens), int(n_draft)))
 
 
 def static_scratch_bytes() -> int:

@@ -42,18 +42,6 @@
 namespace oasis {
 
 constexpr int kAtThreads = 224;                             // producer, Q K^T issuer, P V issuer, four softmax warps
-constexpr int kAtTileCols = 4;                              // blocks per tile
-constexpr int kAtTileKeys = kAtTileCols * kBlock;           // 64
-constexpr int kAtStageBytes = kAtTileCols * kEntryBytes;    // 32 KiB: one 8 KiB image per block
-// Shared-memory image of one block (one 5-D tensor copy): [row group 0..1][dim half 0..1][K, V][8 rows][128 B].
-constexpr int kImgGroup = 4096, kImgHalf = 2048, kImgPart = 1024;
-constexpr int kAtSBufs = 4;                                 // S / P buffers in tensor memory (Q K^T runs 3 tiles ahead)
-constexpr int kAtQBytes = 0;                                // Q lives in tensor memory
-constexpr int kAtMaxStages = 7;
-constexpr int kAtTmemCols = 512;                            // S buffers [0,256), O [256,384), Q [384,448)
-constexpr float kAtLog2e = 1.4426950408889634f;
-constexpr float kAtLn2 = 0.6931471805599453f;
-
 struct AttnTcParams {
     const uint8_t *q;
     const int32_t *slot_tbl;
@@ -67,65 +55,6 @@ struct AttnTcParams {
     float scale_log2;
     int T, Hq, Hkv, G, n_cols, R, n_splits, cols_per_split, stages;
 };
-
-__device__ __forceinline__ void tc_mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                               uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&v)[16])
-{
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
-          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
-        : "memory");
-}
-__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t (&v)[8])
-{
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                 ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
-                 : "memory");
-}
-__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-// K-major operand with 128-byte rows and the 128-byte swizzle is described by smem_desc_sw128().
-// MN-major operand (V: rows = keys, 64 dims = 128 bytes per row and half): 8-key groups 1024 bytes
-// apart, the second 64-dim half `half_stride` bytes further.
-__device__ __forceinline__ uint64_t smem_desc_sw128_mn(uint32_t addr, uint32_t half_stride, uint32_t group_stride)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3ffffu) >> 4);
-    d |= (uint64_t)((half_stride >> 4) & 0x3fffu) << 16;   // leading-dimension byte offset
-    d |= (uint64_t)((group_stride >> 4) & 0x3fffu) << 32;  // stride between 8-key groups
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
-// K-major operand, 128-byte swizzle, 8-row groups `group_stride` bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sw128_k(uint32_t addr, uint32_t group_stride)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3ffffu) >> 4);
-    d |= (uint64_t)1 << 16;
-    d |= (uint64_t)((group_stride >> 4) & 0x3fffu) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
-__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, int c3, int c4,
-                                            uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
-        : "memory");
-}
 
 // MMA_M = 64 halves the tensor work when the query rows fit; its rows live in tensor-memory lanes
 // (m % 16) + 32 * (m / 16), i.e. sixteen per softmax warp.

@@ -1,0 +1,800 @@
+// Steps 4 + 1 of one layer in a single launch (Sec. 4.2.2: attention over the working set staged by the
+// previous step and the look-ahead scoring for the next step are independent pieces of work of the
+// same layer).  Run as two kernels they each need every SM -- one CTA per SM with almost all of its
+// shared memory -- so they can only alternate, and every alternation costs a CTA launch, a set-up,
+// a pipeline fill and a drain per SM, while the 20 SMs that get no attention row wait.  Here one
+// persistent CTA per SM does both over one ring of shared memory:
+//   phase A  (CTAs 0 .. rows-1)  the sparse attention of one (request, KV head) row, exactly as in
+//            attn_tc.cu (5-D TMA entry copies, Q K^T and P V issued by two warps, one softmax thread
+//            per MMA row with row copies);
+//   phase B  (every CTA)         a contiguous range of the layer's scoring tiles, exactly as in
+//            score_tc.cu (2-D TMA tiles of 128 summaries, swap-AB contraction against (q^- | q^+)).
+// The ring's six 32 KiB stages serve phase B as three 64 KiB stages; the producer starts the scoring
+// copies into a stage pair as soon as the attention tiles that last used it have been consumed, so
+// the stream of bytes into the SM never stops between the phases.  The scoring ranges are sized so
+// that every SM moves the same number of bytes: a CTA with an attention row of n tiles (32 KiB each)
+// gets n / 2 fewer scoring tiles (64 KiB each) than a CTA without one.
+//   warp 0     TMA producer of both phases
+//   warp 1     issues Q K^T (phase A), then the scoring MMAs (phase B)
+//   warp 2     issues P V (phase A)
+//   warps 3-6  softmax and write-out of the attention row, then the scoring epilogue
+//   warp 7     builds the (q^- | q^+) operands of the CTA's scoring range ahead of time
+// Every wait is bounded; a time-out records a code in the error word and the CTA winds down.
+// Algorithmic traffic: 8 KiB per (request, KV head, column) + Q / O, and 512 B + 4 B per scored block.
+#include <cuda.h>
+#include <math_constants.h>
+
+#include "common.cuh"
+#include "tc_common.cuh"
+
+namespace oasis {
+
+constexpr int kLyThreads = 256;
+constexpr int kLyStages = 6;                                // 32 KiB stages (phase A); three 64 KiB pairs (phase B)
+constexpr int kLyPairs = kLyStages / 2;
+constexpr int kLyTileBlocks = 128;                          // summaries per scoring tile
+constexpr int kLyATileBytes = kLyTileBlocks * kSummaryBytes;   // 64 KiB
+constexpr int kLySubTileBytes = kLyTileBlocks * 128;        // one 64-element K chunk of a scoring tile: 16 KiB
+constexpr int kLyTmemCols = 512;                            // S [0,256), O [256,384), Q [384,448), scoring accumulators [448,512)
+constexpr int kLyAccCol = 448;
+
+struct LayerTcParams {
+    // phase A: attention
+    const uint8_t *q;
+    const int32_t *slot_tbl;
+    const int32_t *blk_tbl;
+    const int32_t *seq_len;
+    uint8_t *out;
+    float *lse;
+    float scale_log2;
+    int T, Hq, Hkv, G, n_cols, R, rows;
+    // phase B: scoring
+    const uint8_t *q_draft;
+    long long q_batch_stride;
+    const int32_t *n_full;
+    float *scores;
+    int Rs, N, max_blocks, tiles_per_bh, reduce_sum;
+    long long total_tiles;
+    double w_row, w_free;       // scoring tiles of a CTA with / without an attention row
+    int32_t *err;
+};
+
+template <int MMA_M, int COPIES>
+__global__ void __launch_bounds__(kLyThreads, 1)
+layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap_summ,
+                const LayerTcParams p)
+{
+    constexpr int RPC = MMA_M / COPIES;                     // MMA rows per copy of the query rows
+    constexpr int LANES = MMA_M / 4;                        // lanes of each softmax warp that hold an MMA row
+    constexpr int BPC = kAtTileCols / COPIES;               // blocks of a tile each copy handles
+    constexpr int KPC = BPC * kBlock;                       // keys of a tile each copy handles
+    constexpr int kStageF = COPIES > 1 ? 20 : 0;            // floats per MMA row of the copy-merge staging (16 + pad)
+    constexpr int kAtQBytes = 0;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t kv_u32 = base;                                    // [6][32 KiB] = [3][64 KiB]
+    const uint32_t b_bytes = (uint32_t)p.N * kSummaryBytes;
+    const uint32_t b_u32 = kv_u32 + kLyStages * kAtStageBytes;       // [2][N][512 B] as 4 sub-tiles of N x 128 B
+    uint8_t *b_ptr = base_ptr + (size_t)kLyStages * kAtStageBytes;
+    float *o_sm = reinterpret_cast<float *>(b_ptr + 2 * b_bytes);    // [MMA_M][kStageF]
+    float *m_sm = o_sm + MMA_M * kStageF;                            // [MMA_M]
+    float *l_sm = m_sm + MMA_M;                                      // [MMA_M]
+    uint8_t *misc = reinterpret_cast<uint8_t *>(l_sm + MMA_M);
+    const uint32_t bar_u32 = smem_u32(misc);
+    // phase A barriers
+    auto bar_full = [&](int s) { return bar_u32 + 8u * s; };
+    auto bar_empty = [&](int s) { return bar_u32 + 8u * (kLyStages + s); };
+    auto bar_s_full = [&](int a) { return bar_u32 + 8u * (2 * kLyStages + a); };
+    auto bar_p_full = [&](int a) { return bar_u32 + 8u * (2 * kLyStages + kAtSBufs + a); };
+    // phase B barriers
+    constexpr int kB0 = 2 * kLyStages + 2 * kAtSBufs;
+    auto sbar_full = [&](int s) { return bar_u32 + 8u * (kB0 + s); };
+    auto sbar_empty = [&](int s) { return bar_u32 + 8u * (kB0 + kLyPairs + s); };
+    auto bar_acc_full = [&](int a) { return bar_u32 + 8u * (kB0 + 2 * kLyPairs + a); };
+    auto bar_acc_empty = [&](int a) { return bar_u32 + 8u * (kB0 + 2 * kLyPairs + 2 + a); };
+    auto bar_b_full = [&](int a) { return bar_u32 + 8u * (kB0 + 2 * kLyPairs + 4 + a); };
+    auto bar_b_empty = [&](int a) { return bar_u32 + 8u * (kB0 + 2 * kLyPairs + 6 + a); };
+    constexpr int kNBars = kB0 + 2 * kLyPairs + 8;                   // 34
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 8 * kNBars);
+    int32_t *tile_blk = reinterpret_cast<int32_t *>(misc + 8 * kNBars + 16);   // [stages][4]
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // ---- phase A geometry: CTA c < rows owns row c ------------------------------------------------------
+    const bool cta_has_row = (int)blockIdx.x < p.rows;
+    const int bh = cta_has_row ? blockIdx.x : 0;
+    const int b = bh / p.Hkv, h = bh % p.Hkv;
+    const int c0 = 0, c1 = p.n_cols;
+    const int n_tiles = cta_has_row ? (p.n_cols + kAtTileCols - 1) / kAtTileCols : 0;
+    const int L = p.seq_len[b];
+    const int32_t *slot_row = p.slot_tbl + (long long)bh * p.n_cols;
+    const int32_t *blk_row = p.blk_tbl + (long long)bh * p.n_cols;
+    // ---- phase B geometry: scoring tiles [t0, t1) ---------------------------------------------------------
+    auto tiles_before = [&](int c) {
+        const double w = c <= p.rows ? c * p.w_row : p.rows * p.w_row + (c - p.rows) * p.w_free;
+        long long t = (long long)w;
+        return t < p.total_tiles ? t : p.total_tiles;
+    };
+    const long long t0 = tiles_before(blockIdx.x);
+    const long long t1 = blockIdx.x + 1 == gridDim.x ? p.total_tiles : tiles_before(blockIdx.x + 1);
+
+    // First tile at or after t (and before t1) that has candidate blocks; t1 if there is none.
+    auto next_active = [&](long long t) {
+        for (; t < t1; ++t) {
+            const long long sbh = t / p.tiles_per_bh;
+            const int j0 = (int)(t % p.tiles_per_bh) * kLyTileBlocks;
+            if (j0 < p.n_full[(int)(sbh / p.Hkv)]) break;
+        }
+        return t;
+    };
+    // (q^- | q^+) rows of one (request, KV head), K-major, 128-byte swizzle: element k of row n
+    // lives in sub-tile k / 64.  `nthr` threads (index `me`) share the work; loads are issued
+    // eight at a time so their latencies overlap.
+    auto build_b = [&](long long bh, int buf, int me, int nthr) {
+        const int b = (int)(bh / p.Hkv), h = (int)(bh % p.Hkv);
+        uint8_t *dstb = b_ptr + (size_t)buf * b_bytes;
+        const int tasks = p.N * 16;                              // 16-byte chunks of the query rows
+        for (int i0 = me; i0 < tasks; i0 += nthr * 8) {
+            uint4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + nthr * u;
+                v[u] = make_uint4(0, 0, 0, 0);
+                const int n = i >> 4, c = i & 15;
+                if (i < tasks && (n < p.Rs || !p.reduce_sum)) {
+                    const int r = n % p.Rs;
+                    const int tq = r / p.G, a = h * p.G + r % p.G;
+                    v[u] = *reinterpret_cast<const uint4 *>(
+                        p.q_draft + ((long long)b * p.q_batch_stride + ((long long)tq * p.Hq + a) * kHeadDim) * 2 + c * 16);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + nthr * u;
+                if (i >= tasks) continue;
+                const int n = i >> 4, c = i & 15;
+                const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f);
+                uint4 neg, pos;
+                const __nv_bfloat162 *f = reinterpret_cast<const __nv_bfloat162 *>(&v[u]);
+                __nv_bfloat162 *n2 = reinterpret_cast<__nv_bfloat162 *>(&neg);
+                __nv_bfloat162 *p2 = reinterpret_cast<__nv_bfloat162 *>(&pos);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    n2[e] = __hmin2(f[e], zero2);
+                    p2[e] = __hmax2(f[e], zero2);
+                }
+                const int sub = c >> 3, ch = (c & 7) ^ (n & 7);
+                uint8_t *row = dstb + n * 128 + ch * 16;
+                *reinterpret_cast<uint4 *>(row + (size_t)sub * p.N * 128) = neg;          // k in [0, 128): min rows
+                *reinterpret_cast<uint4 *>(row + (size_t)(2 + sub) * p.N * 128) = pos;    // k in [128, 256): max rows
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    };
+
+    // ---- set-up: barriers, tensor memory, Q ---------------------------------------------------------------
+    if (tid == 0) {
+        for (int s = 0; s < kLyStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+        for (int a = 0; a < kAtSBufs; ++a) { mbar_init(bar_s_full(a), 1); mbar_init(bar_p_full(a), 4); }
+        for (int s = 0; s < kLyPairs; ++s) { mbar_init(sbar_full(s), 1); mbar_init(sbar_empty(s), 1); }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(bar_acc_full(a), 1);
+            mbar_init(bar_acc_empty(a), 4);
+            mbar_init(bar_b_full(a), 1);
+            mbar_init(bar_b_empty(a), 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncthreads();                             // the barriers exist; the producer starts copying right away
+    uint32_t tmem_base = 0, tmem_o = 0, tmem_q = 0;
+    if (warp != 0) {
+        // Meanwhile: warp 1 allocates the tensor memory, and every softmax thread, owner of one MMA row, loads
+        // that row of Q (rows are replicated across the copies, rows past R are zero) and then stores it to its
+        // tensor-memory lane.
+        if (warp == 1) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)kLyTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
+        uint4 v[16];
+        if (warp >= 3 && warp < 7 && cta_has_row) {
+            const int m_row = (warp & 3) * LANES + lane;
+            const int r = m_row % RPC;
+#pragma unroll
+            for (int c = 0; c < 16; ++c) v[c] = make_uint4(0, 0, 0, 0);
+            if (lane < LANES && r < p.R) {
+                const int tq = r / p.G, a = h * p.G + r % p.G;
+                const uint4 *src = reinterpret_cast<const uint4 *>(p.q + ((((long long)b * p.T + tq) * p.Hq + a) * kHeadDim) * 2);
+#pragma unroll
+                for (int c = 0; c < 16; ++c) v[c] = src[c];
+            }
+        }
+        tc_fence_before();
+        asm volatile("bar.sync 2, %0;" ::"n"(kLyThreads - 32) : "memory");
+        tc_fence_after();
+        tmem_base = *tmem_slot;
+        tmem_o = tmem_base + kAtSBufs * kAtTileKeys;
+        tmem_q = tmem_o + kHeadDim;                                  // Q as the A operand: 128 rows x 64 packed columns
+        if (warp >= 3 && warp < 7 && cta_has_row) {
+            const uint32_t q_lane = tmem_q + ((uint32_t)((warp & 3) * 32) << 16);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t w[16] = {v[4 * c].x, v[4 * c].y, v[4 * c].z, v[4 * c].w, v[4 * c + 1].x, v[4 * c + 1].y,
+                                        v[4 * c + 1].z, v[4 * c + 1].w, v[4 * c + 2].x, v[4 * c + 2].y, v[4 * c + 2].z,
+                                        v[4 * c + 2].w, v[4 * c + 3].x, v[4 * c + 3].y, v[4 * c + 3].z, v[4 * c + 3].w};
+                tc_st16(q_lane + c * 16, w);
+            }
+            tc_wait_st();
+        }
+        tc_fence_before();
+        asm volatile("bar.sync 2, %0;" ::"n"(kLyThreads - 32) : "memory");
+        tc_fence_after();
+    }
+    const long long t_first = next_active(t0);
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- producer
+        bool alive = true;
+        // Table entries are read 32 columns (eight tiles) at a time, lane j holding column j of the window, and the
+        // next window is requested as soon as the current one starts, so no table load sits on the critical path.
+        auto load_window = [&](int first_col, int &wblk, int &wslot) {
+            const int c = first_col + lane;
+            wblk = c < c1 ? blk_row[c] : -1;
+            wslot = c < c1 ? slot_row[c] : -1;
+        };
+        int cur_blk, cur_slot, nxt_blk = -1, nxt_slot = -1;
+        load_window(c0, cur_blk, cur_slot);
+        int s = 0;
+        uint32_t ph = 1;                                             // parity of the "empty" phase to wait for
+        for (int i = 0; i < n_tiles && alive; ++i, ph ^= (s + 1 == kLyStages), s = (s + 1 == kLyStages) ? 0 : s + 1) {
+            if ((i & 7) == 0) {
+                if (i > 0) { cur_blk = nxt_blk; cur_slot = nxt_slot; }
+                load_window(c0 + (i + 8) * kAtTileCols, nxt_blk, nxt_slot);
+            }
+            const int src_lane = (i & 7) * kAtTileCols + (lane & 3);
+            int blk = __shfl_sync(0xffffffffu, cur_blk, src_lane);
+            const int slot = __shfl_sync(0xffffffffu, cur_slot, src_lane);
+            if (lane >= kAtTileCols) blk = -1;
+            if (lane == 0) alive = mbar_wait(bar_empty(s), ph, p.err, 41);
+            alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
+            if (!alive) break;
+            const unsigned valid = __ballot_sync(0xffffffffu, lane < kAtTileCols && blk >= 0);
+            if (lane < kAtTileCols) {
+                tile_blk[s * kAtTileCols + lane] = blk;
+                if (blk < 0) {
+                    // a missing block contributes P = 0, which must not meet stale NaN bit patterns in V
+                    uint8_t *img = base_ptr + kAtQBytes + (size_t)s * kAtStageBytes + lane * kEntryBytes;
+                    for (int u = 0; u < 4; ++u)                      // (row group, dim half) units of the V part
+                        for (int j = 0; j < kImgPart / 16; ++j)
+                            *reinterpret_cast<uint4 *>(img + (u >> 1) * kImgGroup + (u & 1) * kImgHalf + kImgPart + j * 16) =
+                                make_uint4(0, 0, 0, 0);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive_expect_tx(bar_full(s), (uint32_t)__popc(valid) * kEntryBytes);
+            __syncwarp();
+            if (lane < kAtTileCols && blk >= 0)                       // the whole 8 KiB entry in one copy
+                tma_load_5d(kv_u32 + s * kAtStageBytes + lane * kEntryBytes, &tmap, 0, 0, 2 * slot, 0, 0, bar_full(s));
+        }
+        {
+            // ---------------------------------------------------------------- phase B: scoring tiles
+            int it = 0;
+            long long t = t_first;
+            while (t < t1 && alive) {
+                const long long bh = t / p.tiles_per_bh;
+                const int j0 = (int)(t % p.tiles_per_bh) * kLyTileBlocks;
+                if (lane == 0) {
+                    const int s = it % kLyPairs;
+                    if (it < kLyPairs) {
+                        // first use of this 64 KiB stage: the attention tiles that last used its two halves must be done
+    #pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const int st = 2 * s + u;
+                            const int uses = n_tiles > st ? (n_tiles - st + kLyStages - 1) / kLyStages : 0;
+                            if (uses > 0) alive = alive && mbar_wait(bar_empty(st), (uses - 1) & 1, p.err, 14);
+                        }
+                    }
+                    alive = alive && mbar_wait(sbar_empty(s), ((it / kLyPairs) & 1) ^ 1, p.err, 12);
+                    if (alive) {
+                        mbar_arrive_expect_tx(sbar_full(s), kLyATileBytes);
+                        const int y = (int)(bh * p.max_blocks + j0);
+    #pragma unroll
+                        for (int kc = 0; kc < 4; ++kc)
+                            tma_load_2d(kv_u32 + s * kLyATileBytes + kc * kLySubTileBytes, &tmap_summ, kc * 64, y, sbar_full(s));
+                    }
+                }
+                alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
+                ++it;
+                const long long tn = next_active(t + 1);
+                t = tn;
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- Q K^T issuer
+        if (lane == 0) {
+            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAtTileKeys >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
+            // descriptors: the operand start address occupies the low 14 bits (16-byte units), so offsets are added there
+            const uint64_t k_desc0 = smem_desc_sw128_k(kv_u32, kImgGroup);
+            bool alive = true;
+            int s = 0, sb = 0, s_old = 0;                            // stage and S buffer of tile i; stage of tile i - kAtSBufs
+            uint32_t ph = 0, ph_old = 0;
+            for (int i = 0; i < n_tiles && alive; ++i) {
+                // the S buffer also held P of tile i - kAtSBufs: its P V must have completed
+                if (i >= kAtSBufs) {
+                    alive = mbar_wait(bar_empty(s_old), ph_old, p.err, 51);
+                    ph_old ^= (s_old + 1 == kLyStages);
+                    s_old = (s_old + 1 == kLyStages) ? 0 : s_old + 1;
+                }
+                alive = alive && mbar_wait(bar_full(s), ph, p.err, 52);
+                if (!alive) break;
+                tc_fence_after();
+                const uint64_t k_desc = k_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(sb * kAtTileKeys);
+#pragma unroll
+                for (int kc = 0; kc < 2; ++kc)
+#pragma unroll
+                    for (int k4 = 0; k4 < 4; ++k4)
+                        tc_mma_bf16_ts(d_tmem, tmem_q + (kc * 4 + k4) * 8, k_desc + (uint64_t)((kc * kImgHalf + k4 * 32) >> 4),
+                                       idesc_qk, (kc | k4) ? 1u : 0u);
+                tc_commit(bar_s_full(sb));
+                ph ^= (s + 1 == kLyStages);
+                s = (s + 1 == kLyStages) ? 0 : s + 1;
+                sb = (sb + 1) & (kAtSBufs - 1);
+            }
+        }
+        {
+            // ---------------------------------------------------------------- phase B: scoring MMAs
+            if (lane == 0) {
+                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.N >> 3) << 17) |
+                                       ((uint32_t)(kLyTileBlocks >> 4) << 24);
+                int it = 0, bo = -1;
+                long long cur_bh = -1;
+                bool alive = true;
+                for (long long t = t0; t < t1 && alive; ++t) {
+                    const long long bh = t / p.tiles_per_bh;
+                    const int j0 = (int)(t % p.tiles_per_bh) * kLyTileBlocks;
+                    const int b = (int)(bh / p.Hkv);
+                    if (j0 >= p.n_full[b]) continue;
+                    if (bh != cur_bh) {
+                        if (bo >= 0) tc_commit(bar_b_empty(bo % 2));   // earlier MMAs no longer read that operand
+                        cur_bh = bh;
+                        ++bo;
+                        alive = mbar_wait(bar_b_full(bo % 2), (bo / 2) & 1, p.err, 21);
+                        if (!alive) break;
+                    }
+                    const int acc = it & 1, s = it % kLyPairs;
+                    alive = mbar_wait(bar_acc_empty(acc), ((it >> 1) & 1) ^ 1, p.err, 22) &&
+                            mbar_wait(sbar_full(s), (it / kLyPairs) & 1, p.err, 23);
+                    if (!alive) break;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + kLyAccCol + (uint32_t)(acc * p.N);
+                    const uint32_t a_tile = kv_u32 + s * kLyATileBytes;
+                    const uint32_t b_tile = b_u32 + (bo % 2) * b_bytes;
+    #pragma unroll
+                    for (int kc = 0; kc < 4; ++kc) {
+    #pragma unroll
+                        for (int k4 = 0; k4 < 4; ++k4) {
+                            const uint64_t ad = smem_desc_sw128(a_tile + kc * kLySubTileBytes + k4 * 32);
+                            const uint64_t bd = smem_desc_sw128(b_tile + kc * p.N * 128 + k4 * 32);
+                            tc_mma_bf16(d_tmem, ad, bd, idesc, (kc | k4) ? 1u : 0u);
+                        }
+                    }
+                    tc_commit(sbar_empty(s));         // the stage may be refilled once these MMAs have read it
+                    tc_commit(bar_acc_full(acc));    // the accumulator is complete
+                    ++it;
+                }
+            }
+        }
+    } else if (warp == 2) {
+        // ---------------------------------------------------------------- P V issuer
+        if (lane == 0) {
+            const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
+            const uint64_t v_desc0 = smem_desc_sw128_mn(kv_u32 + kImgPart, kImgHalf, kImgGroup);
+            bool alive = true;
+            int s = 0, sb = 0;
+            uint32_t ph_p = 0;
+            for (int i = 0; i < n_tiles && alive; ++i) {
+                alive = mbar_wait(bar_p_full(sb), ph_p, p.err, 53);
+                if (!alive) break;
+                tc_fence_after();
+                const uint64_t v_desc = v_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
+                const uint32_t p_tmem = tmem_base + (uint32_t)(sb * kAtTileKeys);
+#pragma unroll
+                for (int ks = 0; ks < kAtTileCols; ++ks)               // 16 keys per MMA = one block image
+                    tc_mma_bf16_ts(tmem_o, p_tmem + ks * 8, v_desc + (uint64_t)((ks * kEntryBytes) >> 4), idesc_pv,
+                                   (i | ks) ? 1u : 0u);
+                tc_commit(bar_empty(s));                             // stage free, and O complete up to this tile
+                s = (s + 1 == kLyStages) ? 0 : s + 1;
+                sb = (sb + 1) & (kAtSBufs - 1);
+                ph_p ^= (sb == 0);
+            }
+        }
+    } else if (warp == 7) {
+        // ---------------------------------------------------------------- operand builder
+        // Walks the CTA's scoring tiles ahead of everyone else and builds (q^- | q^+) of every (request, KV head)
+        // as soon as an operand buffer is free -- normally while phase A is still running.
+        int bo = -1;
+        bool alive = true;
+        long long cur_bh = -1;
+        for (long long t = t_first; t < t1 && alive; t = next_active(t + 1)) {
+            const long long bh = t / p.tiles_per_bh;
+            if (bh == cur_bh) continue;
+            cur_bh = bh;
+            ++bo;
+            const int buf = bo % 2;
+            if (lane == 0) alive = mbar_wait(bar_b_empty(buf), ((bo / 2) & 1) ^ 1, p.err, 11);
+            alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
+            if (!alive) break;
+            build_b(bh, buf, lane, 32);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_b_full(buf));
+        }
+    } else {
+        // ---------------------------------------------------------------- softmax, one thread per MMA row
+        const int quarter = warp & 3;
+        const int m_row = quarter * LANES + (lane % LANES);         // MMA row held by this tensor-memory lane
+        const int copy = m_row / RPC, row = m_row % RPC;            // which copy of the rows, which query row
+        const bool has_row = lane < LANES;
+        const bool live_row = has_row && row < p.R;
+        const bool live_warp = (quarter * LANES) % RPC < p.R;       // some lane of this warp holds a query row
+        const int limit = live_row ? L + row / p.G : -1;            // last visible position of this row
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        float m_ref = -CUDART_INF_F, l_sum = 0.f;
+        bool alive = true;
+        int s = 0, s_prev = 0;                                      // ring stage of tile i and of tile i - 1
+        uint32_t ph_prev = 0;                                       // parity of the "empty" phase that ends tile i - 1
+        for (int i = 0; i < n_tiles && alive; ++i) {
+            alive = mbar_wait(bar_s_full(i % kAtSBufs), (i / kAtSBufs) & 1, p.err, 61);
+            if (!alive) break;
+            tc_fence_after();
+            const uint32_t s_tmem = tmem_base + lane_base + (uint32_t)((i % kAtSBufs) * kAtTileKeys);
+            if (live_warp) {
+                int nvis[BPC];                                      // visible keys of each of this copy's blocks
+                bool masked = false;
+#pragma unroll
+                for (int c = 0; c < BPC; ++c) {
+                    const int blk = tile_blk[s * kAtTileCols + copy * BPC + c];
+                    int n = blk < 0 ? 0 : limit - blk * kBlock + 1;
+                    n = max(0, min(n, kBlock));
+                    nvis[c] = n;
+                    masked |= n < kBlock;
+                }
+                masked = __any_sync(0xffffffffu, masked);
+                float x[KPC];
+                {
+                    uint32_t v[BPC][16];
+#pragma unroll
+                    for (int c = 0; c < BPC; ++c) tc_ld16_nowait(s_tmem + (copy * BPC + c) * 16, v[c]);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int c = 0; c < BPC; ++c)
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) x[c * 16 + e] = __uint_as_float(v[c][e]);
+                }
+                if (masked) {
+#pragma unroll
+                    for (int c = 0; c < BPC; ++c)
+#pragma unroll
+                        for (int e = 0; e < 16; ++e)
+                            if (e >= nvis[c]) x[c * 16 + e] = -CUDART_INF_F;
+                }
+                float mx4[4] = {x[0], x[1], x[2], x[3]};
+#pragma unroll
+                for (int e = 4; e < KPC; e += 4) {
+                    mx4[0] = fmaxf(mx4[0], x[e]); mx4[1] = fmaxf(mx4[1], x[e + 1]);
+                    mx4[2] = fmaxf(mx4[2], x[e + 2]); mx4[3] = fmaxf(mx4[3], x[e + 3]);
+                }
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                const float mxs = mx * p.scale_log2;
+                const bool raise = mxs > m_ref + 8.0f;
+                if (__any_sync(0xffffffffu, raise)) {
+                    // the O rows must be complete up to tile i-1 before they are rescaled
+                    // (its stage is released by the commit that follows that P V; with at least four stages in the
+                    // ring the phase parity of that barrier is unambiguous)
+                    if (i > 0) alive = mbar_wait(bar_empty(s_prev), ph_prev, p.err, 62);
+                    tc_fence_after();
+                    const float m_new = raise ? mxs : m_ref;
+                    const float alpha = m_new == -CUDART_INF_F ? 1.f : fast_exp2(m_ref - m_new);
+                    m_ref = m_new;
+                    l_sum *= alpha;
+                    if (i > 0) {
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            uint32_t v[16];
+                            tc_ld16(tmem_o + lane_base + c * 16, v);
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
+                            tc_st16(tmem_o + lane_base + c * 16, v);
+                        }
+                        tc_wait_st();
+                    }
+                }
+                const float neg_m = m_ref == -CUDART_INF_F ? 0.f : -m_ref;
+                float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+                // P of the whole tile is 32 packed columns; this copy owns columns [copy*KPC/2, +KPC/2), the rest is 0
+                uint32_t pk[KPC / 2];
+#pragma unroll
+                for (int e = 0; e < KPC / 2; ++e) {
+                    const float p0 = fast_exp2(fmaf(x[2 * e], p.scale_log2, neg_m));
+                    const float p1 = fast_exp2(fmaf(x[2 * e + 1], p.scale_log2, neg_m));
+                    sum4[e & 3] += p0 + p1;
+                    pk[e] = pack_bf16x2(p0, p1);
+                }
+                l_sum += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+#pragma unroll
+                for (int g8 = 0; g8 < 4; ++g8) {                    // four groups of 8 packed columns = four blocks
+                    uint32_t w8[8];
+                    const int own = g8 - copy * BPC;                // index among this copy's blocks, if in [0, BPC)
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        uint32_t val = 0u;
+#pragma unroll
+                        for (int c = 0; c < BPC; ++c)
+                            if (own == c) val = pk[c * 8 + e];
+                        w8[e] = val;
+                    }
+                    tc_st8(s_tmem + g8 * 8, w8);
+                }
+                tc_wait_st();
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_p_full(i % kAtSBufs));
+            if (i > 0) ph_prev ^= (s_prev + 1 == kLyStages);
+            s_prev = s;
+            s = (s + 1 == kLyStages) ? 0 : s + 1;
+        }
+        // ---- write the attention row out: merge the copies, normalise ------------------------------------------
+        if (cta_has_row) {
+            if (alive) alive = mbar_wait(bar_empty((n_tiles - 1) % kLyStages), ((n_tiles - 1) / kLyStages) & 1, p.err, 63);
+            tc_fence_after();
+            // From here on the four softmax warps meet at named barriers, which have no time-out: go on only if
+            // none of them has given up (every thread gets here, because all its waits above are bounded).
+            alive = softmax_warps_all(alive);
+            const int t_task = quarter * 32 + lane;
+            // writes 16 output dims [d0, d0 + 16) of query row `orow`
+            auto emit = [&](int orow, int d0, const float (&acc)[16], float mx, float den) {
+                const float inv = den > 0.f ? 1.f / den : 0.f;
+                const int tq = orow / p.G, a = h * p.G + orow % p.G;
+                const long long o_row = ((long long)b * p.T + tq) * p.Hq + a;
+                uint4 *dst = reinterpret_cast<uint4 *>(p.out + (o_row * kHeadDim + d0) * 2);
+#pragma unroll
+                for (int e = 0; e < 2; ++e)
+                    dst[e] = make_uint4(pack_bf16x2(acc[8 * e] * inv, acc[8 * e + 1] * inv),
+                                        pack_bf16x2(acc[8 * e + 2] * inv, acc[8 * e + 3] * inv),
+                                        pack_bf16x2(acc[8 * e + 4] * inv, acc[8 * e + 5] * inv),
+                                        pack_bf16x2(acc[8 * e + 6] * inv, acc[8 * e + 7] * inv));
+                if (p.lse && d0 == 0) p.lse[o_row] = den > 0.f ? (mx + log2f(den)) * kAtLn2 : -CUDART_INF_F;
+            };
+            if (alive && COPIES > 1) {
+                // the ring now belongs to phase B, so the copies meet in a small staging area, 16 dims at a time
+                // (small enough that the selection kernels of other streams still fit beside this CTA)
+                if (lane < LANES) {
+                    m_sm[m_row] = m_ref;
+                    l_sm[m_row] = l_sum;
+                }
+                float mx = -CUDART_INF_F, den = 0.f, wt[COPIES];
+                for (int rd = 0; rd < 8; ++rd) {
+                    if (live_warp) {
+                        uint32_t v[16];
+                        tc_ld16(tmem_o + lane_base + rd * 16, v);
+                        float4 *dst = reinterpret_cast<float4 *>(o_sm + m_row * kStageF);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            if (lane < LANES) dst[e] = make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]),
+                                                                   __uint_as_float(v[4 * e + 2]), __uint_as_float(v[4 * e + 3]));
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");  // the four softmax warps
+                    if (t_task < RPC && t_task < p.R) {
+                        if (rd == 0) {
+#pragma unroll
+                            for (int c = 0; c < COPIES; ++c) mx = fmaxf(mx, m_sm[c * RPC + t_task]);
+#pragma unroll
+                            for (int c = 0; c < COPIES; ++c) {
+                                wt[c] = mx == -CUDART_INF_F ? 0.f : fast_exp2(m_sm[c * RPC + t_task] - mx);
+                                den += wt[c] * l_sm[c * RPC + t_task];
+                            }
+                        }
+                        float acc[16];
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+#pragma unroll
+                        for (int c = 0; c < COPIES; ++c) {
+                            if (wt[c] == 0.f) continue;             // a copy that saw no key holds no O row
+                            const float4 *src = reinterpret_cast<const float4 *>(o_sm + (c * RPC + t_task) * kStageF);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float4 v4 = src[e];
+                                acc[4 * e] += wt[c] * v4.x; acc[4 * e + 1] += wt[c] * v4.y;
+                                acc[4 * e + 2] += wt[c] * v4.z; acc[4 * e + 3] += wt[c] * v4.w;
+                            }
+                        }
+                        emit(t_task, rd * 16, acc, mx, den);
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");  // the staging rows are rewritten next round
+                }
+            } else if (alive) {
+                for (int rd = 0; rd < 8; ++rd) {                    // the thread's own O row, read by the whole warp
+                    float acc[16];
+                    uint32_t v[16];
+                    if (live_warp) tc_ld16(tmem_o + lane_base + rd * 16, v);
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) acc[e] = live_warp ? __uint_as_float(v[e]) : 0.f;
+                    if (live_row) emit(row, rd * 16, acc, m_ref, l_sum);
+                }
+            }
+        }
+        {
+            // ---------------------------------------------------------------- phase B: scoring epilogue
+            int it = 0;
+            bool alive = true;
+            for (long long t = t0; t < t1 && alive; ++t) {
+                const long long bh = t / p.tiles_per_bh;
+                const int j0 = (int)(t % p.tiles_per_bh) * kLyTileBlocks;
+                const int b = (int)(bh / p.Hkv);
+                const int nf = p.n_full[b];
+                const int j = j0 + quarter * 32 + lane;
+                float *out = p.scores + bh * p.max_blocks;
+                if (j0 >= nf) {
+                    if (j < p.max_blocks) out[j] = -CUDART_INF_F;
+                    continue;
+                }
+                const int acc = it & 1;
+                alive = mbar_wait(bar_acc_full(acc), (it >> 1) & 1, p.err, 31);
+                if (!alive) break;
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + kLyAccCol + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.N);
+                float res = p.reduce_sum ? 0.f : -CUDART_INF_F;
+                for (int c = 0; c < p.N; c += 16) {
+                    uint32_t v[16];
+                    tc_ld16(taddr + c, v);
+    #pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const float f = __uint_as_float(v[e]);
+                        res = p.reduce_sum ? res + f : fmaxf(res, f);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_acc_empty(acc));
+                if (j < p.max_blocks) out[j] = j < nf ? res : -CUDART_INF_F;
+                ++it;
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kLyTmemCols)
+                     : "memory");
+    }
+}
+
+// ---- host side -----------------------------------------------------------------------------------------
+
+static size_t layer_tc_smem_bytes(int mma_m, int copies, int N)
+{
+    return 1024 + (size_t)kLyStages * kAtStageBytes + 2 * (size_t)N * kSummaryBytes +
+           (size_t)mma_m * ((copies > 1 ? 20 : 0) + 2) * sizeof(float) + 512;
+}
+
+// Whether the fused launch takes these shapes: every (request, KV head) row an SM of its own and more rows than
+// half the SMs, the scoring accumulators beside the attention's tensor memory, everything within shared memory.
+static bool layer_tc_supported(const oasis_dims_t *dims, int n_q_tokens, int n_draft, size_t *smem_out)
+{
+    const int G = dims->n_q_heads / dims->n_kv_heads;
+    const int R = n_q_tokens * G, Rs = n_draft * G;
+    const long long rows = (long long)dims->batch * dims->n_kv_heads;
+    const int sms = sm_count();
+    const int N = (Rs + 15) / 16 * 16;
+    const int mma_m = R <= 32 ? 64 : 128, copies = R <= 16 ? 4 : (R <= 64 ? 2 : 1);
+    const size_t smem = layer_tc_smem_bytes(mma_m, copies, N);
+    if (smem_out) *smem_out = smem;
+    return R >= 1 && R <= 128 && Rs >= 1 && Rs <= 32 && rows <= sms && rows * 2 > sms && smem <= 227 * 1024;
+}
+
+}  // namespace oasis
+
+extern "C" int oasis_attn_and_score_supported(const oasis_dims_t *dims, int32_t n_q_tokens, int32_t n_draft)
+{
+    using namespace oasis;
+    if (check_dims(dims) != OASIS_OK || n_q_tokens < 1 || n_draft < 1 || dims->batch == 0) return 0;
+    return layer_tc_supported(dims, n_q_tokens, n_draft, nullptr) ? 1 : 0;
+}
+
+extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int32_t n_q_tokens, const void *hbm_pool,
+                                    const int32_t *slot_tbl, const int32_t *blk_tbl, int32_t n_cols,
+                                    const int32_t *seq_len, float scale, void *out, float *lse, const void *q_draft,
+                                    int64_t q_batch_stride, int32_t n_draft, const void *summaries,
+                                    const int32_t *n_full_blocks, int32_t reduce_mode, float *scores, void *stream)
+{
+    using namespace oasis;
+    const char *who = "oasis_attn_and_score";
+    if (int rc = check_dims(dims)) return rc;
+    if (!q || !hbm_pool || !slot_tbl || !blk_tbl || !seq_len || !out || !q_draft || !summaries || !n_full_blocks || !scores)
+        return fail(OASIS_ERR_INVALID_ARG, "%s: NULL pointer argument", who);
+    if (!aligned16(q) || !aligned16(hbm_pool) || !aligned16(out) || !aligned16(q_draft) || !aligned16(summaries))
+        return fail(OASIS_ERR_INVALID_ARG, "%s: q, hbm_pool, out, q_draft and summaries must be 16-byte aligned", who);
+    if (n_q_tokens < 1 || n_cols < 1 || n_draft < 1)
+        return fail(OASIS_ERR_INVALID_ARG, "%s: n_q_tokens %d, n_cols %d, n_draft %d", who, n_q_tokens, n_cols, n_draft);
+    if (reduce_mode != OASIS_REDUCE_MAX && reduce_mode != OASIS_REDUCE_SUM)
+        return fail(OASIS_ERR_INVALID_ARG, "%s: reduce_mode %d", who, reduce_mode);
+    const int G = dims->n_q_heads / dims->n_kv_heads;
+    const int R = n_q_tokens * G, Rs = n_draft * G;
+    if (q_batch_stride == 0) q_batch_stride = (int64_t)n_draft * dims->n_q_heads * kHeadDim;
+    if ((q_batch_stride * 2) % 16 != 0) return fail(OASIS_ERR_INVALID_ARG, "%s: q_batch_stride %lld", who, (long long)q_batch_stride);
+    if (dims->batch == 0) return OASIS_OK;
+    // The fused launch covers the shapes where every (request, KV head) row gets an SM of its own and the scoring
+    // accumulators fit beside the attention's tensor memory; other shapes take the two separate calls.
+    const long long rows = (long long)dims->batch * dims->n_kv_heads;
+    const int sms = sm_count();
+    const int N = (Rs + 15) / 16 * 16;
+    size_t smem = 0;
+    if (!layer_tc_supported(dims, n_q_tokens, n_draft, &smem))
+        return fail(OASIS_ERR_UNSUPPORTED,
+                    "%s: %lld rows on %d SMs, %d attention rows and %d scoring rows per KV head are outside the fused "
+                    "launch; call oasis_sparse_attn and oasis_score_blocks", who, rows, sms, R, Rs);
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return fail(OASIS_ERR_CUDA, "%s: cuTensorMapEncodeTiled is not available", who);
+    CUtensorMap tmap_kv, tmap_summ;
+    {
+        // the pool as 8 KiB entries (see attn_tc.cu): one box = one entry, landing as [group][half][part][8 rows][128 B]
+        const cuuint64_t gdim[5] = {64, 8, (cuuint64_t)1 << 31, 2, 2};
+        const cuuint64_t gstride[4] = {256, 4096, 128, 2048};
+        const cuuint32_t box[5] = {64, 8, 2, 2, 2};
+        const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+        CUresult cr = encode(&tmap_kv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(hbm_pool), gdim, gstride, box,
+                             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (cr != CUDA_SUCCESS) return fail(OASIS_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed (%d)", who, (int)cr);
+    }
+    {
+        // the summaries as rows of 256 bf16 (see score_tc.cu): one box = 64 elements of 128 consecutive blocks
+        const cuuint64_t gdim[2] = {256, (cuuint64_t)(rows * dims->max_blocks)};
+        const cuuint64_t gstride[1] = {(cuuint64_t)kSummaryBytes};
+        const cuuint32_t box[2] = {64, (cuuint32_t)kLyTileBlocks};
+        const cuuint32_t estr[2] = {1, 1};
+        CUresult cr = encode(&tmap_summ, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(summaries), gdim, gstride,
+                             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (cr != CUDA_SUCCESS) return fail(OASIS_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed (%d)", who, (int)cr);
+    }
+    LayerTcParams p;
+    p.q = (const uint8_t *)q; p.slot_tbl = slot_tbl; p.blk_tbl = blk_tbl; p.seq_len = seq_len;
+    p.out = (uint8_t *)out; p.lse = lse;
+    p.scale_log2 = scale * kAtLog2e;
+    p.T = n_q_tokens; p.Hq = dims->n_q_heads; p.Hkv = dims->n_kv_heads; p.G = G;
+    p.n_cols = n_cols; p.R = R; p.rows = (int)rows;
+    p.q_draft = (const uint8_t *)q_draft; p.q_batch_stride = q_batch_stride; p.n_full = n_full_blocks; p.scores = scores;
+    p.Rs = Rs; p.N = N; p.max_blocks = dims->max_blocks;
+    p.tiles_per_bh = (dims->max_blocks + kLyTileBlocks - 1) / kLyTileBlocks;
+    p.reduce_sum = reduce_mode == OASIS_REDUCE_SUM;
+    p.total_tiles = rows * p.tiles_per_bh;
+    p.err = error_word();
+    // Equal bytes per SM: an attention tile is 32 KiB, a scoring tile 64 KiB.
+    const int grid = sms;
+    const double nt_a = (n_cols + kAtTileCols - 1) / kAtTileCols;
+    const double units = ((double)rows * nt_a + 2.0 * (double)p.total_tiles) / grid;
+    double w_row = (units - nt_a) / 2.0;
+    if (w_row < 0.0) w_row = 0.0;
+    p.w_row = grid > rows ? w_row : (double)p.total_tiles / (double)rows;
+    p.w_free = grid > rows ? ((double)p.total_tiles - (double)rows * p.w_row) / (double)(grid - rows) : 0.0;
+    cudaError_t e;
+    cudaStream_t st = (cudaStream_t)stream;
+#define OASIS_LAYER_TC_LAUNCH(M, C)                                                                              \
+    do {                                                                                                         \
+        e = cudaFuncSetAttribute(layer_tc_kernel<M, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
+        if (e == cudaSuccess) layer_tc_kernel<M, C><<<grid, kLyThreads, smem, st>>>(tmap_kv, tmap_summ, p);       \
+    } while (0)
+    if (R <= 16) OASIS_LAYER_TC_LAUNCH(64, 4);
+    else if (R <= 32) OASIS_LAYER_TC_LAUNCH(64, 2);
+    else if (R <= 64) OASIS_LAYER_TC_LAUNCH(128, 2);
+    else OASIS_LAYER_TC_LAUNCH(128, 1);
+#undef OASIS_LAYER_TC_LAUNCH
+    if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "%s: shared memory %zu B: %s", who, smem, cudaGetErrorString(e));
+    return check_launch(who);
+}

@@ -75,6 +75,14 @@ class DecodeLayer:
                           self.out, lse=self.lse, workspace=self.workspace, stream=stream)
         return self.out
 
+    # steps 4 + 1 in one launch (shapes permitting)
+    def attend_and_score(self, q, seq_len, n_full_next, blk_tbl=None, slot_tbl=None, stream=None):
+        oasis.attn_and_score(self.dims, q, self.T, self.pool, self.slot_tbl if slot_tbl is None else slot_tbl,
+                             self.sel if blk_tbl is None else blk_tbl, self.cols, seq_len, self.scale, self.out,
+                             q[:, 1:], self.T - 1, self.summaries, n_full_next, self.scores, lse=self.lse,
+                             q_batch_stride=self.T * self.Hq * 128, stream=stream)
+        return self.out
+
 
 class DecodeEngine:
     """Sequencing of one decode step across layers, after the paper's asynchronous prefetch
@@ -94,10 +102,13 @@ class DecodeEngine:
     mode "fetch_all": every selected block is gathered each step (k + 2 requests per row).
     mode "delta": delta selection with capped eviction (Sec. 4.2.3) bounds the gather to
     `cap` blocks per (request, KV head) per step plus the local blocks.
+    fused (default: whenever the library takes the shapes): a layer's attention and its scoring run
+    as one launch on the foreground stream (`oasis_attn_and_score`); the summary updates of all
+    layers are then issued at the start of the step on the prediction stream.
     """
 
     def __init__(self, batch, n_q_heads, n_kv_heads, max_blocks, k, n_q_tokens, n_layers,
-                 device="cuda", mode="fetch_all", cap=None):
+                 device="cuda", mode="fetch_all", cap=None, fused=None):
         assert mode in ("fetch_all", "delta")
         self.mode, self.k, self.T, self.n_layers = mode, k, n_q_tokens, n_layers
         self.device = torch.device(device)
@@ -112,6 +123,8 @@ class DecodeEngine:
         self.copy = torch.cuda.Stream(device=self.device)     # end-to-end mode: query upload, output download
         self.launches = 0
         self.cap = cap
+        can_fuse = n_layers > 0 and n_q_tokens > 1 and oasis.attn_and_score_supported(self.layers[0].dims, n_q_tokens, n_q_tokens - 1)
+        self.fused = can_fuse if fused is None else (bool(fused) and can_fuse)
         self.stage_done = [None] * n_layers          # event of the layer's latest transfer
         if mode == "delta":
             assert cap is not None and 0 <= cap <= k
@@ -146,17 +159,19 @@ class DecodeEngine:
         timers[name].append((start, ev))
 
     def _predict(self, l, q, first_block, n_new, max_new, n_full_next, seq_next, stamp, timers,
-                 attn_done=None, plan=None):
-        """Prediction chain of one layer on the prediction stream; returns the event after which
-        the layer's gather may start."""
+                 attn_done=None, plan=None, scored=None):
+        """Prediction chain of one layer; returns the event after which the layer's gather may start.
+        `scored`: the scores were already produced (by the fused launch) and this event marks them."""
         L, ps, qs = self.layers[l], self.pred, self.selq
-        with torch.cuda.stream(ps):
-            L.build_summaries(self.kv[l], self.table[l], first_block, n_new, max_new)
-            t0 = self._tick(timers, "score", ps)
-            L.score(q, n_full_next)
-            self._tock(timers, "score", t0, ps)
-            scored = torch.cuda.Event()
-            scored.record(ps)
+        own_score = scored is None
+        if own_score:
+            with torch.cuda.stream(ps):
+                L.build_summaries(self.kv[l], self.table[l], first_block, n_new, max_new)
+                t0 = self._tick(timers, "score", ps)
+                L.score(q, n_full_next)
+                self._tock(timers, "score", t0, ps)
+                scored = torch.cuda.Event()
+                scored.record(ps)
         # top-k and the transfer plan run on their own stream, so that waiting for this layer's attention does
         # not hold back the next layer's scoring
         with torch.cuda.stream(qs):
@@ -166,7 +181,7 @@ class DecodeEngine:
             t0 = self._tick(timers, "select", qs)
             L.select(n_full_next, seq_next, self.table[l])
             self._tock(timers, "select", t0, qs)
-            self.launches += 3
+            self.launches += 3 if own_score else 1      # (summary update, scoring,) top-k
             if self.mode == "delta":
                 plan_idx = self.plan_idx[l] if plan is None else plan[0]
                 plan_slots = self.plan_slots[l] if plan is None else plan[1]
@@ -256,6 +271,15 @@ class DecodeEngine:
                     q_ready[l] = torch.cuda.Event()
                     q_ready[l].record(cs)
             self.side.wait_event(q_ready[-1])
+        summ_ready = [None] * self.n_layers
+        if self.fused:
+            # the summary updates (one newly completed block per request every 16 steps) only depend on this step's
+            # KV append: all layers' updates go first, on the prediction stream
+            with torch.cuda.stream(self.pred):
+                for l in range(self.n_layers):
+                    self.layers[l].build_summaries(self.kv[l], self.table[l], first_block, n_new, 1)
+                    summ_ready[l] = torch.cuda.Event()
+                    summ_ready[l].record(self.pred)
         for l in range(self.n_layers):
             L = self.layers[l]
             with torch.cuda.stream(ms):
@@ -263,20 +287,27 @@ class DecodeEngine:
                     ms.wait_event(q_ready[l])
                 if self.stage_done[l] is not None:
                     ms.wait_event(self.stage_done[l])
-                t0 = self._tick(timers, "attn", ms)
-                L.attend(q_list[l], seq_len, blk_tbl=self.blk_tbl(l))
-                self._tock(timers, "attn", t0, ms)
-                self.launches += 2 if self._splits else 1
+                if self.fused:
+                    ms.wait_event(summ_ready[l])
+                    t0 = self._tick(timers, "layer", ms)
+                    L.attend_and_score(q_list[l], seq_len, n_full_next, blk_tbl=self.blk_tbl(l))
+                    self._tock(timers, "layer", t0, ms)
+                    self.launches += 2                 # the fused launch and the layer's summary update
+                else:
+                    t0 = self._tick(timers, "attn", ms)
+                    L.attend(q_list[l], seq_len, blk_tbl=self.blk_tbl(l))
+                    self._tock(timers, "attn", t0, ms)
+                    self.launches += 2 if self._splits else 1
                 attn_done = torch.cuda.Event()
                 attn_done.record(ms)
             if out_host is not None:
                 cs.wait_event(attn_done)
                 with torch.cuda.stream(cs):
                     out_host[l].copy_(L.out, non_blocking=True)
-            if q_ready[l] is not None:
+            if q_ready[l] is not None and not self.fused:
                 self.pred.wait_event(q_ready[l])
             ready = self._predict(l, q_list[l], first_block, n_new, 1, n_full_next, seq_next, step_stamp, timers,
-                                  attn_done=attn_done)
+                                  attn_done=attn_done, scored=attn_done if self.fused else None)
             self._transfer(l, ready, timers)
         if out_host is not None:
             ev = torch.cuda.Event()                  # the next step's attention overwrites the output buffers

@@ -446,3 +446,49 @@ def test_error_word_registration(gpu):
         assert int(word.item()) == 0
     finally:
         binding.set_error_word(None)
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,Td,nd,ctx,k", [(16, 32, 8, 4, 4, 2064, 24), (10, 32, 8, 2, 2, 1296, 16),
+                                                  (12, 64, 8, 1, 1, 1040, 9), (10, 64, 8, 2, 2, 784, 20),
+                                                  (16, 64, 8, 8, 4, 784, 20), (18, 16, 8, 4, 4, 3088, 40),
+                                                  (16, 32, 8, 1, 1, 528, 40)])
+def test_fused_attention_and_scoring_equals_the_two_calls(oracle, gpu, B, Hq, Hkv, Td, nd, ctx, k):
+    """oasis_attn_and_score is steps 4 and 1 in one launch with unchanged arithmetic: outputs, log-sum-exps and
+    scores must equal those of oasis_sparse_attn and oasis_score_blocks bit for bit (the separate calls are the
+    ones checked against the oracle everywhere else), for 76-148 rows, ragged lengths and every row-count variant
+    (nd = draft tokens that score)."""
+    binding, pipeline = gpu
+    dev = torch.device("cuda")
+    cfg = synth.scaled(synth.C1, batch=B, n_q_heads=Hq, n_kv_heads=Hkv, context=ctx, k_blocks=k, n_draft=Td)
+    lay = synth.make_layer(cfg, seed=12, ragged=True, permute_table=True)
+    L = pipeline.DecodeLayer(B, Hq, Hkv, cfg.max_blocks, k, cfg.n_q_tokens, dev, want_lse=True)
+    kv = lay.host_kv.to(dev)
+    table, n_full, seq, q = (t.to(dev) for t in (lay.block_table, lay.n_full, lay.seq_len, lay.q))
+    stride = cfg.n_q_tokens * Hq * 128
+    L.build_summaries(kv, table, torch.zeros_like(n_full), n_full, cfg.max_blocks)
+    L.score(q, n_full)                                      # the selection uses all draft tokens
+    L.select(n_full, seq, table)
+    L.stage(kv)
+    L.attend(q, seq)
+    binding.score_blocks(L.dims, q[:, 1:1 + nd], nd, L.summaries, n_full, L.scores, q_batch_stride=stride)
+    torch.cuda.synchronize()
+    want_out, want_lse, want_scores = L.out.clone(), L.lse.clone(), L.scores.clone()
+    L.out.fill_(float("nan")); L.lse.fill_(float("nan")); L.scores.fill_(float("nan"))
+    assert binding.attn_and_score_supported(L.dims, cfg.n_q_tokens, nd)
+    binding.attn_and_score(L.dims, q, cfg.n_q_tokens, L.pool, L.slot_tbl, L.sel, L.cols, seq, L.scale, L.out,
+                           q[:, 1:1 + nd], nd, L.summaries, n_full, L.scores, lse=L.lse, q_batch_stride=stride)
+    torch.cuda.synchronize()
+    assert torch.equal(L.out.view(torch.int16), want_out.view(torch.int16))
+    assert torch.equal(L.lse, want_lse)
+    assert torch.equal(L.scores.view(torch.int32), want_scores.view(torch.int32))
+
+
+def test_fused_call_rejects_shapes_outside_its_range(gpu):
+    binding, _ = gpu
+    dev = torch.device("cuda")
+    dims = binding.Dims(2, 32, 8, 64)                               # 16 rows: far fewer than half the SMs
+    z16 = torch.zeros(1 << 16, dtype=torch.bfloat16, device=dev)
+    zi = torch.zeros(1 << 12, dtype=torch.int32, device=dev)
+    zf = torch.zeros(1 << 12, dtype=torch.float32, device=dev)
+    with pytest.raises(binding.OasisError, match="outside the fused"):
+        binding.attn_and_score(dims, z16, 5, z16, zi, zi, 10, zi, 0.1, z16, z16, 4, z16, zi, zf)
