@@ -53,4 +53,17 @@ __device__ __forceinline__ float fast_exp2(float x)
     return y;
 }
 
+// The small kernels of the other streams (top-k, plan, gather, summaries) ask for the largest shared-memory
+// carve-out although they need little: an SM they have configured otherwise could not take a thread block of the
+// attention / scoring kernels (which need nearly all of it) until they have left.
+template <typename K>
+inline void prefer_max_shared_carveout(K kernel)
+{
+    static bool done = false;          // per kernel type; a race here only repeats an idempotent call
+    if (!done) {
+        cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+        done = true;
+    }
+}
+
 }  // namespace oasis

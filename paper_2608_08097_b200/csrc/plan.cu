@@ -187,6 +187,7 @@ extern "C" int oasis_plan_delta(const oasis_dims_t *dims, const int32_t *sel, in
         cudaError_t e = cudaFuncSetAttribute(plan_delta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "oasis_plan_delta: shared memory %zu B: %s", smem, cudaGetErrorString(e));
     }
+    prefer_max_shared_carveout(plan_delta_kernel);
     plan_delta_kernel<<<dims->batch * dims->n_kv_heads, kPlanThreads, smem, (cudaStream_t)stream>>>(p);
     return check_launch("oasis_plan_delta");
 }

@@ -297,6 +297,7 @@ extern "C" int oasis_select_topk(const oasis_dims_t *dims, const float *scores,
         cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "oasis_select_topk: shared memory %zu B: %s", smem, cudaGetErrorString(e));
     }
+    prefer_max_shared_carveout(select_topk_kernel);
     select_topk_kernel<<<dims->batch * dims->n_kv_heads, threads, smem, (cudaStream_t)stream>>>(p);
     return check_launch("oasis_select_topk");
 }

@@ -48,6 +48,7 @@ extern "C" int oasis_stage_blocks(const void *host_kv, const int64_t *idx, const
     const int max_ctas = 16 * sm_count();
     int grid = (n + kStageWarps - 1) / kStageWarps;
     if (grid > max_ctas) grid = max_ctas;
+    prefer_max_shared_carveout(stage_blocks_kernel);
     stage_blocks_kernel<<<grid, kStageWarps * 32, 0, (cudaStream_t)stream>>>(
         (const uint8_t *)host_kv, (const long long *)idx, slots, n, (uint8_t *)hbm_pool);
     return check_launch("oasis_stage_blocks");

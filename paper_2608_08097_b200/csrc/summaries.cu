@@ -94,6 +94,7 @@ extern "C" int oasis_build_summaries(const oasis_dims_t *dims, const void *kv_po
     if (n_items == 0) return OASIS_OK;
     const long long grid = (n_items + kSummWarps - 1) / kSummWarps;
     if (grid > 0x7fffffffLL) return fail(OASIS_ERR_UNSUPPORTED, "oasis_build_summaries: too many blocks");
+    prefer_max_shared_carveout(build_summaries_kernel);
     build_summaries_kernel<<<(unsigned)grid, kSummWarps * 32, 0, (cudaStream_t)stream>>>(
         (const uint8_t *)kv_pool, block_table, first_block, n_blocks, (uint8_t *)summaries,
         dims->batch, dims->n_kv_heads, dims->max_blocks, max_new_blocks, n_items);
