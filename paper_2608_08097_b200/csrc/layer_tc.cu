@@ -95,7 +95,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     auto bar_acc_empty = [&](int a) { return bar_u32 + 8u * (kB0 + 2 * kLyPairs + 2 + a); };
     auto bar_b_full = [&](int a) { return bar_u32 + 8u * (kB0 + 2 * kLyPairs + 4 + a); };
     auto bar_b_empty = [&](int a) { return bar_u32 + 8u * (kB0 + 2 * kLyPairs + 6 + a); };
-    constexpr int kNBars = kB0 + 2 * kLyPairs + 8;                   // 34
+    const uint32_t bar_q = bar_u32 + 8u * (kB0 + 2 * kLyPairs + 8);  // Q is in tensor memory
+    constexpr int kNBars = kB0 + 2 * kLyPairs + 9;                   // 35
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 8 * kNBars);
     int32_t *tile_blk = reinterpret_cast<int32_t *>(misc + 8 * kNBars + 16);   // [stages][4]
 
@@ -172,7 +173,10 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     };
 
-    // ---- set-up: barriers, tensor memory, Q ---------------------------------------------------------------
+    // The next launch on the stream may start as soon as an SM has room for one of its thread blocks (its scoring
+    // phase needs nothing from this one); it waits for this grid before its attention phase.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // ---- set-up: barriers, tensor memory --------------------------------------------------------------------
     if (tid == 0) {
         for (int s = 0; s < kLyStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
         for (int a = 0; a < kAtSBufs; ++a) { mbar_init(bar_s_full(a), 1); mbar_init(bar_p_full(a), 4); }
@@ -183,32 +187,18 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             mbar_init(bar_b_full(a), 1);
             mbar_init(bar_b_empty(a), 1);
         }
+        mbar_init(bar_q, 4);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();                             // the barriers exist; the producer starts copying right away
     uint32_t tmem_base = 0, tmem_o = 0, tmem_q = 0;
     if (warp != 0) {
-        // Meanwhile: warp 1 allocates the tensor memory, and every softmax thread, owner of one MMA row, loads
-        // that row of Q (rows are replicated across the copies, rows past R are zero) and then stores it to its
-        // tensor-memory lane.
+        // Meanwhile warp 1 allocates the tensor memory.
         if (warp == 1) {
             asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                          ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)kLyTmemCols) : "memory");
             asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-        }
-        uint4 v[16];
-        if (warp >= 3 && warp < 7 && cta_has_row) {
-            const int m_row = (warp & 3) * LANES + lane;
-            const int r = m_row % RPC;
-#pragma unroll
-            for (int c = 0; c < 16; ++c) v[c] = make_uint4(0, 0, 0, 0);
-            if (lane < LANES && r < p.R) {
-                const int tq = r / p.G, a = h * p.G + r % p.G;
-                const uint4 *src = reinterpret_cast<const uint4 *>(p.q + ((((long long)b * p.T + tq) * p.Hq + a) * kHeadDim) * 2);
-#pragma unroll
-                for (int c = 0; c < 16; ++c) v[c] = src[c];
-            }
         }
         tc_fence_before();
         asm volatile("bar.sync 2, %0;" ::"n"(kLyThreads - 32) : "memory");
@@ -216,26 +206,35 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         tmem_base = *tmem_slot;
         tmem_o = tmem_base + kAtSBufs * kAtTileKeys;
         tmem_q = tmem_o + kHeadDim;                                  // Q as the A operand: 128 rows x 64 packed columns
-        if (warp >= 3 && warp < 7 && cta_has_row) {
-            const uint32_t q_lane = tmem_q + ((uint32_t)((warp & 3) * 32) << 16);
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const uint32_t w[16] = {v[4 * c].x, v[4 * c].y, v[4 * c].z, v[4 * c].w, v[4 * c + 1].x, v[4 * c + 1].y,
-                                        v[4 * c + 1].z, v[4 * c + 1].w, v[4 * c + 2].x, v[4 * c + 2].y, v[4 * c + 2].z,
-                                        v[4 * c + 2].w, v[4 * c + 3].x, v[4 * c + 3].y, v[4 * c + 3].z, v[4 * c + 3].w};
-                tc_st16(q_lane + c * 16, w);
-            }
-            tc_wait_st();
-        }
-        tc_fence_before();
-        asm volatile("bar.sync 2, %0;" ::"n"(kLyThreads - 32) : "memory");
-        tc_fence_after();
     }
     const long long t_first = next_active(t0);
-
     if (warp == 0) {
-        // ---------------------------------------------------------------- producer
         bool alive = true;
+        int it = 0;                                                  // scoring tiles issued
+        {
+            // ---------------------------------------------------------------- phase B: scoring tiles
+            long long t = t_first;
+            while (t < t1 && alive) {
+                const long long bh = t / p.tiles_per_bh;
+                const int j0 = (int)(t % p.tiles_per_bh) * kLyTileBlocks;
+                if (lane == 0) {
+                    const int s = it % kLyPairs;
+                    alive = alive && mbar_wait(sbar_empty(s), ((it / kLyPairs) & 1) ^ 1, p.err, 12);
+                    if (alive) {
+                        mbar_arrive_expect_tx(sbar_full(s), kLyATileBytes);
+                        const int y = (int)(bh * p.max_blocks + j0);
+    #pragma unroll
+                        for (int kc = 0; kc < 4; ++kc)
+                            tma_load_2d(kv_u32 + s * kLyATileBytes + kc * kLySubTileBytes, &tmap_summ, kc * 64, y, sbar_full(s));
+                    }
+                }
+                alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
+                ++it;
+                const long long tn = next_active(t + 1);
+                t = tn;
+            }
+        }
+        // ---------------------------------------------------------------- producer
         // Table entries are read 32 columns (eight tiles) at a time, lane j holding column j of the window, and the
         // next window is requested as soon as the current one starts, so no table load sits on the critical path.
         auto load_window = [&](int first_col, int &wblk, int &wslot) {
@@ -243,6 +242,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             wblk = c < c1 ? blk_row[c] : -1;
             wslot = c < c1 ? slot_row[c] : -1;
         };
+        // phase A reads what the previous layer may have produced: wait for it (no-op without a programmatic launch)
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         int cur_blk, cur_slot, nxt_blk = -1, nxt_slot = -1;
         load_window(c0, cur_blk, cur_slot);
         int s = 0;
@@ -256,7 +257,13 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             int blk = __shfl_sync(0xffffffffu, cur_blk, src_lane);
             const int slot = __shfl_sync(0xffffffffu, cur_slot, src_lane);
             if (lane >= kAtTileCols) blk = -1;
-            if (lane == 0) alive = mbar_wait(bar_empty(s), ph, p.err, 41);
+            if (lane == 0 && i < kLyStages) {
+                // first use of this stage: the scoring tiles that last used its 64 KiB pair must have been consumed
+                const int pr = s >> 1;
+                const int uses = it > pr ? (it - pr + kLyPairs - 1) / kLyPairs : 0;
+                if (uses > 0) alive = mbar_wait(sbar_empty(pr), (uses - 1) & 1, p.err, 14);
+            }
+            if (lane == 0) alive = alive && mbar_wait(bar_empty(s), ph, p.err, 41);
             alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
             if (!alive) break;
             const unsigned valid = __ballot_sync(0xffffffffu, lane < kAtTileCols && blk >= 0);
@@ -278,72 +285,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             if (lane < kAtTileCols && blk >= 0)                       // the whole 8 KiB entry in one copy
                 tma_load_5d(kv_u32 + s * kAtStageBytes + lane * kEntryBytes, &tmap, 0, 0, 2 * slot, 0, 0, bar_full(s));
         }
-        {
-            // ---------------------------------------------------------------- phase B: scoring tiles
-            int it = 0;
-            long long t = t_first;
-            while (t < t1 && alive) {
-                const long long bh = t / p.tiles_per_bh;
-                const int j0 = (int)(t % p.tiles_per_bh) * kLyTileBlocks;
-                if (lane == 0) {
-                    const int s = it % kLyPairs;
-                    if (it < kLyPairs) {
-                        // first use of this 64 KiB stage: the attention tiles that last used its two halves must be done
-    #pragma unroll
-                        for (int u = 0; u < 2; ++u) {
-                            const int st = 2 * s + u;
-                            const int uses = n_tiles > st ? (n_tiles - st + kLyStages - 1) / kLyStages : 0;
-                            if (uses > 0) alive = alive && mbar_wait(bar_empty(st), (uses - 1) & 1, p.err, 14);
-                        }
-                    }
-                    alive = alive && mbar_wait(sbar_empty(s), ((it / kLyPairs) & 1) ^ 1, p.err, 12);
-                    if (alive) {
-                        mbar_arrive_expect_tx(sbar_full(s), kLyATileBytes);
-                        const int y = (int)(bh * p.max_blocks + j0);
-    #pragma unroll
-                        for (int kc = 0; kc < 4; ++kc)
-                            tma_load_2d(kv_u32 + s * kLyATileBytes + kc * kLySubTileBytes, &tmap_summ, kc * 64, y, sbar_full(s));
-                    }
-                }
-                alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
-                ++it;
-                const long long tn = next_active(t + 1);
-                t = tn;
-            }
-        }
     } else if (warp == 1) {
-        // ---------------------------------------------------------------- Q K^T issuer
-        if (lane == 0) {
-            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAtTileKeys >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
-            // descriptors: the operand start address occupies the low 14 bits (16-byte units), so offsets are added there
-            const uint64_t k_desc0 = smem_desc_sw128_k(kv_u32, kImgGroup);
-            bool alive = true;
-            int s = 0, sb = 0, s_old = 0;                            // stage and S buffer of tile i; stage of tile i - kAtSBufs
-            uint32_t ph = 0, ph_old = 0;
-            for (int i = 0; i < n_tiles && alive; ++i) {
-                // the S buffer also held P of tile i - kAtSBufs: its P V must have completed
-                if (i >= kAtSBufs) {
-                    alive = mbar_wait(bar_empty(s_old), ph_old, p.err, 51);
-                    ph_old ^= (s_old + 1 == kLyStages);
-                    s_old = (s_old + 1 == kLyStages) ? 0 : s_old + 1;
-                }
-                alive = alive && mbar_wait(bar_full(s), ph, p.err, 52);
-                if (!alive) break;
-                tc_fence_after();
-                const uint64_t k_desc = k_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
-                const uint32_t d_tmem = tmem_base + (uint32_t)(sb * kAtTileKeys);
-#pragma unroll
-                for (int kc = 0; kc < 2; ++kc)
-#pragma unroll
-                    for (int k4 = 0; k4 < 4; ++k4)
-                        tc_mma_bf16_ts(d_tmem, tmem_q + (kc * 4 + k4) * 8, k_desc + (uint64_t)((kc * kImgHalf + k4 * 32) >> 4),
-                                       idesc_qk, (kc | k4) ? 1u : 0u);
-                tc_commit(bar_s_full(sb));
-                ph ^= (s + 1 == kLyStages);
-                s = (s + 1 == kLyStages) ? 0 : s + 1;
-                sb = (sb + 1) & (kAtSBufs - 1);
-            }
-        }
         {
             // ---------------------------------------------------------------- phase B: scoring MMAs
             if (lane == 0) {
@@ -385,6 +327,39 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                     tc_commit(bar_acc_full(acc));    // the accumulator is complete
                     ++it;
                 }
+            }
+        }
+        // ---------------------------------------------------------------- Q K^T issuer
+        if (lane == 0) {
+            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAtTileKeys >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
+            // descriptors: the operand start address occupies the low 14 bits (16-byte units), so offsets are added there
+            const uint64_t k_desc0 = smem_desc_sw128_k(kv_u32, kImgGroup);
+            bool alive = n_tiles == 0 || mbar_wait(bar_q, 0, p.err, 55);          // Q is in tensor memory
+            tc_fence_after();
+            int s = 0, sb = 0, s_old = 0;                            // stage and S buffer of tile i; stage of tile i - kAtSBufs
+            uint32_t ph = 0, ph_old = 0;
+            for (int i = 0; i < n_tiles && alive; ++i) {
+                // the S buffer also held P of tile i - kAtSBufs: its P V must have completed
+                if (i >= kAtSBufs) {
+                    alive = mbar_wait(bar_empty(s_old), ph_old, p.err, 51);
+                    ph_old ^= (s_old + 1 == kLyStages);
+                    s_old = (s_old + 1 == kLyStages) ? 0 : s_old + 1;
+                }
+                alive = alive && mbar_wait(bar_full(s), ph, p.err, 52);
+                if (!alive) break;
+                tc_fence_after();
+                const uint64_t k_desc = k_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(sb * kAtTileKeys);
+#pragma unroll
+                for (int kc = 0; kc < 2; ++kc)
+#pragma unroll
+                    for (int k4 = 0; k4 < 4; ++k4)
+                        tc_mma_bf16_ts(d_tmem, tmem_q + (kc * 4 + k4) * 8, k_desc + (uint64_t)((kc * kImgHalf + k4 * 32) >> 4),
+                                       idesc_qk, (kc | k4) ? 1u : 0u);
+                tc_commit(bar_s_full(sb));
+                ph ^= (s + 1 == kLyStages);
+                s = (s + 1 == kLyStages) ? 0 : s + 1;
+                sb = (sb + 1) & (kAtSBufs - 1);
             }
         }
     } else if (warp == 2) {
@@ -441,6 +416,69 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         const bool live_warp = (quarter * LANES) % RPC < p.R;       // some lane of this warp holds a query row
         const int limit = live_row ? L + row / p.G : -1;            // last visible position of this row
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        {
+            // ---------------------------------------------------------------- phase B: scoring epilogue
+            int it = 0;
+            bool alive = true;
+            for (long long t = t0; t < t1 && alive; ++t) {
+                const long long bh = t / p.tiles_per_bh;
+                const int j0 = (int)(t % p.tiles_per_bh) * kLyTileBlocks;
+                const int b = (int)(bh / p.Hkv);
+                const int nf = p.n_full[b];
+                const int j = j0 + quarter * 32 + lane;
+                float *out = p.scores + bh * p.max_blocks;
+                if (j0 >= nf) {
+                    if (j < p.max_blocks) out[j] = -CUDART_INF_F;
+                    continue;
+                }
+                const int acc = it & 1;
+                alive = mbar_wait(bar_acc_full(acc), (it >> 1) & 1, p.err, 31);
+                if (!alive) break;
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + kLyAccCol + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.N);
+                float res = p.reduce_sum ? 0.f : -CUDART_INF_F;
+                for (int c = 0; c < p.N; c += 16) {
+                    uint32_t v[16];
+                    tc_ld16(taddr + c, v);
+    #pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const float f = __uint_as_float(v[e]);
+                        res = p.reduce_sum ? res + f : fmaxf(res, f);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_acc_empty(acc));
+                if (j < p.max_blocks) out[j] = j < nf ? res : -CUDART_INF_F;
+                ++it;
+            }
+        }
+        // ---- phase A: this thread's Q row goes to its tensor-memory lane (rows are replicated across the copies, rows
+        // past R are zero); q may come from the previous layer: wait for it (no-op without a programmatic launch)
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (cta_has_row) {
+            uint4 v[16];
+#pragma unroll
+            for (int c = 0; c < 16; ++c) v[c] = make_uint4(0, 0, 0, 0);
+            if (live_row) {
+                const int tq = row / p.G, a = h * p.G + row % p.G;
+                const uint4 *src = reinterpret_cast<const uint4 *>(p.q + ((((long long)b * p.T + tq) * p.Hq + a) * kHeadDim) * 2);
+#pragma unroll
+                for (int c = 0; c < 16; ++c) v[c] = src[c];
+            }
+            const uint32_t q_lane = tmem_q + lane_base;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t w[16] = {v[4 * c].x, v[4 * c].y, v[4 * c].z, v[4 * c].w, v[4 * c + 1].x, v[4 * c + 1].y,
+                                        v[4 * c + 1].z, v[4 * c + 1].w, v[4 * c + 2].x, v[4 * c + 2].y, v[4 * c + 2].z,
+                                        v[4 * c + 2].w, v[4 * c + 3].x, v[4 * c + 3].y, v[4 * c + 3].z, v[4 * c + 3].w};
+                tc_st16(q_lane + c * 16, w);
+            }
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_q);
+        }
         float m_ref = -CUDART_INF_F, l_sum = 0.f;
         bool alive = true;
         int s = 0, s_prev = 0;                                      // ring stage of tile i and of tile i - 1
@@ -626,43 +664,6 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 }
             }
         }
-        {
-            // ---------------------------------------------------------------- phase B: scoring epilogue
-            int it = 0;
-            bool alive = true;
-            for (long long t = t0; t < t1 && alive; ++t) {
-                const long long bh = t / p.tiles_per_bh;
-                const int j0 = (int)(t % p.tiles_per_bh) * kLyTileBlocks;
-                const int b = (int)(bh / p.Hkv);
-                const int nf = p.n_full[b];
-                const int j = j0 + quarter * 32 + lane;
-                float *out = p.scores + bh * p.max_blocks;
-                if (j0 >= nf) {
-                    if (j < p.max_blocks) out[j] = -CUDART_INF_F;
-                    continue;
-                }
-                const int acc = it & 1;
-                alive = mbar_wait(bar_acc_full(acc), (it >> 1) & 1, p.err, 31);
-                if (!alive) break;
-                tc_fence_after();
-                const uint32_t taddr = tmem_base + kLyAccCol + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.N);
-                float res = p.reduce_sum ? 0.f : -CUDART_INF_F;
-                for (int c = 0; c < p.N; c += 16) {
-                    uint32_t v[16];
-                    tc_ld16(taddr + c, v);
-    #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const float f = __uint_as_float(v[e]);
-                        res = p.reduce_sum ? res + f : fmaxf(res, f);
-                    }
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_acc_empty(acc));
-                if (j < p.max_blocks) out[j] = j < nf ? res : -CUDART_INF_F;
-                ++it;
-            }
-        }
     }
 
     tc_fence_before();
@@ -785,16 +786,29 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     p.w_free = grid > rows ? ((double)p.total_tiles - (double)rows * p.w_row) / (double)(grid - rows) : 0.0;
     cudaError_t e;
     cudaStream_t st = (cudaStream_t)stream;
+    // Programmatic dependent launch: behind another launch of this kernel on the same stream the thread blocks start
+    // as soon as an SM has room (their scoring phase depends on nothing the predecessor writes) and wait for the
+    // predecessor only before their attention phase (griddepcontrol.wait in the kernel).
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kLyThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
 #define OASIS_LAYER_TC_LAUNCH(M, C)                                                                              \
     do {                                                                                                         \
         e = cudaFuncSetAttribute(layer_tc_kernel<M, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
-        if (e == cudaSuccess) layer_tc_kernel<M, C><<<grid, kLyThreads, smem, st>>>(tmap_kv, tmap_summ, p);       \
+        if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, layer_tc_kernel<M, C>, tmap_kv, tmap_summ, p);         \
     } while (0)
     if (R <= 16) OASIS_LAYER_TC_LAUNCH(64, 4);
     else if (R <= 32) OASIS_LAYER_TC_LAUNCH(64, 2);
     else if (R <= 64) OASIS_LAYER_TC_LAUNCH(128, 2);
     else OASIS_LAYER_TC_LAUNCH(128, 1);
 #undef OASIS_LAYER_TC_LAUNCH
-    if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "%s: shared memory %zu B: %s", who, smem, cudaGetErrorString(e));
+    if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "%s: launch with %zu B of shared memory: %s", who, smem, cudaGetErrorString(e));
     return check_launch(who);
 }
