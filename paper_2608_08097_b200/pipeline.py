@@ -117,9 +117,13 @@ class DecodeEngine:
         self.kv = [None] * n_layers
         self.table = [None] * n_layers
         self.main = torch.cuda.Stream(device=self.device)
-        self.pred = torch.cuda.Stream(device=self.device)
-        self.selq = torch.cuda.Stream(device=self.device)
-        self.side = torch.cuda.Stream(device=self.device)
+        # The small kernels go to higher-priority streams: the block scheduler then places their few thread blocks
+        # ahead of the big kernels' waiting ones instead of behind a partially dispatched grid.
+        import os
+        prio = int(os.environ.get("OASIS_SMALL_PRIO", "-1"))
+        self.pred = torch.cuda.Stream(device=self.device, priority=prio)
+        self.selq = torch.cuda.Stream(device=self.device, priority=prio)
+        self.side = torch.cuda.Stream(device=self.device, priority=prio)
         self.copy = torch.cuda.Stream(device=self.device)     # end-to-end mode: query upload, output download
         self.launches = 0
         self.cap = cap
@@ -182,14 +186,19 @@ class DecodeEngine:
             L.select(n_full_next, seq_next, self.table[l])
             self._tock(timers, "select", t0, qs)
             self.launches += 3 if own_score else 1      # (summary update, scoring,) top-k
-            if self.mode == "delta":
+            ev = torch.cuda.Event()
+            ev.record(qs)
+        if self.mode == "delta":
+            # the transfer plan runs on the transfer stream, so the next layer's top-k does not queue behind it
+            with torch.cuda.stream(self.side):
+                self.side.wait_event(ev)
                 plan_idx = self.plan_idx[l] if plan is None else plan[0]
                 plan_slots = self.plan_slots[l] if plan is None else plan[1]
                 oasis.plan_delta(L.dims, L.sel, self.k, self.table[l], self.resident[l], self.stamp[l],
                                  L.cols, plan_idx.shape[-1] - 2, stamp, plan_idx, plan_slots, n_local=2)
                 self.launches += 1
-            ev = torch.cuda.Event()
-            ev.record(qs)
+                ev = torch.cuda.Event()
+                ev.record(self.side)
         return ev
 
     def _transfer(self, l, ready, timers, plan=None):
