@@ -119,11 +119,9 @@ class DecodeEngine:
         self.main = torch.cuda.Stream(device=self.device)
         # The small kernels go to higher-priority streams: the block scheduler then places their few thread blocks
         # ahead of the big kernels' waiting ones instead of behind a partially dispatched grid.
-        import os
-        prio = int(os.environ.get("OASIS_SMALL_PRIO", "-1"))
-        self.pred = torch.cuda.Stream(device=self.device, priority=prio)
-        self.selq = torch.cuda.Stream(device=self.device, priority=prio)
-        self.side = torch.cuda.Stream(device=self.device, priority=prio)
+        self.pred = torch.cuda.Stream(device=self.device, priority=-1)
+        self.selq = torch.cuda.Stream(device=self.device, priority=-1)
+        self.side = torch.cuda.Stream(device=self.device, priority=-1)
         self.copy = torch.cuda.Stream(device=self.device)     # end-to-end mode: query upload, output download
         self.launches = 0
         self.cap = cap
