@@ -1,23 +1,29 @@
-// Steps 4 + 1 of one layer in a single launch (Sec. 4.2.2: attention over the working set staged by the
-// previous step and the look-ahead scoring for the next step are independent pieces of work of the
-// same layer).  Run as two kernels they each need every SM -- one CTA per SM with almost all of its
-// shared memory -- so they can only alternate, and every alternation costs a CTA launch, a set-up,
-// a pipeline fill and a drain per SM, while the 20 SMs that get no attention row wait.  Here one
-// persistent CTA per SM does both over one ring of shared memory:
-//   phase A  (CTAs 0 .. rows-1)  the sparse attention of one (request, KV head) row, exactly as in
-//            attn_tc.cu (5-D TMA entry copies, Q K^T and P V issued by two warps, one softmax thread
-//            per MMA row with row copies);
-//   phase B  (every CTA)         a contiguous range of the layer's scoring tiles, exactly as in
-//            score_tc.cu (2-D TMA tiles of 128 summaries, swap-AB contraction against (q^- | q^+)).
-// The ring's six 32 KiB stages serve phase B as three 64 KiB stages; the producer starts the scoring
-// copies into a stage pair as soon as the attention tiles that last used it have been consumed, so
-// the stream of bytes into the SM never stops between the phases.  The scoring ranges are sized so
-// that every SM moves the same number of bytes: a CTA with an attention row of n tiles (32 KiB each)
-// gets n / 2 fewer scoring tiles (64 KiB each) than a CTA without one.
+// Steps 1 + 4 of one layer in a single launch (Sec. 4.2.2: the look-ahead scoring for the next step and
+// the attention over the working set staged by the previous step are independent pieces of work of
+// the same layer).  Run as two kernels they each need every SM -- one CTA per SM with almost all of
+// its shared memory -- so they can only alternate, and every alternation costs a CTA launch, a
+// set-up, a pipeline fill and a drain per SM, while the 20 SMs that get no attention row wait.  Here
+// one persistent CTA per SM does both over one ring of shared memory:
+//   scoring phase    (every CTA)         a contiguous range of the layer's scoring tiles, exactly as in
+//                    score_tc.cu (2-D TMA tiles of 128 summaries, swap-AB contraction against (q^- | q^+));
+//   attention phase  (CTAs 0 .. rows-1)  the sparse attention of one (request, KV head) row, exactly as
+//                    in attn_tc.cu (5-D TMA entry copies, Q K^T and P V issued by two warps, one softmax
+//                    thread per MMA row with row copies).
+// The ring's six 32 KiB stages serve the scoring phase as three 64 KiB stages; the producer starts the
+// attention copies into a stage as soon as the scoring tiles that last used its pair have been
+// consumed, so the stream of bytes into the SM never stops between the phases.  The scoring ranges
+// are sized so that every SM moves the same number of bytes: a CTA with an attention row of n tiles
+// (32 KiB each) gets n / 2 fewer scoring tiles (64 KiB each) than a CTA without one.
+// Scoring comes first because it needs nothing from the previous layer (draft queries and summaries
+// exist before the step), whereas the attention's queries do: the kernel is launched with programmatic
+// stream serialization, so behind another launch of itself its CTAs start as soon as an SM has room
+// (griddepcontrol.launch_dependents at the top), score, and only then wait for the predecessor
+// (griddepcontrol.wait) before touching the attention inputs.  SMs are thus handed from one layer to
+// the next one by one, without the idle time around a kernel boundary.
 //   warp 0     TMA producer of both phases
-//   warp 1     issues Q K^T (phase A), then the scoring MMAs (phase B)
-//   warp 2     issues P V (phase A)
-//   warps 3-6  softmax and write-out of the attention row, then the scoring epilogue
+//   warp 1     issues the scoring MMAs, then Q K^T
+//   warp 2     issues P V
+//   warps 3-6  scoring epilogue, then Q into tensor memory, softmax and write-out of the attention row
 //   warp 7     builds the (q^- | q^+) operands of the CTA's scoring range ahead of time
 // Every wait is bounded; a time-out records a code in the error word and the CTA winds down.
 // Algorithmic traffic: 8 KiB per (request, KV head, column) + Q / O, and 512 B + 4 B per scored block.
@@ -30,7 +36,7 @@
 namespace oasis {
 
 constexpr int kLyThreads = 256;
-constexpr int kLyStages = 6;                                // 32 KiB stages (phase A); three 64 KiB pairs (phase B)
+constexpr int kLyStages = 6;                                // 32 KiB stages (attention); three 64 KiB pairs (scoring)
 constexpr int kLyPairs = kLyStages / 2;
 constexpr int kLyTileBlocks = 128;                          // summaries per scoring tile
 constexpr int kLyATileBytes = kLyTileBlocks * kSummaryBytes;   // 64 KiB
@@ -39,7 +45,7 @@ constexpr int kLyTmemCols = 512;                            // S [0,256), O [256
 constexpr int kLyAccCol = 448;
 
 struct LayerTcParams {
-    // phase A: attention
+    // attention phase
     const uint8_t *q;
     const int32_t *slot_tbl;
     const int32_t *blk_tbl;
@@ -48,7 +54,7 @@ struct LayerTcParams {
     float *lse;
     float scale_log2;
     int T, Hq, Hkv, G, n_cols, R, rows;
-    // phase B: scoring
+    // scoring phase
     const uint8_t *q_draft;
     long long q_batch_stride;
     const int32_t *n_full;
@@ -82,12 +88,12 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     float *l_sm = m_sm + MMA_M;                                      // [MMA_M]
     uint8_t *misc = reinterpret_cast<uint8_t *>(l_sm + MMA_M);
     const uint32_t bar_u32 = smem_u32(misc);
-    // phase A barriers
+    // attention-phase barriers
     auto bar_full = [&](int s) { return bar_u32 + 8u * s; };
     auto bar_empty = [&](int s) { return bar_u32 + 8u * (kLyStages + s); };
     auto bar_s_full = [&](int a) { return bar_u32 + 8u * (2 * kLyStages + a); };
     auto bar_p_full = [&](int a) { return bar_u32 + 8u * (2 * kLyStages + kAtSBufs + a); };
-    // phase B barriers
+    // scoring-phase barriers
     constexpr int kB0 = 2 * kLyStages + 2 * kAtSBufs;
     auto sbar_full = [&](int s) { return bar_u32 + 8u * (kB0 + s); };
     auto sbar_empty = [&](int s) { return bar_u32 + 8u * (kB0 + kLyPairs + s); };
@@ -101,7 +107,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     int32_t *tile_blk = reinterpret_cast<int32_t *>(misc + 8 * kNBars + 16);   // [stages][4]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // ---- phase A geometry: CTA c < rows owns row c ------------------------------------------------------
+    // ---- attention geometry: CTA c < rows owns row c ------------------------------------------------------
     const bool cta_has_row = (int)blockIdx.x < p.rows;
     const int bh = cta_has_row ? blockIdx.x : 0;
     const int b = bh / p.Hkv, h = bh % p.Hkv;
@@ -110,7 +116,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     const int L = p.seq_len[b];
     const int32_t *slot_row = p.slot_tbl + (long long)bh * p.n_cols;
     const int32_t *blk_row = p.blk_tbl + (long long)bh * p.n_cols;
-    // ---- phase B geometry: scoring tiles [t0, t1) ---------------------------------------------------------
+    // ---- scoring geometry: tiles [t0, t1) ---------------------------------------------------------
     auto tiles_before = [&](int c) {
         const double w = c <= p.rows ? c * p.w_row : p.rows * p.w_row + (c - p.rows) * p.w_free;
         long long t = (long long)w;
@@ -212,7 +218,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         bool alive = true;
         int it = 0;                                                  // scoring tiles issued
         {
-            // ---------------------------------------------------------------- phase B: scoring tiles
+            // ---------------------------------------------------------------- scoring phase: tiles
             long long t = t_first;
             while (t < t1 && alive) {
                 const long long bh = t / p.tiles_per_bh;
@@ -242,7 +248,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             wblk = c < c1 ? blk_row[c] : -1;
             wslot = c < c1 ? slot_row[c] : -1;
         };
-        // phase A reads what the previous layer may have produced: wait for it (no-op without a programmatic launch)
+        // the attention phase reads what the previous layer may have produced: wait for it (no-op without a programmatic launch)
         asm volatile("griddepcontrol.wait;" ::: "memory");
         int cur_blk, cur_slot, nxt_blk = -1, nxt_slot = -1;
         load_window(c0, cur_blk, cur_slot);
@@ -287,7 +293,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         }
     } else if (warp == 1) {
         {
-            // ---------------------------------------------------------------- phase B: scoring MMAs
+            // ---------------------------------------------------------------- scoring phase: MMAs
             if (lane == 0) {
                 const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.N >> 3) << 17) |
                                        ((uint32_t)(kLyTileBlocks >> 4) << 24);
@@ -389,7 +395,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     } else if (warp == 7) {
         // ---------------------------------------------------------------- operand builder
         // Walks the CTA's scoring tiles ahead of everyone else and builds (q^- | q^+) of every (request, KV head)
-        // as soon as an operand buffer is free -- normally while phase A is still running.
+        // as soon as an operand buffer is free.
         int bo = -1;
         bool alive = true;
         long long cur_bh = -1;
@@ -417,7 +423,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         const int limit = live_row ? L + row / p.G : -1;            // last visible position of this row
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         {
-            // ---------------------------------------------------------------- phase B: scoring epilogue
+            // ---------------------------------------------------------------- scoring phase: epilogue
             int it = 0;
             bool alive = true;
             for (long long t = t0; t < t1 && alive; ++t) {
@@ -453,7 +459,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 ++it;
             }
         }
-        // ---- phase A: this thread's Q row goes to its tensor-memory lane (rows are replicated across the copies, rows
+        // ---- attention phase: this thread's Q row goes to its tensor-memory lane (rows are replicated across the copies, rows
         // past R are zero); q may come from the previous layer: wait for it (no-op without a programmatic launch)
         asm volatile("griddepcontrol.wait;" ::: "memory");
         if (cta_has_row) {
@@ -607,8 +613,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 if (p.lse && d0 == 0) p.lse[o_row] = den > 0.f ? (mx + log2f(den)) * kAtLn2 : -CUDART_INF_F;
             };
             if (alive && COPIES > 1) {
-                // the ring now belongs to phase B, so the copies meet in a small staging area, 16 dims at a time
-                // (small enough that the selection kernels of other streams still fit beside this CTA)
+                // the copies meet in a small staging area, 16 dims at a time (small enough that the selection kernels
+                // of other streams still fit beside this CTA, and the ring may already belong to the next phase)
                 if (lane < LANES) {
                     m_sm[m_row] = m_ref;
                     l_sm[m_row] = l_sum;
