@@ -166,3 +166,42 @@ def test_handover_from_dense_pool_then_decode(oracle, gpu):
     torch.cuda.synchronize()
     ref = oracle.sparse_attn(pu.np_u16(lay.q_steps[0]), pool, slot_tbl, sel, seq[0].numpy(), SCALE, Hkv)
     pu.assert_attn_close(pu.bf16_to_f32_np(eng.layers[0].out), ref["out32"])
+
+
+@pytest.mark.parametrize("mode,cap", [("fetch_all", None), ("delta", 2)])
+def test_fused_engine_equals_unfused_engine(gpu, mode, cap):
+    """With 128 (request, KV head) rows the engine makes one fused launch per layer (attention + scoring,
+    overlapping consecutive layers through programmatic dependent launch); its outputs, selections and working
+    sets must equal, bit for bit, those of the engine that makes the two separate launches."""
+    binding, pipeline = gpu
+    dev = torch.device("cuda")
+    n_layers, S = 3, 6
+    cfg = synth.scaled(synth.C2, batch=16, context=1040, k_blocks=12, layers=n_layers, steps=S)
+    lays = [synth.make_layer(cfg, seed=51, layer=l, device=dev) for l in range(n_layers)]
+    seq = lays[0].seq_len_steps
+    to_dev = lambda t: t.to(torch.int32).contiguous().to(dev)
+    engines = []
+    for fused in (True, False):
+        eng = pipeline.DecodeEngine(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_blocks, cfg.k_blocks,
+                                    cfg.n_q_tokens, n_layers, dev, mode=mode, cap=cap, fused=fused)
+        assert eng.fused == fused
+        for l, lay in enumerate(lays):
+            eng.attach(l, lay.host_kv.to(dev), lay.block_table.to(dev))
+        engines.append(eng)
+    q_dev = [lay.q_steps.to(dev) for lay in lays]
+    for eng in engines:
+        eng.prime([q_dev[l][0] for l in range(n_layers)], to_dev(seq[0] // 16), to_dev(seq[0]))
+    for s in range(S):
+        args = ([q_dev[l][s] for l in range(n_layers)], to_dev(seq[s]), to_dev(seq[s] // 16),
+                to_dev((seq[s] + 1) // 16 - seq[s] // 16), to_dev((seq[s] + 1) // 16), to_dev(seq[s] + 1))
+        graphs = [eng.capture_step(*args, step_stamp=s + 1) for eng in engines]
+        for eng, g in zip(engines, graphs):
+            eng.replay(g)
+        torch.cuda.synchronize()
+        a, b = engines
+        for l in range(n_layers):
+            assert torch.equal(a.layers[l].out.view(torch.int16), b.layers[l].out.view(torch.int16))
+            assert torch.equal(a.layers[l].scores.view(torch.int32), b.layers[l].scores.view(torch.int32))
+            assert torch.equal(a.layers[l].sel, b.layers[l].sel)
+            assert torch.equal(a.blk_tbl(l), b.blk_tbl(l))
+            assert torch.equal(a.layers[l].pool.view(torch.int16), b.layers[l].pool.view(torch.int16))
