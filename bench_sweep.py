@@ -1,6 +1,6 @@
 """Secondary measurements of the sparse-decode path on one B200 (not part of the `bench.py` contract).
 
-    python bench_sweep.py [--layers 8] [--steps 16] [--what ratio,c5,stage]
+    python bench_sweep.py [--layers 8] [--steps 16] [--what ratio,c5,stage,shapes]
 
 Prints one JSON line per section:
   ratio   configs[1] (reasoning-style decode) at several fetch ratios of the capped delta gather
@@ -12,6 +12,9 @@ Prints one JSON line per section:
           scoring / top-k / attention, and lookahead recall per cell.
   stage   the gather kernel alone on random entries of a pinned pool, against the DMA copy peak, and the
           dense -> sparse hand-over (device blocks -> pinned entries + summaries) alone.
+  shapes  the kernels alone at the shapes of configs[1], configs[2] and configs[3] (one layer, random
+          summaries and pools): scoring, top-k, attention, and the fused attention + scoring launch where
+          it takes the shape, each against the measured copy peak.
 Inputs are synthetic (the generators of `synth`); nothing here touches the CPU oracle.
 """
 import argparse
@@ -194,6 +197,55 @@ def section_stage(args, dev, hbm_peak):
     print(json.dumps({"section": "stage", "pinned_h2d_peak_GBps": round(h2d_peak, 2), "rows": rows, "offload": offload}))
 
 
+def section_shapes(args, dev, hbm_peak):
+    """Kernels alone at the shapes of configs[1..3] (graph replay over 3 rotating working sets)."""
+    from paper_2608_08097_b200 import binding, pipeline
+    rows = []
+    for name, base in (("configs[1]", synth.C2), ("configs[2]", synth.C3), ("configs[3]", synth.C4)):
+        cfg = synth.scaled(base, layers=1, steps=1)
+        Bq, Hq, Hkv, T, mb, K = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.n_q_tokens, cfg.max_blocks, cfg.k_blocks
+        n_rot = 3
+        Ls = [pipeline.DecodeLayer(Bq, Hq, Hkv, mb, K, T, dev) for _ in range(n_rot)]
+        g = torch.Generator(device=dev)
+        g.manual_seed(args.seed)
+        q = torch.randn((Bq, T, Hq, 128), device=dev, generator=g).to(torch.bfloat16)
+        nf = cfg.context // 16
+        n_full = torch.full((Bq,), nf, dtype=torch.int32, device=dev)
+        seq = torch.full((Bq,), cfg.context, dtype=torch.int32, device=dev)
+        table = torch.arange(Bq * mb, dtype=torch.int32, device=dev).view(Bq, mb)
+        for L in Ls:
+            L.summaries.copy_(torch.randn(L.summaries.shape, device=dev, generator=g).to(torch.bfloat16))
+            L.pool.copy_(torch.randn(L.pool.shape, device=dev, generator=g).to(torch.bfloat16))
+            L.score(q, n_full)
+            L.select(n_full, seq, table)
+        torch.cuda.synchronize()
+        Td, stride = T - 1, T * Hq * 128
+        sb = Bq * Hkv * nf * 516
+        ab = Bq * Hkv * (K + 1) * 8192 + 2 * Bq * T * Hq * 256
+        t_score = graph_time(lambda i: Ls[i].score(q, n_full), n_rot)
+        t_sel = graph_time(lambda i: Ls[i].select(n_full, seq, table), n_rot)
+        t_attn = graph_time(lambda i: Ls[i].attend(q, seq), n_rot)
+        row = {"shape": name, "batch": Bq, "rows": Bq * Hkv, "context": cfg.context, "K": K, "Td": Td, "G": Hq // Hkv,
+               "score_us": round(t_score, 1), "score_frac": round(sb / t_score / 1e3 / hbm_peak, 3),
+               "select_us": round(t_sel, 1), "attn_us": round(t_attn, 1),
+               "attn_frac": round(ab / t_attn / 1e3 / hbm_peak, 3), "layer_us": None, "layer_frac": None}
+        if binding.attn_and_score_supported(Ls[0].dims, T, Td):
+            def fused(i):
+                L = Ls[i]
+                binding.attn_and_score(L.dims, q, T, L.pool, L.slot_tbl, L.sel, L.cols, seq, L.scale, L.out, q[:, 1:], Td,
+                                       L.summaries, n_full, L.scores, q_batch_stride=stride)
+            t_layer = graph_time(fused, n_rot)
+            row["layer_us"] = round(t_layer, 1)
+            row["layer_frac"] = round((sb + ab) / t_layer / 1e3 / hbm_peak, 3)
+        rows.append(row)
+        del Ls
+        torch.cuda.empty_cache()
+    print(json.dumps({"section": "shapes", "workload": "one layer of configs[1..3], 3 rotating copies of summaries and "
+                      "pools (random contents), kernels alone by graph replay; frac = algorithmic bytes / time / measured "
+                      "copy peak; layer = the fused attention + scoring launch (null where it does not take the shape)",
+                      "hbm_peak_GBps": hbm_peak, "rows": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--layers", type=int, default=8)
@@ -209,7 +261,7 @@ def main():
     build.build()
     hbm_peak, _ = B.measured_peaks()
     for what in args.what.split(","):
-        {"ratio": section_ratio, "c5": section_c5, "stage": section_stage}[what](args, dev, hbm_peak)
+        {"ratio": section_ratio, "c5": section_c5, "stage": section_stage, "shapes": section_shapes}[what](args, dev, hbm_peak)
         torch.cuda.empty_cache()
 
 

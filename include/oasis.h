@@ -179,10 +179,10 @@ size_t oasis_attn_workspace_bytes(const oasis_dims_t *dims, int32_t n_q_tokens,
  * Steps 4 and 1 of one layer in a single launch (Sec. 4.2.2: a layer's attention over the working set
  * staged by the previous step and its look-ahead scoring for the next step are independent).  Same
  * arguments, arithmetic and results as oasis_sparse_attn (q .. lse) followed by oasis_score_blocks
- * (q_draft .. scores); no workspace is needed.  One persistent thread block per SM first attends one
- * (request, KV head) row and then scores its share of the layer's blocks over the same shared-memory
- * ring, the shares sized so that every SM moves the same number of bytes.
- * Only shapes with  SMs / 2 < B * Hkv <= SMs,  n_q_tokens * (Hq/Hkv) <= 128,  n_draft * (Hq/Hkv) <= 32
+ * (q_draft .. scores); no workspace is needed.  One persistent thread block per SM scores its share of
+ * the layer's blocks and attends (request, KV head) rows c, c + SMs, c + 2 SMs, ... over the same
+ * shared-memory ring, the shares sized so that every SM moves the same number of bytes.
+ * Only shapes with  B * Hkv > SMs / 2,  n_q_tokens * (Hq/Hkv) <= 128,  n_draft * (Hq/Hkv) <= 32
  * and a shared-memory footprint within 227 KiB are taken (oasis_attn_and_score_supported tells); others
  * return OASIS_ERR_UNSUPPORTED: make the two calls.
  *   q_batch_stride   elements between consecutive requests of q_draft (0 = dense)

@@ -6,14 +6,17 @@
 // one persistent CTA per SM does both over one ring of shared memory:
 //   scoring phase    (every CTA)         a contiguous range of the layer's scoring tiles, exactly as in
 //                    score_tc.cu (2-D TMA tiles of 128 summaries, swap-AB contraction against (q^- | q^+));
-//   attention phase  (CTAs 0 .. rows-1)  the sparse attention of one (request, KV head) row, exactly as
-//                    in attn_tc.cu (5-D TMA entry copies, Q K^T and P V issued by two warps, one softmax
-//                    thread per MMA row with row copies).
+//   attention phase  (CTA c: rows c, c + grid, c + 2 grid, ...)  the sparse attention of whole (request,
+//                    KV head) rows, one after the other, exactly as in attn_tc.cu (5-D TMA entry copies,
+//                    Q K^T and P V issued by two warps, one softmax thread per MMA row with row copies).
+//                    Tiles are counted through all rows of the CTA, so the ring and the S buffers never
+//                    drain between rows; Q of the next row goes to tensor memory while the row before it
+//                    is written out.
 // The ring's six 32 KiB stages serve the scoring phase as three 64 KiB stages; the producer starts the
 // attention copies into a stage as soon as the scoring tiles that last used its pair have been
 // consumed, so the stream of bytes into the SM never stops between the phases.  The scoring ranges
-// are sized so that every SM moves the same number of bytes: a CTA with an attention row of n tiles
-// (32 KiB each) gets n / 2 fewer scoring tiles (64 KiB each) than a CTA without one.
+// are sized so that every SM moves the same number of bytes: a CTA with one more attention row of n
+// tiles (32 KiB each) gets n / 2 fewer scoring tiles (64 KiB each) than the others.
 // Scoring comes first because it needs nothing from the previous layer (draft queries and summaries
 // exist before the step), whereas the attention's queries do: the kernel is launched with programmatic
 // stream serialization, so behind another launch of itself its CTAs start as soon as an SM has room
@@ -54,6 +57,7 @@ struct LayerTcParams {
     float *lse;
     float scale_log2;
     int T, Hq, Hkv, G, n_cols, R, rows;
+    int n_more;                 // CTAs 0 .. n_more-1 attend one row more than the others
     // scoring phase
     const uint8_t *q_draft;
     long long q_batch_stride;
@@ -61,11 +65,11 @@ struct LayerTcParams {
     float *scores;
     int Rs, N, max_blocks, tiles_per_bh, reduce_sum;
     long long total_tiles;
-    double w_row, w_free;       // scoring tiles of a CTA with / without an attention row
+    double w_row, w_free;       // scoring tiles of a CTA with the larger / the smaller number of attention rows
     int32_t *err;
 };
 
-template <int MMA_M, int COPIES>
+template <int MMA_M, int COPIES, bool MULTI>                // MULTI: more rows than thread blocks, several rows per block
 __global__ void __launch_bounds__(kLyThreads, 1)
 layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap_summ,
                 const LayerTcParams p)
@@ -108,17 +112,16 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // ---- attention geometry: CTA c < rows owns row c ------------------------------------------------------
-    const bool cta_has_row = (int)blockIdx.x < p.rows;
-    const int bh = cta_has_row ? blockIdx.x : 0;
-    const int b = bh / p.Hkv, h = bh % p.Hkv;
+    const int n_my_rows = (int)blockIdx.x < p.rows ? (MULTI ? (p.rows - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 1) : 0;
+    const bool cta_has_row = n_my_rows > 0;
+    auto my_row = [&](int k) { return (int)blockIdx.x + k * (int)gridDim.x; };     // k-th row of this CTA
     const int c0 = 0, c1 = p.n_cols;
-    const int n_tiles = cta_has_row ? (p.n_cols + kAtTileCols - 1) / kAtTileCols : 0;
-    const int L = p.seq_len[b];
-    const int32_t *slot_row = p.slot_tbl + (long long)bh * p.n_cols;
-    const int32_t *blk_row = p.blk_tbl + (long long)bh * p.n_cols;
+    const int tpr = (p.n_cols + kAtTileCols - 1) / kAtTileCols;     // tiles per row
+    const int n_tiles = n_my_rows * tpr;                             // attention tiles of this CTA, all rows
+    const int L0 = p.seq_len[(cta_has_row ? (int)blockIdx.x : 0) / p.Hkv];   // length of the request of the first row
     // ---- scoring geometry: tiles [t0, t1) ---------------------------------------------------------
     auto tiles_before = [&](int c) {
-        const double w = c <= p.rows ? c * p.w_row : p.rows * p.w_row + (c - p.rows) * p.w_free;
+        const double w = c <= p.n_more ? c * p.w_row : p.n_more * p.w_row + (c - p.n_more) * p.w_free;
         long long t = (long long)w;
         return t < p.total_tiles ? t : p.total_tiles;
     };
@@ -243,6 +246,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         // ---------------------------------------------------------------- producer
         // Table entries are read 32 columns (eight tiles) at a time, lane j holding column j of the window, and the
         // next window is requested as soon as the current one starts, so no table load sits on the critical path.
+        const int32_t *slot_row = p.slot_tbl, *blk_row = p.blk_tbl;
         auto load_window = [&](int first_col, int &wblk, int &wslot) {
             const int c = first_col + lane;
             wblk = c < c1 ? blk_row[c] : -1;
@@ -250,11 +254,14 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         };
         // the attention phase reads what the previous layer may have produced: wait for it (no-op without a programmatic launch)
         asm volatile("griddepcontrol.wait;" ::: "memory");
+        int s = 0, gi = 0;                                           // ring stage and index of the tile among all rows
+        uint32_t ph = 1;                                             // parity of the "empty" phase to wait for
+        for (int k = 0; k < n_my_rows && alive; ++k) {
+        slot_row = p.slot_tbl + (long long)my_row(k) * p.n_cols;
+        blk_row = p.blk_tbl + (long long)my_row(k) * p.n_cols;
         int cur_blk, cur_slot, nxt_blk = -1, nxt_slot = -1;
         load_window(c0, cur_blk, cur_slot);
-        int s = 0;
-        uint32_t ph = 1;                                             // parity of the "empty" phase to wait for
-        for (int i = 0; i < n_tiles && alive; ++i, ph ^= (s + 1 == kLyStages), s = (s + 1 == kLyStages) ? 0 : s + 1) {
+        for (int i = 0; i < tpr && alive; ++i, ++gi, ph ^= (s + 1 == kLyStages), s = (s + 1 == kLyStages) ? 0 : s + 1) {
             if ((i & 7) == 0) {
                 if (i > 0) { cur_blk = nxt_blk; cur_slot = nxt_slot; }
                 load_window(c0 + (i + 8) * kAtTileCols, nxt_blk, nxt_slot);
@@ -263,7 +270,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             int blk = __shfl_sync(0xffffffffu, cur_blk, src_lane);
             const int slot = __shfl_sync(0xffffffffu, cur_slot, src_lane);
             if (lane >= kAtTileCols) blk = -1;
-            if (lane == 0 && i < kLyStages) {
+            if (lane == 0 && gi < kLyStages) {
                 // first use of this stage: the scoring tiles that last used its 64 KiB pair must have been consumed
                 const int pr = s >> 1;
                 const int uses = it > pr ? (it - pr + kLyPairs - 1) / kLyPairs : 0;
@@ -290,6 +297,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             __syncwarp();
             if (lane < kAtTileCols && blk >= 0)                       // the whole 8 KiB entry in one copy
                 tma_load_5d(kv_u32 + s * kAtStageBytes + lane * kEntryBytes, &tmap, 0, 0, 2 * slot, 0, 0, bar_full(s));
+        }
         }
     } else if (warp == 1) {
         {
@@ -340,11 +348,14 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAtTileKeys >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
             // descriptors: the operand start address occupies the low 14 bits (16-byte units), so offsets are added there
             const uint64_t k_desc0 = smem_desc_sw128_k(kv_u32, kImgGroup);
-            bool alive = n_tiles == 0 || mbar_wait(bar_q, 0, p.err, 55);          // Q is in tensor memory
-            tc_fence_after();
+            bool alive = true;
             int s = 0, sb = 0, s_old = 0;                            // stage and S buffer of tile i; stage of tile i - kAtSBufs
             uint32_t ph = 0, ph_old = 0;
-            for (int i = 0; i < n_tiles && alive; ++i) {
+            int i = 0;                                               // index of the tile among all rows of this CTA
+            for (int k = 0; k < n_my_rows && alive; ++k) {
+            alive = mbar_wait(bar_q, (uint32_t)(k & 1), p.err, 55);  // the row's Q is in tensor memory
+            tc_fence_after();
+            for (int it = 0; it < tpr && alive; ++it, ++i) {
                 // the S buffer also held P of tile i - kAtSBufs: its P V must have completed
                 if (i >= kAtSBufs) {
                     alive = mbar_wait(bar_empty(s_old), ph_old, p.err, 51);
@@ -367,6 +378,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 s = (s + 1 == kLyStages) ? 0 : s + 1;
                 sb = (sb + 1) & (kAtSBufs - 1);
             }
+            }
         }
     } else if (warp == 2) {
         // ---------------------------------------------------------------- P V issuer
@@ -376,7 +388,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             bool alive = true;
             int s = 0, sb = 0;
             uint32_t ph_p = 0;
-            for (int i = 0; i < n_tiles && alive; ++i) {
+            for (int k = 0; k < n_my_rows && alive; ++k)
+            for (int it = 0; it < tpr && alive; ++it) {
                 alive = mbar_wait(bar_p_full(sb), ph_p, p.err, 53);
                 if (!alive) break;
                 tc_fence_after();
@@ -385,7 +398,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
 #pragma unroll
                 for (int ks = 0; ks < kAtTileCols; ++ks)               // 16 keys per MMA = one block image
                     tc_mma_bf16_ts(tmem_o, p_tmem + ks * 8, v_desc + (uint64_t)((ks * kEntryBytes) >> 4), idesc_pv,
-                                   (i | ks) ? 1u : 0u);
+                                   (it | ks) ? 1u : 0u);             // O starts afresh with every row
                 tc_commit(bar_empty(s));                             // stage free, and O complete up to this tile
                 s = (s + 1 == kLyStages) ? 0 : s + 1;
                 sb = (sb + 1) & (kAtSBufs - 1);
@@ -420,7 +433,6 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         const bool has_row = lane < LANES;
         const bool live_row = has_row && row < p.R;
         const bool live_warp = (quarter * LANES) % RPC < p.R;       // some lane of this warp holds a query row
-        const int limit = live_row ? L + row / p.G : -1;            // last visible position of this row
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         {
             // ---------------------------------------------------------------- scoring phase: epilogue
@@ -462,7 +474,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         // ---- attention phase: this thread's Q row goes to its tensor-memory lane (rows are replicated across the copies, rows
         // past R are zero); q may come from the previous layer: wait for it (no-op without a programmatic launch)
         asm volatile("griddepcontrol.wait;" ::: "memory");
-        if (cta_has_row) {
+        auto load_q = [&](int bh) {
+            const int b = bh / p.Hkv, h = bh % p.Hkv;
             uint4 v[16];
 #pragma unroll
             for (int c = 0; c < 16; ++c) v[c] = make_uint4(0, 0, 0, 0);
@@ -484,12 +497,17 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_q);
-        }
-        float m_ref = -CUDART_INF_F, l_sum = 0.f;
+        };
+        if (cta_has_row) load_q(my_row(0));
         bool alive = true;
         int s = 0, s_prev = 0;                                      // ring stage of tile i and of tile i - 1
         uint32_t ph_prev = 0;                                       // parity of the "empty" phase that ends tile i - 1
-        for (int i = 0; i < n_tiles && alive; ++i) {
+        int i = 0;                                                  // index of the tile among all rows of this CTA
+        for (int k = 0; k < n_my_rows; ++k) {
+        const int bh = my_row(k), b = bh / p.Hkv, h = bh % p.Hkv;
+        const int limit = live_row ? (k == 0 ? L0 : p.seq_len[b]) + row / p.G : -1;     // last visible position of this row
+        float m_ref = -CUDART_INF_F, l_sum = 0.f;
+        for (int it = 0; it < tpr && alive; ++it, ++i) {
             alive = mbar_wait(bar_s_full(i % kAtSBufs), (i / kAtSBufs) & 1, p.err, 61);
             if (!alive) break;
             tc_fence_after();
@@ -537,13 +555,13 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                     // the O rows must be complete up to tile i-1 before they are rescaled
                     // (its stage is released by the commit that follows that P V; with at least four stages in the
                     // ring the phase parity of that barrier is unambiguous)
-                    if (i > 0) alive = mbar_wait(bar_empty(s_prev), ph_prev, p.err, 62);
+                    if (it > 0) alive = mbar_wait(bar_empty(s_prev), ph_prev, p.err, 62);
                     tc_fence_after();
                     const float m_new = raise ? mxs : m_ref;
                     const float alpha = m_new == -CUDART_INF_F ? 1.f : fast_exp2(m_ref - m_new);
                     m_ref = m_new;
                     l_sum *= alpha;
-                    if (i > 0) {
+                    if (it > 0) {
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
                             uint32_t v[16];
@@ -590,9 +608,12 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             s_prev = s;
             s = (s + 1 == kLyStages) ? 0 : s + 1;
         }
-        // ---- write the attention row out: merge the copies, normalise ------------------------------------------
-        if (cta_has_row) {
-            if (alive) alive = mbar_wait(bar_empty((n_tiles - 1) % kLyStages), ((n_tiles - 1) / kLyStages) & 1, p.err, 63);
+        // ---- Q of the CTA's next row goes to tensor memory first (this warp has seen S of the row's last tile, so
+        // every Q K^T of the row has completed), then the row is written out: merge the copies, normalise.  The
+        // next row's first P V, which overwrites O, needs P of that tile from these warps, so it comes later.
+        {
+            if (MULTI && alive && k + 1 < n_my_rows) load_q(my_row(k + 1));
+            if (alive) alive = mbar_wait(bar_empty(s_prev), ph_prev, p.err, 63);   // the row's last P V has completed
             tc_fence_after();
             // From here on the four softmax warps meet at named barriers, which have no time-out: go on only if
             // none of them has given up (every thread gets here, because all its waits above are bounded).
@@ -669,6 +690,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                     if (live_row) emit(row, rd * 16, acc, m_ref, l_sum);
                 }
             }
+            if (!alive) break;
+        }
         }
     }
 
@@ -689,8 +712,9 @@ static size_t layer_tc_smem_bytes(int mma_m, int copies, int N)
            (size_t)mma_m * ((copies > 1 ? 20 : 0) + 2) * sizeof(float) + 512;
 }
 
-// Whether the fused launch takes these shapes: every (request, KV head) row an SM of its own and more rows than
-// half the SMs, the scoring accumulators beside the attention's tensor memory, everything within shared memory.
+// Whether the fused launch takes these shapes: more (request, KV head) rows than half the SMs (with fewer the
+// attention wants its column lists split), the scoring accumulators beside the attention's tensor memory,
+// everything within shared memory.  With more rows than SMs a CTA attends rows c, c + grid, c + 2 grid, ...
 static bool layer_tc_supported(const oasis_dims_t *dims, int n_q_tokens, int n_draft, size_t *smem_out)
 {
     const int G = dims->n_q_heads / dims->n_kv_heads;
@@ -701,7 +725,7 @@ static bool layer_tc_supported(const oasis_dims_t *dims, int n_q_tokens, int n_d
     const int mma_m = R <= 32 ? 64 : 128, copies = R <= 16 ? 4 : (R <= 64 ? 2 : 1);
     const size_t smem = layer_tc_smem_bytes(mma_m, copies, N);
     if (smem_out) *smem_out = smem;
-    return R >= 1 && R <= 128 && Rs >= 1 && Rs <= 32 && rows <= sms && rows * 2 > sms && smem <= 227 * 1024;
+    return R >= 1 && R <= 128 && Rs >= 1 && Rs <= 32 && rows * 2 > sms && rows <= 0x7fffffffLL && smem <= 227 * 1024;
 }
 
 }  // namespace oasis
@@ -735,7 +759,7 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     if (q_batch_stride == 0) q_batch_stride = (int64_t)n_draft * dims->n_q_heads * kHeadDim;
     if ((q_batch_stride * 2) % 16 != 0) return fail(OASIS_ERR_INVALID_ARG, "%s: q_batch_stride %lld", who, (long long)q_batch_stride);
     if (dims->batch == 0) return OASIS_OK;
-    // The fused launch covers the shapes where every (request, KV head) row gets an SM of its own and the scoring
+    // The fused launch covers the shapes with more (request, KV head) rows than half the SMs whose scoring
     // accumulators fit beside the attention's tensor memory; other shapes take the two separate calls.
     const long long rows = (long long)dims->batch * dims->n_kv_heads;
     const int sms = sm_count();
@@ -782,14 +806,24 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     p.reduce_sum = reduce_mode == OASIS_REDUCE_SUM;
     p.total_tiles = rows * p.tiles_per_bh;
     p.err = error_word();
-    // Equal bytes per SM: an attention tile is 32 KiB, a scoring tile 64 KiB.
+    // Equal bytes per SM: an attention tile is 32 KiB, a scoring tile 64 KiB.  The first `n_more` CTAs attend
+    // one row more than the others and take correspondingly fewer scoring tiles.
     const int grid = sms;
     const double nt_a = (n_cols + kAtTileCols - 1) / kAtTileCols;
-    const double units = ((double)rows * nt_a + 2.0 * (double)p.total_tiles) / grid;
-    double w_row = (units - nt_a) / 2.0;
-    if (w_row < 0.0) w_row = 0.0;
-    p.w_row = grid > rows ? w_row : (double)p.total_tiles / (double)rows;
-    p.w_free = grid > rows ? ((double)p.total_tiles - (double)rows * p.w_row) / (double)(grid - rows) : 0.0;
+    const long long m_rows = rows / grid;
+    const int rem = (int)(rows % grid);
+    if (rem == 0) {
+        p.n_more = grid;
+        p.w_row = (double)p.total_tiles / (double)grid;
+        p.w_free = 0.0;
+    } else {
+        const double units = ((double)rows * nt_a + 2.0 * (double)p.total_tiles) / grid;
+        double w_more = (units - (double)(m_rows + 1) * nt_a) / 2.0;
+        if (w_more < 0.0) w_more = 0.0;
+        p.n_more = rem;
+        p.w_row = w_more;
+        p.w_free = ((double)p.total_tiles - (double)rem * w_more) / (double)(grid - rem);
+    }
     cudaError_t e;
     cudaStream_t st = (cudaStream_t)stream;
     // Programmatic dependent launch: behind another launch of this kernel on the same stream the thread blocks start
@@ -805,16 +839,22 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-#define OASIS_LAYER_TC_LAUNCH(M, C)                                                                              \
-    do {                                                                                                         \
-        e = cudaFuncSetAttribute(layer_tc_kernel<M, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
-        if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, layer_tc_kernel<M, C>, tmap_kv, tmap_summ, p);         \
+#define OASIS_LAYER_TC_LAUNCH_1(M, C, MU)                                                                            \
+    do {                                                                                                             \
+        e = cudaFuncSetAttribute(layer_tc_kernel<M, C, MU>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
+        if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, layer_tc_kernel<M, C, MU>, tmap_kv, tmap_summ, p);         \
+    } while (0)
+#define OASIS_LAYER_TC_LAUNCH(M, C)                      \
+    do {                                                 \
+        if (rows > grid) OASIS_LAYER_TC_LAUNCH_1(M, C, true); \
+        else OASIS_LAYER_TC_LAUNCH_1(M, C, false);       \
     } while (0)
     if (R <= 16) OASIS_LAYER_TC_LAUNCH(64, 4);
     else if (R <= 32) OASIS_LAYER_TC_LAUNCH(64, 2);
     else if (R <= 64) OASIS_LAYER_TC_LAUNCH(128, 2);
     else OASIS_LAYER_TC_LAUNCH(128, 1);
 #undef OASIS_LAYER_TC_LAUNCH
+#undef OASIS_LAYER_TC_LAUNCH_1
     if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "%s: launch with %zu B of shared memory: %s", who, smem, cudaGetErrorString(e));
     return check_launch(who);
 }

@@ -451,12 +451,14 @@ def test_error_word_registration(gpu):
 @pytest.mark.parametrize("B,Hq,Hkv,Td,nd,ctx,k", [(16, 32, 8, 4, 4, 2064, 24), (10, 32, 8, 2, 2, 1296, 16),
                                                   (12, 64, 8, 1, 1, 1040, 9), (10, 64, 8, 2, 2, 784, 20),
                                                   (16, 64, 8, 8, 4, 784, 20), (18, 16, 8, 4, 4, 3088, 40),
-                                                  (16, 32, 8, 1, 1, 528, 40)])
+                                                  (16, 32, 8, 1, 1, 528, 40), (20, 32, 8, 4, 4, 1040, 24),
+                                                  (38, 32, 8, 2, 2, 784, 9), (37, 32, 8, 1, 1, 528, 3),
+                                                  (24, 64, 8, 4, 2, 784, 20), (19, 128, 8, 6, 2, 528, 12)])
 def test_fused_attention_and_scoring_equals_the_two_calls(oracle, gpu, B, Hq, Hkv, Td, nd, ctx, k):
     """oasis_attn_and_score is steps 4 and 1 in one launch with unchanged arithmetic: outputs, log-sum-exps and
     scores must equal those of oasis_sparse_attn and oasis_score_blocks bit for bit (the separate calls are the
-    ones checked against the oracle everywhere else), for 76-148 rows, ragged lengths and every row-count variant
-    (nd = draft tokens that score)."""
+    ones checked against the oracle everywhere else), for 76 to 304 rows (none to three per thread block, evenly
+    and unevenly spread), ragged lengths and every row-count variant (nd = draft tokens that score)."""
     binding, pipeline = gpu
     dev = torch.device("cuda")
     cfg = synth.scaled(synth.C1, batch=B, n_q_heads=Hq, n_kv_heads=Hkv, context=ctx, k_blocks=k, n_draft=Td)
