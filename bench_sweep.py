@@ -229,7 +229,7 @@ def section_shapes(args, dev, hbm_peak):
                "score_us": round(t_score, 1), "score_frac": round(sb / t_score / 1e3 / hbm_peak, 3),
                "select_us": round(t_sel, 1), "attn_us": round(t_attn, 1),
                "attn_frac": round(ab / t_attn / 1e3 / hbm_peak, 3), "layer_us": None, "layer_frac": None}
-        if binding.attn_and_score_supported(Ls[0].dims, T, Td):
+        if binding.attn_and_score_supported(Ls[0].dims, T, Ls[0].cols, Td):
             def fused(i):
                 L = Ls[i]
                 binding.attn_and_score(L.dims, q, T, L.pool, L.slot_tbl, L.sel, L.cols, seq, L.scale, L.out, q[:, 1:], Td,

@@ -182,8 +182,9 @@ size_t oasis_attn_workspace_bytes(const oasis_dims_t *dims, int32_t n_q_tokens,
  * (q_draft .. scores); no workspace is needed.  One persistent thread block per SM scores its share of
  * the layer's blocks and attends (request, KV head) rows c, c + SMs, c + 2 SMs, ... over the same
  * shared-memory ring, the shares sized so that every SM moves the same number of bytes.
- * Only shapes with  B * Hkv > SMs / 2,  n_q_tokens * (Hq/Hkv) <= 128,  n_draft * (Hq/Hkv) <= 32
- * and a shared-memory footprint within 227 KiB are taken (oasis_attn_and_score_supported tells); others
+ * Only shapes with  n_q_tokens * (Hq/Hkv) <= 128,  n_draft * (Hq/Hkv) <= 64,  a shared-memory footprint
+ * within 227 KiB and attention rows that do not make stragglers (B * Hkv > SMs / 2, or rows of at most 1.25
+ * times an SM's equal share of the launch's bytes) are taken (oasis_attn_and_score_supported tells); others
  * return OASIS_ERR_UNSUPPORTED: make the two calls.
  *   q_batch_stride   elements between consecutive requests of q_draft (0 = dense)
  */
@@ -194,7 +195,8 @@ int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int32_t n_q_to
                          const int32_t *n_full_blocks, int32_t reduce_mode, float *scores, void *stream);
 
 /* 1 if oasis_attn_and_score takes these shapes on the current device, else 0. */
-int oasis_attn_and_score_supported(const oasis_dims_t *dims, int32_t n_q_tokens, int32_t n_draft);
+int oasis_attn_and_score_supported(const oasis_dims_t *dims, int32_t n_q_tokens, int32_t n_cols,
+                                   int32_t n_draft);
 
 /*
  * Sparse attention with built-in scratch memory.  (This entry point has no counterpart in the

@@ -82,7 +82,7 @@ def lib():
         L.oasis_attn_and_score.argtypes = [dp, vp, i32, vp, vp, vp, i32, vp, ctypes.c_float, vp, vp, vp, ctypes.c_int64, i32, vp, vp,
                                            i32, vp, vp]
         L.oasis_attn_and_score.restype = ctypes.c_int
-        L.oasis_attn_and_score_supported.argtypes = [dp, i32, i32]
+        L.oasis_attn_and_score_supported.argtypes = [dp, i32, i32, i32]
         L.oasis_attn_and_score_supported.restype = ctypes.c_int
         L.oasis_union_blocks.restype = ctypes.c_int
         L.oasis_set_error_word.argtypes = [vp]
@@ -225,10 +225,10 @@ def attn_and_score(dims, q, n_q_tokens, hbm_pool, slot_tbl, blk_tbl, n_cols, seq
         int(reduce_mode), _ptr(scores, torch.float32, "scores"), _stream(stream)), "oasis_attn_and_score")
 
 
-def attn_and_score_supported(dims, n_q_tokens, n_draft) -> bool:
+def attn_and_score_supported(dims, n_q_tokens, n_cols, n_draft) -> bool:
     """Whether oasis_attn_and_score takes these shapes on the current device."""
     d = dims.c()
-    return bool(lib().oasis_attn_and_score_supported(ctypes.byref(d), int(n_q_tokens), int(n_draft)))
+    return bool(lib().oasis_attn_and_score_supported(ctypes.byref(d), int(n_q_tokens), int(n_cols), int(n_draft)))
 
 
 def static_scratch_bytes() -> int:

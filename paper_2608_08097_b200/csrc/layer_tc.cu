@@ -39,13 +39,11 @@
 namespace oasis {
 
 constexpr int kLyThreads = 256;
-constexpr int kLyStages = 6;                                // 32 KiB stages (attention); three 64 KiB pairs (scoring)
-constexpr int kLyPairs = kLyStages / 2;
+constexpr int kLyMaxStages = 6;                             // 32 KiB stages (attention) = three 64 KiB pairs (scoring)
 constexpr int kLyTileBlocks = 128;                          // summaries per scoring tile
 constexpr int kLyATileBytes = kLyTileBlocks * kSummaryBytes;   // 64 KiB
 constexpr int kLySubTileBytes = kLyTileBlocks * 128;        // one 64-element K chunk of a scoring tile: 16 KiB
-constexpr int kLyTmemCols = 512;                            // S [0,256), O [256,384), Q [384,448), scoring accumulators [448,512)
-constexpr int kLyAccCol = 448;
+constexpr int kLyTmemCols = 512;                            // S [0,256), O [256,384), Q [384,448), narrow scoring accumulators [448,512)
 
 struct LayerTcParams {
     // attention phase
@@ -64,16 +62,20 @@ struct LayerTcParams {
     const int32_t *n_full;
     float *scores;
     int Rs, N, max_blocks, tiles_per_bh, reduce_sum;
+    int acc_col;                // first tensor-memory column of the two scoring accumulators
     long long total_tiles;
     double w_row, w_free;       // scoring tiles of a CTA with the larger / the smaller number of attention rows
     int32_t *err;
 };
 
-template <int MMA_M, int COPIES, bool MULTI>                // MULTI: more rows than thread blocks, several rows per block
+// MULTI: more rows than thread blocks, several rows per block.  STAGES: 32 KiB stages of the ring (6, or 4 where the
+// scoring operands or the copy-merge staging need the room).
+template <int MMA_M, int COPIES, bool MULTI, int STAGES>
 __global__ void __launch_bounds__(kLyThreads, 1)
 layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap_summ,
                 const LayerTcParams p)
 {
+    constexpr int kLyStages = STAGES, kLyPairs = STAGES / 2;
     constexpr int RPC = MMA_M / COPIES;                     // MMA rows per copy of the query rows
     constexpr int LANES = MMA_M / 4;                        // lanes of each softmax warp that hold an MMA row
     constexpr int BPC = kAtTileCols / COPIES;               // blocks of a tile each copy handles
@@ -83,7 +85,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t kv_u32 = base;                                    // [6][32 KiB] = [3][64 KiB]
+    const uint32_t kv_u32 = base;                                    // [STAGES][32 KiB] = [STAGES / 2][64 KiB]
     const uint32_t b_bytes = (uint32_t)p.N * kSummaryBytes;
     const uint32_t b_u32 = kv_u32 + kLyStages * kAtStageBytes;       // [2][N][512 B] as 4 sub-tiles of N x 128 B
     uint8_t *b_ptr = base_ptr + (size_t)kLyStages * kAtStageBytes;
@@ -106,7 +108,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     auto bar_b_full = [&](int a) { return bar_u32 + 8u * (kB0 + 2 * kLyPairs + 4 + a); };
     auto bar_b_empty = [&](int a) { return bar_u32 + 8u * (kB0 + 2 * kLyPairs + 6 + a); };
     const uint32_t bar_q = bar_u32 + 8u * (kB0 + 2 * kLyPairs + 8);  // Q is in tensor memory
-    constexpr int kNBars = kB0 + 2 * kLyPairs + 9;                   // 35
+    constexpr int kNBars = kB0 + 2 * kLyPairs + 9;                   // 35 with six stages
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 8 * kNBars);
     int32_t *tile_blk = reinterpret_cast<int32_t *>(misc + 8 * kNBars + 16);   // [stages][4]
 
@@ -325,7 +327,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                             mbar_wait(sbar_full(s), (it / kLyPairs) & 1, p.err, 23);
                     if (!alive) break;
                     tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + kLyAccCol + (uint32_t)(acc * p.N);
+                    const uint32_t d_tmem = tmem_base + (uint32_t)p.acc_col + (uint32_t)(acc * p.N);
                     const uint32_t a_tile = kv_u32 + s * kLyATileBytes;
                     const uint32_t b_tile = b_u32 + (bo % 2) * b_bytes;
     #pragma unroll
@@ -453,7 +455,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 alive = mbar_wait(bar_acc_full(acc), (it >> 1) & 1, p.err, 31);
                 if (!alive) break;
                 tc_fence_after();
-                const uint32_t taddr = tmem_base + kLyAccCol + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.N);
+                const uint32_t taddr = tmem_base + (uint32_t)p.acc_col + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.N);
                 float res = p.reduce_sum ? 0.f : -CUDART_INF_F;
                 for (int c = 0; c < p.N; c += 16) {
                     uint32_t v[16];
@@ -706,35 +708,59 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
 
 // ---- host side -----------------------------------------------------------------------------------------
 
-static size_t layer_tc_smem_bytes(int mma_m, int copies, int N)
+static size_t layer_tc_smem_bytes(int mma_m, int copies, int N, int stages)
 {
-    return 1024 + (size_t)kLyStages * kAtStageBytes + 2 * (size_t)N * kSummaryBytes +
+    return 1024 + (size_t)stages * kAtStageBytes + 2 * (size_t)N * kSummaryBytes +
            (size_t)mma_m * ((copies > 1 ? 20 : 0) + 2) * sizeof(float) + 512;
 }
 
-// Whether the fused launch takes these shapes: more (request, KV head) rows than half the SMs (with fewer the
-// attention wants its column lists split), the scoring accumulators beside the attention's tensor memory,
-// everything within shared memory.  With more rows than SMs a CTA attends rows c, c + grid, c + 2 grid, ...
-static bool layer_tc_supported(const oasis_dims_t *dims, int n_q_tokens, int n_draft, size_t *smem_out)
+struct LayerTcPlan {
+    int R, Rs, N, mma_m, copies, stages;
+    size_t smem;
+};
+
+// Whether the fused launch takes these shapes, and with which variant.  Wanted: at most 128 attention rows and 64
+// scoring rows per KV head (two accumulators of up to 32 columns fit beside the attention's tensor memory, wider
+// ones take the place of the S buffers, which the attention phase only touches after the last scoring epilogue);
+// a footprint within 227 KiB with six ring stages, or with four for the 128-row variants; and attention rows that
+// do not make stragglers: more rows than half the SMs, or rows whose tiles stay within 1.25 times an SM's equal
+// share of the launch (with fewer and longer rows the attention wants its column lists split over several SMs).
+// With more rows than SMs a CTA attends rows c, c + grid, c + 2 grid, ...
+static bool layer_tc_plan(const oasis_dims_t *dims, int n_q_tokens, int n_cols, int n_draft, LayerTcPlan *out)
 {
+    LayerTcPlan pl;
     const int G = dims->n_q_heads / dims->n_kv_heads;
-    const int R = n_q_tokens * G, Rs = n_draft * G;
+    pl.R = n_q_tokens * G;
+    pl.Rs = n_draft * G;
     const long long rows = (long long)dims->batch * dims->n_kv_heads;
     const int sms = sm_count();
-    const int N = (Rs + 15) / 16 * 16;
-    const int mma_m = R <= 32 ? 64 : 128, copies = R <= 16 ? 4 : (R <= 64 ? 2 : 1);
-    const size_t smem = layer_tc_smem_bytes(mma_m, copies, N);
-    if (smem_out) *smem_out = smem;
-    return R >= 1 && R <= 128 && Rs >= 1 && Rs <= 32 && rows * 2 > sms && rows <= 0x7fffffffLL && smem <= 227 * 1024;
+    pl.N = (pl.Rs + 15) / 16 * 16;
+    pl.mma_m = pl.R <= 32 ? 64 : 128;
+    pl.copies = pl.R <= 16 ? 4 : (pl.R <= 64 ? 2 : 1);
+    pl.stages = kLyMaxStages;
+    pl.smem = layer_tc_smem_bytes(pl.mma_m, pl.copies, pl.N, pl.stages);
+    if (pl.smem > 227 * 1024 && pl.mma_m == 128) {
+        pl.stages = 4;
+        pl.smem = layer_tc_smem_bytes(pl.mma_m, pl.copies, pl.N, pl.stages);
+    }
+    if (out) *out = pl;
+    if (pl.R < 1 || pl.R > 128 || pl.Rs < 1 || pl.Rs > 64 || n_cols < 1 || rows < 1 || rows > 0x7fffffffLL ||
+        pl.smem > 227 * 1024)
+        return false;
+    if (rows * 2 > sms) return true;
+    const double nt_a = (n_cols + kAtTileCols - 1) / kAtTileCols;
+    const double tiles_s = (double)rows * ((dims->max_blocks + kLyTileBlocks - 1) / kLyTileBlocks);
+    const double share = ((double)rows * nt_a + 2.0 * tiles_s) / sms;     // 32 KiB units per SM
+    return nt_a <= 1.25 * share;
 }
 
 }  // namespace oasis
 
-extern "C" int oasis_attn_and_score_supported(const oasis_dims_t *dims, int32_t n_q_tokens, int32_t n_draft)
+extern "C" int oasis_attn_and_score_supported(const oasis_dims_t *dims, int32_t n_q_tokens, int32_t n_cols, int32_t n_draft)
 {
     using namespace oasis;
-    if (check_dims(dims) != OASIS_OK || n_q_tokens < 1 || n_draft < 1 || dims->batch == 0) return 0;
-    return layer_tc_supported(dims, n_q_tokens, n_draft, nullptr) ? 1 : 0;
+    if (check_dims(dims) != OASIS_OK || n_q_tokens < 1 || n_cols < 1 || n_draft < 1 || dims->batch == 0) return 0;
+    return layer_tc_plan(dims, n_q_tokens, n_cols, n_draft, nullptr) ? 1 : 0;
 }
 
 extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int32_t n_q_tokens, const void *hbm_pool,
@@ -755,20 +781,19 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     if (reduce_mode != OASIS_REDUCE_MAX && reduce_mode != OASIS_REDUCE_SUM)
         return fail(OASIS_ERR_INVALID_ARG, "%s: reduce_mode %d", who, reduce_mode);
     const int G = dims->n_q_heads / dims->n_kv_heads;
-    const int R = n_q_tokens * G, Rs = n_draft * G;
     if (q_batch_stride == 0) q_batch_stride = (int64_t)n_draft * dims->n_q_heads * kHeadDim;
     if ((q_batch_stride * 2) % 16 != 0) return fail(OASIS_ERR_INVALID_ARG, "%s: q_batch_stride %lld", who, (long long)q_batch_stride);
     if (dims->batch == 0) return OASIS_OK;
-    // The fused launch covers the shapes with more (request, KV head) rows than half the SMs whose scoring
-    // accumulators fit beside the attention's tensor memory; other shapes take the two separate calls.
+    // Shapes outside the fused launch (see layer_tc_plan) take the two separate calls.
     const long long rows = (long long)dims->batch * dims->n_kv_heads;
     const int sms = sm_count();
-    const int N = (Rs + 15) / 16 * 16;
-    size_t smem = 0;
-    if (!layer_tc_supported(dims, n_q_tokens, n_draft, &smem))
+    LayerTcPlan pl;
+    if (!layer_tc_plan(dims, n_q_tokens, n_cols, n_draft, &pl))
         return fail(OASIS_ERR_UNSUPPORTED,
-                    "%s: %lld rows on %d SMs, %d attention rows and %d scoring rows per KV head are outside the fused "
-                    "launch; call oasis_sparse_attn and oasis_score_blocks", who, rows, sms, R, Rs);
+                    "%s: %lld rows of %d columns on %d SMs, %d attention rows and %d scoring rows per KV head are outside "
+                    "the fused launch; call oasis_sparse_attn and oasis_score_blocks", who, rows, n_cols, sms, pl.R, pl.Rs);
+    const int R = pl.R, Rs = pl.Rs, N = pl.N;
+    const size_t smem = pl.smem;
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return fail(OASIS_ERR_CUDA, "%s: cuTensorMapEncodeTiled is not available", who);
     CUtensorMap tmap_kv, tmap_summ;
@@ -802,6 +827,7 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     p.n_cols = n_cols; p.R = R; p.rows = (int)rows;
     p.q_draft = (const uint8_t *)q_draft; p.q_batch_stride = q_batch_stride; p.n_full = n_full_blocks; p.scores = scores;
     p.Rs = Rs; p.N = N; p.max_blocks = dims->max_blocks;
+    p.acc_col = N <= 32 ? 448 : 0;
     p.tiles_per_bh = (dims->max_blocks + kLyTileBlocks - 1) / kLyTileBlocks;
     p.reduce_sum = reduce_mode == OASIS_REDUCE_SUM;
     p.total_tiles = rows * p.tiles_per_bh;
@@ -839,22 +865,24 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-#define OASIS_LAYER_TC_LAUNCH_1(M, C, MU)                                                                            \
-    do {                                                                                                             \
-        e = cudaFuncSetAttribute(layer_tc_kernel<M, C, MU>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
-        if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, layer_tc_kernel<M, C, MU>, tmap_kv, tmap_summ, p);         \
+#define OASIS_LAYER_TC_LAUNCH_2(M, C, MU, ST)                                                                            \
+    do {                                                                                                                 \
+        e = cudaFuncSetAttribute(layer_tc_kernel<M, C, MU, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
+        if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, layer_tc_kernel<M, C, MU, ST>, tmap_kv, tmap_summ, p);         \
     } while (0)
-#define OASIS_LAYER_TC_LAUNCH(M, C)                      \
-    do {                                                 \
-        if (rows > grid) OASIS_LAYER_TC_LAUNCH_1(M, C, true); \
-        else OASIS_LAYER_TC_LAUNCH_1(M, C, false);       \
+#define OASIS_LAYER_TC_LAUNCH(M, C, ST)                          \
+    do {                                                         \
+        if (rows > grid) OASIS_LAYER_TC_LAUNCH_2(M, C, true, ST); \
+        else OASIS_LAYER_TC_LAUNCH_2(M, C, false, ST);           \
     } while (0)
-    if (R <= 16) OASIS_LAYER_TC_LAUNCH(64, 4);
-    else if (R <= 32) OASIS_LAYER_TC_LAUNCH(64, 2);
-    else if (R <= 64) OASIS_LAYER_TC_LAUNCH(128, 2);
-    else OASIS_LAYER_TC_LAUNCH(128, 1);
+    if (R <= 16) OASIS_LAYER_TC_LAUNCH(64, 4, 6);
+    else if (R <= 32) OASIS_LAYER_TC_LAUNCH(64, 2, 6);
+    else if (R <= 64 && pl.stages == 6) OASIS_LAYER_TC_LAUNCH(128, 2, 6);
+    else if (R <= 64) OASIS_LAYER_TC_LAUNCH(128, 2, 4);
+    else if (pl.stages == 6) OASIS_LAYER_TC_LAUNCH(128, 1, 6);
+    else OASIS_LAYER_TC_LAUNCH(128, 1, 4);
 #undef OASIS_LAYER_TC_LAUNCH
-#undef OASIS_LAYER_TC_LAUNCH_1
+#undef OASIS_LAYER_TC_LAUNCH_2
     if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "%s: launch with %zu B of shared memory: %s", who, smem, cudaGetErrorString(e));
     return check_launch(who);
 }

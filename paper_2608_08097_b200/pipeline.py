@@ -125,7 +125,7 @@ class DecodeEngine:
         self.copy = torch.cuda.Stream(device=self.device)     # end-to-end mode: query upload, output download
         self.launches = 0
         self.cap = cap
-        can_fuse = n_layers > 0 and n_q_tokens > 1 and oasis.attn_and_score_supported(self.layers[0].dims, n_q_tokens, n_q_tokens - 1)
+        can_fuse = n_layers > 0 and n_q_tokens > 1 and oasis.attn_and_score_supported(self.layers[0].dims, n_q_tokens, self.layers[0].cols, n_q_tokens - 1)
         self.fused = can_fuse if fused is None else (bool(fused) and can_fuse)
         self.stage_done = [None] * n_layers          # event of the layer's latest transfer
         if mode == "delta":
