@@ -5,7 +5,9 @@
 // with a bitonic sort of (empty first, last-selected step, column) keys; the candidates keep
 // their rank order through a ballot/prefix-sum compaction; the first min(cap, candidates,
 // targets) pairs are applied to the resident table and emitted as gather requests.
-// Integer work on a few hundred elements per row: latency bound, no roofline to speak of.
+// Integer work on a few hundred elements per row: latency bound, no roofline to speak of.  The loops are kept
+// rolled: the kernel shares SMs with the attention / scoring kernel, whose instruction fetches a large
+// co-resident kernel slows down.
 #include "common.cuh"
 
 namespace oasis {
@@ -43,13 +45,16 @@ plan_delta_kernel(const PlanParams p)
     int32_t *stp = p.stamp + (long long)row * p.res_stride;
     const int plan_cols = p.cap + p.n_local;
 
+#pragma unroll 1
     for (int i = tid; i < 2 * p.bitmap_words; i += kPlanThreads) pred_bits[i] = 0;
     if (tid == 0) sh_n_target = 0;
     __syncthreads();
+#pragma unroll 1
     for (int r = tid; r < p.k; r += kPlanThreads) {
         const int j = pred[r];
         if (j >= 0 && j < p.max_blocks) atomicOr(&pred_bits[j >> 5], 1u << (j & 31));
     }
+#pragma unroll 1
     for (int c = tid; c < p.n_res; c += kPlanThreads) {
         const int j = res[c];
         if (j >= 0 && j < p.max_blocks) atomicOr(&res_bits[j >> 5], 1u << (j & 31));
@@ -57,6 +62,7 @@ plan_delta_kernel(const PlanParams p)
     __syncthreads();
 
     // ---- hits keep their column; everything else is an eviction target ------------------------------
+#pragma unroll 1
     for (int c = tid; c < p.sort_len; c += kPlanThreads) {
         unsigned long long key = ~0ull;                       // non-targets sort to the end
         if (c < p.n_res) {
@@ -73,8 +79,11 @@ plan_delta_kernel(const PlanParams p)
         tkey[c] = key;
     }
     __syncthreads();
+#pragma unroll 1
     for (int size = 2; size <= p.sort_len; size <<= 1) {
+#pragma unroll 1
         for (int stride = size >> 1; stride > 0; stride >>= 1) {
+#pragma unroll 1
             for (int i = tid; i < (p.sort_len >> 1); i += kPlanThreads) {
                 const int pos = 2 * i - (i & (stride - 1));
                 const unsigned long long x = tkey[pos], y = tkey[pos + stride];
@@ -91,6 +100,7 @@ plan_delta_kernel(const PlanParams p)
     // ---- candidates: predicted blocks that are not resident, in rank order -----------------------------
     uint32_t n_cand = 0;
     const int k_pad = (p.k + kPlanThreads - 1) / kPlanThreads * kPlanThreads;
+#pragma unroll 1
     for (int base = 0; base < k_pad; base += kPlanThreads) {
         const int r = base + tid;
         const int j = r < p.k ? pred[r] : -1;
@@ -117,6 +127,7 @@ plan_delta_kernel(const PlanParams p)
 
     // ---- pair candidates with targets, bounded by the cap ------------------------------------------------
     const int n_pair = min(p.cap, min((int)n_cand, (int)sh_n_target));
+#pragma unroll 1
     for (int i = tid; i < p.cap; i += kPlanThreads) {
         long long idx = -1;
         int slot = 0;
@@ -132,6 +143,7 @@ plan_delta_kernel(const PlanParams p)
         p.plan_slots[(long long)row * plan_cols + i] = slot;
     }
     // the always-kept local blocks (Sec. 4.3: selected blocks plus a local window)
+#pragma unroll 1
     for (int i = tid; i < p.n_local; i += kPlanThreads) {
         const int j = pred[p.k + i];
         res[p.n_res + i] = j;

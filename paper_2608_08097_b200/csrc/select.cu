@@ -7,7 +7,7 @@
 //      which the row's keys actually differ (warp-aggregated shared-memory histograms);
 //   3. index-ordered compaction: every key above the threshold, and the lowest-index keys
 //      equal to it until K are taken (ballot + prefix sums), so ties go to the lowest id;
-//   4. bitonic sort of the K winners by (score descending, id ascending);
+//   4. sort of the K winners by (score descending, id ascending): rank sort for up to 256, else bitonic;
 //   5. sel row, local block ids, and the optional gather lists.
 // The work is integer and shared-memory bound; it moves 4 B per block in and (k+2) * 16 B out.
 #include "common.cuh"
@@ -53,6 +53,7 @@ select_topk_kernel(const SelectParams p)
 
     // ---- 1. keys, min, max ---------------------------------------------------------------
     uint32_t lo = 0xffffffffu, hi = 0u;
+#pragma unroll 1
     for (int j = tid; j < n; j += nthreads) {
         const uint32_t key = score_key(srow[j]);
         keys[j] = key;
@@ -86,11 +87,13 @@ select_topk_kernel(const SelectParams p)
     uint32_t prefix = 0;
     uint32_t rank = (uint32_t)k_eff;              // wanted: rank-th largest among keys matching prefix
     if (k_eff > 0) {
+#pragma unroll 1
         for (int pass = npass - 1; pass >= 0; --pass) {
             const int shift = pass * 8;
             const uint32_t hi_mask = (shift + 8 >= 32) ? 0u : (0xffffffffu << (shift + 8));
             for (int i = tid; i < 256; i += nthreads) hist[i] = 0;
             __syncthreads();
+#pragma unroll 1
             for (int j = tid; j < n_pad; j += nthreads) {
                 const bool valid = j < n;
                 const uint32_t kr = valid ? keys[j] - kmin : 0u;
@@ -141,6 +144,7 @@ select_topk_kernel(const SelectParams p)
     // ---- 3. index-ordered compaction ------------------------------------------------------------
     uint32_t equal_before = 0;                    // equal keys in earlier tiles
     if (k_eff > 0) {
+#pragma unroll 1
         for (int base = 0; base < n_pad; base += nthreads) {
             const int j = base + tid;
             const bool valid = j < n;
@@ -176,54 +180,38 @@ select_topk_kernel(const SelectParams p)
             __syncthreads();                       // warp_a / warp_b / sh_rank reused by the next tile
         }
     }
+#pragma unroll 1
     for (int i = k_eff + tid; i < p.sort_len; i += nthreads) cand[i] = 0ull;   // sorts to the end
     __syncthreads();
 
-    // ---- 4. bitonic sort, descending ------------------------------------------------------------
-    if (k_eff > 1 && p.sort_len <= 128) {
-        // up to 128 winners: one warp sorts them in registers (element e = 32 * j + lane), exchanging
-        // across lanes with shuffles -- no CTA-wide barrier per stage
-        if (warp == 0) {
-            unsigned long long v[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) v[j] = (32 * j + lane < p.sort_len) ? cand[32 * j + lane] : 0ull;
-#pragma unroll
-            for (int size = 2; size <= 128; size <<= 1) {
-#pragma unroll
-                for (int stride = size >> 1; stride > 0; stride >>= 1) {
-                    if (stride >= 32) {                       // partner lives in the same lane
-                        const int dj = stride >> 5;
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            if ((j & dj) == 0) {
-                                const int e = 32 * j + lane;
-                                const bool descending = (e & size) == 0;
-                                const unsigned long long x = v[j], y = v[j | dj];
-                                if ((x < y) == descending) { v[j] = y; v[j | dj] = x; }
-                            }
-                        }
-                    } else {                                   // partner lives in lane ^ stride
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int e = 32 * j + lane;
-                            const unsigned long long other = __shfl_xor_sync(0xffffffffu, v[j], stride);
-                            const bool lower = (lane & stride) == 0;          // this lane holds the pair's first element
-                            const bool descending = (e & size) == 0;
-                            const bool keep_max = lower == descending;
-                            v[j] = keep_max ? (v[j] > other ? v[j] : other) : (v[j] < other ? v[j] : other);
-                        }
-                    }
-                }
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (32 * j + lane < p.sort_len) cand[32 * j + lane] = v[j];
+    // ---- 4. sort, descending ----------------------------------------------------------------------
+    // Plain loops over shared memory keep the code small: a large kernel that shares SMs with the attention /
+    // scoring kernel costs that kernel instruction-cache misses even where little of it executes (a fully
+    // unrolled register-resident sorting network made this kernel 75 KB and the decode step 8 % slower).
+    if (k_eff > 1 && p.sort_len <= 256 && p.max_blocks >= 2 * p.sort_len) {
+        // few winners: every thread ranks one of them against all others (the 64-bit keys are distinct) and
+        // drops it at its rank; the key array, no longer needed, is the second buffer
+        unsigned long long *sorted = reinterpret_cast<unsigned long long *>(keys);
+        __syncthreads();
+#pragma unroll 1
+        for (int i = tid; i < p.sort_len; i += nthreads) {
+            const unsigned long long mine = cand[i];
+            int rank_i = 0;
+#pragma unroll 4
+            for (int o = 0; o < p.sort_len; ++o) rank_i += cand[o] > mine;
+            if (mine != 0ull) sorted[rank_i] = mine;          // padding zeros stay behind the k_eff winners
         }
+        __syncthreads();
+#pragma unroll 1
+        for (int i = tid; i < k_eff; i += nthreads) cand[i] = sorted[i];
         __syncthreads();
     } else if (k_eff > 1) {
         const int len = p.sort_len;
+#pragma unroll 1
         for (int size = 2; size <= len; size <<= 1) {
+#pragma unroll 1
             for (int stride = size >> 1; stride > 0; stride >>= 1) {
+#pragma unroll 1
                 for (int i = tid; i < (len >> 1); i += nthreads) {
                     const int pos = 2 * i - (i & (stride - 1));
                     const unsigned long long x = cand[pos], y = cand[pos + stride];
@@ -241,6 +229,7 @@ select_topk_kernel(const SelectParams p)
     // ---- 5. outputs --------------------------------------------------------------------------------
     const int cols = p.k + 2;
     const int end_block = (p.seq_len[b] + p.n_q_tokens + kBlock - 1) / kBlock;   // exclusive
+#pragma unroll 1
     for (int c = tid; c < cols; c += nthreads) {
         int v = -1;
         if (c < k_eff) {
