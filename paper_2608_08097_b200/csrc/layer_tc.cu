@@ -63,7 +63,7 @@ struct LayerTcParams {
     float *scores;
     int Rs, N, max_blocks, tiles_per_bh, reduce_sum;
     int acc_col;                // first tensor-memory column of the two scoring accumulators
-    long long total_tiles;
+    int total_tiles;            // rows * tiles_per_bh (the host checks that summaries rows fit 31 bits)
     double w_row, w_free;       // scoring tiles of a CTA with the larger / the smaller number of attention rows
     int32_t *err;
 };
@@ -124,16 +124,17 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     // ---- scoring geometry: tiles [t0, t1) ---------------------------------------------------------
     auto tiles_before = [&](int c) {
         const double w = c <= p.n_more ? c * p.w_row : p.n_more * p.w_row + (c - p.n_more) * p.w_free;
-        long long t = (long long)w;
+        int t = (int)w;
         return t < p.total_tiles ? t : p.total_tiles;
     };
-    const long long t0 = tiles_before(blockIdx.x);
-    const long long t1 = blockIdx.x + 1 == gridDim.x ? p.total_tiles : tiles_before(blockIdx.x + 1);
+    const int t0 = tiles_before(blockIdx.x);
+    const int t1 = blockIdx.x + 1 == gridDim.x ? p.total_tiles : tiles_before(blockIdx.x + 1);
 
     // First tile at or after t (and before t1) that has candidate blocks; t1 if there is none.
-    auto next_active = [&](long long t) {
+    auto next_active = [&](int t) {
+#pragma unroll 1
         for (; t < t1; ++t) {
-            const long long sbh = t / p.tiles_per_bh;
+            const int sbh = t / p.tiles_per_bh;
             const int j0 = (int)(t % p.tiles_per_bh) * kLyTileBlocks;
             if (j0 < p.n_full[(int)(sbh / p.Hkv)]) break;
         }
@@ -142,10 +143,11 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     // (q^- | q^+) rows of one (request, KV head), K-major, 128-byte swizzle: element k of row n
     // lives in sub-tile k / 64.  `nthr` threads (index `me`) share the work; loads are issued
     // eight at a time so their latencies overlap.
-    auto build_b = [&](long long bh, int buf, int me, int nthr) {
+    auto build_b = [&](int bh, int buf, int me, int nthr) {
         const int b = (int)(bh / p.Hkv), h = (int)(bh % p.Hkv);
         uint8_t *dstb = b_ptr + (size_t)buf * b_bytes;
         const int tasks = p.N * 16;                              // 16-byte chunks of the query rows
+#pragma unroll 1
         for (int i0 = me; i0 < tasks; i0 += nthr * 8) {
             uint4 v[8];
 #pragma unroll
@@ -218,22 +220,22 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         tmem_o = tmem_base + kAtSBufs * kAtTileKeys;
         tmem_q = tmem_o + kHeadDim;                                  // Q as the A operand: 128 rows x 64 packed columns
     }
-    const long long t_first = next_active(t0);
+    const int t_first = next_active(t0);
     if (warp == 0) {
         bool alive = true;
         int it = 0;                                                  // scoring tiles issued
         {
             // ---------------------------------------------------------------- scoring phase: tiles
-            long long t = t_first;
+            int t = t_first;
             while (t < t1 && alive) {
-                const long long bh = t / p.tiles_per_bh;
+                const int bh = t / p.tiles_per_bh;
                 const int j0 = (int)(t % p.tiles_per_bh) * kLyTileBlocks;
                 if (lane == 0) {
                     const int s = it % kLyPairs;
                     alive = alive && mbar_wait(sbar_empty(s), ((it / kLyPairs) & 1) ^ 1, p.err, 12);
                     if (alive) {
                         mbar_arrive_expect_tx(sbar_full(s), kLyATileBytes);
-                        const int y = (int)(bh * p.max_blocks + j0);
+                        const int y = bh * p.max_blocks + j0;
     #pragma unroll
                         for (int kc = 0; kc < 4; ++kc)
                             tma_load_2d(kv_u32 + s * kLyATileBytes + kc * kLySubTileBytes, &tmap_summ, kc * 64, y, sbar_full(s));
@@ -241,7 +243,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 }
                 alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
                 ++it;
-                const long long tn = next_active(t + 1);
+                const int tn = next_active(t + 1);
                 t = tn;
             }
         }
@@ -258,11 +260,13 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         asm volatile("griddepcontrol.wait;" ::: "memory");
         int s = 0, gi = 0;                                           // ring stage and index of the tile among all rows
         uint32_t ph = 1;                                             // parity of the "empty" phase to wait for
+#pragma unroll 1
         for (int k = 0; k < n_my_rows && alive; ++k) {
         slot_row = p.slot_tbl + (long long)my_row(k) * p.n_cols;
         blk_row = p.blk_tbl + (long long)my_row(k) * p.n_cols;
         int cur_blk, cur_slot, nxt_blk = -1, nxt_slot = -1;
         load_window(c0, cur_blk, cur_slot);
+#pragma unroll 1
         for (int i = 0; i < tpr && alive; ++i, ++gi, ph ^= (s + 1 == kLyStages), s = (s + 1 == kLyStages) ? 0 : s + 1) {
             if ((i & 7) == 0) {
                 if (i > 0) { cur_blk = nxt_blk; cur_slot = nxt_slot; }
@@ -287,7 +291,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 if (blk < 0) {
                     // a missing block contributes P = 0, which must not meet stale NaN bit patterns in V
                     uint8_t *img = base_ptr + kAtQBytes + (size_t)s * kAtStageBytes + lane * kEntryBytes;
+#pragma unroll 1
                     for (int u = 0; u < 4; ++u)                      // (row group, dim half) units of the V part
+#pragma unroll 1
                         for (int j = 0; j < kImgPart / 16; ++j)
                             *reinterpret_cast<uint4 *>(img + (u >> 1) * kImgGroup + (u & 1) * kImgHalf + kImgPart + j * 16) =
                                 make_uint4(0, 0, 0, 0);
@@ -308,10 +314,11 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.N >> 3) << 17) |
                                        ((uint32_t)(kLyTileBlocks >> 4) << 24);
                 int it = 0, bo = -1;
-                long long cur_bh = -1;
+                int cur_bh = -1;
                 bool alive = true;
-                for (long long t = t0; t < t1 && alive; ++t) {
-                    const long long bh = t / p.tiles_per_bh;
+#pragma unroll 1
+                for (int t = t0; t < t1 && alive; ++t) {
+                    const int bh = t / p.tiles_per_bh;
                     const int j0 = (int)(t % p.tiles_per_bh) * kLyTileBlocks;
                     const int b = (int)(bh / p.Hkv);
                     if (j0 >= p.n_full[b]) continue;
@@ -354,9 +361,11 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             int s = 0, sb = 0, s_old = 0;                            // stage and S buffer of tile i; stage of tile i - kAtSBufs
             uint32_t ph = 0, ph_old = 0;
             int i = 0;                                               // index of the tile among all rows of this CTA
+#pragma unroll 1
             for (int k = 0; k < n_my_rows && alive; ++k) {
             alive = mbar_wait(bar_q, (uint32_t)(k & 1), p.err, 55);  // the row's Q is in tensor memory
             tc_fence_after();
+#pragma unroll 1
             for (int it = 0; it < tpr && alive; ++it, ++i) {
                 // the S buffer also held P of tile i - kAtSBufs: its P V must have completed
                 if (i >= kAtSBufs) {
@@ -390,7 +399,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             bool alive = true;
             int s = 0, sb = 0;
             uint32_t ph_p = 0;
+#pragma unroll 1
             for (int k = 0; k < n_my_rows && alive; ++k)
+#pragma unroll 1
             for (int it = 0; it < tpr && alive; ++it) {
                 alive = mbar_wait(bar_p_full(sb), ph_p, p.err, 53);
                 if (!alive) break;
@@ -413,9 +424,10 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         // as soon as an operand buffer is free.
         int bo = -1;
         bool alive = true;
-        long long cur_bh = -1;
-        for (long long t = t_first; t < t1 && alive; t = next_active(t + 1)) {
-            const long long bh = t / p.tiles_per_bh;
+        int cur_bh = -1;
+#pragma unroll 1
+        for (int t = t_first; t < t1 && alive; t = next_active(t + 1)) {
+            const int bh = t / p.tiles_per_bh;
             if (bh == cur_bh) continue;
             cur_bh = bh;
             ++bo;
@@ -440,13 +452,14 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             // ---------------------------------------------------------------- scoring phase: epilogue
             int it = 0;
             bool alive = true;
-            for (long long t = t0; t < t1 && alive; ++t) {
-                const long long bh = t / p.tiles_per_bh;
+#pragma unroll 1
+            for (int t = t0; t < t1 && alive; ++t) {
+                const int bh = t / p.tiles_per_bh;
                 const int j0 = (int)(t % p.tiles_per_bh) * kLyTileBlocks;
                 const int b = (int)(bh / p.Hkv);
                 const int nf = p.n_full[b];
                 const int j = j0 + quarter * 32 + lane;
-                float *out = p.scores + bh * p.max_blocks;
+                float *out = p.scores + (long long)bh * p.max_blocks;
                 if (j0 >= nf) {
                     if (j < p.max_blocks) out[j] = -CUDART_INF_F;
                     continue;
@@ -457,6 +470,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + (uint32_t)p.acc_col + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.N);
                 float res = p.reduce_sum ? 0.f : -CUDART_INF_F;
+#pragma unroll 1
                 for (int c = 0; c < p.N; c += 16) {
                     uint32_t v[16];
                     tc_ld16(taddr + c, v);
@@ -505,10 +519,12 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         int s = 0, s_prev = 0;                                      // ring stage of tile i and of tile i - 1
         uint32_t ph_prev = 0;                                       // parity of the "empty" phase that ends tile i - 1
         int i = 0;                                                  // index of the tile among all rows of this CTA
+#pragma unroll 1
         for (int k = 0; k < n_my_rows; ++k) {
         const int bh = my_row(k), b = bh / p.Hkv, h = bh % p.Hkv;
         const int limit = live_row ? (k == 0 ? L0 : p.seq_len[b]) + row / p.G : -1;     // last visible position of this row
         float m_ref = -CUDART_INF_F, l_sum = 0.f;
+#pragma unroll 1
         for (int it = 0; it < tpr && alive; ++it, ++i) {
             alive = mbar_wait(bar_s_full(i % kAtSBufs), (i / kAtSBufs) & 1, p.err, 61);
             if (!alive) break;
@@ -643,6 +659,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                     l_sm[m_row] = l_sum;
                 }
                 float mx = -CUDART_INF_F, den = 0.f, wt[COPIES];
+#pragma unroll 1
                 for (int rd = 0; rd < 8; ++rd) {
                     if (live_warp) {
                         uint32_t v[16];
@@ -683,6 +700,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                     asm volatile("bar.sync 1, 128;" ::: "memory");  // the staging rows are rewritten next round
                 }
             } else if (alive) {
+#pragma unroll 1
                 for (int rd = 0; rd < 8; ++rd) {                    // the thread's own O row, read by the whole warp
                     float acc[16];
                     uint32_t v[16];
@@ -744,8 +762,8 @@ static bool layer_tc_plan(const oasis_dims_t *dims, int n_q_tokens, int n_cols, 
         pl.smem = layer_tc_smem_bytes(pl.mma_m, pl.copies, pl.N, pl.stages);
     }
     if (out) *out = pl;
-    if (pl.R < 1 || pl.R > 128 || pl.Rs < 1 || pl.Rs > 64 || n_cols < 1 || rows < 1 || rows > 0x7fffffffLL ||
-        pl.smem > 227 * 1024)
+    if (pl.R < 1 || pl.R > 128 || pl.Rs < 1 || pl.Rs > 64 || n_cols < 1 || rows < 1 ||
+        rows * (long long)dims->max_blocks > 0x7fffffffLL || pl.smem > 227 * 1024)      // summary rows are indexed with 31 bits
         return false;
     if (rows * 2 > sms) return true;
     const double nt_a = (n_cols + kAtTileCols - 1) / kAtTileCols;
@@ -830,7 +848,7 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     p.acc_col = N <= 32 ? 448 : 0;
     p.tiles_per_bh = (dims->max_blocks + kLyTileBlocks - 1) / kLyTileBlocks;
     p.reduce_sum = reduce_mode == OASIS_REDUCE_SUM;
-    p.total_tiles = rows * p.tiles_per_bh;
+    p.total_tiles = (int)(rows * p.tiles_per_bh);
     p.err = error_word();
     // Equal bytes per SM: an attention tile is 32 KiB, a scoring tile 64 KiB.  The first `n_more` CTAs attend
     // one row more than the others and take correspondingly fewer scoring tiles.
