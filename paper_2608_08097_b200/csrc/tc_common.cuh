@@ -25,6 +25,7 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 // Bounded wait: false (and an error code) if the phase did not complete within the spin limit.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t *err, int code)
 {
+#pragma unroll 1                 // the compiler otherwise unrolls the spin loop at every call site (half the kernel's code)
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         uint32_t done;
         asm volatile(
