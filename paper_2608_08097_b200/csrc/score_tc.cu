@@ -74,6 +74,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
 
     // First tile at or after t (and before t1) that has candidate blocks; t1 if there is none.
     auto next_active = [&](long long t) {
+#pragma unroll 1
         for (; t < t1; ++t) {
             const long long bh = t / p.tiles_per_bh;
             const int j0 = (int)(t % p.tiles_per_bh) * kTileBlocks;
@@ -88,6 +89,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
         const int b = (int)(bh / p.Hkv), h = (int)(bh % p.Hkv);
         uint8_t *dstb = b_ptr + (size_t)buf * b_bytes;
         const int tasks = p.N * 16;                              // 16-byte chunks of the query rows
+#pragma unroll 1
         for (int i0 = me; i0 < tasks; i0 += nthr * 8) {
             uint4 v[8];
 #pragma unroll
@@ -160,6 +162,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
         int it = 0;
         bool alive = true;
         long long t = t_first;
+#pragma unroll 1
         while (t < t1 && alive) {
             const long long bh = t / p.tiles_per_bh;
             const int j0 = (int)(t % p.tiles_per_bh) * kTileBlocks;
@@ -187,6 +190,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
             int it = 0, bo = -1;
             long long cur_bh = -1;
             bool alive = true;
+#pragma unroll 1
             for (long long t = t0; t < t1 && alive; ++t) {
                 const long long bh = t / p.tiles_per_bh;
                 const int j0 = (int)(t % p.tiles_per_bh) * kTileBlocks;
@@ -228,6 +232,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
         int bo = 0;
         bool alive = true;
         long long cur_bh = t_first < t1 ? t_first / p.tiles_per_bh : -1;
+#pragma unroll 1
         for (long long t = t_first < t1 ? next_active(t_first + 1) : t1; t < t1 && alive; t = next_active(t + 1)) {
             const long long bh = t / p.tiles_per_bh;
             if (bh == cur_bh) continue;
@@ -246,6 +251,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
         const int quarter = warp & 3;            // TMEM lanes [32 * quarter, +32) belong to this warp
         int it = 0;
         bool alive = true;
+#pragma unroll 1
         for (long long t = t0; t < t1 && alive; ++t) {
             const long long bh = t / p.tiles_per_bh;
             const int j0 = (int)(t % p.tiles_per_bh) * kTileBlocks;
@@ -263,6 +269,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.N);
             float res = p.reduce_sum ? 0.f : -CUDART_INF_F;
+#pragma unroll 1
             for (int c = 0; c < p.N; c += 16) {
                 uint32_t v[16];
                 tc_ld16(taddr + c, v);
