@@ -9,7 +9,7 @@ Prints one JSON line per section:
           admitted entries per (request, KV head) per step, and the break-even fetch fraction
           rho* = link bandwidth x compute time / cold bytes.
   c5      the budget x draft-length sweep (configs[4]): solo kernel times and roofline fractions of
-          scoring / top-k / attention, and lookahead recall per cell.
+          scoring / top-k / attention and of the fused attention + scoring launch, and lookahead recall per cell.
   stage   the gather kernel alone on random entries of a pinned pool, against the DMA copy peak, and the
           dense -> sparse hand-over (device blocks -> pinned entries + summaries) alone.
   shapes  the kernels alone at the shapes of configs[1], configs[2] and configs[3] (one layer, random
@@ -113,7 +113,7 @@ def section_ratio(args, dev, hbm_peak):
 
 def section_c5(args, dev, hbm_peak):
     """Budget x draft-length sweep: kernels alone (graph replay over rotating working sets) and recall."""
-    from paper_2608_08097_b200 import pipeline
+    from paper_2608_08097_b200 import binding, pipeline
     base = synth.scaled(synth.C5, n_draft=8, layers=1, steps=1)
     lay = synth.make_layer(base, seed=args.seed, layer=0, device=dev)
     kv = lay.host_kv.to(dev)
@@ -138,6 +138,9 @@ def section_c5(args, dev, hbm_peak):
             t_score = graph_time(lambda i: Ls[i].score(q, n_full), n_rot)
             t_sel = graph_time(lambda i: Ls[i].select(n_full, seq, table), n_rot)
             t_attn = graph_time(lambda i: Ls[i].attend(q, seq), n_rot)
+            t_layer = None
+            if binding.attn_and_score_supported(Ls[0].dims, T, Ls[0].cols, Td):
+                t_layer = graph_time(lambda i: Ls[i].attend_and_score(q, seq, n_full), n_rot)
             sel_draft = Ls[0].sel.clone()
             sel_true = torch.empty_like(sel_draft)
             Ls[0].score_queries(q_true, n_full)
@@ -150,13 +153,17 @@ def section_c5(args, dev, hbm_peak):
             cells.append({"K": K, "Td": Td, "score_us": round(t_score, 1), "score_frac": round(sb / t_score / 1e3 / hbm_peak, 3),
                           "select_us": round(t_sel, 1), "attn_us": round(t_attn, 1),
                           "attn_frac": round(ab / t_attn / 1e3 / hbm_peak, 3),
+                          "layer_us": None if t_layer is None else round(t_layer, 1),
+                          "layer_frac": None if t_layer is None else round((sb + ab) / t_layer / 1e3 / hbm_peak, 3),
                           "tokens_per_s_per_layer": round(Bq / ((t_score + t_sel + t_attn) * 1e-6), 1),
+                          "tokens_per_s_per_layer_fused": None if t_layer is None else round(Bq / ((t_layer + t_sel) * 1e-6), 1),
                           "recall": round(recall, 4)})
             del Ls
             torch.cuda.empty_cache()
     print(json.dumps({"section": "c5", "workload": "configs[4]: batch 16, 32q/8kv heads, context 65536, one layer "
                       "(3 rotating copies of the summaries and pools), kernels alone; frac = algorithmic bytes / time / "
-                      "measured copy peak; tokens/s/layer from the serial sum score + top-k + attention",
+                      "measured copy peak; layer = the fused attention + scoring launch; tokens/s/layer from the serial sum score + "
+                      "top-k + attention (and fused launch + top-k)",
                       "hbm_peak_GBps": hbm_peak, "cells": cells}))
 
 

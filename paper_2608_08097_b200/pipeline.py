@@ -108,7 +108,7 @@ class DecodeEngine:
     """
 
     def __init__(self, batch, n_q_heads, n_kv_heads, max_blocks, k, n_q_tokens, n_layers,
-                 device="cuda", mode="fetch_all", cap=None, fused=None):
+                 device="cuda", mode="fetch_all", cap=None, fused=None, transfer_streams=1):
         assert mode in ("fetch_all", "delta")
         self.mode, self.k, self.T, self.n_layers = mode, k, n_q_tokens, n_layers
         self.device = torch.device(device)
@@ -123,6 +123,10 @@ class DecodeEngine:
         self.selq = torch.cuda.Stream(device=self.device, priority=-1)
         self.side = torch.cuda.Stream(device=self.device, priority=-1)
         self.copy = torch.cuda.Stream(device=self.device)     # end-to-end mode: query upload, output download
+        # consecutive layers' gathers may alternate between several transfer streams, so that one gather's
+        # requests are already in flight while the previous one's last ones come back over the host link
+        self.xfer = [self.side] + [torch.cuda.Stream(device=self.device, priority=-1)
+                                   for _ in range(max(1, int(transfer_streams)) - 1)]
         self.launches = 0
         self.cap = cap
         can_fuse = n_layers > 0 and n_q_tokens > 1 and oasis.attn_and_score_supported(self.layers[0].dims, n_q_tokens, self.layers[0].cols, n_q_tokens - 1)
@@ -200,7 +204,7 @@ class DecodeEngine:
         return ev
 
     def _transfer(self, l, ready, timers, plan=None):
-        L, ss = self.layers[l], self.side
+        L, ss = self.layers[l], self.xfer[l % len(self.xfer)]
         with torch.cuda.stream(ss):
             ss.wait_event(ready)
             t0 = self._tick(timers, "stage", ss)
@@ -250,7 +254,8 @@ class DecodeEngine:
                                   step_stamp, None, plan=plan)
             self._transfer(l, ready, None, plan=plan)
             if plan is not None:
-                self.side.synchronize()  # the shared priming plan is reused by the next layer
+                for st in self.xfer:     # the shared priming plan is reused by the next layer
+                    st.synchronize()
         torch.cuda.synchronize(self.device)
         self.stage_done = [None] * self.n_layers     # everything has completed
 
@@ -277,7 +282,8 @@ class DecodeEngine:
                     q_list[l].copy_(q_host[l], non_blocking=True)
                     q_ready[l] = torch.cuda.Event()
                     q_ready[l].record(cs)
-            self.side.wait_event(q_ready[-1])
+            for st in self.xfer:
+                st.wait_event(q_ready[-1])
         summ_ready = [None] * self.n_layers
         if self.fused:
             # the summary updates (one newly completed block per request every 16 steps) only depend on this step's
@@ -323,7 +329,7 @@ class DecodeEngine:
 
     def join(self):
         """Makes the foreground stream wait for everything the other streams have in flight."""
-        for st in (self.pred, self.selq, self.side, self.copy):
+        for st in (self.pred, self.selq, self.copy, *self.xfer):
             ev = torch.cuda.Event()
             ev.record(st)
             self.main.wait_event(ev)
@@ -342,7 +348,8 @@ class DecodeEngine:
             fork.record(self.main)
             self.pred.wait_event(fork)
             self.selq.wait_event(fork)
-            self.side.wait_event(fork)
+            for st in self.xfer:
+                st.wait_event(fork)
             self.copy.wait_event(fork)
             self.step(*args, **kwargs)
             self.join()
