@@ -182,8 +182,10 @@ def test_fused_engine_equals_unfused_engine(gpu, mode, cap):
     to_dev = lambda t: t.to(torch.int32).contiguous().to(dev)
     engines = []
     for fused in (True, False):
+        # the fused engine also alternates its gathers between three transfer streams
         eng = pipeline.DecodeEngine(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_blocks, cfg.k_blocks,
-                                    cfg.n_q_tokens, n_layers, dev, mode=mode, cap=cap, fused=fused)
+                                    cfg.n_q_tokens, n_layers, dev, mode=mode, cap=cap, fused=fused,
+                                    transfer_streams=3 if fused else 1)
         assert eng.fused == fused
         for l, lay in enumerate(lays):
             eng.attach(l, lay.host_kv.to(dev), lay.block_table.to(dev))
