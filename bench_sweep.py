@@ -12,7 +12,7 @@ Prints one JSON line per section:
           scoring / top-k / attention and of the fused attention + scoring launch, and lookahead recall per cell.
   stage   the gather kernel alone on random entries of a pinned pool, against the DMA copy peak, and the
           dense -> sparse hand-over (device blocks -> pinned entries + summaries) alone.
-  shapes  the kernels alone at the shapes of configs[1], configs[2] and configs[3] (one layer, random
+  shapes  the kernels alone at the shapes of configs[0] to configs[3] (one layer, random
           summaries and pools): scoring, top-k, attention, and the fused attention + scoring launch where
           it takes the shape, each against the measured copy peak.
 Inputs are synthetic (the generators of `synth`); nothing here touches the CPU oracle.
@@ -205,10 +205,10 @@ def section_stage(args, dev, hbm_peak):
 
 
 def section_shapes(args, dev, hbm_peak):
-    """Kernels alone at the shapes of configs[1..3] (graph replay over 3 rotating working sets)."""
+    """Kernels alone at the shapes of configs[0..3] (graph replay over 3 rotating working sets)."""
     from paper_2608_08097_b200 import binding, pipeline
     rows = []
-    for name, base in (("configs[1]", synth.C2), ("configs[2]", synth.C3), ("configs[3]", synth.C4)):
+    for name, base in (("configs[0]", synth.C1), ("configs[1]", synth.C2), ("configs[2]", synth.C3), ("configs[3]", synth.C4)):
         cfg = synth.scaled(base, layers=1, steps=1)
         Bq, Hq, Hkv, T, mb, K = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.n_q_tokens, cfg.max_blocks, cfg.k_blocks
         n_rot = 3
@@ -240,14 +240,14 @@ def section_shapes(args, dev, hbm_peak):
             def fused(i):
                 L = Ls[i]
                 binding.attn_and_score(L.dims, q, T, L.pool, L.slot_tbl, L.sel, L.cols, seq, L.scale, L.out, q[:, 1:], Td,
-                                       L.summaries, n_full, L.scores, q_batch_stride=stride)
+                                       L.summaries, n_full, L.scores, q_batch_stride=stride, workspace=L.workspace)
             t_layer = graph_time(fused, n_rot)
             row["layer_us"] = round(t_layer, 1)
             row["layer_frac"] = round((sb + ab) / t_layer / 1e3 / hbm_peak, 3)
         rows.append(row)
         del Ls
         torch.cuda.empty_cache()
-    print(json.dumps({"section": "shapes", "workload": "one layer of configs[1..3], 3 rotating copies of summaries and "
+    print(json.dumps({"section": "shapes", "workload": "one layer of configs[0..3], 3 rotating copies of summaries and "
                       "pools (random contents), kernels alone by graph replay; frac = algorithmic bytes / time / measured "
                       "copy peak; layer = the fused attention + scoring launch (null where it does not take the shape)",
                       "hbm_peak_GBps": hbm_peak, "rows": rows}))

@@ -179,12 +179,15 @@ size_t oasis_attn_workspace_bytes(const oasis_dims_t *dims, int32_t n_q_tokens,
  * Steps 4 and 1 of one layer in a single launch (Sec. 4.2.2: a layer's attention over the working set
  * staged by the previous step and its look-ahead scoring for the next step are independent).  Same
  * arguments, arithmetic and results as oasis_sparse_attn (q .. lse) followed by oasis_score_blocks
- * (q_draft .. scores); no workspace is needed.  One persistent thread block per SM scores its share of
- * the layer's blocks and attends (request, KV head) rows c, c + SMs, c + 2 SMs, ... over the same
- * shared-memory ring, the shares sized so that every SM moves the same number of bytes.
- * Only shapes with  n_q_tokens * (Hq/Hkv) <= 128,  n_draft * (Hq/Hkv) <= 64,  a shared-memory footprint
- * within 227 KiB and attention rows that do not make stragglers (B * Hkv > SMs / 2, or rows of at most 1.25
- * times an SM's equal share of the launch's bytes) are taken (oasis_attn_and_score_supported tells); others
+ * (q_draft .. scores).  One persistent thread block per SM scores its share of the layer's blocks and
+ * attends (request, KV head) rows c, c + SMs, c + 2 SMs, ... over the same shared-memory ring, the
+ * shares sized so that every SM moves the same number of bytes.  With B * Hkv <= SMs / 2 and rows too
+ * long to be attended whole, the column lists are split as oasis_sparse_attn splits them, each split a
+ * work item, and a second, small launch merges the parts: pass a `workspace` of
+ * oasis_attn_workspace_bytes() bytes (16-byte aligned, contents undefined before and after; may be
+ * NULL where that is 0).
+ * Only shapes with  n_q_tokens * (Hq/Hkv) <= 128,  n_draft * (Hq/Hkv) <= 64  and a shared-memory
+ * footprint within 227 KiB are taken (oasis_attn_and_score_supported tells); others
  * return OASIS_ERR_UNSUPPORTED: make the two calls.
  *   q_batch_stride   elements between consecutive requests of q_draft (0 = dense)
  */
@@ -192,7 +195,8 @@ int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int32_t n_q_to
                          const int32_t *slot_tbl, const int32_t *blk_tbl, int32_t n_cols,
                          const int32_t *seq_len, float scale, void *out, float *lse, const void *q_draft,
                          int64_t q_batch_stride, int32_t n_draft, const void *summaries,
-                         const int32_t *n_full_blocks, int32_t reduce_mode, float *scores, void *stream);
+                         const int32_t *n_full_blocks, int32_t reduce_mode, float *scores, void *workspace,
+                         size_t workspace_bytes, void *stream);
 
 /* 1 if oasis_attn_and_score takes these shapes on the current device, else 0. */
 int oasis_attn_and_score_supported(const oasis_dims_t *dims, int32_t n_q_tokens, int32_t n_cols,

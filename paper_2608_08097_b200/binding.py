@@ -80,7 +80,7 @@ def lib():
         L.oasis_offload_blocks.argtypes = [dp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
         L.oasis_offload_blocks.restype = ctypes.c_int
         L.oasis_attn_and_score.argtypes = [dp, vp, i32, vp, vp, vp, i32, vp, ctypes.c_float, vp, vp, vp, ctypes.c_int64, i32, vp, vp,
-                                           i32, vp, vp]
+                                           i32, vp, vp, ctypes.c_size_t, vp]
         L.oasis_attn_and_score.restype = ctypes.c_int
         L.oasis_attn_and_score_supported.argtypes = [dp, i32, i32, i32]
         L.oasis_attn_and_score_supported.restype = ctypes.c_int
@@ -210,10 +210,13 @@ def offload_blocks(dims, dense_k, dense_v, gpu_table, block_table, first_block, 
 
 
 def attn_and_score(dims, q, n_q_tokens, hbm_pool, slot_tbl, blk_tbl, n_cols, seq_len, scale, out, q_draft, n_draft,
-                   summaries, n_full_blocks, scores, lse=None, reduce_mode=REDUCE_MAX, q_batch_stride=None, stream=None):
+                   summaries, n_full_blocks, scores, lse=None, reduce_mode=REDUCE_MAX, q_batch_stride=None, workspace=None,
+                   stream=None):
     """Steps 4 and 1 of one layer in one launch; raises OasisError (status 2) for shapes outside the fused
-    launch, which take sparse_attn + score_blocks instead."""
+    launch, which take sparse_attn + score_blocks instead.  `workspace`: attn_workspace_bytes() bytes where
+    that is not zero (few rows: the column lists are split)."""
     d = dims.c()
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     if q_batch_stride is None:
         q_batch_stride = n_draft * dims.n_q_heads * 128
     _check(lib().oasis_attn_and_score(
@@ -222,7 +225,8 @@ def attn_and_score(dims, q, n_q_tokens, hbm_pool, slot_tbl, blk_tbl, n_cols, seq
         _ptr(seq_len, torch.int32, "seq_len"), ctypes.c_float(scale), _ptr(out, torch.bfloat16, "out"),
         _ptr(lse, torch.float32, "lse"), ctypes.c_void_p(q_draft.data_ptr()), ctypes.c_int64(int(q_batch_stride)),
         int(n_draft), _ptr(summaries, torch.bfloat16, "summaries"), _ptr(n_full_blocks, torch.int32, "n_full_blocks"),
-        int(reduce_mode), _ptr(scores, torch.float32, "scores"), _stream(stream)), "oasis_attn_and_score")
+        int(reduce_mode), _ptr(scores, torch.float32, "scores"), _ptr(workspace, None, "workspace"), ws_bytes,
+        _stream(stream)), "oasis_attn_and_score")
 
 
 def attn_and_score_supported(dims, n_q_tokens, n_cols, n_draft) -> bool:

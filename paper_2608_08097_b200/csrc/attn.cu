@@ -28,15 +28,21 @@ struct AttnParams {
 };
 
 // Merges the splits of one (request, KV head, row): out = sum_s w_s o_s / sum_s w_s with
-// w_s = 2^(lse_s - max lse).  One CTA of 128 threads per row.
-__global__ void __launch_bounds__(128)
-attn_combine_kernel(const AttnParams p)
+// w_s = 2^(lse_s - max lse).  CTAs of 256 threads take the `total` rows in turn, two at a time.  Launched behind the fused layer
+// kernel with programmatic stream serialization it lets the launch after it start early and itself waits for the
+// partials (both instructions do nothing in an ordinary launch).
+__global__ void __launch_bounds__(256)
+attn_combine_kernel(const AttnParams p, long long total)
 {
-    const int row = blockIdx.x % p.R;
-    const int bh = blockIdx.x / p.R;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+#pragma unroll 1
+    for (long long wi = 2ll * blockIdx.x + (threadIdx.x >> 7); wi < total; wi += 2ll * gridDim.x) {
+    const int row = (int)(wi % p.R);
+    const int bh = (int)(wi / p.R);
     const int b = bh / p.Hkv, h = bh % p.Hkv;
     const int grp = row / p.rows_per_group, r = row % p.rows_per_group;
-    const int d = threadIdx.x;
+    const int d = threadIdx.x & 127;
     float mx = -CUDART_INF_F;
     for (int s = 0; s < p.n_splits; ++s) {
         const long long item = ((long long)bh * p.n_splits + s) * p.n_groups + grp;
@@ -55,6 +61,7 @@ attn_combine_kernel(const AttnParams p)
     const long long orow = ((long long)b * p.T + tq) * p.Hq + a;
     reinterpret_cast<__nv_bfloat16 *>(p.out)[orow * kHeadDim + d] = __float2bfloat16_rn(den > 0.f ? acc / den : 0.f);
     if (p.lse && d == 0) p.lse[orow] = den > 0.f ? (mx + log2f(den)) * kLn2 : -CUDART_INF_F;
+    }
 }
 
 // Launch geometry shared by the entry point and the workspace query.
@@ -102,10 +109,47 @@ static int launch_attn(const oasis_dims_t *dims, const AttnPlan &pl, const AttnP
                                 p.part_o, p.part_lse, pl.n_splits, pl.cols_per_split, kAttnStages, error_word(), st, who))
         return rc;
     if (pl.n_splits > 1) {
-        attn_combine_kernel<<<(unsigned)combine_ctas, 128, 0, st>>>(p);
+        attn_combine_kernel<<<(unsigned)((combine_ctas + 1) / 2), 256, 0, st>>>(p, combine_ctas);
         return check_launch(who);
     }
     return OASIS_OK;
+}
+
+// How the attention splits the column lists for these shapes (the fused layer launch splits the same way, so
+// that its results equal the separate call's bit for bit) and the scratch bytes the partials need.
+void attn_split_plan(const oasis_dims_t *dims, int T, int n_cols, int *n_splits, int *cols_per_split, size_t *workspace)
+{
+    const AttnPlan pl = attn_plan(dims, T, n_cols);
+    *n_splits = pl.n_splits;
+    *cols_per_split = pl.cols_per_split;
+    *workspace = pl.workspace;
+}
+
+// The combine launch behind the fused layer kernel: a few CTAs per SM that are all resident at once, started
+// early by programmatic stream serialization (the kernel itself waits for the partials).
+int launch_attn_combine_after(const oasis_dims_t *dims, int T, void *out, float *lse, float *part_o, float *part_lse,
+                              int n_splits, cudaStream_t st, const char *who)
+{
+    AttnParams p = {};
+    p.out = (uint8_t *)out; p.lse = lse; p.part_o = part_o; p.part_lse = part_lse;
+    p.T = T; p.Hq = dims->n_q_heads; p.Hkv = dims->n_kv_heads; p.G = dims->n_q_heads / dims->n_kv_heads;
+    p.R = T * p.G; p.n_splits = n_splits; p.n_groups = 1; p.rows_per_group = p.R;
+    const long long total = (long long)dims->batch * dims->n_kv_heads * p.R;
+    long long grid = (long long)sm_count() * 2;          // all resident beside the fused kernel's thread blocks
+    if (grid > (total + 1) / 2) grid = (total + 1) / 2;
+    prefer_max_shared_carveout(attn_combine_kernel);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_combine_kernel, p, total);
+    if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "%s: combine launch: %s", who, cudaGetErrorString(e));
+    return check_launch(who);
 }
 
 }  // namespace oasis

@@ -54,7 +54,10 @@ struct LayerTcParams {
     uint8_t *out;
     float *lse;
     float scale_log2;
-    int T, Hq, Hkv, G, n_cols, R, rows;
+    int T, Hq, Hkv, G, n_cols, R;
+    int items;                  // attention work items: (request, KV head) rows x splits of their column lists
+    int n_splits, cols_per_split;
+    float *part_o, *part_lse;   // split runs: normalised partial outputs [items][R][128] and their log2 sum-exps [items][R]
     int n_more;                 // CTAs 0 .. n_more-1 attend one row more than the others
     // scoring phase
     const uint8_t *q_draft;
@@ -68,13 +71,17 @@ struct LayerTcParams {
     int32_t *err;
 };
 
-// MULTI: more rows than thread blocks, several rows per block.  STAGES: 32 KiB stages of the ring (6, or 4 where the
-// scoring operands or the copy-merge staging need the room).
-template <int MMA_M, int COPIES, bool MULTI, int STAGES>
+// MODE: 0 = at most one whole row per thread block; 1 = more rows than thread blocks, several whole rows per block;
+// 2 = fewer rows than half the SMs, their column lists split into one work item per thread block.  Separate
+// instantiations because the kernel is sensitive to every instruction its issuing threads execute (the row loop
+// costs mode 0 1.5 us at 128 rows, the split arithmetic 0.5 us).  STAGES: 32 KiB stages of the ring (6, or 4 where
+// the scoring operands or the copy-merge staging need the room).
+template <int MMA_M, int COPIES, int MODE, int STAGES>
 __global__ void __launch_bounds__(kLyThreads, 1)
 layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap_summ,
                 const LayerTcParams p)
 {
+    constexpr bool MULTI = MODE == 1, SPLIT = MODE == 2;
     constexpr int kLyStages = STAGES, kLyPairs = STAGES / 2;
     constexpr int RPC = MMA_M / COPIES;                     // MMA rows per copy of the query rows
     constexpr int LANES = MMA_M / 4;                        // lanes of each softmax warp that hold an MMA row
@@ -114,13 +121,19 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // ---- attention geometry: CTA c < rows owns row c ------------------------------------------------------
-    const int n_my_rows = (int)blockIdx.x < p.rows ? (MULTI ? (p.rows - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 1) : 0;
+    // An attention work item is one (request, KV head) row, or one split of its column list where there are fewer
+    // rows than half the SMs (items of a row are consecutive: item = row * n_splits + split).
+    const int n_my_rows = (int)blockIdx.x < p.items ? (MULTI ? (p.items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 1) : 0;
     const bool cta_has_row = n_my_rows > 0;
-    auto my_row = [&](int k) { return (int)blockIdx.x + k * (int)gridDim.x; };     // k-th row of this CTA
-    const int c0 = 0, c1 = p.n_cols;
-    const int tpr = (p.n_cols + kAtTileCols - 1) / kAtTileCols;     // tiles per row
-    const int n_tiles = n_my_rows * tpr;                             // attention tiles of this CTA, all rows
-    const int L0 = p.seq_len[(cta_has_row ? (int)blockIdx.x : 0) / p.Hkv];   // length of the request of the first row
+    auto my_row = [&](int k) { return (int)blockIdx.x + k * (int)gridDim.x; };     // k-th item of this CTA
+    auto row_of = [&](int item) { return SPLIT ? item / p.n_splits : item; };
+    auto first_col = [&](int item) { return SPLIT ? (item % p.n_splits) * p.cols_per_split : 0; };
+    auto end_col = [&](int item) { return SPLIT ? min(first_col(item) + p.cols_per_split, p.n_cols) : p.n_cols; };
+    // tiles of 4 columns an item covers: the same for every whole row; a split item is its thread block's only one
+    const int tiles_first = ((SPLIT && cta_has_row ? end_col((int)blockIdx.x) - first_col((int)blockIdx.x) : p.n_cols) +
+                             kAtTileCols - 1) / kAtTileCols;
+    auto tiles_of = [&](int) { return tiles_first; };
+    const int L0 = p.seq_len[(cta_has_row ? row_of((int)blockIdx.x) : 0) / p.Hkv];   // length of the request of the first item
     // ---- scoring geometry: tiles [t0, t1) ---------------------------------------------------------
     auto tiles_before = [&](int c) {
         const double w = c <= p.n_more ? c * p.w_row : p.n_more * p.w_row + (c - p.n_more) * p.w_free;
@@ -250,20 +263,21 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         // ---------------------------------------------------------------- producer
         // Table entries are read 32 columns (eight tiles) at a time, lane j holding column j of the window, and the
         // next window is requested as soon as the current one starts, so no table load sits on the critical path.
-        const int32_t *slot_row = p.slot_tbl, *blk_row = p.blk_tbl;
-        auto load_window = [&](int first_col, int &wblk, int &wslot) {
-            const int c = first_col + lane;
-            wblk = c < c1 ? blk_row[c] : -1;
-            wslot = c < c1 ? slot_row[c] : -1;
-        };
         // the attention phase reads what the previous layer may have produced: wait for it (no-op without a programmatic launch)
         asm volatile("griddepcontrol.wait;" ::: "memory");
         int s = 0, gi = 0;                                           // ring stage and index of the tile among all rows
         uint32_t ph = 1;                                             // parity of the "empty" phase to wait for
 #pragma unroll 1
         for (int k = 0; k < n_my_rows && alive; ++k) {
-        slot_row = p.slot_tbl + (long long)my_row(k) * p.n_cols;
-        blk_row = p.blk_tbl + (long long)my_row(k) * p.n_cols;
+        const int item = my_row(k), tpr = tiles_of(item);
+        const int32_t *slot_row = p.slot_tbl + (long long)row_of(item) * p.n_cols;
+        const int32_t *blk_row = p.blk_tbl + (long long)row_of(item) * p.n_cols;
+        const int c0 = first_col(item), c1 = end_col(item);          // column range of the item
+        auto load_window = [&](int first, int &wblk, int &wslot) {
+            const int c = first + lane;
+            wblk = c < c1 ? blk_row[c] : -1;
+            wslot = c < c1 ? slot_row[c] : -1;
+        };
         int cur_blk, cur_slot, nxt_blk = -1, nxt_slot = -1;
         load_window(c0, cur_blk, cur_slot);
 #pragma unroll 1
@@ -363,6 +377,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             int i = 0;                                               // index of the tile among all rows of this CTA
 #pragma unroll 1
             for (int k = 0; k < n_my_rows && alive; ++k) {
+            const int tpr = tiles_of(my_row(k));
             alive = mbar_wait(bar_q, (uint32_t)(k & 1), p.err, 55);  // the row's Q is in tensor memory
             tc_fence_after();
 #pragma unroll 1
@@ -400,7 +415,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             int s = 0, sb = 0;
             uint32_t ph_p = 0;
 #pragma unroll 1
-            for (int k = 0; k < n_my_rows && alive; ++k)
+            for (int k = 0; k < n_my_rows && alive; ++k) {
+            const int tpr = tiles_of(my_row(k));
 #pragma unroll 1
             for (int it = 0; it < tpr && alive; ++it) {
                 alive = mbar_wait(bar_p_full(sb), ph_p, p.err, 53);
@@ -416,6 +432,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 s = (s + 1 == kLyStages) ? 0 : s + 1;
                 sb = (sb + 1) & (kAtSBufs - 1);
                 ph_p ^= (sb == 0);
+            }
             }
         }
     } else if (warp == 7) {
@@ -514,14 +531,15 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_q);
         };
-        if (cta_has_row) load_q(my_row(0));
+        if (cta_has_row) load_q(row_of(my_row(0)));
         bool alive = true;
         int s = 0, s_prev = 0;                                      // ring stage of tile i and of tile i - 1
         uint32_t ph_prev = 0;                                       // parity of the "empty" phase that ends tile i - 1
         int i = 0;                                                  // index of the tile among all rows of this CTA
 #pragma unroll 1
         for (int k = 0; k < n_my_rows; ++k) {
-        const int bh = my_row(k), b = bh / p.Hkv, h = bh % p.Hkv;
+        const int item = my_row(k), tpr = tiles_of(item);
+        const int bh = row_of(item), b = bh / p.Hkv, h = bh % p.Hkv;
         const int limit = live_row ? (k == 0 ? L0 : p.seq_len[b]) + row / p.G : -1;     // last visible position of this row
         float m_ref = -CUDART_INF_F, l_sum = 0.f;
 #pragma unroll 1
@@ -640,6 +658,15 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             // writes 16 output dims [d0, d0 + 16) of query row `orow`
             auto emit = [&](int orow, int d0, const float (&acc)[16], float mx, float den) {
                 const float inv = den > 0.f ? 1.f / den : 0.f;
+                if (SPLIT) {
+                    // one split of the row: normalised partial and its log2 sum-exp, merged by the combine launch
+                    float4 *dstp = reinterpret_cast<float4 *>(p.part_o + ((long long)item * p.R + orow) * kHeadDim + d0);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        dstp[e] = make_float4(acc[4 * e] * inv, acc[4 * e + 1] * inv, acc[4 * e + 2] * inv, acc[4 * e + 3] * inv);
+                    if (d0 == 0) p.part_lse[(long long)item * p.R + orow] = den > 0.f ? mx + log2f(den) : -CUDART_INF_F;
+                    return;
+                }
                 const int tq = orow / p.G, a = h * p.G + orow % p.G;
                 const long long o_row = ((long long)b * p.T + tq) * p.Hq + a;
                 uint4 *dst = reinterpret_cast<uint4 *>(p.out + (o_row * kHeadDim + d0) * 2);
@@ -734,16 +761,21 @@ static size_t layer_tc_smem_bytes(int mma_m, int copies, int N, int stages)
 
 struct LayerTcPlan {
     int R, Rs, N, mma_m, copies, stages;
-    size_t smem;
+    int n_splits, cols_per_split;       // of every row's column list (1 = rows are attended whole)
+    size_t smem, workspace;
 };
+
+void attn_split_plan(const oasis_dims_t *dims, int T, int n_cols, int *n_splits, int *cols_per_split, size_t *workspace);
+int launch_attn_combine_after(const oasis_dims_t *dims, int T, void *out, float *lse, float *part_o, float *part_lse,
+                              int n_splits, cudaStream_t st, const char *who);                       // attn.cu
 
 // Whether the fused launch takes these shapes, and with which variant.  Wanted: at most 128 attention rows and 64
 // scoring rows per KV head (two accumulators of up to 32 columns fit beside the attention's tensor memory, wider
-// ones take the place of the S buffers, which the attention phase only touches after the last scoring epilogue);
-// a footprint within 227 KiB with six ring stages, or with four for the 128-row variants; and attention rows that
-// do not make stragglers: more rows than half the SMs, or rows whose tiles stay within 1.25 times an SM's equal
-// share of the launch (with fewer and longer rows the attention wants its column lists split over several SMs).
-// With more rows than SMs a CTA attends rows c, c + grid, c + 2 grid, ...
+// ones take the place of the S buffers, which the attention phase only touches after the last scoring epilogue)
+// and a footprint within 227 KiB with six ring stages, or with four for the 128-row variants.
+// With more rows than SMs a CTA attends rows c, c + grid, c + 2 grid, ...; with fewer rows than half the SMs, and
+// rows too long to be attended whole without making stragglers, the column lists are split exactly as
+// oasis_sparse_attn splits them, each split a work item of its own, and a combine launch merges the parts.
 static bool layer_tc_plan(const oasis_dims_t *dims, int n_q_tokens, int n_cols, int n_draft, LayerTcPlan *out)
 {
     LayerTcPlan pl;
@@ -761,15 +793,23 @@ static bool layer_tc_plan(const oasis_dims_t *dims, int n_q_tokens, int n_cols, 
         pl.stages = 4;
         pl.smem = layer_tc_smem_bytes(pl.mma_m, pl.copies, pl.N, pl.stages);
     }
+    pl.n_splits = 1;
+    pl.cols_per_split = n_cols;
+    pl.workspace = 0;
+    if (rows * 2 <= sms && rows >= 1 && pl.R >= 1 && pl.R <= 128 && n_cols >= 1) {
+        // Few rows.  Whole rows are still fine while a row's tiles stay within 1.25 times an SM's equal share of the
+        // launch (the thread blocks without a row score instead); longer rows would be stragglers and are split.
+        const double nt_a = (n_cols + kAtTileCols - 1) / kAtTileCols;
+        const double tiles_s = (double)rows * ((dims->max_blocks + kLyTileBlocks - 1) / kLyTileBlocks);
+        const double share = ((double)rows * nt_a + 2.0 * tiles_s) / sms;     // 32 KiB units per SM
+        if (nt_a > 1.25 * share)
+            attn_split_plan(dims, n_q_tokens, n_cols, &pl.n_splits, &pl.cols_per_split, &pl.workspace);
+    }
     if (out) *out = pl;
     if (pl.R < 1 || pl.R > 128 || pl.Rs < 1 || pl.Rs > 64 || n_cols < 1 || rows < 1 ||
         rows * (long long)dims->max_blocks > 0x7fffffffLL || pl.smem > 227 * 1024)      // summary rows are indexed with 31 bits
         return false;
-    if (rows * 2 > sms) return true;
-    const double nt_a = (n_cols + kAtTileCols - 1) / kAtTileCols;
-    const double tiles_s = (double)rows * ((dims->max_blocks + kLyTileBlocks - 1) / kLyTileBlocks);
-    const double share = ((double)rows * nt_a + 2.0 * tiles_s) / sms;     // 32 KiB units per SM
-    return nt_a <= 1.25 * share;
+    return rows * (long long)pl.n_splits <= 0x7fffffffLL;
 }
 
 }  // namespace oasis
@@ -785,7 +825,8 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
                                     const int32_t *slot_tbl, const int32_t *blk_tbl, int32_t n_cols,
                                     const int32_t *seq_len, float scale, void *out, float *lse, const void *q_draft,
                                     int64_t q_batch_stride, int32_t n_draft, const void *summaries,
-                                    const int32_t *n_full_blocks, int32_t reduce_mode, float *scores, void *stream)
+                                    const int32_t *n_full_blocks, int32_t reduce_mode, float *scores, void *workspace,
+                                    size_t workspace_bytes, void *stream)
 {
     using namespace oasis;
     const char *who = "oasis_attn_and_score";
@@ -812,6 +853,11 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
                     "the fused launch; call oasis_sparse_attn and oasis_score_blocks", who, rows, n_cols, sms, pl.R, pl.Rs);
     const int R = pl.R, Rs = pl.Rs, N = pl.N;
     const size_t smem = pl.smem;
+    if (pl.workspace > 0) {
+        if (!workspace || workspace_bytes < pl.workspace)
+            return fail(OASIS_ERR_WORKSPACE, "%s: workspace of %zu bytes required, %zu given", who, pl.workspace, workspace_bytes);
+        if (!aligned16(workspace)) return fail(OASIS_ERR_INVALID_ARG, "%s: workspace must be 16-byte aligned", who);
+    }
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return fail(OASIS_ERR_CUDA, "%s: cuTensorMapEncodeTiled is not available", who);
     CUtensorMap tmap_kv, tmap_summ;
@@ -842,7 +888,10 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     p.out = (uint8_t *)out; p.lse = lse;
     p.scale_log2 = scale * kAtLog2e;
     p.T = n_q_tokens; p.Hq = dims->n_q_heads; p.Hkv = dims->n_kv_heads; p.G = G;
-    p.n_cols = n_cols; p.R = R; p.rows = (int)rows;
+    p.n_cols = n_cols; p.R = R; p.items = (int)(rows * pl.n_splits);
+    p.n_splits = pl.n_splits; p.cols_per_split = pl.cols_per_split;
+    p.part_o = (float *)workspace;
+    p.part_lse = p.part_o ? p.part_o + (size_t)p.items * R * kHeadDim : nullptr;
     p.q_draft = (const uint8_t *)q_draft; p.q_batch_stride = q_batch_stride; p.n_full = n_full_blocks; p.scores = scores;
     p.Rs = Rs; p.N = N; p.max_blocks = dims->max_blocks;
     p.acc_col = N <= 32 ? 448 : 0;
@@ -853,15 +902,19 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     // Equal bytes per SM: an attention tile is 32 KiB, a scoring tile 64 KiB.  The first `n_more` CTAs attend
     // one row more than the others and take correspondingly fewer scoring tiles.
     const int grid = sms;
-    const double nt_a = (n_cols + kAtTileCols - 1) / kAtTileCols;
-    const long long m_rows = rows / grid;
-    const int rem = (int)(rows % grid);
+    const long long items = p.items;
+    long long row_tiles = 0;                                   // attention tiles of one row, over its splits
+    for (int c0 = 0; c0 < n_cols; c0 += pl.cols_per_split)
+        row_tiles += ((c0 + pl.cols_per_split < n_cols ? pl.cols_per_split : n_cols - c0) + kAtTileCols - 1) / kAtTileCols;
+    const double nt_a = (double)row_tiles / pl.n_splits;        // per work item
+    const long long m_rows = items / grid;
+    const int rem = (int)(items % grid);
     if (rem == 0) {
         p.n_more = grid;
         p.w_row = (double)p.total_tiles / (double)grid;
         p.w_free = 0.0;
     } else {
-        const double units = ((double)rows * nt_a + 2.0 * (double)p.total_tiles) / grid;
+        const double units = ((double)items * nt_a + 2.0 * (double)p.total_tiles) / grid;
         double w_more = (units - (double)(m_rows + 1) * nt_a) / 2.0;
         if (w_more < 0.0) w_more = 0.0;
         p.n_more = rem;
@@ -890,8 +943,9 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     } while (0)
 #define OASIS_LAYER_TC_LAUNCH(M, C, ST)                          \
     do {                                                         \
-        if (rows > grid) OASIS_LAYER_TC_LAUNCH_2(M, C, true, ST); \
-        else OASIS_LAYER_TC_LAUNCH_2(M, C, false, ST);           \
+        if (pl.n_splits > 1) OASIS_LAYER_TC_LAUNCH_2(M, C, 2, ST);  \
+        else if (items > grid) OASIS_LAYER_TC_LAUNCH_2(M, C, 1, ST); \
+        else OASIS_LAYER_TC_LAUNCH_2(M, C, 0, ST);               \
     } while (0)
     if (R <= 16) OASIS_LAYER_TC_LAUNCH(64, 4, 6);
     else if (R <= 32) OASIS_LAYER_TC_LAUNCH(64, 2, 6);
@@ -902,5 +956,8 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
 #undef OASIS_LAYER_TC_LAUNCH
 #undef OASIS_LAYER_TC_LAUNCH_2
     if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "%s: launch with %zu B of shared memory: %s", who, smem, cudaGetErrorString(e));
-    return check_launch(who);
+    if (int rc = check_launch(who)) return rc;
+    if (pl.n_splits > 1)
+        return launch_attn_combine_after(dims, n_q_tokens, out, lse, p.part_o, p.part_lse, pl.n_splits, st, who);
+    return OASIS_OK;
 }

@@ -80,7 +80,7 @@ class DecodeLayer:
         oasis.attn_and_score(self.dims, q, self.T, self.pool, self.slot_tbl if slot_tbl is None else slot_tbl,
                              self.sel if blk_tbl is None else blk_tbl, self.cols, seq_len, self.scale, self.out,
                              q[:, 1:], self.T - 1, self.summaries, n_full_next, self.scores, lse=self.lse,
-                             q_batch_stride=self.T * self.Hq * 128, stream=stream)
+                             q_batch_stride=self.T * self.Hq * 128, workspace=self.workspace, stream=stream)
         return self.out
 
 
@@ -305,7 +305,7 @@ class DecodeEngine:
                     t0 = self._tick(timers, "layer", ms)
                     L.attend_and_score(q_list[l], seq_len, n_full_next, blk_tbl=self.blk_tbl(l))
                     self._tock(timers, "layer", t0, ms)
-                    self.launches += 2                 # the fused launch and the layer's summary update
+                    self.launches += 3 if self._splits else 2      # the fused launch (and the merge of split rows), the summary update
                 else:
                     t0 = self._tick(timers, "attn", ms)
                     L.attend(q_list[l], seq_len, blk_tbl=self.blk_tbl(l))
