@@ -253,7 +253,9 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
         const bool has_row = lane < LANES;
         const bool live_row = has_row && row < p.R;
         const bool live_warp = (quarter * LANES) % RPC < p.R;       // some lane of this warp holds a query row
-        const int limit = live_row ? L + row / p.G : -1;            // last visible position of this row
+        // last visible position of this row; MMA rows past R hold zero queries and need no masking (masking them would
+        // send their whole warp down the masked path on every tile), lanes without an MMA row see nothing
+        const int limit = live_row ? L + row / p.G : (has_row ? 0x3fffffff : -1);
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         float m_ref = -CUDART_INF_F, l_sum = 0.f;
         bool alive = true;

@@ -540,7 +540,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         for (int k = 0; k < n_my_rows; ++k) {
         const int item = my_row(k), tpr = tiles_of(item);
         const int bh = row_of(item), b = bh / p.Hkv, h = bh % p.Hkv;
-        const int limit = live_row ? (k == 0 ? L0 : p.seq_len[b]) + row / p.G : -1;     // last visible position of this row
+        // last visible position of this row; MMA rows past R hold zero queries and need no masking (masking them would
+        // send their whole warp down the masked path on every tile), lanes without an MMA row see nothing
+        const int limit = live_row ? (k == 0 ? L0 : p.seq_len[b]) + row / p.G : (has_row ? 0x3fffffff : -1);
         float m_ref = -CUDART_INF_F, l_sum = 0.f;
 #pragma unroll 1
         for (int it = 0; it < tpr && alive; ++it, ++i) {
