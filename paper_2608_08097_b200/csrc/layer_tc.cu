@@ -559,7 +559,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                     int n = blk < 0 ? 0 : limit - blk * kBlock + 1;
                     n = max(0, min(n, kBlock));
                     nvis[c] = n;
-                    masked |= n < kBlock;
+                    masked |= has_row && n < kBlock;         // lanes without an MMA row are zeroed below instead
                 }
                 masked = __any_sync(0xffffffffu, masked);
                 float x[KPC];
@@ -586,7 +586,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                     mx4[0] = fmaxf(mx4[0], x[e]); mx4[1] = fmaxf(mx4[1], x[e + 1]);
                     mx4[2] = fmaxf(mx4[2], x[e + 2]); mx4[3] = fmaxf(mx4[3], x[e + 3]);
                 }
-                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                // a lane without an MMA row read whatever its tensor-memory lane held: it must not raise the reference
+                const float mx = has_row ? fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) : -CUDART_INF_F;
                 const float mxs = mx * p.scale_log2;
                 const bool raise = mxs > m_ref + 8.0f;
                 if (__any_sync(0xffffffffu, raise)) {
@@ -623,6 +624,10 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                     pk[e] = pack_bf16x2(p0, p1);
                 }
                 l_sum += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                if (!has_row) {
+#pragma unroll
+                    for (int e = 0; e < KPC / 2; ++e) pk[e] = 0u;   // and it stores P = 0
+                }
 #pragma unroll
                 for (int g8 = 0; g8 < 4; ++g8) {                    // four groups of 8 packed columns = four blocks
                     uint32_t w8[8];
