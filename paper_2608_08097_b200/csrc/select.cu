@@ -280,7 +280,7 @@ extern "C" int oasis_select_topk(const oasis_dims_t *dims, const float *scores,
     while (sort_len < k) sort_len <<= 1;
     p.sort_len = sort_len;
     int threads = 128;
-    while (threads < 1024 && threads * 16 < dims->max_blocks) threads <<= 1;   // ~16 keys per thread
+    while (threads < 1024 && threads * 8 < dims->max_blocks) threads <<= 1;    // ~8 keys per thread
     const size_t smem = (size_t)sort_len * 8 + (size_t)dims->max_blocks * 4;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
