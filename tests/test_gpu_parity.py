@@ -509,3 +509,18 @@ def test_fused_call_rejects_shapes_outside_its_range(gpu):
     zf = torch.zeros(1 << 12, dtype=torch.float32, device=dev)
     with pytest.raises(binding.OasisError, match="outside the fused"):
         binding.attn_and_score(dims, z16, 5, z16, zi, zi, 10, zi, 0.1, z16, z16, 20, z16, zi, zf)
+
+
+def test_fused_call_wants_its_workspace_when_it_splits(gpu):
+    """With few, long rows the fused launch splits the column lists and needs the attention's workspace; without
+    it the call must fail before anything is launched."""
+    binding, _ = gpu
+    dev = torch.device("cuda")
+    dims = binding.Dims(1, 32, 8, 512)                              # 8 rows of 130 columns: split
+    assert binding.attn_workspace_bytes(dims, 5, 130) > 0
+    assert binding.attn_and_score_supported(dims, 5, 130, 4)
+    z16 = torch.zeros(1 << 20, dtype=torch.bfloat16, device=dev)
+    zi = torch.zeros(1 << 12, dtype=torch.int32, device=dev)
+    zf = torch.zeros(1 << 12, dtype=torch.float32, device=dev)
+    with pytest.raises(binding.OasisError, match="workspace"):
+        binding.attn_and_score(dims, z16, 5, z16, zi, zi, 130, zi, 0.1, z16, z16, 4, z16, zi, zf)
