@@ -686,13 +686,61 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 if (p.lse && d0 == 0) p.lse[o_row] = den > 0.f ? (mx + log2f(den)) * kAtLn2 : -CUDART_INF_F;
             };
             if (alive && COPIES > 1) {
-                // the copies meet in a small staging area, 16 dims at a time (small enough that the selection kernels
-                // of other streams still fit beside this CTA, and the ring may already belong to the next phase)
+                // with several rows per thread block the ring already holds the next row's tiles: the copies meet in a
+                // small staging area, 16 dims at a time (small enough that the selection kernels of other streams still
+                // fit beside this CTA)
                 if (lane < LANES) {
                     m_sm[m_row] = m_ref;
                     l_sm[m_row] = l_sum;
                 }
                 float mx = -CUDART_INF_F, den = 0.f, wt[COPIES];
+                if (!MULTI) {
+                    // the thread block's only work item: the ring is idle, so whole O rows meet there in one round
+                    // ([MMA_M][132] floats) and the (row, slice of the dims) tasks go to the first MMA_M threads
+                    float *o_big = reinterpret_cast<float *>(base_ptr + kAtQBytes);
+                    if (live_warp) {
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            uint32_t v[16];
+                            tc_ld16(tmem_o + lane_base + c * 16, v);
+                            float4 *dst = reinterpret_cast<float4 *>(o_big + m_row * 132 + c * 16);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                if (lane < LANES) dst[e] = make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]),
+                                                                       __uint_as_float(v[4 * e + 2]), __uint_as_float(v[4 * e + 3]));
+                        }
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");  // the four softmax warps
+                    constexpr int DLEN = kHeadDim / COPIES;
+                    const int orow = t_task % RPC, d_first = (t_task / RPC) * DLEN;
+                    if (t_task < MMA_M && orow < p.R) {
+#pragma unroll
+                        for (int c = 0; c < COPIES; ++c) mx = fmaxf(mx, m_sm[c * RPC + orow]);
+#pragma unroll
+                        for (int c = 0; c < COPIES; ++c) {
+                            wt[c] = mx == -CUDART_INF_F ? 0.f : fast_exp2(m_sm[c * RPC + orow] - mx);
+                            den += wt[c] * l_sm[c * RPC + orow];
+                        }
+#pragma unroll 1
+                        for (int d0 = d_first; d0 < d_first + DLEN; d0 += 16) {
+                            float acc[16];
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+#pragma unroll
+                            for (int c = 0; c < COPIES; ++c) {
+                                if (wt[c] == 0.f) continue;         // a copy that saw no key holds no O row
+                                const float4 *src = reinterpret_cast<const float4 *>(o_big + (c * RPC + orow) * 132 + d0);
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const float4 v4 = src[e];
+                                    acc[4 * e] += wt[c] * v4.x; acc[4 * e + 1] += wt[c] * v4.y;
+                                    acc[4 * e + 2] += wt[c] * v4.z; acc[4 * e + 3] += wt[c] * v4.w;
+                                }
+                            }
+                            emit(orow, d0, acc, mx, den);
+                        }
+                    }
+                } else
 #pragma unroll 1
                 for (int rd = 0; rd < 8; ++rd) {
                     if (live_warp) {
