@@ -202,18 +202,14 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     // The next launch on the stream may start as soon as an SM has room for one of its thread blocks (its scoring
     // phase needs nothing from this one); it waits for this grid before its attention phase.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    // ---- set-up: barriers, tensor memory --------------------------------------------------------------------
-    if (tid == 0) {
-        for (int s = 0; s < kLyStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
-        for (int a = 0; a < kAtSBufs; ++a) { mbar_init(bar_s_full(a), 1); mbar_init(bar_p_full(a), 4); }
-        for (int s = 0; s < kLyPairs; ++s) { mbar_init(sbar_full(s), 1); mbar_init(sbar_empty(s), 1); }
-        for (int a = 0; a < 2; ++a) {
-            mbar_init(bar_acc_full(a), 1);
-            mbar_init(bar_acc_empty(a), 4);
-            mbar_init(bar_b_full(a), 1);
-            mbar_init(bar_b_empty(a), 1);
-        }
-        mbar_init(bar_q, 4);
+    // the first scoring tile with candidates: asked for now, so that the look-up's trip to global memory overlaps the set-up
+    const int t_first = next_active(t0);
+    // ---- set-up: barriers (one thread each), tensor memory ---------------------------------------------------
+    if (tid < kNBars) {
+        // arrival counts: the four softmax / epilogue warps arrive on P-written, accumulator-read and Q-written
+        const bool four = (tid >= 2 * kLyStages + kAtSBufs && tid < kB0) ||
+                          (tid >= kB0 + 2 * kLyPairs + 2 && tid < kB0 + 2 * kLyPairs + 4) || tid == kB0 + 2 * kLyPairs + 8;
+        mbar_init(bar_u32 + 8u * tid, four ? 4 : 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -233,7 +229,6 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         tmem_o = tmem_base + kAtSBufs * kAtTileKeys;
         tmem_q = tmem_o + kHeadDim;                                  // Q as the A operand: 128 rows x 64 packed columns
     }
-    const int t_first = next_active(t0);
     if (warp == 0) {
         bool alive = true;
         int it = 0;                                                  // scoring tiles issued
