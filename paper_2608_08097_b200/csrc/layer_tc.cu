@@ -689,8 +689,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                     l_sm[m_row] = l_sum;
                 }
                 float mx = -CUDART_INF_F, den = 0.f, wt[COPIES];
-                if (!MULTI) {
-                    // the thread block's only work item: the ring is idle, so whole O rows meet there in one round
+                if (!MULTI || k + 1 == n_my_rows) {
+                    // the thread block's only (or last) work item: the ring is idle, so whole O rows meet there in one round
                     // ([MMA_M][132] floats) and the (row, slice of the dims) tasks go to the first MMA_M threads
                     float *o_big = reinterpret_cast<float *>(base_ptr + kAtQBytes);
                     if (live_warp) {
