@@ -244,6 +244,16 @@ def section_shapes(args, dev, hbm_peak):
             t_layer = graph_time(fused, n_rot)
             row["layer_us"] = round(t_layer, 1)
             row["layer_frac"] = round((sb + ab) / t_layer / 1e3 / hbm_peak, 3)
+        if name == "configs[1]":
+            # step 0 at full size: the summaries of every full block of the layer from a device-resident pool
+            kvs = [torch.randn((Bq * mb, Hkv, 2, 16, 128), device=dev, generator=g, dtype=torch.float32).to(torch.bfloat16)
+                   for _ in range(n_rot)]
+            zeros = torch.zeros(Bq, dtype=torch.int32, device=dev)
+            torch.cuda.synchronize()
+            t_sum = graph_time(lambda i: Ls[i].build_summaries(kvs[i], table, zeros, n_full, mb), n_rot, iters=12)
+            row["summaries_full_build_us"] = round(t_sum, 1)
+            row["summaries_full_build_frac"] = round(Bq * Hkv * nf * (4096 + 512) / t_sum / 1e3 / hbm_peak, 3)
+            del kvs
         rows.append(row)
         del Ls
         torch.cuda.empty_cache()
