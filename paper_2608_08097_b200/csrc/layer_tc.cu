@@ -6,12 +6,15 @@
 // one persistent CTA per SM does both over one ring of shared memory:
 //   scoring phase    (every CTA)         a contiguous range of the layer's scoring tiles, exactly as in
 //                    score_tc.cu (2-D TMA tiles of 128 summaries, swap-AB contraction against (q^- | q^+));
-//   attention phase  (CTA c: rows c, c + grid, c + 2 grid, ...)  the sparse attention of whole (request,
-//                    KV head) rows, one after the other, exactly as in attn_tc.cu (5-D TMA entry copies,
-//                    Q K^T and P V issued by two warps, one softmax thread per MMA row with row copies).
-//                    Tiles are counted through all rows of the CTA, so the ring and the S buffers never
-//                    drain between rows; Q of the next row goes to tensor memory while the row before it
-//                    is written out.
+//   attention phase  (CTA c: work items c, c + grid, c + 2 grid, ...)  the sparse attention of whole
+//                    (request, KV head) rows, one after the other, exactly as in attn_tc.cu (5-D TMA entry
+//                    copies, Q K^T and P V issued by two warps, one softmax thread per MMA row with row
+//                    copies).  Tiles are counted through all rows of the CTA, so the ring and the S buffers
+//                    never drain between rows; Q of the next row goes to tensor memory while the row before
+//                    it is written out.  With fewer rows than half the SMs and rows too long to attend
+//                    whole, a work item is one split of a row's column list (split as attn.cu splits) and
+//                    writes a normalised partial; the merge launch follows on the stream.
+//                    The row copies of a CTA's last work item meet in the ring, idle by then, in one round.
 // The ring's six 32 KiB stages serve the scoring phase as three 64 KiB stages; the producer starts the
 // attention copies into a stage as soon as the scoring tiles that last used its pair have been
 // consumed, so the stream of bytes into the SM never stops between the phases.  The scoring ranges
