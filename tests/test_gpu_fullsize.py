@@ -95,6 +95,20 @@ def test_full_size_config(oracle, gpu, name, cfg, sample):
     kth = picked[..., -1:]
     assert ((sc > kth).sum(-1) <= k - 1).all()                        # nothing better was left out
     assert np.isfinite(pu.bf16_to_f32_np(L.out)).all()
+    # the fused attention + scoring launch (what the decode engine and bench.py run) at the same full size:
+    # scores bit for bit, outputs bit for bit unless it attends whole rows where the separate call splits them
+    binding = gpu[0]
+    T = q_dev.shape[1]
+    if binding.attn_and_score_supported(L.dims, T, L.cols, T - 1):
+        want_out, want_scores = L.out.clone(), L.scores.clone()
+        L.out.fill_(float("nan"))
+        L.scores.fill_(float("nan"))
+        L.attend_and_score(q_dev, seq_len, n_full)
+        torch.cuda.synchronize()
+        assert torch.equal(L.scores.view(torch.int32), want_scores.view(torch.int32))
+        if not torch.equal(L.out.view(torch.int16), want_out.view(torch.int16)):
+            assert 2 * cfg.batch * cfg.n_kv_heads <= torch.cuda.get_device_properties(dev).multi_processor_count
+            torch.testing.assert_close(L.out.float(), want_out.float(), atol=2e-3, rtol=1e-2)
 
 
 def test_full_size_budget_and_draft_sweep(oracle, gpu):
