@@ -108,7 +108,7 @@ class DecodeEngine:
     """
 
     def __init__(self, batch, n_q_heads, n_kv_heads, max_blocks, k, n_q_tokens, n_layers,
-                 device="cuda", mode="fetch_all", cap=None, fused=None, transfer_streams=1):
+                 device="cuda", mode="fetch_all", cap=None, fused=None, transfer_streams=1, defer_tail=False):
         assert mode in ("fetch_all", "delta")
         self.mode, self.k, self.T, self.n_layers = mode, k, n_q_tokens, n_layers
         self.device = torch.device(device)
@@ -129,6 +129,12 @@ class DecodeEngine:
                                    for _ in range(max(1, int(transfer_streams)) - 1)]
         self.launches = 0
         self.cap = cap
+        # defer_tail: the last layer's prediction chain (top-k, plan, gather) of a step is launched at the start of
+        # the next step instead of at its end, where nothing would overlap it (the next step's attention of that
+        # layer comes last and waits for it as usual); `flush()` launches a chain that is still pending.
+        self.defer_tail = bool(defer_tail)
+        self._deferred = None
+        self._capturing = False
         can_fuse = n_layers > 0 and n_q_tokens > 1 and oasis.attn_and_score_supported(self.layers[0].dims, n_q_tokens, self.layers[0].cols, n_q_tokens - 1)
         self.fused = can_fuse if fused is None else (bool(fused) and can_fuse)
         self.stage_done = [None] * n_layers          # event of the layer's latest transfer
@@ -181,7 +187,8 @@ class DecodeEngine:
         # top-k and the transfer plan run on their own stream, so that waiting for this layer's attention does
         # not hold back the next layer's scoring
         with torch.cuda.stream(qs):
-            qs.wait_event(scored)
+            if scored != "completed":                # (a chain deferred into the next captured step: all done)
+                qs.wait_event(scored)
             if attn_done is not None:
                 qs.wait_event(attn_done)            # sel / resident are read by this step's attention
             t0 = self._tick(timers, "select", qs)
@@ -266,6 +273,7 @@ class DecodeEngine:
         out_host (pinned tensors per layer) the step's queries are copied in and its outputs
         copied out inside the step (end-to-end mode)."""
         ms, cs = self.main, self.copy
+        self._launch_deferred(timers)
         q_ready = [None] * self.n_layers
         if q_host is not None or out_host is not None:
             # the copy stream starts after everything the previous step left on the other streams
@@ -319,6 +327,10 @@ class DecodeEngine:
                     out_host[l].copy_(L.out, non_blocking=True)
             if q_ready[l] is not None and not self.fused:
                 self.pred.wait_event(q_ready[l])
+            if self.defer_tail and self.fused and l == self.n_layers - 1:
+                self._deferred = (l, q_list[l], first_block, n_new, n_full_next, seq_next, step_stamp, attn_done,
+                                  self._capturing)
+                continue
             ready = self._predict(l, q_list[l], first_block, n_new, 1, n_full_next, seq_next, step_stamp, timers,
                                   attn_done=attn_done, scored=attn_done if self.fused else None)
             self._transfer(l, ready, timers)
@@ -326,6 +338,25 @@ class DecodeEngine:
             ev = torch.cuda.Event()                  # the next step's attention overwrites the output buffers
             ev.record(cs)
             ms.wait_event(ev)
+
+    def _launch_deferred(self, timers=None):
+        if self._deferred is None:
+            return
+        l, q, first_block, n_new, n_full_next, seq_next, stamp, attn_done, was_captured = self._deferred
+        self._deferred = None
+        if self._capturing:
+            attn_done = None                         # a graph starts after everything before it has completed
+        elif was_captured:
+            attn_done = torch.cuda.Event()           # the step was a graph replayed on the foreground stream
+            attn_done.record(self.main)
+        ready = self._predict(l, q, first_block, n_new, 1, n_full_next, seq_next, stamp, timers,
+                              attn_done=attn_done, scored="completed")
+        self._transfer(l, ready, timers)
+
+    def flush(self):
+        """Launches the prediction chain that `defer_tail` left pending (after the last step, or before reading the
+        last layer's selection state)."""
+        self._launch_deferred()
 
     def join(self):
         """Makes the foreground stream wait for everything the other streams have in flight."""
@@ -344,6 +375,7 @@ class DecodeEngine:
         before = self.launches
         g = torch.cuda.CUDAGraph()
         fork = torch.cuda.Event()
+        self._capturing = True
         with torch.cuda.graph(g, stream=self.main, capture_error_mode="thread_local"):
             fork.record(self.main)
             self.pred.wait_event(fork)
@@ -353,6 +385,7 @@ class DecodeEngine:
             self.copy.wait_event(fork)
             self.step(*args, **kwargs)
             self.join()
+        self._capturing = False
         g.launches = self.launches - before
         self.launches = before
         return g

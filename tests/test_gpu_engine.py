@@ -207,3 +207,53 @@ def test_fused_engine_equals_unfused_engine(gpu, mode, cap):
             assert torch.equal(a.layers[l].sel, b.layers[l].sel)
             assert torch.equal(a.blk_tbl(l), b.blk_tbl(l))
             assert torch.equal(a.layers[l].pool.view(torch.int16), b.layers[l].pool.view(torch.int16))
+
+
+@pytest.mark.parametrize("graph", [True, False])
+def test_deferred_tail_engine_equals_plain_engine(gpu, graph):
+    """defer_tail launches the last layer's prediction chain at the start of the next step instead of at the end
+    of its own: every step's outputs, and after a final flush every layer's selection, working set and pool, must
+    equal those of the engine that does not defer."""
+    binding, pipeline = gpu
+    dev = torch.device("cuda")
+    n_layers, S = 3, 7
+    cfg = synth.scaled(synth.C2, batch=16, context=1040, k_blocks=12, layers=n_layers, steps=S)
+    lays = [synth.make_layer(cfg, seed=52, layer=l, device=dev) for l in range(n_layers)]
+    seq = lays[0].seq_len_steps
+    to_dev = lambda t: t.to(torch.int32).contiguous().to(dev)
+    engines = []
+    for defer in (True, False):
+        eng = pipeline.DecodeEngine(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_blocks, cfg.k_blocks,
+                                    cfg.n_q_tokens, n_layers, dev, mode="delta", cap=2, defer_tail=defer)
+        assert eng.fused
+        for l, lay in enumerate(lays):
+            eng.attach(l, lay.host_kv.to(dev), lay.block_table.to(dev))
+        engines.append(eng)
+    q_dev = [lay.q_steps.to(dev) for lay in lays]
+    for eng in engines:
+        eng.prime([q_dev[l][0] for l in range(n_layers)], to_dev(seq[0] // 16), to_dev(seq[0]))
+    keep = []                                                       # the graphs' argument tensors stay alive
+    for s in range(S):
+        args = ([q_dev[l][s] for l in range(n_layers)], to_dev(seq[s]), to_dev(seq[s] // 16),
+                to_dev((seq[s] + 1) // 16 - seq[s] // 16), to_dev((seq[s] + 1) // 16), to_dev(seq[s] + 1))
+        keep.append(args)
+        for eng in engines:
+            if graph:
+                g = eng.capture_step(*args, step_stamp=s + 1)
+                keep.append(g)
+                eng.replay(g)
+            else:
+                eng.step(*args, step_stamp=s + 1)
+                eng.join()
+        torch.cuda.synchronize()
+        a, b = engines
+        for l in range(n_layers):
+            assert torch.equal(a.layers[l].out.view(torch.int16), b.layers[l].out.view(torch.int16)), (s, l)
+    engines[0].flush()
+    engines[0].join()
+    torch.cuda.synchronize()
+    a, b = engines
+    for l in range(n_layers):
+        assert torch.equal(a.layers[l].sel, b.layers[l].sel)
+        assert torch.equal(a.blk_tbl(l), b.blk_tbl(l))
+        assert torch.equal(a.layers[l].pool.view(torch.int16), b.layers[l].pool.view(torch.int16))
