@@ -87,7 +87,9 @@ class ClockSampler:
         self.index, self.thread, self.stop_flag = index, None, threading.Event()
         self.clocks, self.reason_bits, self.max_mhz = [], 0, None
 
-    def _run(self):
+    def _open(self):
+        """NVML set-up, done before the timed region starts (the first nvmlInit of a process can take longer than a
+        short timed region)."""
         try:
             import pynvml
             pynvml.nvmlInit()
@@ -98,19 +100,28 @@ class ClockSampler:
                     idx = int(visible.split(",")[self.index])
                 except ValueError:
                     pass
-            h = pynvml.nvmlDeviceGetHandleByIndex(idx)
-            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM)
-            while not self.stop_flag.is_set():
-                self.clocks.append(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM))
-                self.reason_bits |= int(pynvml.nvmlDeviceGetCurrentClocksEventReasons(h))
-                time.sleep(0.004)
+            self._nvml = pynvml
+            self._handle = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._handle, pynvml.NVML_CLOCK_SM)
         except Exception:          # NVML missing or refused: report no samples
+            self._nvml = self._handle = None
+
+    def _run(self):
+        try:
+            nv, h = self._nvml, self._handle
+            while not self.stop_flag.is_set():
+                self.clocks.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(h))
+                time.sleep(0.002)
+        except Exception:
             pass
 
     def start(self):
+        self._open()
+        if self._handle is None:
+            return
         self.thread = threading.Thread(target=self._run, daemon=True)
         self.thread.start()
-        time.sleep(0.02)
 
     def stop(self):
         self.stop_flag.set()
@@ -215,13 +226,10 @@ class Bench:
         cfg = self.cfg
         # gathers from pinned host memory alternate between three transfer streams (about 3 % on the end-to-end step:
         # a gather's first requests are in flight while the previous gather's last ones come back)
-        # With the pool in HBM the last layer's prediction chain of a step is launched at the start of the next step
-        # (its 35 us would otherwise run alone at the end of every step); the chain left over by the last timed step
-        # is launched, and waited for, inside the timed region.
         host_pool = len(kv_list) > 0 and not kv_list[0].is_cuda
         eng = self.pipeline.DecodeEngine(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_blocks, cfg.k_blocks,
                                          cfg.n_q_tokens, self.n_layers, self.dev, mode=mode, cap=cap,
-                                         transfer_streams=3 if host_pool else 1, defer_tail=not host_pool)
+                                         transfer_streams=3 if host_pool else 1)
         for l in range(self.n_layers):
             eng.attach(l, kv_list[l], self.tables[l])
         eng.prime([self.q_dev[l][0] for l in range(self.n_layers)], self.first_dev[0].contiguous(), self.seq_dev[0].contiguous())
