@@ -105,6 +105,12 @@ class DecodeEngine:
     fused (default: whenever the library takes the shapes): a layer's attention and its scoring run
     as one launch on the foreground stream (`oasis_attn_and_score`); the summary updates of all
     layers are then issued at the start of the step on the prediction stream.
+    transfer_streams: consecutive layers' gathers alternate between this many transfer streams (useful
+    when the pool is in host memory: one gather's requests are in flight while the previous one's last
+    ones come back).
+    defer_tail: the last layer's prediction chain of a step is launched at the start of the next step
+    (`flush()` launches a chain still pending); the state of that layer is then one step behind
+    between steps.
     """
 
     def __init__(self, batch, n_q_heads, n_kv_heads, max_blocks, k, n_q_tokens, n_layers,
