@@ -75,6 +75,18 @@ int oasis_build_summaries(const oasis_dims_t *dims, const void *kv_pool,
                           void *stream);
 
 /*
+ * Step 0 for several layers in one launch: the same as one oasis_build_summaries call per layer with that
+ * layer's pool, block table and summaries (host arrays of n_layers device pointers; first_block, n_blocks
+ * and max_new_blocks are shared, as a decode step appends the same positions to every layer's cache).
+ * n_layers may not exceed OASIS_MAX_LAYERS.
+ */
+#define OASIS_MAX_LAYERS 128
+int oasis_build_summaries_layers(const oasis_dims_t *dims, int32_t n_layers, const void *const *kv_pools,
+                                 const int32_t *const *block_tables, const int32_t *first_block,
+                                 const int32_t *n_blocks, int32_t max_new_blocks, void *const *summaries,
+                                 void *stream);
+
+/*
  * Dense -> sparse hand-over (Sec. 4.3: a request prefills and decodes densely; once its context
  * exceeds the sparsification threshold the full KV cache is copied to CPU memory and only the
  * selected blocks and a local window stay on the GPU; both pools keep their blocks in

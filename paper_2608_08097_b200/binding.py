@@ -21,7 +21,8 @@ SYMBOLS = ("oasis_build_summaries", "oasis_score_blocks", "oasis_select_topk",
            "oasis_stage_blocks", "oasis_sparse_attn", "oasis_attn_workspace_bytes",
            "oasis_plan_delta", "oasis_last_error", "oasis_version",
            "oasis_sparse_attn_static_scratch", "oasis_static_scratch_bytes", "oasis_set_error_word", "oasis_union_blocks",
-           "oasis_offload_blocks", "oasis_attn_and_score", "oasis_attn_and_score_supported")
+           "oasis_offload_blocks", "oasis_attn_and_score", "oasis_attn_and_score_supported",
+           "oasis_build_summaries_layers")
 
 
 class OasisError(RuntimeError):
@@ -82,6 +83,8 @@ def lib():
         L.oasis_attn_and_score.argtypes = [dp, vp, i32, vp, vp, vp, i32, vp, ctypes.c_float, vp, vp, vp, ctypes.c_int64, i32, vp, vp,
                                            i32, vp, vp, ctypes.c_size_t, vp]
         L.oasis_attn_and_score.restype = ctypes.c_int
+        L.oasis_build_summaries_layers.argtypes = [dp, i32, vp, vp, vp, vp, i32, vp, vp]
+        L.oasis_build_summaries_layers.restype = ctypes.c_int
         L.oasis_attn_and_score_supported.argtypes = [dp, i32, i32, i32]
         L.oasis_attn_and_score_supported.restype = ctypes.c_int
         L.oasis_union_blocks.restype = ctypes.c_int
@@ -133,6 +136,26 @@ def build_summaries(dims, kv_pool, block_table, first_block, n_blocks, max_new_b
         _ptr(block_table, torch.int32, "block_table"), _ptr(first_block, torch.int32, "first_block"),
         _ptr(n_blocks, torch.int32, "n_blocks"), int(max_new_blocks),
         _ptr(summaries, torch.bfloat16, "summaries"), _stream(stream)), "oasis_build_summaries")
+
+
+MAX_LAYERS = 128
+
+
+def build_summaries_layers(dims, kv_pools, block_tables, first_block, n_blocks, max_new_blocks, summaries,
+                           stream=None):
+    """oasis_build_summaries for several layers in one launch: lists of per-layer tensors."""
+    n = len(kv_pools)
+    if not (len(block_tables) == n and len(summaries) == n):
+        raise ValueError("kv_pools, block_tables and summaries must have one tensor per layer")
+    d = dims.c()
+    arr = ctypes.c_void_p * max(n, 1)
+    kv = arr(*[_ptr(t, torch.bfloat16, "kv_pools").value for t in kv_pools])
+    bt = arr(*[_ptr(t, torch.int32, "block_tables").value for t in block_tables])
+    sm = arr(*[_ptr(t, torch.bfloat16, "summaries").value for t in summaries])
+    _check(lib().oasis_build_summaries_layers(
+        ctypes.byref(d), n, kv, bt, _ptr(first_block, torch.int32, "first_block"),
+        _ptr(n_blocks, torch.int32, "n_blocks"), int(max_new_blocks), sm, _stream(stream)),
+        "oasis_build_summaries_layers")
 
 
 def score_blocks(dims, q_draft, n_draft, summaries, n_full_blocks, scores, reduce_mode=REDUCE_MAX,

@@ -25,11 +25,10 @@ __device__ __forceinline__ uint32_t max2(uint32_t a, uint32_t b)
     return r;
 }
 
-__global__ void __launch_bounds__(kSummWarps * 32)
-build_summaries_kernel(const uint8_t *__restrict__ kv_pool, const int32_t *__restrict__ block_table,
-                       const int32_t *__restrict__ first_block, const int32_t *__restrict__ n_blocks,
-                       uint8_t *__restrict__ summaries, int B, int Hkv, int max_blocks,
-                       int max_new, long long n_items)
+__device__ __forceinline__ void
+summarise_item(const uint8_t *__restrict__ kv_pool, const int32_t *__restrict__ block_table,
+               const int32_t *__restrict__ first_block, const int32_t *__restrict__ n_blocks,
+               uint8_t *__restrict__ summaries, int Hkv, int max_blocks, int max_new, long long n_items)
 {
     const int lane = threadIdx.x & 31;
     const long long item = (long long)blockIdx.x * kSummWarps + (threadIdx.x >> 5);
@@ -74,6 +73,32 @@ build_summaries_kernel(const uint8_t *__restrict__ kv_pool, const int32_t *__res
     *reinterpret_cast<uint4 *>(dst + lane * 16) = o;
 }
 
+__global__ void __launch_bounds__(kSummWarps * 32)
+build_summaries_kernel(const uint8_t *__restrict__ kv_pool, const int32_t *__restrict__ block_table,
+                       const int32_t *__restrict__ first_block, const int32_t *__restrict__ n_blocks,
+                       uint8_t *__restrict__ summaries, int B, int Hkv, int max_blocks,
+                       int max_new, long long n_items)
+{
+    summarise_item(kv_pool, block_table, first_block, n_blocks, summaries, Hkv, max_blocks, max_new, n_items);
+}
+
+// The same for several layers in one launch (blockIdx.y = layer): a decode step appends to every layer's cache
+// at once, and one launch instead of one per layer keeps 31 small launches out of the step.
+struct SummLayers {
+    const uint8_t *kv_pool[OASIS_MAX_LAYERS];
+    const int32_t *block_table[OASIS_MAX_LAYERS];
+    uint8_t *summaries[OASIS_MAX_LAYERS];
+};
+
+__global__ void __launch_bounds__(kSummWarps * 32)
+build_summaries_layers_kernel(const __grid_constant__ SummLayers ly, const int32_t *__restrict__ first_block,
+                              const int32_t *__restrict__ n_blocks, int Hkv, int max_blocks, int max_new, long long n_items)
+{
+    const int l = blockIdx.y;
+    summarise_item(ly.kv_pool[l], ly.block_table[l], first_block, n_blocks, ly.summaries[l], Hkv, max_blocks, max_new,
+                   n_items);
+}
+
 }  // namespace oasis
 
 extern "C" int oasis_build_summaries(const oasis_dims_t *dims, const void *kv_pool,
@@ -99,4 +124,38 @@ extern "C" int oasis_build_summaries(const oasis_dims_t *dims, const void *kv_po
         (const uint8_t *)kv_pool, block_table, first_block, n_blocks, (uint8_t *)summaries,
         dims->batch, dims->n_kv_heads, dims->max_blocks, max_new_blocks, n_items);
     return check_launch("oasis_build_summaries");
+}
+
+extern "C" int oasis_build_summaries_layers(const oasis_dims_t *dims, int32_t n_layers, const void *const *kv_pools,
+                                            const int32_t *const *block_tables, const int32_t *first_block,
+                                            const int32_t *n_blocks, int32_t max_new_blocks, void *const *summaries,
+                                            void *stream)
+{
+    using namespace oasis;
+    const char *who = "oasis_build_summaries_layers";
+    if (int rc = check_dims(dims)) return rc;
+    if (n_layers < 0 || n_layers > OASIS_MAX_LAYERS)
+        return fail(OASIS_ERR_INVALID_ARG, "%s: n_layers %d outside [0, %d]", who, n_layers, OASIS_MAX_LAYERS);
+    if (!kv_pools || !block_tables || !summaries || !first_block || !n_blocks)
+        return fail(OASIS_ERR_INVALID_ARG, "%s: NULL pointer argument", who);
+    if (max_new_blocks < 0 || max_new_blocks > dims->max_blocks)
+        return fail(OASIS_ERR_INVALID_ARG, "%s: max_new_blocks %d outside [0, %d]", who, max_new_blocks, dims->max_blocks);
+    SummLayers ly = {};
+    for (int l = 0; l < n_layers; ++l) {
+        if (!kv_pools[l] || !block_tables[l] || !summaries[l])
+            return fail(OASIS_ERR_INVALID_ARG, "%s: NULL pointer for layer %d", who, l);
+        if (!aligned16(kv_pools[l]) || !aligned16(summaries[l]))
+            return fail(OASIS_ERR_INVALID_ARG, "%s: kv_pools and summaries must be 16-byte aligned (layer %d)", who, l);
+        ly.kv_pool[l] = (const uint8_t *)kv_pools[l];
+        ly.block_table[l] = block_tables[l];
+        ly.summaries[l] = (uint8_t *)summaries[l];
+    }
+    const long long n_items = (long long)dims->batch * dims->n_kv_heads * max_new_blocks;
+    if (n_items == 0 || n_layers == 0) return OASIS_OK;
+    const long long grid = (n_items + kSummWarps - 1) / kSummWarps;
+    if (grid > 0x7fffffffLL) return fail(OASIS_ERR_UNSUPPORTED, "%s: too many blocks", who);
+    prefer_max_shared_carveout(build_summaries_layers_kernel);
+    build_summaries_layers_kernel<<<dim3((unsigned)grid, (unsigned)n_layers), kSummWarps * 32, 0, (cudaStream_t)stream>>>(
+        ly, first_block, n_blocks, dims->n_kv_heads, dims->max_blocks, max_new_blocks, n_items);
+    return check_launch(who);
 }

@@ -303,10 +303,16 @@ class DecodeEngine:
             # the summary updates (one newly completed block per request every 16 steps) only depend on this step's
             # KV append: all layers' updates go first, on the prediction stream
             with torch.cuda.stream(self.pred):
-                for l in range(self.n_layers):
-                    self.layers[l].build_summaries(self.kv[l], self.table[l], first_block, n_new, 1)
-                    summ_ready[l] = torch.cuda.Event()
-                    summ_ready[l].record(self.pred)
+                for l0 in range(0, self.n_layers, oasis.MAX_LAYERS):       # one launch for (up to 128) layers
+                    l1 = min(l0 + oasis.MAX_LAYERS, self.n_layers)
+                    oasis.build_summaries_layers(self.layers[l0].dims, self.kv[l0:l1], self.table[l0:l1], first_block,
+                                                 n_new, 1, [L.summaries for L in self.layers[l0:l1]])
+                    self.launches += 1
+                    # only the group's first fused launch waits for it: the later ones follow that launch on the
+                    # foreground stream (a wait for the same, already awaited launch before every fused launch made
+                    # the captured graph drop the programmatic edges between consecutive fused launches)
+                    summ_ready[l0] = torch.cuda.Event()
+                    summ_ready[l0].record(self.pred)
         for l in range(self.n_layers):
             L = self.layers[l]
             with torch.cuda.stream(ms):
@@ -315,11 +321,12 @@ class DecodeEngine:
                 if self.stage_done[l] is not None:
                     ms.wait_event(self.stage_done[l])
                 if self.fused:
-                    ms.wait_event(summ_ready[l])
+                    if summ_ready[l] is not None:
+                        ms.wait_event(summ_ready[l])
                     t0 = self._tick(timers, "layer", ms)
                     L.attend_and_score(q_list[l], seq_len, n_full_next, blk_tbl=self.blk_tbl(l))
                     self._tock(timers, "layer", t0, ms)
-                    self.launches += 3 if self._splits else 2      # the fused launch (and the merge of split rows), the summary update
+                    self.launches += 2 if self._splits else 1      # the fused launch (and the merge of split rows)
                 else:
                     t0 = self._tick(timers, "attn", ms)
                     L.attend(q_list[l], seq_len, blk_tbl=self.blk_tbl(l))

@@ -524,3 +524,29 @@ def test_fused_call_wants_its_workspace_when_it_splits(gpu):
     zf = torch.zeros(1 << 12, dtype=torch.float32, device=dev)
     with pytest.raises(binding.OasisError, match="workspace"):
         binding.attn_and_score(dims, z16, 5, z16, zi, zi, 130, zi, 0.1, z16, z16, 4, z16, zi, zf)
+
+
+def test_build_summaries_layers_equals_per_layer_calls(gpu):
+    """One launch for several layers writes exactly what one oasis_build_summaries call per layer writes
+    (which the other tests check against the oracle), and nothing else."""
+    binding, pipeline = gpu
+    dev = torch.device("cuda")
+    cfg = synth.scaled(synth.C1, batch=3, context=1040, k_blocks=8)
+    n_layers = 5
+    lays = [synth.make_layer(cfg, seed=70 + l, ragged=True, permute_table=True) for l in range(n_layers)]
+    dims = binding.Dims(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_blocks)
+    kvs = [lay.host_kv.to(dev) for lay in lays]
+    tables = [lay.block_table.to(dev) for lay in lays]
+    n_full = lays[0].n_full.to(dev)
+    first = torch.tensor([0, 3, 7], dtype=torch.int32, device=dev)
+    n_new = torch.minimum(n_full - first, torch.tensor([40, 1, 9], dtype=torch.int32, device=dev)).contiguous()
+    shape = (cfg.batch, cfg.n_kv_heads, cfg.max_blocks, 2, 128)
+    want = [torch.full(shape, 7.0, dtype=torch.bfloat16, device=dev) for _ in range(n_layers)]
+    got = [torch.full(shape, 7.0, dtype=torch.bfloat16, device=dev) for _ in range(n_layers)]
+    for l in range(n_layers):
+        binding.build_summaries(dims, kvs[l], tables[l], first, n_new, 40, want[l])
+    binding.build_summaries_layers(dims, kvs, tables, first, n_new, 40, got)
+    torch.cuda.synchronize()
+    for l in range(n_layers):
+        assert torch.equal(got[l].view(torch.int16), want[l].view(torch.int16))
+    assert not torch.equal(want[0].view(torch.int16), torch.full(shape, 7.0, dtype=torch.bfloat16, device=dev).view(torch.int16))
