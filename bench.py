@@ -32,7 +32,7 @@ import torch  # noqa: E402
 from paper_2608_08097_b200 import synth  # noqa: E402
 
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (configs[1] shapes)
-TRAFFIC_BYTES = {"score": 139.0e6, "attn": 140.3e6, "layer": 275.6e6}
+TRAFFIC_BYTES = {"score": 139.0e6, "attn": 140.3e6, "layer": 277.3e6}
 
 METRIC = "sparse decode-attn+select tokens/s per layer"
 UNIT = "tokens/s/layer"
