@@ -177,6 +177,10 @@ int oasis_stage_blocks(const void *host_kv, const int64_t *idx, const int32_t *s
  *               May be NULL when that function returns 0.
  * n_q_tokens * (Hq/Hkv) may not exceed 128.  A query row that sees no key yields zeros
  * (lse = -inf).
+ * Every byte of an entry named by a column with blk_tbl >= 0 must be a finite bf16 pattern, also the
+ * token rows that lie past the visible positions (the unwritten tail of the local block): masked keys
+ * enter the P V product with weight zero, and 0 x NaN or 0 x Inf is NaN.  A pool that was zeroed
+ * once and only ever receives real keys and values satisfies this.
  */
 int oasis_sparse_attn(const oasis_dims_t *dims, const void *q, int32_t n_q_tokens,
                       const void *hbm_pool, const int32_t *slot_tbl, const int32_t *blk_tbl,
@@ -202,6 +206,14 @@ size_t oasis_attn_workspace_bytes(const oasis_dims_t *dims, int32_t n_q_tokens,
  * footprint within 227 KiB are taken (oasis_attn_and_score_supported tells); others
  * return OASIS_ERR_UNSUPPORTED: make the two calls.
  *   q_batch_stride   elements between consecutive requests of q_draft (0 = dense)
+ * Stream ordering.  The kernel is launched with programmatic stream serialization and its scoring phase
+ * runs before it waits for the previous launch of `stream`: q_draft, summaries, n_full_blocks and seq_len
+ * are read, and scores written, while that previous launch may still be running, and the launch after this
+ * one may start as soon as this one has begun.  So the previous launch on `stream` must neither produce
+ * those inputs nor still use `scores` (an oasis_attn_and_score of another layer is the intended
+ * predecessor); separate such producers and consumers from this call by an event on another stream or by
+ * another launch in between.  Everything the attention phase touches (q,
+ * hbm_pool, the tables, out, lse, workspace) is ordered as usual.
  */
 int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int32_t n_q_tokens, const void *hbm_pool,
                          const int32_t *slot_tbl, const int32_t *blk_tbl, int32_t n_cols,
@@ -294,6 +306,16 @@ int oasis_union_blocks(const oasis_dims_t *dims, const int32_t *sel, int32_t sel
  * process-wide and is only ever written with a compare-and-swap from zero.
  */
 int oasis_set_error_word(int32_t *device_word);
+
+/*
+ * Self-test of the bounded waits behind oasis_set_error_word (no counterpart in the paper).  One small
+ * launch waits, with a bound of `probes` polls (1 .. 2^20), on a barrier that nothing ever completes; the
+ * wait gives up, the kernel records code 99 in the registered error word (if one is registered and still
+ * zero), releases what it holds and returns -- the path the real kernels take when a copy or tensor-core
+ * operation never signals.  result (device, int32[2], may be NULL) receives {1 if the wait gave up else 0,
+ * the code}.  Nothing is left in flight; later calls work as usual.
+ */
+int oasis_selftest_wait_timeout(uint32_t probes, int32_t *result, void *stream);
 
 /* Description of the calling thread's most recent error ("" if none). Static storage. */
 const char *oasis_last_error(void);

@@ -69,8 +69,8 @@ void oasis_oracle_bf16_to_f32(const uint16_t *src, float *dst, int64_t n)
 }
 
 /* ---------------------------------------------------------------- step 0: summaries
- * Sec. 4.2.1 ("Quest-style summaries ... coordinate-wise minimum and maximum of the
- * keys in each logical block"), Fig. "Look-ahead attention" (per-block min/max pooling),
+ * Sec. 4.2.1 (per logical block and KV head, one summary row holds the smallest and one
+ * the largest value of every key coordinate), Fig. "Look-ahead attention" (min/max pooling),
  * Sec. 5.2 (two summary rows per block = 1/16 of the KV size, hence bf16 like the KV).
  * For request b, logical blocks first_block[b] .. first_block[b]+n_blocks[b]-1.
  */
@@ -102,8 +102,8 @@ void oasis_oracle_build_summaries(int32_t B, int32_t Hkv, int32_t d, int32_t bs,
 }
 
 /* ---------------------------------------------------------------- step 1: scores
- * Sec. 4.2.1: "each draft query scans these summaries and ranks all logical blocks
- * independently for every KV head".  The estimate for one query row q and block j is
+ * Sec. 4.2.1: the draft queries are compared with every block's summary, separately for
+ * each KV head, and the blocks are ranked by the result.  The estimate for one query row q and block j is
  * the Quest upper bound  U(q, j) = sum_x max(q_x * min_jx, q_x * max_jx), summed over
  * x ascending.  The Td draft tokens and the G = Hq/Hkv query heads that share KV head
  * h give R = Td*G rows; they are reduced with max (reduce_mode 0) or sum (1), rows
@@ -503,8 +503,8 @@ void oasis_oracle_union_blocks(int32_t B, int32_t Hkv, int32_t max_blocks, int32
 }
 
 /* ---------------------------------------------------------------- dense -> sparse hand-over
- * Sec. 4.3: "A request initially performs prefill and decoding densely ...  Once its context
- * exceeds the sparsification threshold, [the system] copies the full KV cache to CPU memory";
+ * Sec. 4.3: a request starts out dense (prefill and the first decode steps); when its context
+ * grows past the sparsification threshold its whole KV cache is moved to the CPU pool;
  * both pools keep their blocks in Head-Token-Dimension order and each has its own page table.
  * The dense GPU pool holds keys and values separately, dense_k / dense_v [P_gpu][Hkv][bs][d];
  * the CPU pool holds one entry [K part | V part] per (block, head).  For request b and logical
@@ -544,6 +544,92 @@ void oasis_oracle_offload_blocks(int32_t B, int32_t Hkv, int32_t d, int32_t bs, 
                     }
                     row_min[x] = lo;
                     row_max[x] = hi;
+                }
+            }
+        }
+    }
+}
+
+/* ---------------------------------------------------------------- local window and KV append
+ * Sec. 4.3 keeps, next to the selected blocks, a local window in GPU memory; Sec. 5.2 calls it the
+ * active local block (the block being written), kept on top of the K selected ones.  The paper does
+ * not say how the newest tokens reach the CPU pool; the reading taken here is write-through: the
+ * tokens a step produces are written into the local window of the GPU working set (they are produced
+ * on the GPU and never cross the host link in that direction), and the ones the step commits are
+ * also written to the CPU full-KV pool, so that a block that fills up is complete there and can be
+ * summarised, selected and gathered like any other.
+ *
+ * Geometry.  With L = seq_len[b] history tokens and T verify-step tokens, token t sits at position
+ * L + t, i.e. row (L + t) % bs of logical block (L + t) / bs.  The local blocks are lo = L / bs ..
+ * hi = (L + T - 1) / bs (T <= bs, so at most two).  Local block j lives in column local_col + (j & 1)
+ * of its (b, h) row: a block keeps its column, hence its slot, for as long as it is local, and the
+ * column of the other parity is free again by the time block j + 2 needs it.
+ *
+ * oasis_oracle_local_window: blk_tbl[b][h][local_col + (lo & 1)] = lo; the other local column = hi
+ * if hi > lo else -1.  When stage_idx / stage_slots are given ([B][Hkv][2]) request r of a row
+ * (re)loads the block of column local_col + r from the CPU pool: idx = block_table[b][j] * Hkv + h
+ * (-1 for an empty column), slot = row * slot_stride + local_col + r.
+ */
+void oasis_oracle_local_window(int32_t B, int32_t Hkv, int32_t bs, int32_t max_blocks,
+                               const int32_t *seq_len, int32_t n_q_tokens,
+                               const int32_t *block_table, int32_t *blk_tbl, int32_t n_cols,
+                               int32_t local_col, int32_t slot_stride, int64_t *stage_idx,
+                               int32_t *stage_slots)
+{
+    for (int32_t b = 0; b < B; ++b) {
+        int32_t lo = seq_len[b] / bs;
+        int32_t hi = (seq_len[b] + n_q_tokens - 1) / bs;
+        for (int32_t h = 0; h < Hkv; ++h) {
+            int64_t row = (int64_t)b * Hkv + h;
+            int32_t *cols = blk_tbl + row * n_cols + local_col;
+            cols[lo & 1] = lo;
+            cols[(lo & 1) ^ 1] = hi > lo ? hi : -1;
+            if (stage_idx && stage_slots) {
+                for (int32_t r = 0; r < 2; ++r) {
+                    int32_t j = cols[r];
+                    stage_slots[row * 2 + r] = (int32_t)(row * slot_stride + local_col + r);
+                    stage_idx[row * 2 + r] =
+                        j < 0 ? -1 : (int64_t)block_table[(int64_t)b * max_blocks + j] * Hkv + h;
+                }
+            }
+        }
+    }
+}
+
+/* oasis_oracle_append_kv: the KV append of one decode step.
+ * new_kv [B][T][Hkv][2][d] bf16: key row then value row of token t for KV head h.
+ *   1. the local columns of blk_tbl are set as in oasis_oracle_local_window;
+ *   2. every token t < T is written to row (L + t) % bs of the K part and of the V part of the pool
+ *      entry slot_tbl[b][h][local_col + (j & 1)], j = (L + t) / bs;
+ *   3. the first n_commit tokens are also written to the same rows of entry
+ *      (block_table[b][j], h) of the CPU pool host_kv (skipped when host_kv is NULL).
+ * Nothing else is touched: the rows of a local entry that earlier steps wrote stay as they are.
+ */
+void oasis_oracle_append_kv(int32_t B, int32_t T, int32_t Hkv, int32_t d, int32_t bs,
+                            int32_t max_blocks, int32_t n_commit, const uint16_t *new_kv,
+                            const int32_t *seq_len, const int32_t *block_table,
+                            const int32_t *slot_tbl, int32_t *blk_tbl, int32_t n_cols,
+                            int32_t local_col, uint16_t *pool, uint16_t *host_kv)
+{
+    const int64_t part = (int64_t)bs * d;
+    oasis_oracle_local_window(B, Hkv, bs, max_blocks, seq_len, T, block_table, blk_tbl, n_cols,
+                              local_col, 0, NULL, NULL);
+    for (int32_t b = 0; b < B; ++b) {
+        for (int32_t t = 0; t < T; ++t) {
+            int32_t pos = seq_len[b] + t;
+            int32_t j = pos / bs, i = pos % bs;
+            for (int32_t h = 0; h < Hkv; ++h) {
+                int64_t row = (int64_t)b * Hkv + h;
+                const uint16_t *src = new_kv + ((((int64_t)b * T + t) * Hkv + h) * 2) * d;
+                int64_t slot = slot_tbl[row * n_cols + local_col + (j & 1)];
+                uint16_t *entry = pool + slot * 2 * part;
+                memcpy(entry + (int64_t)i * d, src, sizeof(uint16_t) * (size_t)d);
+                memcpy(entry + part + (int64_t)i * d, src + d, sizeof(uint16_t) * (size_t)d);
+                if (host_kv && t < n_commit) {
+                    int64_t phys = block_table[(int64_t)b * max_blocks + j];
+                    uint16_t *he = host_kv + (phys * Hkv + h) * 2 * part;
+                    memcpy(he + (int64_t)i * d, src, sizeof(uint16_t) * (size_t)d);
+                    memcpy(he + part + (int64_t)i * d, src + d, sizeof(uint16_t) * (size_t)d);
                 }
             }
         }

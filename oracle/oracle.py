@@ -176,3 +176,35 @@ def offload_blocks(dense_k, dense_v, gpu_table, block_table, first_block, n_bloc
     lib().oasis_oracle_offload_blocks(B, Hkv, d, bs, max_blocks, _p(dense_k), _p(dense_v), _p(gpu_table),
                                       _p(block_table), _p(first_block), _p(n_blocks), _p(host_kv), _p(summaries))
     return host_kv
+
+
+def local_window(seq_len, n_q_tokens, block_table, blk_tbl, local_col, slot_stride, want_stage=True, bs=16):
+    """Sets the two local columns of blk_tbl [B][Hkv][n_cols] (in place) by block parity; returns
+    (stage_idx int64 [B][Hkv][2], stage_slots int32 [B][Hkv][2]) that reload them from the CPU pool."""
+    seq_len, block_table = _i32(seq_len), _i32(block_table)
+    assert blk_tbl.dtype == np.int32 and blk_tbl.flags.c_contiguous
+    B, Hkv, n_cols = blk_tbl.shape
+    max_blocks = block_table.shape[-1]
+    idx = np.empty((B, Hkv, 2), dtype=np.int64) if want_stage else None
+    slots = np.empty((B, Hkv, 2), dtype=np.int32) if want_stage else None
+    lib().oasis_oracle_local_window(B, Hkv, bs, max_blocks, _p(seq_len), int(n_q_tokens), _p(block_table),
+                                    _p(blk_tbl), n_cols, int(local_col), int(slot_stride), _p(idx), _p(slots))
+    return idx, slots
+
+
+def append_kv(new_kv, n_commit, seq_len, block_table, slot_tbl, blk_tbl, local_col, pool, host_kv=None):
+    """new_kv [B][T][Hkv][2][d] u16; pool [n_slots][2][bs][d] and host_kv [P][Hkv][2][bs][d] u16 and blk_tbl
+    [B][Hkv][n_cols] int32 are updated in place."""
+    new_kv = _u16(new_kv)
+    B, T, Hkv, _, d = new_kv.shape
+    seq_len, block_table, slot_tbl = _i32(seq_len), _i32(block_table), _i32(slot_tbl)
+    assert blk_tbl.dtype == np.int32 and blk_tbl.flags.c_contiguous
+    assert pool.dtype == np.uint16 and pool.flags.c_contiguous
+    if host_kv is not None:
+        assert host_kv.dtype == np.uint16 and host_kv.flags.c_contiguous
+    bs = pool.shape[-2]
+    n_cols = blk_tbl.shape[-1]
+    max_blocks = block_table.shape[-1]
+    lib().oasis_oracle_append_kv(B, T, Hkv, d, bs, max_blocks, int(n_commit), _p(new_kv), _p(seq_len),
+                                 _p(block_table), _p(slot_tbl), _p(blk_tbl), n_cols, int(local_col), _p(pool),
+                                 _p(host_kv))

@@ -22,7 +22,7 @@ SYMBOLS = ("oasis_build_summaries", "oasis_score_blocks", "oasis_select_topk",
            "oasis_plan_delta", "oasis_last_error", "oasis_version",
            "oasis_sparse_attn_static_scratch", "oasis_static_scratch_bytes", "oasis_set_error_word", "oasis_union_blocks",
            "oasis_offload_blocks", "oasis_attn_and_score", "oasis_attn_and_score_supported",
-           "oasis_build_summaries_layers")
+           "oasis_build_summaries_layers", "oasis_selftest_wait_timeout")
 
 
 class OasisError(RuntimeError):
@@ -88,6 +88,8 @@ def lib():
         L.oasis_attn_and_score_supported.argtypes = [dp, i32, i32, i32]
         L.oasis_attn_and_score_supported.restype = ctypes.c_int
         L.oasis_union_blocks.restype = ctypes.c_int
+        L.oasis_selftest_wait_timeout.argtypes = [ctypes.c_uint32, vp, vp]
+        L.oasis_selftest_wait_timeout.restype = ctypes.c_int
         L.oasis_set_error_word.argtypes = [vp]
         L.oasis_set_error_word.restype = ctypes.c_int
         L.oasis_last_error.restype = ctypes.c_char_p
@@ -101,6 +103,13 @@ def set_error_word(word):
     wait time-out; None unregisters."""
     _check(lib().oasis_set_error_word(None if word is None else ctypes.c_void_p(word.data_ptr())),
            "oasis_set_error_word")
+
+
+def selftest_wait_timeout(probes, result=None, stream=None):
+    """Runs the bounded-wait self-test: a wait of `probes` polls that nothing completes.  result: int32[2]
+    device tensor receiving (gave_up, code)."""
+    _check(lib().oasis_selftest_wait_timeout(int(probes), _ptr(result, torch.int32, "result"), _stream(stream)),
+           "oasis_selftest_wait_timeout")
 
 
 def last_error() -> str:

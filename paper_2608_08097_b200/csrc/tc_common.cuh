@@ -22,11 +22,11 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Bounded wait: false (and an error code) if the phase did not complete within the spin limit.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t *err, int code)
+// Bounded wait: false (and an error code in *err) if the phase did not complete within `limit` probes.
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, int32_t *err, int code, uint32_t limit)
 {
 #pragma unroll 1                 // the compiler otherwise unrolls the spin loop at every call site (half the kernel's code)
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    for (uint32_t i = 0; i < limit; ++i) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -39,6 +39,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t
     }
     if (err) atomicCAS(err, 0, code);
     return false;
+}
+// The wait every kernel uses: the compile-time limit of about four million probes (tens of milliseconds).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t *err, int code)
+{
+    return mbar_wait_limit(bar, parity, err, code, kSpinLimit);
 }
 // One non-blocking probe of a phase.
 __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)

@@ -144,6 +144,7 @@ class DecodeEngine:
         can_fuse = n_layers > 0 and n_q_tokens > 1 and oasis.attn_and_score_supported(self.layers[0].dims, n_q_tokens, self.layers[0].cols, n_q_tokens - 1)
         self.fused = can_fuse if fused is None else (bool(fused) and can_fuse)
         self.stage_done = [None] * n_layers          # event of the layer's latest transfer
+        self.sel_done = [None] * n_layers            # event of the layer's latest top-k (it reads the scores)
         if mode == "delta":
             assert cap is not None and 0 <= cap <= k
             dev, rows = self.device, (batch, n_kv_heads)
@@ -184,6 +185,9 @@ class DecodeEngine:
         own_score = scored is None
         if own_score:
             with torch.cuda.stream(ps):
+                # the scores buffer is rewritten: the previous step's top-k of this layer must have read it
+                if self.sel_done[l] is not None:
+                    ps.wait_event(self.sel_done[l])
                 L.build_summaries(self.kv[l], self.table[l], first_block, n_new, max_new)
                 t0 = self._tick(timers, "score", ps)
                 L.score(q, n_full_next)
@@ -203,6 +207,7 @@ class DecodeEngine:
             self.launches += 3 if own_score else 1      # (summary update, scoring,) top-k
             ev = torch.cuda.Event()
             ev.record(qs)
+            self.sel_done[l] = ev
         if self.mode == "delta":
             # the transfer plan runs on the transfer stream, so the next layer's top-k does not queue behind it
             with torch.cuda.stream(self.side):
@@ -271,6 +276,7 @@ class DecodeEngine:
                     st.synchronize()
         torch.cuda.synchronize(self.device)
         self.stage_done = [None] * self.n_layers     # everything has completed
+        self.sel_done = [None] * self.n_layers
 
     def step(self, q_list, seq_len, first_block, n_new, n_full_next, seq_next, step_stamp=0,
              timers=None, q_host=None, out_host=None):
@@ -385,6 +391,7 @@ class DecodeEngine:
         completes only when all streams' work of the step has completed."""
         torch.cuda.synchronize(self.device)
         self.stage_done = [None] * self.n_layers
+        self.sel_done = [None] * self.n_layers
         before = self.launches
         g = torch.cuda.CUDAGraph()
         fork = torch.cuda.Event()
@@ -399,6 +406,7 @@ class DecodeEngine:
             self.step(*args, **kwargs)
             self.join()
         self._capturing = False
+        self.sel_done = [None] * self.n_layers       # events recorded inside a capture mean nothing outside it
         g.launches = self.launches - before
         self.launches = before
         return g

@@ -1,8 +1,8 @@
 """GPU parity at the full sizes of the five benchmark configurations, in the launch
 configuration bench.py times (full batch): one layer is generated at full size, the whole
-path runs on the GPU, and sampled requests are checked against the CPU oracle element by
-element (summaries and gather exactly, indices with the fp32 near-tie rule, attention within
-atol 2e-3 / rtol 1e-2).  The oracle handles one request at a time, so it finishes in seconds."""
+path runs on the GPU, and EVERY request of the batch is checked against the CPU oracle element
+by element (summaries and gather exactly, indices with the fp32 near-tie rule, attention within
+atol 2e-3 / rtol 1e-2).  The oracle handles one request at a time (0.1 - 1 s each)."""
 import math
 
 import numpy as np
@@ -65,11 +65,11 @@ def run_full(pipeline, cfg, lay, k, q_dev, kv):
     return L, table, n_full, seq_len
 
 
-FULL = [("c1", synth.C1, [0]), ("c2", synth.C2, [0, 15]), ("c3", synth.C3, [0, 31]), ("c4", synth.C4, [0, 7])]
+FULL = [("c1", synth.C1), ("c2", synth.C2), ("c3", synth.C3), ("c4", synth.C4)]
 
 
-@pytest.mark.parametrize("name,cfg,sample", FULL, ids=[f[0] for f in FULL])
-def test_full_size_config(oracle, gpu, name, cfg, sample):
+@pytest.mark.parametrize("name,cfg", FULL, ids=[f[0] for f in FULL])
+def test_full_size_config(oracle, gpu, name, cfg):
     _, pipeline = gpu
     dev = torch.device("cuda")
     cfg = synth.scaled(cfg, layers=1, steps=1)
@@ -83,7 +83,7 @@ def test_full_size_config(oracle, gpu, name, cfg, sample):
     L.stage(lay.host_kv)
     L.attend(q_dev, seq_len)
     torch.cuda.synchronize()
-    for b in sample:
+    for b in range(cfg.batch):
         check_request(oracle, cfg, lay, L, b, k, lay.q)
     # properties that hold for every row, checked over the whole batch
     sel = L.sel.cpu().numpy()
@@ -109,6 +109,9 @@ def test_full_size_config(oracle, gpu, name, cfg, sample):
         if not torch.equal(L.out.view(torch.int16), want_out.view(torch.int16)):
             assert 2 * cfg.batch * cfg.n_kv_heads <= torch.cuda.get_device_properties(dev).multi_processor_count
             torch.testing.assert_close(L.out.float(), want_out.float(), atol=2e-3, rtol=1e-2)
+        # and the fused launch's own scores and outputs directly against the oracle, every request
+        for b in range(cfg.batch):
+            check_request(oracle, cfg, lay, L, b, k, lay.q)
 
 
 def test_full_size_budget_and_draft_sweep(oracle, gpu):
@@ -131,13 +134,15 @@ def test_full_size_budget_and_draft_sweep(oracle, gpu):
             L.stage(lay.host_kv)
             L.attend(q_dev, seq_len)
             torch.cuda.synchronize()
-            check_request(oracle, cfg, lay, L, (k + td) % cfg.batch, k, q_cpu)
+            for b in range(cfg.batch):
+                check_request(oracle, cfg, lay, L, b, k, q_cpu)
             del L
 
 
 def test_full_size_engine_steps(oracle, gpu):
     """configs[1] through the multi-layer engine exactly as bench.py drives it (full batch,
-    two layers, three consecutive steps): sampled attention outputs against the oracle."""
+    two layers, three consecutive steps): every request's selection (near-ties adjudicated with the
+    oracle's double-precision scores) and attention outputs against the oracle."""
     _, pipeline = gpu
     dev = torch.device("cuda")
     n_layers, S = 2, 3
@@ -151,24 +156,31 @@ def test_full_size_engine_steps(oracle, gpu):
     q_dev = [lay.q_steps.to(dev) for lay in lays]
     to_dev = lambda t: t.to(torch.int32).contiguous().to(dev)
     eng.prime([q_dev[l][0] for l in range(n_layers)], to_dev(seq[0] // 16), to_dev(seq[0]))
+    torch.cuda.synchronize()
+    used_sel = [eng.layers[l].sel.cpu().numpy() for l in range(n_layers)]     # what the next attention reads
     prev_q = 0
+    table = np.arange(mb, dtype=np.int32).reshape(1, mb)
     for s in range(S):
         eng.step([q_dev[l][s] for l in range(n_layers)], to_dev(seq[s]), to_dev(seq[s] // 16),
                  to_dev((seq[s] + 1) // 16 - seq[s] // 16), to_dev((seq[s] + 1) // 16), to_dev(seq[s] + 1))
         eng.join()
         torch.cuda.synchronize()
         for l in range(n_layers):
-            for b in (3, 12):
+            for b in range(B):
                 kv = pu.np_u16(lays[l].host_kv[b * mb:(b + 1) * mb])
-                table = np.arange(mb, dtype=np.int32).reshape(1, mb)
                 n_full = (seq[s][b:b + 1] // 16).numpy()
                 sq = seq[s][b:b + 1].numpy()
                 summ = oracle.build_summaries(kv, table, np.zeros(1, np.int32), n_full)
                 qp = pu.np_u16(lays[l].q_steps[prev_q][b:b + 1])            # the drafts that predicted this step
                 s32, s64 = oracle.score_blocks(qp[:, 1:], summ, n_full)
                 sel, idx, slots = oracle.select_topk(s32, n_full, sq, cfg.n_q_tokens, k, table)
+                gsel = used_sel[l][b:b + 1]
+                pu.assert_sel_parity(gsel, sel, s64, k)
+                # the attention ran over the GPU's own (adjudicated) selection
+                gidx = np.where(gsel < 0, -1, gsel.astype(np.int64) * Hkv + np.arange(Hkv)[None, :, None])
                 pool = np.zeros((Hkv * (k + 2), 2, 16, 128), np.uint16)
-                oracle.stage_blocks(kv.reshape(-1, 2, 16, 128), idx, slots, pool)
-                ref = oracle.sparse_attn(pu.np_u16(lays[l].q_steps[s][b:b + 1]), pool, slots, sel, sq, SCALE, Hkv)
+                oracle.stage_blocks(kv.reshape(-1, 2, 16, 128), gidx, slots, pool)
+                ref = oracle.sparse_attn(pu.np_u16(lays[l].q_steps[s][b:b + 1]), pool, slots, gsel, sq, SCALE, Hkv)
                 pu.assert_attn_close(pu.bf16_to_f32_np(eng.layers[l].out[b:b + 1]), ref["out32"])
+        used_sel = [eng.layers[l].sel.cpu().numpy() for l in range(n_layers)]
         prev_q = s

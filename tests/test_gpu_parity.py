@@ -550,3 +550,103 @@ def test_build_summaries_layers_equals_per_layer_calls(gpu):
     for l in range(n_layers):
         assert torch.equal(got[l].view(torch.int16), want[l].view(torch.int16))
     assert not torch.equal(want[0].view(torch.int16), torch.full(shape, 7.0, dtype=torch.bfloat16, device=dev).view(torch.int16))
+
+
+FUSED_DIRECT = [
+    ("rows128", dict(base="c2_reasoning", batch=16, context=2064, k_blocks=24, layers=1, steps=1), dict(ragged=True)),
+    ("rows24_split", dict(base="c1_single", batch=3, context=2064, k_blocks=40), dict(ragged=True, permute_table=True)),
+    ("rows304", dict(base="c5_sweep", batch=38, context=784, k_blocks=9, n_draft=2), dict(ragged=True)),
+    ("gqa8", dict(base="c4_gqa8", batch=10, context=1296, k_blocks=20, layers=1), dict(ragged=True)),
+]
+
+
+@pytest.mark.parametrize("name,spec,kw", FUSED_DIRECT, ids=[s[0] for s in FUSED_DIRECT])
+def test_fused_launch_against_the_oracle(oracle, gpu, name, spec, kw):
+    """oasis_attn_and_score checked directly against the oracle (not through the separate calls): its scores
+    within 1e-5 relative of the double-precision scores, the selection made from ITS scores equal to the oracle's
+    (near-ties adjudicated), its attention within tolerance of the oracle's attention on that selection."""
+    binding, pipeline = gpu
+    dev = torch.device("cuda")
+    cfg = make_cfg(spec)
+    lay = synth.make_layer(cfg, seed=21, **kw)
+    k, T = cfg.k_blocks, cfg.n_q_tokens
+    ref = pu.oracle_layer(oracle, lay, k)
+    L = pipeline.DecodeLayer(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_blocks, k, T, dev, want_lse=True)
+    assert binding.attn_and_score_supported(L.dims, T, L.cols, T - 1)
+    kv = lay.host_kv.to(dev)
+    table, n_full, seq, q = (t.to(dev) for t in (lay.block_table, lay.n_full, lay.seq_len, lay.q))
+    L.build_summaries(kv, table, torch.zeros_like(n_full), n_full, cfg.max_blocks)
+    # the working set the attention phase reads: the oracle's selection and the oracle's staged pool
+    L.pool.copy_(torch.from_numpy(ref["pool"].view(np.int16)).view(torch.bfloat16).to(dev))
+    blk = torch.from_numpy(ref["sel"]).to(dev)
+    L.scores.fill_(float("nan"))
+    L.attend_and_score(q, seq, n_full, blk_tbl=blk)
+    L.select(n_full, seq, table)                       # top-k of the fused launch's own scores
+    torch.cuda.synchronize()
+    pu.assert_scores_close(L.scores.cpu().numpy(), ref["s32"], ref["s64"], ref["n_full"])
+    pu.assert_sel_parity(L.sel.cpu().numpy(), ref["sel"], ref["s64"], k)
+    pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref["attn"]["out32"])
+    np.testing.assert_allclose(L.lse.cpu().numpy(), ref["attn"]["lse"], rtol=1e-3, atol=2e-3)
+
+
+def test_wait_timeout_selftest_reports_and_leaves_the_library_usable(oracle, gpu):
+    """A bounded wait that nothing completes must give up, record its code in the registered error word and
+    return; the next ordinary call must work and leave the (re-zeroed) word at zero."""
+    binding, pipeline = gpu
+    dev = torch.device("cuda")
+    word = torch.zeros(1, dtype=torch.int32, device=dev)
+    result = torch.full((2,), -1, dtype=torch.int32, device=dev)
+    binding.set_error_word(word)
+    try:
+        binding.selftest_wait_timeout(4096, result)
+        torch.cuda.synchronize()
+        assert result.tolist() == [1, 99]
+        assert int(word.item()) == 99
+        # the word is only ever written from zero: a second time-out does not overwrite a code already there
+        word.fill_(7)
+        binding.selftest_wait_timeout(64, result)
+        torch.cuda.synchronize()
+        assert int(word.item()) == 7
+        word.zero_()
+        cfg = synth.scaled(synth.C1, batch=2, context=1040, k_blocks=24)
+        lay = synth.make_layer(cfg, seed=11)
+        compare_path(oracle, pipeline, lay, cfg.k_blocks)
+        assert int(word.item()) == 0
+    finally:
+        binding.set_error_word(None)
+    with pytest.raises(binding.OasisError, match="probes"):
+        binding.selftest_wait_timeout(0, result)
+
+
+def test_unwritten_tail_of_the_local_block_may_hold_any_finite_pattern(oracle, gpu):
+    """Token rows of the local block past the visible positions are masked; whatever finite bit patterns they
+    hold (here the largest finite bf16, in keys and values) must not change the result."""
+    binding, pipeline = gpu
+    dev = torch.device("cuda")
+    cfg = synth.scaled(synth.C1, batch=2, context=1029, k_blocks=12)          # 5 tokens in the local block
+    lay = synth.make_layer(cfg, seed=23)
+    k, T = cfg.k_blocks, cfg.n_q_tokens
+    ref = pu.oracle_layer(oracle, lay, k)
+    L, dv = run_gpu_path(pipeline, lay, k)
+    want = L.out.clone()
+    # overwrite every row past position seq_len + T - 1 of the local entries with 0x7f7f (3.39e38)
+    pool = L.pool.view(torch.int16)
+    sel = L.sel.cpu().numpy()
+    slots = L.slot_tbl.cpu().numpy()
+    touched = 0
+    for b in range(cfg.batch):
+        last = int(lay.seq_len[b]) + T - 1
+        for h in range(cfg.n_kv_heads):
+            for c in (k, k + 1):
+                j = int(sel[b, h, c])
+                if j < 0:
+                    continue
+                first_hidden = max(0, last + 1 - j * 16)
+                if first_hidden < 16:
+                    pool[int(slots[b, h, c]), :, first_hidden:, :] = 0x7f7f
+                    touched += 1
+    assert touched > 0
+    L.attend(dv["q"], dv["seq_len"])
+    torch.cuda.synchronize()
+    assert torch.equal(L.out.view(torch.int16), want.view(torch.int16))
+    pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref["attn"]["out32"])
