@@ -696,3 +696,142 @@ def test_offload_summaries_are_the_min_and_max_of_the_copied_keys(oracle):
     sel = [(b, j) for b in range(B) for j in range(mb) if first[b] <= j < first[b] + n[b]]
     for b, j in sel:
         assert np.array_equal(summ[b, :, j], again[b, :, j])
+
+
+# --------------------------------------------------------------------------- local window, KV append
+
+
+def test_local_window_hand_worked_columns_and_requests(oracle):
+    """bs = 16, T = 3, local columns 4 and 5 (block parity picks the column).
+    L = 30: tokens at 30, 31 (block 1) and 32 (block 2)  -> column 5 = block 1, column 4 = block 2.
+    L = 32: tokens 32..34, all in block 2                -> column 4 = block 2, column 5 = -1.
+    L = 45: tokens 45..47, all in block 2                -> as before (a block keeps its column).
+    L = 46: tokens 46, 47 (block 2) and 48 (block 3)     -> column 4 = block 2, column 5 = block 3."""
+    Hkv, n_cols, mb = 2, 6, 8
+    seq = np.array([30, 32, 45, 46], np.int32)
+    table = (np.arange(4 * mb, dtype=np.int32).reshape(4, mb) * 3 + 1)            # some non-identity table
+    blk = np.full((4, Hkv, n_cols), 77, np.int32)
+    idx, slots = oracle.local_window(seq, 3, table, blk, 4, 10)
+    assert blk[:, :, :4].tolist() == np.full((4, Hkv, 4), 77).tolist()            # other columns untouched
+    assert blk[:, 0, 4:].tolist() == [[2, 1], [2, -1], [2, -1], [2, 3]]
+    assert np.array_equal(blk[:, 0], blk[:, 1])
+    for b, (c4, c5) in enumerate([(2, 1), (2, -1), (2, -1), (2, 3)]):
+        for h in range(Hkv):
+            row = b * Hkv + h
+            assert slots[b, h].tolist() == [row * 10 + 4, row * 10 + 5]
+            want = [(table[b, j] * Hkv + h) if j >= 0 else -1 for j in (c4, c5)]
+            assert idx[b, h].tolist() == want
+
+
+def _token_stream(rng, n_tok, Hkv, d):
+    """A contiguous per-request K/V sequence [n_tok][Hkv][2][d] as (bits, values)."""
+    return rand_bf16(rng, (n_tok, Hkv, 2, d))
+
+
+def test_append_over_many_steps_rebuilds_the_blocks_in_the_cpu_pool(oracle):
+    """Tokens appended one committed token per step (T = 5 written, 1 committed) over 40 steps: every position
+    that was committed must sit in the CPU pool exactly where a plain numpy reshape of the contiguous token
+    sequence into [block][head][K,V][row][dim] puts it, nothing else in the CPU pool may change, and the GPU
+    working set's local slots must hold the tokens written last at each position."""
+    rng = np.random.default_rng(5)
+    B, Hkv, d, bs, T, mb, k = 2, 3, 8, 16, 5, 8, 2
+    n_cols, steps = k + 2, 40
+    L0 = np.array([21, 48], np.int32)
+    table = rng.permutation(B * mb).astype(np.int32).reshape(B, mb)
+    n_tok = mb * bs
+    sbits, _ = _token_stream(rng, B * n_tok, Hkv, d)
+    sbits = sbits.reshape(B, n_tok, Hkv, 2, d)
+    # the layout a reshape gives: [block][row][head][part][d] -> [block][head][part][row][d]
+    want_blocks = sbits.reshape(B, mb, bs, Hkv, 2, d).transpose(0, 1, 3, 4, 2, 5)
+    canary = np.uint16(0xABCD)
+    host = np.full((B * mb, Hkv, 2, bs, d), canary, np.uint16)
+    pool = np.full((B * Hkv * n_cols, 2, bs, d), canary, np.uint16)
+    slot_tbl = rng.permutation(B * Hkv * n_cols).astype(np.int32).reshape(B, Hkv, n_cols)
+    blk = np.full((B, Hkv, n_cols), -1, np.int32)
+    latest = {}                                     # (b, position) -> step that wrote it last
+    for s in range(steps):
+        seq = (L0 + s).astype(np.int32)
+        new = np.stack([sbits[b, seq[b]:seq[b] + T] for b in range(B)])           # [B][T][Hkv][2][d]
+        new = new + np.uint16(s % 3)                # drafts differ from what is committed later (bit noise)
+        new[:, 0] = np.stack([sbits[b, seq[b]] for b in range(B)])                # the committed token is the true one
+        oracle.append_kv(new, 1, seq, table, slot_tbl, blk, k, pool, host)
+        for b in range(B):
+            lo, hi = seq[b] // bs, (seq[b] + T - 1) // bs
+            assert blk[b, 0, k + (lo & 1)] == lo
+            assert blk[b, 0, k + 1 - (lo & 1)] == (hi if hi > lo else -1)
+            for t in range(T):
+                latest[(b, int(seq[b]) + t)] = (s, t, new[b, t].copy())
+    for b in range(B):
+        first, last = int(L0[b]), int(L0[b]) + steps - 1
+        for j in range(mb):
+            got = host[table[b, j]]                                               # [Hkv][2][bs][d]
+            for i in range(bs):
+                p = j * bs + i
+                if first <= p <= last:
+                    assert np.array_equal(got[:, :, i], want_blocks[b, j][:, :, i]), (b, p)
+                else:
+                    assert (got[:, :, i] == canary).all(), (b, p)
+        # local slots: the last two local blocks hold, row by row, what was written last
+        seq = int(L0[b]) + steps - 1
+        for j in range(seq // bs, (seq + T - 1) // bs + 1):
+            for h in range(Hkv):
+                e = pool[slot_tbl[b, h, k + (j & 1)]]
+                for i in range(bs):
+                    p = j * bs + i
+                    if (b, p) in latest and p >= seq - bs:     # still inside the two-block window
+                        assert np.array_equal(e[:, i], latest[(b, p)][2][h]), (b, p, h)
+    # slots of the k selected columns were never touched
+    for b in range(B):
+        for h in range(Hkv):
+            for c in range(k):
+                assert (pool[slot_tbl[b, h, c]] == canary).all()
+
+
+@pytest.mark.parametrize("L0", [33, 45, 47])
+def test_append_then_attention_equals_dense_attention(oracle, L0):
+    """The local window written by the append (not gathered from the CPU pool) together with a full budget of
+    gathered blocks must reproduce brute-force dense causal attention over the contiguous token sequence;
+    L0 = 45 and 47 with T = 4 put tokens into two local blocks, and the steps before cross a block boundary."""
+    rng = np.random.default_rng(17 + L0)
+    B, Hq, Hkv, d, bs, T = 2, 4, 2, 8, 16, 4
+    mb, k = 6, 6
+    n_cols = k + 2
+    n_tok = mb * bs
+    sbits, svals = _token_stream(rng, B * n_tok, Hkv, d)
+    sbits, svals = sbits.reshape(B, n_tok, Hkv, 2, d), svals.reshape(B, n_tok, Hkv, 2, d)
+    table = rng.permutation(B * mb).astype(np.int32).reshape(B, mb)
+    host = np.zeros((B * mb, Hkv, 2, bs, d), np.uint16)
+    pool = np.zeros((B * Hkv * n_cols, 2, bs, d), np.uint16)
+    slot_tbl = identity_tables(B, Hkv, n_cols)
+    blk = np.full((B, Hkv, n_cols), -1, np.int32)
+    start = np.array([L0 - 20, L0 - 20 - 7], np.int32)
+    # history before `start` is already in the CPU pool (as after a hand-over)
+    for b in range(B):
+        for p in range(int(start[b])):
+            host[table[b, p // bs], :, :, p % bs] = sbits[b, p]
+    # the partially filled block at `start` is loaded into its local slot once
+    idx, slots = oracle.local_window(start, T, table, blk, k, n_cols)
+    oracle.stage_blocks(host.reshape(-1, 2, bs, d), idx, slots, pool)
+    scale = float(np.float32(1.0 / math.sqrt(d)))
+    qbits, q = rand_bf16(rng, (B, T, Hq, d))
+    for s in range(21):
+        seq = (start + s).astype(np.int32)
+        new = np.stack([sbits[b, seq[b]:seq[b] + T] for b in range(B)])
+        oracle.append_kv(new, 1, seq, table, slot_tbl, blk, k, pool, host)
+        # full budget: every full block is selected and gathered from the CPU pool
+        n_full = seq // bs
+        for b in range(B):
+            for h in range(Hkv):
+                blk[b, h, :k] = -1
+                blk[b, h, :n_full[b]] = np.arange(n_full[b])
+        gidx = np.where(blk[:, :, :k] < 0, -1,
+                        np.take_along_axis(np.broadcast_to(table[:, None, :], (B, Hkv, mb)), np.maximum(blk[:, :, :k], 0), axis=2)
+                        .astype(np.int64) * Hkv + np.arange(Hkv)[None, :, None])
+        oracle.stage_blocks(host.reshape(-1, 2, bs, d), gidx, slot_tbl[:, :, :k].copy(), pool)
+        res = oracle.sparse_attn(qbits, pool, slot_tbl, blk, seq, scale, Hkv)
+        for b in range(B):
+            K = svals[b, :, :, 0].transpose(1, 0, 2)
+            V = svals[b, :, :, 1].transpose(1, 0, 2)
+            want, want_lse = dense_attention_f64(q[b], K, V, int(seq[b]), scale)
+            np.testing.assert_allclose(res["out64"][b], want, rtol=1e-12, atol=1e-12)
+            np.testing.assert_allclose(res["lse"][b], want_lse, rtol=1e-5, atol=1e-5)
