@@ -286,6 +286,54 @@ int oasis_plan_delta(const oasis_dims_t *dims, const int32_t *sel, int32_t sel_c
                      int32_t *n_admitted, void *stream);
 
 /*
+ * Local window (Sec. 4.3: the selected blocks and a local window stay in GPU memory; Sec. 5.2: the active
+ * local block is kept on top of the K selected blocks).  With L = seq_len[b] and T = n_q_tokens (1..16),
+ * the step's tokens sit at positions L .. L+T-1, in the local blocks lo = L / 16 .. hi = (L+T-1) / 16 (at
+ * most two).  Local block j lives in column local_col + (j & 1) of its (request, KV head) row, so a block
+ * keeps its column, and with it its slot, for as long as it is local.
+ * oasis_local_window sets   blk_tbl[b][h][local_col + (lo & 1)] = lo   and the other local column to hi
+ * (if hi > lo) or -1, and leaves every other column alone.  Optionally (both lists, or both NULL) it emits
+ * two gather requests per row that load the local blocks from the CPU pool with oasis_stage_blocks -- used
+ * once, when a request enters sparse decoding with a partially filled block:
+ *   stage_idx   [B][Hkv][2] int64: block_table[b][j] * Hkv + h for the block j of column local_col + r, or -1
+ *   stage_slots [B][Hkv][2] int32: (b * Hkv + h) * slot_stride + local_col + r
+ */
+int oasis_local_window(const oasis_dims_t *dims, const int32_t *seq_len, int32_t n_q_tokens,
+                       const int32_t *block_table, int32_t *blk_tbl, int32_t n_cols, int32_t local_col,
+                       int32_t slot_stride, int64_t *stage_idx, int32_t *stage_slots, void *stream);
+
+/*
+ * KV append of one decode step.  The paper keeps the newest tokens in the GPU-resident local window (Sec. 4.3,
+ * 5.2) and does not say how they reach the CPU pool; this library writes them through: the step's tokens are
+ * produced on the GPU and go straight into the local window, and the tokens the step commits are also stored
+ * into the CPU full-KV pool, so that a block that fills up is complete there and is summarised, selected and
+ * gathered like any other.  The local blocks therefore never cross the host link towards the GPU.
+ *   1. the local columns of blk_tbl are set as by oasis_local_window;
+ *   2. token t < n_q_tokens of request b, KV head h (key row, then value row, of new_kv) is written to row
+ *      (L + t) % 16 of the K part and of the V part of entry slot_tbl[b][h][local_col + (j & 1)] of hbm_pool,
+ *      j = (L + t) / 16;
+ *   3. the first n_commit tokens are also written to the same rows of entry (block_table[b][j], h) of host_kv.
+ *   new_kv      [B][n_q_tokens][Hkv][2][128] bf16 (device)
+ *   slot_tbl    [B][Hkv][n_cols] int32 (device), blk_tbl the same shape, updated in place
+ *   host_kv     the CPU full-KV pool (mapped pinned memory, or device memory); may be NULL when n_commit = 0
+ * Rows of a local entry that earlier steps wrote are left as they are.  1 <= n_q_tokens <= 16,
+ * 0 <= n_commit <= n_q_tokens, local_col + 2 <= n_cols.
+ * oasis_append_kv_layers does the same for n_layers <= OASIS_MAX_APPEND_LAYERS layers in one launch (host
+ * arrays of per-layer device pointers; seq_len is shared, as a step appends the same positions in every layer).
+ */
+int oasis_append_kv(const oasis_dims_t *dims, const void *new_kv, int32_t n_q_tokens, int32_t n_commit,
+                    const int32_t *seq_len, const int32_t *block_table, const int32_t *slot_tbl,
+                    int32_t *blk_tbl, int32_t n_cols, int32_t local_col, void *hbm_pool, void *host_kv,
+                    void *stream);
+
+#define OASIS_MAX_APPEND_LAYERS 64
+int oasis_append_kv_layers(const oasis_dims_t *dims, int32_t n_layers, const void *const *new_kv,
+                           int32_t n_q_tokens, int32_t n_commit, const int32_t *seq_len,
+                           const int32_t *const *block_tables, const int32_t *const *slot_tbls,
+                           int32_t *const *blk_tbls, int32_t n_cols, int32_t local_col,
+                           void *const *hbm_pools, void *const *host_kvs, void *stream);
+
+/*
  * Head-union block set (Sec. 4.4.1, partial transfer: per layer the per-head selected sets are
  * united at block granularity -- a block is included if at least one KV head selected it -- and
  * the index of every included block is sent with its data).

@@ -635,3 +635,57 @@ void oasis_oracle_append_kv(int32_t B, int32_t T, int32_t Hkv, int32_t d, int32_
         }
     }
 }
+
+/* ---------------------------------------------------------------- attention mass per block
+ * Second reading of "the exact set of the true next-token query" in the agreement figures of Sec. 3 and
+ * Sec. 4.2.1: the blocks that matter are those that receive the attention of the true query.  For
+ * request b and every query row (t, a) of q_true [B][Tq][Hq][d] -- row t sits at position seq_len[b] + t
+ * and sees every position <= its own -- dense causal softmax attention over the WHOLE context read from
+ * the full-KV pool (two passes, double precision) gives a probability per key; the probabilities of
+ * a block's keys are added up, and the rows that share KV head h are reduced with max:
+ *   mass[b][h][j] = max_{t, a in head group h}  sum_{i : j*bs+i visible} softmax_{t,a}(j*bs + i)
+ * for every logical block j that holds a visible key (0 for the others).
+ */
+void oasis_oracle_block_mass(int32_t B, int32_t Tq, int32_t Hq, int32_t Hkv, int32_t d, int32_t bs,
+                             int32_t max_blocks, const uint16_t *q_true, const uint16_t *kv_pool,
+                             const int32_t *block_table, const int32_t *seq_len, float scale,
+                             double *mass)
+{
+    const int32_t G = Hq / Hkv;
+    const int64_t part = (int64_t)bs * d;
+    double *logit = (double *)malloc(sizeof(double) * (size_t)max_blocks * (size_t)bs);
+    for (int64_t o = 0; o < (int64_t)B * Hkv * max_blocks; ++o) mass[o] = 0.0;
+    for (int32_t b = 0; b < B; ++b) {
+        for (int32_t t = 0; t < Tq; ++t) {
+            int64_t n_vis = (int64_t)seq_len[b] + t + 1;
+            if (n_vis > (int64_t)max_blocks * bs) n_vis = (int64_t)max_blocks * bs;
+            for (int32_t a = 0; a < Hq; ++a) {
+                const int32_t h = a / G;
+                const uint16_t *qv = q_true + (((int64_t)b * Tq + t) * Hq + a) * d;
+                double mx = -INFINITY;
+                for (int64_t p = 0; p < n_vis; ++p) {
+                    int64_t phys = block_table[(int64_t)b * max_blocks + p / bs];
+                    const uint16_t *kr = kv_pool + (phys * Hkv + h) * 2 * part + (p % bs) * d;
+                    double s = 0.0;
+                    for (int32_t x = 0; x < d; ++x)
+                        s = s + (double)bf16_to_f32(qv[x]) * (double)bf16_to_f32(kr[x]);
+                    logit[p] = s * (double)scale;
+                    if (logit[p] > mx) mx = logit[p];
+                }
+                double den = 0.0;
+                for (int64_t p = 0; p < n_vis; ++p) {
+                    logit[p] = exp(logit[p] - mx);
+                    den = den + logit[p];
+                }
+                for (int64_t j = 0; j * bs < n_vis; ++j) {
+                    double m = 0.0;
+                    for (int64_t p = j * bs; p < (j + 1) * bs && p < n_vis; ++p) m = m + logit[p];
+                    m = m / den;
+                    double *dst = mass + ((int64_t)b * Hkv + h) * max_blocks + j;
+                    if (m > *dst) *dst = m;
+                }
+            }
+        }
+    }
+    free(logit);
+}

@@ -208,3 +208,18 @@ def append_kv(new_kv, n_commit, seq_len, block_table, slot_tbl, blk_tbl, local_c
     lib().oasis_oracle_append_kv(B, T, Hkv, d, bs, max_blocks, int(n_commit), _p(new_kv), _p(seq_len),
                                  _p(block_table), _p(slot_tbl), _p(blk_tbl), n_cols, int(local_col), _p(pool),
                                  _p(host_kv))
+
+
+def block_mass(q_true, kv_pool, block_table, seq_len, scale):
+    """q_true [B][Tq][Hq][d] u16 (row t at position seq_len[b] + t), kv_pool [P][Hkv][2][bs][d] u16 ->
+    mass [B][Hkv][max_blocks] fp64: the largest share of a sharing query row's dense attention that falls on
+    each block."""
+    q_true, kv_pool = _u16(q_true), _u16(kv_pool)
+    block_table, seq_len = _i32(block_table), _i32(seq_len)
+    B, Tq, Hq, d = q_true.shape
+    _, Hkv, _, bs, _ = kv_pool.shape
+    max_blocks = block_table.shape[-1]
+    mass = np.empty((B, Hkv, max_blocks), dtype=np.float64)
+    lib().oasis_oracle_block_mass(B, Tq, Hq, Hkv, d, bs, max_blocks, _p(q_true), _p(kv_pool), _p(block_table),
+                                  _p(seq_len), ctypes.c_float(scale), _p(mass))
+    return mass

@@ -22,7 +22,8 @@ SYMBOLS = ("oasis_build_summaries", "oasis_score_blocks", "oasis_select_topk",
            "oasis_plan_delta", "oasis_last_error", "oasis_version",
            "oasis_sparse_attn_static_scratch", "oasis_static_scratch_bytes", "oasis_set_error_word", "oasis_union_blocks",
            "oasis_offload_blocks", "oasis_attn_and_score", "oasis_attn_and_score_supported",
-           "oasis_build_summaries_layers", "oasis_selftest_wait_timeout")
+           "oasis_build_summaries_layers", "oasis_selftest_wait_timeout",
+           "oasis_local_window", "oasis_append_kv", "oasis_append_kv_layers")
 
 
 class OasisError(RuntimeError):
@@ -88,6 +89,12 @@ def lib():
         L.oasis_attn_and_score_supported.argtypes = [dp, i32, i32, i32]
         L.oasis_attn_and_score_supported.restype = ctypes.c_int
         L.oasis_union_blocks.restype = ctypes.c_int
+        L.oasis_local_window.argtypes = [dp, vp, i32, vp, vp, i32, i32, i32, vp, vp, vp]
+        L.oasis_local_window.restype = ctypes.c_int
+        L.oasis_append_kv.argtypes = [dp, vp, i32, i32, vp, vp, vp, vp, i32, i32, vp, vp, vp]
+        L.oasis_append_kv.restype = ctypes.c_int
+        L.oasis_append_kv_layers.argtypes = [dp, i32, vp, i32, i32, vp, vp, vp, vp, i32, i32, vp, vp, vp]
+        L.oasis_append_kv_layers.restype = ctypes.c_int
         L.oasis_selftest_wait_timeout.argtypes = [ctypes.c_uint32, vp, vp]
         L.oasis_selftest_wait_timeout.restype = ctypes.c_int
         L.oasis_set_error_word.argtypes = [vp]
@@ -286,14 +293,61 @@ def sparse_attn_static_scratch(dims, q, n_q_tokens, hbm_pool, slot_tbl, blk_tbl,
 
 
 def plan_delta(dims, sel, k, block_table, resident, stamp, slot_stride, cap, step, plan_idx,
-               plan_slots, n_admitted=None, n_local=0, stream=None):
-    """resident / stamp are [B][Hkv][n_res + n_local]; plan lists [B][Hkv][cap + n_local]."""
+               plan_slots, n_admitted=None, n_local=0, n_res=None, stream=None):
+    """resident / stamp are [B][Hkv][res_stride] with the n_res eviction-managed columns first (default:
+    all but the last n_local); plan lists [B][Hkv][cap + n_local]."""
     d = dims.c()
     res_stride = int(resident.shape[-1])
+    n_res = res_stride - int(n_local) if n_res is None else int(n_res)
     _check(lib().oasis_plan_delta(
         ctypes.byref(d), _ptr(sel, torch.int32, "sel"), int(sel.shape[-1]), int(k),
         _ptr(block_table, torch.int32, "block_table"), _ptr(resident, torch.int32, "resident"),
-        _ptr(stamp, torch.int32, "stamp"), res_stride - int(n_local), res_stride, int(n_local),
+        _ptr(stamp, torch.int32, "stamp"), n_res, res_stride, int(n_local),
         int(slot_stride), int(cap), int(step), _ptr(plan_idx, torch.int64, "plan_idx"),
         _ptr(plan_slots, torch.int32, "plan_slots"), _ptr(n_admitted, torch.int32, "n_admitted"),
         _stream(stream)), "oasis_plan_delta")
+
+
+MAX_APPEND_LAYERS = 64
+
+
+def local_window(dims, seq_len, n_q_tokens, block_table, blk_tbl, local_col, slot_stride=0, stage_idx=None,
+                 stage_slots=None, stream=None):
+    """Sets the two local columns of blk_tbl [B][Hkv][n_cols] (block parity picks the column) and, when the
+    lists [B][Hkv][2] are given, emits the gather requests that load the local blocks from the CPU pool."""
+    d = dims.c()
+    _check(lib().oasis_local_window(
+        ctypes.byref(d), _ptr(seq_len, torch.int32, "seq_len"), int(n_q_tokens),
+        _ptr(block_table, torch.int32, "block_table"), _ptr(blk_tbl, torch.int32, "blk_tbl"), int(blk_tbl.shape[-1]),
+        int(local_col), int(slot_stride), _ptr(stage_idx, torch.int64, "stage_idx"),
+        _ptr(stage_slots, torch.int32, "stage_slots"), _stream(stream)), "oasis_local_window")
+
+
+def append_kv(dims, new_kv, n_commit, seq_len, block_table, slot_tbl, blk_tbl, local_col, hbm_pool, host_kv=None,
+              stream=None):
+    """KV append of one step: new_kv [B][T][Hkv][2][128] into the local window of hbm_pool, its first n_commit
+    tokens also into the CPU pool host_kv."""
+    d = dims.c()
+    _check(lib().oasis_append_kv(
+        ctypes.byref(d), _ptr(new_kv, torch.bfloat16, "new_kv"), int(new_kv.shape[1]), int(n_commit),
+        _ptr(seq_len, torch.int32, "seq_len"), _ptr(block_table, torch.int32, "block_table"),
+        _ptr(slot_tbl, torch.int32, "slot_tbl"), _ptr(blk_tbl, torch.int32, "blk_tbl"), int(blk_tbl.shape[-1]),
+        int(local_col), _ptr(hbm_pool, torch.bfloat16, "hbm_pool"), _ptr(host_kv, torch.bfloat16, "host_kv"),
+        _stream(stream)), "oasis_append_kv")
+
+
+def append_kv_layers(dims, new_kv, n_commit, seq_len, block_tables, slot_tbls, blk_tbls, local_col, hbm_pools,
+                     host_kvs, stream=None):
+    """oasis_append_kv for several layers in one launch: lists of per-layer tensors."""
+    n = len(new_kv)
+    if not all(len(x) == n for x in (block_tables, slot_tbls, blk_tbls, hbm_pools, host_kvs)):
+        raise ValueError("one tensor per layer is needed in every list")
+    d = dims.c()
+    arr = ctypes.c_void_p * max(n, 1)
+    mk = lambda ts, dt, nm: arr(*[None if t is None else _ptr(t, dt, nm).value for t in ts])
+    _check(lib().oasis_append_kv_layers(
+        ctypes.byref(d), n, mk(new_kv, torch.bfloat16, "new_kv"), int(new_kv[0].shape[1]) if n else 1, int(n_commit),
+        _ptr(seq_len, torch.int32, "seq_len"), mk(block_tables, torch.int32, "block_tables"),
+        mk(slot_tbls, torch.int32, "slot_tbls"), mk(blk_tbls, torch.int32, "blk_tbls"),
+        int(blk_tbls[0].shape[-1]) if n else 2, int(local_col), mk(hbm_pools, torch.bfloat16, "hbm_pools"),
+        mk(host_kvs, torch.bfloat16, "host_kvs"), _stream(stream)), "oasis_append_kv_layers")

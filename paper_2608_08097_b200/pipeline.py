@@ -85,37 +85,49 @@ class DecodeLayer:
 
 
 class DecodeEngine:
-    """Sequencing of one decode step across layers, after the paper's asynchronous prefetch
-    pipeline (Sec. 4.2.2).  Four streams:
+    """Sequencing of decode steps across layers, after the paper's asynchronous prefetch pipeline
+    (Sec. 4.2.2).  Streams:
       foreground  attention of every layer over the working set that the previous step's
                   prediction staged;
-      prediction  summary update for newly completed blocks and scoring with the draft queries;
-      selection   top-k and (delta mode) the transfer plan -- the tables a layer's attention
-                  reads are only rewritten after that attention has finished;
-      transfer    the gather of what was selected, awaited, per layer, only by the next step's
-                  attention of that same layer.
-    In end-to-end mode a fifth stream uploads the step's queries (all layers, before the first
-    gather) and downloads each layer's output.
-    A whole step can be captured into a CUDA graph (`capture_step`) and replayed, which removes
-    the host launch cost of its ~250 kernels.
+      prediction  the step's KV append and summary update for newly completed blocks, and (unfused)
+                  scoring with the draft queries;
+      selection   top-k -- the tables a layer's attention reads are only rewritten after that
+                  attention has finished;
+      transfer    the transfer plan and the gather of what was selected, awaited, per layer, only by
+                  the next step's attention of that same layer.
+    In end-to-end mode an upload stream brings each layer's queries from pinned host memory and a
+    download stream returns each layer's output.
+    Every dependency is per layer and carries over from one step to the next, so consecutive steps
+    overlap exactly as far as the data allows: a layer's gather may still be running while the next
+    step's first layers attend.  Steps can be captured into CUDA graphs, one or several per graph
+    (`capture_steps`); only the end of a graph is a synchronisation point.
 
     mode "fetch_all": every selected block is gathered each step (k + 2 requests per row).
     mode "delta": delta selection with capped eviction (Sec. 4.2.3) bounds the gather to
-    `cap` blocks per (request, KV head) per step plus the local blocks.
+    `cap` blocks per (request, KV head) per step.
+    append (delta mode): every step is given its new keys and values (`new_kv`), which `oasis_append_kv`
+    writes into the GPU-resident local window (the committed token also through to the full-KV pool),
+    so the local blocks never cross the host link; without it the local blocks are gathered from the
+    full-KV pool like selected ones.
     fused (default: whenever the library takes the shapes): a layer's attention and its scoring run
     as one launch on the foreground stream (`oasis_attn_and_score`); the summary updates of all
     layers are then issued at the start of the step on the prediction stream.
     transfer_streams: consecutive layers' gathers alternate between this many transfer streams (useful
     when the pool is in host memory: one gather's requests are in flight while the previous one's last
     ones come back).
-    defer_tail: the last layer's prediction chain of a step is launched at the start of the next step
-    (`flush()` launches a chain still pending); the state of that layer is then one step behind
-    between steps.
+    wait_group: the foreground stream picks up the other streams' events (a layer's transfer, query
+    upload and output download of the previous step) for `wait_group` layers at a time, in front of the
+    group's first launch.  A fused launch that follows a cross-stream wait is fully serialised behind
+    its predecessor, the others overlap it through programmatic dependent launch; so fewer waits keep
+    more of that overlap, at the price of a coarser dependency.
     """
 
     def __init__(self, batch, n_q_heads, n_kv_heads, max_blocks, k, n_q_tokens, n_layers,
-                 device="cuda", mode="fetch_all", cap=None, fused=None, transfer_streams=1, defer_tail=False):
+                 device="cuda", mode="fetch_all", cap=None, fused=None, transfer_streams=1, wait_group=8,
+                 append=False):
         assert mode in ("fetch_all", "delta")
+        assert not append or mode == "delta", "the KV append goes with delta selection"
+        self.append = bool(append)
         self.mode, self.k, self.T, self.n_layers = mode, k, n_q_tokens, n_layers
         self.device = torch.device(device)
         self.layers = [DecodeLayer(batch, n_q_heads, n_kv_heads, max_blocks, k, n_q_tokens, device)
@@ -128,31 +140,36 @@ class DecodeEngine:
         self.pred = torch.cuda.Stream(device=self.device, priority=-1)
         self.selq = torch.cuda.Stream(device=self.device, priority=-1)
         self.side = torch.cuda.Stream(device=self.device, priority=-1)
-        self.copy = torch.cuda.Stream(device=self.device)     # end-to-end mode: query upload, output download
+        self.up = torch.cuda.Stream(device=self.device)       # end-to-end mode: query upload
+        self.down = torch.cuda.Stream(device=self.device)     # end-to-end mode: output download
         # consecutive layers' gathers may alternate between several transfer streams, so that one gather's
         # requests are already in flight while the previous one's last ones come back over the host link
         self.xfer = [self.side] + [torch.cuda.Stream(device=self.device, priority=-1)
                                    for _ in range(max(1, int(transfer_streams)) - 1)]
         self.launches = 0
         self.cap = cap
-        # defer_tail: the last layer's prediction chain (top-k, plan, gather) of a step is launched at the start of
-        # the next step instead of at its end, where nothing would overlap it (the next step's attention of that
-        # layer comes last and waits for it as usual); `flush()` launches a chain that is still pending.
-        self.defer_tail = bool(defer_tail)
-        self._deferred = None
-        self._capturing = False
+        self.wait_group = max(1, int(wait_group))
         can_fuse = n_layers > 0 and n_q_tokens > 1 and oasis.attn_and_score_supported(self.layers[0].dims, n_q_tokens, self.layers[0].cols, n_q_tokens - 1)
         self.fused = can_fuse if fused is None else (bool(fused) and can_fuse)
-        self.stage_done = [None] * n_layers          # event of the layer's latest transfer
-        self.sel_done = [None] * n_layers            # event of the layer's latest top-k (it reads the scores)
+        self._reset_events()
         if mode == "delta":
             assert cap is not None and 0 <= cap <= k
             dev, rows = self.device, (batch, n_kv_heads)
             self.resident = [torch.full(rows + (k + 2,), -1, dtype=torch.int32, device=dev) for _ in range(n_layers)]
             self.stamp = [torch.zeros(rows + (k + 2,), dtype=torch.int32, device=dev) for _ in range(n_layers)]
-            self.plan_idx = [torch.empty(rows + (cap + 2,), dtype=torch.int64, device=dev) for _ in range(n_layers)]
-            self.plan_slots = [torch.empty(rows + (cap + 2,), dtype=torch.int32, device=dev) for _ in range(n_layers)]
+            n_req = cap + (0 if append else 2)       # requests per row: the admitted pairs (and the local blocks)
+            self.plan_idx = [torch.empty(rows + (n_req,), dtype=torch.int64, device=dev) for _ in range(n_layers)]
+            self.plan_slots = [torch.empty(rows + (n_req,), dtype=torch.int32, device=dev) for _ in range(n_layers)]
         self._splits = oasis.attn_workspace_bytes(self.layers[0].dims, n_q_tokens, k + 2) > 0 if n_layers else False
+
+    def _reset_events(self):
+        """Forgets the previous step's events (everything before has completed)."""
+        n = self.n_layers
+        self.stage_done = [None] * n         # the layer's latest transfer
+        self.sel_done = [None] * n           # the layer's latest top-k (it reads the scores)
+        self.attn_done = [None] * n          # the layer's latest attention (it reads q, the tables and the pool)
+        self.score_done = [None] * n         # unfused: the layer's latest scoring (it reads q)
+        self.out_done = [None] * n           # end to end: the download of the layer's latest output
 
     def attach(self, layer, kv_src, block_table):
         """kv_src: the layer's full-KV pool (pinned host memory, or device memory)."""
@@ -177,8 +194,14 @@ class DecodeEngine:
         ev.record(stream)
         timers[name].append((start, ev))
 
+    @staticmethod
+    def _event(stream):
+        ev = torch.cuda.Event()
+        ev.record(stream)
+        return ev
+
     def _predict(self, l, q, first_block, n_new, max_new, n_full_next, seq_next, stamp, timers,
-                 attn_done=None, plan=None, scored=None):
+                 attn_done=None, plan=None, scored=None, n_local=2, sel_log=None):
         """Prediction chain of one layer; returns the event after which the layer's gather may start.
         `scored`: the scores were already produced (by the fused launch) and this event marks them."""
         L, ps, qs = self.layers[l], self.pred, self.selq
@@ -192,21 +215,21 @@ class DecodeEngine:
                 t0 = self._tick(timers, "score", ps)
                 L.score(q, n_full_next)
                 self._tock(timers, "score", t0, ps)
-                scored = torch.cuda.Event()
-                scored.record(ps)
-        # top-k and the transfer plan run on their own stream, so that waiting for this layer's attention does
+                scored = self._event(ps)
+                self.score_done[l] = scored
+        # top-k and the transfer plan run on their own streams, so that waiting for this layer's attention does
         # not hold back the next layer's scoring
         with torch.cuda.stream(qs):
-            if scored != "completed":                # (a chain deferred into the next captured step: all done)
-                qs.wait_event(scored)
+            qs.wait_event(scored)
             if attn_done is not None:
                 qs.wait_event(attn_done)            # sel / resident are read by this step's attention
             t0 = self._tick(timers, "select", qs)
             L.select(n_full_next, seq_next, self.table[l])
             self._tock(timers, "select", t0, qs)
+            if sel_log is not None:
+                sel_log.copy_(L.sel, non_blocking=True)  # a record of this step's selection (tests, analysis)
             self.launches += 3 if own_score else 1      # (summary update, scoring,) top-k
-            ev = torch.cuda.Event()
-            ev.record(qs)
+            ev = self._event(qs)
             self.sel_done[l] = ev
         if self.mode == "delta":
             # the transfer plan runs on the transfer stream, so the next layer's top-k does not queue behind it
@@ -215,10 +238,10 @@ class DecodeEngine:
                 plan_idx = self.plan_idx[l] if plan is None else plan[0]
                 plan_slots = self.plan_slots[l] if plan is None else plan[1]
                 oasis.plan_delta(L.dims, L.sel, self.k, self.table[l], self.resident[l], self.stamp[l],
-                                 L.cols, plan_idx.shape[-1] - 2, stamp, plan_idx, plan_slots, n_local=2)
+                                 L.cols, plan_idx.shape[-1] - n_local, stamp, plan_idx, plan_slots, n_local=n_local,
+                                 n_res=self.k)
                 self.launches += 1
-                ev = torch.cuda.Event()
-                ev.record(self.side)
+                ev = self._event(self.side)
         return ev
 
     def _transfer(self, l, ready, timers, plan=None):
@@ -234,9 +257,7 @@ class DecodeEngine:
                 L.stage(self.kv[l])
             self._tock(timers, "stage", t0, ss)
             self.launches += 1
-            ev = torch.cuda.Event()
-            ev.record(ss)
-        self.stage_done[l] = ev
+            self.stage_done[l] = self._event(ss)
 
     def handover(self, layer, dense_k, dense_v, gpu_table, seq_len):
         """Dense -> sparse transition of one layer (Sec. 4.3): every block of the dense GPU pool that
@@ -257,159 +278,148 @@ class DecodeEngine:
 
     def prime(self, q_list, n_full_next, seq_next, step_stamp=0, summaries_ready=False):
         """Before the first step: build every summary (unless the hand-over already did) and run one
-        prediction + transfer per layer, as the step before the first one would have done."""
+        prediction + transfer per layer, as the step before the first one would have done.  With the KV
+        append the (partially filled) local block is loaded from the full-KV pool into the local window
+        once, here."""
         B = self.layers[0].B
         zeros = torch.zeros(B, dtype=torch.int32, device=self.device)
         n_build = zeros if summaries_ready else n_full_next
         torch.cuda.current_stream(self.device).synchronize()      # `zeros` is read on the engine's own streams
         plan = None
+        n_local = 0 if self.append else 2
         if self.mode == "delta":        # the initial working set is admitted whole (cap = k)
-            rows = (B, self.layers[0].Hkv, self.k + 2)
+            rows = (B, self.layers[0].Hkv, self.k + n_local)
             plan = (torch.empty(rows, dtype=torch.int64, device=self.device),
                     torch.empty(rows, dtype=torch.int32, device=self.device))
         for l in range(self.n_layers):
-            ready = self._predict(l, q_list[l], zeros, n_build, self.layers[l].mb, n_full_next, seq_next,
-                                  step_stamp, None, plan=plan)
+            L = self.layers[l]
+            ready = self._predict(l, q_list[l], zeros, n_build, L.mb, n_full_next, seq_next,
+                                  step_stamp, None, plan=plan, n_local=n_local)
             self._transfer(l, ready, None, plan=plan)
+            if self.append:
+                with torch.cuda.stream(self.side):
+                    self.side.wait_event(self.stage_done[l])
+                    idx = torch.empty((B, L.Hkv, 2), dtype=torch.int64, device=self.device)
+                    slots = torch.empty((B, L.Hkv, 2), dtype=torch.int32, device=self.device)
+                    oasis.local_window(L.dims, seq_next, self.T, self.table[l], self.resident[l], self.k, L.cols, idx, slots)
+                    oasis.stage_blocks(self.kv[l], idx, slots, idx.numel(), L.pool)
+                    self.launches += 2
             if plan is not None:
                 for st in self.xfer:     # the shared priming plan is reused by the next layer
                     st.synchronize()
         torch.cuda.synchronize(self.device)
-        self.stage_done = [None] * self.n_layers     # everything has completed
-        self.sel_done = [None] * self.n_layers
+        self._reset_events()                         # everything has completed
 
     def step(self, q_list, seq_len, first_block, n_new, n_full_next, seq_next, step_stamp=0,
-             timers=None, q_host=None, out_host=None):
+             timers=None, q_host=None, out_host=None, new_kv=None, sel_log=None):
         """One decode step over all layers.  seq_len: history tokens of this step; the
         prediction works on the next step's view (n_full_next, seq_next).  With q_host /
         out_host (pinned tensors per layer) the step's queries are copied in and its outputs
-        copied out inside the step (end-to-end mode)."""
-        ms, cs = self.main, self.copy
-        self._launch_deferred(timers)
-        q_ready = [None] * self.n_layers
-        if q_host is not None or out_host is not None:
-            # the copy stream starts after everything the previous step left on the other streams
-            for st in (ms, self.pred):
-                ev = torch.cuda.Event()
-                ev.record(st)
-                cs.wait_event(ev)
+        copied out inside the step (end-to-end mode).  new_kv (one [B][T][Hkv][2][128] tensor per
+        layer; engines built with append=True): the step's new keys and values.  sel_log (one tensor like
+        `layers[l].sel` per layer): receives a copy of each layer's selection of this step."""
+        ms, n = self.main, self.n_layers
+        if self.append != (new_kv is not None):
+            raise ValueError("new_kv must be given exactly when the engine was built with append=True")
+        q_ready = [None] * n
         if q_host is not None:
-            # All of the step's queries cross the host link before its first gather: the zero-copy gathers keep
-            # thousands of reads in flight on the link and would starve DMA copies queued beside them, which
-            # would serialise gather(l) -> attention(l + 1).
-            with torch.cuda.stream(cs):
-                for l in range(self.n_layers):
+            # a layer's queries are uploaded as soon as the previous step no longer reads the staging tensor
+            with torch.cuda.stream(self.up):
+                for l in range(n):
+                    for ev in (self.attn_done[l], self.score_done[l]):
+                        if ev is not None:
+                            self.up.wait_event(ev)
                     q_list[l].copy_(q_host[l], non_blocking=True)
-                    q_ready[l] = torch.cuda.Event()
-                    q_ready[l].record(cs)
-            for st in self.xfer:
-                st.wait_event(q_ready[-1])
-        summ_ready = [None] * self.n_layers
-        if self.fused:
-            # the summary updates (one newly completed block per request every 16 steps) only depend on this step's
-            # KV append: all layers' updates go first, on the prediction stream
-            with torch.cuda.stream(self.pred):
-                for l0 in range(0, self.n_layers, oasis.MAX_LAYERS):       # one launch for (up to 128) layers
-                    l1 = min(l0 + oasis.MAX_LAYERS, self.n_layers)
+                    q_ready[l] = self._event(self.up)
+        head_ready = None
+        with torch.cuda.stream(self.pred):
+            if self.append:
+                # the previous step's attention read the local window and the local columns that are rewritten now
+                if self.attn_done[n - 1] is not None:
+                    self.pred.wait_event(self.attn_done[n - 1])
+                for l0 in range(0, n, oasis.MAX_APPEND_LAYERS):
+                    l1 = min(l0 + oasis.MAX_APPEND_LAYERS, n)
+                    oasis.append_kv_layers(self.layers[l0].dims, new_kv[l0:l1], 1, seq_len, self.table[l0:l1],
+                                           [L.slot_tbl for L in self.layers[l0:l1]], self.resident[l0:l1], self.k,
+                                           [L.pool for L in self.layers[l0:l1]], self.kv[l0:l1])
+                    self.launches += 1
+                head_ready = self._event(self.pred)
+            if self.fused:
+                # the summary updates (one newly completed block per request every 16 steps) only depend on this step's
+                # KV append: all layers' updates go first, on the prediction stream.  Only the step's first fused
+                # launch waits for them (the later ones follow it on the foreground stream).
+                for l0 in range(0, n, oasis.MAX_LAYERS):       # one launch for (up to 128) layers
+                    l1 = min(l0 + oasis.MAX_LAYERS, n)
                     oasis.build_summaries_layers(self.layers[l0].dims, self.kv[l0:l1], self.table[l0:l1], first_block,
                                                  n_new, 1, [L.summaries for L in self.layers[l0:l1]])
                     self.launches += 1
-                    # only the group's first fused launch waits for it: the later ones follow that launch on the
-                    # foreground stream (a wait for the same, already awaited launch before every fused launch made
-                    # the captured graph drop the programmatic edges between consecutive fused launches)
-                    summ_ready[l0] = torch.cuda.Event()
-                    summ_ready[l0].record(self.pred)
-        for l in range(self.n_layers):
+                head_ready = self._event(self.pred)
+        for l in range(n):
             L = self.layers[l]
             with torch.cuda.stream(ms):
-                if q_ready[l] is not None:
-                    ms.wait_event(q_ready[l])
-                if self.stage_done[l] is not None:
-                    ms.wait_event(self.stage_done[l])
+                if l % self.wait_group == 0:
+                    # what the other streams did for the layers of this group: queries uploaded, the previous step's
+                    # transfer landed, the previous step's output downloaded
+                    for g in range(l, min(l + self.wait_group, n)):
+                        for ev in (q_ready[g], self.stage_done[g], self.out_done[g]):
+                            if ev is not None:
+                                ms.wait_event(ev)
+                if l == 0 and head_ready is not None:
+                    ms.wait_event(head_ready)
                 if self.fused:
-                    if summ_ready[l] is not None:
-                        ms.wait_event(summ_ready[l])
                     t0 = self._tick(timers, "layer", ms)
                     L.attend_and_score(q_list[l], seq_len, n_full_next, blk_tbl=self.blk_tbl(l))
                     self._tock(timers, "layer", t0, ms)
-                    self.launches += 2 if self._splits else 1      # the fused launch (and the merge of split rows)
                 else:
                     t0 = self._tick(timers, "attn", ms)
                     L.attend(q_list[l], seq_len, blk_tbl=self.blk_tbl(l))
                     self._tock(timers, "attn", t0, ms)
-                    self.launches += 2 if self._splits else 1
-                attn_done = torch.cuda.Event()
-                attn_done.record(ms)
+                self.launches += 2 if self._splits else 1      # the launch (and the merge of split rows)
+                attn_done = self._event(ms)
+                self.attn_done[l] = attn_done
             if out_host is not None:
-                cs.wait_event(attn_done)
-                with torch.cuda.stream(cs):
+                with torch.cuda.stream(self.down):
+                    self.down.wait_event(attn_done)
                     out_host[l].copy_(L.out, non_blocking=True)
+                    self.out_done[l] = self._event(self.down)
             if q_ready[l] is not None and not self.fused:
                 self.pred.wait_event(q_ready[l])
-            if self.defer_tail and self.fused and l == self.n_layers - 1:
-                self._deferred = (l, q_list[l], first_block, n_new, n_full_next, seq_next, step_stamp, attn_done,
-                                  self._capturing)
-                continue
             ready = self._predict(l, q_list[l], first_block, n_new, 1, n_full_next, seq_next, step_stamp, timers,
-                                  attn_done=attn_done, scored=attn_done if self.fused else None)
+                                  attn_done=attn_done, scored=attn_done if self.fused else None,
+                                  n_local=0 if self.append else 2, sel_log=None if sel_log is None else sel_log[l])
             self._transfer(l, ready, timers)
-        if out_host is not None:
-            ev = torch.cuda.Event()                  # the next step's attention overwrites the output buffers
-            ev.record(cs)
-            ms.wait_event(ev)
-
-    def _launch_deferred(self, timers=None):
-        if self._deferred is None:
-            return
-        l, q, first_block, n_new, n_full_next, seq_next, stamp, attn_done, was_captured = self._deferred
-        self._deferred = None
-        if self._capturing:
-            attn_done = None                         # a graph starts after everything before it has completed
-        elif was_captured:
-            attn_done = torch.cuda.Event()           # the step was a graph replayed on the foreground stream
-            attn_done.record(self.main)
-        ready = self._predict(l, q, first_block, n_new, 1, n_full_next, seq_next, stamp, timers,
-                              attn_done=attn_done, scored="completed")
-        self._transfer(l, ready, timers)
-
-    def flush(self):
-        """Launches the prediction chain that `defer_tail` left pending (after the last step, or before reading the
-        last layer's selection state)."""
-        self._launch_deferred()
 
     def join(self):
         """Makes the foreground stream wait for everything the other streams have in flight."""
-        for st in (self.pred, self.selq, self.copy, *self.xfer):
-            ev = torch.cuda.Event()
-            ev.record(st)
-            self.main.wait_event(ev)
-        self.stage_done = [None] * self.n_layers
+        for st in (self.pred, self.selq, self.up, self.down, *self.xfer):
+            self.main.wait_event(self._event(st))
 
-    def capture_step(self, *args, **kwargs):
-        """Captures one step (same arguments as `step`) into a CUDA graph on the foreground
-        stream and returns it; `graph.replay()` must be issued on that stream, and a replay
-        completes only when all streams' work of the step has completed."""
+    def capture_steps(self, steps):
+        """Captures consecutive steps -- a list of (args, kwargs) of `step` -- into one CUDA graph on the
+        foreground stream and returns it.  Inside the graph the steps overlap as far as their per-layer
+        dependencies allow; `graph.replay()` must be issued on that stream, and a replay completes only when
+        all streams' work of its last step has completed."""
         torch.cuda.synchronize(self.device)
-        self.stage_done = [None] * self.n_layers
-        self.sel_done = [None] * self.n_layers
+        self._reset_events()
         before = self.launches
         g = torch.cuda.CUDAGraph()
         fork = torch.cuda.Event()
-        self._capturing = True
         with torch.cuda.graph(g, stream=self.main, capture_error_mode="thread_local"):
             fork.record(self.main)
-            self.pred.wait_event(fork)
-            self.selq.wait_event(fork)
-            for st in self.xfer:
+            for st in (self.pred, self.selq, self.up, self.down, *self.xfer):
                 st.wait_event(fork)
-            self.copy.wait_event(fork)
-            self.step(*args, **kwargs)
+            for args, kwargs in steps:
+                self.step(*args, **kwargs)
             self.join()
-        self._capturing = False
-        self.sel_done = [None] * self.n_layers       # events recorded inside a capture mean nothing outside it
+        self._reset_events()                         # events recorded inside a capture mean nothing outside it
         g.launches = self.launches - before
+        g.n_steps = len(steps)
         self.launches = before
         return g
+
+    def capture_step(self, *args, **kwargs):
+        """One step (same arguments as `step`) as a CUDA graph."""
+        return self.capture_steps([(args, kwargs)])
 
     def replay(self, graph):
         with torch.cuda.stream(self.main):

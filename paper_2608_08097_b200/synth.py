@@ -237,6 +237,33 @@ def make_layer(cfg: Config, seed: int = 0, layer: int = 0, device="cpu", pin: bo
                  extra=extra)
 
 
+def new_kv_steps(lay: Layer, kv: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """The keys and values each step appends, read out of the pre-generated pool: element [s][b][t][h] is the
+    (key row, value row) of position seq_len_steps[s][b] + t.  Shape [S][B][T][Hkv][2][d], on kv's device."""
+    cfg = lay.cfg
+    kv = lay.host_kv if kv is None else kv
+    pos = lay.seq_len_steps.to(torch.int64)[:, :, None] + torch.arange(cfg.n_q_tokens)[None, None, :]   # [S][B][T]
+    blk, row = pos // cfg.block_size, pos % cfg.block_size
+    phys = torch.gather(lay.block_table.to(torch.int64)[None].expand(pos.shape[0], -1, -1), 2, blk)
+    return kv[phys.to(kv.device), :, :, row.to(kv.device)].contiguous()
+
+
+def blank_future(kv: torch.Tensor, lay: Layer) -> torch.Tensor:
+    """Zeroes, in place, every position of the pool at or beyond each request's first-step history length: the
+    state of a cache whose later tokens have not been produced yet."""
+    cfg = lay.cfg
+    bs = cfg.block_size
+    for b in range(cfg.batch):
+        L = int(lay.seq_len_steps[0][b])
+        lo = L // bs
+        table = lay.block_table[b].to(torch.int64)
+        if L % bs:
+            kv[table[lo], :, :, L % bs:] = 0
+            lo += 1
+        kv[table[lo:]] = 0
+    return kv
+
+
 def u16(t: torch.Tensor):
     """bf16 CPU tensor -> numpy uint16 bit patterns (shares memory)."""
     import numpy as np

@@ -650,3 +650,63 @@ def test_unwritten_tail_of_the_local_block_may_hold_any_finite_pattern(oracle, g
     torch.cuda.synchronize()
     assert torch.equal(L.out.view(torch.int16), want.view(torch.int16))
     pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref["attn"]["out32"])
+
+
+@pytest.mark.parametrize("host_on", ["pinned", "device"])
+def test_append_kv_and_local_window_match_oracle(oracle, gpu, host_on):
+    """The KV append (single-layer call and the several-layers launch) and the local-window set-up against the
+    oracle, byte for byte, over steps that fill a block, cross a block boundary with the draft tokens and roll
+    the local window over; canaries around everything that must stay untouched."""
+    binding, _ = gpu
+    dev = torch.device("cuda")
+    rng = np.random.default_rng(9)
+    B, Hkv, T, mb, k, n_layers, steps = 5, 8, 5, 12, 6, 3, 24
+    n_cols = k + 2
+    dims = binding.Dims(B, 4 * Hkv, Hkv, mb)
+    L0 = np.array([33, 16, 47, 60, 79], np.int32)
+    tables = [rng.permutation(B * mb).astype(np.int32).reshape(B, mb) for _ in range(n_layers)]
+    slot_tbls = [rng.permutation(B * Hkv * n_cols).astype(np.int32).reshape(B, Hkv, n_cols) for _ in range(n_layers)]
+    host_ref = [rng.integers(0, 0x7f00, (B * mb, Hkv, 2, 16, 128)).astype(np.uint16) for _ in range(n_layers)]
+    pool_ref = [rng.integers(0, 0x7f00, (B * Hkv * n_cols, 2, 16, 128)).astype(np.uint16) for _ in range(n_layers)]
+    blk_ref = [np.full((B, Hkv, n_cols), -5, np.int32) for _ in range(n_layers)]
+    bf = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
+    host_gpu = [bf(a).pin_memory() if host_on == "pinned" else bf(a).to(dev) for a in host_ref]
+    pool_gpu = [bf(a).to(dev) for a in pool_ref]
+    blk_gpu = [torch.from_numpy(a).to(dev) for a in blk_ref]
+    tab_gpu = [torch.from_numpy(a).to(dev) for a in tables]
+    slot_gpu = [torch.from_numpy(a).to(dev) for a in slot_tbls]
+
+    # local-window set-up with gather requests (layer 0), then the requests replayed on both sides
+    seq0 = torch.from_numpy(L0).to(dev)
+    idx_g = torch.empty((B, Hkv, 2), dtype=torch.int64, device=dev)
+    slots_g = torch.empty((B, Hkv, 2), dtype=torch.int32, device=dev)
+    binding.local_window(dims, seq0, T, tab_gpu[0], blk_gpu[0], k, n_cols, idx_g, slots_g)
+    idx_r, slots_r = oracle.local_window(L0, T, tables[0], blk_ref[0], k, n_cols)
+    torch.cuda.synchronize()
+    assert np.array_equal(idx_g.cpu().numpy(), idx_r) and np.array_equal(slots_g.cpu().numpy(), slots_r)
+    assert np.array_equal(blk_gpu[0].cpu().numpy(), blk_ref[0])
+
+    for s in range(steps):
+        seq = (L0 + s).astype(np.int32)
+        seq_g = torch.from_numpy(seq).to(dev)
+        new = [rng.integers(0, 0x7f00, (B, T, Hkv, 2, 128)).astype(np.uint16) for _ in range(n_layers)]
+        new_g = [bf(a).to(dev) for a in new]
+        n_commit = 1 if s % 5 else 2
+        for l in range(n_layers):
+            oracle.append_kv(new[l], n_commit, seq, tables[l], slot_tbls[l], blk_ref[l], k, pool_ref[l], host_ref[l])
+        if s % 2:
+            binding.append_kv_layers(dims, new_g, n_commit, seq_g, tab_gpu, slot_gpu, blk_gpu, k, pool_gpu, host_gpu)
+        else:
+            for l in range(n_layers):
+                binding.append_kv(dims, new_g[l], n_commit, seq_g, tab_gpu[l], slot_gpu[l], blk_gpu[l], k, pool_gpu[l],
+                                  host_gpu[l])
+        torch.cuda.synchronize()
+        for l in range(n_layers):
+            assert np.array_equal(blk_gpu[l].cpu().numpy(), blk_ref[l]), (s, l)
+            assert np.array_equal(pu.np_u16(pool_gpu[l]), pool_ref[l]), (s, l)
+            assert np.array_equal(pu.np_u16(host_gpu[l]), host_ref[l]), (s, l)
+    # no write-back without a CPU pool
+    binding.append_kv(dims, new_g[0], 0, seq_g, tab_gpu[0], slot_gpu[0], blk_gpu[0], k, pool_gpu[0], None)
+    torch.cuda.synchronize()
+    with pytest.raises(binding.OasisError, match="n_commit"):
+        binding.append_kv(dims, new_g[0], 1, seq_g, tab_gpu[0], slot_gpu[0], blk_gpu[0], k, pool_gpu[0], None)

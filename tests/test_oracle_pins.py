@@ -835,3 +835,48 @@ def test_append_then_attention_equals_dense_attention(oracle, L0):
             want, want_lse = dense_attention_f64(q[b], K, V, int(seq[b]), scale)
             np.testing.assert_allclose(res["out64"][b], want, rtol=1e-12, atol=1e-12)
             np.testing.assert_allclose(res["lse"][b], want_lse, rtol=1e-5, atol=1e-5)
+
+
+# --------------------------------------------------------------------------- attention mass per block
+
+
+def test_block_mass_equals_dense_softmax_summed_per_block(oracle):
+    """Brute force with numpy on contiguous keys: softmax over the visible prefix, reshaped into blocks and
+    summed, then the maximum over the query rows that share the KV head."""
+    rng = np.random.default_rng(29)
+    B, Tq, Hq, Hkv, d, bs, mb = 2, 3, 4, 2, 8, 4, 9
+    bits, vals = make_pool(rng, B * mb, Hkv, bs, d)
+    table = rng.permutation(B * mb).astype(np.int32).reshape(B, mb)
+    seq = np.array([22, 13], np.int32)
+    qbits, q = rand_bf16(rng, (B, Tq, Hq, d), scale=2.0)
+    scale = float(np.float32(0.37))
+    got = oracle.block_mass(qbits, bits, table, seq, scale)
+    G = Hq // Hkv
+    for b in range(B):
+        K, _ = contiguous_kv(vals, table[b], Hkv)                       # [Hkv][mb*bs][d]
+        want = np.zeros((Hkv, mb))
+        for t in range(Tq):
+            n = int(seq[b]) + t + 1
+            for a in range(Hq):
+                h = a // G
+                logits = (K[h, :n].astype(np.float64) @ q[b, t, a].astype(np.float64)) * scale
+                w = np.exp(logits - logits.max())
+                prob = np.zeros(mb * bs)
+                prob[:n] = w / w.sum()
+                want[h] = np.maximum(want[h], prob.reshape(mb, bs).sum(1))
+        np.testing.assert_allclose(got[b], want, rtol=1e-12, atol=1e-15)
+
+
+def test_block_mass_closed_form_for_identical_keys(oracle):
+    """All keys equal: every visible key gets 1/n, so a full block's mass is bs/n for the row that sees the
+    fewest keys (t = 0, the maximum over rows), and the partially visible last block gets its visible share
+    at the row that sees the most."""
+    B, Tq, Hq, Hkv, d, bs, mb = 1, 2, 2, 1, 4, 4, 5
+    key = rand_bf16(np.random.default_rng(1), (d,))[0]
+    bits = np.zeros((mb, Hkv, 2, bs, d), np.uint16)
+    bits[:, :, 0] = key
+    table = np.arange(mb, dtype=np.int32).reshape(1, mb)
+    seq = np.array([13], np.int32)                                       # rows see 14 and 15 keys
+    qbits, _ = rand_bf16(np.random.default_rng(2), (B, Tq, Hq, d))
+    got = oracle.block_mass(qbits, bits, table, seq, 1.0)[0, 0]
+    np.testing.assert_allclose(got, [4 / 14, 4 / 14, 4 / 14, 3 / 15, 0.0], rtol=1e-12)
