@@ -1,24 +1,33 @@
 #!/usr/bin/env python
 """Benchmark of the OasisKV decode hot path on B200: one JSON line per run.
 
-A "step" is one decode step of the reasoning-style workload (batch 16, 32 layers, 32 q / 8 KV
-heads, 32,768-token context in 16-token blocks, budget 2,048 tokens, 4 draft tokens, drifting
-heavy hitters): per layer, sparse attention over the working set staged by the previous step,
-then summary update, block scoring with the draft queries, top-k, and the gather of the
-selected blocks on a side stream.  metric = tokens/s per layer = batch / (step time / layers).
+A "step" is one decode step of a workload: per layer, the KV append of the step's tokens into the
+GPU-resident local window (the committed token written through to the CPU pool), sparse attention over
+the working set staged by the previous step fused with block scoring by the draft queries, summary
+update, top-k, delta selection with capped eviction, and the gather of the admitted blocks from the
+full-KV pool in PINNED HOST MEMORY on side streams.  metric = tokens/s per layer = batch / (step time / layers).
 
-  value : full-KV pool mirrored in HBM (all inputs resident in HBM), fetch-all gather.
-  e2e   : full-KV pool in pinned host memory (the gather crosses the host link), queries copied
-          host->device and outputs device->host inside every step, fetch-all gather.
-Extra keys report the capped-delta gather, the gather's GB/s against the measured pinned
-host->device peak, the per-kernel HBM rooflines, lookahead recall and the CPU-oracle baseline.
+  value            : queries resident in HBM, full KV in pinned host memory (the gather crosses the host link).
+  e2e              : the same, plus every layer's queries copied host->device and outputs device->host inside
+                     every step.
+  value_hbm_mirror : the full KV mirrored in HBM (no host link): the compute-only step, for the exposed
+                     transfer time  value.ms_per_step - value_hbm_mirror.ms_per_step.
+Consecutive steps are captured into CUDA graphs of `--group` steps; inside a graph a layer's transfer only
+has to land before that layer's next-step attention (Sec. 4.2.2), so steps overlap.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config 0..4] [--fetch-ratio R] [--group G]
+                  [--repeats R] [--sweep-ratios 0.01,0.02,...] [--summary FILE] [--impl reference]
+
+--config picks the workload (default 1, the reasoning-style decode the metric is quoted on; 0 and 4 rotate
+over independent copies of their single layer so that every launch reads cold data; 4 prints one line with
+a cell per budget x draft length).  --sweep-ratios repeats value / value_hbm_mirror / e2e for several fetch
+caps (Sec. 5.5.1) and reports the exposed time per layer; --summary writes the numbers as a markdown table.
 """
 import argparse
 import json
 import math
 import os
+import re
 import sys
 import threading
 import time
@@ -31,41 +40,60 @@ import torch  # noqa: E402
 
 from paper_2608_08097_b200 import synth  # noqa: E402
 
-# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (configs[1] shapes)
-TRAFFIC_BYTES = {"score": 139.0e6, "attn": 140.3e6, "layer": 277.3e6}
-
 METRIC = "sparse decode-attn+select tokens/s per layer"
 UNIT = "tokens/s/layer"
+BUDGETS = (32, 64, 128, 256, 512)        # configs[4]: K blocks = 512 .. 8,192 tokens
+DRAFTS = (1, 2, 4, 8)
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=48)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--layers", type=int, default=None, help="override the number of layers (debugging)")
+    ap.add_argument("--config", type=int, default=1, choices=[0, 1, 2, 3, 4])
+    ap.add_argument("--layers", type=int, default=None, help="override the number of layers (debugging, profiling)")
     ap.add_argument("--batch", type=int, default=None, help="override the batch (debugging)")
     ap.add_argument("--context", type=int, default=None, help="override the context length (debugging)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--fetch-ratio", type=float, default=0.05, help="cap of the delta gather, fraction of K")
+    ap.add_argument("--group", type=int, default=0, help="decode steps per CUDA graph (0: all timed steps in one)")
+    ap.add_argument("--wait-group", type=int, default=8, help="layers per pick-up of the side streams' events")
+    ap.add_argument("--transfer-group", type=int, default=0,
+                    help="layers per gather launch when the pool is in host memory (0: 4 when the host link bounds the step, else 1)")
+    ap.add_argument("--repeats", type=int, default=1, help="replay the timed steps this many times in a second, long "
+                                                            "timed region (reported as `sustained`)")
+    ap.add_argument("--sweep-ratios", default="", help="comma-separated fetch ratios to sweep (e.g. 0.01,0.02,0.05)")
+    ap.add_argument("--summary", default="", help="write a markdown summary of the numbers to this file")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
+    ap.add_argument("--skip-mirror", action="store_true")
     return ap.parse_args()
 
 
 def workload(args):
+    """(configuration, description).  configs[0] and configs[4] have one layer: they run as 32 / 4 independent
+    copies of it (different seeds), so that consecutive launches read different data."""
+    base = (synth.C1, synth.C2, synth.C3, synth.C4, synth.C5)[args.config]
     kw = {}
+    if args.config == 0:
+        kw["layers"] = 32
+    if args.config == 4:
+        kw.update(layers=4, n_draft=max(DRAFTS))
     if args.layers:
         kw["layers"] = args.layers
     if args.batch:
         kw["batch"] = args.batch
     if args.context:
         kw["context"] = args.context
-    need_steps = args.steps + max(args.warmup, 3) + 1
-    if need_steps > synth.C2.steps:
-        kw["steps"] = need_steps
-    return synth.scaled(synth.C2, **kw) if kw else synth.C2
+    kw["steps"] = max(base.steps, args.steps + max(args.warmup, 3) + 1)
+    cfg = synth.scaled(base, **kw)
+    names = ("configs[0] single layer, batch 1 (run as %d independent copies)" % cfg.layers,
+             "configs[1] reasoning-style decode", "configs[2] long-context large batch",
+             "configs[3] larger-model GQA-8 shape",
+             "configs[4] budget x draft-length sweep (one layer run as %d independent copies)" % cfg.layers)
+    return cfg, names[args.config]
 
 
 def measured_peaks():
@@ -75,6 +103,21 @@ def measured_peaks():
             d = json.load(f)
         return float(d["hbm_gbs"]), "measured"
     return 6650.0, "fallback"
+
+
+def profile_traffic(name="c2_layer_tcgen05_kernel.md"):
+    """DRAM bytes (read + write) per launch of the fused kernel from the tracked ncu summary of the configs[1]
+    shapes: the mean of the 'traffic (read + write)' row."""
+    try:
+        with open(os.path.join(ROOT, "profiles", name)) as f:
+            for line in f:
+                if line.startswith("| traffic (read + write)"):
+                    vals = [float(x) for x in re.findall(r"([0-9.]+) MB", line)]
+                    if vals:
+                        return sum(vals) / len(vals) * 1e6
+    except OSError:
+        pass
+    return None
 
 
 class ClockSampler:
@@ -161,9 +204,6 @@ def max_over_ranks(x, world, device):
     return float(t.item())
 
 
-# ------------------------------------------------------------------------------------------- ours
-
-
 def time_pinned_h2d(device):
     """Pinned host -> device copy bandwidth, 1 GiB, best of 10 (GB/s)."""
     n = 1 << 30
@@ -181,6 +221,31 @@ def time_pinned_h2d(device):
     return best
 
 
+# ------------------------------------------------------------------------------------------- ours
+
+
+class Work:
+    """One (budget, draft length) view of the generated workload: contiguous per-layer query / new-KV tensors."""
+
+    def __init__(self, bench, k, td):
+        cfg = bench.cfg
+        self.k, self.td, self.T = k, td, td + 1
+        full = td == cfg.n_draft
+        self.q_dev = [q if full else q[:, :, :self.T].contiguous() for q in bench.q_dev]              # [S][B][T][Hq][d]
+        self.q_true_dev = [q if full else q[:, :, :td].contiguous() for q in bench.q_true_dev]        # [S][B][Td][Hq][d]
+        self.new_kv = [t if full else t[:, :, :self.T].contiguous() for t in bench.new_kv]            # [S][B][T][Hkv][2][d]
+        self.q_pinned = None
+
+    def e2e_buffers(self, bench):
+        cfg = bench.cfg
+        if self.q_pinned is None:
+            self.q_pinned = [q.cpu().pin_memory() for q in self.q_dev]
+            self.q_stage = [torch.empty_like(self.q_dev[l][0]) for l in range(cfg.layers)]
+            self.out_pinned = [torch.empty((cfg.batch, self.T, cfg.n_q_heads, 128), dtype=torch.bfloat16, pin_memory=True)
+                               for _ in range(cfg.layers)]
+        return self.q_pinned, self.q_stage, self.out_pinned
+
+
 class Bench:
     def __init__(self, args, cfg, device, rank):
         from paper_2608_08097_b200 import build
@@ -191,8 +256,15 @@ class Bench:
         self.binding, self.pipeline = binding, pipeline
         self.n_layers = cfg.layers
         self.host_kv, self.mirror, self.tables = [], [], []
-        self.q_dev, self.q_true_dev = [], []
+        self.q_dev, self.q_true_dev, self.new_kv = [], [], []
         self.sample_layer = None
+        self.err_word = torch.zeros(1, dtype=torch.int32, device=device)
+        binding.set_error_word(self.err_word)
+
+    def check_error_word(self, where):
+        code = int(self.err_word.item())
+        if code != 0:
+            raise RuntimeError("a kernel's bounded wait ran out (code %d) during %s: the numbers are void" % (code, where))
 
     def generate(self, want_mirror, want_host):
         cfg = self.cfg
@@ -204,6 +276,7 @@ class Bench:
             self.tables.append(lay.block_table.to(self.dev))
             self.q_dev.append(lay.q_steps.to(self.dev))
             self.q_true_dev.append(lay.q_true_steps.to(self.dev))
+            self.new_kv.append(synth.new_kv_steps(lay).to(self.dev))
             if want_mirror:
                 self.mirror.append(host.to(self.dev, non_blocking=False))
             if want_host:
@@ -213,7 +286,6 @@ class Bench:
                 self.sample_layer = lay if want_host else None
             if not want_host:
                 del host
-        S = cfg.steps
         seq = self.seq_steps                                            # [S][B] int32 (host)
         self.seq_dev = seq.to(self.dev)
         self.first_dev = (seq // 16).to(torch.int32).to(self.dev)       # full blocks before the step's commit
@@ -222,40 +294,57 @@ class Bench:
         self.n_new_dev = (self.nfull_next_dev - self.first_dev).contiguous()
         self.gen_seconds = time.time() - t0
 
-    def engine(self, mode, kv_list, cap=None):
+    def transfer_group(self, w, cap):
+        """Layers per gather launch from pinned host memory.  Where the link bounds the step (the gathered bytes of a
+        layer take longer than its scoring + attention), four layers per launch keep the link busier (0.89 against 0.85
+        of the copy-engine rate); where compute bounds it, one launch per layer disturbs the compute least."""
+        if self.args.transfer_group > 0:
+            return self.args.transfer_group
         cfg = self.cfg
-        # gathers from pinned host memory alternate between three transfer streams (about 3 % on the end-to-end step:
-        # a gather's first requests are in flight while the previous gather's last ones come back)
+        link_us = cap * cfg.batch * cfg.n_kv_heads * 8192 / (0.9 * self.h2d_peak * 1e3)
+        score, attn = algorithmic_bytes(cfg, w.k, w.T, self.seq_steps, [0])
+        compute_us = (score + attn) / (0.85 * self.hbm_peak * 1e3)
+        return 4 if link_us > compute_us else 1
+
+    def engine(self, w, kv_list, cap):
+        cfg = self.cfg
+        # gathers from pinned host memory alternate between three transfer streams (a gather's first requests are in
+        # flight while the previous gather's last ones come back)
         host_pool = len(kv_list) > 0 and not kv_list[0].is_cuda
-        eng = self.pipeline.DecodeEngine(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_blocks, cfg.k_blocks,
-                                         cfg.n_q_tokens, self.n_layers, self.dev, mode=mode, cap=cap,
-                                         transfer_streams=3 if host_pool else 1)
+        eng = self.pipeline.DecodeEngine(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_blocks, w.k, w.T,
+                                         self.n_layers, self.dev, mode="delta", cap=cap, append=True,
+                                         transfer_streams=getattr(self.args, "transfer_streams", 1),
+                                         plan_stream=getattr(self.args, "plan_stream", "own"), wait_group=self.args.wait_group,
+                                         n_commit=getattr(self.args, "n_commit", 1),
+                                         transfer_ctas=getattr(self.args, "transfer_ctas", 0) if host_pool else 0,
+                                         transfer_group=self.transfer_group(w, cap) if host_pool else 1)
         for l in range(self.n_layers):
             eng.attach(l, kv_list[l], self.tables[l])
-        eng.prime([self.q_dev[l][0] for l in range(self.n_layers)], self.first_dev[0].contiguous(), self.seq_dev[0].contiguous())
+        eng.prime([w.q_dev[l][0] for l in range(self.n_layers)], self.first_dev[0].contiguous(), self.seq_dev[0].contiguous())
         return eng
 
-    def step_args(self, s, e2e, q_pinned, q_stage, out_pinned):
+    def step_args(self, w, s, e2e):
+        n = self.n_layers
+        kw = dict(step_stamp=s + 1, new_kv=[w.new_kv[l][s] for l in range(n)])
         if e2e:
+            q_pinned, q_stage, out_pinned = w.e2e_buffers(self)
             q_list = q_stage
-            q_host = [q_pinned[l][s] for l in range(self.n_layers)]
+            kw.update(q_host=[q_pinned[l][s] for l in range(n)], out_host=out_pinned)
         else:
-            q_list = [self.q_dev[l][s] for l in range(self.n_layers)]
-            q_host = None
+            q_list = [w.q_dev[l][s] for l in range(n)]
         args = (q_list, self.seq_dev[s], self.first_dev[s], self.n_new_dev[s], self.nfull_next_dev[s],
                 self.seq_next_dev[s])
-        kw = dict(step_stamp=s + 1, q_host=q_host, out_host=out_pinned if e2e else None)
         return args, kw
 
-    def timed(self, eng, world, W, K, e2e=False, q_pinned=None, out_pinned=None, q_stage=None):
-        """Every step is captured into a CUDA graph; W warm-up replays, then exactly K timed
-        replays bracketed by barrier + synchronize.  Returns (ms per step, clocks, launches)."""
-        graphs = []
-        for s in range(W + K):
-            args, kw = self.step_args(s, e2e, q_pinned, q_stage, out_pinned)
-            graphs.append(eng.capture_step(*args, **kw))
-        for s in range(W):
-            eng.replay(graphs[s])
+    def timed(self, eng, w, world, W, K, e2e=False, repeats=1):
+        """The steps are captured into CUDA graphs of `--group` consecutive steps (default: all K timed steps in
+        one); W warm-up steps are replayed, then exactly K timed steps bracketed by barrier + synchronize.
+        Returns (ms per step, clocks, launches, sustained) -- `sustained`: the K steps replayed `repeats` times."""
+        group = self.args.group if self.args.group > 0 else K
+        warm = eng.capture_steps([self.step_args(w, s, e2e) for s in range(W)])
+        graphs = [eng.capture_steps([self.step_args(w, s, e2e) for s in range(s0, min(s0 + group, W + K))])
+                  for s0 in range(W, W + K, group)]
+        eng.replay(warm)
         torch.cuda.synchronize()
         sampler = ClockSampler(self.dev.index or 0)
         sampler.start()
@@ -264,90 +353,113 @@ class Bench:
         start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         l0 = eng.launches
         start.record(eng.main)
-        for s in range(W, W + K):
-            eng.replay(graphs[s])
-        eng.flush()                                  # a prediction chain deferred by the last step (defer_tail)
-        eng.join()
+        for g in graphs:
+            eng.replay(g)
         end.record(eng.main)
         torch.cuda.synchronize()
         barrier(world)
         clocks = sampler.stop()
+        launches = eng.launches - l0
         ms = max_over_ranks(start.elapsed_time(end) / K, world, self.dev)
-        return ms, clocks, eng.launches - l0
+        self.check_error_word("the timed steps")
+        sustained = None
+        if repeats > 1:
+            # a long timed region: the same K steps again and again (the working sets keep evolving; the shapes and
+            # the per-step traffic stay what they are), with the clocks sampled throughout
+            sampler = ClockSampler(self.dev.index or 0)
+            sampler.start()
+            torch.cuda.synchronize()
+            start.record(eng.main)
+            for _ in range(repeats):
+                for g in graphs:
+                    eng.replay(g)
+            end.record(eng.main)
+            torch.cuda.synchronize()
+            c = sampler.stop()
+            ms_r = max_over_ranks(start.elapsed_time(end) / (K * repeats), world, self.dev)
+            sustained = {"ms_per_step": round(ms_r, 4), "seconds": round(ms_r * K * repeats * 1e-3, 2), "repeats": repeats,
+                         "sm_mhz_median": c["sm_mhz"], "reasons": c["reasons"],
+                         "ms_x_mhz": None if c["sm_mhz"] is None else round(ms_r * c["sm_mhz"], 1)}
+            self.check_error_word("the repeated steps")
+        return ms, clocks, launches, sustained
 
-    def kernel_times(self, eng, W, K, e2e=False, q_pinned=None, out_pinned=None, q_stage=None):
-        """Per-kernel durations (us per launch) with CUDA events on the launching streams, over
-        the same steps launched eagerly on the engine's streams."""
-        timers = {"score": [], "select": [], "attn": [], "layer": [], "stage": []}
-        for s in range(W, W + K):
-            args, kw = self.step_args(s, e2e, q_pinned, q_stage, out_pinned)
-            eng.step(*args, timers=timers, **kw)
-        eng.flush()
-        eng.join()
-        torch.cuda.synchronize()
-        return {n: sum(a.elapsed_time(b) for a, b in p) / len(p) * 1e3 for n, p in timers.items() if p}
-
-    def kernel_solo_times(self, eng, s):
-        """Average launch duration (us) of the scoring and of the attention kernel on their own: one launch per
-        layer (all layers' distinct buffers, far more than L2) captured into a CUDA graph on one stream and
-        replayed, timed with CUDA events on that stream."""
-        out = {}
+    def kernel_solo_times(self, eng, w, s):
+        """Launch durations (us) of the scoring, the attention and the fused kernel on their own.
+        graph: one launch per layer (all layers' distinct buffers, far more than L2) captured into a CUDA graph on
+        one stream and replayed, timed with CUDA events on that stream -- consecutive fused launches overlap there
+        through programmatic dependent launch, as they do in the step.
+        single: one launch alone with cold caches: a graph of [write 512 MB, the launch] minus a graph of [write
+        512 MB] (the write flushes L2, keeps the neighbours apart, and its own time and the host's launch latency
+        cancel in the difference); the median over up to four layers."""
+        out, single = {}, {}
         st = eng.main
+        flush = torch.empty(512 << 20, dtype=torch.uint8, device=self.dev)
         calls = {
-            "score": lambda l: eng.layers[l].score(self.q_dev[l][s], self.nfull_next_dev[s]),
-            "attn": lambda l: eng.layers[l].attend(self.q_dev[l][s], self.seq_dev[s], blk_tbl=eng.blk_tbl(l)),
+            "score": lambda l: eng.layers[l].score(w.q_dev[l][s], self.nfull_next_dev[s]),
+            "attn": lambda l: eng.layers[l].attend(w.q_dev[l][s], self.seq_dev[s], blk_tbl=eng.blk_tbl(l)),
         }
         if eng.fused:        # the launch the step actually makes: attention + scoring of a layer in one kernel
-            calls["layer"] = lambda l: eng.layers[l].attend_and_score(self.q_dev[l][s], self.seq_dev[s], self.nfull_next_dev[s],
+            calls["layer"] = lambda l: eng.layers[l].attend_and_score(w.q_dev[l][s], self.seq_dev[s], self.nfull_next_dev[s],
                                                                       blk_tbl=eng.blk_tbl(l))
-        for name, fn in calls.items():
+
+        def graph_of(fn):
             torch.cuda.synchronize()
             with torch.cuda.stream(st):
-                for l in range(self.n_layers):
-                    fn(l)
+                fn()
             torch.cuda.synchronize()
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=st, capture_error_mode="thread_local"):
-                for l in range(self.n_layers):
-                    fn(l)
+                fn()
+            return g
+
+        def best_of(g, reps=5):
             best = None
-            for _ in range(5):
+            for _ in range(reps):
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 with torch.cuda.stream(st):
                     a.record(st)
                     g.replay()
                     b.record(st)
                 torch.cuda.synchronize()
-                t = a.elapsed_time(b) * 1e3 / self.n_layers
+                t = a.elapsed_time(b) * 1e3
                 best = t if best is None else min(best, t)
-            out[name] = best
-        return out
+            return best
 
-    def recall(self, eng, steps):
-        """Share of the draft-predicted top-k also chosen by the true next-step queries."""
-        cfg = self.cfg
+        t_flush = best_of(graph_of(lambda: flush.zero_()))
+        for name, fn in calls.items():
+            out[name] = best_of(graph_of(lambda: [fn(l) for l in range(self.n_layers)])) / self.n_layers
+            ts = []
+            for l in range(0, self.n_layers, max(1, self.n_layers // 4)):
+                ts.append(best_of(graph_of(lambda: (flush.zero_(), fn(l)))) - t_flush)
+            ts.sort()
+            single[name] = ts[len(ts) // 2]
+        del flush
+        return out, single
+
+    def recall(self, eng, w, steps):
+        """Share of the draft-predicted top-k also chosen by the true next-step queries (same estimator)."""
         tot, n = 0.0, 0
         for l in range(0, self.n_layers, max(1, self.n_layers // 4)):
             L = eng.layers[l]
             sel_true = torch.empty_like(L.sel)
             for s in steps:
                 with torch.cuda.stream(eng.main):
-                    L.score(self.q_dev[l][s], self.nfull_next_dev[s])
+                    L.score(w.q_dev[l][s], self.nfull_next_dev[s])
                     L.select(self.nfull_next_dev[s], self.seq_next_dev[s], self.tables[l])
                     sel_draft = L.sel.clone()
-                    L.score_queries(self.q_true_dev[l][s], self.nfull_next_dev[s])
+                    L.score_queries(w.q_true_dev[l][s], self.nfull_next_dev[s])
                     L.select(self.nfull_next_dev[s], self.seq_next_dev[s], self.tables[l], sel=sel_true)
                 eng.main.synchronize()
-                a = sel_draft[..., :cfg.k_blocks]
-                b = sel_true[..., :cfg.k_blocks]
+                a = sel_draft[..., :w.k]
+                b = sel_true[..., :w.k]
                 hit = (a[..., :, None] == b[..., None, :]).any(-1).float().mean().item()
                 tot, n = tot + hit, n + 1
         return tot / max(n, 1)
 
 
-def algorithmic_bytes(cfg, seq_steps, steps):
+def algorithmic_bytes(cfg, k, T, seq_steps, steps):
     """Per-launch algorithmic bytes of the scoring and attention kernels, averaged over steps."""
-    B, Hkv, T, Hq = cfg.batch, cfg.n_kv_heads, cfg.n_q_tokens, cfg.n_q_heads
+    B, Hkv, Hq = cfg.batch, cfg.n_kv_heads, cfg.n_q_heads
     score, attn = 0.0, 0.0
     for s in steps:
         L = seq_steps[s].to(torch.int64)
@@ -355,44 +467,59 @@ def algorithmic_bytes(cfg, seq_steps, steps):
         score += float((nfull_next * Hkv * (512 + 4)).sum())
         nfull = L // 16
         n_local = (L + T + 15) // 16 - nfull
-        cols = torch.minimum(nfull, torch.tensor(cfg.k_blocks)) + n_local
+        cols = torch.minimum(nfull, torch.tensor(k)) + n_local
         attn += float((cols * Hkv * 8192).sum()) + 2.0 * B * T * Hq * 128 * 2
     return score / len(steps), attn / len(steps)
 
 
-def cpu_baseline(cfg, lay, budget_s=20.0):
-    """The oracle, as it stands, on this host: one layer of one step, request by request
-    (score + top-k + gather + attention), until about `budget_s` seconds are spent."""
+def cpu_leg(bench, w, cfg, sel_gpu, s_sel, budget_s=20.0, mass_requests=2):
+    """What runs on the host cores: (1) the oracle, as it stands, on one layer of one step, request by request
+    (score + top-k + gather + attention), until about `budget_s` seconds are spent; (2) the secondary recall: the
+    GPU's lookahead selection of step `s_sel` (layer 0) against the top-K blocks by the attention mass that the true
+    next-step queries put on them, computed by the oracle's dense softmax for the first `mass_requests` requests."""
     import numpy as np
     from oracle import oracle
     oracle.lib()
+    lay = bench.sample_layer
     kv = synth.u16(lay.host_kv)
     table = lay.block_table.numpy()
-    mb = cfg.max_blocks
+    scale = np.float32(1.0 / math.sqrt(128.0))
     done, t_used = 0, 0.0
     for b in range(cfg.batch):
         tb = table[b:b + 1]
         n_full = lay.n_full.numpy()[b:b + 1]
         seq = lay.seq_len.numpy()[b:b + 1]
-        q = synth.u16(lay.q[b:b + 1])
+        q = synth.u16(lay.q[b:b + 1, :w.T].contiguous())
         summ = oracle.build_summaries(kv, tb, np.zeros(1, np.int32), n_full)          # set-up, not timed
         t0 = time.perf_counter()
         s32, _ = oracle.score_blocks(q[:, 1:], summ, n_full)
-        sel, idx, slots = oracle.select_topk(s32, n_full, seq, cfg.n_q_tokens, cfg.k_blocks, tb)
-        pool = np.zeros((cfg.n_kv_heads * (cfg.k_blocks + 2), 2, 16, 128), np.uint16)
+        sel, idx, slots = oracle.select_topk(s32, n_full, seq, w.T, w.k, tb)
+        pool = np.zeros((cfg.n_kv_heads * (w.k + 2), 2, 16, 128), np.uint16)
         oracle.stage_blocks(kv.reshape(-1, 2, 16, 128), idx, slots, pool)
-        oracle.sparse_attn(q, pool, slots.reshape(1, cfg.n_kv_heads, -1), sel, seq,
-                           np.float32(1.0 / math.sqrt(128.0)), cfg.n_kv_heads)
+        oracle.sparse_attn(q, pool, slots.reshape(1, cfg.n_kv_heads, -1), sel, seq, scale, cfg.n_kv_heads)
         t_used += time.perf_counter() - t0
         done += 1
         if t_used >= budget_s:
             break
-    return {"value": done / t_used, "unit": UNIT, "cores": 1, "kind": "oracle",
+    base = {"value": done / t_used, "unit": UNIT, "cores": 1, "host_cores": os.cpu_count(), "kind": "oracle",
             "sample": "layer 0, step 0, %d of %d requests, score+top-k+gather+attention, single thread (%.1f s)"
                       % (done, cfg.batch, t_used)}
+    # secondary recall (attention mass): the true queries of steps s+1.. sit at positions L_s + 1 + t
+    recall_mass = None
+    if sel_gpu is not None:
+        nb = min(mass_requests, cfg.batch)
+        seq_next = (lay.seq_len_steps[s_sel][:nb] + 1).numpy().astype(np.int32)
+        q_true = synth.u16(lay.q_true_steps[s_sel][:nb, :w.td].contiguous())
+        mass = oracle.block_mass(q_true, kv, table[:nb], seq_next, scale)
+        n_full_next = (seq_next // 16).astype(np.int32)
+        sel_mass = oracle.select_topk(mass.astype(np.float32), n_full_next, seq_next, w.T, w.k, table[:nb], want_stage=False)
+        recall_mass = {"value": round(oracle.topk_recall(sel_gpu[:nb], sel_mass, w.k), 4),
+                       "sample": "layer 0, step %d, requests 0..%d: GPU lookahead selection vs top-%d blocks by the true "
+                                 "next-step queries' dense softmax mass (oracle, fp64)" % (s_sel, nb - 1, w.k)}
+    return base, recall_mass
 
 
-def kernel_rooflines(per_kernel, score_bytes, attn_bytes, hbm_peak):
+def kernel_rooflines(per_kernel, single, score_bytes, attn_bytes, hbm_peak):
     kern = {}
     for name, nbytes in (("score", score_bytes), ("attn", attn_bytes), ("layer", score_bytes + attn_bytes)):
         if name in per_kernel:
@@ -400,17 +527,146 @@ def kernel_rooflines(per_kernel, score_bytes, attn_bytes, hbm_peak):
             kern[name] = {"us": round(per_kernel[name], 2), "algorithmic_MB": round(nbytes / 1e6, 2),
                           "GBps": round(gbs, 1), "frac_of_measured": round(gbs / hbm_peak, 3),
                           "frac_of_8TBps": round(gbs / 8000.0, 3)}
-    for name in ("select", "stage"):
-        if name in per_kernel:
-            kern[name] = {"us": round(per_kernel[name], 2)}
+            if name in single:
+                kern[name]["us_single_launch"] = round(single[name], 2)
+                kern[name]["frac_single_launch"] = round(nbytes / (single[name] * 1e-6) / 1e9 / hbm_peak, 3)
     return kern
 
 
-def staged_entries(eng):
-    """Gather requests actually issued by the last step, per layer (delta mode: admitted pairs + local blocks)."""
-    if eng.mode == "delta":
-        return sum(int((p >= 0).sum().item()) for p in eng.plan_idx) / max(1, eng.n_layers)
-    return sum(int((L.stage_idx >= 0).sum().item()) for L in eng.layers) / max(1, eng.n_layers)
+def admitted_entries(eng):
+    """Gather requests actually issued by the last step, per layer."""
+    return sum(int((p >= 0).sum().item()) for p in eng.plan_idx) / max(1, eng.n_layers)
+
+
+def measure(bench, w, world, W, K, cap, hbm_peak, h2d_peak, want_mirror=True, want_host=True, want_e2e=True,
+            want_kernels=True, repeats=1):
+    """All timings of one (workload view, cap): the step with the pool mirrored in HBM, with the pool in pinned host
+    memory, end to end; the kernels alone; recall."""
+    cfg = bench.cfg
+    n = cfg.layers
+    steps = range(W, W + K)
+    score_bytes, attn_bytes = algorithmic_bytes(cfg, w.k, w.T, bench.seq_steps, steps)
+    tok = cfg.batch * world * n          # tokens/s/layer = batch / (step time / layers)
+    qo_bytes = cfg.batch * w.T * cfg.n_q_heads * 128 * 2
+    commit_bytes = cfg.batch * cfg.n_kv_heads * 512
+    r = {"k_blocks": w.k, "n_draft": w.td, "cap": cap, "algorithmic_MB_per_layer": round((score_bytes + attn_bytes) / 1e6, 2)}
+    sel_gpu = None
+    if want_mirror and bench.mirror:
+        eng = bench.engine(w, bench.mirror, cap)
+        ms, clocks, launches, _ = bench.timed(eng, w, world, W, K)
+        r["mirror"] = {"ms_per_step": round(ms, 4), "value": round(tok / (ms * 1e-3), 1), "launches": launches}
+        gbs = (score_bytes + attn_bytes) * n / (ms * 1e-3) / 1e9
+        r["step_hbm"] = {"achieved_GBps": round(gbs, 1), "frac_of_measured": round(gbs / hbm_peak, 3),
+                         "note": "scoring + attention bytes of all layers / step time, full KV mirrored in HBM"}
+        r["recall_lookahead_topk"] = round(bench.recall(eng, w, range(W, min(W + 4, W + K))), 4)
+        if want_kernels:
+            solo, single = bench.kernel_solo_times(eng, w, W)
+            kern = kernel_rooflines(solo, single, score_bytes, attn_bytes, hbm_peak)
+            r["kernels"] = kern
+            r["dominant"] = "layer" if "layer" in solo else max(("score", "attn"), key=lambda x: solo.get(x, 0.0))
+        bench.check_error_word("the HBM-mirror runs")
+        del eng
+        torch.cuda.empty_cache()
+    if want_host and bench.host_kv:
+        eng = bench.engine(w, bench.host_kv, cap)
+        ms, clocks, launches, sustained = bench.timed(eng, w, world, W, K, repeats=repeats)
+        n_req = admitted_entries(eng)
+        gather = n * n_req * 8192
+        r["host"] = {"ms_per_step": round(ms, 4), "value": round(tok / (ms * 1e-3), 1), "launches": launches,
+                     "clocks": clocks, "requests_per_layer": round(n_req, 1),
+                     "h2d_bytes_per_step": int(gather), "d2h_bytes_per_step": int(n * commit_bytes),
+                     "gather_GBps_over_step": round(gather / (ms * 1e-3) / 1e9, 2),
+                     "gather_frac_of_h2d_peak": round(gather / (ms * 1e-3) / 1e9 / h2d_peak, 3)}
+        if sustained:
+            r["host"]["sustained"] = sustained
+        if "mirror" in r:
+            r["host"]["exposed_us_per_layer"] = round((ms - r["mirror"]["ms_per_step"]) * 1e3 / n, 2)
+            r["host"]["compute_to_host_step_ratio"] = round(r["mirror"]["ms_per_step"] / ms, 3)
+        # the GPU's lookahead selection of the last timed step, layer 0 (for the secondary recall on the host)
+        sel_gpu = eng.layers[0].sel.cpu().numpy()
+        r["_sel_step"] = W + K - 1
+        del eng
+        torch.cuda.empty_cache()
+    if want_e2e and bench.host_kv:
+        eng = bench.engine(w, bench.host_kv, cap)
+        ms, clocks, launches, _ = bench.timed(eng, w, world, W, K, e2e=True)
+        n_req = admitted_entries(eng)
+        gather = n * n_req * 8192
+        h2d = gather + n * qo_bytes
+        r["e2e"] = {"value": round(tok / (ms * 1e-3), 1), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                    "d2h_bytes_per_step": int(n * (qo_bytes + commit_bytes)), "ms_per_step": round(ms, 4), "steps": K,
+                    "launches": launches, "requests_per_layer": round(n_req, 1),
+                    "gather_GBps_over_step": round(gather / (ms * 1e-3) / 1e9, 2),
+                    "gather_frac_of_h2d_peak": round(gather / (ms * 1e-3) / 1e9 / h2d_peak, 3),
+                    "h2d_GBps_over_step": round(h2d / (ms * 1e-3) / 1e9, 2),
+                    "h2d_frac_of_h2d_peak": round(h2d / (ms * 1e-3) / 1e9 / h2d_peak, 3),
+                    "gather": "capped delta: at most %d new blocks per (request, KV head) per step, zero-copy from pinned "
+                              "host memory; the local blocks are appended on the GPU and never cross the link; the "
+                              "committed token's K/V is written through to the host pool (counted in d2h)" % cap}
+        if "mirror" in r:
+            r["e2e"]["exposed_us_per_layer"] = round((ms - r["mirror"]["ms_per_step"]) * 1e3 / n, 2)
+        del eng
+        torch.cuda.empty_cache()
+    r["_sel_gpu"] = sel_gpu
+    return r
+
+
+def cap_of(ratio, k):
+    return max(1, int(math.floor(ratio * k)))          # Sec. 5.5.1: at most this fraction of the K selected blocks
+
+
+def write_summary(path, line, rows_sweep, cells, cmd):
+    """A short markdown summary of one run: the numbers the JSON line carries, as tables."""
+    out = ["# %s" % line["config"]["workload"], "", "Command: `%s`" % cmd, "",
+           "One B200; SM clock median %s MHz of %s, throttle reasons %s; pinned H2D peak %.1f GB/s; HBM copy peak %.1f GB/s (%s)."
+           % (line["clocks"]["sm_mhz"], line["clocks"]["sm_max_mhz"], line["clocks"]["reasons"] or "none",
+              line["staged"]["pinned_h2d_peak_GBps"], line["roofline"]["peak"], line["roofline"]["peak_kind"]), ""]
+    if cells:
+        out += ["| K blocks | drafts | cap | step in HBM ms | host-KV step ms | e2e step ms | tokens/s/layer (host KV) | fused kernel us (frac of copy peak) | recall |",
+                "|---|---|---|---|---|---|---|---|---|"]
+        for c in cells:
+            kl = c.get("kernels", {}).get("layer", {})
+            out.append("| %d | %d | %d | %s | %s | %s | %s | %s (%s) | %s |" % (
+                c["k_blocks"], c["n_draft"], c["cap"], c.get("mirror", {}).get("ms_per_step"), c.get("host", {}).get("ms_per_step"),
+                c.get("e2e", {}).get("ms_per_step"), c.get("host", {}).get("value"), kl.get("us"), kl.get("frac_of_measured"),
+                c.get("recall_lookahead_topk")))
+    else:
+        v, m, e = line, line.get("value_hbm_mirror") or {}, line.get("e2e") or {}
+        out += ["| quantity | value |", "|---|---|",
+                "| step, full KV in pinned host memory (`value`) | %.4f ms = %.1f us/layer = %.0f tokens/s/layer |"
+                % (v["ms_per_step"], v["ms_per_step"] * 1e3 / line["config"]["layers"], v["value"]),
+                "| step, full KV mirrored in HBM | %s ms |" % m.get("ms_per_step"),
+                "| end-to-end step (queries H2D, outputs D2H) | %s ms = %s tokens/s/layer |" % (e.get("ms_per_step"), e.get("value")),
+                "| exposed transfer per layer (host-KV step - HBM step) | %s us |" % line["staged"].get("exposed_us_per_layer"),
+                "| gathered bytes over the host-KV step | %s GB/s = %s of the pinned peak |"
+                % (line["staged"].get("gather_GBps_over_step"), line["staged"].get("gather_frac_of_h2d_peak")),
+                "| gathered bytes over the e2e step | %s GB/s = %s of the pinned peak (all H2D bytes: %s) |"
+                % (e.get("gather_GBps_over_step"), e.get("gather_frac_of_h2d_peak"), e.get("h2d_frac_of_h2d_peak")),
+                "| fused kernel, graph of one launch per layer | %s us = %s of the copy peak |"
+                % (line["roofline"].get("us"), line["roofline"].get("frac")),
+                "| fused kernel, one launch alone | %s of the copy peak |" % line["roofline"].get("frac_single_launch"),
+                "| scoring + attention bytes over the HBM step | %s of the copy peak |" % line["roofline"].get("frac_in_step"),
+                "| recall (lookahead vs true-query estimator) / (vs attention mass) | %s / %s |"
+                % (line.get("recall_lookahead_topk"), (line.get("recall_attention_mass") or {}).get("value"))]
+    if rows_sweep:
+        out += ["", "Fetch-ratio sweep (cap = floor(ratio x K) blocks per (request, KV head) per step; exposed = step with the pool in "
+                "pinned host memory minus step with the pool in HBM):", "",
+                "| fetch ratio (cap) | step in HBM us/layer | host-KV us/layer | exposed us/layer | e2e us/layer | e2e exposed us/layer | "
+                "gathered MB/layer | gather GB/s over host-KV step (frac of pinned peak) | e2e tokens/s/layer |",
+                "|---|---|---|---|---|---|---|---|---|"]
+        n = line["config"]["layers"]
+        for r in rows_sweep:
+            out.append("| %s (%d) | %.1f | %.1f | %.1f | %.1f | %.1f | %.2f | %.1f (%.2f) | %.0f |" % (
+                r["fetch_ratio"], r["cap"], r["mirror"]["ms_per_step"] * 1e3 / n, r["host"]["ms_per_step"] * 1e3 / n,
+                r["host"]["exposed_us_per_layer"], r["e2e"]["ms_per_step"] * 1e3 / n, r["e2e"]["exposed_us_per_layer"],
+                r["host"]["h2d_bytes_per_step"] / n / 1e6, r["host"]["gather_GBps_over_step"],
+                r["host"]["gather_frac_of_h2d_peak"], r["e2e"]["value"]))
+    with open(path, "w") as f:
+        f.write("\n".join(out) + "\n")
+
+
+def strip_private(r):
+    return {k: v for k, v in r.items() if not k.startswith("_")}
 
 
 def run_ours(args):
@@ -419,127 +675,96 @@ def run_ours(args):
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    cfg = workload(args)
+    cfg, name = workload(args)
     W, K = max(args.warmup, 3), args.steps
     hbm_peak, peak_kind = measured_peaks()
     bench = Bench(args, cfg, dev, rank)
     h2d_peak = time_pinned_h2d(dev)
-    bench.generate(want_mirror=True, want_host=not args.skip_e2e)
-    cap = max(1, int(math.floor(args.fetch_ratio * cfg.k_blocks)))
-    steps = range(W, W + K)
-    score_bytes, attn_bytes = algorithmic_bytes(cfg, bench.seq_steps, steps)
-    tok = cfg.batch * world * cfg.layers          # tokens/s/layer = batch / (step time / layers)
-    extra = {}
+    bench.h2d_peak, bench.hbm_peak = h2d_peak, hbm_peak
+    bench.generate(want_mirror=not args.skip_mirror, want_host=True)
+    cells, rows_sweep = [], []
+    if args.config == 4:
+        # budget x draft-length cells; the headline cell is budget 2,048 tokens, 4 draft tokens
+        for k in BUDGETS:
+            for td in DRAFTS:
+                w = Work(bench, k, td)
+                c = measure(bench, w, world, W, K, cap_of(args.fetch_ratio, k), hbm_peak, h2d_peak,
+                            want_mirror=not args.skip_mirror, want_e2e=not args.skip_e2e)
+                cells.append(c)
+                del w
+        main = next(c for c in cells if c["k_blocks"] == 128 and c["n_draft"] == 4)
+        w = Work(bench, 128, 4)
+    else:
+        w = Work(bench, cfg.k_blocks, cfg.n_draft)
+        main = measure(bench, w, world, W, K, cap_of(args.fetch_ratio, w.k), hbm_peak, h2d_peak,
+                       want_mirror=not args.skip_mirror, want_e2e=not args.skip_e2e, repeats=args.repeats)
+        for tok in [t for t in args.sweep_ratios.split(",") if t]:
+            ratio = float(tok)
+            r = main if abs(ratio - args.fetch_ratio) < 1e-9 else \
+                measure(bench, w, world, W, K, cap_of(ratio, w.k), hbm_peak, h2d_peak, want_kernels=False)
+            r = dict(r)
+            r["fetch_ratio"] = tok
+            rows_sweep.append(r)
 
-    # ---- value: everything resident in HBM, capped-delta gather (the paper's default operating point) ----
-    eng = bench.engine("delta", bench.mirror, cap=cap)
-    ms, clocks, launches = bench.timed(eng, world, W, K)
-    value = tok / (ms * 1e-3)
-    recall = bench.recall(eng, range(W, min(W + 4, W + K)))
-    del eng
-    eng = bench.engine("delta", bench.mirror, cap=cap)        # instrumented eager pass, fresh state
-    for s in range(W):
-        a, kw = bench.step_args(s, False, None, None, None)
-        eng.step(*a, **kw)
-    per_kernel = bench.kernel_times(eng, W, min(K, 16))
-    solo = bench.kernel_solo_times(eng, W)
-    kern = kernel_rooflines(solo, score_bytes, attn_bytes, hbm_peak)
-    for name, us in per_kernel.items():          # the same launches inside the four-stream step (they share HBM there)
-        kern.setdefault(name, {})["us_in_step"] = round(us, 2)
-    dominant = "layer" if "layer" in solo else max(("score", "attn"), key=lambda n: solo.get(n, 0.0))
-    fused = "layer" in solo
-    del eng
-    # the whole step against the HBM roofline: scoring + attention bytes of all layers over the step time
-    step_gbs = (score_bytes + attn_bytes) * cfg.layers / (ms * 1e-3) / 1e9
-    extra["step_hbm"] = {"algorithmic_MB_per_layer": round((score_bytes + attn_bytes) / 1e6, 2),
-                         "achieved_GBps": round(step_gbs, 1), "frac_of_measured": round(step_gbs / hbm_peak, 3),
-                         "note": "scoring + attention bytes of all layers / step time"}
-    eng = bench.engine("fetch_all", bench.mirror)
-    ms_f, _, _ = bench.timed(eng, world, W, K)
-    extra["value_fetch_all"] = {"ms_per_step": round(ms_f, 4), "value": round(tok / (ms_f * 1e-3), 1),
-                                "gather": "all K+1 blocks per (request, KV head) every step, HBM mirror -> pool"}
-    del eng
-    bench.mirror.clear()
-    torch.cuda.empty_cache()
-
-    # ---- e2e: KV in pinned host memory, queries in / outputs out every step --------------------------------
-    e2e = None
-    if not args.skip_e2e:
-        q_pinned = [q.cpu().pin_memory() for q in bench.q_dev]
-        q_stage = [torch.empty_like(bench.q_dev[l][0]) for l in range(cfg.layers)]
-        out_pinned = [torch.empty((cfg.batch, cfg.n_q_tokens, cfg.n_q_heads, 128), dtype=torch.bfloat16,
-                                  pin_memory=True) for _ in range(cfg.layers)]
-        kw = dict(q_pinned=q_pinned, out_pinned=out_pinned, q_stage=q_stage)
-        qo_bytes = cfg.batch * cfg.n_q_tokens * cfg.n_q_heads * 128 * 2
-        eng = bench.engine("delta", bench.host_kv, cap=cap)
-        ms_e, _, _ = bench.timed(eng, world, W, K, e2e=True, **kw)
-        n_req = staged_entries(eng)
-        pk = bench.kernel_times(eng, W, min(K, 8), e2e=True, **kw)
-        e2e = {"value": round(tok / (ms_e * 1e-3), 1), "unit": UNIT,
-               "h2d_bytes_per_step": int(cfg.layers * (n_req * 8192 + qo_bytes)),
-               "d2h_bytes_per_step": int(cfg.layers * qo_bytes), "ms_per_step": round(ms_e, 4), "steps": K,
-               "gather": "capped delta: at most %d new blocks per (request, KV head) per step + local blocks, "
-                         "zero-copy from pinned host memory" % cap}
-        # consecutive gathers overlap (alternating transfer streams), so the link rate is taken over the whole step
-        gbs = cfg.layers * n_req * 8192 / (ms_e * 1e-3) / 1e9
-        h2d = e2e["h2d_bytes_per_step"] / (ms_e * 1e-3) / 1e9
-        extra["staged_delta"] = {"requests_per_layer": round(n_req, 1), "gather_GBps_over_step": round(gbs, 2),
-                                 "h2d_GBps_over_step": round(h2d, 2), "pinned_h2d_peak_GBps": round(h2d_peak, 2),
-                                 "frac_of_h2d_peak": round(h2d / h2d_peak, 3),
-                                 "launch_us_in_step": round(pk["stage"], 1) if "stage" in pk else None,
-                                 "note": "gathered bytes (and all host-to-device bytes: gathers + queries) / end-to-end step "
-                                         "time; the gather kernel alone is measured by bench_sweep.py --what stage"}
-        del eng
-        Ke = min(K, 8)
-        eng = bench.engine("fetch_all", bench.host_kv)
-        ms_ef, _, _ = bench.timed(eng, world, W, Ke, e2e=True, **kw)
-        n_req_f = staged_entries(eng)
-        pk_f = bench.kernel_times(eng, W, min(Ke, 4), e2e=True, **kw)
-        extra["e2e_fetch_all"] = {"ms_per_step": round(ms_ef, 3), "value": round(tok / (ms_ef * 1e-3), 1), "steps": Ke,
-                                  "h2d_bytes_per_step": int(cfg.layers * (n_req_f * 8192 + qo_bytes))}
-        h2d = extra["e2e_fetch_all"]["h2d_bytes_per_step"] / (ms_ef * 1e-3) / 1e9
-        extra["staged_fetch_all"] = {"h2d_GBps_over_step": round(h2d, 2), "pinned_h2d_peak_GBps": round(h2d_peak, 2),
-                                     "frac_of_h2d_peak": round(h2d / h2d_peak, 3),
-                                     "launch_us_in_step": round(pk_f["stage"], 1) if "stage" in pk_f else None}
-        del eng
-
-    cpu = None
+    cpu, recall_mass = None, None
     if rank == 0 and world == 1 and not args.skip_cpu and bench.sample_layer is not None:
-        cpu = cpu_baseline(cfg, bench.sample_layer)
+        cpu, recall_mass = cpu_leg(bench, w, cfg, main.get("_sel_gpu"), main.get("_sel_step", 0))
 
     if rank == 0:
-        d = kern.get(dominant, {})
+        host, mirror = main.get("host", {}), main.get("mirror", {})
+        kern = main.get("kernels", {})
+        dom = main.get("dominant", "layer")
+        d = kern.get(dom, {})
+        cap = main["cap"]
         line = {
-            "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-            "ms_per_step": round(ms, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "metric": METRIC, "value": host.get("value"), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": host.get("ms_per_step"), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "configs[1] reasoning-style decode: batch %d, %d layers, %dq/%dkv heads, d128, "
-                                   "context %d (+1 per step), 16-token blocks, budget %d tokens, %d draft tokens"
-                                   % (cfg.batch, cfg.layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.context,
-                                      cfg.k_blocks * 16, cfg.n_draft),
-                       "global_batch": cfg.batch * world, "parallelism": "replicas x%d" % world,
+            "config": {"workload": "%s: batch %d, %d layers, %dq/%dkv heads, d128, context %d (+1 per step), 16-token blocks, "
+                                   "budget %d tokens, %d draft tokens" % (name, cfg.batch, cfg.layers, cfg.n_q_heads, cfg.n_kv_heads,
+                                                                          cfg.context, main["k_blocks"] * 16, main["n_draft"]),
+                       "layers": cfg.layers, "global_batch": cfg.batch * world, "parallelism": "replicas x%d" % world,
                        "l2": "inputs larger than L2: each step streams %d layers x %.0f MB of distinct summaries + staged KV"
-                             % (cfg.layers, (score_bytes + attn_bytes) / 1e6),
-                       "gather": "delta selection with capped eviction, fetch ratio %.2f (cap %d blocks per head per "
-                                 "step); full KV in an HBM mirror (value) / pinned host memory (e2e)" % (args.fetch_ratio, cap),
-                       "launch": "each decode step is one CUDA graph over four streams (six end to end: three alternating transfer streams); a layer's attention and scoring are "
-                                 "one fused launch (oasis_attn_and_score)" if fused else
-                                 "each decode step is one CUDA graph over four streams (attention / scoring / selection / transfer)"},
-            "gpu_launches": launches,
-            "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
-                       "samples": clocks["samples"]},
-            "roofline": {"bound": "hbm", "kernel": dominant, "achieved": d.get("GBps"), "peak": hbm_peak,
-                         "unit": "GB/s", "frac": d.get("frac_of_measured"), "traffic": TRAFFIC_BYTES.get(dominant),
+                             % (cfg.layers, main["algorithmic_MB_per_layer"]),
+                       "kv": "full KV in pinned host memory (value, e2e); value_hbm_mirror: the same pool copied to HBM",
+                       "gather": "delta selection with capped eviction, fetch ratio %.2f (cap %d blocks per head per step); local "
+                                 "blocks appended on the GPU" % (args.fetch_ratio, cap),
+                       "launch": "CUDA graphs of %d consecutive decode steps over 6-10 streams; a layer's attention and scoring are "
+                                 "one fused launch (oasis_attn_and_score); gathers of %d layers per launch; side-stream events "
+                                 "picked up every %d layers" % (args.group if args.group > 0 else K, bench.transfer_group(w, cap),
+                                                                 args.wait_group)},
+            "gpu_launches": host.get("launches"),
+            "clocks": {kk: (host.get("clocks") or {}).get(kk) for kk in ("sm_mhz", "sm_max_mhz", "reasons", "samples")},
+            "roofline": {"bound": "hbm", "kernel": dom, "achieved": d.get("GBps"), "peak": hbm_peak, "unit": "GB/s",
+                         "frac": d.get("frac_of_measured"), "us": d.get("us"),
+                         "frac_single_launch": d.get("frac_single_launch"),
+                         "frac_in_step": (main.get("step_hbm") or {}).get("frac_of_measured"),
+                         "traffic": profile_traffic() if args.config == 1 and not (args.batch or args.context) else None,
                          "peak_kind": peak_kind + " (STREAM-style copy)",
-                         "timing": "CUDA events around a graph of one launch per layer (32 distinct working sets), "
-                                   "kernel alone on its stream; us_in_step = same launch inside the four-stream step; "
-                                   "'layer' = the fused attention + scoring launch the step makes, 'score' and 'attn' = "
-                                   "the two separate kernels, for comparison"},
+                         "timing": "frac: CUDA events around a graph of one launch per layer (distinct working sets, consecutive "
+                                   "launches overlap through programmatic dependent launch as in the step); frac_single_launch: "
+                                   "events around one launch alone, median over the layers; frac_in_step: scoring + attention bytes "
+                                   "of all layers over the whole step with the KV mirrored in HBM; traffic: dram bytes per launch "
+                                   "from the tracked ncu summary of these shapes"},
             "kernels": kern,
-            "recall_lookahead_topk": round(recall, 4),
-            "e2e": e2e, "cpu_baseline": cpu, "setup_seconds": round(bench.gen_seconds, 1),
+            "recall_lookahead_topk": main.get("recall_lookahead_topk"), "recall_attention_mass": recall_mass,
+            "e2e": main.get("e2e"), "cpu_baseline": cpu, "setup_seconds": round(bench.gen_seconds, 1),
+            "value_hbm_mirror": mirror or None, "step_hbm": main.get("step_hbm"),
+            "staged": {"pinned_h2d_peak_GBps": round(h2d_peak, 2), "requests_per_layer": host.get("requests_per_layer"),
+                       "gather_GBps_over_step": host.get("gather_GBps_over_step"),
+                       "gather_frac_of_h2d_peak": host.get("gather_frac_of_h2d_peak"),
+                       "exposed_us_per_layer": host.get("exposed_us_per_layer"),
+                       "compute_to_host_step_ratio": host.get("compute_to_host_step_ratio"),
+                       "h2d_bytes_per_step": host.get("h2d_bytes_per_step"), "d2h_bytes_per_step": host.get("d2h_bytes_per_step")},
         }
-        line.update(extra)
+        if host.get("sustained"):
+            line["sustained"] = host["sustained"]
+        if cells:
+            line["cells"] = [strip_private(c) for c in cells]
+        if rows_sweep:
+            line["sweep"] = [{kk: r[kk] for kk in ("fetch_ratio", "cap", "mirror", "host", "e2e") if kk in r} for r in rows_sweep]
+        if args.summary:
+            write_summary(args.summary, line, rows_sweep, cells, "python bench.py " + " ".join(sys.argv[1:]))
         print(json.dumps(line))
 
 
@@ -556,8 +781,10 @@ def run_reference(args):
     import numpy as np
     from oracle import oracle
     oracle.lib()
-    cfg = workload(args)
-    one = synth.scaled(cfg, batch=1, layers=1, steps=1)
+    cfg, name = workload(args)
+    k = 128 if args.config == 4 else cfg.k_blocks
+    td = 4 if args.config == 4 else cfg.n_draft
+    one = synth.scaled(cfg, batch=1, layers=1, steps=1, n_draft=td)
     lay = synth.make_layer(one, seed=args.seed, layer=0, device="cpu")
     kv = synth.u16(lay.host_kv)
     table, n_full, seq = lay.block_table.numpy(), lay.n_full.numpy(), lay.seq_len.numpy()
@@ -566,8 +793,8 @@ def run_reference(args):
 
     def one_step():
         s32, _ = oracle.score_blocks(q[:, 1:], summ, n_full)
-        sel, idx, slots = oracle.select_topk(s32, n_full, seq, one.n_q_tokens, one.k_blocks, table)
-        pool = np.zeros((one.n_kv_heads * (one.k_blocks + 2), 2, 16, 128), np.uint16)
+        sel, idx, slots = oracle.select_topk(s32, n_full, seq, one.n_q_tokens, k, table)
+        pool = np.zeros((one.n_kv_heads * (k + 2), 2, 16, 128), np.uint16)
         oracle.stage_blocks(kv.reshape(-1, 2, 16, 128), idx, slots, pool)
         oracle.sparse_attn(q, pool, slots.reshape(1, one.n_kv_heads, -1), sel, seq,
                            np.float32(1.0 / math.sqrt(128.0)), one.n_kv_heads)
@@ -584,8 +811,9 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world,
             "steps": K, "warmup": W, "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": "configs[1] reasoning-style decode (bounded sample): %s" % sample},
-            "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "config": {"workload": "%s (bounded sample): %s" % (name, sample)},
+            "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": 1, "host_cores": os.cpu_count(), "kind": "oracle",
+                             "sample": sample},
             "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))

@@ -1,13 +1,9 @@
 """Secondary measurements of the sparse-decode path on one B200 (not part of the `bench.py` contract).
 
-    python bench_sweep.py [--layers 8] [--steps 16] [--what ratio,c5,stage,shapes]
+    python bench_sweep.py [--what c5,stage,shapes]
 
+Kernels alone (the whole step, every configuration and the fetch-ratio sweep are `bench.py --config / --sweep-ratios`).
 Prints one JSON line per section:
-  ratio   configs[1] (reasoning-style decode) at several fetch ratios of the capped delta gather
-          (Sec. 5.5.1) plus the uncapped delta and fetch-all: step time with everything in HBM,
-          end-to-end step time with the KV pool in pinned host memory, the exposed transfer time,
-          admitted entries per (request, KV head) per step, and the break-even fetch fraction
-          rho* = link bandwidth x compute time / cold bytes.
   c5      the budget x draft-length sweep (configs[4]): solo kernel times and roofline fractions of
           scoring / top-k / attention and of the fused attention + scoring launch, and lookahead recall per cell.
   stage   the gather kernel alone on random entries of a pinned pool, against the DMA copy peak, and the
@@ -53,62 +49,6 @@ def graph_time(fn, n_rot, iters=32, warm=4):
         ts.append(a.elapsed_time(b) * 1e3 / iters)
     ts.sort()
     return ts[2]
-
-
-def section_ratio(args, dev, hbm_peak):
-    """Fetch-ratio sweep on the reasoning-style workload (fewer layers than the bench, same per-layer sizes)."""
-    W, K = 3, args.steps
-    cfg = synth.scaled(synth.C2, layers=args.layers, steps=W + K + 2)
-    ns = argparse.Namespace(seed=args.seed, skip_e2e=False, skip_cpu=True, fetch_ratio=0.05, layers=args.layers,
-                            batch=None, context=None, gpus=1, steps=K, warmup=W)
-    bench = B.Bench(ns, cfg, dev, 0)
-    h2d_peak = B.time_pinned_h2d(dev)
-    bench.generate(want_mirror=True, want_host=True)
-    q_pinned = [q.cpu().pin_memory() for q in bench.q_dev]
-    q_stage = [torch.empty_like(bench.q_dev[l][0]) for l in range(cfg.layers)]
-    out_pinned = [torch.empty((cfg.batch, cfg.n_q_tokens, cfg.n_q_heads, 128), dtype=torch.bfloat16, pin_memory=True)
-                  for _ in range(cfg.layers)]
-    kw = dict(q_pinned=q_pinned, out_pinned=out_pinned, q_stage=q_stage)
-    rows = cfg.batch * cfg.n_kv_heads
-    cold_bytes = rows * (cfg.k_blocks + 1) * 8192                       # per layer: every selected block + the local one
-    out = []
-    for ratio in (0.01, 0.02, 0.05, 0.10, 0.20, 1.0, None):              # 1.0: uncapped delta; None: fetch all
-        if ratio is None:
-            mode, cap, name = "fetch_all", None, "all"
-        else:
-            mode, cap, name = "delta", max(1, int(math.floor(ratio * cfg.k_blocks))), "%.2f" % ratio
-        eng = bench.engine(mode, bench.mirror, cap=cap)
-        ms_v, _, _ = bench.timed(eng, 1, W, K)
-        del eng
-        eng = bench.engine(mode, bench.host_kv, cap=cap)
-        ms_e, _, _ = bench.timed(eng, 1, W, K, e2e=True, **kw)
-        if mode == "delta":
-            adm = sum(int((p[..., :cap] >= 0).sum().item()) for p in eng.plan_idx) / (cfg.layers * rows)
-            loc = sum(int((p[..., cap:] >= 0).sum().item()) for p in eng.plan_idx) / (cfg.layers * rows)
-        else:
-            adm = sum(int((L.stage_idx[..., :cfg.k_blocks] >= 0).sum().item()) for L in eng.layers) / (cfg.layers * rows)
-            loc = sum(int((L.stage_idx[..., cfg.k_blocks:] >= 0).sum().item()) for L in eng.layers) / (cfg.layers * rows)
-        del eng
-        bytes_layer = rows * (adm + loc) * 8192
-        out.append({
-            "fetch_ratio": name, "cap_blocks": cap,
-            "value_us_per_layer": round(ms_v * 1e3 / cfg.layers, 1),
-            "e2e_us_per_layer": round(ms_e * 1e3 / cfg.layers, 1),
-            "exposed_us_per_layer": round((ms_e - ms_v) * 1e3 / cfg.layers, 1),
-            "tokens_per_s_per_layer_value": round(cfg.batch * cfg.layers / (ms_v * 1e-3), 1),
-            "tokens_per_s_per_layer_e2e": round(cfg.batch * cfg.layers / (ms_e * 1e-3), 1),
-            "admitted_per_row_last_step": round(adm, 2), "local_per_row": round(loc, 2),
-            "fetched_fraction_of_budget": round(adm / cfg.k_blocks, 4),
-            "staged_MB_per_layer": round(bytes_layer / 1e6, 2),
-            "staged_GBps_over_e2e_step": round(bytes_layer / (ms_e * 1e-3 / cfg.layers) / 1e9, 2),
-        })
-    t_compute = out[2]["value_us_per_layer"] * 1e-6                      # the default operating point
-    link = 0.91 * h2d_peak * 1e9                                         # what the zero-copy gather reaches alone
-    print(json.dumps({"section": "ratio", "workload": "configs[1], %d layers, %d timed steps" % (cfg.layers, K),
-                      "pinned_h2d_peak_GBps": round(h2d_peak, 2), "cold_MB_per_layer": round(cold_bytes / 1e6, 1),
-                      "break_even_fetch_fraction": round(link * t_compute / cold_bytes, 4),
-                      "break_even_note": "rho* = 0.91 x pinned peak x value-mode time per layer / cold bytes per layer",
-                      "rows": out}))
 
 
 def section_c5(args, dev, hbm_peak):
@@ -265,10 +205,8 @@ def section_shapes(args, dev, hbm_peak):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--layers", type=int, default=8)
-    ap.add_argument("--steps", type=int, default=16)
     ap.add_argument("--seed", type=int, default=0)
-    ap.add_argument("--what", default="ratio,c5,stage")
+    ap.add_argument("--what", default="c5,stage,shapes")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("bench_sweep.py needs a CUDA device: the product path has no CPU fallback")
@@ -278,7 +216,7 @@ def main():
     build.build()
     hbm_peak, _ = B.measured_peaks()
     for what in args.what.split(","):
-        {"ratio": section_ratio, "c5": section_c5, "stage": section_stage, "shapes": section_shapes}[what](args, dev, hbm_peak)
+        {"c5": section_c5, "stage": section_stage, "shapes": section_shapes}[what](args, dev, hbm_peak)
         torch.cuda.empty_cache()
 
 

@@ -162,6 +162,19 @@ int oasis_stage_blocks(const void *host_kv, const int64_t *idx, const int32_t *s
                        int32_t n, void *hbm_pool, void *stream);
 
 /*
+ * Step 3 for several layers in one launch: the same as one oasis_stage_blocks call per layer with that layer's
+ * pool, lists (each of length n) and working-set pool (host arrays of n_layers <= OASIS_MAX_STAGE_LAYERS device
+ * pointers).  A few large gathers keep the host link busier than many small ones.
+ *   max_ctas   thread blocks of the launch (each keeps 64 KiB of reads in flight); 0 = the library's default of
+ *              64, which is what the host link of a B200 takes before its rate drops.  A small value makes a
+ *              low-intensity copy that can run beside another gather (e.g. the upload of a step's queries).
+ */
+#define OASIS_MAX_STAGE_LAYERS 64
+int oasis_stage_blocks_layers(int32_t n_layers, const void *const *host_kvs, const int64_t *const *idx,
+                              const int32_t *const *slots, int32_t n, void *const *hbm_pools, int32_t max_ctas,
+                              void *stream);
+
+/*
  * Step 4 -- sparse paged decode attention over the staged working set (Sec. 4.2.1: the
  * stacked normal and draft queries run over one resident KV working set in one call;
  * Sec. 4.3: the selected key and value blocks share one ordering).

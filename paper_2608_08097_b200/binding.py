@@ -23,7 +23,7 @@ SYMBOLS = ("oasis_build_summaries", "oasis_score_blocks", "oasis_select_topk",
            "oasis_sparse_attn_static_scratch", "oasis_static_scratch_bytes", "oasis_set_error_word", "oasis_union_blocks",
            "oasis_offload_blocks", "oasis_attn_and_score", "oasis_attn_and_score_supported",
            "oasis_build_summaries_layers", "oasis_selftest_wait_timeout",
-           "oasis_local_window", "oasis_append_kv", "oasis_append_kv_layers")
+           "oasis_local_window", "oasis_append_kv", "oasis_append_kv_layers", "oasis_stage_blocks_layers")
 
 
 class OasisError(RuntimeError):
@@ -89,6 +89,8 @@ def lib():
         L.oasis_attn_and_score_supported.argtypes = [dp, i32, i32, i32]
         L.oasis_attn_and_score_supported.restype = ctypes.c_int
         L.oasis_union_blocks.restype = ctypes.c_int
+        L.oasis_stage_blocks_layers.argtypes = [i32, vp, vp, vp, i32, vp, i32, vp]
+        L.oasis_stage_blocks_layers.restype = ctypes.c_int
         L.oasis_local_window.argtypes = [dp, vp, i32, vp, vp, i32, i32, i32, vp, vp, vp]
         L.oasis_local_window.restype = ctypes.c_int
         L.oasis_append_kv.argtypes = [dp, vp, i32, i32, vp, vp, vp, vp, i32, i32, vp, vp, vp]
@@ -351,3 +353,18 @@ def append_kv_layers(dims, new_kv, n_commit, seq_len, block_tables, slot_tbls, b
         mk(slot_tbls, torch.int32, "slot_tbls"), mk(blk_tbls, torch.int32, "blk_tbls"),
         int(blk_tbls[0].shape[-1]) if n else 2, int(local_col), mk(hbm_pools, torch.bfloat16, "hbm_pools"),
         mk(host_kvs, torch.bfloat16, "host_kvs"), _stream(stream)), "oasis_append_kv_layers")
+
+
+MAX_STAGE_LAYERS = 64
+
+
+def stage_blocks_layers(host_kvs, idx, slots, n, hbm_pools, max_ctas=0, stream=None):
+    """oasis_stage_blocks for several layers in one launch: lists of per-layer tensors, every list of length n."""
+    nl = len(host_kvs)
+    if not all(len(x) == nl for x in (idx, slots, hbm_pools)):
+        raise ValueError("one tensor per layer is needed in every list")
+    arr = ctypes.c_void_p * max(nl, 1)
+    mk = lambda ts, dt, nm: arr(*[_ptr(t, dt, nm).value for t in ts])
+    _check(lib().oasis_stage_blocks_layers(
+        nl, mk(host_kvs, torch.bfloat16, "host_kvs"), mk(idx, torch.int64, "idx"), mk(slots, torch.int32, "slots"), int(n),
+        mk(hbm_pools, torch.bfloat16, "hbm_pools"), int(max_ctas), _stream(stream)), "oasis_stage_blocks_layers")

@@ -115,6 +115,9 @@ class DecodeEngine:
     transfer_streams: consecutive layers' gathers alternate between this many transfer streams (useful
     when the pool is in host memory: one gather's requests are in flight while the previous one's last
     ones come back).
+    transfer_group: the gathers of this many consecutive layers are one launch (`oasis_stage_blocks_layers`): a
+    few large gathers keep the host link busier than many small ones; a layer's next-step attention then waits
+    for its group's launch.
     wait_group: the foreground stream picks up the other streams' events (a layer's transfer, query
     upload and output download of the previous step) for `wait_group` layers at a time, in front of the
     group's first launch.  A fused launch that follows a cross-stream wait is fully serialised behind
@@ -124,10 +127,12 @@ class DecodeEngine:
 
     def __init__(self, batch, n_q_heads, n_kv_heads, max_blocks, k, n_q_tokens, n_layers,
                  device="cuda", mode="fetch_all", cap=None, fused=None, transfer_streams=1, wait_group=8,
-                 append=False):
+                 append=False, transfer_group=1, plan_stream="own", n_commit=1, transfer_ctas=0):
         assert mode in ("fetch_all", "delta")
         assert not append or mode == "delta", "the KV append goes with delta selection"
         self.append = bool(append)
+        self.transfer_ctas = int(transfer_ctas)  # thread blocks per gather launch (0: the library's default)
+        self.n_commit = int(n_commit)            # tokens per step that the KV append also writes to the full-KV pool
         self.mode, self.k, self.T, self.n_layers = mode, k, n_q_tokens, n_layers
         self.device = torch.device(device)
         self.layers = [DecodeLayer(batch, n_q_heads, n_kv_heads, max_blocks, k, n_q_tokens, device)
@@ -140,6 +145,8 @@ class DecodeEngine:
         self.pred = torch.cuda.Stream(device=self.device, priority=-1)
         self.selq = torch.cuda.Stream(device=self.device, priority=-1)
         self.side = torch.cuda.Stream(device=self.device, priority=-1)
+        # transfer plans: a stream of their own (never queued behind a gather), or the first transfer stream
+        self.planq = torch.cuda.Stream(device=self.device, priority=-1) if plan_stream == "own" else self.side
         self.up = torch.cuda.Stream(device=self.device)       # end-to-end mode: query upload
         self.down = torch.cuda.Stream(device=self.device)     # end-to-end mode: output download
         # consecutive layers' gathers may alternate between several transfer streams, so that one gather's
@@ -149,6 +156,7 @@ class DecodeEngine:
         self.launches = 0
         self.cap = cap
         self.wait_group = max(1, int(wait_group))
+        self.transfer_group = max(1, min(int(transfer_group), oasis.MAX_STAGE_LAYERS))
         can_fuse = n_layers > 0 and n_q_tokens > 1 and oasis.attn_and_score_supported(self.layers[0].dims, n_q_tokens, self.layers[0].cols, n_q_tokens - 1)
         self.fused = can_fuse if fused is None else (bool(fused) and can_fuse)
         self._reset_events()
@@ -232,32 +240,42 @@ class DecodeEngine:
             ev = self._event(qs)
             self.sel_done[l] = ev
         if self.mode == "delta":
-            # the transfer plan runs on the transfer stream, so the next layer's top-k does not queue behind it
-            with torch.cuda.stream(self.side):
-                self.side.wait_event(ev)
+            # the transfer plan runs on a stream of its own, so neither the next layer's top-k nor this plan queues
+            # behind a gather
+            with torch.cuda.stream(self.planq):
+                self.planq.wait_event(ev)
                 plan_idx = self.plan_idx[l] if plan is None else plan[0]
                 plan_slots = self.plan_slots[l] if plan is None else plan[1]
                 oasis.plan_delta(L.dims, L.sel, self.k, self.table[l], self.resident[l], self.stamp[l],
                                  L.cols, plan_idx.shape[-1] - n_local, stamp, plan_idx, plan_slots, n_local=n_local,
                                  n_res=self.k)
                 self.launches += 1
-                ev = self._event(self.side)
+                ev = self._event(self.planq)
         return ev
 
-    def _transfer(self, l, ready, timers, plan=None):
-        L, ss = self.layers[l], self.xfer[l % len(self.xfer)]
+    def _transfer(self, ls, readies, timers, plan=None):
+        """The gather of the consecutive layers `ls` (one launch), after their plans / selections `readies`."""
+        ss = self.xfer[(ls[0] // self.transfer_group) % len(self.xfer)]
         with torch.cuda.stream(ss):
-            ss.wait_event(ready)
+            for ev in readies:
+                ss.wait_event(ev)
             t0 = self._tick(timers, "stage", ss)
             if self.mode == "delta":
-                plan_idx = self.plan_idx[l] if plan is None else plan[0]
-                plan_slots = self.plan_slots[l] if plan is None else plan[1]
-                oasis.stage_blocks(self.kv[l], plan_idx, plan_slots, plan_idx.numel(), L.pool)
+                idx = [self.plan_idx[l] if plan is None else plan[0] for l in ls]
+                slots = [self.plan_slots[l] if plan is None else plan[1] for l in ls]
             else:
-                L.stage(self.kv[l])
+                idx = [self.layers[l].stage_idx for l in ls]
+                slots = [self.layers[l].stage_slots for l in ls]
+            if len(ls) == 1 and self.transfer_ctas == 0:
+                oasis.stage_blocks(self.kv[ls[0]], idx[0], slots[0], idx[0].numel(), self.layers[ls[0]].pool)
+            else:
+                oasis.stage_blocks_layers([self.kv[l] for l in ls], idx, slots, idx[0].numel(),
+                                          [self.layers[l].pool for l in ls], max_ctas=self.transfer_ctas)
             self._tock(timers, "stage", t0, ss)
             self.launches += 1
-            self.stage_done[l] = self._event(ss)
+            ev = self._event(ss)
+            for l in ls:
+                self.stage_done[l] = ev
 
     def handover(self, layer, dense_k, dense_v, gpu_table, seq_len):
         """Dense -> sparse transition of one layer (Sec. 4.3): every block of the dense GPU pool that
@@ -295,7 +313,7 @@ class DecodeEngine:
             L = self.layers[l]
             ready = self._predict(l, q_list[l], zeros, n_build, L.mb, n_full_next, seq_next,
                                   step_stamp, None, plan=plan, n_local=n_local)
-            self._transfer(l, ready, None, plan=plan)
+            self._transfer([l], [ready], None, plan=plan)
             if self.append:
                 with torch.cuda.stream(self.side):
                     self.side.wait_event(self.stage_done[l])
@@ -331,41 +349,44 @@ class DecodeEngine:
                             self.up.wait_event(ev)
                     q_list[l].copy_(q_host[l], non_blocking=True)
                     q_ready[l] = self._event(self.up)
-        head_ready = None
-        with torch.cuda.stream(self.pred):
-            if self.append:
-                # the previous step's attention read the local window and the local columns that are rewritten now
-                if self.attn_done[n - 1] is not None:
-                    self.pred.wait_event(self.attn_done[n - 1])
-                for l0 in range(0, n, oasis.MAX_APPEND_LAYERS):
-                    l1 = min(l0 + oasis.MAX_APPEND_LAYERS, n)
-                    oasis.append_kv_layers(self.layers[l0].dims, new_kv[l0:l1], 1, seq_len, self.table[l0:l1],
-                                           [L.slot_tbl for L in self.layers[l0:l1]], self.resident[l0:l1], self.k,
-                                           [L.pool for L in self.layers[l0:l1]], self.kv[l0:l1])
-                    self.launches += 1
-                head_ready = self._event(self.pred)
-            if self.fused:
-                # the summary updates (one newly completed block per request every 16 steps) only depend on this step's
-                # KV append: all layers' updates go first, on the prediction stream.  Only the step's first fused
-                # launch waits for them (the later ones follow it on the foreground stream).
-                for l0 in range(0, n, oasis.MAX_LAYERS):       # one launch for (up to 128) layers
-                    l1 = min(l0 + oasis.MAX_LAYERS, n)
-                    oasis.build_summaries_layers(self.layers[l0].dims, self.kv[l0:l1], self.table[l0:l1], first_block,
-                                                 n_new, 1, [L.summaries for L in self.layers[l0:l1]])
-                    self.launches += 1
-                head_ready = self._event(self.pred)
+        # Per group of `wait_group` layers, on the prediction stream: the KV append (the previous step's attention of
+        # the group's layers read the local window and the local columns that are rewritten now) and, for the fused
+        # launch, the summary updates (one newly completed block per request every 16 steps), which only depend on the
+        # append.  Only the group's first launch on the foreground stream waits for them.
+        head_ready = {}
+        if self.append or self.fused:
+            with torch.cuda.stream(self.pred):
+                for l0 in range(0, n, self.wait_group):
+                    l1 = min(l0 + self.wait_group, n)
+                    if self.append:
+                        if self.attn_done[l1 - 1] is not None:
+                            self.pred.wait_event(self.attn_done[l1 - 1])
+                        for a0 in range(l0, l1, oasis.MAX_APPEND_LAYERS):
+                            a1 = min(a0 + oasis.MAX_APPEND_LAYERS, l1)
+                            oasis.append_kv_layers(self.layers[a0].dims, new_kv[a0:a1], self.n_commit, seq_len, self.table[a0:a1],
+                                                   [L.slot_tbl for L in self.layers[a0:a1]], self.resident[a0:a1], self.k,
+                                                   [L.pool for L in self.layers[a0:a1]], self.kv[a0:a1])
+                            self.launches += 1
+                    if self.fused:
+                        for a0 in range(l0, l1, oasis.MAX_LAYERS):
+                            a1 = min(a0 + oasis.MAX_LAYERS, l1)
+                            oasis.build_summaries_layers(self.layers[a0].dims, self.kv[a0:a1], self.table[a0:a1], first_block,
+                                                         n_new, 1, [L.summaries for L in self.layers[a0:a1]])
+                            self.launches += 1
+                    head_ready[l0] = self._event(self.pred)
+        pending, readies = [], []
         for l in range(n):
             L = self.layers[l]
             with torch.cuda.stream(ms):
                 if l % self.wait_group == 0:
                     # what the other streams did for the layers of this group: queries uploaded, the previous step's
-                    # transfer landed, the previous step's output downloaded
+                    # transfer landed, the previous step's output downloaded, this step's tokens appended
                     for g in range(l, min(l + self.wait_group, n)):
                         for ev in (q_ready[g], self.stage_done[g], self.out_done[g]):
                             if ev is not None:
                                 ms.wait_event(ev)
-                if l == 0 and head_ready is not None:
-                    ms.wait_event(head_ready)
+                    if l in head_ready:
+                        ms.wait_event(head_ready[l])
                 if self.fused:
                     t0 = self._tick(timers, "layer", ms)
                     L.attend_and_score(q_list[l], seq_len, n_full_next, blk_tbl=self.blk_tbl(l))
@@ -387,11 +408,15 @@ class DecodeEngine:
             ready = self._predict(l, q_list[l], first_block, n_new, 1, n_full_next, seq_next, step_stamp, timers,
                                   attn_done=attn_done, scored=attn_done if self.fused else None,
                                   n_local=0 if self.append else 2, sel_log=None if sel_log is None else sel_log[l])
-            self._transfer(l, ready, timers)
+            pending.append(l)
+            readies.append(ready)
+            if len(pending) == self.transfer_group or l == n - 1:
+                self._transfer(pending, readies, timers)
+                pending, readies = [], []
 
     def join(self):
         """Makes the foreground stream wait for everything the other streams have in flight."""
-        for st in (self.pred, self.selq, self.up, self.down, *self.xfer):
+        for st in (self.pred, self.selq, self.planq, self.up, self.down, *self.xfer):
             self.main.wait_event(self._event(st))
 
     def capture_steps(self, steps):
@@ -406,7 +431,7 @@ class DecodeEngine:
         fork = torch.cuda.Event()
         with torch.cuda.graph(g, stream=self.main, capture_error_mode="thread_local"):
             fork.record(self.main)
-            for st in (self.pred, self.selq, self.up, self.down, *self.xfer):
+            for st in (self.pred, self.selq, self.planq, self.up, self.down, *self.xfer):
                 st.wait_event(fork)
             for args, kwargs in steps:
                 self.step(*args, **kwargs)

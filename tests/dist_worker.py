@@ -19,7 +19,7 @@ def main():
     ms = bench.max_over_ranks(10.0 + 5.0 * rank, world, torch.device("cpu"))
     bench.barrier(world)
     if rank == 0:
-        cfg = bench.workload(args)
+        cfg, _ = bench.workload(args)
         print(json.dumps({"world": world, "ms": ms, "value": cfg.batch * world / (ms * 1e-3 / cfg.layers)}))
     if world > 1:
         import torch.distributed as dist

@@ -59,7 +59,8 @@ def test_engine_steps_match_oracle(oracle, gpu, mode, cap, append, chunk, graph,
     k, B, Hkv, T = cfg.k_blocks, cfg.batch, cfg.n_kv_heads, cfg.n_q_tokens
     lays = [synth.make_layer(cfg, seed=31, layer=l) for l in range(n_layers)]
     eng = pipeline.DecodeEngine(B, cfg.n_q_heads, Hkv, cfg.max_blocks, k, T, n_layers, dev,
-                                mode=mode, cap=cap, append=append, fused=fused, transfer_streams=2, wait_group=2)
+                                mode=mode, cap=cap, append=append, fused=fused, transfer_streams=2, wait_group=2,
+                                transfer_group=2 if (append or chunk == 3) else 1)
     new_kv = [synth.new_kv_steps(lay) for lay in lays] if append else None     # [S][B][T][Hkv][2][128] per layer
     # with the KV append the pools start without the tokens that the steps will produce
     kvs = [(synth.blank_future(lay.host_kv.clone(), lay) if append else lay.host_kv).pin_memory() for lay in lays]
