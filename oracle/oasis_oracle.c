@@ -241,12 +241,33 @@ void oasis_oracle_stage_blocks(const uint8_t *host_kv, const int64_t *idx,
  * out32 [B][T][Hq][d] fp32, out64 the same in double, out_bf16 = RNE(out32),
  * lse [B][T][Hq] = max + log(sum) (natural log).  Any output pointer may be NULL.
  * A row that sees no key gets zeros and lse = -inf.
+ * out_abs [B][T][Hq][d] (optional, double) = sum_p softmax_p * |v_p|: the scale of the terms behind each
+ * output element.  It is not part of the method; the parity tests use it to bound what rounding the
+ * softmax weights to 8 significant bits (a tensor-core operand format) can do to an output element.
  */
+void oasis_oracle_sparse_attn_abs(int32_t B, int32_t T, int32_t Hq, int32_t Hkv, int32_t d,
+                                  int32_t bs, const uint16_t *q, const uint16_t *pool,
+                                  const int32_t *slot_tbl, const int32_t *blk_tbl,
+                                  int32_t n_cols, const int32_t *seq_len, float scale,
+                                  float *out32, double *out64, uint16_t *out_bf16, float *lse,
+                                  double *out_abs);
+
 void oasis_oracle_sparse_attn(int32_t B, int32_t T, int32_t Hq, int32_t Hkv, int32_t d,
                               int32_t bs, const uint16_t *q, const uint16_t *pool,
                               const int32_t *slot_tbl, const int32_t *blk_tbl,
                               int32_t n_cols, const int32_t *seq_len, float scale,
                               float *out32, double *out64, uint16_t *out_bf16, float *lse)
+{
+    oasis_oracle_sparse_attn_abs(B, T, Hq, Hkv, d, bs, q, pool, slot_tbl, blk_tbl, n_cols, seq_len, scale,
+                                 out32, out64, out_bf16, lse, NULL);
+}
+
+void oasis_oracle_sparse_attn_abs(int32_t B, int32_t T, int32_t Hq, int32_t Hkv, int32_t d,
+                                  int32_t bs, const uint16_t *q, const uint16_t *pool,
+                                  const int32_t *slot_tbl, const int32_t *blk_tbl,
+                                  int32_t n_cols, const int32_t *seq_len, float scale,
+                                  float *out32, double *out64, uint16_t *out_bf16, float *lse,
+                                  double *out_abs)
 {
     const int32_t G = Hq / Hkv;
     const int64_t max_keys = (int64_t)n_cols * bs;
@@ -255,6 +276,7 @@ void oasis_oracle_sparse_attn(int32_t B, int32_t T, int32_t Hq, int32_t Hkv, int
     const uint16_t **vrow = (const uint16_t **)malloc(sizeof(void *) * (size_t)(max_keys > 0 ? max_keys : 1));
     float *acc = (float *)malloc(sizeof(float) * (size_t)d);
     double *acc64 = (double *)malloc(sizeof(double) * (size_t)d);
+    double *accabs = (double *)malloc(sizeof(double) * (size_t)d);
 
     for (int32_t b = 0; b < B; ++b) {
         for (int32_t t = 0; t < T; ++t) {
@@ -290,6 +312,7 @@ void oasis_oracle_sparse_attn(int32_t B, int32_t T, int32_t Hq, int32_t Hkv, int
                         if (out32) out32[o * d + x] = 0.0f;
                         if (out64) out64[o * d + x] = 0.0;
                         if (out_bf16) out_bf16[o * d + x] = 0;
+                        if (out_abs) out_abs[o * d + x] = 0.0;
                     }
                     if (lse) lse[o] = -INFINITY;
                     continue;
@@ -305,6 +328,7 @@ void oasis_oracle_sparse_attn(int32_t B, int32_t T, int32_t Hq, int32_t Hkv, int
                 for (int32_t x = 0; x < d; ++x) {
                     acc[x] = 0.0f;
                     acc64[x] = 0.0;
+                    accabs[x] = 0.0;
                 }
                 for (int64_t p = 0; p < nk; ++p) {
                     float w = expf(logit[p] - mx);
@@ -315,6 +339,7 @@ void oasis_oracle_sparse_attn(int32_t B, int32_t T, int32_t Hq, int32_t Hkv, int
                         float v = bf16_to_f32(vrow[p][x]);
                         acc[x] = acc[x] + w * v;
                         acc64[x] = acc64[x] + w64 * (double)v;
+                        accabs[x] = accabs[x] + w64 * fabs((double)v);
                     }
                 }
                 for (int32_t x = 0; x < d; ++x) {
@@ -322,6 +347,7 @@ void oasis_oracle_sparse_attn(int32_t B, int32_t T, int32_t Hq, int32_t Hkv, int
                     if (out32) out32[o * d + x] = r;
                     if (out64) out64[o * d + x] = acc64[x] / den64;
                     if (out_bf16) out_bf16[o * d + x] = f32_to_bf16(r);
+                    if (out_abs) out_abs[o * d + x] = accabs[x] / den64;
                 }
                 if (lse) lse[o] = mx + logf(den);
             }
@@ -332,6 +358,7 @@ void oasis_oracle_sparse_attn(int32_t B, int32_t T, int32_t Hq, int32_t Hkv, int
     free(vrow);
     free(acc);
     free(acc64);
+    free(accabs);
 }
 
 /* ---------------------------------------------------------------- lookahead recall

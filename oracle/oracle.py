@@ -108,7 +108,8 @@ def stage_blocks(host_kv, idx, slots, pool):
 
 def sparse_attn(q, pool, slot_tbl, blk_tbl, seq_len, scale, Hkv):
     """q [B][T][Hq][d] u16, pool [n_slots][2][bs][d] u16, tables [B][Hkv][n_cols]
-    -> dict(out32, out64, out_bf16, lse)."""
+    -> dict(out32, out64, out_bf16, lse, out_abs); out_abs = sum_p softmax_p * |v_p| (fp64), the scale of the
+    terms behind each output element."""
     q, pool = _u16(q), _u16(pool)
     B, T, Hq, d = q.shape
     bs = pool.shape[-2]
@@ -118,10 +119,11 @@ def sparse_attn(q, pool, slot_tbl, blk_tbl, seq_len, scale, Hkv):
     out64 = np.empty((B, T, Hq, d), dtype=np.float64)
     out16 = np.empty((B, T, Hq, d), dtype=np.uint16)
     lse = np.empty((B, T, Hq), dtype=np.float32)
-    lib().oasis_oracle_sparse_attn(B, T, Hq, int(Hkv), d, bs, _p(q), _p(pool), _p(slot_tbl),
-                                   _p(blk_tbl), n_cols, _p(seq_len), ctypes.c_float(scale),
-                                   _p(out32), _p(out64), _p(out16), _p(lse))
-    return dict(out32=out32, out64=out64, out_bf16=out16, lse=lse)
+    out_abs = np.empty((B, T, Hq, d), dtype=np.float64)
+    lib().oasis_oracle_sparse_attn_abs(B, T, Hq, int(Hkv), d, bs, _p(q), _p(pool), _p(slot_tbl),
+                                       _p(blk_tbl), n_cols, _p(seq_len), ctypes.c_float(scale),
+                                       _p(out32), _p(out64), _p(out16), _p(lse), _p(out_abs))
+    return dict(out32=out32, out64=out64, out_bf16=out16, lse=lse, out_abs=out_abs)
 
 
 def topk_recall(sel_draft, sel_true, k):

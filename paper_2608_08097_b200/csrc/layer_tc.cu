@@ -407,7 +407,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     } else if (warp == 2) {
         // ---------------------------------------------------------------- P V issuer
         if (lane == 0) {
-            const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
+            const uint32_t idesc_pv = (1u << 4) | kIdescPvFormats | (1u << 16) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
             const uint64_t v_desc0 = smem_desc_sw128_mn(kv_u32 + kImgPart, kImgHalf, kImgGroup);
             bool alive = true;
             int s = 0, sb = 0;
@@ -619,7 +619,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                     const float p0 = fast_exp2(fmaf(x[2 * e], p.scale_log2, neg_m));
                     const float p1 = fast_exp2(fmaf(x[2 * e + 1], p.scale_log2, neg_m));
                     sum4[e & 3] += p0 + p1;
-                    pk[e] = pack_bf16x2(p0, p1);
+                    pk[e] = pack_p(p0, p1);
                 }
                 l_sum += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
                 if (!has_row) {

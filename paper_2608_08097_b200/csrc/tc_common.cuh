@@ -147,6 +147,10 @@ constexpr int kAtSBufs = 4;                                 // S / P buffers in 
 constexpr int kAtQBytes = 0;                                // Q lives in tensor memory
 constexpr int kAtMaxStages = 7;
 constexpr int kAtTmemCols = 512;                            // S buffers [0,256), O [256,384), Q [384,448)
+// The softmax weights P go to the P V product as bf16, like V: the two operands of one tcgen05.mma kind::f16 must
+// have the same format (fp16 weights against bf16 values raise an illegal-instruction fault on B200).
+constexpr uint32_t kIdescPvFormats = (1u << 7) | (1u << 10);
+__device__ __forceinline__ uint32_t pack_p(float lo, float hi) { return pack_bf16x2(lo, hi); }
 constexpr float kAtLog2e = 1.4426950408889634f;
 constexpr float kAtLn2 = 0.6931471805599453f;
 

@@ -78,12 +78,33 @@ def assert_sel_parity(gpu_sel, ref_sel, s64, k):
     return len(diff)
 
 
-def assert_attn_close(gpu_out, ref32):
+BF16_HALF_ULP = 2.0 ** -9           # relative rounding error of a value kept to 8 significant bits
+MAX_BOUND_FRACTION = 1e-5           # share of the elements that may need the arithmetic bound instead of the tolerance
+
+
+def assert_attn_close(gpu_out, ref):
+    """ref: the oracle's result dict (or just its fp32 output).  Every element must lie within
+    atol 2e-3 + rtol 1e-2 of the oracle.  The tensor core takes the softmax weights as bf16, which perturbs an
+    output element by up to 2^-9 * sum_p w_p |v_p| whatever the element's own size; in rows whose softmax is carried
+    by a few keys with large values that can exceed atol at a small element.  Such elements -- at most 1e-5 of
+    all -- must then lie within the worst case of that arithmetic, 2^-9 * (2 * sum_p w_p |v_p| + |out|) (weights
+    rounded in the numerator, exact in the denominator, output rounded to bf16), which the oracle's out_abs gives."""
+    ref32 = ref["out32"] if isinstance(ref, dict) else ref
     g = gpu_out.astype(np.float64)
     r = ref32.astype(np.float64)
-    err = np.abs(g - r) - (ATTN_ATOL + ATTN_RTOL * np.abs(r))
-    worst = err.max(initial=-1.0)
-    assert worst <= 0, "attention off by %.3g beyond tolerance (max abs err %.3g)" % (worst, np.abs(g - r).max())
+    err = np.abs(g - r)
+    over = err - (ATTN_ATOL + ATTN_RTOL * np.abs(r))
+    worst = over.max(initial=-1.0)
+    if worst <= 0:
+        return
+    assert isinstance(ref, dict) and "out_abs" in ref, \
+        "attention off by %.3g beyond tolerance (max abs err %.3g)" % (worst, err.max())
+    bad = over > 0
+    bound = BF16_HALF_ULP * (2.0 * ref["out_abs"] + np.abs(r)) + 1e-6
+    assert (err[bad] <= bound[bad]).all(), \
+        "attention off by %.3g beyond tolerance and beyond the bf16-weight bound (max abs err %.3g)" % (worst, err.max())
+    assert bad.sum() <= max(1, int(MAX_BOUND_FRACTION * bad.size)), \
+        "%d of %d elements beyond tolerance (worst by %.3g): more than rounding of the weights explains" % (bad.sum(), bad.size, worst)
 
 
 def bf16_to_f32_np(t):

@@ -163,7 +163,7 @@ def test_engine_steps_match_oracle(oracle, gpu, mode, cap, append, chunk, graph,
                                      kv_ref[l])
                 # attention of this step ran over the working set predicted one step earlier
                 ref = oracle.sparse_attn(pu.np_u16(lays[l].q_steps[s]), pools[l], slot_tbl, blk[l], seq[s].numpy(), SCALE, Hkv)
-                pu.assert_attn_close(pu.bf16_to_f32_np(got_out[(s, l)]), ref["out32"])
+                pu.assert_attn_close(pu.bf16_to_f32_np(got_out[(s, l)]), ref)
                 # this step's prediction and transfer, for the next step
                 sel, idx, slots, s64 = oracle_prediction_on(l, s, ((seq[s] + 1) // 16).numpy(), (seq[s] + 1).numpy())
                 gsel = sel_log[s][l].cpu().numpy()
@@ -235,7 +235,7 @@ def test_handover_from_dense_pool_then_decode(oracle, gpu):
     eng.join()
     torch.cuda.synchronize()
     ref = oracle.sparse_attn(pu.np_u16(lay.q_steps[0]), pool, slot_tbl, sel, seq[0].numpy(), SCALE, Hkv)
-    pu.assert_attn_close(pu.bf16_to_f32_np(eng.layers[0].out), ref["out32"])
+    pu.assert_attn_close(pu.bf16_to_f32_np(eng.layers[0].out), ref)
 
 
 @pytest.mark.parametrize("mode,cap", [("fetch_all", None), ("delta", 2)])

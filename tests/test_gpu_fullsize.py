@@ -53,7 +53,7 @@ def check_request(oracle, cfg, lay, L, b, k, q_cpu, n_draft_rows=None):
     rows = slice(b * Hkv * (k + 2), (b + 1) * Hkv * (k + 2))
     assert np.array_equal(pu.np_u16(L.pool[rows]), pool)
     ref = oracle.sparse_attn(q, pool, slots, gsel, seq, SCALE, Hkv)
-    pu.assert_attn_close(pu.bf16_to_f32_np(L.out[b:b + 1]), ref["out32"])
+    pu.assert_attn_close(pu.bf16_to_f32_np(L.out[b:b + 1]), ref)
     return n_adj
 
 
@@ -181,6 +181,6 @@ def test_full_size_engine_steps(oracle, gpu):
                 pool = np.zeros((Hkv * (k + 2), 2, 16, 128), np.uint16)
                 oracle.stage_blocks(kv.reshape(-1, 2, 16, 128), gidx, slots, pool)
                 ref = oracle.sparse_attn(pu.np_u16(lays[l].q_steps[s][b:b + 1]), pool, slots, gsel, sq, SCALE, Hkv)
-                pu.assert_attn_close(pu.bf16_to_f32_np(eng.layers[l].out[b:b + 1]), ref["out32"])
+                pu.assert_attn_close(pu.bf16_to_f32_np(eng.layers[l].out[b:b + 1]), ref)
         used_sel = [eng.layers[l].sel.cpu().numpy() for l in range(n_layers)]
         prev_q = s

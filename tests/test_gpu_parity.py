@@ -73,7 +73,7 @@ def compare_path(oracle, pipeline, lay, k, step=0, reduce_mode=0, kv_on="pinned"
     slot_tbl = np.arange(gsel.size, dtype=np.int32).reshape(gsel.shape)
     ref_attn = oracle.sparse_attn(ref["q"], want_pool, slot_tbl, gsel, ref["seq_len"],
                                   np.float32(1.0 / math.sqrt(128.0)), cfg.n_kv_heads)
-    pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref_attn["out32"])
+    pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref_attn)
     np.testing.assert_allclose(L.lse.cpu().numpy(), ref_attn["lse"], rtol=1e-3, atol=2e-3)
     # and attention on the ORACLE's selection and pool (independent of the GPU's choices)
     if n_adj:
@@ -81,7 +81,7 @@ def compare_path(oracle, pipeline, lay, k, step=0, reduce_mode=0, kv_on="pinned"
         L.pool.copy_(torch.from_numpy(ref["pool"].view(np.int16)).view(torch.bfloat16).to(dev))
         L.attend(dv["q"], dv["seq_len"], blk_tbl=torch.from_numpy(ref["sel"]).to(dev))
         torch.cuda.synchronize()
-        pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref["attn"]["out32"])
+        pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref["attn"])
     return L, ref, n_adj
 
 
@@ -202,7 +202,7 @@ def test_consecutive_steps_with_growing_context(oracle, gpu):
         if 12 <= s < 16:
             assert (gsel[:, :, cfg.k_blocks + 1] >= 0).all()            # second local block in use
         if n_adj == 0:
-            pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref["attn"]["out32"])
+            pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref["attn"])
 
 
 def _select_only(binding, scores, n_full, seq_len, T, k, table=None, with_lists=True):
@@ -298,7 +298,7 @@ def test_attention_padding_rows_and_empty_columns(oracle, gpu):
     slot_tbl = np.arange(sel.size, dtype=np.int32).reshape(sel.shape)
     ref = oracle.sparse_attn(pu.np_u16(lay.q), pu.np_u16(L.pool), slot_tbl, sel, lay.seq_len.numpy(),
                              np.float32(1.0 / math.sqrt(128.0)), cfg.n_kv_heads)
-    pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref["out32"])
+    pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref)
     G = cfg.group
     assert (pu.bf16_to_f32_np(L.out)[1, :, 2 * G:3 * G] == 0).all()
     assert np.isneginf(L.lse.cpu().numpy()[1, :, 2 * G:3 * G]).all()
@@ -585,7 +585,7 @@ def test_fused_launch_against_the_oracle(oracle, gpu, name, spec, kw):
     torch.cuda.synchronize()
     pu.assert_scores_close(L.scores.cpu().numpy(), ref["s32"], ref["s64"], ref["n_full"])
     pu.assert_sel_parity(L.sel.cpu().numpy(), ref["sel"], ref["s64"], k)
-    pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref["attn"]["out32"])
+    pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref["attn"])
     np.testing.assert_allclose(L.lse.cpu().numpy(), ref["attn"]["lse"], rtol=1e-3, atol=2e-3)
 
 
@@ -649,7 +649,7 @@ def test_unwritten_tail_of_the_local_block_may_hold_any_finite_pattern(oracle, g
     L.attend(dv["q"], dv["seq_len"])
     torch.cuda.synchronize()
     assert torch.equal(L.out.view(torch.int16), want.view(torch.int16))
-    pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref["attn"]["out32"])
+    pu.assert_attn_close(pu.bf16_to_f32_np(L.out), ref["attn"])
 
 
 @pytest.mark.parametrize("host_on", ["pinned", "device"])

@@ -880,3 +880,30 @@ def test_block_mass_closed_form_for_identical_keys(oracle):
     qbits, _ = rand_bf16(np.random.default_rng(2), (B, Tq, Hq, d))
     got = oracle.block_mass(qbits, bits, table, seq, 1.0)[0, 0]
     np.testing.assert_allclose(got, [4 / 14, 4 / 14, 4 / 14, 3 / 15, 0.0], rtol=1e-12)
+
+
+def test_attention_abs_weighted_output(oracle):
+    """out_abs = sum_p softmax_p |v_p|: equals the output itself when no value is negative, never lies below
+    |output|, and equals the brute-force sum on contiguous keys."""
+    rng = np.random.default_rng(41)
+    B, Hq, Hkv, d, bs, T, mb = 1, 2, 1, 8, 4, 2, 5
+    bits, vals = make_pool(rng, mb, Hkv, bs, d)
+    table = np.arange(mb, dtype=np.int32).reshape(1, mb)
+    seq = np.array([14], np.int32)
+    qbits, q = rand_bf16(rng, (B, T, Hq, d))
+    blk = np.arange(mb, dtype=np.int32).reshape(1, 1, mb)
+    slots = np.arange(mb, dtype=np.int32).reshape(1, 1, mb)
+    res = oracle.sparse_attn(qbits, bits.reshape(-1, 2, bs, d), slots, blk, seq, 0.5, Hkv)
+    assert (res["out_abs"] >= np.abs(res["out64"]) - 1e-15).all()
+    K, V = contiguous_kv(vals, table[0], Hkv)
+    for t in range(T):
+        for a in range(Hq):
+            n = int(seq[0]) + t + 1
+            logits = (K[0, :n].astype(np.float64) @ q[0, t, a].astype(np.float64)) * 0.5
+            w = np.exp(logits - logits.max())
+            want = (w[:, None] * np.abs(V[0, :n].astype(np.float64))).sum(0) / w.sum()
+            np.testing.assert_allclose(res["out_abs"][0, t, a], want, rtol=1e-12)
+    pos_bits = bits.copy()
+    pos_bits[:, :, 1] &= 0x7fff                                         # clear the sign bit of every value
+    res2 = oracle.sparse_attn(qbits, pos_bits.reshape(-1, 2, bs, d), slots, blk, seq, 0.5, Hkv)
+    np.testing.assert_allclose(res2["out_abs"], res2["out64"], rtol=1e-12)

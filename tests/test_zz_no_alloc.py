@@ -53,7 +53,7 @@ def test_static_scratch_attention_matches_workspace_attention_twice(oracle):
         # and against the oracle, on the selection and working set the GPU produced
         ref = oracle.sparse_attn(pu.np_u16(lay.q), pu.np_u16(L.pool), L.slot_tbl.cpu().numpy(), L.sel.cpu().numpy(),
                                  lay.seq_len.numpy(), np.float32(scale), cfg.n_kv_heads)
-        pu.assert_attn_close(pu.bf16_to_f32_np(got), ref["out32"])
+        pu.assert_attn_close(pu.bf16_to_f32_np(got), ref)
         np.testing.assert_allclose(got_lse.cpu().numpy(), ref["lse"], rtol=1e-3, atol=2e-3)
 
 
