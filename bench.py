@@ -59,9 +59,10 @@ def parse_args():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--fetch-ratio", type=float, default=0.05, help="cap of the delta gather, fraction of K")
     ap.add_argument("--group", type=int, default=0, help="decode steps per CUDA graph (0: all timed steps in one)")
-    ap.add_argument("--wait-group", type=int, default=8, help="layers per pick-up of the side streams' events")
+    ap.add_argument("--wait-group", type=int, default=0,
+                    help="layers per pick-up of the side streams' events (0: a quarter of the layers, at most 8)")
     ap.add_argument("--transfer-group", type=int, default=0,
-                    help="layers per gather launch when the pool is in host memory (0: 4 when the host link bounds the step, else 1)")
+                    help="layers per gather launch when the pool is in host memory (0: up to 4 when the host link bounds the step, else 1)")
     ap.add_argument("--repeats", type=int, default=1, help="replay the timed steps this many times in a second, long "
                                                             "timed region (reported as `sustained`)")
     ap.add_argument("--sweep-ratios", default="", help="comma-separated fetch ratios to sweep (e.g. 0.01,0.02,0.05)")
@@ -304,7 +305,13 @@ class Bench:
         link_us = cap * cfg.batch * cfg.n_kv_heads * 8192 / (0.9 * self.h2d_peak * 1e3)
         score, attn = algorithmic_bytes(cfg, w.k, w.T, self.seq_steps, [0])
         compute_us = (score + attn) / (0.85 * self.hbm_peak * 1e3)
-        return 4 if link_us > compute_us else 1
+        return max(1, min(4, cfg.layers // 4)) if link_us > compute_us else 1
+
+    def wait_group(self):
+        """Layers whose side-stream events the foreground stream picks up together: few enough that a step's last
+        transfers overlap the next step's first layers, many enough to keep most consecutive fused launches
+        overlapping."""
+        return self.args.wait_group if self.args.wait_group > 0 else max(1, min(8, self.cfg.layers // 4))
 
     def engine(self, w, kv_list, cap):
         cfg = self.cfg
@@ -314,7 +321,7 @@ class Bench:
         eng = self.pipeline.DecodeEngine(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.max_blocks, w.k, w.T,
                                          self.n_layers, self.dev, mode="delta", cap=cap, append=True,
                                          transfer_streams=getattr(self.args, "transfer_streams", 1),
-                                         plan_stream=getattr(self.args, "plan_stream", "own"), wait_group=self.args.wait_group,
+                                         plan_stream=getattr(self.args, "plan_stream", "own"), wait_group=self.wait_group(),
                                          n_commit=getattr(self.args, "n_commit", 1),
                                          transfer_ctas=getattr(self.args, "transfer_ctas", 0) if host_pool else 0,
                                          transfer_group=self.transfer_group(w, cap) if host_pool else 1)
@@ -732,7 +739,7 @@ def run_ours(args):
                        "launch": "CUDA graphs of %d consecutive decode steps over 6-10 streams; a layer's attention and scoring are "
                                  "one fused launch (oasis_attn_and_score); gathers of %d layers per launch; side-stream events "
                                  "picked up every %d layers" % (args.group if args.group > 0 else K, bench.transfer_group(w, cap),
-                                                                 args.wait_group)},
+                                                                 bench.wait_group())},
             "gpu_launches": host.get("launches"),
             "clocks": {kk: (host.get("clocks") or {}).get(kk) for kk in ("sm_mhz", "sm_max_mhz", "reasons", "samples")},
             "roofline": {"bound": "hbm", "kernel": dom, "achieved": d.get("GBps"), "peak": hbm_peak, "unit": "GB/s",

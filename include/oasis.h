@@ -369,6 +369,22 @@ int oasis_union_blocks(const oasis_dims_t *dims, const int32_t *sel, int32_t sel
 int oasis_set_error_word(int32_t *device_word);
 
 /*
+ * Bounds-check build (no counterpart in the paper: a debugging aid of this library).  The library also builds
+ * with -DOASIS_BOUNDS_CHECK (liboasis_checked.so).  In that build every index that a kernel reads from a device
+ * array is range-checked on the device before use: entries of the full-KV pool (block_table[..] * Hkv + h, idx[])
+ * against n_host_entries, slots (slots[], slot_tbl[..], computed plan slots) against n_slots, logical block ids
+ * against dims->max_blocks, per-request block counts and ranges against dims->max_blocks.  A violation writes
+ * its code into the error word registered with oasis_set_error_word (the first violation wins: 201 host entry,
+ * 202 slot, 203 block id, 204 block count) and the access is skipped -- the request is dropped, the column is
+ * treated as missing, the count is clamped; nothing traps or asserts.  The attention's tensor map then also
+ * declares the pool's real extent.  oasis_set_extents declares the two extents (process-wide, like the error
+ * word; 0 = unknown = unchecked); in the regular build it is accepted and has no effect.
+ * oasis_bounds_checked() tells which build is loaded (1 = checked).
+ */
+int oasis_set_extents(int64_t n_host_entries, int64_t n_slots);
+int oasis_bounds_checked(void);
+
+/*
  * Self-test of the bounded waits behind oasis_set_error_word (no counterpart in the paper).  One small
  * launch waits, with a bound of `probes` polls (1 .. 2^20), on a barrier that nothing ever completes; the
  * wait gives up, the kernel records code 99 in the registered error word (if one is registered and still

@@ -13,7 +13,8 @@ from dataclasses import dataclass
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "liboasis.so")
+# OASIS_LIB selects another build of the library for the whole process (the bounds-check build liboasis_checked.so)
+LIB_PATH = os.environ.get("OASIS_LIB") or os.path.join(_HERE, "liboasis.so")
 
 REDUCE_MAX, REDUCE_SUM = 0, 1
 ENTRY_BYTES = 8192
@@ -23,7 +24,8 @@ SYMBOLS = ("oasis_build_summaries", "oasis_score_blocks", "oasis_select_topk",
            "oasis_sparse_attn_static_scratch", "oasis_static_scratch_bytes", "oasis_set_error_word", "oasis_union_blocks",
            "oasis_offload_blocks", "oasis_attn_and_score", "oasis_attn_and_score_supported",
            "oasis_build_summaries_layers", "oasis_selftest_wait_timeout",
-           "oasis_local_window", "oasis_append_kv", "oasis_append_kv_layers", "oasis_stage_blocks_layers")
+           "oasis_local_window", "oasis_append_kv", "oasis_append_kv_layers", "oasis_stage_blocks_layers",
+           "oasis_set_extents", "oasis_bounds_checked")
 
 
 class OasisError(RuntimeError):
@@ -99,6 +101,10 @@ def lib():
         L.oasis_append_kv_layers.restype = ctypes.c_int
         L.oasis_selftest_wait_timeout.argtypes = [ctypes.c_uint32, vp, vp]
         L.oasis_selftest_wait_timeout.restype = ctypes.c_int
+        L.oasis_set_extents.argtypes = [i64, i64]
+        L.oasis_set_extents.restype = ctypes.c_int
+        L.oasis_bounds_checked.argtypes = []
+        L.oasis_bounds_checked.restype = ctypes.c_int
         L.oasis_set_error_word.argtypes = [vp]
         L.oasis_set_error_word.restype = ctypes.c_int
         L.oasis_last_error.restype = ctypes.c_char_p
@@ -112,6 +118,17 @@ def set_error_word(word):
     wait time-out; None unregisters."""
     _check(lib().oasis_set_error_word(None if word is None else ctypes.c_void_p(word.data_ptr())),
            "oasis_set_error_word")
+
+
+def set_extents(n_host_entries, n_slots):
+    """Declares the sizes the bounds-check build checks indices against (entries of the full-KV pool, slots of
+    the working-set pool; 0 = unknown)."""
+    _check(lib().oasis_set_extents(int(n_host_entries), int(n_slots)), "oasis_set_extents")
+
+
+def bounds_checked() -> bool:
+    """Whether the loaded library is the bounds-check build."""
+    return bool(lib().oasis_bounds_checked())
 
 
 def selftest_wait_timeout(probes, result=None, stream=None):

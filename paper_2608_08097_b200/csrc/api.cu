@@ -65,6 +65,9 @@ int sm_count()
 static int32_t *g_error_word = nullptr;
 int32_t *error_word() { return g_error_word; }
 
+static long long g_n_entries = 1ll << 62, g_n_slots = 1ll << 31;
+Bounds bounds() { return Bounds{g_n_entries, g_n_slots, g_error_word}; }
+
 }  // namespace oasis
 
 extern "C" int oasis_set_error_word(int32_t *device_word)
@@ -72,6 +75,19 @@ extern "C" int oasis_set_error_word(int32_t *device_word)
     oasis::g_error_word = device_word;
     return OASIS_OK;
 }
+
+extern "C" int oasis_set_extents(int64_t n_host_entries, int64_t n_slots)
+{
+    using namespace oasis;
+    if (n_host_entries < 0 || n_slots < 0 || n_slots > (1ll << 31))
+        return fail(OASIS_ERR_INVALID_ARG, "oasis_set_extents: n_host_entries %lld, n_slots %lld", (long long)n_host_entries,
+                    (long long)n_slots);
+    g_n_entries = n_host_entries > 0 ? n_host_entries : 1ll << 62;
+    g_n_slots = n_slots > 0 ? n_slots : 1ll << 31;
+    return OASIS_OK;
+}
+
+extern "C" int oasis_bounds_checked(void) { return oasis::kBoundsCheck ? 1 : 0; }
 
 extern "C" const char *oasis_last_error(void) { return oasis::g_last_error; }
 extern "C" const char *oasis_version(void) { return "0.1"; }

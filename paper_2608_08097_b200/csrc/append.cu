@@ -38,7 +38,7 @@ __device__ __forceinline__ void set_local_columns(int32_t *cols, int lo, int hi)
 }
 
 __global__ void __launch_bounds__(kAppendWarps * 32)
-append_kv_kernel(const __grid_constant__ AppendLayers ly_all, const AppendParams p)
+append_kv_kernel(const __grid_constant__ AppendLayers ly_all, const AppendParams p, const Bounds bd)
 {
     const int l = blockIdx.y;
     struct {
@@ -61,10 +61,12 @@ append_kv_kernel(const __grid_constant__ AppendLayers ly_all, const AppendParams
         const uint4 v = *reinterpret_cast<const uint4 *>(ly.new_kv + (long long)w * 2 * kRowBytes + part * kRowBytes + off);
         const long long slot = ly.slot_tbl[row * p.n_cols + p.local_col + (j & 1)];
         const long long in_entry = (long long)part * kPartBytes + (long long)i * kRowBytes + off;
-        *reinterpret_cast<uint4 *>(ly.pool + slot * kEntryBytes + in_entry) = v;
-        if (ly.host_kv && t < p.n_commit) {
+        if (in_range(slot, bd.n_slots, bd, kErrSlot))
+            *reinterpret_cast<uint4 *>(ly.pool + slot * kEntryBytes + in_entry) = v;
+        if (ly.host_kv && t < p.n_commit && in_range(j, p.max_blocks, bd, kErrBlockId)) {
             const long long phys = ly.block_table[(long long)b * p.max_blocks + j];
-            *reinterpret_cast<uint4 *>(ly.host_kv + (phys * p.Hkv + h) * kEntryBytes + in_entry) = v;
+            if (in_range(phys * p.Hkv + h, bd.n_entries, bd, kErrHostEntry))
+                *reinterpret_cast<uint4 *>(ly.host_kv + (phys * p.Hkv + h) * kEntryBytes + in_entry) = v;
         }
     }
 }
@@ -72,7 +74,7 @@ append_kv_kernel(const __grid_constant__ AppendLayers ly_all, const AppendParams
 __global__ void __launch_bounds__(128)
 local_window_kernel(const int32_t *__restrict__ seq_len, const int32_t *__restrict__ block_table,
                     int32_t *__restrict__ blk_tbl, long long *__restrict__ stage_idx, int32_t *__restrict__ stage_slots,
-                    int B, int T, int Hkv, int max_blocks, int n_cols, int local_col, int slot_stride)
+                    int B, int T, int Hkv, int max_blocks, int n_cols, int local_col, int slot_stride, const Bounds bd)
 {
     const int row = blockIdx.x * blockDim.x + threadIdx.x;
     if (row >= B * Hkv) return;
@@ -86,7 +88,8 @@ local_window_kernel(const int32_t *__restrict__ seq_len, const int32_t *__restri
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
             stage_slots[row * 2 + r] = row * slot_stride + local_col + r;
-            stage_idx[row * 2 + r] = c[r] < 0 ? -1ll : (long long)block_table[(long long)b * max_blocks + c[r]] * Hkv + h;
+            stage_idx[row * 2 + r] = (c[r] < 0 || !in_range(c[r], max_blocks, bd, kErrBlockId))
+                                         ? -1ll : (long long)block_table[(long long)b * max_blocks + c[r]] * Hkv + h;
         }
     }
 }
@@ -140,7 +143,7 @@ static int launch_append(const oasis_dims_t *dims, int n_layers, const void *con
     long long grid = (total + kAppendWarps - 1) / kAppendWarps;
     if (grid > 4096) grid = 4096;
     prefer_max_shared_carveout(append_kv_kernel);
-    append_kv_kernel<<<dim3((unsigned)grid, (unsigned)n_layers), kAppendWarps * 32, 0, st>>>(ly, p);
+    append_kv_kernel<<<dim3((unsigned)grid, (unsigned)n_layers), kAppendWarps * 32, 0, st>>>(ly, p, bounds());
     return check_launch(who);
 }
 
@@ -183,6 +186,6 @@ extern "C" int oasis_local_window(const oasis_dims_t *dims, const int32_t *seq_l
     prefer_max_shared_carveout(local_window_kernel);
     local_window_kernel<<<(rows + 127) / 128, 128, 0, (cudaStream_t)stream>>>(
         seq_len, block_table, blk_tbl, (long long *)stage_idx, stage_slots, dims->batch, n_q_tokens, dims->n_kv_heads,
-        dims->max_blocks, n_cols, local_col, slot_stride);
+        dims->max_blocks, n_cols, local_col, slot_stride, bounds());
     return check_launch(who);
 }

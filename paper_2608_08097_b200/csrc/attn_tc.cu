@@ -54,6 +54,7 @@ struct AttnTcParams {
     int32_t *err;
     float scale_log2;
     int T, Hq, Hkv, G, n_cols, R, n_splits, cols_per_split, stages;
+    long long n_slots;          // bounds-check build: slots of the working-set pool (else unused)
 };
 
 // MMA_M = 64 halves the tensor work when the query rows fit; its rows live in tensor-memory lanes
@@ -152,6 +153,7 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
             const int c = first_col + lane;
             wblk = c < c1 ? blk_row[c] : -1;
             wslot = c < c1 ? slot_row[c] : -1;
+            if (kBoundsCheck && wblk >= 0 && !in_range(wslot, p.n_slots, Bounds{0, 0, p.err}, kErrSlot)) wblk = -1;
         };
         int cur_blk, cur_slot, nxt_blk = -1, nxt_slot = -1;
         load_window(c0, cur_blk, cur_slot);
@@ -496,7 +498,11 @@ int launch_attn_tc(const oasis_dims_t *dims, const void *q, int n_q_tokens, cons
     // the two 64-dim halves of a row | the two 8-row groups of a part.  One box = one whole 8 KiB entry, landing as
     // [group][half][part][8 rows][128 B], so that 8-row groups of consecutive blocks are uniformly 4096 bytes apart.
     CUtensorMap tmap;
-    const cuuint64_t gdim[5] = {64, 8, (cuuint64_t)1 << 31, 2, 2};
+    // (bounds-check build with declared extents: the map covers exactly the pool's slots, so a copy by a slot id
+    // outside them would read the fill value instead of foreign memory -- and such ids are dropped before that)
+    const cuuint64_t pool_parts = (kBoundsCheck && bounds().n_slots < (1ll << 30)) ? (cuuint64_t)(2 * bounds().n_slots)
+                                               : (cuuint64_t)1 << 31;
+    const cuuint64_t gdim[5] = {64, 8, pool_parts, 2, 2};
     const cuuint64_t gstride[4] = {256, 4096, 128, 2048};
     const cuuint32_t box[5] = {64, 8, 2, 2, 2};
     const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
@@ -512,6 +518,7 @@ int launch_attn_tc(const oasis_dims_t *dims, const void *q, int n_q_tokens, cons
     p.T = n_q_tokens; p.Hq = dims->n_q_heads; p.Hkv = dims->n_kv_heads; p.G = p.Hq / p.Hkv;
     p.n_cols = n_cols; p.R = n_q_tokens * p.G; p.n_splits = n_splits; p.cols_per_split = cols_per_split;
     p.stages = stages;
+    p.n_slots = bounds().n_slots;
     const size_t smem = attn_tc_smem_bytes(stages);
     const long long grid = (long long)dims->batch * dims->n_kv_heads * n_splits;
     cudaError_t e;

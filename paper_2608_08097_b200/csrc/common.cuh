@@ -23,6 +23,36 @@ int check_launch(const char *what);   // cudaGetLastError() -> status
 int sm_count();                       // multiprocessors of the current device (148 if unknown)
 int32_t *error_word();                // device word registered with oasis_set_error_word (or NULL)
 
+// ---- bounds-check build (-DOASIS_BOUNDS_CHECK) ---------------------------------------------------------
+// In that build every index a kernel reads from a device array -- an entry of the full-KV pool, a slot of the
+// working-set pool, a logical block id, a per-request block count -- is range-checked before it is used; a
+// violation records a code in the registered error word (first one wins) and the access is skipped.  Nothing
+// traps.  In the regular build the checks compile to nothing.
+#ifdef OASIS_BOUNDS_CHECK
+constexpr bool kBoundsCheck = true;
+#else
+constexpr bool kBoundsCheck = false;
+#endif
+constexpr int kErrHostEntry = 201;   // index into the full-KV pool outside [0, n_host_entries)
+constexpr int kErrSlot = 202;        // slot outside [0, n_slots)
+constexpr int kErrBlockId = 203;     // logical block id outside [0, max_blocks)
+constexpr int kErrBlockCount = 204;  // per-request block count / range beyond max_blocks
+
+struct Bounds {
+    long long n_entries;   // entries ((block, head) pairs) of the full-KV pool
+    long long n_slots;     // entries of the working-set pool
+    int32_t *err;          // the registered error word (may be NULL)
+};
+Bounds bounds();           // what oasis_set_extents declared (huge when nothing was declared) + the error word
+
+__device__ __forceinline__ bool in_range(long long v, long long n, const Bounds &bd, int code)
+{
+    if constexpr (!kBoundsCheck) return true;
+    if (v >= 0 && v < n) return true;
+    if (bd.err) atomicCAS(bd.err, 0, code);
+    return false;
+}
+
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // ---- device helpers -----------------------------------------------------------------

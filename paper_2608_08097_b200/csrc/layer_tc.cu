@@ -72,6 +72,7 @@ struct LayerTcParams {
     int total_tiles;            // rows * tiles_per_bh (the host checks that summaries rows fit 31 bits)
     double w_row, w_free;       // scoring tiles of a CTA with the larger / the smaller number of attention rows
     int32_t *err;
+    long long n_slots;          // bounds-check build: slots of the working-set pool (else unused)
 };
 
 // MODE: 0 = at most one whole row per thread block; 1 = more rows than thread blocks, several whole rows per block;
@@ -275,6 +276,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             const int c = first + lane;
             wblk = c < c1 ? blk_row[c] : -1;
             wslot = c < c1 ? slot_row[c] : -1;
+            if (kBoundsCheck && wblk >= 0 && !in_range(wslot, p.n_slots, Bounds{0, 0, p.err}, kErrSlot)) wblk = -1;
         };
         int cur_blk, cur_slot, nxt_blk = -1, nxt_slot = -1;
         load_window(c0, cur_blk, cur_slot);
@@ -473,6 +475,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 const int j0 = (int)(t % p.tiles_per_bh) * kLyTileBlocks;
                 const int b = (int)(bh / p.Hkv);
                 const int nf = p.n_full[b];
+                if (kBoundsCheck && lane == 0 && nf > p.max_blocks) in_range(nf, p.max_blocks + 1, Bounds{0, 0, p.err}, kErrBlockCount);
                 const int j = j0 + quarter * 32 + lane;
                 float *out = p.scores + (long long)bh * p.max_blocks;
                 if (j0 >= nf) {
@@ -916,7 +919,11 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     CUtensorMap tmap_kv, tmap_summ;
     {
         // the pool as 8 KiB entries (see attn_tc.cu): one box = one entry, landing as [group][half][part][8 rows][128 B]
-        const cuuint64_t gdim[5] = {64, 8, (cuuint64_t)1 << 31, 2, 2};
+        // (bounds-check build with declared extents: the map covers exactly the pool's slots, so a copy by a slot id
+        // outside them would read the fill value instead of foreign memory -- and such ids are dropped before that)
+        const cuuint64_t pool_parts = (kBoundsCheck && bounds().n_slots < (1ll << 30)) ? (cuuint64_t)(2 * bounds().n_slots)
+                                                                                       : (cuuint64_t)1 << 31;
+        const cuuint64_t gdim[5] = {64, 8, pool_parts, 2, 2};
         const cuuint64_t gstride[4] = {256, 4096, 128, 2048};
         const cuuint32_t box[5] = {64, 8, 2, 2, 2};
         const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
@@ -952,6 +959,7 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     p.reduce_sum = reduce_mode == OASIS_REDUCE_SUM;
     p.total_tiles = (int)(rows * p.tiles_per_bh);
     p.err = error_word();
+    p.n_slots = bounds().n_slots;
     // Equal bytes per SM: an attention tile is 32 KiB, a scoring tile 64 KiB.  The first `n_more` CTAs attend
     // one row more than the others and take correspondingly fewer scoring tiles.
     const int grid = sms;

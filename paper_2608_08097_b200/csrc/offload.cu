@@ -34,7 +34,7 @@ offload_blocks_kernel(const uint8_t *__restrict__ dense_k, const uint8_t *__rest
                       const int32_t *__restrict__ gpu_table, const int32_t *__restrict__ block_table,
                       const int32_t *__restrict__ first_block, const int32_t *__restrict__ n_blocks,
                       uint8_t *__restrict__ host_kv, uint8_t *__restrict__ summaries, int Hkv, int max_blocks,
-                      int max_new, long long n_items)
+                      int max_new, long long n_items, const Bounds bd)
 {
     const int lane = threadIdx.x & 31;
     const long long item = (long long)blockIdx.x * kOffloadWarps + (threadIdx.x >> 5);
@@ -44,9 +44,13 @@ offload_blocks_kernel(const uint8_t *__restrict__ dense_k, const uint8_t *__rest
     const int b = (int)(item / ((long long)Hkv * max_new));
     if (jj >= n_blocks[b]) return;
     const int j = first_block[b] + jj;
-    if (j < 0 || j >= max_blocks) return;
+    if (j < 0 || j >= max_blocks) {
+        in_range(j, max_blocks, bd, kErrBlockCount);       // (checked build: reported; always skipped)
+        return;
+    }
     const long long src_blk = gpu_table[(long long)b * max_blocks + j];
     const long long dst_blk = block_table[(long long)b * max_blocks + j];
+    if (!in_range(dst_blk * Hkv + h, bd.n_entries, bd, kErrHostEntry)) return;
     constexpr int kPart = kEntryBytes / 2;                          // 4 KiB of keys, 4 KiB of values
     const uint8_t *ksrc = dense_k + (src_blk * Hkv + h) * (long long)kPart + lane * 16;
     const uint8_t *vsrc = dense_v + (src_blk * Hkv + h) * (long long)kPart + lane * 16;
@@ -112,6 +116,6 @@ extern "C" int oasis_offload_blocks(const oasis_dims_t *dims, const void *dense_
     if (grid > 0x7fffffffLL) return fail(OASIS_ERR_UNSUPPORTED, "oasis_offload_blocks: too many blocks");
     offload_blocks_kernel<<<(unsigned)grid, kOffloadWarps * 32, 0, (cudaStream_t)stream>>>(
         (const uint8_t *)dense_k, (const uint8_t *)dense_v, gpu_table, block_table, first_block, n_blocks,
-        (uint8_t *)host_kv, (uint8_t *)summaries, dims->n_kv_heads, dims->max_blocks, max_new_blocks, n_items);
+        (uint8_t *)host_kv, (uint8_t *)summaries, dims->n_kv_heads, dims->max_blocks, max_new_blocks, n_items, bounds());
     return check_launch("oasis_offload_blocks");
 }

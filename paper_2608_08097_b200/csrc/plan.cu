@@ -21,6 +21,7 @@ struct PlanParams {
     int32_t *plan_slots;
     int32_t *n_admitted;
     int Hkv, max_blocks, sel_cols, k, n_res, res_stride, n_local, slot_stride, cap, step, sort_len, bitmap_words;
+    Bounds bd;
 };
 
 constexpr int kPlanThreads = 256;
@@ -53,6 +54,7 @@ plan_delta_kernel(const PlanParams p)
     for (int r = tid; r < p.k; r += kPlanThreads) {
         const int j = pred[r];
         if (j >= 0 && j < p.max_blocks) atomicOr(&pred_bits[j >> 5], 1u << (j & 31));
+        else if (kBoundsCheck && j >= p.max_blocks) in_range(j, p.max_blocks, p.bd, kErrBlockId);
     }
 #pragma unroll 1
     for (int c = tid; c < p.n_res; c += kPlanThreads) {
@@ -138,6 +140,7 @@ plan_delta_kernel(const PlanParams p)
             stp[c] = p.step;
             idx = (long long)p.block_table[(long long)b * p.max_blocks + j] * p.Hkv + h;
             slot = row * p.slot_stride + c;
+            if (!in_range(idx, p.bd.n_entries, p.bd, kErrHostEntry) || !in_range(slot, p.bd.n_slots, p.bd, kErrSlot)) idx = -1;
         }
         p.plan_idx[(long long)row * plan_cols + i] = idx;
         p.plan_slots[(long long)row * plan_cols + i] = slot;
@@ -148,8 +151,12 @@ plan_delta_kernel(const PlanParams p)
         const int j = pred[p.k + i];
         res[p.n_res + i] = j;
         p.plan_slots[(long long)row * plan_cols + p.cap + i] = row * p.slot_stride + p.n_res + i;
-        p.plan_idx[(long long)row * plan_cols + p.cap + i] =
-            (j < 0 || j >= p.max_blocks) ? -1ll : (long long)p.block_table[(long long)b * p.max_blocks + j] * p.Hkv + h;
+        long long lidx = (j < 0 || j >= p.max_blocks) ? -1ll : (long long)p.block_table[(long long)b * p.max_blocks + j] * p.Hkv + h;
+        if (kBoundsCheck && j >= p.max_blocks) in_range(j, p.max_blocks, p.bd, kErrBlockId);
+        if (lidx >= 0 && (!in_range(lidx, p.bd.n_entries, p.bd, kErrHostEntry) ||
+                          !in_range((long long)row * p.slot_stride + p.n_res + i, p.bd.n_slots, p.bd, kErrSlot)))
+            lidx = -1;
+        p.plan_idx[(long long)row * plan_cols + p.cap + i] = lidx;
     }
     if (tid == 0 && p.n_admitted) p.n_admitted[row] = n_pair;
 }
@@ -190,6 +197,7 @@ extern "C" int oasis_plan_delta(const oasis_dims_t *dims, const int32_t *sel, in
     p.plan_idx = (long long *)plan_idx; p.plan_slots = plan_slots; p.n_admitted = n_admitted;
     p.Hkv = dims->n_kv_heads; p.max_blocks = dims->max_blocks; p.sel_cols = sel_cols; p.k = k;
     p.n_res = n_res; p.res_stride = res_stride; p.n_local = n_local; p.slot_stride = slot_stride; p.cap = cap; p.step = step;
+    p.bd = bounds();
     int sort_len = 2;
     while (sort_len < n_res) sort_len <<= 1;
     p.sort_len = sort_len;

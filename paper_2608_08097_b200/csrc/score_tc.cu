@@ -257,6 +257,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
             const int j0 = (int)(t % p.tiles_per_bh) * kTileBlocks;
             const int b = (int)(bh / p.Hkv);
             const int nf = p.n_full[b];
+            if (kBoundsCheck && lane == 0 && nf > p.max_blocks) in_range(nf, p.max_blocks + 1, Bounds{0, 0, p.err}, kErrBlockCount);
             const int j = j0 + quarter * 32 + lane;
             float *out = p.scores + bh * p.max_blocks;
             if (j0 >= nf) {

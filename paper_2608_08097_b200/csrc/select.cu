@@ -23,6 +23,7 @@ struct SelectParams {
     long long *stage_idx;
     int32_t *stage_slots;
     int Hkv, max_blocks, k, n_q_tokens, sort_len;   // sort_len: power of two >= k
+    Bounds bd;
 };
 
 __device__ __forceinline__ uint32_t score_key(float f)
@@ -47,6 +48,7 @@ select_topk_kernel(const SelectParams p)
     const int b = row / p.Hkv, h = row % p.Hkv;
     const int n_full_raw = p.n_full[b];
     const int n = max(0, min(n_full_raw, p.max_blocks));
+    if (kBoundsCheck && threadIdx.x == 0 && n != n_full_raw) in_range(n_full_raw, p.max_blocks + 1, p.bd, kErrBlockCount);
     const int k_eff = min(p.k, n);
     const int n_pad = (n + 31) & ~31;
     const float *srow = p.scores + (long long)row * p.max_blocks;
@@ -242,9 +244,13 @@ select_topk_kernel(const SelectParams p)
         p.sel[o] = v;
         if (p.stage_idx) {
             p.stage_slots[o] = (int32_t)o;
-            p.stage_idx[o] = (v < 0 || v >= p.max_blocks)
-                                 ? -1ll
-                                 : (long long)p.block_table[(long long)b * p.max_blocks + v] * p.Hkv + h;
+            long long src = (v < 0 || v >= p.max_blocks)
+                                ? -1ll
+                                : (long long)p.block_table[(long long)b * p.max_blocks + v] * p.Hkv + h;
+            if (src >= 0 && (!in_range(src, p.bd.n_entries, p.bd, kErrHostEntry) || !in_range(o, p.bd.n_slots, p.bd, kErrSlot)))
+                src = -1ll;
+            if (kBoundsCheck && v >= p.max_blocks) in_range(v, p.max_blocks, p.bd, kErrBlockId);
+            p.stage_idx[o] = src;
         }
     }
 }
@@ -274,6 +280,7 @@ extern "C" int oasis_select_topk(const oasis_dims_t *dims, const float *scores,
 
     SelectParams p;
     p.scores = scores; p.n_full = n_full_blocks; p.seq_len = seq_len; p.block_table = block_table;
+    p.bd = bounds();
     p.sel = sel; p.stage_idx = (long long *)stage_idx; p.stage_slots = stage_slots;
     p.Hkv = dims->n_kv_heads; p.max_blocks = dims->max_blocks; p.k = k; p.n_q_tokens = n_q_tokens;
     int sort_len = 2;

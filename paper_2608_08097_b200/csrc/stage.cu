@@ -21,13 +21,14 @@ constexpr int kStageDefaultCtas = 128;
 
 __global__ void __launch_bounds__(kStageWarps * 32)
 stage_blocks_kernel(const uint8_t *__restrict__ host_kv, const long long *__restrict__ idx,
-                    const int32_t *__restrict__ slots, int n, uint8_t *__restrict__ pool)
+                    const int32_t *__restrict__ slots, int n, uint8_t *__restrict__ pool, const Bounds bd)
 {
     const int lane = threadIdx.x & 31;
     const int warps_total = gridDim.x * kStageWarps;
     for (int i = blockIdx.x * kStageWarps + (threadIdx.x >> 5); i < n; i += warps_total) {
         const long long src_entry = idx[i];
         if (src_entry < 0) continue;
+        if (!in_range(src_entry, bd.n_entries, bd, kErrHostEntry) || !in_range(slots[i], bd.n_slots, bd, kErrSlot)) continue;
         const uint8_t *src = host_kv + src_entry * (long long)kEntryBytes + lane * 16;
         uint8_t *dst = pool + (long long)slots[i] * kEntryBytes + lane * 16;
         uint4 v[16];
@@ -49,7 +50,7 @@ struct StageLayers {
 };
 
 __global__ void __launch_bounds__(kStageWarps * 32)
-stage_blocks_layers_kernel(const __grid_constant__ StageLayers ly, int n)
+stage_blocks_layers_kernel(const __grid_constant__ StageLayers ly, int n, const Bounds bd)
 {
     const int l = blockIdx.y;
     const uint8_t *host_kv = ly.host_kv[l];
@@ -61,6 +62,7 @@ stage_blocks_layers_kernel(const __grid_constant__ StageLayers ly, int n)
     for (int i = blockIdx.x * kStageWarps + (threadIdx.x >> 5); i < n; i += warps_total) {
         const long long src_entry = idx[i];
         if (src_entry < 0) continue;
+        if (!in_range(src_entry, bd.n_entries, bd, kErrHostEntry) || !in_range(slots[i], bd.n_slots, bd, kErrSlot)) continue;
         const uint8_t *src = host_kv + src_entry * (long long)kEntryBytes + lane * 16;
         uint8_t *dst = pool + (long long)slots[i] * kEntryBytes + lane * 16;
         uint4 v[16];
@@ -102,7 +104,7 @@ extern "C" int oasis_stage_blocks_layers(int32_t n_layers, const void *const *ho
     int grid = (n + kStageWarps - 1) / kStageWarps;
     if (grid > max_ctas) grid = max_ctas;
     prefer_max_shared_carveout(stage_blocks_layers_kernel);
-    stage_blocks_layers_kernel<<<dim3((unsigned)grid, (unsigned)n_layers), kStageWarps * 32, 0, (cudaStream_t)stream>>>(ly, n);
+    stage_blocks_layers_kernel<<<dim3((unsigned)grid, (unsigned)n_layers), kStageWarps * 32, 0, (cudaStream_t)stream>>>(ly, n, bounds());
     return check_launch(who);
 }
 
@@ -121,6 +123,6 @@ extern "C" int oasis_stage_blocks(const void *host_kv, const int64_t *idx, const
     if (grid > max_ctas) grid = max_ctas;
     prefer_max_shared_carveout(stage_blocks_kernel);
     stage_blocks_kernel<<<grid, kStageWarps * 32, 0, (cudaStream_t)stream>>>(
-        (const uint8_t *)host_kv, (const long long *)idx, slots, n, (uint8_t *)hbm_pool);
+        (const uint8_t *)host_kv, (const long long *)idx, slots, n, (uint8_t *)hbm_pool, bounds());
     return check_launch("oasis_stage_blocks");
 }

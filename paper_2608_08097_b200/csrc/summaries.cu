@@ -28,7 +28,7 @@ __device__ __forceinline__ uint32_t max2(uint32_t a, uint32_t b)
 __device__ __forceinline__ void
 summarise_item(const uint8_t *__restrict__ kv_pool, const int32_t *__restrict__ block_table,
                const int32_t *__restrict__ first_block, const int32_t *__restrict__ n_blocks,
-               uint8_t *__restrict__ summaries, int Hkv, int max_blocks, int max_new, long long n_items)
+               uint8_t *__restrict__ summaries, int Hkv, int max_blocks, int max_new, long long n_items, const Bounds &bd)
 {
     const int lane = threadIdx.x & 31;
     const long long item = (long long)blockIdx.x * kSummWarps + (threadIdx.x >> 5);
@@ -38,8 +38,12 @@ summarise_item(const uint8_t *__restrict__ kv_pool, const int32_t *__restrict__ 
     const int b = (int)(item / ((long long)Hkv * max_new));
     if (jj >= n_blocks[b]) return;
     const int j = first_block[b] + jj;
-    if (j < 0 || j >= max_blocks) return;
+    if (j < 0 || j >= max_blocks) {
+        in_range(j, max_blocks, bd, kErrBlockCount);       // (checked build: reported; always skipped)
+        return;
+    }
     const long long phys = block_table[(long long)b * max_blocks + j];
+    if (!in_range(phys * Hkv + h, bd.n_entries, bd, kErrHostEntry)) return;
     const uint8_t *src = kv_pool + (phys * Hkv + h) * (long long)kEntryBytes;
 
     // lane -> 16-byte chunk (lane & 15) of token (lane >> 4) + 2*i
@@ -77,9 +81,9 @@ __global__ void __launch_bounds__(kSummWarps * 32)
 build_summaries_kernel(const uint8_t *__restrict__ kv_pool, const int32_t *__restrict__ block_table,
                        const int32_t *__restrict__ first_block, const int32_t *__restrict__ n_blocks,
                        uint8_t *__restrict__ summaries, int B, int Hkv, int max_blocks,
-                       int max_new, long long n_items)
+                       int max_new, long long n_items, const Bounds bd)
 {
-    summarise_item(kv_pool, block_table, first_block, n_blocks, summaries, Hkv, max_blocks, max_new, n_items);
+    summarise_item(kv_pool, block_table, first_block, n_blocks, summaries, Hkv, max_blocks, max_new, n_items, bd);
 }
 
 // The same for several layers in one launch (blockIdx.y = layer): a decode step appends to every layer's cache
@@ -92,11 +96,12 @@ struct SummLayers {
 
 __global__ void __launch_bounds__(kSummWarps * 32)
 build_summaries_layers_kernel(const __grid_constant__ SummLayers ly, const int32_t *__restrict__ first_block,
-                              const int32_t *__restrict__ n_blocks, int Hkv, int max_blocks, int max_new, long long n_items)
+                              const int32_t *__restrict__ n_blocks, int Hkv, int max_blocks, int max_new, long long n_items,
+                              const Bounds bd)
 {
     const int l = blockIdx.y;
     summarise_item(ly.kv_pool[l], ly.block_table[l], first_block, n_blocks, ly.summaries[l], Hkv, max_blocks, max_new,
-                   n_items);
+                   n_items, bd);
 }
 
 }  // namespace oasis
@@ -122,7 +127,7 @@ extern "C" int oasis_build_summaries(const oasis_dims_t *dims, const void *kv_po
     prefer_max_shared_carveout(build_summaries_kernel);
     build_summaries_kernel<<<(unsigned)grid, kSummWarps * 32, 0, (cudaStream_t)stream>>>(
         (const uint8_t *)kv_pool, block_table, first_block, n_blocks, (uint8_t *)summaries,
-        dims->batch, dims->n_kv_heads, dims->max_blocks, max_new_blocks, n_items);
+        dims->batch, dims->n_kv_heads, dims->max_blocks, max_new_blocks, n_items, bounds());
     return check_launch("oasis_build_summaries");
 }
 
@@ -156,6 +161,6 @@ extern "C" int oasis_build_summaries_layers(const oasis_dims_t *dims, int32_t n_
     if (grid > 0x7fffffffLL) return fail(OASIS_ERR_UNSUPPORTED, "%s: too many blocks", who);
     prefer_max_shared_carveout(build_summaries_layers_kernel);
     build_summaries_layers_kernel<<<dim3((unsigned)grid, (unsigned)n_layers), kSummWarps * 32, 0, (cudaStream_t)stream>>>(
-        ly, first_block, n_blocks, dims->n_kv_heads, dims->max_blocks, max_new_blocks, n_items);
+        ly, first_block, n_blocks, dims->n_kv_heads, dims->max_blocks, max_new_blocks, n_items, bounds());
     return check_launch(who);
 }
