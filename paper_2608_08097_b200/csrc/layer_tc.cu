@@ -551,100 +551,10 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             if (!alive) break;
             tc_fence_after();
             const uint32_t s_tmem = tmem_base + lane_base + (uint32_t)((i % kAtSBufs) * kAtTileKeys);
-            if (live_warp) {
-                int nvis[BPC];                                      // visible keys of each of this copy's blocks
-                bool masked = false;
-#pragma unroll
-                for (int c = 0; c < BPC; ++c) {
-                    const int blk = tile_blk[s * kAtTileCols + copy * BPC + c];
-                    int n = blk < 0 ? 0 : limit - blk * kBlock + 1;
-                    n = max(0, min(n, kBlock));
-                    nvis[c] = n;
-                    masked |= has_row && n < kBlock;         // lanes without an MMA row are zeroed below instead
-                }
-                masked = __any_sync(0xffffffffu, masked);
-                float x[KPC];
-                {
-                    uint32_t v[BPC][16];
-#pragma unroll
-                    for (int c = 0; c < BPC; ++c) tc_ld16_nowait(s_tmem + (copy * BPC + c) * 16, v[c]);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int c = 0; c < BPC; ++c)
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) x[c * 16 + e] = __uint_as_float(v[c][e]);
-                }
-                if (masked) {
-#pragma unroll
-                    for (int c = 0; c < BPC; ++c)
-#pragma unroll
-                        for (int e = 0; e < 16; ++e)
-                            if (e >= nvis[c]) x[c * 16 + e] = -CUDART_INF_F;
-                }
-                float mx4[4] = {x[0], x[1], x[2], x[3]};
-#pragma unroll
-                for (int e = 4; e < KPC; e += 4) {
-                    mx4[0] = fmaxf(mx4[0], x[e]); mx4[1] = fmaxf(mx4[1], x[e + 1]);
-                    mx4[2] = fmaxf(mx4[2], x[e + 2]); mx4[3] = fmaxf(mx4[3], x[e + 3]);
-                }
-                // a lane without an MMA row read whatever its tensor-memory lane held: it must not raise the reference
-                const float mx = has_row ? fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) : -CUDART_INF_F;
-                const float mxs = mx * p.scale_log2;
-                const bool raise = mxs > m_ref + 8.0f;
-                if (__any_sync(0xffffffffu, raise)) {
-                    // the O rows must be complete up to tile i-1 before they are rescaled
-                    // (its stage is released by the commit that follows that P V; with at least four stages in the
-                    // ring the phase parity of that barrier is unambiguous)
-                    if (it > 0) alive = mbar_wait(bar_empty(s_prev), ph_prev, p.err, 62);
-                    tc_fence_after();
-                    const float m_new = raise ? mxs : m_ref;
-                    const float alpha = m_new == -CUDART_INF_F ? 1.f : fast_exp2(m_ref - m_new);
-                    m_ref = m_new;
-                    l_sum *= alpha;
-                    if (it > 0) {
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) {
-                            uint32_t v[16];
-                            tc_ld16(tmem_o + lane_base + c * 16, v);
-#pragma unroll
-                            for (int e = 0; e < 16; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
-                            tc_st16(tmem_o + lane_base + c * 16, v);
-                        }
-                        tc_wait_st();
-                    }
-                }
-                const float neg_m = m_ref == -CUDART_INF_F ? 0.f : -m_ref;
-                float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-                // P of the whole tile is 32 packed columns; this copy owns columns [copy*KPC/2, +KPC/2), the rest is 0
-                uint32_t pk[KPC / 2];
-#pragma unroll
-                for (int e = 0; e < KPC / 2; ++e) {
-                    const float p0 = fast_exp2(fmaf(x[2 * e], p.scale_log2, neg_m));
-                    const float p1 = fast_exp2(fmaf(x[2 * e + 1], p.scale_log2, neg_m));
-                    sum4[e & 3] += p0 + p1;
-                    pk[e] = pack_p(p0, p1);
-                }
-                l_sum += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-                if (!has_row) {
-#pragma unroll
-                    for (int e = 0; e < KPC / 2; ++e) pk[e] = 0u;   // and it stores P = 0
-                }
-#pragma unroll
-                for (int g8 = 0; g8 < 4; ++g8) {                    // four groups of 8 packed columns = four blocks
-                    uint32_t w8[8];
-                    const int own = g8 - copy * BPC;                // index among this copy's blocks, if in [0, BPC)
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        uint32_t val = 0u;
-#pragma unroll
-                        for (int c = 0; c < BPC; ++c)
-                            if (own == c) val = pk[c * 8 + e];
-                        w8[e] = val;
-                    }
-                    tc_st8(s_tmem + g8 * 8, w8);
-                }
-                tc_wait_st();
-            }
+            if (live_warp)
+                alive = softmax_tile<COPIES>(s_tmem, tmem_o + lane_base, tile_blk + s * kAtTileCols, copy, limit, has_row,
+                                             p.scale_log2, m_ref, l_sum, it > 0,
+                                             [&] { return mbar_wait(bar_empty(s_prev), ph_prev, p.err, 62); });
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_p_full(i % kAtSBufs));

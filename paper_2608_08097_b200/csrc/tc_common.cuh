@@ -3,6 +3,7 @@
 // descriptors, and the host-side tensor-map encoder lookup.
 #pragma once
 #include <cuda.h>
+#include <math_constants.h>
 
 #include "common.cuh"
 
@@ -225,6 +226,164 @@ __device__ __forceinline__ bool softmax_warps_all(bool pred)
         "selp.u32 %0, 1, 0, q;\n\t}"
         : "=r"(r) : "r"((uint32_t)pred) : "memory");
     return r != 0;
+}
+
+// ---- packed fp32 arithmetic (two lanes per instruction) and the three-input maximum of sm_100 ------------------
+__device__ __forceinline__ uint64_t f32x2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f32x2_split(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// ---- one 64-key tile of the online softmax, shared by the attention kernel and the fused layer kernel --------
+// The calling thread owns one MMA row (one tensor-memory lane).  It reads its row of S = Q K^T for the blocks of
+// its copy, masks positions past `limit` (only tiles that hold a block of the local window need it), raises the
+// reference maximum lazily -- only when a logit exceeds it by 2^8; the O row in tensor memory is then rescaled,
+// after `wait_prev()` has made sure that the previous tile's P V has completed -- and writes P = 2^(s - m_ref),
+// rounded to bf16, back over S; the columns of the other copies' blocks get P = 0.  Running maximum and sum stay
+// in the thread's registers; there is no cross-thread reduction.
+//   s_tmem      tensor-memory address of the tile's S buffer at this thread's lane
+//   o_tmem      tensor-memory address of the O rows at this thread's lane
+//   tile_blk    the four block ids of the tile (shared memory), -1 = missing
+//   copy        which copy of the query rows this thread belongs to (0 when COPIES == 1)
+//   have_o      O already holds earlier tiles of this row (else there is nothing to rescale)
+// Returns false if wait_prev() gave up.
+template <int COPIES, class WaitPrev>
+__device__ __forceinline__ bool softmax_tile(const uint32_t s_tmem, const uint32_t o_tmem, const int32_t *tile_blk, const int copy_in,
+                                             const int limit, const bool has_row, const float scale_log2, float &m_ref, float &l_sum,
+                                             const bool have_o, WaitPrev &&wait_prev)
+{
+    constexpr int BPC = kAtTileCols / COPIES;               // blocks of a tile each copy handles
+    constexpr int KPC = BPC * kBlock;                       // keys of a tile each copy handles
+    const int copy = COPIES == 1 ? 0 : copy_in;
+    bool alive = true;
+    int nvis[BPC];                                          // visible keys of each of this copy's blocks
+    bool masked = false;
+#pragma unroll
+    for (int c = 0; c < BPC; ++c) {
+        const int blk = tile_blk[copy * BPC + c];
+        int n = blk < 0 ? 0 : limit - blk * kBlock + 1;
+        n = max(0, min(n, kBlock));
+        nvis[c] = n;
+        masked |= has_row && n < kBlock;                    // lanes without an MMA row are zeroed below instead
+    }
+    masked = __any_sync(0xffffffffu, masked);
+    float x[KPC];
+    {
+        uint32_t v[BPC][16];
+#pragma unroll
+        for (int c = 0; c < BPC; ++c) tc_ld16_nowait(s_tmem + (copy * BPC + c) * 16, v[c]);
+        tc_wait_ld();
+#pragma unroll
+        for (int c = 0; c < BPC; ++c)
+#pragma unroll
+            for (int e = 0; e < 16; ++e) x[c * 16 + e] = __uint_as_float(v[c][e]);
+    }
+    if (masked) {
+#pragma unroll
+        for (int c = 0; c < BPC; ++c)
+#pragma unroll
+            for (int e = 0; e < 16; ++e)
+                if (e >= nvis[c]) x[c * 16 + e] = -CUDART_INF_F;
+    }
+    float mx4[4] = {x[0], x[1], x[2], x[3]};
+#pragma unroll
+    for (int e = 4; e < KPC; e += 8) {                      // three-input maxima: two elements per instruction
+        mx4[0] = max3(mx4[0], x[e], x[e + 4]);
+        mx4[1] = max3(mx4[1], x[e + 1], x[e + 5]);
+        mx4[2] = max3(mx4[2], x[e + 2], x[e + 6]);
+        mx4[3] = max3(mx4[3], x[e + 3], x[e + 7]);
+    }
+    // a lane without an MMA row read whatever its tensor-memory lane held: it must not raise the reference
+    const float mx = has_row ? fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) : -CUDART_INF_F;
+    const float mxs = mx * scale_log2;
+    const bool raise = mxs > m_ref + 8.0f;
+    if (__any_sync(0xffffffffu, raise)) {
+        // the O rows must be complete up to the previous tile before they are rescaled
+        if (have_o) alive = wait_prev();
+        tc_fence_after();
+        const float m_new = raise ? mxs : m_ref;
+        const float alpha = m_new == -CUDART_INF_F ? 1.f : fast_exp2(m_ref - m_new);
+        m_ref = m_new;
+        l_sum *= alpha;
+        if (have_o) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                uint32_t v[16];
+                tc_ld16(o_tmem + c * 16, v);
+#pragma unroll
+                for (int e = 0; e < 16; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
+                tc_st16(o_tmem + c * 16, v);
+            }
+            tc_wait_st();
+        }
+    }
+    const float neg_m = m_ref == -CUDART_INF_F ? 0.f : -m_ref;
+    const uint64_t scale2 = f32x2(scale_log2, scale_log2), neg_m2 = f32x2(neg_m, neg_m);
+    uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};            // eight partial sums, two per packed accumulator
+    // P of the whole tile is 32 packed columns; this copy owns columns [copy*KPC/2, +KPC/2), the rest is 0
+    uint32_t pk[KPC / 2];
+#pragma unroll
+    for (int e = 0; e < KPC / 2; ++e) {
+        float t0, t1;
+        f32x2_split(fma_f32x2(f32x2(x[2 * e], x[2 * e + 1]), scale2, neg_m2), t0, t1);
+        const float p0 = fast_exp2(t0), p1 = fast_exp2(t1);
+        sum2[e & 3] = add_f32x2(sum2[e & 3], f32x2(p0, p1));
+        pk[e] = pack_p(p0, p1);
+    }
+    {
+        float lo, hi;
+        f32x2_split(add_f32x2(add_f32x2(sum2[0], sum2[1]), add_f32x2(sum2[2], sum2[3])), lo, hi);
+        l_sum += lo + hi;
+    }
+    if (!has_row) {
+#pragma unroll
+        for (int e = 0; e < KPC / 2; ++e) pk[e] = 0u;       // and it stores P = 0
+    }
+#pragma unroll
+    for (int g8 = 0; g8 < 4; ++g8) {                        // four groups of 8 packed columns = four blocks
+        uint32_t w8[8];
+        if (COPIES == 1) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) w8[e] = pk[g8 * 8 + e];
+        } else {
+            const int own = g8 - copy * BPC;                // index among this copy's blocks, if in [0, BPC)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                uint32_t val = 0u;
+#pragma unroll
+                for (int c = 0; c < BPC; ++c)
+                    if (own == c) val = pk[c * 8 + e];
+                w8[e] = val;
+            }
+        }
+        tc_st8(s_tmem + g8 * 8, w8);
+    }
+    tc_wait_st();
+    return alive;
 }
 
 }  // namespace oasis
