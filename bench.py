@@ -479,7 +479,7 @@ def algorithmic_bytes(cfg, k, T, seq_steps, steps):
     return score / len(steps), attn / len(steps)
 
 
-def cpu_leg(bench, w, cfg, sel_gpu, s_sel, budget_s=20.0, mass_requests=2):
+def cpu_leg(bench, w, cfg, sel_gpu, s_sel, budget_s=12.0, mass_requests=2):
     """What runs on the host cores: (1) the oracle, as it stands, on one layer of one step, request by request
     (score + top-k + gather + attention), until about `budget_s` seconds are spent; (2) the secondary recall: the
     GPU's lookahead selection of step `s_sel` (layer 0) against the top-K blocks by the attention mass that the true
@@ -491,26 +491,30 @@ def cpu_leg(bench, w, cfg, sel_gpu, s_sel, budget_s=20.0, mass_requests=2):
     kv = synth.u16(lay.host_kv)
     table = lay.block_table.numpy()
     scale = np.float32(1.0 / math.sqrt(128.0))
-    done, t_used = 0, 0.0
-    for b in range(cfg.batch):
-        tb = table[b:b + 1]
-        n_full = lay.n_full.numpy()[b:b + 1]
-        seq = lay.seq_len.numpy()[b:b + 1]
-        q = synth.u16(lay.q[b:b + 1, :w.T].contiguous())
-        summ = oracle.build_summaries(kv, tb, np.zeros(1, np.int32), n_full)          # set-up, not timed
-        t0 = time.perf_counter()
-        s32, _ = oracle.score_blocks(q[:, 1:], summ, n_full)
-        sel, idx, slots = oracle.select_topk(s32, n_full, seq, w.T, w.k, tb)
-        pool = np.zeros((cfg.n_kv_heads * (w.k + 2), 2, 16, 128), np.uint16)
-        oracle.stage_blocks(kv.reshape(-1, 2, 16, 128), idx, slots, pool)
-        oracle.sparse_attn(q, pool, slots.reshape(1, cfg.n_kv_heads, -1), sel, seq, scale, cfg.n_kv_heads)
-        t_used += time.perf_counter() - t0
-        done += 1
+    done, t_used, steps_used = 0, 0.0, 0
+    for s in range(min(lay.seq_len_steps.shape[0], 16)):           # step by step, request by request, until the budget is spent
+        for b in range(cfg.batch):
+            tb = table[b:b + 1]
+            n_full = lay.n_full_steps[s].numpy()[b:b + 1]
+            seq = lay.seq_len_steps[s].numpy()[b:b + 1]
+            q = synth.u16(lay.q_steps[s][b:b + 1, :w.T].contiguous())
+            summ = oracle.build_summaries(kv, tb, np.zeros(1, np.int32), n_full)          # set-up, not timed
+            t0 = time.perf_counter()
+            s32, _ = oracle.score_blocks(q[:, 1:], summ, n_full)
+            sel, idx, slots = oracle.select_topk(s32, n_full, seq, w.T, w.k, tb)
+            pool = np.zeros((cfg.n_kv_heads * (w.k + 2), 2, 16, 128), np.uint16)
+            oracle.stage_blocks(kv.reshape(-1, 2, 16, 128), idx, slots, pool)
+            oracle.sparse_attn(q, pool, slots.reshape(1, cfg.n_kv_heads, -1), sel, seq, scale, cfg.n_kv_heads)
+            t_used += time.perf_counter() - t0
+            done += 1
+            if t_used >= budget_s:
+                break
+        steps_used = s + 1
         if t_used >= budget_s:
             break
     base = {"value": done / t_used, "unit": UNIT, "cores": 1, "host_cores": os.cpu_count(), "kind": "oracle",
-            "sample": "layer 0, step 0, %d of %d requests, score+top-k+gather+attention, single thread (%.1f s)"
-                      % (done, cfg.batch, t_used)}
+            "sample": "layer 0, %d (request, step) units of steps 0..%d (batch %d), score+top-k+gather+attention each, single "
+                      "thread (%.1f s)" % (done, steps_used - 1, cfg.batch, t_used)}
     # secondary recall (attention mass): the true queries of steps s+1.. sit at positions L_s + 1 + t
     recall_mass = None
     if sel_gpu is not None:

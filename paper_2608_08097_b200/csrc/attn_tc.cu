@@ -129,15 +129,7 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
         tmem_o = tmem_base + kAtSBufs * kAtTileKeys;
         tmem_q = tmem_o + kHeadDim;                                  // Q as the A operand: 128 rows x 64 packed columns
         if (warp >= 3) {
-            const uint32_t q_lane = tmem_q + ((uint32_t)((warp & 3) * 32) << 16);
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const uint32_t w[16] = {v[4 * c].x, v[4 * c].y, v[4 * c].z, v[4 * c].w, v[4 * c + 1].x, v[4 * c + 1].y,
-                                        v[4 * c + 1].z, v[4 * c + 1].w, v[4 * c + 2].x, v[4 * c + 2].y, v[4 * c + 2].z,
-                                        v[4 * c + 2].w, v[4 * c + 3].x, v[4 * c + 3].y, v[4 * c + 3].z, v[4 * c + 3].w};
-                tc_st16(q_lane + c * 16, w);
-            }
-            tc_wait_st();
+            q_row_to_tmem(tmem_q + ((uint32_t)((warp & 3) * 32) << 16), v);
         }
         tc_fence_before();
         asm volatile("bar.sync 2, %0;" ::"n"(kAtThreads - 32) : "memory");
@@ -171,29 +163,13 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
             if (lane == 0) alive = mbar_wait(bar_empty(s), ph, p.err, 41);
             alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
             if (!alive) break;
-            const unsigned valid = __ballot_sync(0xffffffffu, lane < kAtTileCols && blk >= 0);
-            if (lane < kAtTileCols) {
-                tile_blk[s * kAtTileCols + lane] = blk;
-                if (blk < 0) {
-                    // a missing block contributes P = 0, which must not meet stale NaN bit patterns in V
-                    uint8_t *img = base_ptr + kAtQBytes + (size_t)s * kAtStageBytes + lane * kEntryBytes;
-                    for (int u = 0; u < 4; ++u)                      // (row group, dim half) units of the V part
-                        for (int j = 0; j < kImgPart / 16; ++j)
-                            *reinterpret_cast<uint4 *>(img + (u >> 1) * kImgGroup + (u & 1) * kImgHalf + kImgPart + j * 16) =
-                                make_uint4(0, 0, 0, 0);
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive_expect_tx(bar_full(s), (uint32_t)__popc(valid) * kEntryBytes);
-            __syncwarp();
-            if (lane < kAtTileCols && blk >= 0)                       // the whole 8 KiB entry in one copy
-                tma_load_5d(kv_u32 + s * kAtStageBytes + lane * kEntryBytes, &tmap, 0, 0, 2 * slot, 0, 0, bar_full(s));
+            stage_attn_tile(lane, blk, slot, tile_blk + s * kAtTileCols, base_ptr + kAtQBytes + (size_t)s * kAtStageBytes,
+                            kv_u32 + s * kAtStageBytes, &tmap, bar_full(s));
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- Q K^T issuer
         if (lane == 0) {
-            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAtTileKeys >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
+            const uint32_t idesc = idesc_qk(MMA_M);
             // descriptors: the operand start address occupies the low 14 bits (16-byte units), so offsets are added there
             const uint64_t k_desc0 = smem_desc_sw128_k(kv_u32, kImgGroup);
             bool alive = true;
@@ -211,12 +187,7 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
                 tc_fence_after();
                 const uint64_t k_desc = k_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
                 const uint32_t d_tmem = tmem_base + (uint32_t)(sb * kAtTileKeys);
-#pragma unroll
-                for (int kc = 0; kc < 2; ++kc)
-#pragma unroll
-                    for (int k4 = 0; k4 < 4; ++k4)
-                        tc_mma_bf16_ts(d_tmem, tmem_q + (kc * 4 + k4) * 8, k_desc + (uint64_t)((kc * kImgHalf + k4 * 32) >> 4),
-                                       idesc_qk, (kc | k4) ? 1u : 0u);
+                issue_qk_tile(d_tmem, tmem_q, k_desc, idesc);
                 tc_commit(bar_s_full(sb));
                 ph ^= (s + 1 == p.stages);
                 s = (s + 1 == p.stages) ? 0 : s + 1;
@@ -226,7 +197,7 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
     } else if (warp == 2) {
         // ---------------------------------------------------------------- P V issuer
         if (lane == 0) {
-            const uint32_t idesc_pv = (1u << 4) | kIdescPvFormats | (1u << 16) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
+            const uint32_t idesc = idesc_pv(MMA_M);
             const uint64_t v_desc0 = smem_desc_sw128_mn(kv_u32 + kImgPart, kImgHalf, kImgGroup);
             bool alive = true;
             int s = 0, sb = 0;
@@ -237,10 +208,7 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
                 tc_fence_after();
                 const uint64_t v_desc = v_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
                 const uint32_t p_tmem = tmem_base + (uint32_t)(sb * kAtTileKeys);
-#pragma unroll
-                for (int ks = 0; ks < kAtTileCols; ++ks)               // 16 keys per MMA = one block image
-                    tc_mma_bf16_ts(tmem_o, p_tmem + ks * 8, v_desc + (uint64_t)((ks * kEntryBytes) >> 4), idesc_pv,
-                                   (i | ks) ? 1u : 0u);
+                issue_pv_tile(tmem_o, p_tmem, v_desc, idesc, i == 0);
                 tc_commit(bar_empty(s));                             // stage free, and O complete up to this tile
                 s = (s + 1 == p.stages) ? 0 : s + 1;
                 sb = (sb + 1) & (kAtSBufs - 1);

@@ -161,46 +161,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     // lives in sub-tile k / 64.  `nthr` threads (index `me`) share the work; loads are issued
     // eight at a time so their latencies overlap.
     auto build_b = [&](int bh, int buf, int me, int nthr) {
-        const int b = (int)(bh / p.Hkv), h = (int)(bh % p.Hkv);
-        uint8_t *dstb = b_ptr + (size_t)buf * b_bytes;
-        const int tasks = p.N * 16;                              // 16-byte chunks of the query rows
-#pragma unroll 1
-        for (int i0 = me; i0 < tasks; i0 += nthr * 8) {
-            uint4 v[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int i = i0 + nthr * u;
-                v[u] = make_uint4(0, 0, 0, 0);
-                const int n = i >> 4, c = i & 15;
-                if (i < tasks && (n < p.Rs || !p.reduce_sum)) {
-                    const int r = n % p.Rs;
-                    const int tq = r / p.G, a = h * p.G + r % p.G;
-                    v[u] = *reinterpret_cast<const uint4 *>(
-                        p.q_draft + ((long long)b * p.q_batch_stride + ((long long)tq * p.Hq + a) * kHeadDim) * 2 + c * 16);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int i = i0 + nthr * u;
-                if (i >= tasks) continue;
-                const int n = i >> 4, c = i & 15;
-                const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f);
-                uint4 neg, pos;
-                const __nv_bfloat162 *f = reinterpret_cast<const __nv_bfloat162 *>(&v[u]);
-                __nv_bfloat162 *n2 = reinterpret_cast<__nv_bfloat162 *>(&neg);
-                __nv_bfloat162 *p2 = reinterpret_cast<__nv_bfloat162 *>(&pos);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    n2[e] = __hmin2(f[e], zero2);
-                    p2[e] = __hmax2(f[e], zero2);
-                }
-                const int sub = c >> 3, ch = (c & 7) ^ (n & 7);
-                uint8_t *row = dstb + n * 128 + ch * 16;
-                *reinterpret_cast<uint4 *>(row + (size_t)sub * p.N * 128) = neg;          // k in [0, 128): min rows
-                *reinterpret_cast<uint4 *>(row + (size_t)(2 + sub) * p.N * 128) = pos;    // k in [128, 256): max rows
-            }
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        build_qpm_operand(b_ptr + (size_t)buf * b_bytes, p.q_draft, p.q_batch_stride, bh / p.Hkv, bh % p.Hkv, p.Rs, p.G, p.Hq, p.N,
+                          p.reduce_sum, me, nthr);
     };
 
     // The next launch on the stream may start as soon as an SM has room for one of its thread blocks (its scoring
@@ -248,9 +210,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                     if (alive) {
                         mbar_arrive_expect_tx(sbar_full(s), kLyATileBytes);
                         const int y = bh * p.max_blocks + j0;
-    #pragma unroll
-                        for (int kc = 0; kc < 4; ++kc)
-                            tma_load_2d(kv_u32 + s * kLyATileBytes + kc * kLySubTileBytes, &tmap_summ, kc * 64, y, sbar_full(s));
+                        load_score_tile(kv_u32 + s * kLyATileBytes, &tmap_summ, y, kLySubTileBytes, sbar_full(s));
                     }
                 }
                 alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
@@ -299,34 +259,15 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             if (lane == 0) alive = alive && mbar_wait(bar_empty(s), ph, p.err, 41);
             alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
             if (!alive) break;
-            const unsigned valid = __ballot_sync(0xffffffffu, lane < kAtTileCols && blk >= 0);
-            if (lane < kAtTileCols) {
-                tile_blk[s * kAtTileCols + lane] = blk;
-                if (blk < 0) {
-                    // a missing block contributes P = 0, which must not meet stale NaN bit patterns in V
-                    uint8_t *img = base_ptr + kAtQBytes + (size_t)s * kAtStageBytes + lane * kEntryBytes;
-#pragma unroll 1
-                    for (int u = 0; u < 4; ++u)                      // (row group, dim half) units of the V part
-#pragma unroll 1
-                        for (int j = 0; j < kImgPart / 16; ++j)
-                            *reinterpret_cast<uint4 *>(img + (u >> 1) * kImgGroup + (u & 1) * kImgHalf + kImgPart + j * 16) =
-                                make_uint4(0, 0, 0, 0);
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive_expect_tx(bar_full(s), (uint32_t)__popc(valid) * kEntryBytes);
-            __syncwarp();
-            if (lane < kAtTileCols && blk >= 0)                       // the whole 8 KiB entry in one copy
-                tma_load_5d(kv_u32 + s * kAtStageBytes + lane * kEntryBytes, &tmap, 0, 0, 2 * slot, 0, 0, bar_full(s));
+            stage_attn_tile(lane, blk, slot, tile_blk + s * kAtTileCols, base_ptr + kAtQBytes + (size_t)s * kAtStageBytes,
+                            kv_u32 + s * kAtStageBytes, &tmap, bar_full(s));
         }
         }
     } else if (warp == 1) {
         {
             // ---------------------------------------------------------------- scoring phase: MMAs
             if (lane == 0) {
-                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.N >> 3) << 17) |
-                                       ((uint32_t)(kLyTileBlocks >> 4) << 24);
+                const uint32_t idesc = idesc_score(p.N, kLyTileBlocks);
                 int it = 0, bo = -1;
                 int cur_bh = -1;
                 bool alive = true;
@@ -351,15 +292,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                     const uint32_t d_tmem = tmem_base + (uint32_t)p.acc_col + (uint32_t)(acc * p.N);
                     const uint32_t a_tile = kv_u32 + s * kLyATileBytes;
                     const uint32_t b_tile = b_u32 + (bo % 2) * b_bytes;
-    #pragma unroll
-                    for (int kc = 0; kc < 4; ++kc) {
-    #pragma unroll
-                        for (int k4 = 0; k4 < 4; ++k4) {
-                            const uint64_t ad = smem_desc_sw128(a_tile + kc * kLySubTileBytes + k4 * 32);
-                            const uint64_t bd = smem_desc_sw128(b_tile + kc * p.N * 128 + k4 * 32);
-                            tc_mma_bf16(d_tmem, ad, bd, idesc, (kc | k4) ? 1u : 0u);
-                        }
-                    }
+                    issue_score_tile(d_tmem, a_tile, b_tile, p.N, kLySubTileBytes, idesc);
                     tc_commit(sbar_empty(s));         // the stage may be refilled once these MMAs have read it
                     tc_commit(bar_acc_full(acc));    // the accumulator is complete
                     ++it;
@@ -368,7 +301,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         }
         // ---------------------------------------------------------------- Q K^T issuer
         if (lane == 0) {
-            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAtTileKeys >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
+            const uint32_t idesc = idesc_qk(MMA_M);
             // descriptors: the operand start address occupies the low 14 bits (16-byte units), so offsets are added there
             const uint64_t k_desc0 = smem_desc_sw128_k(kv_u32, kImgGroup);
             bool alive = true;
@@ -393,12 +326,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 tc_fence_after();
                 const uint64_t k_desc = k_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
                 const uint32_t d_tmem = tmem_base + (uint32_t)(sb * kAtTileKeys);
-#pragma unroll
-                for (int kc = 0; kc < 2; ++kc)
-#pragma unroll
-                    for (int k4 = 0; k4 < 4; ++k4)
-                        tc_mma_bf16_ts(d_tmem, tmem_q + (kc * 4 + k4) * 8, k_desc + (uint64_t)((kc * kImgHalf + k4 * 32) >> 4),
-                                       idesc_qk, (kc | k4) ? 1u : 0u);
+                issue_qk_tile(d_tmem, tmem_q, k_desc, idesc);
                 tc_commit(bar_s_full(sb));
                 ph ^= (s + 1 == kLyStages);
                 s = (s + 1 == kLyStages) ? 0 : s + 1;
@@ -409,7 +337,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     } else if (warp == 2) {
         // ---------------------------------------------------------------- P V issuer
         if (lane == 0) {
-            const uint32_t idesc_pv = (1u << 4) | kIdescPvFormats | (1u << 16) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(MMA_M >> 4) << 24);
+            const uint32_t idesc = idesc_pv(MMA_M);
             const uint64_t v_desc0 = smem_desc_sw128_mn(kv_u32 + kImgPart, kImgHalf, kImgGroup);
             bool alive = true;
             int s = 0, sb = 0;
@@ -424,10 +352,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 tc_fence_after();
                 const uint64_t v_desc = v_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
                 const uint32_t p_tmem = tmem_base + (uint32_t)(sb * kAtTileKeys);
-#pragma unroll
-                for (int ks = 0; ks < kAtTileCols; ++ks)               // 16 keys per MMA = one block image
-                    tc_mma_bf16_ts(tmem_o, p_tmem + ks * 8, v_desc + (uint64_t)((ks * kEntryBytes) >> 4), idesc_pv,
-                                   (it | ks) ? 1u : 0u);             // O starts afresh with every row
+                issue_pv_tile(tmem_o, p_tmem, v_desc, idesc, it == 0);   // O starts afresh with every row
                 tc_commit(bar_empty(s));                             // stage free, and O complete up to this tile
                 s = (s + 1 == kLyStages) ? 0 : s + 1;
                 sb = (sb + 1) & (kAtSBufs - 1);
@@ -487,17 +412,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 if (!alive) break;
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + (uint32_t)p.acc_col + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.N);
-                float res = p.reduce_sum ? 0.f : -CUDART_INF_F;
-#pragma unroll 1
-                for (int c = 0; c < p.N; c += 16) {
-                    uint32_t v[16];
-                    tc_ld16(taddr + c, v);
-    #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const float f = __uint_as_float(v[e]);
-                        res = p.reduce_sum ? res + f : fmaxf(res, f);
-                    }
-                }
+                const float res = reduce_score_row(taddr, p.N, p.reduce_sum);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_acc_empty(acc));
@@ -519,15 +434,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
 #pragma unroll
                 for (int c = 0; c < 16; ++c) v[c] = src[c];
             }
-            const uint32_t q_lane = tmem_q + lane_base;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const uint32_t w[16] = {v[4 * c].x, v[4 * c].y, v[4 * c].z, v[4 * c].w, v[4 * c + 1].x, v[4 * c + 1].y,
-                                        v[4 * c + 1].z, v[4 * c + 1].w, v[4 * c + 2].x, v[4 * c + 2].y, v[4 * c + 2].z,
-                                        v[4 * c + 2].w, v[4 * c + 3].x, v[4 * c + 3].y, v[4 * c + 3].z, v[4 * c + 3].w};
-                tc_st16(q_lane + c * 16, w);
-            }
-            tc_wait_st();
+            q_row_to_tmem(tmem_q + lane_base, v);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_q);

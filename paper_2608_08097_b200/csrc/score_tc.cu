@@ -86,46 +86,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
     // lives in sub-tile k / 64.  `nthr` threads (index `me`) share the work; loads are issued
     // eight at a time so their latencies overlap.
     auto build_b = [&](long long bh, int buf, int me, int nthr) {
-        const int b = (int)(bh / p.Hkv), h = (int)(bh % p.Hkv);
-        uint8_t *dstb = b_ptr + (size_t)buf * b_bytes;
-        const int tasks = p.N * 16;                              // 16-byte chunks of the query rows
-#pragma unroll 1
-        for (int i0 = me; i0 < tasks; i0 += nthr * 8) {
-            uint4 v[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int i = i0 + nthr * u;
-                v[u] = make_uint4(0, 0, 0, 0);
-                const int n = i >> 4, c = i & 15;
-                if (i < tasks && (n < p.R || !p.reduce_sum)) {
-                    const int r = n % p.R;
-                    const int tq = r / p.G, a = h * p.G + r % p.G;
-                    v[u] = *reinterpret_cast<const uint4 *>(
-                        p.q + ((long long)b * p.q_batch_stride + ((long long)tq * p.Hq + a) * kHeadDim) * 2 + c * 16);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int i = i0 + nthr * u;
-                if (i >= tasks) continue;
-                const int n = i >> 4, c = i & 15;
-                const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f);
-                uint4 neg, pos;
-                const __nv_bfloat162 *f = reinterpret_cast<const __nv_bfloat162 *>(&v[u]);
-                __nv_bfloat162 *n2 = reinterpret_cast<__nv_bfloat162 *>(&neg);
-                __nv_bfloat162 *p2 = reinterpret_cast<__nv_bfloat162 *>(&pos);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    n2[e] = __hmin2(f[e], zero2);
-                    p2[e] = __hmax2(f[e], zero2);
-                }
-                const int sub = c >> 3, ch = (c & 7) ^ (n & 7);
-                uint8_t *row = dstb + n * 128 + ch * 16;
-                *reinterpret_cast<uint4 *>(row + (size_t)sub * p.N * 128) = neg;          // k in [0, 128): min rows
-                *reinterpret_cast<uint4 *>(row + (size_t)(2 + sub) * p.N * 128) = pos;    // k in [128, 256): max rows
-            }
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        build_qpm_operand(b_ptr + (size_t)buf * b_bytes, p.q, p.q_batch_stride, (int)(bh / p.Hkv), (int)(bh % p.Hkv), p.R, p.G, p.Hq,
+                          p.N, p.reduce_sum, me, nthr);
     };
 
     if (tid == 0) {
@@ -172,9 +134,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
                 if (alive) {
                     mbar_arrive_expect_tx(bar_full(s), kATileBytes);
                     const int y = (int)(bh * p.max_blocks + j0);
-#pragma unroll
-                    for (int kc = 0; kc < 4; ++kc)
-                        tma_load_2d(a_u32 + s * kATileBytes + kc * kSubTileBytes, &tmap, kc * 64, y, bar_full(s));
+                    load_score_tile(a_u32 + s * kATileBytes, &tmap, y, kSubTileBytes, bar_full(s));
                 }
             }
             alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
@@ -185,8 +145,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.N >> 3) << 17) |
-                                   ((uint32_t)(kTileBlocks >> 4) << 24);
+            const uint32_t idesc = idesc_score(p.N, kTileBlocks);
             int it = 0, bo = -1;
             long long cur_bh = -1;
             bool alive = true;
@@ -211,15 +170,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.N);
                 const uint32_t a_tile = a_u32 + s * kATileBytes;
                 const uint32_t b_tile = b_u32 + (bo % p.n_bbuf) * b_bytes;
-#pragma unroll
-                for (int kc = 0; kc < 4; ++kc) {
-#pragma unroll
-                    for (int k4 = 0; k4 < 4; ++k4) {
-                        const uint64_t ad = smem_desc_sw128(a_tile + kc * kSubTileBytes + k4 * 32);
-                        const uint64_t bd = smem_desc_sw128(b_tile + kc * p.N * 128 + k4 * 32);
-                        tc_mma_bf16(d_tmem, ad, bd, idesc, (kc | k4) ? 1u : 0u);
-                    }
-                }
+                issue_score_tile(d_tmem, a_tile, b_tile, p.N, kSubTileBytes, idesc);
                 tc_commit(bar_empty(s));         // the stage may be refilled once these MMAs have read it
                 tc_commit(bar_acc_full(acc));    // the accumulator is complete
                 ++it;
@@ -269,17 +220,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
             if (!alive) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * p.N);
-            float res = p.reduce_sum ? 0.f : -CUDART_INF_F;
-#pragma unroll 1
-            for (int c = 0; c < p.N; c += 16) {
-                uint32_t v[16];
-                tc_ld16(taddr + c, v);
-#pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const float f = __uint_as_float(v[e]);
-                    res = p.reduce_sum ? res + f : fmaxf(res, f);
-                }
-            }
+            const float res = reduce_score_row(taddr, p.N, p.reduce_sum);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_acc_empty(acc));

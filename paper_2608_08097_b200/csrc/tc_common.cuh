@@ -228,6 +228,159 @@ __device__ __forceinline__ bool softmax_warps_all(bool pred)
     return r != 0;
 }
 
+// ---- pieces shared by the scoring kernel, the attention kernel and the fused layer kernel ----------------------
+// Instruction descriptors (kind::f16): fp32 accumulator (bit 4), operand formats (bits 7-9, 10-12: 1 = bf16),
+// B transposed for the key-major V operand (bit 16), N >> 3 (bits 17-22), M >> 4 (bits 24-28).
+__device__ __forceinline__ uint32_t idesc_qk(int mma_m)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kAtTileKeys >> 3) << 17) | ((uint32_t)(mma_m >> 4) << 24);
+}
+__device__ __forceinline__ uint32_t idesc_pv(int mma_m)
+{
+    return (1u << 4) | kIdescPvFormats | (1u << 16) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(mma_m >> 4) << 24);
+}
+__device__ __forceinline__ uint32_t idesc_score(int n_cols, int tile_blocks)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_cols >> 3) << 17) | ((uint32_t)(tile_blocks >> 4) << 24);
+}
+
+// S = Q K^T of one 64-key tile: Q (128 dims = 8 k-steps) from tensor memory, K from the stage's block images.
+__device__ __forceinline__ void issue_qk_tile(uint32_t d_tmem, uint32_t tmem_q, uint64_t k_desc, uint32_t idesc)
+{
+#pragma unroll
+    for (int kc = 0; kc < 2; ++kc)
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4)
+            tc_mma_bf16_ts(d_tmem, tmem_q + (kc * 4 + k4) * 8, k_desc + (uint64_t)((kc * kImgHalf + k4 * 32) >> 4), idesc,
+                           (kc | k4) ? 1u : 0u);
+}
+// O (+)= P V of one tile: 16 keys (one block image) per MMA, P from tensor memory.
+__device__ __forceinline__ void issue_pv_tile(uint32_t tmem_o, uint32_t p_tmem, uint64_t v_desc, uint32_t idesc, bool first_of_row)
+{
+#pragma unroll
+    for (int ks = 0; ks < kAtTileCols; ++ks)
+        tc_mma_bf16_ts(tmem_o, p_tmem + ks * 8, v_desc + (uint64_t)((ks * kEntryBytes) >> 4), idesc,
+                       (!first_of_row || ks) ? 1u : 0u);
+}
+// D[128 blocks x N] = [min | max][128 x 256] . (q^- | q^+)[256 x N] of one scoring tile: 16 MMAs of K = 16.
+__device__ __forceinline__ void issue_score_tile(uint32_t d_tmem, uint32_t a_tile, uint32_t b_tile, int n_cols, uint32_t sub_tile_bytes,
+                                                 uint32_t idesc)
+{
+#pragma unroll
+    for (int kc = 0; kc < 4; ++kc) {
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4) {
+            const uint64_t ad = smem_desc_sw128(a_tile + kc * sub_tile_bytes + k4 * 32);
+            const uint64_t bd = smem_desc_sw128(b_tile + kc * n_cols * 128 + k4 * 32);
+            tc_mma_bf16(d_tmem, ad, bd, idesc, (kc | k4) ? 1u : 0u);
+        }
+    }
+}
+// The four 2-D tensor copies (128 rows x 128 bytes each) that bring one scoring tile of 128 summaries.
+__device__ __forceinline__ void load_score_tile(uint32_t dst, const CUtensorMap *map, int y, uint32_t sub_tile_bytes, uint32_t bar)
+{
+#pragma unroll
+    for (int kc = 0; kc < 4; ++kc) tma_load_2d(dst + kc * sub_tile_bytes, map, kc * 64, y, bar);
+}
+// One block's score: the reduction (max or sum) over the N query columns of this thread's accumulator row.
+__device__ __forceinline__ float reduce_score_row(uint32_t taddr, int n_cols, bool reduce_sum)
+{
+    float res = reduce_sum ? 0.f : -CUDART_INF_F;
+#pragma unroll 1
+    for (int c = 0; c < n_cols; c += 16) {
+        uint32_t v[16];
+        tc_ld16(taddr + c, v);
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            const float f = __uint_as_float(v[e]);
+            res = reduce_sum ? res + f : fmaxf(res, f);
+        }
+    }
+    return res;
+}
+// The scoring operand (q^- | q^+) of one (request, KV head): rows n = query rows (R = draft tokens x group; rows R..N-1
+// repeat them, or are zero in sum mode), K-major with the 128-byte swizzle: element k of row n lives in sub-tile
+// k / 64; k in [0, 128) holds min(q, 0) (it meets the min rows), k in [128, 256) max(q, 0).  `nthr` threads (index
+// `me`) share the work; loads are issued eight at a time so their latencies overlap.
+__device__ __forceinline__ void build_qpm_operand(uint8_t *dstb, const uint8_t *q, long long q_batch_stride, int b, int h, int R, int G,
+                                                  int Hq, int n_cols, bool reduce_sum, int me, int nthr)
+{
+    const int tasks = n_cols * 16;                           // 16-byte chunks of the query rows
+#pragma unroll 1
+    for (int i0 = me; i0 < tasks; i0 += nthr * 8) {
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = i0 + nthr * u;
+            v[u] = make_uint4(0, 0, 0, 0);
+            const int n = i >> 4, c = i & 15;
+            if (i < tasks && (n < R || !reduce_sum)) {
+                const int r = n % R;
+                const int tq = r / G, a = h * G + r % G;
+                v[u] = *reinterpret_cast<const uint4 *>(q + ((long long)b * q_batch_stride + ((long long)tq * Hq + a) * kHeadDim) * 2 + c * 16);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = i0 + nthr * u;
+            if (i >= tasks) continue;
+            const int n = i >> 4, c = i & 15;
+            const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f);
+            uint4 neg, pos;
+            const __nv_bfloat162 *f = reinterpret_cast<const __nv_bfloat162 *>(&v[u]);
+            __nv_bfloat162 *n2 = reinterpret_cast<__nv_bfloat162 *>(&neg);
+            __nv_bfloat162 *p2 = reinterpret_cast<__nv_bfloat162 *>(&pos);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                n2[e] = __hmin2(f[e], zero2);
+                p2[e] = __hmax2(f[e], zero2);
+            }
+            const int sub = c >> 3, ch = (c & 7) ^ (n & 7);
+            uint8_t *row = dstb + n * 128 + ch * 16;
+            *reinterpret_cast<uint4 *>(row + (size_t)sub * n_cols * 128) = neg;          // k in [0, 128): min rows
+            *reinterpret_cast<uint4 *>(row + (size_t)(2 + sub) * n_cols * 128) = pos;    // k in [128, 256): max rows
+        }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+// Producer side of one attention tile (the producer warp; lanes 0..3 hold one block each): records the block ids for
+// the softmax warps, zeroes the V part of a missing block's image (a missing block contributes P = 0, which must not
+// meet stale NaN bit patterns in V), announces the bytes and issues one 5-D tensor copy per present block (the whole
+// 8 KiB entry, gathered by slot id).
+__device__ __forceinline__ void stage_attn_tile(int lane, int blk, int slot, int32_t *tile_blk_s, uint8_t *stage_ptr, uint32_t stage_u32,
+                                                const CUtensorMap *map, uint32_t bar)
+{
+    const unsigned valid = __ballot_sync(0xffffffffu, lane < kAtTileCols && blk >= 0);
+    if (lane < kAtTileCols) tile_blk_s[lane] = blk;
+    if ((valid & 0xfu) != 0xfu) {
+        // the whole warp zeroes the V part of each missing block: lane -> (row group, dim half) unit lane / 8, 128 bytes of it
+#pragma unroll
+        for (int c = 0; c < kAtTileCols; ++c) {
+            if ((valid >> c) & 1u) continue;
+            uint8_t *dst = stage_ptr + c * kEntryBytes + (lane >> 4) * kImgGroup + ((lane >> 3) & 1) * kImgHalf + kImgPart + (lane & 7) * 128;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) *reinterpret_cast<uint4 *>(dst + j * 16) = make_uint4(0, 0, 0, 0);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive_expect_tx(bar, (uint32_t)__popc(valid) * kEntryBytes);
+    __syncwarp();
+    if (lane < kAtTileCols && blk >= 0) tma_load_5d(stage_u32 + lane * kEntryBytes, map, 0, 0, 2 * slot, 0, 0, bar);
+}
+// One query row (128 dims, 16 x 16 bytes in v) to this thread's tensor-memory lane as the A operand of Q K^T.
+__device__ __forceinline__ void q_row_to_tmem(uint32_t q_lane, const uint4 (&v)[16])
+{
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const uint32_t w[16] = {v[4 * c].x, v[4 * c].y, v[4 * c].z, v[4 * c].w, v[4 * c + 1].x, v[4 * c + 1].y,
+                                v[4 * c + 1].z, v[4 * c + 1].w, v[4 * c + 2].x, v[4 * c + 2].y, v[4 * c + 2].z,
+                                v[4 * c + 2].w, v[4 * c + 3].x, v[4 * c + 3].y, v[4 * c + 3].z, v[4 * c + 3].w};
+        tc_st16(q_lane + c * 16, w);
+    }
+    tc_wait_st();
+}
+
 // ---- packed fp32 arithmetic (two lanes per instruction) and the three-input maximum of sm_100 ------------------
 __device__ __forceinline__ uint64_t f32x2(float lo, float hi)
 {
