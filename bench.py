@@ -238,12 +238,14 @@ class Work:
         self.q_pinned = None
 
     def e2e_buffers(self, bench):
+        """Pinned queries of every step stacked over the layers ([S][n_layers][B][T][Hq][128]), one device staging
+        tensor and one pinned output tensor of the same per-step shape."""
         cfg = bench.cfg
         if self.q_pinned is None:
-            self.q_pinned = [q.cpu().pin_memory() for q in self.q_dev]
-            self.q_stage = [torch.empty_like(self.q_dev[l][0]) for l in range(cfg.layers)]
-            self.out_pinned = [torch.empty((cfg.batch, self.T, cfg.n_q_heads, 128), dtype=torch.bfloat16, pin_memory=True)
-                               for _ in range(cfg.layers)]
+            self.q_pinned = torch.stack([q.cpu() for q in self.q_dev], dim=1).pin_memory()
+            self.q_stage = torch.empty_like(self.q_pinned[0], device=bench.dev)
+            self.out_pinned = torch.empty((cfg.layers, cfg.batch, self.T, cfg.n_q_heads, 128), dtype=torch.bfloat16,
+                                          pin_memory=True)
         return self.q_pinned, self.q_stage, self.out_pinned
 
 
@@ -336,7 +338,7 @@ class Bench:
         if e2e:
             q_pinned, q_stage, out_pinned = w.e2e_buffers(self)
             q_list = q_stage
-            kw.update(q_host=[q_pinned[l][s] for l in range(n)], out_host=out_pinned)
+            kw.update(q_host=q_pinned[s], out_host=out_pinned)
         else:
             q_list = [w.q_dev[l][s] for l in range(n)]
         args = (q_list, self.seq_dev[s], self.first_dev[s], self.n_new_dev[s], self.nfull_next_dev[s],

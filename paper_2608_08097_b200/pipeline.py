@@ -18,7 +18,7 @@ class DecodeLayer:
     """
 
     def __init__(self, batch, n_q_heads, n_kv_heads, max_blocks, k, n_q_tokens, device="cuda",
-                 want_lse=False):
+                 want_lse=False, out=None):
         self.B, self.Hq, self.Hkv, self.mb = batch, n_q_heads, n_kv_heads, max_blocks
         self.k, self.T = k, n_q_tokens
         self.cols = k + 2
@@ -33,7 +33,7 @@ class DecodeLayer:
         self.stage_slots = torch.empty((batch, n_kv_heads, self.cols), dtype=torch.int32, device=dev)
         self.pool = torch.zeros((rows * self.cols, 2, 16, 128), dtype=torch.bfloat16, device=dev)
         self.slot_tbl = torch.arange(rows * self.cols, dtype=torch.int32, device=dev).view(batch, n_kv_heads, self.cols)
-        self.out = torch.empty((batch, n_q_tokens, n_q_heads, 128), dtype=torch.bfloat16, device=dev)
+        self.out = torch.empty((batch, n_q_tokens, n_q_heads, 128), dtype=torch.bfloat16, device=dev) if out is None else out
         self.lse = torch.empty((batch, n_q_tokens, n_q_heads), dtype=torch.float32, device=dev) if want_lse else None
         ws = oasis.attn_workspace_bytes(self.dims, n_q_tokens, self.cols)
         self.workspace = torch.empty((max(ws, 16),), dtype=torch.uint8, device=dev)
@@ -135,8 +135,10 @@ class DecodeEngine:
         self.n_commit = int(n_commit)            # tokens per step that the KV append also writes to the full-KV pool
         self.mode, self.k, self.T, self.n_layers = mode, k, n_q_tokens, n_layers
         self.device = torch.device(device)
-        self.layers = [DecodeLayer(batch, n_q_heads, n_kv_heads, max_blocks, k, n_q_tokens, device)
-                       for _ in range(n_layers)]
+        # the layers' outputs are slices of one tensor, so that several layers' outputs can leave in one copy
+        self.out_all = torch.empty((n_layers, batch, n_q_tokens, n_q_heads, 128), dtype=torch.bfloat16, device=self.device)
+        self.layers = [DecodeLayer(batch, n_q_heads, n_kv_heads, max_blocks, k, n_q_tokens, device, out=self.out_all[l])
+                       for l in range(n_layers)]
         self.kv = [None] * n_layers
         self.table = [None] * n_layers
         self.main = torch.cuda.Stream(device=self.device)
@@ -333,22 +335,33 @@ class DecodeEngine:
         """One decode step over all layers.  seq_len: history tokens of this step; the
         prediction works on the next step's view (n_full_next, seq_next).  With q_host /
         out_host (pinned tensors per layer) the step's queries are copied in and its outputs
-        copied out inside the step (end-to-end mode).  new_kv (one [B][T][Hkv][2][128] tensor per
+        copied out inside the step (end-to-end mode).  When q_list / q_host / out_host are each ONE tensor stacked
+        over the layers ([n_layers][B][T][Hq][128]) the copies are made for `wait_group` layers at a time: a few
+        large copies disturb the gathers on the host link less than many small ones.  new_kv (one [B][T][Hkv][2][128] tensor per
         layer; engines built with append=True): the step's new keys and values.  sel_log (one tensor like
         `layers[l].sel` per layer): receives a copy of each layer's selection of this step."""
         ms, n = self.main, self.n_layers
         if self.append != (new_kv is not None):
             raise ValueError("new_kv must be given exactly when the engine was built with append=True")
         q_ready = [None] * n
+        stacked = isinstance(q_list, torch.Tensor)
         if q_host is not None:
             # a layer's queries are uploaded as soon as the previous step no longer reads the staging tensor
             with torch.cuda.stream(self.up):
-                for l in range(n):
-                    for ev in (self.attn_done[l], self.score_done[l]):
-                        if ev is not None:
-                            self.up.wait_event(ev)
-                    q_list[l].copy_(q_host[l], non_blocking=True)
-                    q_ready[l] = self._event(self.up)
+                grp = self.wait_group if (stacked and isinstance(q_host, torch.Tensor)) else 1
+                for l0 in range(0, n, grp):
+                    l1 = min(l0 + grp, n)
+                    for l in range(l0, l1):
+                        for ev in (self.attn_done[l], self.score_done[l]):
+                            if ev is not None:
+                                self.up.wait_event(ev)
+                    if grp == 1:
+                        q_list[l0].copy_(q_host[l0], non_blocking=True)
+                    else:
+                        q_list[l0:l1].copy_(q_host[l0:l1], non_blocking=True)
+                    ev = self._event(self.up)
+                    for l in range(l0, l1):
+                        q_ready[l] = ev
         # Per group of `wait_group` layers, on the prediction stream: the KV append (the previous step's attention of
         # the group's layers read the local window and the local columns that are rewritten now) and, for the fused
         # launch, the summary updates (one newly completed block per request every 16 steps), which only depend on the
@@ -401,8 +414,15 @@ class DecodeEngine:
             if out_host is not None:
                 with torch.cuda.stream(self.down):
                     self.down.wait_event(attn_done)
-                    out_host[l].copy_(L.out, non_blocking=True)
-                    self.out_done[l] = self._event(self.down)
+                    if not isinstance(out_host, torch.Tensor):
+                        out_host[l].copy_(L.out, non_blocking=True)
+                        self.out_done[l] = self._event(self.down)
+                    elif (l + 1) % self.wait_group == 0 or l == n - 1:
+                        l0 = l - l % self.wait_group
+                        out_host[l0:l + 1].copy_(self.out_all[l0:l + 1], non_blocking=True)
+                        ev = self._event(self.down)
+                        for g in range(l0, l + 1):
+                            self.out_done[g] = ev
             if q_ready[l] is not None and not self.fused:
                 self.pred.wait_event(q_ready[l])
             ready = self._predict(l, q_list[l], first_block, n_new, 1, n_full_next, seq_next, step_stamp, timers,

@@ -73,10 +73,15 @@ def test_engine_steps_match_oracle(oracle, gpu, mode, cap, append, chunk, graph,
     to_dev = lambda t: t.to(torch.int32).contiguous().to(dev)
     # end-to-end mode: the step uploads its queries from pinned memory and downloads its outputs (one pinned output
     # buffer per step and layer, so every step's result can be read after a chunk)
+    stacked = e2e and chunk in (4, 19)           # one tensor over the layers: grouped uploads / downloads
     q_pin = [lay.q_steps.pin_memory() for lay in lays] if e2e else None
     q_stage = [torch.empty_like(q_dev[l][0]) for l in range(n_layers)] if e2e else None
     out_pin = [[torch.zeros((B, T, cfg.n_q_heads, 128), dtype=torch.bfloat16).pin_memory() for _ in range(n_layers)]
                for _ in range(S)] if e2e else None
+    if stacked:
+        q_pin_all = torch.stack([lay.q_steps for lay in lays], dim=1).pin_memory()       # [S][n_layers][B][T][Hq][128]
+        q_stage = torch.empty_like(q_pin_all[0], device=dev)
+        out_pin = [torch.zeros((n_layers, B, T, cfg.n_q_heads, 128), dtype=torch.bfloat16).pin_memory() for _ in range(S)]
     eng.prime([q_dev[l][0] for l in range(n_layers)], to_dev(seq[0] // 16), to_dev(seq[0]))
 
     # oracle-side state
@@ -130,7 +135,7 @@ def test_engine_steps_match_oracle(oracle, gpu, mode, cap, append, chunk, graph,
                     to_dev((seq[s] + 1) // 16 - seq[s] // 16), to_dev((seq[s] + 1) // 16), to_dev(seq[s] + 1))
             kw = dict(step_stamp=s + 1, sel_log=sel_log[s])
             if e2e:
-                kw.update(q_host=[q_pin[l][s] for l in range(n_layers)], out_host=out_pin[s])
+                kw.update(q_host=q_pin_all[s] if stacked else [q_pin[l][s] for l in range(n_layers)], out_host=out_pin[s])
             if append:
                 kw.update(new_kv=[new_dev[l][s] for l in range(n_layers)])
             calls.append((args, kw))
