@@ -661,6 +661,10 @@ def write_summary(path, line, rows_sweep, cells, cmd):
                 "| scoring + attention bytes over the HBM step | %s of the copy peak |" % line["roofline"].get("frac_in_step"),
                 "| recall (lookahead vs true-query estimator) / (vs attention mass) | %s / %s |"
                 % (line.get("recall_lookahead_topk"), (line.get("recall_attention_mass") or {}).get("value"))]
+        if line.get("sustained"):
+            su = line["sustained"]
+            out.append("| host-KV step over %s s (%d replays of the timed graph) | %s ms at a median SM clock of %s MHz, reasons %s |"
+                       % (su["seconds"], su["repeats"], su["ms_per_step"], su["sm_mhz_median"], su["reasons"] or "none"))
     if rows_sweep:
         out += ["", "Fetch-ratio sweep (cap = floor(ratio x K) blocks per (request, KV head) per step; exposed = step with the pool in "
                 "pinned host memory minus step with the pool in HBM):", "",

@@ -139,14 +139,19 @@ def test_full_size_budget_and_draft_sweep(oracle, gpu):
             del L
 
 
-def test_full_size_engine_steps(oracle, gpu):
-    """configs[1] through the multi-layer engine exactly as bench.py drives it (full batch,
-    two layers, three consecutive steps): every request's selection (near-ties adjudicated with the
-    oracle's double-precision scores) and attention outputs against the oracle."""
+ENGINE_FULL = [("c2", synth.C2, 2, 3), ("c3", synth.C3, 1, 2), ("c4", synth.C4, 1, 2)]
+
+
+@pytest.mark.parametrize("name,base,n_layers,S", ENGINE_FULL, ids=[e[0] for e in ENGINE_FULL])
+def test_full_size_engine_steps(oracle, gpu, name, base, n_layers, S):
+    """configs[1], [2] and [3] at full size through the multi-layer engine (full batch, consecutive eager steps, every
+    selected block gathered): every request's selection (near-ties adjudicated with the oracle's double-precision
+    scores) and attention outputs against the oracle.  The fused launch runs in its three arrangements here: one row
+    per thread block (128 rows), several rows per thread block (256 rows), 128 MMA rows with row-less scoring blocks
+    (64 rows of 72 query rows)."""
     _, pipeline = gpu
     dev = torch.device("cuda")
-    n_layers, S = 2, 3
-    cfg = synth.scaled(synth.C2, layers=n_layers, steps=S)
+    cfg = synth.scaled(base, layers=n_layers, steps=S)
     k, B, Hkv, mb = cfg.k_blocks, cfg.batch, cfg.n_kv_heads, cfg.max_blocks
     lays = [synth.make_layer(cfg, seed=0, layer=l, device=dev, pin=True) for l in range(n_layers)]
     eng = pipeline.DecodeEngine(B, cfg.n_q_heads, Hkv, mb, k, cfg.n_q_tokens, n_layers, dev)
@@ -184,3 +189,17 @@ def test_full_size_engine_steps(oracle, gpu):
                 pu.assert_attn_close(pu.bf16_to_f32_np(eng.layers[l].out[b:b + 1]), ref)
         used_sel = [eng.layers[l].sel.cpu().numpy() for l in range(n_layers)]
         prev_q = s
+
+
+def test_full_size_engine_delta_append_graph(oracle, gpu):
+    """configs[1] at full size the way bench.py runs it: delta selection with the paper's default cap, the KV append,
+    three decode steps in ONE CUDA graph, queries uploaded and outputs downloaded inside the steps; every request,
+    two layers, against the oracle (attention of every step, selections, tables, working-set pool, and the blocks of
+    the CPU pool that the write-through can have touched)."""
+    from tests import engine_util
+    _, pipeline = gpu
+    dev = torch.device("cuda")
+    cfg = synth.scaled(synth.C2, layers=2, steps=3)
+    lays = [synth.make_layer(cfg, seed=0, layer=l, device=dev, pin=True) for l in range(cfg.layers)]
+    engine_util.check_engine(oracle, pipeline, cfg, lays, "delta", int(0.05 * cfg.k_blocks), True, 3, True, True, True,
+                             wait_group=1, transfer_group=2, max_adjudicated=64, light=True)
