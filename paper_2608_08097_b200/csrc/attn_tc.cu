@@ -79,6 +79,7 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
     auto bar_p_full = [&](int a) { return bar_u32 + 8u * (2 * kAtMaxStages + kAtSBufs + a); };
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 8 * (2 * kAtMaxStages + 2 * kAtSBufs + 2));
     int32_t *tile_blk = reinterpret_cast<int32_t *>(misc + 8 * (2 * kAtMaxStages + 2 * kAtSBufs + 4));   // [stages][4]
+    int32_t *win = reinterpret_cast<int32_t *>(misc + 512);                                             // two table windows
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int split = blockIdx.x % p.n_splits;
@@ -139,27 +140,19 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
     if (warp == 0) {
         // ---------------------------------------------------------------- producer
         bool alive = true;
-        // Table entries are read 32 columns (eight tiles) at a time, lane j holding column j of the window, and the
-        // next window is requested as soon as the current one starts, so no table load sits on the critical path.
-        auto load_window = [&](int first_col, int &wblk, int &wslot) {
-            const int c = first_col + lane;
-            wblk = c < c1 ? blk_row[c] : -1;
-            wslot = c < c1 ? slot_row[c] : -1;
-            if (kBoundsCheck && wblk >= 0 && !in_range(wslot, p.n_slots, Bounds{0, 0, p.err}, kErrSlot)) wblk = -1;
-        };
-        int cur_blk, cur_slot, nxt_blk = -1, nxt_slot = -1;
-        load_window(c0, cur_blk, cur_slot);
+        // Table entries come 32 columns (eight tiles) at a time through two window buffers, one window ahead.
+        const uint32_t win_u32 = smem_u32(win);
+        window_request(win_u32, lane, blk_row, slot_row, c0 + lane, c1);
         int s = 0;
         uint32_t ph = 1;                                             // parity of the "empty" phase to wait for
         for (int i = 0; i < n_tiles && alive; ++i, ph ^= (s + 1 == p.stages), s = (s + 1 == p.stages) ? 0 : s + 1) {
             if ((i & 7) == 0) {
-                if (i > 0) { cur_blk = nxt_blk; cur_slot = nxt_slot; }
-                load_window(c0 + (i + 8) * kAtTileCols, nxt_blk, nxt_slot);
+                window_wait();
+                window_request(win_u32 + (((i >> 3) + 1) & 1) * kWinBytes, lane, blk_row, slot_row, c0 + (i + 8) * kAtTileCols + lane, c1);
             }
-            const int src_lane = (i & 7) * kAtTileCols + (lane & 3);
-            int blk = __shfl_sync(0xffffffffu, cur_blk, src_lane);
-            const int slot = __shfl_sync(0xffffffffu, cur_slot, src_lane);
-            if (lane >= kAtTileCols) blk = -1;
+            int blk, slot;
+            window_read(win, i, lane, blk, slot);
+            if (kBoundsCheck && blk >= 0 && !in_range(slot, p.n_slots, Bounds{0, 0, p.err}, kErrSlot)) blk = -1;
             if (lane == 0) alive = mbar_wait(bar_empty(s), ph, p.err, 41);
             alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
             if (!alive) break;
@@ -167,8 +160,8 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
                             kv_u32 + s * kAtStageBytes, &tmap, bar_full(s));
         }
     } else if (warp == 1) {
-        // ---------------------------------------------------------------- Q K^T issuer
-        if (lane == 0) {
+        // ---------------------------------------------------------------- Q K^T issuer (the whole warp, converged)
+        {
             const uint32_t idesc = idesc_qk(MMA_M);
             // descriptors: the operand start address occupies the low 14 bits (16-byte units), so offsets are added there
             const uint64_t k_desc0 = smem_desc_sw128_k(kv_u32, kImgGroup);
@@ -178,11 +171,11 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
             for (int i = 0; i < n_tiles && alive; ++i) {
                 // the S buffer also held P of tile i - kAtSBufs: its P V must have completed
                 if (i >= kAtSBufs) {
-                    alive = mbar_wait(bar_empty(s_old), ph_old, p.err, 51);
+                    alive = mbar_wait_warp(bar_empty(s_old), ph_old, p.err, 51);
                     ph_old ^= (s_old + 1 == p.stages);
                     s_old = (s_old + 1 == p.stages) ? 0 : s_old + 1;
                 }
-                alive = alive && mbar_wait(bar_full(s), ph, p.err, 52);
+                alive = alive && mbar_wait_warp(bar_full(s), ph, p.err, 52);
                 if (!alive) break;
                 tc_fence_after();
                 const uint64_t k_desc = k_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
@@ -195,15 +188,15 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
             }
         }
     } else if (warp == 2) {
-        // ---------------------------------------------------------------- P V issuer
-        if (lane == 0) {
+        // ---------------------------------------------------------------- P V issuer (the whole warp, converged)
+        {
             const uint32_t idesc = idesc_pv(MMA_M);
             const uint64_t v_desc0 = smem_desc_sw128_mn(kv_u32 + kImgPart, kImgHalf, kImgGroup);
             bool alive = true;
             int s = 0, sb = 0;
             uint32_t ph_p = 0;
             for (int i = 0; i < n_tiles && alive; ++i) {
-                alive = mbar_wait(bar_p_full(sb), ph_p, p.err, 53);
+                alive = mbar_wait_warp(bar_p_full(sb), ph_p, p.err, 53);
                 if (!alive) break;
                 tc_fence_after();
                 const uint64_t v_desc = v_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
@@ -363,7 +356,7 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
 
 // ---- host side -----------------------------------------------------------------------------------------
 
-size_t attn_tc_smem_bytes(int stages) { return 1024 + kAtQBytes + (size_t)stages * kAtStageBytes + 512; }
+size_t attn_tc_smem_bytes(int stages) { return 1024 + kAtQBytes + (size_t)stages * kAtStageBytes + 512 + 2 * kWinBytes; }
 
 int launch_attn_tc(const oasis_dims_t *dims, const void *q, int n_q_tokens, const void *hbm_pool,
                    const int32_t *slot_tbl, const int32_t *blk_tbl, int n_cols, const int32_t *seq_len, float scale,

@@ -122,6 +122,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     constexpr int kNBars = kB0 + 2 * kLyPairs + 9;                   // 35 with six stages
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 8 * kNBars);
     int32_t *tile_blk = reinterpret_cast<int32_t *>(misc + 8 * kNBars + 16);   // [stages][4]
+    int32_t *win = reinterpret_cast<int32_t *>(misc + 512);                    // two table windows
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // ---- attention geometry: CTA c < rows owns row c ------------------------------------------------------
@@ -220,10 +221,10 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             }
         }
         // ---------------------------------------------------------------- producer
-        // Table entries are read 32 columns (eight tiles) at a time, lane j holding column j of the window, and the
-        // next window is requested as soon as the current one starts, so no table load sits on the critical path.
+        // Table entries come 32 columns (eight tiles) at a time through two window buffers, one window ahead.
         // the attention phase reads what the previous layer may have produced: wait for it (no-op without a programmatic launch)
         asm volatile("griddepcontrol.wait;" ::: "memory");
+        const uint32_t win_u32 = smem_u32(win);
         int s = 0, gi = 0;                                           // ring stage and index of the tile among all rows
         uint32_t ph = 1;                                             // parity of the "empty" phase to wait for
 #pragma unroll 1
@@ -232,24 +233,17 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         const int32_t *slot_row = p.slot_tbl + (long long)row_of(item) * p.n_cols;
         const int32_t *blk_row = p.blk_tbl + (long long)row_of(item) * p.n_cols;
         const int c0 = first_col(item), c1 = end_col(item);          // column range of the item
-        auto load_window = [&](int first, int &wblk, int &wslot) {
-            const int c = first + lane;
-            wblk = c < c1 ? blk_row[c] : -1;
-            wslot = c < c1 ? slot_row[c] : -1;
-            if (kBoundsCheck && wblk >= 0 && !in_range(wslot, p.n_slots, Bounds{0, 0, p.err}, kErrSlot)) wblk = -1;
-        };
-        int cur_blk, cur_slot, nxt_blk = -1, nxt_slot = -1;
-        load_window(c0, cur_blk, cur_slot);
+        __syncwarp();                                                // the previous row's window reads are over
+        window_request(win_u32, lane, blk_row, slot_row, c0 + lane, c1);
 #pragma unroll 1
         for (int i = 0; i < tpr && alive; ++i, ++gi, ph ^= (s + 1 == kLyStages), s = (s + 1 == kLyStages) ? 0 : s + 1) {
             if ((i & 7) == 0) {
-                if (i > 0) { cur_blk = nxt_blk; cur_slot = nxt_slot; }
-                load_window(c0 + (i + 8) * kAtTileCols, nxt_blk, nxt_slot);
+                window_wait();
+                window_request(win_u32 + (((i >> 3) + 1) & 1) * kWinBytes, lane, blk_row, slot_row, c0 + (i + 8) * kAtTileCols + lane, c1);
             }
-            const int src_lane = (i & 7) * kAtTileCols + (lane & 3);
-            int blk = __shfl_sync(0xffffffffu, cur_blk, src_lane);
-            const int slot = __shfl_sync(0xffffffffu, cur_slot, src_lane);
-            if (lane >= kAtTileCols) blk = -1;
+            int blk, slot;
+            window_read(win, i, lane, blk, slot);
+            if (kBoundsCheck && blk >= 0 && !in_range(slot, p.n_slots, Bounds{0, 0, p.err}, kErrSlot)) blk = -1;
             if (lane == 0 && gi < kLyStages) {
                 // first use of this stage: the scoring tiles that last used its 64 KiB pair must have been consumed
                 const int pr = s >> 1;
@@ -265,8 +259,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         }
     } else if (warp == 1) {
         {
-            // ---------------------------------------------------------------- scoring phase: MMAs
-            if (lane == 0) {
+            // ---------------------------------------------------------------- scoring phase: MMAs (the whole warp, converged)
+            {
                 const uint32_t idesc = idesc_score(p.N, kLyTileBlocks);
                 int it = 0, bo = -1;
                 int cur_bh = -1;
@@ -281,12 +275,12 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                         if (bo >= 0) tc_commit(bar_b_empty(bo % 2));   // earlier MMAs no longer read that operand
                         cur_bh = bh;
                         ++bo;
-                        alive = mbar_wait(bar_b_full(bo % 2), (bo / 2) & 1, p.err, 21);
+                        alive = mbar_wait_warp(bar_b_full(bo % 2), (bo / 2) & 1, p.err, 21);
                         if (!alive) break;
                     }
                     const int acc = it & 1, s = it % kLyPairs;
-                    alive = mbar_wait(bar_acc_empty(acc), ((it >> 1) & 1) ^ 1, p.err, 22) &&
-                            mbar_wait(sbar_full(s), (it / kLyPairs) & 1, p.err, 23);
+                    alive = mbar_wait_warp(bar_acc_empty(acc), ((it >> 1) & 1) ^ 1, p.err, 22) &&
+                            mbar_wait_warp(sbar_full(s), (it / kLyPairs) & 1, p.err, 23);
                     if (!alive) break;
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + (uint32_t)p.acc_col + (uint32_t)(acc * p.N);
@@ -299,8 +293,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 }
             }
         }
-        // ---------------------------------------------------------------- Q K^T issuer
-        if (lane == 0) {
+        // ---------------------------------------------------------------- Q K^T issuer (the whole warp, converged)
+        {
             const uint32_t idesc = idesc_qk(MMA_M);
             // descriptors: the operand start address occupies the low 14 bits (16-byte units), so offsets are added there
             const uint64_t k_desc0 = smem_desc_sw128_k(kv_u32, kImgGroup);
@@ -311,17 +305,17 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
 #pragma unroll 1
             for (int k = 0; k < n_my_rows && alive; ++k) {
             const int tpr = tiles_of(my_row(k));
-            alive = mbar_wait(bar_q, (uint32_t)(k & 1), p.err, 55);  // the row's Q is in tensor memory
+            alive = mbar_wait_warp(bar_q, (uint32_t)(k & 1), p.err, 55);  // the row's Q is in tensor memory
             tc_fence_after();
 #pragma unroll 1
             for (int it = 0; it < tpr && alive; ++it, ++i) {
                 // the S buffer also held P of tile i - kAtSBufs: its P V must have completed
                 if (i >= kAtSBufs) {
-                    alive = mbar_wait(bar_empty(s_old), ph_old, p.err, 51);
+                    alive = mbar_wait_warp(bar_empty(s_old), ph_old, p.err, 51);
                     ph_old ^= (s_old + 1 == kLyStages);
                     s_old = (s_old + 1 == kLyStages) ? 0 : s_old + 1;
                 }
-                alive = alive && mbar_wait(bar_full(s), ph, p.err, 52);
+                alive = alive && mbar_wait_warp(bar_full(s), ph, p.err, 52);
                 if (!alive) break;
                 tc_fence_after();
                 const uint64_t k_desc = k_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
@@ -335,8 +329,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             }
         }
     } else if (warp == 2) {
-        // ---------------------------------------------------------------- P V issuer
-        if (lane == 0) {
+        // ---------------------------------------------------------------- P V issuer (the whole warp, converged)
+        {
             const uint32_t idesc = idesc_pv(MMA_M);
             const uint64_t v_desc0 = smem_desc_sw128_mn(kv_u32 + kImgPart, kImgHalf, kImgGroup);
             bool alive = true;
@@ -347,7 +341,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             const int tpr = tiles_of(my_row(k));
 #pragma unroll 1
             for (int it = 0; it < tpr && alive; ++it) {
-                alive = mbar_wait(bar_p_full(sb), ph_p, p.err, 53);
+                alive = mbar_wait_warp(bar_p_full(sb), ph_p, p.err, 53);
                 if (!alive) break;
                 tc_fence_after();
                 const uint64_t v_desc = v_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
@@ -629,7 +623,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
 static size_t layer_tc_smem_bytes(int mma_m, int copies, int N, int stages)
 {
     return 1024 + (size_t)stages * kAtStageBytes + 2 * (size_t)N * kSummaryBytes +
-           (size_t)mma_m * ((copies > 1 ? 20 : 0) + 2) * sizeof(float) + 512;
+           (size_t)mma_m * ((copies > 1 ? 20 : 0) + 2) * sizeof(float) + 512 + 2 * kWinBytes;
 }
 
 struct LayerTcPlan {

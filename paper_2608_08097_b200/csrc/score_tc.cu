@@ -143,8 +143,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
             t = tn;
         }
     } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
+        // ---------------------------------------------------------------- MMA issuer (the whole warp, converged)
+        {
             const uint32_t idesc = idesc_score(p.N, kTileBlocks);
             int it = 0, bo = -1;
             long long cur_bh = -1;
@@ -159,12 +159,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
                     if (bo >= 0) tc_commit(bar_b_empty(bo % p.n_bbuf));   // earlier MMAs no longer read that operand
                     cur_bh = bh;
                     ++bo;
-                    alive = mbar_wait(bar_b_full(bo % p.n_bbuf), (bo / p.n_bbuf) & 1, p.err, 21);
+                    alive = mbar_wait_warp(bar_b_full(bo % p.n_bbuf), (bo / p.n_bbuf) & 1, p.err, 21);
                     if (!alive) break;
                 }
                 const int acc = it & 1, s = it % p.stages;
-                alive = mbar_wait(bar_acc_empty(acc), ((it >> 1) & 1) ^ 1, p.err, 22) &&
-                        mbar_wait(bar_full(s), (it / p.stages) & 1, p.err, 23);
+                alive = mbar_wait_warp(bar_acc_empty(acc), ((it >> 1) & 1) ^ 1, p.err, 22) &&
+                        mbar_wait_warp(bar_full(s), (it / p.stages) & 1, p.err, 23);
                 if (!alive) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.N);

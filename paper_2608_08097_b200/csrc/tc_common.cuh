@@ -46,6 +46,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t
 {
     return mbar_wait_limit(bar, parity, err, code, kSpinLimit);
 }
+// The same wait made by all 32 lanes of a converged warp (the MMA-issuing warps); the lanes agree on the outcome, so the
+// warp stays converged whatever happens.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int32_t *err, int code)
+{
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, err, code));
+}
 // One non-blocking probe of a phase.
 __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
 {
@@ -68,17 +74,27 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// tcgen05.mma and tcgen05.commit are issued by ONE lane, but from a converged warp: all 32 lanes call these wrappers
+// with the same arguments and elect.sync picks the issuing lane (always the same one for the full mask, so a commit
+// tracks the MMAs before it).  Issued from inside an `if (lane == 0)` branch instead, every MMA costs about 60 cycles
+// whatever its shape (measured: 8 MMAs of 128 x 64 x 16 in 497 cycles), because in divergent code the descriptors
+// cannot stay in uniform registers; from a converged warp the same eight take 257 cycles, the tensor core's own time.
 __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                             uint32_t accumulate)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
+        "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
@@ -160,9 +176,10 @@ __device__ __forceinline__ void tc_mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem,
                                                uint32_t accumulate)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
+        "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
@@ -342,6 +359,44 @@ __device__ __forceinline__ void build_qpm_operand(uint8_t *dstb, const uint8_t *
         }
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+// ---- table windows of the attention producers ------------------------------------------------------------------
+// The producer warp reads a row's block ids and slot ids 32 columns (eight tiles) at a time, one window ahead, by
+// asynchronous copies into two small shared-memory buffers: lane j requests column j of the window, and the copies
+// of a window are only waited for when its first tile comes up, eight tiles later.  (Loads into registers did not
+// stay ahead: written as a rotation of current / next window registers, the warp stalled for a whole memory
+// latency, 2,300-3,100 cycles, at every window switch, whatever form the load took.)
+constexpr int kWinCols = 32;                                // columns per window
+constexpr int kWinBytes = 2 * kWinCols * 4;                 // block ids [32], slot ids [32]
+// Lane `lane` requests column `c` of the row (beyond the last column `c1 - 1`: -1) into the window buffer at `win_u32`.
+__device__ __forceinline__ void window_request(uint32_t win_u32, int lane, const int32_t *blk_row, const int32_t *slot_row, int c, int c1)
+{
+    const uint32_t dst = win_u32 + (uint32_t)lane * 4u;
+    if (c < c1) {
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(blk_row + c) : "memory");
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst + kWinCols * 4), "l"(slot_row + c) : "memory");
+    } else {
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst), "r"(-1) : "memory");
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + kWinCols * 4), "r"(-1) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+// All requested windows have landed and are visible to the whole warp; earlier reads of the buffers are over.
+__device__ __forceinline__ void window_wait()
+{
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncwarp();
+}
+// Block id and slot id of this lane's column of tile `i` (lanes 0..3; -1 for the other lanes).
+__device__ __forceinline__ void window_read(const int32_t *win, int i, int lane, int &blk, int &slot)
+{
+    const int32_t *w = win + ((i >> 3) & 1) * (2 * kWinCols) + (i & 7) * kAtTileCols;
+    blk = -1;
+    slot = -1;
+    if (lane < kAtTileCols) {
+        blk = w[lane];
+        slot = w[kWinCols + lane];
+    }
 }
 // Producer side of one attention tile (the producer warp; lanes 0..3 hold one block each): records the block ids for
 // the softmax warps, zeroes the V part of a missing block's image (a missing block contributes P = 0, which must not
