@@ -26,6 +26,18 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 // Bounded wait: false (and an error code in *err) if the phase did not complete within `limit` probes.
 __device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, int32_t *err, int code, uint32_t limit)
 {
+    {
+        // one non-blocking probe first: try_wait on a phase that has already completed costs well over a hundred cycles
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
 #pragma unroll 1                 // the compiler otherwise unrolls the spin loop at every call site (half the kernel's code)
     for (uint32_t i = 0; i < limit; ++i) {
         uint32_t done;
