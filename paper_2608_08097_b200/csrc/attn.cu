@@ -28,39 +28,58 @@ struct AttnParams {
 };
 
 // Merges the splits of one (request, KV head, row): out = sum_s w_s o_s / sum_s w_s with
-// w_s = 2^(lse_s - max lse).  CTAs of 256 threads take the `total` rows in turn, two at a time.  Launched behind the fused layer
-// kernel with programmatic stream serialization it lets the launch after it start early and itself waits for the
-// partials (both instructions do nothing in an ordinary launch).
+// w_s = 2^(lse_s - max lse).  One warp per row, four output dims per thread (16-byte loads of the partials, the loads
+// of four splits in flight at a time); CTAs of 256 threads take the `total` rows in turn, eight at a time.  Launched
+// behind the fused layer kernel with programmatic stream serialization it lets the launch after it start early and
+// itself waits for the partials (both instructions do nothing in an ordinary launch).
 __global__ void __launch_bounds__(256)
 attn_combine_kernel(const AttnParams p, long long total)
 {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int lane = threadIdx.x & 31;
 #pragma unroll 1
-    for (long long wi = 2ll * blockIdx.x + (threadIdx.x >> 7); wi < total; wi += 2ll * gridDim.x) {
-    const int row = (int)(wi % p.R);
-    const int bh = (int)(wi / p.R);
-    const int b = bh / p.Hkv, h = bh % p.Hkv;
-    const int grp = row / p.rows_per_group, r = row % p.rows_per_group;
-    const int d = threadIdx.x & 127;
-    float mx = -CUDART_INF_F;
-    for (int s = 0; s < p.n_splits; ++s) {
-        const long long item = ((long long)bh * p.n_splits + s) * p.n_groups + grp;
-        mx = fmaxf(mx, p.part_lse[item * p.rows_per_group + r]);
-    }
-    float acc = 0.f, den = 0.f;
-    if (mx > -CUDART_INF_F) {
-        for (int s = 0; s < p.n_splits; ++s) {
-            const long long prow = (((long long)bh * p.n_splits + s) * p.n_groups + grp) * p.rows_per_group + r;
-            const float w = fast_exp2(p.part_lse[prow] - mx);
-            acc += w * p.part_o[prow * kHeadDim + d];
-            den += w;
+    for (long long wi = 8ll * blockIdx.x + (threadIdx.x >> 5); wi < total; wi += 8ll * gridDim.x) {
+        const int row = (int)(wi % p.R);
+        const int bh = (int)(wi / p.R);
+        const int b = bh / p.Hkv, h = bh % p.Hkv;
+        const int grp = row / p.rows_per_group, r = row % p.rows_per_group;
+        // partial row of split s: prow0 + s * pstride
+        const long long prow0 = ((long long)bh * p.n_splits * p.n_groups + grp) * p.rows_per_group + r;
+        const long long pstride = (long long)p.n_groups * p.rows_per_group;
+        float mx = -CUDART_INF_F;
+        for (int s = lane; s < p.n_splits; s += 32) mx = fmaxf(mx, p.part_lse[prow0 + s * pstride]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float den = 0.f;
+        if (mx > -CUDART_INF_F) {
+#pragma unroll 1
+            for (int s0 = 0; s0 < p.n_splits; s0 += 4) {
+                float w[4];
+                float4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const bool in = s0 + u < p.n_splits;
+                    const long long prow = prow0 + (in ? s0 + u : s0) * pstride;
+                    w[u] = in ? p.part_lse[prow] : -CUDART_INF_F;
+                    v[u] = reinterpret_cast<const float4 *>(p.part_o + prow * kHeadDim)[lane];
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const float ws = fast_exp2(w[u] - mx);           // 0 for the splits past the last one
+                    acc.x += ws * v[u].x; acc.y += ws * v[u].y; acc.z += ws * v[u].z; acc.w += ws * v[u].w;
+                    den += ws;
+                }
+            }
         }
-    }
-    const int tq = row / p.G, a = h * p.G + row % p.G;
-    const long long orow = ((long long)b * p.T + tq) * p.Hq + a;
-    reinterpret_cast<__nv_bfloat16 *>(p.out)[orow * kHeadDim + d] = __float2bfloat16_rn(den > 0.f ? acc / den : 0.f);
-    if (p.lse && d == 0) p.lse[orow] = den > 0.f ? (mx + log2f(den)) * kLn2 : -CUDART_INF_F;
+        const bool any = den > 0.f;                                  // some split saw a key
+        if (!any) { acc = make_float4(0.f, 0.f, 0.f, 0.f); den = 1.f; }
+        const int tq = row / p.G, a = h * p.G + row % p.G;
+        const long long orow = ((long long)b * p.T + tq) * p.Hq + a;
+        reinterpret_cast<uint2 *>(p.out + orow * kHeadDim * 2)[lane] =
+            make_uint2(pack_bf16x2(acc.x / den, acc.y / den), pack_bf16x2(acc.z / den, acc.w / den));
+        if (p.lse && lane == 0) p.lse[orow] = any ? (mx + log2f(den)) * kLn2 : -CUDART_INF_F;
     }
 }
 
@@ -109,7 +128,7 @@ static int launch_attn(const oasis_dims_t *dims, const AttnPlan &pl, const AttnP
                                 p.part_o, p.part_lse, pl.n_splits, pl.cols_per_split, kAttnStages, error_word(), st, who))
         return rc;
     if (pl.n_splits > 1) {
-        attn_combine_kernel<<<(unsigned)((combine_ctas + 1) / 2), 256, 0, st>>>(p, combine_ctas);
+        attn_combine_kernel<<<(unsigned)((combine_ctas + 7) / 8), 256, 0, st>>>(p, combine_ctas);
         return check_launch(who);
     }
     return OASIS_OK;
@@ -136,7 +155,7 @@ int launch_attn_combine_after(const oasis_dims_t *dims, int T, void *out, float 
     p.R = T * p.G; p.n_splits = n_splits; p.n_groups = 1; p.rows_per_group = p.R;
     const long long total = (long long)dims->batch * dims->n_kv_heads * p.R;
     long long grid = (long long)sm_count() * 2;          // all resident beside the fused kernel's thread blocks
-    if (grid > (total + 1) / 2) grid = (total + 1) / 2;
+    if (grid > (total + 7) / 8) grid = (total + 7) / 8;
     prefer_max_shared_carveout(attn_combine_kernel);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

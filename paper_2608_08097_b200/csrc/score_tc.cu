@@ -163,8 +163,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap, const ScoreTcParams p)
                     if (!alive) break;
                 }
                 const int acc = it & 1, s = it % p.stages;
-                alive = mbar_wait_warp(bar_acc_empty(acc), ((it >> 1) & 1) ^ 1, p.err, 22) &&
-                        mbar_wait_warp(bar_full(s), (it / p.stages) & 1, p.err, 23);
+alive = mbar_wait_warp2(bar_acc_empty(acc), ((it >> 1) & 1) ^ 1, bar_full(s), (it / p.stages) & 1, p.err, 23);
                 if (!alive) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.N);
