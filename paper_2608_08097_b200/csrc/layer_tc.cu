@@ -80,13 +80,15 @@ struct LayerTcParams {
 // instantiations because the kernel is sensitive to every instruction its issuing threads execute (the row loop
 // costs mode 0 1.5 us at 128 rows, the split arithmetic 0.5 us).  STAGES: 32 KiB stages of the ring (6, or 4 where
 // the scoring operands or the copy-merge staging need the room).
-template <int MMA_M, int COPIES, int MODE, int STAGES>
+template <int MMA_M, int COPIES, int MODE, int STAGES, int ASTAGES>
 __global__ void __launch_bounds__(kLyThreads, 1)
 layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap_summ,
                 const LayerTcParams p)
 {
     constexpr bool MULTI = MODE == 1, SPLIT = MODE == 2;
-    constexpr int kLyStages = STAGES, kLyPairs = STAGES / 2;
+    // ASTAGES: stages of the ring in the attention phase.  Where 64 scoring rows leave room for only four stages beside
+    // the two 32 KiB operand buffers, those buffers, idle once the last scoring MMA has completed, are stages 4 and 5.
+    constexpr int kLyStages = ASTAGES, kLyPairs = STAGES / 2;
     constexpr int RPC = MMA_M / COPIES;                     // MMA rows per copy of the query rows
     constexpr int LANES = MMA_M / 4;                        // lanes of each softmax warp that hold an MMA row
     constexpr int BPC = kAtTileCols / COPIES;               // blocks of a tile each copy handles
@@ -98,8 +100,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t kv_u32 = base;                                    // [STAGES][32 KiB] = [STAGES / 2][64 KiB]
     const uint32_t b_bytes = (uint32_t)p.N * kSummaryBytes;
-    const uint32_t b_u32 = kv_u32 + kLyStages * kAtStageBytes;       // [2][N][512 B] as 4 sub-tiles of N x 128 B
-    uint8_t *b_ptr = base_ptr + (size_t)kLyStages * kAtStageBytes;
+    const uint32_t b_u32 = kv_u32 + STAGES * kAtStageBytes;          // [2][N][512 B] as 4 sub-tiles of N x 128 B
+    uint8_t *b_ptr = base_ptr + (size_t)STAGES * kAtStageBytes;
     float *o_sm = reinterpret_cast<float *>(b_ptr + 2 * b_bytes);    // [MMA_M][kStageF]
     float *m_sm = o_sm + MMA_M * kStageF;                            // [MMA_M]
     float *l_sm = m_sm + MMA_M;                                      // [MMA_M]
@@ -119,7 +121,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     auto bar_b_full = [&](int a) { return bar_u32 + 8u * (kB0 + 2 * kLyPairs + 4 + a); };
     auto bar_b_empty = [&](int a) { return bar_u32 + 8u * (kB0 + 2 * kLyPairs + 6 + a); };
     const uint32_t bar_q = bar_u32 + 8u * (kB0 + 2 * kLyPairs + 8);  // Q is in tensor memory
-    constexpr int kNBars = kB0 + 2 * kLyPairs + 9;                   // 35 with six stages
+    const uint32_t bar_score_done = bar_u32 + 8u * (kB0 + 2 * kLyPairs + 9);   // every scoring MMA has completed
+    constexpr int kNBars = kB0 + 2 * kLyPairs + 10;                  // 36 with six stages
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(misc + 8 * kNBars);
     int32_t *tile_blk = reinterpret_cast<int32_t *>(misc + 8 * kNBars + 16);   // [stages][4]
     int32_t *win = reinterpret_cast<int32_t *>(misc + 512);                    // two table windows
@@ -245,10 +248,15 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             window_read(win, i, lane, blk, slot);
             if (kBoundsCheck && blk >= 0 && !in_range(slot, p.n_slots, Bounds{0, 0, p.err}, kErrSlot)) blk = -1;
             if (lane == 0 && gi < kLyStages) {
-                // first use of this stage: the scoring tiles that last used its 64 KiB pair must have been consumed
-                const int pr = s >> 1;
-                const int uses = it > pr ? (it - pr + kLyPairs - 1) / kLyPairs : 0;
-                if (uses > 0) alive = mbar_wait(sbar_empty(pr), (uses - 1) & 1, p.err, 14);
+                if (s < STAGES) {
+                    // first use of this stage: the scoring tiles that last used its 64 KiB pair must have been consumed
+                    const int pr = s >> 1;
+                    const int uses = it > pr ? (it - pr + kLyPairs - 1) / kLyPairs : 0;
+                    if (uses > 0) alive = mbar_wait(sbar_empty(pr), (uses - 1) & 1, p.err, 14);
+                } else {
+                    // a stage in the place of the scoring operands: every scoring MMA must have completed
+                    alive = mbar_wait(bar_score_done, 0, p.err, 15);
+                }
             }
             if (lane == 0) alive = alive && mbar_wait(bar_empty(s), ph, p.err, 41);
             alive = __shfl_sync(0xffffffffu, (int)alive, 0) != 0;
@@ -291,6 +299,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                     tc_commit(bar_acc_full(acc));    // the accumulator is complete
                     ++it;
                 }
+                if (ASTAGES > STAGES) tc_commit(bar_score_done);     // (arrives at once if this thread block scored nothing)
             }
         }
         // ---------------------------------------------------------------- Q K^T issuer (the whole warp, converged)
@@ -627,7 +636,7 @@ static size_t layer_tc_smem_bytes(int mma_m, int copies, int N, int stages)
 }
 
 struct LayerTcPlan {
-    int R, Rs, N, mma_m, copies, stages;
+    int R, Rs, N, mma_m, copies, stages, astages;
     int n_splits, cols_per_split;       // of every row's column list (1 = rows are attended whole)
     size_t smem, workspace;
 };
@@ -660,6 +669,8 @@ static bool layer_tc_plan(const oasis_dims_t *dims, int n_q_tokens, int n_cols, 
         pl.stages = 4;
         pl.smem = layer_tc_smem_bytes(pl.mma_m, pl.copies, pl.N, pl.stages);
     }
+    // attention-phase stages: with four stages and 64 scoring rows the two operand buffers (2 x 32 KiB) are two more
+    pl.astages = (pl.stages == 4 && 2 * (size_t)pl.N * kSummaryBytes >= 2 * (size_t)kAtStageBytes) ? 6 : pl.stages;
     pl.n_splits = 1;
     pl.cols_per_split = n_cols;
     pl.workspace = 0;
@@ -808,23 +819,25 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-#define OASIS_LAYER_TC_LAUNCH_2(M, C, MU, ST)                                                                            \
-    do {                                                                                                                 \
-        e = cudaFuncSetAttribute(layer_tc_kernel<M, C, MU, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
-        if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, layer_tc_kernel<M, C, MU, ST>, tmap_kv, tmap_summ, p);         \
+#define OASIS_LAYER_TC_LAUNCH_2(M, C, MU, ST, AST)                                                                            \
+    do {                                                                                                                      \
+        e = cudaFuncSetAttribute(layer_tc_kernel<M, C, MU, ST, AST>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
+        if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, layer_tc_kernel<M, C, MU, ST, AST>, tmap_kv, tmap_summ, p);         \
     } while (0)
-#define OASIS_LAYER_TC_LAUNCH(M, C, ST)                          \
-    do {                                                         \
-        if (pl.n_splits > 1) OASIS_LAYER_TC_LAUNCH_2(M, C, 2, ST);  \
-        else if (items > grid) OASIS_LAYER_TC_LAUNCH_2(M, C, 1, ST); \
-        else OASIS_LAYER_TC_LAUNCH_2(M, C, 0, ST);               \
+#define OASIS_LAYER_TC_LAUNCH(M, C, ST, AST)                          \
+    do {                                                              \
+        if (pl.n_splits > 1) OASIS_LAYER_TC_LAUNCH_2(M, C, 2, ST, AST);  \
+        else if (items > grid) OASIS_LAYER_TC_LAUNCH_2(M, C, 1, ST, AST); \
+        else OASIS_LAYER_TC_LAUNCH_2(M, C, 0, ST, AST);               \
     } while (0)
-    if (R <= 16) OASIS_LAYER_TC_LAUNCH(64, 4, 6);
-    else if (R <= 32) OASIS_LAYER_TC_LAUNCH(64, 2, 6);
-    else if (R <= 64 && pl.stages == 6) OASIS_LAYER_TC_LAUNCH(128, 2, 6);
-    else if (R <= 64) OASIS_LAYER_TC_LAUNCH(128, 2, 4);
-    else if (pl.stages == 6) OASIS_LAYER_TC_LAUNCH(128, 1, 6);
-    else OASIS_LAYER_TC_LAUNCH(128, 1, 4);
+    if (R <= 16) OASIS_LAYER_TC_LAUNCH(64, 4, 6, 6);
+    else if (R <= 32) OASIS_LAYER_TC_LAUNCH(64, 2, 6, 6);
+    else if (R <= 64 && pl.stages == 6) OASIS_LAYER_TC_LAUNCH(128, 2, 6, 6);
+    else if (R <= 64 && pl.astages == 6) OASIS_LAYER_TC_LAUNCH(128, 2, 4, 6);
+    else if (R <= 64) OASIS_LAYER_TC_LAUNCH(128, 2, 4, 4);
+    else if (pl.stages == 6) OASIS_LAYER_TC_LAUNCH(128, 1, 6, 6);
+    else if (pl.astages == 6) OASIS_LAYER_TC_LAUNCH(128, 1, 4, 6);
+    else OASIS_LAYER_TC_LAUNCH(128, 1, 4, 4);
 #undef OASIS_LAYER_TC_LAUNCH
 #undef OASIS_LAYER_TC_LAUNCH_2
     if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "%s: launch with %zu B of shared memory: %s", who, smem, cudaGetErrorString(e));
