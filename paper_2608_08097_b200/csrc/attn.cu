@@ -128,7 +128,19 @@ static int launch_attn(const oasis_dims_t *dims, const AttnPlan &pl, const AttnP
                                 p.part_o, p.part_lse, pl.n_splits, pl.cols_per_split, kAttnStages, error_word(), st, who))
         return rc;
     if (pl.n_splits > 1) {
-        attn_combine_kernel<<<(unsigned)((combine_ctas + 7) / 8), 256, 0, st>>>(p, combine_ctas);
+        // programmatic stream serialization: the merge's thread blocks become resident while the attention still runs
+        // and wait there for its partials, which hides their launch
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)((combine_ctas + 7) / 8));
+        cfg.blockDim = dim3(256);
+        cfg.stream = st;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, attn_combine_kernel, p, combine_ctas);
+        if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "%s: combine launch: %s", who, cudaGetErrorString(e));
         return check_launch(who);
     }
     return OASIS_OK;

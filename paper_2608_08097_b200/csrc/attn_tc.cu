@@ -9,14 +9,16 @@
 //              by slot id) as [row group][dim half][K, V][8 rows][128 B] with the 128-byte swizzle,
 //              so that the 8-row groups of consecutive blocks are uniformly 4 KiB apart and both
 //              the K operand (K-major) and the V operand (key-major) can be described to the MMA.
-//              Slot / block tables are read 32 columns at a time, one window ahead.
-//   warp 1     one thread issues S = Q K^T (8 x tcgen05.mma M x 64 x 16, Q read from tensor memory,
-//              K from shared memory) into one of four S buffers as soon as a tile has landed and
-//              the buffer's previous P V has completed.
-//   warp 2     one thread issues O += P V (4 x tcgen05.mma M x 128 x 16, P read from tensor memory,
-//              V from shared memory) as soon as the tile's P is written; the commit after P V
-//              releases the stage.  Issuing a tcgen05.mma costs its thread about 50-60 cycles,
-//              so two issuers halve the per-tile issue time, which otherwise bounds the loop.
+//              Slot / block tables come 32 columns at a time, one window ahead, by asynchronous
+//              copies into two small shared-memory buffers.
+//   warp 1     issues S = Q K^T (8 x tcgen05.mma M x 64 x 16, Q read from tensor memory, K from
+//              shared memory) into one of four S buffers as soon as a tile has landed and the
+//              buffer's previous P V has completed.
+//   warp 2     issues O += P V (4 x tcgen05.mma M x 128 x 16, P read from tensor memory, V from
+//              shared memory) as soon as the tile's P is written; the commit after P V releases
+//              the stage.  Both warps run converged and elect.sync picks the issuing lane: from
+//              inside an `if (lane == 0)` branch every tcgen05.mma cost its thread about 60 cycles
+//              whatever its shape, from a converged warp the tensor core's own time.
 //   warps 3-6  softmax, one thread per MMA row: tcgen05.ld of the row's logits, masking on local
 //              blocks only, exp2 against a running reference maximum that is raised lazily (only
 //              when a logit exceeds it by 2^8; the O row is then rescaled in tensor memory),
@@ -82,6 +84,8 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
     int32_t *win = reinterpret_cast<int32_t *>(misc + 512);                                             // two table windows
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // a merge launch behind this one (split runs) may bring its thread blocks onto the SMs already; it waits for the partials
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int split = blockIdx.x % p.n_splits;
     const int bh = blockIdx.x / p.n_splits;
     const int b = bh / p.Hkv, h = bh % p.Hkv;

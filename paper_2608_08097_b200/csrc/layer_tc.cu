@@ -79,7 +79,7 @@ struct LayerTcParams {
 // 2 = fewer rows than half the SMs, their column lists split into one work item per thread block.  Separate
 // instantiations because the kernel is sensitive to every instruction its issuing threads execute (the row loop
 // costs mode 0 1.5 us at 128 rows, the split arithmetic 0.5 us).  STAGES: 32 KiB stages of the ring (6, or 4 where
-// the scoring operands or the copy-merge staging need the room).
+// the scoring operands or the copy-merge staging need the room); ASTAGES: stages in the attention phase.
 template <int MMA_M, int COPIES, int MODE, int STAGES, int ASTAGES>
 __global__ void __launch_bounds__(kLyThreads, 1)
 layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap_summ,

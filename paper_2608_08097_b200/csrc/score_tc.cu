@@ -12,9 +12,10 @@
 //              into a ring of 64 KiB stages, completion on mbarriers.  It starts right after the
 //              barrier set-up, while the other warps allocate the tensor memory and build the
 //              (q^- | q^+) operand of the first (request, KV head) in the same swizzled layout.
-//   warp 1     one thread issues 16 tcgen05.mma (128 x N x 16, bf16 -> fp32) per tile into one of
-//              two TMEM accumulators and commits to the stage's "empty" and the accumulator's
-//              "full" barrier.
+//   warp 1     issues 16 tcgen05.mma (128 x N x 16, bf16 -> fp32) per tile into one of two TMEM
+//              accumulators and commits to the stage's "empty" and the accumulator's "full"
+//              barrier.  The warp runs converged, elect.sync picks the issuing lane, and its two
+//              waits per tile are one predicated probe by two lanes and a ballot.
 //   warps 2-5  epilogue: tcgen05.ld of the thread's TMEM lane (= one block), max / sum over its N
 //              columns, one coalesced fp32 store per block.
 //   warp 6     builds the (q^- | q^+) operand of every further (request, KV head) of the CTA's range
