@@ -224,8 +224,9 @@ size_t oasis_attn_workspace_bytes(const oasis_dims_t *dims, int32_t n_q_tokens,
  * are read, and scores written, while that previous launch may still be running, and the launch after this
  * one may start as soon as this one has begun.  So the previous launch on `stream` must neither produce
  * those inputs nor still use `scores` (an oasis_attn_and_score of another layer is the intended
- * predecessor); separate such producers and consumers from this call by an event on another stream or by
- * another launch in between.  Everything the attention phase touches (q,
+ * predecessor; it, oasis_sparse_attn and their merge launches are the launches of this library that let
+ * a successor start early); separate such producers and consumers from this call by an event on another
+ * stream or by another launch in between.  Everything the attention phase touches (q,
  * hbm_pool, the tables, out, lse, workspace) is ordered as usual.
  */
 int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int32_t n_q_tokens, const void *hbm_pool,
