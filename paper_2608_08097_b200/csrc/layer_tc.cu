@@ -17,7 +17,9 @@
 //                    The row copies of a CTA's last work item meet in the ring, idle by then, in one round.
 // The ring's six 32 KiB stages serve the scoring phase as three 64 KiB stages; the producer starts the
 // attention copies into a stage as soon as the scoring tiles that last used its pair have been
-// consumed, so the stream of bytes into the SM never stops between the phases.  The scoring ranges
+// consumed, so the stream of bytes into the SM never stops between the phases.  (With 64 scoring rows the two
+// 32 KiB operand buffers leave room for four stages only; they become stages 4 and 5 of the attention phase once the
+// last scoring MMA has completed.)  The scoring ranges
 // are sized so that every SM moves the same number of bytes: a CTA with one more attention row of n
 // tiles (32 KiB each) gets n / 2 fewer scoring tiles (64 KiB each) than the others.
 // Scoring comes first because it needs nothing from the previous layer (draft queries and summaries
@@ -27,7 +29,7 @@
 // (griddepcontrol.wait) before touching the attention inputs.  SMs are thus handed from one layer to
 // the next one by one, without the idle time around a kernel boundary.
 //   warp 0     TMA producer of both phases
-//   warp 1     issues the scoring MMAs, then Q K^T
+//   warp 1     issues the scoring MMAs, then Q K^T  (both issuing warps run converged, elect.sync picks the lane)
 //   warp 2     issues P V
 //   warps 3-6  scoring epilogue, then Q into tensor memory, softmax and write-out of the attention row
 //   warp 7     builds the (q^- | q^+) operands of the CTA's scoring range ahead of time
