@@ -62,7 +62,10 @@ def parse_args():
     ap.add_argument("--wait-group", type=int, default=0,
                     help="layers per pick-up of the side streams' events (0: a quarter of the layers, at most 8)")
     ap.add_argument("--transfer-group", type=int, default=0,
-                    help="layers per gather launch when the pool is in host memory (0: up to 4 when the host link bounds the step, else 1)")
+                    help="layers per gather launch when the pool is in host memory (0: up to 8 when the host link bounds the step, else 2)")
+    ap.add_argument("--transfer-kind", default="", choices=["", "warp", "bulk"],
+                    help="gather from host memory: warp per entry, or bulk copies through shared memory (default: bulk where "
+                         "the host link bounds the step)")
     ap.add_argument("--repeats", type=int, default=1, help="replay the timed steps this many times in a second, long "
                                                             "timed region (reported as `sustained`)")
     ap.add_argument("--sweep-ratios", default="", help="comma-separated fetch ratios to sweep (e.g. 0.01,0.02,0.05)")
@@ -299,15 +302,19 @@ class Bench:
 
     def transfer_group(self, w, cap):
         """Layers per gather launch from pinned host memory.  Where the link bounds the step (the gathered bytes of a
-        layer take longer than its scoring + attention), four layers per launch keep the link busier (0.89 against 0.85
-        of the copy-engine rate); where compute bounds it, one launch per layer disturbs the compute least."""
+        layer take longer than its scoring + attention), eight layers per launch of the bulk gather keep the link
+        busiest (0.90 of the copy-engine rate; 0.88 with two); where compute bounds it, two layers per launch of the
+        warp gather with 32 thread blocks disturb the compute and the query uploads least."""
         if self.args.transfer_group > 0:
             return self.args.transfer_group
+        return max(1, min(8 if self.link_bound(w, cap) else 2, self.cfg.layers // 4))
+
+    def link_bound(self, w, cap):
         cfg = self.cfg
         link_us = cap * cfg.batch * cfg.n_kv_heads * 8192 / (0.9 * self.h2d_peak * 1e3)
         score, attn = algorithmic_bytes(cfg, w.k, w.T, self.seq_steps, [0])
         compute_us = (score + attn) / (0.85 * self.hbm_peak * 1e3)
-        return max(1, min(4, cfg.layers // 4)) if link_us > compute_us else 1
+        return link_us > compute_us
 
     def wait_group(self):
         """Layers whose side-stream events the foreground stream picks up together: few enough that a step's last
@@ -325,10 +332,12 @@ class Bench:
                                          transfer_streams=getattr(self.args, "transfer_streams", 1),
                                          plan_stream=getattr(self.args, "plan_stream", "own"), wait_group=self.wait_group(),
                                          n_commit=getattr(self.args, "n_commit", 1),
-                                         # (compute-bound steps: a smaller gather launch disturbs the fused kernel less and
-                                         #  is itself less disturbed -- 1.74 against 1.92-1.98 ms per step at fetch ratio 0.02)
+                                         # (pool in pinned host memory: bulk gather where the link bounds the step, else a
+                                         #  small warp gather -- 32 thread blocks -- that disturbs the fused kernel least)
+                                         transfer_kind=(getattr(self.args, "transfer_kind", "") or
+                                                        ("bulk" if host_pool and self.link_bound(w, cap) else "warp")),
                                          transfer_ctas=(getattr(self.args, "transfer_ctas", 0) or
-                                                        (32 if self.transfer_group(w, cap) == 1 else 0)) if host_pool else 0,
+                                                        (32 if host_pool and not self.link_bound(w, cap) else 0)),
                                          transfer_group=self.transfer_group(w, cap) if host_pool else 1)
         for l in range(self.n_layers):
             eng.attach(l, kv_list[l], self.tables[l])
@@ -750,9 +759,11 @@ def run_ours(args):
                        "gather": "delta selection with capped eviction, fetch ratio %.2f (cap %d blocks per head per step); local "
                                  "blocks appended on the GPU" % (args.fetch_ratio, cap),
                        "launch": "CUDA graphs of %d consecutive decode steps over 6-10 streams; a layer's attention and scoring are "
-                                 "one fused launch (oasis_attn_and_score); gathers of %d layers per launch; side-stream events "
-                                 "picked up every %d layers" % (args.group if args.group > 0 else K, bench.transfer_group(w, cap),
-                                                                 bench.wait_group())},
+                                 "one fused launch (oasis_attn_and_score); %s gathers of %d layers per launch; side-stream "
+                                 "events picked up every %d layers"
+                                 % (args.group if args.group > 0 else K,
+                                    args.transfer_kind or ("bulk (copy unit)" if bench.link_bound(w, cap) else "warp-per-entry"),
+                                    bench.transfer_group(w, cap), bench.wait_group())},
             "gpu_launches": host.get("launches"),
             "clocks": {kk: (host.get("clocks") or {}).get(kk) for kk in ("sm_mhz", "sm_max_mhz", "reasons", "samples")},
             "roofline": {"bound": "hbm", "kernel": dom, "achieved": d.get("GBps"), "peak": hbm_peak, "unit": "GB/s",

@@ -175,6 +175,20 @@ int oasis_stage_blocks_layers(int32_t n_layers, const void *const *host_kvs, con
                               void *stream);
 
 /*
+ * Step 3 for several layers in one launch, through the copy unit: the same result as oasis_stage_blocks_layers, but the
+ * entries move as 8 KiB bulk copies (CPU pool -> shared memory -> working-set pool) issued by one thread of a
+ * small thread block per entry stream, so that the gather runs beside kernels that fill the SMs (the fused
+ * attention + scoring launch) without competing for their issue slots.  Faster than the warp-per-entry gather where
+ * the host link bounds the decode step; no better where compute bounds it.  A copy that does not complete within
+ * the library's bounded wait records code 71 in the error word.
+ *   max_streams   entry streams (thread blocks) of the launch, shared among the layers, each with one 8 KiB copy
+ *                 in flight; 0 = the library's default of 128 (1 MiB in flight).
+ */
+int oasis_stage_blocks_bulk(int32_t n_layers, const void *const *host_kvs, const int64_t *const *idx,
+                            const int32_t *const *slots, int32_t n, void *const *hbm_pools,
+                            int32_t max_streams, void *stream);
+
+/*
  * Step 4 -- sparse paged decode attention over the staged working set (Sec. 4.2.1: the
  * stacked normal and draft queries run over one resident KV working set in one call;
  * Sec. 4.3: the selected key and value blocks share one ordering).

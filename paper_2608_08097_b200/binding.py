@@ -24,7 +24,7 @@ SYMBOLS = ("oasis_build_summaries", "oasis_score_blocks", "oasis_select_topk",
            "oasis_sparse_attn_static_scratch", "oasis_static_scratch_bytes", "oasis_set_error_word", "oasis_union_blocks",
            "oasis_offload_blocks", "oasis_attn_and_score", "oasis_attn_and_score_supported",
            "oasis_build_summaries_layers", "oasis_selftest_wait_timeout",
-           "oasis_local_window", "oasis_append_kv", "oasis_append_kv_layers", "oasis_stage_blocks_layers",
+           "oasis_local_window", "oasis_append_kv", "oasis_append_kv_layers", "oasis_stage_blocks_layers", "oasis_stage_blocks_bulk",
            "oasis_set_extents", "oasis_bounds_checked")
 
 
@@ -93,6 +93,8 @@ def lib():
         L.oasis_union_blocks.restype = ctypes.c_int
         L.oasis_stage_blocks_layers.argtypes = [i32, vp, vp, vp, i32, vp, i32, vp]
         L.oasis_stage_blocks_layers.restype = ctypes.c_int
+        L.oasis_stage_blocks_bulk.argtypes = [i32, vp, vp, vp, i32, vp, i32, vp]
+        L.oasis_stage_blocks_bulk.restype = ctypes.c_int
         L.oasis_local_window.argtypes = [dp, vp, i32, vp, vp, i32, i32, i32, vp, vp, vp]
         L.oasis_local_window.restype = ctypes.c_int
         L.oasis_append_kv.argtypes = [dp, vp, i32, i32, vp, vp, vp, vp, i32, i32, vp, vp, vp]
@@ -385,3 +387,16 @@ def stage_blocks_layers(host_kvs, idx, slots, n, hbm_pools, max_ctas=0, stream=N
     _check(lib().oasis_stage_blocks_layers(
         nl, mk(host_kvs, torch.bfloat16, "host_kvs"), mk(idx, torch.int64, "idx"), mk(slots, torch.int32, "slots"), int(n),
         mk(hbm_pools, torch.bfloat16, "hbm_pools"), int(max_ctas), _stream(stream)), "oasis_stage_blocks_layers")
+
+
+def stage_blocks_bulk(host_kvs, idx, slots, n, hbm_pools, max_streams=0, stream=None):
+    """oasis_stage_blocks_bulk: the several-layers gather through the copy unit (same arguments and result as
+    stage_blocks_layers; `max_streams` entry streams, 0 = the library's default)."""
+    nl = len(host_kvs)
+    if not all(len(x) == nl for x in (idx, slots, hbm_pools)):
+        raise ValueError("one tensor per layer is needed in every list")
+    arr = ctypes.c_void_p * max(nl, 1)
+    mk = lambda ts, dt, nm: arr(*[_ptr(t, dt, nm).value for t in ts])
+    _check(lib().oasis_stage_blocks_bulk(
+        nl, mk(host_kvs, torch.bfloat16, "host_kvs"), mk(idx, torch.int64, "idx"), mk(slots, torch.int32, "slots"), int(n),
+        mk(hbm_pools, torch.bfloat16, "hbm_pools"), int(max_streams), _stream(stream)), "oasis_stage_blocks_bulk")

@@ -118,6 +118,8 @@ class DecodeEngine:
     transfer_group: the gathers of this many consecutive layers are one launch (`oasis_stage_blocks_layers`): a
     few large gathers keep the host link busier than many small ones; a layer's next-step attention then waits
     for its group's launch.
+    transfer_kind: "warp" = the warp-per-entry zero-copy gather, "bulk" = `oasis_stage_blocks_bulk` (8 KiB bulk copies
+    through shared memory: the faster one where the host link bounds the step).
     wait_group: the foreground stream picks up the other streams' events (a layer's transfer, query
     upload and output download of the previous step) for `wait_group` layers at a time, in front of the
     group's first launch.  A fused launch that follows a cross-stream wait is fully serialised behind
@@ -127,11 +129,14 @@ class DecodeEngine:
 
     def __init__(self, batch, n_q_heads, n_kv_heads, max_blocks, k, n_q_tokens, n_layers,
                  device="cuda", mode="fetch_all", cap=None, fused=None, transfer_streams=1, wait_group=8,
-                 append=False, transfer_group=1, plan_stream="own", n_commit=1, transfer_ctas=0):
+                 append=False, transfer_group=1, plan_stream="own", n_commit=1, transfer_ctas=0, transfer_kind="warp"):
         assert mode in ("fetch_all", "delta")
         assert not append or mode == "delta", "the KV append goes with delta selection"
         self.append = bool(append)
         self.transfer_ctas = int(transfer_ctas)  # thread blocks per gather launch (0: the library's default)
+        if transfer_kind not in ("warp", "bulk"):
+            raise ValueError("transfer_kind must be 'warp' or 'bulk'")
+        self.transfer_kind = transfer_kind       # warp-per-entry zero-copy gather, or bulk copies through shared memory
         self.n_commit = int(n_commit)            # tokens per step that the KV append also writes to the full-KV pool
         self.mode, self.k, self.T, self.n_layers = mode, k, n_q_tokens, n_layers
         self.device = torch.device(device)
@@ -268,7 +273,10 @@ class DecodeEngine:
             else:
                 idx = [self.layers[l].stage_idx for l in ls]
                 slots = [self.layers[l].stage_slots for l in ls]
-            if len(ls) == 1 and self.transfer_ctas == 0:
+            if self.transfer_kind == "bulk":
+                oasis.stage_blocks_bulk([self.kv[l] for l in ls], idx, slots, idx[0].numel(),
+                                        [self.layers[l].pool for l in ls], max_streams=self.transfer_ctas)
+            elif len(ls) == 1 and self.transfer_ctas == 0:
                 oasis.stage_blocks(self.kv[ls[0]], idx[0], slots[0], idx[0].numel(), self.layers[ls[0]].pool)
             else:
                 oasis.stage_blocks_layers([self.kv[l] for l in ls], idx, slots, idx[0].numel(),

@@ -283,6 +283,42 @@ def test_stage_skips_negative_and_keeps_other_slots(oracle, gpu):
     binding.stage_blocks(host, torch.from_numpy(idx).to(dev), torch.from_numpy(slots).to(dev), 0, pool)   # n = 0: no-op
 
 
+@pytest.mark.parametrize("src", ["pinned", "device"])
+@pytest.mark.parametrize("n,streams", [(1, 0), (7, 0), (150, 0), (768, 0), (3001, 0), (150, 3), (768, 1024)])
+@pytest.mark.parametrize("kind", ["warp", "bulk"])
+def test_stage_several_layers_in_one_launch(oracle, gpu, kind, src, n, streams):
+    """The several-layers gathers (warp per entry; bulk copies through shared memory): byte-exact per layer against the
+    oracle, skipped requests, untouched slots, lists shorter and longer than the number of thread blocks, the error
+    word stays 0."""
+    binding, _ = gpu
+    dev = torch.device("cuda")
+    rng = np.random.default_rng(17 + n)
+    n_layers, n_host, n_slots = 3, 4000, 3500
+    err = torch.zeros(1, dtype=torch.int32, device=dev)
+    binding.set_error_word(err)
+    try:
+        hosts, idxs, slotss, pools, wants = [], [], [], [], []
+        for l in range(n_layers):
+            h = torch.from_numpy(rng.integers(0, 2 ** 15, (n_host, 2, 16, 128), dtype=np.int16)).view(torch.bfloat16)
+            h = h.pin_memory() if src == "pinned" else h.to(dev)
+            idx = rng.integers(0, n_host, n).astype(np.int64)
+            idx[::5] = -1
+            slots = rng.permutation(n_slots)[:n].astype(np.int32)
+            hosts.append(h); idxs.append(idx); slotss.append(slots)
+            pools.append(torch.from_numpy(np.full((n_slots, 2, 16, 128), 0x3ABC + l, np.int16)).view(torch.bfloat16).to(dev))
+            want = np.full((n_slots, 2, 16, 128), 0x3ABC + l, np.uint16)
+            oracle.stage_blocks(pu.np_u16(h), idx, slots, want)
+            wants.append(want)
+        fn = binding.stage_blocks_layers if kind == "warp" else binding.stage_blocks_bulk
+        fn(hosts, [torch.from_numpy(i).to(dev) for i in idxs], [torch.from_numpy(s_).to(dev) for s_ in slotss], n, pools, streams)
+        torch.cuda.synchronize()
+        for l in range(n_layers):
+            assert np.array_equal(pu.np_u16(pools[l]), wants[l]), "layer %d" % l
+        assert int(err.item()) == 0
+    finally:
+        binding.set_error_word(None)
+
+
 def test_attention_padding_rows_and_empty_columns(oracle, gpu):
     """Columns of -1 anywhere in the table (not only at the end), rows that see nothing."""
     binding, pipeline = gpu
