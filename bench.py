@@ -301,20 +301,38 @@ class Bench:
         self.gen_seconds = time.time() - t0
 
     def transfer_group(self, w, cap):
-        """Layers per gather launch from pinned host memory.  Where the link bounds the step (the gathered bytes of a
-        layer take longer than its scoring + attention), eight layers per launch of the bulk gather keep the link
-        busiest (0.90 of the copy-engine rate; 0.88 with two); where compute bounds it, two layers per launch of the
-        warp gather with 32 thread blocks disturb the compute and the query uploads least."""
+        """Layers per gather launch from pinned host memory, from the ratio of a layer's gather time on the link to its
+        scoring + attention time.  Measured (step in ms, bulk gather unless noted): configs[1] (32 layers, ratio 3): 4.01
+        with 8 layers per launch, 4.03 with 4, 4.11 with 2; configs[3] (8 layers, ratio 2.4): 1.11 with 4, 1.25 with 2,
+        1.27 with 1; configs[2] (4 layers, ratio 1.3): 1.11 with 1, 1.17 with 2, 2.05 with 4 (the whole step's transfers
+        then wait for its last layer); configs[1] at fetch ratio 0.02 (ratio 0.85, warp gather): 1.67 with 2, 1.75
+        with 1 or 4; far below the break-even one launch per layer is best (configs[0]: 0.55-0.60 against 0.67-0.69 end
+        to end)."""
         if self.args.transfer_group > 0:
             return self.args.transfer_group
-        return max(1, min(8 if self.link_bound(w, cap) else 2, self.cfg.layers // 4))
+        r, layers = self.link_ratio(w, cap), self.cfg.layers
+        if r > 2.0 and layers >= 8:
+            return min(8, layers // 2)
+        if r > 1.0:
+            return max(1, min(8, layers // 4))
+        # near the break-even two layers per launch, unless a layer is so short that waiting for the second one's plan
+        # costs more than the launch saves
+        return max(1, min(2, layers // 4)) if r > 0.5 and self.compute_us(w) >= 30.0 else 1
 
-    def link_bound(self, w, cap):
+    def link_ratio(self, w, cap):
+        """A layer's gathered bytes at 0.9 of the pinned copy peak over its scoring + attention bytes at 0.85 of the HBM
+        copy peak: above 1 the host link bounds the step."""
         cfg = self.cfg
         link_us = cap * cfg.batch * cfg.n_kv_heads * 8192 / (0.9 * self.h2d_peak * 1e3)
-        score, attn = algorithmic_bytes(cfg, w.k, w.T, self.seq_steps, [0])
-        compute_us = (score + attn) / (0.85 * self.hbm_peak * 1e3)
-        return link_us > compute_us
+        return link_us / self.compute_us(w)
+
+    def compute_us(self, w):
+        """A layer's scoring + attention bytes at 0.85 of the HBM copy peak, at least the 10 us a fused launch takes."""
+        score, attn = algorithmic_bytes(self.cfg, w.k, w.T, self.seq_steps, [0])
+        return max(10.0, (score + attn) / (0.85 * self.hbm_peak * 1e3))
+
+    def link_bound(self, w, cap):
+        return self.link_ratio(w, cap) > 1.0
 
     def wait_group(self):
         """Layers whose side-stream events the foreground stream picks up together: few enough that a step's last
