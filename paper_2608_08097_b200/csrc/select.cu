@@ -287,7 +287,10 @@ extern "C" int oasis_select_topk(const oasis_dims_t *dims, const float *scores,
     while (sort_len < k) sort_len <<= 1;
     p.sort_len = sort_len;
     int threads = 128;
-    while (threads < 1024 && threads * 8 < dims->max_blocks) threads <<= 1;    // ~8 keys per thread
+    // about 4 keys per thread: the kernel runs beside the fused attention + scoring kernel, and the shorter it is there
+    // the less it costs that kernel (compute-only step of the reasoning-style workload: 1.71 ms with 256 threads per
+    // row, 1.60 with 512, 1.58-1.62 with 1,024; with 128 and fewer the top-k itself becomes the step's bottleneck)
+    while (threads < 1024 && threads * 4 < dims->max_blocks) threads <<= 1;
     const size_t smem = (size_t)sort_len * 8 + (size_t)dims->max_blocks * 4;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
