@@ -124,6 +124,18 @@ def profile_traffic(name="c2_layer_tcgen05_kernel.md"):
     return None
 
 
+def pick_transfer_group(link_ratio, layers, compute_us):
+    """Layers per gather launch for a step whose layers spend `link_ratio` times as long on the host link as on scoring +
+    attention (`compute_us` per layer); the measurements behind the thresholds are listed in Bench.transfer_group."""
+    if link_ratio > 2.0 and layers >= 8:
+        return min(8, layers // 2)
+    if link_ratio > 1.0:
+        return max(1, min(8, layers // 4))
+    # near the break-even two layers per launch, unless a layer is so short that waiting for the second one's plan
+    # costs more than the launch saves
+    return max(1, min(2, layers // 4)) if link_ratio > 0.5 and compute_us >= 30.0 else 1
+
+
 class ClockSampler:
     """Samples the SM clock and the clock-event (throttle) reasons through NVML, read-only,
     every few milliseconds from a thread while a timed region runs."""
@@ -310,14 +322,7 @@ class Bench:
         to end)."""
         if self.args.transfer_group > 0:
             return self.args.transfer_group
-        r, layers = self.link_ratio(w, cap), self.cfg.layers
-        if r > 2.0 and layers >= 8:
-            return min(8, layers // 2)
-        if r > 1.0:
-            return max(1, min(8, layers // 4))
-        # near the break-even two layers per launch, unless a layer is so short that waiting for the second one's plan
-        # costs more than the launch saves
-        return max(1, min(2, layers // 4)) if r > 0.5 and self.compute_us(w) >= 30.0 else 1
+        return pick_transfer_group(self.link_ratio(w, cap), self.cfg.layers, self.compute_us(w))
 
     def link_ratio(self, w, cap):
         """A layer's gathered bytes at 0.9 of the pinned copy peak over its scoring + attention bytes at 0.85 of the HBM

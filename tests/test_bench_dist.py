@@ -44,3 +44,22 @@ def test_reference_arm_under_torchrun_prints_once():
     assert len(lines) == 1 and lines[0]["impl"] == "reference"
     assert lines[0]["cpu_baseline"]["kind"] == "oracle" and lines[0]["e2e"]["h2d_bytes_per_step"] == 0
     assert lines[0]["value"] > 0
+
+
+def test_gather_grouping_follows_the_measured_regimes():
+    """Layers per gather launch as a function of the link / compute ratio of a layer, the layer count and the layer's
+    compute time: the five configurations' operating points and the edges of the rule."""
+    sys.path.insert(0, ROOT)
+    import bench
+    pick = bench.pick_transfer_group
+    assert pick(3.0, 32, 41.0) == 8          # configs[1] at fetch ratio 0.05: strongly link-bound, many layers
+    assert pick(2.4, 8, 51.0) == 4           # configs[3]: half of its 8 layers
+    assert pick(1.3, 4, 196.0) == 1          # configs[2]: mildly link-bound, 4 layers: one launch per layer
+    assert pick(3.0, 4, 60.0) == 1           # few layers never share one launch, however link-bound
+    assert pick(0.85, 32, 44.0) == 2         # configs[1] at fetch ratio 0.02: near the break-even
+    assert pick(0.43, 32, 44.0) == 1         # far below it
+    assert pick(0.8, 32, 10.0) == 1          # configs[0]: layers too short to wait for a second plan
+    for r in (0.0, 0.4, 0.6, 1.0, 1.5, 2.5, 10.0):
+        for layers in (1, 2, 4, 8, 32, 64):
+            g = pick(r, layers, 50.0)
+            assert 1 <= g <= max(1, min(8, layers))
