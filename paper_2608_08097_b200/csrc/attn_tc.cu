@@ -29,6 +29,11 @@
 //              the M rows they are replicated (2 or 4 copies) and each copy takes its share of the
 //              tile's four blocks, writing P = 0 for the others.  The copies' partial (max, sum, O)
 //              are merged through shared memory after the last tile.
+//   warps 7-10 only with 65 to 128 query rows (one copy of the rows in 128 MMA rows): a second set of
+//              softmax warps.  The two sets take alternate tiles, each with a running maximum, sum
+//              and O accumulator of its own (P V of even tiles goes to the first O, of odd tiles to
+//              the second; three S buffers), so that one set's waits and tensor-memory traffic
+//              overlap the other's exponentials; the two threads of a row merge when it is written.
 // After the merge the rows are normalised and written as bf16 (or, when the column list is
 // split, as a normalised partial plus its log-sum-exp to the workspace).
 // Every wait is bounded; a timeout records a code in the error word and the CTA winds down.
@@ -44,6 +49,8 @@
 namespace oasis {
 
 constexpr int kAtThreads = 224;                             // producer, Q K^T issuer, P V issuer, four softmax warps
+// (four more with two softmax sets)
+__host__ __device__ constexpr int at_threads(int mma_m, int copies) { return kAtThreads + (at_softmax_sets(mma_m, copies) - 1) * 128; }
 struct AttnTcParams {
     const uint8_t *q;
     const int32_t *slot_tbl;
@@ -62,13 +69,15 @@ struct AttnTcParams {
 // MMA_M = 64 halves the tensor work when the query rows fit; its rows live in tensor-memory lanes
 // (m % 16) + 32 * (m / 16), i.e. sixteen per softmax warp.
 template <int MMA_M, int COPIES>
-__global__ void __launch_bounds__(kAtThreads, 1)
+__global__ void __launch_bounds__(at_threads(MMA_M, COPIES), 1)
 sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcParams p)
 {
     constexpr int RPC = MMA_M / COPIES;                     // MMA rows per copy of the query rows
     constexpr int LANES = MMA_M / 4;                        // lanes of each softmax warp that hold an MMA row
     constexpr int BPC = kAtTileCols / COPIES;               // blocks of a tile each copy handles
-    constexpr int KPC = BPC * kBlock;                       // keys of a tile each copy handles
+    constexpr int SETS = at_softmax_sets(MMA_M, COPIES);    // softmax warp sets, taking alternate tiles
+    constexpr int SBUFS = at_s_bufs(SETS);                  // S / P buffers in tensor memory
+    constexpr int THREADS = at_threads(MMA_M, COPIES);
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -115,7 +124,7 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
             asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
         }
         uint4 v[16];
-        if (warp >= 3) {
+        if (warp >= 3 && warp < 7) {
             const int m_row = (warp & 3) * LANES + lane;
             const int r = m_row % RPC;
 #pragma unroll
@@ -128,16 +137,16 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
             }
         }
         tc_fence_before();
-        asm volatile("bar.sync 2, %0;" ::"n"(kAtThreads - 32) : "memory");
+        asm volatile("bar.sync 2, %0;" ::"n"(THREADS - 32) : "memory");
         tc_fence_after();
         tmem_base = *tmem_slot;
-        tmem_o = tmem_base + kAtSBufs * kAtTileKeys;
-        tmem_q = tmem_o + kHeadDim;                                  // Q as the A operand: 128 rows x 64 packed columns
-        if (warp >= 3) {
+        tmem_o = tmem_base + SBUFS * kAtTileKeys;
+        tmem_q = tmem_o + SETS * kHeadDim;                           // Q as the A operand: 128 rows x 64 packed columns
+        if (warp >= 3 && warp < 7) {
             q_row_to_tmem(tmem_q + ((uint32_t)((warp & 3) * 32) << 16), v);
         }
         tc_fence_before();
-        asm volatile("bar.sync 2, %0;" ::"n"(kAtThreads - 32) : "memory");
+        asm volatile("bar.sync 2, %0;" ::"n"(THREADS - 32) : "memory");
         tc_fence_after();
     }
 
@@ -170,11 +179,11 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
             // descriptors: the operand start address occupies the low 14 bits (16-byte units), so offsets are added there
             const uint64_t k_desc0 = smem_desc_sw128_k(kv_u32, kImgGroup);
             bool alive = true;
-            int s = 0, sb = 0, s_old = 0;                            // stage and S buffer of tile i; stage of tile i - kAtSBufs
+            int s = 0, sb = 0, s_old = 0;                            // stage and S buffer of tile i; stage of tile i - SBUFS
             uint32_t ph = 0, ph_old = 0;
             for (int i = 0; i < n_tiles && alive; ++i) {
-                // the S buffer also held P of tile i - kAtSBufs: its P V must have completed
-                if (i >= kAtSBufs) {
+                // the S buffer also held P of tile i - SBUFS: its P V must have completed
+                if (i >= SBUFS) {
                     alive = mbar_wait_warp(bar_empty(s_old), ph_old, p.err, 51);
                     ph_old ^= (s_old + 1 == p.stages);
                     s_old = (s_old + 1 == p.stages) ? 0 : s_old + 1;
@@ -188,7 +197,7 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
                 tc_commit(bar_s_full(sb));
                 ph ^= (s + 1 == p.stages);
                 s = (s + 1 == p.stages) ? 0 : s + 1;
-                sb = (sb + 1) & (kAtSBufs - 1);
+                sb = (sb + 1 == SBUFS) ? 0 : sb + 1;
             }
         }
     } else if (warp == 2) {
@@ -205,15 +214,18 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
                 tc_fence_after();
                 const uint64_t v_desc = v_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
                 const uint32_t p_tmem = tmem_base + (uint32_t)(sb * kAtTileKeys);
-                issue_pv_tile(tmem_o, p_tmem, v_desc, idesc, i == 0);
+                // (two softmax sets: even tiles accumulate into the first O, odd tiles into the second)
+                issue_pv_tile(tmem_o + (uint32_t)((i % SETS) * kHeadDim), p_tmem, v_desc, idesc, i < SETS);
                 tc_commit(bar_empty(s));                             // stage free, and O complete up to this tile
                 s = (s + 1 == p.stages) ? 0 : s + 1;
-                sb = (sb + 1) & (kAtSBufs - 1);
+                sb = (sb + 1 == SBUFS) ? 0 : sb + 1;
                 ph_p ^= (sb == 0);
             }
         }
     } else {
-        // ---------------------------------------------------------------- softmax, one thread per MMA row
+        // ---------------------------------------------------------------- softmax, one thread per MMA row (two sets: warps
+        // 3-6 take the even tiles, warps 7-10 the odd ones)
+        const int set = SETS == 2 ? (warp - 3) >> 2 : 0;
         const int quarter = warp & 3;
         const int m_row = quarter * LANES + (lane % LANES);         // MMA row held by this tensor-memory lane
         const int copy = m_row / RPC, row = m_row % RPC;            // which copy of the rows, which query row
@@ -226,25 +238,34 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         float m_ref = -CUDART_INF_F, l_sum = 0.f;
         bool alive = true;
-        int s = 0, s_prev = 0;                                      // ring stage of tile i and of tile i - 1
-        uint32_t ph_prev = 0;                                       // parity of the "empty" phase that ends tile i - 1
-        for (int i = 0; i < n_tiles && alive; ++i) {
-            alive = mbar_wait(bar_s_full(i % kAtSBufs), (i / kAtSBufs) & 1, p.err, 61);
+        int s = 0, s_prev = 0;                                      // ring stage of tile i and of this set's previous tile
+        uint32_t ph = 0, ph_prev = 0;                               // parities of the "empty" phases that end those tiles
+        int sb = set;                                               // S buffer of tile i (SETS < SBUFS)
+        uint32_t ph_s = 0;
+        ring_advance(s, ph, set, p.stages);
+        const uint32_t my_o = tmem_o + (uint32_t)(set * kHeadDim) + lane_base;   // this thread's O row
+        for (int i = set; i < n_tiles && alive; i += SETS) {
+            alive = mbar_wait(bar_s_full(sb), ph_s, p.err, 61);
             if (!alive) break;
             tc_fence_after();
-            const uint32_t s_tmem = tmem_base + lane_base + (uint32_t)((i % kAtSBufs) * kAtTileKeys);
+            const uint32_t s_tmem = tmem_base + lane_base + (uint32_t)(sb * kAtTileKeys);
             if (live_warp)
-                alive = softmax_tile<COPIES>(s_tmem, tmem_o + lane_base, tile_blk + s * kAtTileCols, copy, limit, has_row,
-                                             p.scale_log2, m_ref, l_sum, i > 0,
-                                             // (the previous tile's stage is released by the commit that follows its P V; with
-                                             // at least four stages in the ring the phase parity of that barrier is unambiguous)
+                alive = softmax_tile<COPIES>(s_tmem, my_o, tile_blk + s * kAtTileCols, copy, limit, has_row,
+                                             p.scale_log2, m_ref, l_sum, i >= SETS,
+                                             // (the stage of this set's previous tile is released by the commit that follows its
+                                             // P V; with at least four stages in the ring the phase parity is unambiguous)
                                              [&] { return mbar_wait(bar_empty(s_prev), ph_prev, p.err, 62); });
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_p_full(i % kAtSBufs));
-            if (i > 0) ph_prev ^= (s_prev + 1 == p.stages);
+            if (lane == 0) mbar_arrive(bar_p_full(sb));
             s_prev = s;
-            s = (s + 1 == p.stages) ? 0 : s + 1;
+            ph_prev = ph;
+            ring_advance(s, ph, SETS, p.stages);
+#pragma unroll
+            for (int k = 0; k < SETS; ++k) {
+                sb = (sb + 1 == SBUFS) ? 0 : sb + 1;
+                ph_s ^= (sb == 0);
+            }
         }
         // ---- epilogue: merge the copies, normalise, write out ----------------------------------------------
         if (alive && n_tiles > 0)
@@ -253,8 +274,54 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
         // the K/V ring is idle now: stage the O rows there.  [128 MMA rows][132 floats], then max and sum.
         float *o_sm = reinterpret_cast<float *>(base_ptr + kAtQBytes);
         float *m_sm = o_sm + 128 * 132;
-        float *l_sm = m_sm + 128;
-        if (COPIES > 1) {
+        float *l_sm = m_sm + 128 * SETS;
+        if (SETS == 2) {
+            // the two threads of a row exchange maximum and sum; each then merges and writes one half of the output dims,
+            // reading both O accumulators at its own tensor-memory lane
+            m_sm[set * 128 + m_row] = m_ref;
+            l_sm[set * 128 + m_row] = l_sum;
+            asm volatile("bar.sync 1, 256;" ::: "memory");          // the eight softmax warps
+            const float m_o = m_sm[(set ^ 1) * 128 + m_row], l_o = l_sm[(set ^ 1) * 128 + m_row];
+            const float mx = fmaxf(m_ref, m_o);
+            const float w_me = mx == -CUDART_INF_F ? 0.f : fast_exp2(m_ref - mx), w_ot = mx == -CUDART_INF_F ? 0.f : fast_exp2(m_o - mx);
+            const float den = w_me * l_sum + w_ot * l_o;
+            const float inv = den > 0.f ? 1.f / den : 0.f;
+            const float lse2 = den > 0.f ? mx + log2f(den) : -CUDART_INF_F;
+            const float w_a = set == 0 ? w_me : w_ot, w_b = set == 0 ? w_ot : w_me;   // weights of the first and second accumulator
+            const int tq = row / p.G, a = h * p.G + row % p.G;
+            const long long orow = ((long long)b * p.T + tq) * p.Hq + a;
+            const bool run = n_tiles > 0 && live_warp && alive;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                const int d0 = set * 64 + c * 16;
+                uint32_t va[16], vb[16];
+                if (run) {
+                    tc_ld16(tmem_o + lane_base + d0, va);
+                    tc_ld16(tmem_o + kHeadDim + lane_base + d0, vb);
+                }
+                if (!(live_row && alive)) continue;
+                float acc[16];
+                // an accumulator whose set saw no key (weight 0) was never written: its contents do not enter
+#pragma unroll
+                for (int e = 0; e < 16; ++e)
+                    acc[e] = ((w_a != 0.f ? w_a * __uint_as_float(va[e]) : 0.f) + (w_b != 0.f ? w_b * __uint_as_float(vb[e]) : 0.f)) * inv;
+                if (p.n_splits == 1) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(p.out + (orow * kHeadDim + d0) * 2);
+#pragma unroll
+                    for (int e = 0; e < 2; ++e)
+                        dst[e] = make_uint4(pack_bf16x2(acc[8 * e], acc[8 * e + 1]), pack_bf16x2(acc[8 * e + 2], acc[8 * e + 3]),
+                                            pack_bf16x2(acc[8 * e + 4], acc[8 * e + 5]), pack_bf16x2(acc[8 * e + 6], acc[8 * e + 7]));
+                } else {
+                    float4 *dst = reinterpret_cast<float4 *>(p.part_o + ((long long)blockIdx.x * p.R + row) * kHeadDim + d0);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) dst[e] = make_float4(acc[4 * e], acc[4 * e + 1], acc[4 * e + 2], acc[4 * e + 3]);
+                }
+            }
+            if (live_row && alive && set == 0) {
+                if (p.n_splits == 1) { if (p.lse) p.lse[orow] = lse2 * kAtLn2; }
+                else p.part_lse[(long long)blockIdx.x * p.R + row] = lse2;
+            }
+        } else if (COPIES > 1) {
             if (live_warp && alive && n_tiles > 0) {
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
@@ -273,7 +340,7 @@ sparse_attn_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnTcPara
             }
             asm volatile("bar.sync 1, 128;" ::: "memory");          // the four softmax warps
         }
-        {
+        if (SETS == 1) {
             // thread -> (query row, slice of the 128 output dims)
             // one copy: the thread that holds a row writes it; several copies: the MMA_M (row, slice) tasks go to
             // the first MMA_M softmax threads
@@ -402,7 +469,7 @@ int launch_attn_tc(const oasis_dims_t *dims, const void *q, int n_q_tokens, cons
 #define OASIS_ATTN_TC_LAUNCH(M, C)                                                                                     \
     do {                                                                                                               \
         e = cudaFuncSetAttribute(sparse_attn_tc_kernel<M, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
-        if (e == cudaSuccess) sparse_attn_tc_kernel<M, C><<<(unsigned)grid, kAtThreads, smem, st>>>(tmap, p);          \
+        if (e == cudaSuccess) sparse_attn_tc_kernel<M, C><<<(unsigned)grid, at_threads(M, C), smem, st>>>(tmap, p);          \
     } while (0)
     if (p.R <= 16) OASIS_ATTN_TC_LAUNCH(64, 4);          // four copies of <= 16 rows, one block of a tile each
     else if (p.R <= 32) OASIS_ATTN_TC_LAUNCH(64, 2);     // two copies of <= 32 rows, two blocks each

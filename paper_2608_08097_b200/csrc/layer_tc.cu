@@ -33,6 +33,8 @@
 //   warp 2     issues P V
 //   warps 3-6  scoring epilogue, then Q into tensor memory, softmax and write-out of the attention row
 //   warp 7     builds the (q^- | q^+) operands of the CTA's scoring range ahead of time
+//   warps 8-11 only with 65 to 128 query rows: the second set of softmax warps (alternate tiles, own O accumulator;
+//              see attn_tc.cu); idle in the scoring phase
 // Every wait is bounded; a time-out records a code in the error word and the CTA winds down.
 // Algorithmic traffic: 8 KiB per (request, KV head, column) + Q / O, and 512 B + 4 B per scored block.
 #include <cuda.h>
@@ -43,7 +45,8 @@
 
 namespace oasis {
 
-constexpr int kLyThreads = 256;
+constexpr int kLyThreads = 256;                             // (128 more with two softmax sets: warps 8-11)
+__host__ __device__ constexpr int ly_threads(int mma_m, int copies) { return kLyThreads + (at_softmax_sets(mma_m, copies) - 1) * 128; }
 constexpr int kLyMaxStages = 6;                             // 32 KiB stages (attention) = three 64 KiB pairs (scoring)
 constexpr int kLyTileBlocks = 128;                          // summaries per scoring tile
 constexpr int kLyATileBytes = kLyTileBlocks * kSummaryBytes;   // 64 KiB
@@ -83,7 +86,7 @@ struct LayerTcParams {
 // costs mode 0 1.5 us at 128 rows, the split arithmetic 0.5 us).  STAGES: 32 KiB stages of the ring (6, or 4 where
 // the scoring operands or the copy-merge staging need the room); ASTAGES: stages in the attention phase.
 template <int MMA_M, int COPIES, int MODE, int STAGES, int ASTAGES>
-__global__ void __launch_bounds__(kLyThreads, 1)
+__global__ void __launch_bounds__(ly_threads(MMA_M, COPIES), 1)
 layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap_summ,
                 const LayerTcParams p)
 {
@@ -96,6 +99,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     constexpr int BPC = kAtTileCols / COPIES;               // blocks of a tile each copy handles
     constexpr int KPC = BPC * kBlock;                       // keys of a tile each copy handles
     constexpr int kStageF = COPIES > 1 ? 20 : 0;            // floats per MMA row of the copy-merge staging (16 + pad)
+    constexpr int SETS = at_softmax_sets(MMA_M, COPIES);    // softmax warp sets, taking alternate tiles of a row
+    constexpr int SBUFS = at_s_bufs(SETS);                  // S / P buffers in tensor memory
+    constexpr int THREADS = ly_threads(MMA_M, COPIES);
     constexpr int kAtQBytes = 0;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -105,9 +111,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
     const uint32_t b_u32 = kv_u32 + STAGES * kAtStageBytes;          // [2][N][512 B] as 4 sub-tiles of N x 128 B
     uint8_t *b_ptr = base_ptr + (size_t)STAGES * kAtStageBytes;
     float *o_sm = reinterpret_cast<float *>(b_ptr + 2 * b_bytes);    // [MMA_M][kStageF]
-    float *m_sm = o_sm + MMA_M * kStageF;                            // [MMA_M]
-    float *l_sm = m_sm + MMA_M;                                      // [MMA_M]
-    uint8_t *misc = reinterpret_cast<uint8_t *>(l_sm + MMA_M);
+    float *m_sm = o_sm + MMA_M * kStageF;                            // [SETS][MMA_M]
+    float *l_sm = m_sm + MMA_M * SETS;                               // [SETS][MMA_M]
+    uint8_t *misc = reinterpret_cast<uint8_t *>(l_sm + MMA_M * SETS);
     const uint32_t bar_u32 = smem_u32(misc);
     // attention-phase barriers
     auto bar_full = [&](int s) { return bar_u32 + 8u * s; };
@@ -195,11 +201,11 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
         }
         tc_fence_before();
-        asm volatile("bar.sync 2, %0;" ::"n"(kLyThreads - 32) : "memory");
+        asm volatile("bar.sync 2, %0;" ::"n"(THREADS - 32) : "memory");
         tc_fence_after();
         tmem_base = *tmem_slot;
-        tmem_o = tmem_base + kAtSBufs * kAtTileKeys;
-        tmem_q = tmem_o + kHeadDim;                                  // Q as the A operand: 128 rows x 64 packed columns
+        tmem_o = tmem_base + SBUFS * kAtTileKeys;
+        tmem_q = tmem_o + SETS * kHeadDim;                                // Q as the A operand: 128 rows x 64 packed columns
     }
     if (warp == 0) {
         bool alive = true;
@@ -310,7 +316,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             // descriptors: the operand start address occupies the low 14 bits (16-byte units), so offsets are added there
             const uint64_t k_desc0 = smem_desc_sw128_k(kv_u32, kImgGroup);
             bool alive = true;
-            int s = 0, sb = 0, s_old = 0;                            // stage and S buffer of tile i; stage of tile i - kAtSBufs
+            int s = 0, sb = 0, s_old = 0;                            // stage and S buffer of tile i; stage of tile i - SBUFS
             uint32_t ph = 0, ph_old = 0;
             int i = 0;                                               // index of the tile among all rows of this CTA
 #pragma unroll 1
@@ -320,8 +326,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             tc_fence_after();
 #pragma unroll 1
             for (int it = 0; it < tpr && alive; ++it, ++i) {
-                // the S buffer also held P of tile i - kAtSBufs: its P V must have completed
-                if (i >= kAtSBufs) {
+                // the S buffer also held P of tile i - SBUFS: its P V must have completed
+                if (i >= SBUFS) {
                     alive = mbar_wait_warp(bar_empty(s_old), ph_old, p.err, 51);
                     ph_old ^= (s_old + 1 == kLyStages);
                     s_old = (s_old + 1 == kLyStages) ? 0 : s_old + 1;
@@ -335,7 +341,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 tc_commit(bar_s_full(sb));
                 ph ^= (s + 1 == kLyStages);
                 s = (s + 1 == kLyStages) ? 0 : s + 1;
-                sb = (sb + 1) & (kAtSBufs - 1);
+                sb = (sb + 1 == SBUFS) ? 0 : sb + 1;
             }
             }
         }
@@ -357,10 +363,11 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                 tc_fence_after();
                 const uint64_t v_desc = v_desc0 + (uint64_t)((s * kAtStageBytes) >> 4);
                 const uint32_t p_tmem = tmem_base + (uint32_t)(sb * kAtTileKeys);
-                issue_pv_tile(tmem_o, p_tmem, v_desc, idesc, it == 0);   // O starts afresh with every row
+                // O starts afresh with every row (two softmax sets: even tiles of the row go to the first O, odd ones to the second)
+                issue_pv_tile(tmem_o + (uint32_t)((it % SETS) * kHeadDim), p_tmem, v_desc, idesc, it < SETS);
                 tc_commit(bar_empty(s));                             // stage free, and O complete up to this tile
                 s = (s + 1 == kLyStages) ? 0 : s + 1;
-                sb = (sb + 1) & (kAtSBufs - 1);
+                sb = (sb + 1 == SBUFS) ? 0 : sb + 1;
                 ph_p ^= (sb == 0);
             }
             }
@@ -387,7 +394,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             if (lane == 0) mbar_arrive(bar_b_full(buf));
         }
     } else {
-        // ---------------------------------------------------------------- softmax, one thread per MMA row
+        // ---------------------------------------------------------------- softmax, one thread per MMA row (two sets: warps
+        // 3-6 take the even tiles of a row, warps 8-11 the odd ones; the first set alone has a part in the scoring phase)
+        const int set = SETS == 2 ? (warp >= 8 ? 1 : 0) : 0;
         const int quarter = warp & 3;
         const int m_row = quarter * LANES + (lane % LANES);         // MMA row held by this tensor-memory lane
         const int copy = m_row / RPC, row = m_row % RPC;            // which copy of the rows, which query row
@@ -395,7 +404,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         const bool live_row = has_row && row < p.R;
         const bool live_warp = (quarter * LANES) % RPC < p.R;       // some lane of this warp holds a query row
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        {
+        if (set == 0) {
             // ---------------------------------------------------------------- scoring phase: epilogue
             int it = 0;
             bool alive = true;
@@ -444,11 +453,10 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_q);
         };
-        if (cta_has_row) load_q(row_of(my_row(0)));
+        if (set == 0 && cta_has_row) load_q(row_of(my_row(0)));
         bool alive = true;
-        int s = 0, s_prev = 0;                                      // ring stage of tile i and of tile i - 1
-        uint32_t ph_prev = 0;                                       // parity of the "empty" phase that ends tile i - 1
-        int i = 0;                                                  // index of the tile among all rows of this CTA
+        int i0 = 0;                                                 // index of the row's first tile among all tiles of this CTA
+        const uint32_t my_o = tmem_o + (uint32_t)(set * kHeadDim) + lane_base;   // this thread's O row
 #pragma unroll 1
         for (int k = 0; k < n_my_rows; ++k) {
         const int item = my_row(k), tpr = tiles_of(item);
@@ -457,33 +465,40 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
         // send their whole warp down the masked path on every tile), lanes without an MMA row see nothing
         const int limit = live_row ? (k == 0 ? L0 : p.seq_len[b]) + row / p.G : (has_row ? 0x3fffffff : -1);
         float m_ref = -CUDART_INF_F, l_sum = 0.f;
+        // Tile g of the CTA (counted through all its rows) lives in ring stage g % stages and S buffer g % SBUFS; the
+        // barriers of its stage / buffer complete for it with parity (g / stages) & 1, (g / SBUFS) & 1.
 #pragma unroll 1
-        for (int it = 0; it < tpr && alive; ++it, ++i) {
-            alive = mbar_wait(bar_s_full(i % kAtSBufs), (i / kAtSBufs) & 1, p.err, 61);
+        for (int it = set; it < tpr && alive; it += SETS) {
+            const int g = i0 + it, sb = g % SBUFS, s = g % kLyStages;
+            alive = mbar_wait(bar_s_full(sb), (uint32_t)((g / SBUFS) & 1), p.err, 61);
             if (!alive) break;
             tc_fence_after();
-            const uint32_t s_tmem = tmem_base + lane_base + (uint32_t)((i % kAtSBufs) * kAtTileKeys);
+            const uint32_t s_tmem = tmem_base + lane_base + (uint32_t)(sb * kAtTileKeys);
             if (live_warp)
-                alive = softmax_tile<COPIES>(s_tmem, tmem_o + lane_base, tile_blk + s * kAtTileCols, copy, limit, has_row,
-                                             p.scale_log2, m_ref, l_sum, it > 0,
-                                             [&] { return mbar_wait(bar_empty(s_prev), ph_prev, p.err, 62); });
+                alive = softmax_tile<COPIES>(s_tmem, my_o, tile_blk + s * kAtTileCols, copy, limit, has_row,
+                                             p.scale_log2, m_ref, l_sum, it >= SETS,
+                                             // the P V of this set's previous tile of the row
+                                             [&] { return mbar_wait(bar_empty((g - SETS) % kLyStages), (uint32_t)(((g - SETS) / kLyStages) & 1), p.err, 62); });
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_p_full(i % kAtSBufs));
-            if (i > 0) ph_prev ^= (s_prev + 1 == kLyStages);
-            s_prev = s;
-            s = (s + 1 == kLyStages) ? 0 : s + 1;
+            if (lane == 0) mbar_arrive(bar_p_full(sb));
         }
         // ---- Q of the CTA's next row goes to tensor memory first (this warp has seen S of the row's last tile, so
         // every Q K^T of the row has completed), then the row is written out: merge the copies, normalise.  The
         // next row's first P V, which overwrites O, needs P of that tile from these warps, so it comes later.
         {
-            if (MULTI && alive && k + 1 < n_my_rows) load_q(my_row(k + 1));
-            if (alive) alive = mbar_wait(bar_empty(s_prev), ph_prev, p.err, 63);   // the row's last P V has completed
+            // (with two softmax sets the first one has not seen the row's odd tiles: it loads Q after the last P V instead)
+            if (SETS == 1 && MULTI && alive && k + 1 < n_my_rows) load_q(my_row(k + 1));
+            if (alive && tpr > 0) {                                  // the row's last P V has completed
+                const int g = i0 + tpr - 1;
+                alive = mbar_wait(bar_empty(g % kLyStages), (uint32_t)((g / kLyStages) & 1), p.err, 63);
+            }
             tc_fence_after();
+            if (SETS == 2 && MULTI && alive && set == 0 && k + 1 < n_my_rows) load_q(my_row(k + 1));
+            i0 += tpr;
             // From here on the four softmax warps meet at named barriers, which have no time-out: go on only if
             // none of them has given up (every thread gets here, because all its waits above are bounded).
-            alive = softmax_warps_all(alive);
+            alive = softmax_warps_all<128 * SETS>(alive);
             const int t_task = quarter * 32 + lane;
             // writes 16 output dims [d0, d0 + 16) of query row `orow`
             auto emit = [&](int orow, int d0, const float (&acc)[16], float mx, float den) {
@@ -508,7 +523,34 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
                                         pack_bf16x2(acc[8 * e + 6] * inv, acc[8 * e + 7] * inv));
                 if (p.lse && d0 == 0) p.lse[o_row] = den > 0.f ? (mx + log2f(den)) * kAtLn2 : -CUDART_INF_F;
             };
-            if (alive && COPIES > 1) {
+            if (alive && SETS == 2) {
+                // the two threads of a row exchange maximum and sum; each then merges and writes one half of the output dims,
+                // reading both O accumulators at its own tensor-memory lane
+                m_sm[set * MMA_M + m_row] = m_ref;
+                l_sm[set * MMA_M + m_row] = l_sum;
+                asm volatile("bar.sync 1, 256;" ::: "memory");      // the eight softmax warps
+                const float m_o = m_sm[(set ^ 1) * MMA_M + m_row], l_o = l_sm[(set ^ 1) * MMA_M + m_row];
+                const float mx = fmaxf(m_ref, m_o);
+                const float w_me = mx == -CUDART_INF_F ? 0.f : fast_exp2(m_ref - mx), w_ot = mx == -CUDART_INF_F ? 0.f : fast_exp2(m_o - mx);
+                const float den = w_me * l_sum + w_ot * l_o;
+                const float w_a = set == 0 ? w_me : w_ot, w_b = set == 0 ? w_ot : w_me;   // weights of the first and second accumulator
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    const int d0 = set * 64 + c * 16;
+                    uint32_t va[16], vb[16];
+                    if (live_warp) {
+                        tc_ld16(tmem_o + lane_base + d0, va);
+                        tc_ld16(tmem_o + kHeadDim + lane_base + d0, vb);
+                    }
+                    float acc[16];
+                    // an accumulator whose set saw no key (weight 0) was never written: its contents do not enter
+#pragma unroll
+                    for (int e = 0; e < 16; ++e)
+                        acc[e] = live_warp ? (w_a != 0.f ? w_a * __uint_as_float(va[e]) : 0.f) + (w_b != 0.f ? w_b * __uint_as_float(vb[e]) : 0.f) : 0.f;
+                    if (live_row) emit(row, d0, acc, mx, den);
+                }
+                asm volatile("bar.sync 1, 256;" ::: "memory");      // the exchange area is rewritten for the next row
+            } else if (alive && COPIES > 1) {
                 // with several rows per thread block the ring already holds the next row's tiles: the copies meet in a
                 // small staging area, 16 dims at a time (small enough that the selection kernels of other streams still
                 // fit beside this CTA)
@@ -634,7 +676,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant_
 static size_t layer_tc_smem_bytes(int mma_m, int copies, int N, int stages)
 {
     return 1024 + (size_t)stages * kAtStageBytes + 2 * (size_t)N * kSummaryBytes +
-           (size_t)mma_m * ((copies > 1 ? 20 : 0) + 2) * sizeof(float) + 512 + 2 * kWinBytes;
+           (size_t)mma_m * ((copies > 1 ? 20 : 0) + 2 * at_softmax_sets(mma_m, copies)) * sizeof(float) + 512 + 2 * kWinBytes;
 }
 
 struct LayerTcPlan {
@@ -671,8 +713,13 @@ static bool layer_tc_plan(const oasis_dims_t *dims, int n_q_tokens, int n_cols, 
         pl.stages = 4;
         pl.smem = layer_tc_smem_bytes(pl.mma_m, pl.copies, pl.N, pl.stages);
     }
-    // attention-phase stages: with four stages and 64 scoring rows the two operand buffers (2 x 32 KiB) are two more
-    pl.astages = (pl.stages == 4 && 2 * (size_t)pl.N * kSummaryBytes >= 2 * (size_t)kAtStageBytes) ? 6 : pl.stages;
+    // attention-phase stages: with four stages the two operand buffers (2 x N x 512 B: 64 KiB at 64 scoring rows, 32 KiB
+    // at 32) are one or two more
+    pl.astages = pl.stages;
+    if (pl.stages == 4) {
+        const int extra = (int)(2 * (size_t)pl.N * kSummaryBytes / kAtStageBytes);
+        pl.astages = 4 + (extra > 2 ? 2 : extra);
+    }
     pl.n_splits = 1;
     pl.cols_per_split = n_cols;
     pl.workspace = 0;
@@ -778,7 +825,9 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     p.part_lse = p.part_o ? p.part_o + (size_t)p.items * R * kHeadDim : nullptr;
     p.q_draft = (const uint8_t *)q_draft; p.q_batch_stride = q_batch_stride; p.n_full = n_full_blocks; p.scores = scores;
     p.Rs = Rs; p.N = N; p.max_blocks = dims->max_blocks;
-    p.acc_col = N <= 32 ? 448 : 0;
+    // two accumulators of up to 32 columns fit behind Q; wider ones, and all with two softmax sets (whose second O takes that
+    // place), use the S buffers' columns, which the attention phase only touches after the last scoring epilogue
+    p.acc_col = (N <= 32 && at_softmax_sets(pl.mma_m, pl.copies) == 1) ? 448 : 0;
     p.tiles_per_bh = (dims->max_blocks + kLyTileBlocks - 1) / kLyTileBlocks;
     p.reduce_sum = reduce_mode == OASIS_REDUCE_SUM;
     p.total_tiles = (int)(rows * p.tiles_per_bh);
@@ -823,6 +872,7 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     cfg.numAttrs = 1;
 #define OASIS_LAYER_TC_LAUNCH_2(M, C, MU, ST, AST)                                                                            \
     do {                                                                                                                      \
+        cfg.blockDim = dim3(ly_threads(M, C));                                                                                \
         e = cudaFuncSetAttribute(layer_tc_kernel<M, C, MU, ST, AST>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
         if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, layer_tc_kernel<M, C, MU, ST, AST>, tmap_kv, tmap_summ, p);         \
     } while (0)
@@ -836,9 +886,11 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     else if (R <= 32) OASIS_LAYER_TC_LAUNCH(64, 2, 6, 6);
     else if (R <= 64 && pl.stages == 6) OASIS_LAYER_TC_LAUNCH(128, 2, 6, 6);
     else if (R <= 64 && pl.astages == 6) OASIS_LAYER_TC_LAUNCH(128, 2, 4, 6);
+    else if (R <= 64 && pl.astages == 5) OASIS_LAYER_TC_LAUNCH(128, 2, 4, 5);
     else if (R <= 64) OASIS_LAYER_TC_LAUNCH(128, 2, 4, 4);
     else if (pl.stages == 6) OASIS_LAYER_TC_LAUNCH(128, 1, 6, 6);
     else if (pl.astages == 6) OASIS_LAYER_TC_LAUNCH(128, 1, 4, 6);
+    else if (pl.astages == 5) OASIS_LAYER_TC_LAUNCH(128, 1, 4, 5);
     else OASIS_LAYER_TC_LAUNCH(128, 1, 4, 4);
 #undef OASIS_LAYER_TC_LAUNCH
 #undef OASIS_LAYER_TC_LAUNCH_2

@@ -281,16 +281,17 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
-// Named barrier 1 over the four softmax warps (128 threads), returning the AND of their predicates.
+// Named barrier 1 over the softmax warps (THREADS = 128 per set), returning the AND of their predicates.
+template <int THREADS = 128>
 __device__ __forceinline__ bool softmax_warps_all(bool pred)
 {
     uint32_t r;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.u32 p, %1, 0;\n\t"
-        "bar.red.and.pred q, 1, 128, p;\n\t"
+        "bar.red.and.pred q, 1, %2, p;\n\t"
         "selp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(r) : "r"((uint32_t)pred) : "memory");
+        : "=r"(r) : "r"((uint32_t)pred), "n"(THREADS) : "memory");
     return r != 0;
 }
 
@@ -319,6 +320,24 @@ __device__ __forceinline__ void issue_qk_tile(uint32_t d_tmem, uint32_t tmem_q, 
         for (int k4 = 0; k4 < 4; ++k4)
             tc_mma_bf16_ts(d_tmem, tmem_q + (kc * 4 + k4) * 8, k_desc + (uint64_t)((kc * kImgHalf + k4 * 32) >> 4), idesc,
                            (kc | k4) ? 1u : 0u);
+}
+// Two softmax warp sets (the 128-row kernels with a single copy of the query rows, 65 to 128 rows).  A softmax warp
+// with full 64-key rows needs 950-1,000 cycles per tile (64 ex2 at 8 cycles per warp instruction, about 240 other
+// instructions at 2 or more), of which a lone warp per scheduler loses the latencies between dependent instructions
+// and around its waits.  So the rows get two threads each, in two warps of the same scheduler, that take alternate
+// tiles of the row; each set keeps a running maximum and sum and an O accumulator of its own (P V of the row's even
+// tiles goes to the first, of its odd tiles to the second), merged when the row is written.  Tensor memory then holds
+// three S buffers, the two O accumulators and Q.
+__host__ __device__ constexpr int at_softmax_sets(int mma_m, int copies) { return (mma_m == 128 && copies == 1) ? 2 : 1; }
+__host__ __device__ constexpr int at_s_bufs(int sets) { return sets == 2 ? 3 : kAtSBufs; }
+// Ring stage and completion parity of the tile `n` tiles further on (run-time stage count: no division per tile).
+__device__ __forceinline__ void ring_advance(int &s, uint32_t &ph, int n, int stages)
+{
+#pragma unroll
+    for (int k = 0; k < n; ++k) {
+        ph ^= (s + 1 == stages);
+        s = (s + 1 == stages) ? 0 : s + 1;
+    }
 }
 // O (+)= P V of one tile: 16 keys (one block image) per MMA, P from tensor memory.
 __device__ __forceinline__ void issue_pv_tile(uint32_t tmem_o, uint32_t p_tmem, uint64_t v_desc, uint32_t idesc, bool first_of_row)
