@@ -152,14 +152,18 @@ def test_kv_pool_in_device_memory(oracle, gpu):
     compare_path(oracle, pipeline, lay, cfg.k_blocks, kv_on="device")
 
 
-@pytest.mark.parametrize("Hq,Hkv,Td", [(8, 8, 1), (16, 8, 1), (32, 8, 2), (32, 8, 7), (64, 8, 5), (40, 8, 8), (128, 8, 8)])
-def test_row_counts(oracle, gpu, Hq, Hkv, Td):
-    """R = Td*G from 1 to 128 score rows; T*G from 2 to 144 would exceed 128, so Td is capped."""
+@pytest.mark.parametrize("Hq,Hkv,Td,B", [(8, 8, 1, 1), (16, 8, 1, 1), (32, 8, 2, 1), (32, 8, 7, 1), (64, 8, 5, 1), (40, 8, 8, 1),
+                                         (128, 8, 8, 1),
+                                         # KV head counts other than the five configurations' 8 (one head per GPU is the
+                                         # tensor-parallel shape of the larger models, Sec. 5.3.1), odd group sizes
+                                         (8, 1, 4, 5), (1, 1, 1, 3), (4, 2, 4, 3), (12, 4, 2, 2), (48, 16, 3, 2), (9, 3, 8, 7)])
+def test_row_counts(oracle, gpu, Hq, Hkv, Td, B):
+    """R = Td*G from 1 to 128 score rows; T*G from 2 to 144 would exceed 128, so Td is capped.  1 to 16 KV heads."""
     _, pipeline = gpu
     G = Hq // Hkv
     if (Td + 1) * G > 128:
         Td = 128 // G - 1
-    cfg = synth.scaled(synth.C1, batch=1, n_q_heads=Hq, n_kv_heads=Hkv, context=656, k_blocks=12, n_draft=Td)
+    cfg = synth.scaled(synth.C1, batch=B, n_q_heads=Hq, n_kv_heads=Hkv, context=656, k_blocks=12, n_draft=Td)
     lay = synth.make_layer(cfg, seed=6)
     compare_path(oracle, pipeline, lay, cfg.k_blocks)
 
@@ -493,7 +497,9 @@ def test_error_word_registration(gpu):
                                                   (16, 32, 8, 8, 8, 2064, 24), (16, 32, 8, 14, 14, 1040, 12),
                                                   (8, 64, 8, 8, 8, 10256, 38), (24, 64, 8, 8, 8, 1040, 12),
                                                   (1, 32, 8, 4, 4, 2064, 30), (3, 32, 8, 4, 4, 1040, 21),
-                                                  (5, 64, 8, 2, 2, 784, 127), (9, 32, 8, 4, 4, 528, 16)])
+                                                  (5, 64, 8, 2, 2, 784, 127), (9, 32, 8, 4, 4, 528, 16),
+                                                  (16, 8, 1, 4, 4, 1040, 24), (150, 4, 1, 4, 4, 528, 8),
+                                                  (30, 12, 4, 3, 3, 1040, 17), (5, 48, 16, 2, 2, 784, 9)])
 def test_fused_attention_and_scoring_equals_the_two_calls(oracle, gpu, B, Hq, Hkv, Td, nd, ctx, k):
     """oasis_attn_and_score is steps 4 and 1 in one launch with unchanged arithmetic: outputs, log-sum-exps and
     scores must equal those of oasis_sparse_attn and oasis_score_blocks bit for bit (the separate calls are the
