@@ -13,7 +13,9 @@ full-KV pool in PINNED HOST MEMORY on side streams.  metric = tokens/s per layer
   value_hbm_mirror : the full KV mirrored in HBM (no host link): the compute-only step, for the exposed
                      transfer time  value.ms_per_step - value_hbm_mirror.ms_per_step.
 Consecutive steps are captured into CUDA graphs of `--group` steps; inside a graph a layer's transfer only
-has to land before that layer's next-step attention (Sec. 4.2.2), so steps overlap.
+has to land before that layer's next-step attention (Sec. 4.2.2), so steps overlap.  The graphs of the timed
+steps are instantiated and uploaded to the device before the timed region (the first replay of a graph of some
+thousand nodes otherwise spends about 3 ms on the host before the device sees its first node).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config 0..4] [--fetch-ratio R] [--group G]
                   [--repeats R] [--sweep-ratios 0.01,0.02,...] [--summary FILE] [--impl reference]
@@ -389,6 +391,8 @@ class Bench:
         graphs = [eng.capture_steps([self.step_args(w, s, e2e) for s in range(s0, min(s0 + group, W + K))])
                   for s0 in range(W, W + K, group)]
         eng.replay(warm)
+        for g in graphs:                # instantiated and uploaded ahead of the timed region, like any other set-up
+            eng.upload(g)
         torch.cuda.synchronize()
         sampler = ClockSampler(self.dev.index or 0)
         sampler.start()
@@ -781,7 +785,8 @@ def run_ours(args):
                        "kv": "full KV in pinned host memory (value, e2e); value_hbm_mirror: the same pool copied to HBM",
                        "gather": "delta selection with capped eviction, fetch ratio %.2f (cap %d blocks per head per step); local "
                                  "blocks appended on the GPU" % (args.fetch_ratio, cap),
-                       "launch": "CUDA graphs of %d consecutive decode steps over 6-10 streams; a layer's attention and scoring are "
+                       "launch": "CUDA graphs of %d consecutive decode steps over 6-10 streams, instantiated and uploaded to the device "
+                                 "before the timed region; a layer's attention and scoring are "
                                  "one fused launch (oasis_attn_and_score); %s gathers of %d layers per launch; side-stream "
                                  "events picked up every %d layers"
                                  % (args.group if args.group > 0 else K,

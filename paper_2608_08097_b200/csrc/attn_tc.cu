@@ -469,6 +469,7 @@ int launch_attn_tc(const oasis_dims_t *dims, const void *q, int n_q_tokens, cons
 #define OASIS_ATTN_TC_LAUNCH(M, C)                                                                                     \
     do {                                                                                                               \
         e = cudaFuncSetAttribute(sparse_attn_tc_kernel<M, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
+        if (e == cudaSuccess) prefer_max_shared_carveout(sparse_attn_tc_kernel<M, C>);                                \
         if (e == cudaSuccess) sparse_attn_tc_kernel<M, C><<<(unsigned)grid, at_threads(M, C), smem, st>>>(tmap, p);          \
     } while (0)
     if (p.R <= 16) OASIS_ATTN_TC_LAUNCH(64, 4);          // four copies of <= 16 rows, one block of a tile each

@@ -4,6 +4,7 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <mutex>
 
 #include "../../include/oasis.h"
 
@@ -92,15 +93,28 @@ __device__ __forceinline__ float fast_exp2(float x)
 
 // The small kernels of the other streams (top-k, plan, gather, summaries) ask for the largest shared-memory
 // carve-out although they need little: an SM they have configured otherwise could not take a thread block of the
-// attention / scoring kernels (which need nearly all of it) until they have left.
+// attention / scoring kernels (which need nearly all of it) until they have left.  The attention / scoring kernels ask
+// for it too: an instantiation with four ring stages needs 173 KiB, the driver then configured the SM for the next
+// size up, and a top-k thread block (20 KiB at 4,096 blocks per row) no longer fitted beside it and a gather thread
+// block -- every gather waited for the following layer's launch (budget x draft sweep, 8 draft tokens: 0.75 -> 0.52 ms).
+inline void prefer_max_shared_carveout_of(const void *kernel)
+{
+    // once per kernel (per instantiation: instantiations of one template share their pointer TYPE, so the flag cannot be
+    // a static of a function template over that type)
+    static std::mutex lock;
+    static const void *seen[256];
+    static int n_seen = 0;
+    std::lock_guard<std::mutex> guard(lock);
+    for (int i = 0; i < n_seen; ++i)
+        if (seen[i] == kernel) return;
+    cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+    if (n_seen < 256) seen[n_seen++] = kernel;
+}
+
 template <typename K>
 inline void prefer_max_shared_carveout(K kernel)
 {
-    static bool done = false;          // per kernel type; a race here only repeats an idempotent call
-    if (!done) {
-        cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
-        done = true;
-    }
+    prefer_max_shared_carveout_of(reinterpret_cast<const void *>(kernel));
 }
 
 }  // namespace oasis

@@ -874,6 +874,7 @@ extern "C" int oasis_attn_and_score(const oasis_dims_t *dims, const void *q, int
     do {                                                                                                                      \
         cfg.blockDim = dim3(ly_threads(M, C));                                                                                \
         e = cudaFuncSetAttribute(layer_tc_kernel<M, C, MU, ST, AST>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);  \
+        if (e == cudaSuccess) prefer_max_shared_carveout(layer_tc_kernel<M, C, MU, ST, AST>);                                 \
         if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, layer_tc_kernel<M, C, MU, ST, AST>, tmap_kv, tmap_summ, p);         \
     } while (0)
 #define OASIS_LAYER_TC_LAUNCH(M, C, ST, AST)                          \

@@ -280,6 +280,7 @@ int score_blocks_tc(const oasis_dims_t *dims, const void *q_draft, int64_t q_bat
     const size_t smem = 1024 + (size_t)p.stages * kATileBytes + (size_t)p.n_bbuf * N * kSummaryBytes + 256;
     cudaError_t e = cudaFuncSetAttribute(score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "oasis_score_blocks: shared memory %zu B: %s", smem, cudaGetErrorString(e));
+    prefer_max_shared_carveout(score_tc_kernel);
     long long grid = p.total_tiles < sm_count() ? p.total_tiles : sm_count();
     score_tc_kernel<<<(unsigned)grid, kTcThreads, smem, st>>>(tmap, p);
     return check_launch("oasis_score_blocks");

@@ -196,6 +196,7 @@ extern "C" int oasis_stage_blocks_bulk(int32_t n_layers, const void *const *host
     int per_layer = (max_streams > 0 ? max_streams : kStageDefaultCtas) / n_layers;
     if (per_layer < 1) per_layer = 1;
     const int grid = n < per_layer ? n : per_layer;
+    prefer_max_shared_carveout(stage_blocks_bulk_kernel);
     stage_blocks_bulk_kernel<<<dim3((unsigned)grid, (unsigned)n_layers), 32, (size_t)kStageBulkBufs * kEntryBytes, (cudaStream_t)stream>>>(
         ly, n, kStageBulkBufs, error_word(), bounds());
     return check_launch(who);

@@ -91,6 +91,7 @@ extern "C" int oasis_union_blocks(const oasis_dims_t *dims, const int32_t *sel, 
         cudaError_t e = cudaFuncSetAttribute(union_blocks_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return fail(OASIS_ERR_CUDA, "oasis_union_blocks: shared memory %zu B: %s", smem, cudaGetErrorString(e));
     }
+    prefer_max_shared_carveout(union_blocks_kernel);
     union_blocks_kernel<<<dims->batch, kUnionThreads, smem, (cudaStream_t)stream>>>(
         sel, dims->n_kv_heads, dims->max_blocks, sel_cols, k, max_union, n_words, union_idx, n_union);
     return check_launch("oasis_union_blocks");

@@ -3,11 +3,15 @@
 This is host-side bookkeeping only (allocation through torch, call sequencing, stream
 choice); every step of the path runs inside liboasis.so through `binding`.
 """
+import ctypes
 import math
 
 import torch
 
 from . import binding as oasis
+
+
+_libcuda = None                      # the driver library, loaded on the first DecodeEngine.upload
 
 
 class DecodeLayer:
@@ -473,6 +477,19 @@ class DecodeEngine:
     def capture_step(self, *args, **kwargs):
         """One step (same arguments as `step`) as a CUDA graph."""
         return self.capture_steps([(args, kwargs)])
+
+    def upload(self, graph):
+        """Makes an instantiated graph resident on the device ahead of its first replay (the driver's cuGraphUpload
+        on the foreground stream): the first replay of a graph of some thousand nodes otherwise spends milliseconds
+        on the host before the device sees its first node."""
+        global _libcuda
+        if _libcuda is None:
+            _libcuda = ctypes.CDLL("libcuda.so.1")
+            _libcuda.cuGraphUpload.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+            _libcuda.cuGraphUpload.restype = ctypes.c_int
+        rc = _libcuda.cuGraphUpload(ctypes.c_void_p(graph.raw_cuda_graph_exec()), ctypes.c_void_p(self.main.cuda_stream))
+        if rc != 0:
+            raise RuntimeError("cuGraphUpload failed with CUresult %d" % rc)
 
     def replay(self, graph):
         with torch.cuda.stream(self.main):
