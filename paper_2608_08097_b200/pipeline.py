@@ -481,15 +481,23 @@ class DecodeEngine:
     def upload(self, graph):
         """Makes an instantiated graph resident on the device ahead of its first replay (the driver's cuGraphUpload
         on the foreground stream): the first replay of a graph of some thousand nodes otherwise spends milliseconds
-        on the host before the device sees its first node."""
+        on the host before the device sees its first node.  Returns False, having done nothing, where the driver
+        library or the graph's handle cannot be had (the replay then uploads the graph itself)."""
         global _libcuda
         if _libcuda is None:
-            _libcuda = ctypes.CDLL("libcuda.so.1")
-            _libcuda.cuGraphUpload.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
-            _libcuda.cuGraphUpload.restype = ctypes.c_int
+            try:
+                lib = ctypes.CDLL("libcuda.so.1")
+                lib.cuGraphUpload.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+                lib.cuGraphUpload.restype = ctypes.c_int
+                _libcuda = lib
+            except (OSError, AttributeError):
+                _libcuda = False
+        if not _libcuda or not hasattr(graph, "raw_cuda_graph_exec"):
+            return False
         rc = _libcuda.cuGraphUpload(ctypes.c_void_p(graph.raw_cuda_graph_exec()), ctypes.c_void_p(self.main.cuda_stream))
         if rc != 0:
             raise RuntimeError("cuGraphUpload failed with CUresult %d" % rc)
+        return True
 
     def replay(self, graph):
         with torch.cuda.stream(self.main):
