@@ -179,7 +179,7 @@ int oasis_stage_blocks_layers(int32_t n_layers, const void *const *host_kvs, con
  * entries move as 8 KiB bulk copies (CPU pool -> shared memory -> working-set pool) issued by one thread of a
  * small thread block per entry stream, so that the gather runs beside kernels that fill the SMs (the fused
  * attention + scoring launch) without competing for their issue slots.  Faster than the warp-per-entry gather where
- * the host link bounds the decode step; no better where compute bounds it.  A copy that does not complete within
+ * the host link bounds the decode step and also carries the step's query uploads; no better otherwise.  A copy that does not complete within
  * the library's bounded wait records code 71 in the error word.
  *   max_streams   entry streams (thread blocks) of the launch, shared among the layers, each with one 8 KiB copy
  *                 in flight; 0 = the library's default of 128 (1 MiB in flight).

@@ -80,12 +80,12 @@ stage_blocks_layers_kernel(const __grid_constant__ StageLayers ly, int n, const 
 // The several-layers gather through the copy unit: one thread per CTA moves its share of the list as 8 KiB bulk
 // copies, CPU pool -> shared memory -> working-set pool, one buffer per CTA; no warp spends an instruction on the
 // bytes, and the CTA (32 threads, 8 KiB of shared memory) fits on an SM beside the fused attention + scoring CTA.
-// Alone it moves what the warp-per-entry kernel moves (49-51 GB/s from pinned memory).  Inside a decode step that the
-// host link bounds it is the faster one at 128 entry streams per launch and eight layers per launch (host-KV step
-// 4.01-4.03 against 4.05-4.07 ms at fetch ratio 0.05, end to end 4.47 against 4.60 ms); where compute bounds the step
-// the two are equal (1.66-1.67 ms at fetch ratio 0.02, two layers per launch) and the warp kernel disturbs the query
-// uploads of the end-to-end step less (2.07 against 2.41 ms).  Two buffers per CTA no longer fit beside the fused
-// CTA and are slower.
+// Alone it moves what the warp-per-entry kernel moves (49-51 GB/s from pinned memory), and so it does inside a decode
+// step that the host link bounds while the queries are resident (3.99 ms either way at fetch ratio 0.05, 128 entry
+// streams and eight layers per launch); end to end, with the query uploads on the same link, it is the faster one (4.45-4.47
+// against 4.55-4.60 ms).  Where compute bounds the step the two are equal (1.66-1.67 ms at fetch ratio 0.02, two layers
+// per launch) and the warp kernel disturbs the query uploads of the end-to-end step less (2.07 against 2.41 ms).  Two
+// buffers per CTA no longer fit beside the fused CTA and are slower.
 __global__ void __launch_bounds__(32)
 stage_blocks_bulk_kernel(const __grid_constant__ StageLayers ly, int n, int nbuf, int32_t *err, const Bounds bd)
 {
