@@ -63,3 +63,17 @@ def test_gather_grouping_follows_the_measured_regimes():
         for layers in (1, 2, 4, 8, 32, 64):
             g = pick(r, layers, 50.0)
             assert 1 <= g <= max(1, min(8, layers))
+
+
+def test_graph_upload_is_skipped_without_a_graph_handle():
+    """DecodeEngine.upload is an optimisation of the first replay: where the graph object has no handle to give (or
+    the driver library is not there) it reports False and does nothing."""
+    from paper_2608_08097_b200 import pipeline
+
+    class NoHandle:
+        pass
+
+    class Engine:
+        main = None
+
+    assert pipeline.DecodeEngine.upload(Engine(), NoHandle()) is False
