@@ -317,7 +317,7 @@ class Bench:
     def transfer_group(self, w, cap):
         """Layers per gather launch from pinned host memory, from the ratio of a layer's gather time on the link to its
         scoring + attention time.  Measured (step in ms, bulk gather unless noted): configs[1] (32 layers, ratio 3): 4.01
-        with 8 layers per launch, 4.03 with 4, 4.11 with 2; configs[3] (8 layers, ratio 2.4): 1.11 with 4, 1.25 with 2,
+        with 8 layers per launch (16: the same; all 32: 5.37), 4.03 with 4, 4.11 with 2; configs[3] (8 layers, ratio 2.4): 1.11 with 4, 1.25 with 2,
         1.27 with 1; configs[2] (4 layers, ratio 1.3): 1.11 with 1, 1.17 with 2, 2.05 with 4 (the whole step's transfers
         then wait for its last layer); configs[1] at fetch ratio 0.02 (ratio 0.85, warp gather): 1.67 with 2, 1.75
         with 1 or 4; far below the break-even one launch per layer is best (configs[0]: 0.55-0.60 against 0.67-0.69 end
