@@ -100,7 +100,7 @@ __device__ __forceinline__ float fast_exp2(float x)
 inline void prefer_max_shared_carveout_of(const void *kernel)
 {
     // once per kernel (per instantiation: instantiations of one template share their pointer TYPE, so the flag cannot be
-    // a static of a function template over that type)
+    // a static of a function template over that type); a process drives one GPU, so once per process is once per device
     static std::mutex lock;
     static const void *seen[256];
     static int n_seen = 0;
