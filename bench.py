@@ -15,7 +15,10 @@ full-KV pool in PINNED HOST MEMORY on side streams.  metric = tokens/s per layer
 Consecutive steps are captured into CUDA graphs of `--group` steps; inside a graph a layer's transfer only
 has to land before that layer's next-step attention (Sec. 4.2.2), so steps overlap.  The graphs of the timed
 steps are instantiated and uploaded to the device before the timed region (the first replay of a graph of some
-thousand nodes otherwise spends about 3 ms on the host before the device sees its first node).
+thousand nodes otherwise spends about 3 ms on the host before the device sees its first node).  After the timed
+region the same K steps are replayed `--again` more times (default 2), each replay timed by itself and reported as
+`ms_per_step_again` beside `value` and `e2e` (never part of them): the host link of a shared machine does not always
+deliver the same rate, and a reader should see whether the timed region repeats.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config 0..4] [--fetch-ratio R] [--group G]
                   [--repeats R] [--sweep-ratios 0.01,0.02,...] [--summary FILE] [--impl reference]
@@ -70,6 +73,8 @@ def parse_args():
                          "the host link bounds the step)")
     ap.add_argument("--repeats", type=int, default=1, help="replay the timed steps this many times in a second, long "
                                                             "timed region (reported as `sustained`)")
+    ap.add_argument("--again", type=int, default=2, help="further replays of the timed steps, each timed by itself and "
+                                                         "reported as ms_per_step_again (not part of value)")
     ap.add_argument("--sweep-ratios", default="", help="comma-separated fetch ratios to sweep (e.g. 0.01,0.02,0.05)")
     ap.add_argument("--summary", default="", help="write a markdown summary of the numbers to this file")
     ap.add_argument("--skip-e2e", action="store_true")
@@ -410,6 +415,17 @@ class Bench:
         launches = eng.launches - l0
         ms = max_over_ranks(start.elapsed_time(end) / K, world, self.dev)
         self.check_error_word("the timed steps")
+        # the same K steps twice more, each replay timed by itself: not part of `value`, reported beside it so that a
+        # reader sees how far one timed region on this (shared) machine repeats
+        self.again_ms = []
+        for _ in range(max(0, self.args.again)):
+            torch.cuda.synchronize()
+            start.record(eng.main)
+            for g in graphs:
+                eng.replay(g)
+            end.record(eng.main)
+            torch.cuda.synchronize()
+            self.again_ms.append(round(max_over_ranks(start.elapsed_time(end) / K, world, self.dev), 4))
         sustained = None
         if repeats > 1:
             # a long timed region: the same K steps again and again (the working sets keep evolving; the shapes and
@@ -629,6 +645,7 @@ def measure(bench, w, world, W, K, cap, hbm_peak, h2d_peak, want_mirror=True, wa
                      "h2d_bytes_per_step": int(gather), "d2h_bytes_per_step": int(n * commit_bytes),
                      "gather_GBps_over_step": round(gather / (ms * 1e-3) / 1e9, 2),
                      "gather_frac_of_h2d_peak": round(gather / (ms * 1e-3) / 1e9 / h2d_peak, 3)}
+        r["host"]["ms_per_step_again"] = list(bench.again_ms)
         if sustained:
             r["host"]["sustained"] = sustained
         if "mirror" in r:
@@ -647,6 +664,7 @@ def measure(bench, w, world, W, K, cap, hbm_peak, h2d_peak, want_mirror=True, wa
         h2d = gather + n * qo_bytes
         r["e2e"] = {"value": round(tok / (ms * 1e-3), 1), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                     "d2h_bytes_per_step": int(n * (qo_bytes + commit_bytes)), "ms_per_step": round(ms, 4), "steps": K,
+                    "ms_per_step_again": list(bench.again_ms),
                     "launches": launches, "requests_per_layer": round(n_req, 1),
                     "gather_GBps_over_step": round(gather / (ms * 1e-3) / 1e9, 2),
                     "gather_frac_of_h2d_peak": round(gather / (ms * 1e-3) / 1e9 / h2d_peak, 3),
@@ -814,7 +832,8 @@ def run_ours(args):
                        "gather_frac_of_h2d_peak": host.get("gather_frac_of_h2d_peak"),
                        "exposed_us_per_layer": host.get("exposed_us_per_layer"),
                        "compute_to_host_step_ratio": host.get("compute_to_host_step_ratio"),
-                       "h2d_bytes_per_step": host.get("h2d_bytes_per_step"), "d2h_bytes_per_step": host.get("d2h_bytes_per_step")},
+                       "h2d_bytes_per_step": host.get("h2d_bytes_per_step"), "d2h_bytes_per_step": host.get("d2h_bytes_per_step"),
+                       "ms_per_step_again": host.get("ms_per_step_again")},
         }
         if host.get("sustained"):
             line["sustained"] = host["sustained"]
